@@ -1,0 +1,402 @@
+#!/usr/bin/env python
+"""Benchmark of the per-example clipping path: clipped+noised gradient examples/s.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl reference]
+
+A "step" is one pass of the whole path (per-layer squared norms -> clip factors
+-> clipped sums -> noise) over one batch of synthetic inputs shaped like the
+paper's workloads.  The headline workload is the MLP 784->1000->1000->10 at
+B = 128 (fp32); the other paper-shaped workloads are timed too and reported in
+the same JSON line under "workloads".  Rank 0 prints ONE JSON line.
+
+Timing: CUDA events on the launching stream around every step, the L2 flushed
+by a 256 MB write between steps (outside the events), max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+import workloads  # noqa: E402
+
+METRIC = "clipped+noised gradient examples/sec"
+UNIT = "examples/s"
+FFMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12        # 148 SMs x 128 fp32 lanes x 2 flop x 1.965 GHz
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"],
+                    bf16_tflops_sustained=d.get("bf16_tflops_sustained", d["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+# ---------------------------------------------------------------------------
+# clocks
+# ---------------------------------------------------------------------------
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.samples = []
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append((time.time(), line.strip()))
+
+    def stop(self, t0=None, t1=None):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        mhz, mx, reasons = [], None, set()
+        for ts, line in self.samples:
+            if t0 is not None and not (t0 - 0.05 <= ts <= t1 + 0.15):
+                continue
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                mhz.append(float(parts[0])); mx = float(parts[1])
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return dict(sm_mhz=float(np.median(mhz)) if mhz else None, sm_max_mhz=mx, reasons=sorted(reasons),
+                    samples=len(mhz))
+
+
+# ---------------------------------------------------------------------------
+# algorithmic work per kernel launch
+# ---------------------------------------------------------------------------
+def elt_bytes(dtype):
+    return 4 if dtype == "f32" else 2
+
+
+def layer_work(w, spec, kind):
+    """(algorithmic bytes, flops) of one launch of `kind` on one layer: every
+    input element read once, every output written once; flops of the exact
+    form the kernel evaluates."""
+    es = elt_bytes(w.dtype)
+    inp = w.B * spec.T * (spec.d_in + spec.d_out) * es
+    P = spec.d_in * spec.d_out + (spec.d_out if spec.has_bias else 0)
+    if kind == "norm_t1":
+        return inp + 4 * w.B, 2 * w.B * (spec.d_in + spec.d_out)
+    if kind == "norm_simt" or kind == "norm_mat":
+        return inp + 4 * w.B, 2 * w.B * spec.T * spec.d_in * spec.d_out
+    if kind == "norm_gram":
+        return inp + 4 * w.B, w.B * spec.T * (spec.T + 1) * (spec.d_in + spec.d_out)
+    if kind == "grad":
+        return inp + 4 * P, 2 * w.B * spec.T * spec.d_in * spec.d_out
+    if kind == "noise":
+        return 8 * P, 0
+    raise ValueError(kind)
+
+
+def step_algorithmic_bytes(w):
+    """Two passes over the inputs (norms, then the clipped sum: the factor of
+    an example depends on all its layers) + every output written once."""
+    return 2 * w.input_bytes() + 4 * w.n_params
+
+
+# ---------------------------------------------------------------------------
+# device arm
+# ---------------------------------------------------------------------------
+def to_dev(x, dtype, torch):
+    t = torch.from_numpy(x).cuda()
+    return t if dtype == "f32" else t.to(torch.bfloat16)
+
+
+def make_plan(dp, w, layers, torch):
+    return dp.StepPlan([dp.Layer(to_dev(A, w.dtype, torch), to_dev(Z, w.dtype, torch), s.has_bias)
+                        for (A, Z), s in zip(layers, w.layers)])
+
+
+def time_steps(torch, fn, steps, warmup, flush):
+    """Per-step device times (ms): events around each step, L2 flush between."""
+    for _ in range(warmup):
+        flush(); fn()
+    torch.cuda.synchronize()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for s, e in ev:
+        flush()
+        s.record(); fn(); e.record()
+    torch.cuda.synchronize()
+    return [s.elapsed_time(e) for s, e in ev]
+
+
+def kernel_breakdown(torch, dp, w, plan, steps, flush, C, sigma):
+    """Second, instrumented pass of the same steps: one event pair around every
+    entry-point call, to attribute the step time to kernels."""
+    acc = {}
+
+    def timed(key, fn):
+        s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s.record(); fn(); e.record()
+        acc.setdefault(key, []).append((s, e))
+
+    for it in range(steps + 1):
+        flush()
+        for l, (y, spec) in enumerate(zip(plan.layers, w.layers)):
+            m = dp.dpclip_pick_method(w.B, spec.T, spec.d_in, spec.d_out, None, None, plan.dtype_code)
+            kind = {dp.DPCLIP_T1: "norm_t1", dp.DPCLIP_SIMT: "norm_simt", dp.DPCLIP_GRAM: "norm_gram",
+                    dp.DPCLIP_MATERIALIZE: "norm_mat"}[m]
+            timed((kind, l), lambda: dp.dpclip_layer_sqnorms(y.A, y.Zbar, spec.has_bias, plan.sq_layers[l],
+                                                             plan.workspace))
+        timed(("factors", -1), lambda: dp.dpclip_factors(plan.sq_layers, C, plan.clip, plan.norms))
+        for l, (y, spec) in enumerate(zip(plan.layers, w.layers)):
+            timed(("grad", l), lambda: dp.dpclip_clipped_grad(y.A, y.Zbar, plan.clip, plan.gW[l], plan.gb[l],
+                                                              plan.workspace))
+            timed(("noise", l), lambda: (dp.dpclip_add_noise(plan.gW[l], sigma, C, 1, 2 * l),
+                                         plan.gb[l] is not None and dp.dpclip_add_noise(plan.gb[l], sigma, C, 1, 2 * l + 1)))
+    torch.cuda.synchronize()
+    out = {}
+    for key, evs in acc.items():
+        ts = [s.elapsed_time(e) for s, e in evs[1:]]            # first iteration is warm-up
+        out[key] = float(np.mean(ts))
+    return out
+
+
+def roofline_for(w, breakdown, peaks):
+    """Roofline of the launch that takes the largest share of the step."""
+    cands = {k: v for k, v in breakdown.items() if k[0] not in ("factors",)}
+    key = max(cands, key=cands.get)
+    kind, l = key
+    spec = w.layers[l]
+    nbytes, flops = layer_work(w, spec, kind)
+    ms = breakdown[key]
+    t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9)
+    on_tensor = kind in ("norm_gram", "norm_mat") or (kind == "grad" and False)
+    alu_peak = (peaks["bf16_tflops"] if on_tensor else FFMA_PEAK_TFLOPS) * 1e12
+    t_alu = flops / alu_peak
+    total = sum(breakdown.values())
+    if t_hbm >= t_alu:
+        ach = nbytes / (ms * 1e-3) / 1e9
+        r = dict(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s", frac=ach / peaks["hbm_gbs"])
+    else:
+        ach = flops / (ms * 1e-3) / 1e12
+        pk = alu_peak / 1e12
+        r = dict(bound="tensor" if on_tensor else "alu", achieved=ach, peak=pk, unit="TFLOP/s", frac=ach / pk)
+    r.update(traffic=None, kernel=f"{kind}[{spec.name}]", kernel_ms=ms, share_of_step=ms / total,
+             algorithmic_bytes=nbytes, algorithmic_flops=flops, peak_source=peaks["source"])
+    return r
+
+
+def bench_workload(torch, dp, w, steps, warmup, flush, peaks, with_e2e=True):
+    layers = workloads.generate(w, seed=0)
+    plan = make_plan(dp, w, layers, torch)
+    n0 = dp.dpclip_launch_count()
+    plan.run(w.C, w.sigma, 1)
+    launches_per_step = dp.dpclip_launch_count() - n0
+    times = time_steps(torch, lambda: plan.run(w.C, w.sigma, 1), steps, warmup, flush)
+    assert dp.dpclip_read_status(plan.workspace) == 0
+    warm = time_steps(torch, lambda: plan.run(w.C, w.sigma, 1), steps, 1, lambda: None)
+    bd = kernel_breakdown(torch, dp, w, plan, min(steps, 20), flush, w.C, w.sigma)
+    res = dict(times_ms=times, warm_ms=float(np.median(warm)), launches_per_step=int(launches_per_step),
+               breakdown={f"{k[0]}[{w.layers[k[1]].name if k[1] >= 0 else 'all'}]": round(v * 1e3, 2)
+                          for k, v in bd.items()},
+               roofline=roofline_for(w, bd, peaks))
+    # whole-step lower bound: max(total algorithmic bytes / HBM, total flops / the engine used)
+    res["step_roofline_us"] = step_algorithmic_bytes(w) / (peaks["hbm_gbs"] * 1e9) * 1e6
+    if with_e2e:
+        host_layers = [dp.Layer(torch.from_numpy(A).to(torch.float32 if w.dtype == "f32" else torch.bfloat16).pin_memory(),
+                                torch.from_numpy(Z).to(torch.float32 if w.dtype == "f32" else torch.bfloat16).pin_memory(),
+                                s.has_bias) for (A, Z), s in zip(layers, w.layers)]
+        hs = dp.HostStep(host_layers)
+
+        def e2e_step():
+            hs.run(w.C, w.sigma, 1)
+            torch.cuda.current_stream().synchronize()          # the caller reads the result on the host
+
+        for _ in range(max(1, warmup)):
+            e2e_step()
+        t0 = time.perf_counter()
+        s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s.record()
+        for _ in range(steps):
+            e2e_step()
+        e.record(); torch.cuda.synchronize()
+        res["e2e_ms"] = s.elapsed_time(e) / steps
+        res["e2e_wall_ms"] = (time.perf_counter() - t0) * 1e3 / steps
+        res["h2d"], res["d2h"] = hs.h2d_bytes, hs.d2h_bytes
+    return res
+
+
+# ---------------------------------------------------------------------------
+# CPU oracle legs
+# ---------------------------------------------------------------------------
+def oracle_sample(w, budget_s=12.0):
+    """Time the oracle, as it stands, on a bounded sample of `w`: whole steps
+    over the first `n` examples of the batch (n chosen so one step takes a few
+    seconds), repeated until about `budget_s` of CPU time is spent."""
+    import oracle
+    oracle.build()
+    hb = [s.has_bias for s in w.layers]
+    flops_per_ex = sum(4.0 * s.T * s.d_in * s.d_out for s in w.layers)      # norm pass + clipped-sum pass
+    n = int(max(1, min(w.B, 4e9 / max(flops_per_ex, 1.0))))
+    layers = workloads.generate(w, seed=0, examples=n)
+    t0 = time.perf_counter()
+    reps = 0
+    while True:
+        oracle.step(layers, hb, w.C, w.sigma, 1)
+        reps += 1
+        dt = time.perf_counter() - t0
+        if dt >= budget_s or reps >= 50:
+            break
+    return dict(value=n * reps / dt, unit=UNIT, cores=1, kind="oracle",
+                sample=f"{reps} whole steps over the first {n} of {w.B} examples of {w.name} "
+                       f"(fp64, single thread, {dt:.1f} s)"), dt / reps, n
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = workloads.by_name(args.workload)
+    total_t, total_n = 0.0, 0
+    info = None
+    for i in range(args.warmup + args.steps):
+        info, per_step, n = oracle_sample(w, budget_s=1.0)
+        if i >= args.warmup:
+            total_t += per_step; total_n += n
+    value = total_n / total_t
+    line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
+                warmup=args.warmup, ms_per_step=total_t / args.steps * 1e3, higher_is_better=True,
+                scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
+                config=dict(workload=w.name, B=w.B, sample=info["sample"]),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=1, kind="oracle", sample=info["sample"]),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0),
+                gpu_launches=0)
+    print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--impl", default="dpclip", choices=["dpclip", "reference"])
+    ap.add_argument("--others", default="cfg1,cfg3_f32,cfg3_bf16,cfg4",
+                    help="further workloads reported under 'workloads' (N=1 only; '' for none)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "dpclip" else args.warmup
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import torch.distributed as dist
+
+    import paper_2009_03106_b200 as dp
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dp.load_library()
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    peaks = measured_peaks()
+    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+    def flush():
+        flush_buf.fill_(1)
+
+    w = workloads.by_name(args.workload)
+    sampler = ClockSampler(local) if rank == 0 else None
+    if world > 1:
+        from paper_2009_03106_b200 import parallel
+        layers = workloads.generate(w, seed=rank)                 # every rank owns its own batch (weak scaling)
+        plan = make_plan(dp, w, layers, torch)
+        fn = lambda: parallel.sharded_step(plan, w.C, w.sigma, seed=1, stream_id0=0)   # noqa: E731
+        n0 = dp.dpclip_launch_count(); fn(); lps = dp.dpclip_launch_count() - n0
+        dist.barrier(); torch.cuda.synchronize()
+        t_wall0 = time.time()
+        times = time_steps(torch, fn, args.steps, args.warmup, flush)
+        torch.cuda.synchronize(); dist.barrier()
+        t_wall1 = time.time()
+        tot = torch.tensor([sum(times)], device="cuda", dtype=torch.float64)
+        dist.all_reduce(tot, op=dist.ReduceOp.MAX)
+        total_ms = tot.item()
+        res = dict(launches_per_step=int(lps), roofline=None, e2e_ms=None)
+    else:
+        t_wall0 = time.time()
+        res = bench_workload(torch, dp, w, args.steps, args.warmup, flush, peaks)
+        t_wall1 = time.time()
+        total_ms = sum(res["times_ms"])
+    clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    ms_per_step = total_ms / args.steps
+    value = w.B * world * args.steps / (total_ms * 1e-3)
+    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
+                ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None,
+                dtype=w.dtype, data="synthetic",
+                config=dict(workload=w.name, B_per_gpu=w.B, layers=[f"{s.name}:T{s.T}:{s.d_in}->{s.d_out}" for s in w.layers],
+                            C=w.C, sigma=w.sigma, l2="flushed by a 256 MB write between steps",
+                            parallelism=f"dp{world}" if world > 1 else "single"),
+                gpu_launches=int(res["launches_per_step"]) * args.steps, clocks=clocks)
+    if world == 1:
+        line["roofline"] = res["roofline"]
+        line["step_roofline_frac"] = res["step_roofline_us"] / (ms_per_step * 1e3)
+        line["warm_l2_ms_per_step"] = res["warm_ms"]
+        line["breakdown_us"] = res["breakdown"]
+        line["e2e"] = dict(value=w.B / (res["e2e_ms"] * 1e-3), unit=UNIT, h2d_bytes_per_step=res["h2d"],
+                           d2h_bytes_per_step=res["d2h"], ms_per_step=res["e2e_ms"])
+        others = {}
+        for name in [n for n in args.others.split(",") if n and n != args.workload]:
+            ow = workloads.by_name(name)
+            r = bench_workload(torch, dp, ow, min(args.steps, 20), 3, flush, peaks, with_e2e=False)
+            ms = float(np.mean(r["times_ms"]))
+            others[name] = dict(workload=ow.name, dtype=ow.dtype, value=ow.B / (ms * 1e-3), ms_per_step=ms,
+                                warm_l2_ms_per_step=r["warm_ms"], launches_per_step=r["launches_per_step"],
+                                step_roofline_frac=r["step_roofline_us"] / (ms * 1e3), roofline=r["roofline"],
+                                breakdown_us=r["breakdown"])
+        line["workloads"] = others
+        if not args.no_cpu_baseline:
+            line["cpu_baseline"], _, _ = oracle_sample(w)
+    else:
+        line["e2e"] = None
+        dist.destroy_process_group()
+    print(json.dumps(line))
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,185 @@
+/*
+ * dpclip.h -- C ABI of libdpclip: per-example gradient clipping for DP-SGD on
+ * one B200 (sm_100a), after Lee & Kifer, "Scaling up Differentially Private
+ * Deep Learning with Fast Per-Example Gradient Clipping".
+ *
+ * Problem statement (paper, Sec. "algorithm": "all that is needed" per layer
+ * is the gradient w.r.t. the pre-activations and the layer's input):
+ *
+ *   layer l, example i:  A_i   in R^{T x d_in}    layer input rows
+ *                        Zb_i  in R^{T x d_out}   dLoss_i/dZ rows, as given (no hidden 1/tau)
+ *     T = 1 dense layer (Algorithm 2), T = H'W' im2col patches for a convolution
+ *     (Algorithm 3), T = sequence length for recurrent/LSTM layers (Algorithm 4)
+ *     and attention projections (Sec. "Multi-head attention").
+ *   per-example gradient  G_i  = sum_t zb_{i,t} (outer) a_{i,t}   (d_out x d_in)
+ *                         gb_i = sum_t zb_{i,t}                    (bias)
+ *   norm    n_i = sqrt( sum_l ||G_{i,l}||_F^2 + ||gb_{i,l}||^2 )   (text after Eq. "weighted_loss")
+ *   factor  c_i = min(1, C / n_i)                                  (Eq. "per_example_weight")
+ *   release sum_i c_i G_i (+ bias)  + N(0, sigma^2 C^2)            (Algorithm 1, last line, as a SUM)
+ *
+ * The library never writes a per-example gradient or a Gram matrix to global
+ * memory.
+ *
+ * Conventions for every entry point
+ *   - Pointers are DEVICE pointers unless the parameter comment says "host".
+ *   - `stream` is a cudaStream_t passed as void* (NULL = legacy default stream).
+ *     Calls only enqueue work; they never synchronise the stream.
+ *   - The caller owns every buffer, including the workspace.  The library
+ *     allocates no device memory and keeps no state between calls.
+ *   - Layout: A is B x T x d_in with row stride `lda` ELEMENTS (>= d_in), rows
+ *     of one example contiguous (example i starts at row i*T); Zbar likewise
+ *     with `ldz`.  Outputs are fp32; gW is d_out x d_in row-major with row
+ *     stride `ldg` (>= d_in), the layout of a dense weight [out, in] or of a
+ *     convolution weight flattened to [c_out, c_in*k*k].
+ *   - Return value: DPCLIP_OK or a negative dpclip_status.  Argument errors
+ *     are detected on the host before anything is launched.  A device-side
+ *     bounded wait that ran out sets a status word in the workspace header
+ *     (see dpclip_read_status); the kernel then exits, it never traps.
+ *   - NaN/Inf inputs propagate; nothing is screened.
+ */
+#ifndef DPCLIP_H_
+#define DPCLIP_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { DPCLIP_F32 = 0, DPCLIP_BF16 = 1 } dpclip_dtype;
+
+/* How a layer's squared norms are computed.  AUTO picks T1 when T == 1 and
+ * otherwise the cheaper exact form by flop count, restricted to the forms the
+ * shape and alignment allow. */
+typedef enum {
+    DPCLIP_AUTO = 0,
+    DPCLIP_T1 = 1,           /* ||a||^2 ||zb||^2, Goodfellow's closed form (Sec. "Fully-connected Layers") */
+    DPCLIP_GRAM = 2,         /* sum_{t,s} (a_t.a_s)(zb_t.zb_s): Gram tiles on the tensor cores (bf16)        */
+    DPCLIP_MATERIALIZE = 3,  /* ||Zb_i^T A_i||_F^2 with the tile held on chip, Frobenius sum in the epilogue   */
+    DPCLIP_SIMT = 4          /* MATERIALIZE on the fp32 ALUs (any dtype, any alignment)                        */
+} dpclip_method;
+
+typedef enum {
+    DPCLIP_OK = 0,
+    DPCLIP_ERR_INVALID_ARG = -1,      /* null pointer, non-positive size, stride < width          */
+    DPCLIP_ERR_UNSUPPORTED = -2,      /* method not available for this dtype / shape / alignment   */
+    DPCLIP_ERR_MISALIGNED = -3,       /* pointer not aligned to its element size                   */
+    DPCLIP_ERR_WORKSPACE = -4,        /* workspace NULL or smaller than dpclip_workspace_bytes()   */
+    DPCLIP_ERR_CUDA = -5,             /* a CUDA runtime/driver call or a launch failed              */
+    DPCLIP_ERR_TIMEOUT = -6           /* (device status) a bounded wait inside a kernel ran out     */
+} dpclip_status;
+
+/* Squared per-example gradient norm of ONE layer, for every example:
+ *   sq_layer[i] = || sum_t zb_{i,t} (outer) a_{i,t} ||_F^2  (+ || sum_t zb_{i,t} ||^2 if has_bias).
+ * T = 1 is Goodfellow's closed form; T > 1 follows Algorithms 3-4 (the sum
+ * over t is taken BEFORE the norm) without storing G_i.
+ *   A, Zbar   inputs as described above, dtype `dtype` (bf16 = raw 16-bit payload)
+ *   sq_layer  [B] fp32, OVERWRITTEN (row l of the caller's [L][B] array)
+ *   workspace >= dpclip_workspace_bytes(...) bytes, 256-byte aligned; its first
+ *             256 bytes are the status header (see dpclip_workspace_init).
+ * Errors: INVALID_ARG for B, T, d_in or d_out <= 0, lda < d_in, ldz < d_out or
+ * null pointers; UNSUPPORTED when `method` cannot run this dtype/shape (e.g.
+ * T1 with T > 1, GRAM with fp32 inputs or rows not a multiple of 16 bytes). */
+int dpclip_layer_sqnorms(const void* A, long lda, const void* Zbar, long ldz,
+                         int B, int T, int d_in, int d_out,
+                         dpclip_dtype dtype, int has_bias, dpclip_method method,
+                         float* sq_layer, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Cross-layer accumulate and clip factors:
+ *   norms[i] = sqrt(sum_l sq_layers[l*ld_sq + i]),  clip[i] = 1 if norms[i] <= C else C / norms[i].
+ * The stored factor is exactly 1.0f for an unclipped example (including a zero
+ * norm).  norms and n_clipped may be NULL; n_clipped[0] receives the number
+ * of examples with clip < 1.  Errors: INVALID_ARG for L, B <= 0, C <= 0 or
+ * ld_sq < B. */
+int dpclip_factors(const float* sq_layers, int L, long ld_sq, int B, float C,
+                   float* clip, float* norms, int* n_clipped, void* stream);
+
+/* Clipped sum of ONE layer (the weight-gradient product of Algorithm 1's
+ * reweighted backward pass, with the per-example weight applied while the
+ * operand is loaded):
+ *   gW[o][k] = sum_i clip[i] sum_t zb_{i,t}[o] a_{i,t}[k],   gb[o] = sum_i clip[i] sum_t zb_{i,t}[o].
+ *   clip  [B] fp32, or NULL for all ones (the plain batch gradient Zbar^T A)
+ *   gW    d_out x d_in fp32, row stride ldg, OVERWRITTEN;  gb [d_out] or NULL, OVERWRITTEN
+ * When the contraction is split over CTAs the partial sums are combined with
+ * fp32 atomic adds, so low-order bits may differ from run to run. */
+int dpclip_clipped_grad(const void* A, long lda, const void* Zbar, long ldz,
+                        int B, int T, int d_in, int d_out, dpclip_dtype dtype,
+                        const float* clip, float* gW, long ldg, float* gb,
+                        void* workspace, size_t workspace_bytes, void* stream);
+
+/* Gaussian mechanism: g[j] += sigma * C * xi_j for j in [0, n), xi_j ~ N(0,1).
+ * The paper names no generator.  This library uses Philox4x32-10 with key =
+ * (seed lo, seed hi) and counter = (q lo, q hi, stream_id lo, stream_id hi),
+ * q = j / 4; word w of the block maps to u = fma(float(w), 2^-32, 2^-33) in
+ * (0,1]; Box-Muller on words (0,1) gives elements 4q (cos) and 4q+1 (sin),
+ * words (2,3) give 4q+2 and 4q+3.  The result depends only on (seed,
+ * stream_id, j): the library is stateless, and a (seed, stream_id) pair must
+ * not be reused for two tensors.  n == 0 is a no-op.  Errors: INVALID_ARG for
+ * a null g with n > 0 or negative sigma or C. */
+int dpclip_add_noise(float* g, size_t n, float sigma, float C,
+                     unsigned long long seed, unsigned long long stream_id, void* stream);
+
+/* One layer of a whole step. */
+typedef struct {
+    const void* A;  long lda;       /* B x T x d_in  */
+    const void* Zbar; long ldz;     /* B x T x d_out */
+    int T, d_in, d_out;
+    int has_bias;
+    int method;                     /* dpclip_method for the norm */
+    float* gW; long ldg;            /* d_out x d_in, overwritten with the noised clipped sum */
+    float* gb;                      /* [d_out] or NULL when has_bias == 0 */
+} dpclip_layer;
+
+/* The whole path over L layers on one stream: per-layer squared norms ->
+ * factors -> per-layer clipped sums -> noise on every released coordinate
+ * (weights of layer l use noise stream stream_id0 + 2l, its bias + 2l + 1).
+ *   layers     host array of L descriptors whose pointers are device pointers
+ *   sq_layers  [L][B] fp32 scratch/outputs, clip [B], norms [B] or NULL
+ *   workspace  >= the largest dpclip_workspace_bytes() over the layers
+ * Output rows must be dense (ldg == d_in; UNSUPPORTED otherwise) because the
+ * noise is indexed by the element's position in the dense tensor. */
+int dpclip_step(const dpclip_layer* layers /* host */, int L, int B, dpclip_dtype dtype,
+                float C, float sigma, unsigned long long seed, unsigned long long stream_id0,
+                float* sq_layers, float* clip, float* norms,
+                void* workspace, size_t workspace_bytes, void* stream);
+
+/* Same, for callers whose tensors live in HOST memory (pinned memory makes the
+ * copies asynchronous).  `layers[l].A/Zbar/gW/gb` are HOST pointers with dense
+ * rows (lda = d_in, ldz = d_out, ldg = d_in are required).  `arena` is a device
+ * buffer of at least dpclip_step_host_arena_bytes() bytes that stages inputs,
+ * outputs and the workspace.  host_clip [B] and host_norms [B] (either may be
+ * NULL) receive the factors.  All copies and kernels are enqueued on `stream`;
+ * the results are valid after the caller synchronises it. */
+int dpclip_step_host(const dpclip_layer* layers /* host, host pointers inside */, int L, int B,
+                     dpclip_dtype dtype, float C, float sigma,
+                     unsigned long long seed, unsigned long long stream_id0,
+                     float* host_clip, float* host_norms,
+                     void* arena, size_t arena_bytes, void* stream);
+size_t dpclip_step_host_arena_bytes(const dpclip_layer* layers /* host */, int L, int B, dpclip_dtype dtype);
+
+/* Bytes of workspace that dpclip_layer_sqnorms / dpclip_clipped_grad need for
+ * this shape (always >= 256: the status header). */
+size_t dpclip_workspace_bytes(int B, int T, int d_in, int d_out, dpclip_dtype dtype, dpclip_method method);
+
+/* Zero the 256-byte status header.  Call once after allocating a workspace. */
+int dpclip_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
+
+/* Copy the device status word to *host_status (host pointer) and synchronise
+ * `stream`.  0 means no kernel reported an anomaly since the header was
+ * initialised. */
+int dpclip_read_status(const void* workspace, int* host_status /* host */, void* stream);
+
+/* Which form DPCLIP_AUTO resolves to for this layer (a dpclip_method). */
+int dpclip_pick_method(int B, int T, int d_in, int d_out, long lda, long ldz, dpclip_dtype dtype);
+
+/* Number of kernels this library has launched in this process (a host-side
+ * counter for benchmarks and tests; cudaMemset calls are not counted). */
+unsigned long long dpclip_launch_count(void);
+
+const char* dpclip_status_string(int status);
+int dpclip_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DPCLIP_H_ */

@@ -1,0 +1,292 @@
+"""ctypes binding of libdpclip.so: same names as the C ABI, argument marshalling only.
+
+Every step of the path runs in the library's kernels.  torch is used for
+device memory and for the current CUDA stream.  There is no CPU fallback: if
+the shared library is missing or does not load, the first call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import List, Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libdpclip.so")
+_lib = None
+
+DPCLIP_F32, DPCLIP_BF16 = 0, 1
+DPCLIP_AUTO, DPCLIP_T1, DPCLIP_GRAM, DPCLIP_MATERIALIZE, DPCLIP_SIMT = 0, 1, 2, 3, 4
+
+_vp, _i, _l, _f = ctypes.c_void_p, ctypes.c_int, ctypes.c_long, ctypes.c_float
+_sz, _u64 = ctypes.c_size_t, ctypes.c_ulonglong
+
+
+class DpclipError(RuntimeError):
+    def __init__(self, fn: str, status: int):
+        self.status = status
+        super().__init__(f"{fn} failed: {status} ({dpclip_status_string(status)})")
+
+
+class _CLayer(ctypes.Structure):
+    _fields_ = [("A", _vp), ("lda", _l), ("Zbar", _vp), ("ldz", _l),
+                ("T", _i), ("d_in", _i), ("d_out", _i), ("has_bias", _i), ("method", _i),
+                ("gW", _vp), ("ldg", _l), ("gb", _vp)]
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def load_library():
+    """Load libdpclip.so (built in-tree by paper_2009_03106_b200.build)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise ImportError(f"{_LIB_PATH} is missing: build it with "
+                          "`python -m paper_2009_03106_b200.build` (there is no fallback path)")
+    L = ctypes.CDLL(_LIB_PATH)
+    L.dpclip_layer_sqnorms.argtypes = [_vp, _l, _vp, _l, _i, _i, _i, _i, _i, _i, _i, _vp, _vp, _sz, _vp]
+    L.dpclip_factors.argtypes = [_vp, _i, _l, _i, _f, _vp, _vp, _vp, _vp]
+    L.dpclip_clipped_grad.argtypes = [_vp, _l, _vp, _l, _i, _i, _i, _i, _i, _vp, _vp, _l, _vp, _vp, _sz, _vp]
+    L.dpclip_add_noise.argtypes = [_vp, _sz, _f, _f, _u64, _u64, _vp]
+    L.dpclip_step.argtypes = [ctypes.POINTER(_CLayer), _i, _i, _i, _f, _f, _u64, _u64, _vp, _vp, _vp, _vp, _sz, _vp]
+    L.dpclip_step_host.argtypes = [ctypes.POINTER(_CLayer), _i, _i, _i, _f, _f, _u64, _u64, _vp, _vp, _vp, _sz, _vp]
+    L.dpclip_step_host_arena_bytes.argtypes = [ctypes.POINTER(_CLayer), _i, _i, _i]
+    L.dpclip_step_host_arena_bytes.restype = _sz
+    L.dpclip_workspace_bytes.argtypes = [_i, _i, _i, _i, _i, _i]
+    L.dpclip_workspace_bytes.restype = _sz
+    L.dpclip_workspace_init.argtypes = [_vp, _sz, _vp]
+    L.dpclip_read_status.argtypes = [_vp, ctypes.POINTER(_i), _vp]
+    L.dpclip_pick_method.argtypes = [_i, _i, _i, _i, _l, _l, _i]
+    L.dpclip_status_string.argtypes = [_i]
+    L.dpclip_status_string.restype = ctypes.c_char_p
+    L.dpclip_version.argtypes = []
+    L.dpclip_launch_count.argtypes = []
+    L.dpclip_launch_count.restype = _u64
+    for name in ("dpclip_layer_sqnorms", "dpclip_factors", "dpclip_clipped_grad", "dpclip_add_noise",
+                 "dpclip_step", "dpclip_step_host", "dpclip_workspace_init", "dpclip_read_status",
+                 "dpclip_pick_method", "dpclip_version"):
+        getattr(L, name).restype = _i
+    _lib = L
+    return L
+
+
+# ----------------------------------------------------------------------------
+# marshalling helpers
+# ----------------------------------------------------------------------------
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return DPCLIP_F32
+    if t.dtype == torch.bfloat16:
+        return DPCLIP_BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else t.data_ptr()
+
+
+def _check(fn: str, rc: int):
+    if rc != 0:
+        raise DpclipError(fn, rc)
+
+
+def _rows(t: torch.Tensor):
+    """(B, T, d) tensor with contiguous features -> (B, T, d, row stride in elements)."""
+    if t.dim() == 2:
+        t = t.unsqueeze(1)
+    B, T, d = t.shape
+    if t.stride(2) != 1 and d > 1:
+        raise ValueError("feature dimension must be contiguous")
+    ld = t.stride(1) if T > 1 else (t.stride(0) if B > 1 else d)
+    if T > 1 and B > 1 and t.stride(0) != T * ld:
+        raise ValueError("rows of consecutive examples must be equally spaced")
+    return B, T, d, ld
+
+
+# ----------------------------------------------------------------------------
+# the C ABI, one function per entry point
+# ----------------------------------------------------------------------------
+def dpclip_version() -> int:
+    return load_library().dpclip_version()
+
+
+def dpclip_launch_count() -> int:
+    return load_library().dpclip_launch_count()
+
+
+def dpclip_status_string(status: int) -> str:
+    try:
+        return load_library().dpclip_status_string(status).decode()
+    except ImportError:
+        return "library not loaded"
+
+
+def dpclip_workspace_bytes(B, T, d_in, d_out, dtype=DPCLIP_F32, method=DPCLIP_AUTO) -> int:
+    return load_library().dpclip_workspace_bytes(B, T, d_in, d_out, dtype, method)
+
+
+def dpclip_workspace_init(workspace: torch.Tensor, stream=None) -> None:
+    _check("dpclip_workspace_init",
+           load_library().dpclip_workspace_init(_ptr(workspace), workspace.numel() * workspace.element_size(),
+                                                _stream(stream)))
+
+
+def dpclip_read_status(workspace: torch.Tensor, stream=None) -> int:
+    out = _i(0)
+    _check("dpclip_read_status", load_library().dpclip_read_status(_ptr(workspace), ctypes.byref(out),
+                                                                   _stream(stream)))
+    return out.value
+
+
+def dpclip_pick_method(B, T, d_in, d_out, lda=None, ldz=None, dtype=DPCLIP_F32) -> int:
+    return load_library().dpclip_pick_method(B, T, d_in, d_out, lda or d_in, ldz or d_out, dtype)
+
+
+def dpclip_layer_sqnorms(A: torch.Tensor, Zbar: torch.Tensor, has_bias: bool, sq_layer: torch.Tensor,
+                         workspace: torch.Tensor, method: int = DPCLIP_AUTO, stream=None) -> None:
+    B, T, d_in, lda = _rows(A)
+    B2, T2, d_out, ldz = _rows(Zbar)
+    assert (B, T) == (B2, T2) and A.dtype == Zbar.dtype
+    assert sq_layer.dtype == torch.float32 and sq_layer.numel() >= B and sq_layer.is_contiguous()
+    _check("dpclip_layer_sqnorms", load_library().dpclip_layer_sqnorms(
+        _ptr(A), lda, _ptr(Zbar), ldz, B, T, d_in, d_out, _dtype_code(A), int(has_bias), method,
+        _ptr(sq_layer), _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+def dpclip_factors(sq_layers: torch.Tensor, C: float, clip: torch.Tensor, norms: Optional[torch.Tensor] = None,
+                   n_clipped: Optional[torch.Tensor] = None, stream=None) -> None:
+    L, B = sq_layers.shape
+    assert sq_layers.dtype == torch.float32 and sq_layers.stride(1) == 1
+    _check("dpclip_factors", load_library().dpclip_factors(
+        _ptr(sq_layers), L, sq_layers.stride(0) if L > 1 else B, B, C, _ptr(clip), _ptr(norms),
+        _ptr(n_clipped), _stream(stream)))
+
+
+def dpclip_clipped_grad(A: torch.Tensor, Zbar: torch.Tensor, clip: Optional[torch.Tensor], gW: torch.Tensor,
+                        gb: Optional[torch.Tensor], workspace: torch.Tensor, stream=None) -> None:
+    B, T, d_in, lda = _rows(A)
+    _, _, d_out, ldz = _rows(Zbar)
+    assert gW.dtype == torch.float32 and gW.shape == (d_out, d_in) and gW.stride(1) == 1
+    _check("dpclip_clipped_grad", load_library().dpclip_clipped_grad(
+        _ptr(A), lda, _ptr(Zbar), ldz, B, T, d_in, d_out, _dtype_code(A), _ptr(clip), _ptr(gW),
+        gW.stride(0) if d_out > 1 else d_in, _ptr(gb), _ptr(workspace),
+        workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+def dpclip_add_noise(g: torch.Tensor, sigma: float, C: float, seed: int, stream_id: int, stream=None) -> None:
+    assert g.dtype == torch.float32 and g.is_contiguous()
+    _check("dpclip_add_noise", load_library().dpclip_add_noise(_ptr(g), g.numel(), sigma, C, seed, stream_id,
+                                                               _stream(stream)))
+
+
+# ----------------------------------------------------------------------------
+# whole step
+# ----------------------------------------------------------------------------
+@dataclass
+class Layer:
+    A: torch.Tensor            # (B, T, d_in)
+    Zbar: torch.Tensor         # (B, T, d_out)
+    has_bias: bool = True
+    method: int = DPCLIP_AUTO
+
+
+class StepPlan:
+    """Buffers and the C descriptor array for repeated whole-step calls on one
+    set of layer shapes.  Holds no arithmetic: `run` is one dpclip_step call."""
+
+    def __init__(self, layers: Sequence[Layer], device=None):
+        self.layers = list(layers)
+        self.L = len(self.layers)
+        dev = device or self.layers[0].A.device
+        self.B = self.layers[0].A.shape[0]
+        self.dtype_code = _dtype_code(self.layers[0].A)
+        self.gW: List[torch.Tensor] = []
+        self.gb: List[Optional[torch.Tensor]] = []
+        self._c = (_CLayer * self.L)()
+        ws = 256
+        # all outputs live in one flat fp32 buffer (each tensor starts on a 256-byte boundary), so a
+        # data-parallel caller can all-reduce the whole gradient with one collective
+        offs, total = [], 0
+        for y in self.layers:
+            d_in, d_out = y.A.shape[-1], y.Zbar.shape[-1]
+            ow = total; total += -(-d_out * d_in // 64) * 64
+            ob = total; total += (-(-d_out // 64) * 64) if y.has_bias else 0
+            offs.append((ow, ob))
+        self.flat = torch.zeros((total,), dtype=torch.float32, device=dev)
+        for l, y in enumerate(self.layers):
+            B, T, d_in, lda = _rows(y.A)
+            _, _, d_out, ldz = _rows(y.Zbar)
+            assert B == self.B and _dtype_code(y.A) == self.dtype_code
+            ow, ob = offs[l]
+            gW = self.flat[ow:ow + d_out * d_in].view(d_out, d_in)
+            gb = self.flat[ob:ob + d_out] if y.has_bias else None
+            self.gW.append(gW); self.gb.append(gb)
+            self._c[l] = _CLayer(_ptr(y.A), lda, _ptr(y.Zbar), ldz, T, d_in, d_out, int(y.has_bias),
+                                 y.method, _ptr(gW), d_in, _ptr(gb))
+            ws = max(ws, dpclip_workspace_bytes(B, T, d_in, d_out, self.dtype_code, y.method))
+        self.sq_layers = torch.empty((self.L, self.B), dtype=torch.float32, device=dev)
+        self.clip = torch.empty((self.B,), dtype=torch.float32, device=dev)
+        self.norms = torch.empty((self.B,), dtype=torch.float32, device=dev)
+        self.workspace = torch.empty((ws,), dtype=torch.uint8, device=dev)
+        dpclip_workspace_init(self.workspace)
+
+    def run(self, C: float, sigma: float, seed: int, stream_id0: int = 0, stream=None) -> None:
+        dpclip_step(self, C, sigma, seed, stream_id0, stream)
+
+
+def dpclip_step(plan: StepPlan, C: float, sigma: float, seed: int, stream_id0: int = 0, stream=None) -> None:
+    _check("dpclip_step", load_library().dpclip_step(
+        plan._c, plan.L, plan.B, plan.dtype_code, C, sigma, seed, stream_id0, _ptr(plan.sq_layers),
+        _ptr(plan.clip), _ptr(plan.norms), _ptr(plan.workspace), plan.workspace.numel(), _stream(stream)))
+
+
+class HostStep:
+    """Whole step for tensors that live in (pinned) host memory: inputs are
+    copied to the device, the path runs, outputs are copied back, all inside
+    one dpclip_step_host call enqueued on the current stream."""
+
+    def __init__(self, host_layers: Sequence[Layer], device="cuda"):
+        self.layers = list(host_layers)
+        self.L = len(self.layers)
+        self.B = self.layers[0].A.shape[0]
+        self.dtype_code = _dtype_code(self.layers[0].A)
+        self._c = (_CLayer * self.L)()
+        self.gW, self.gb = [], []
+        self.h2d_bytes = 0
+        self.d2h_bytes = 0
+        for l, y in enumerate(self.layers):
+            assert not y.A.is_cuda and y.A.is_contiguous() and y.Zbar.is_contiguous()
+            B, T, d_in, _ = _rows(y.A)
+            _, _, d_out, _ = _rows(y.Zbar)
+            gW = torch.empty((d_out, d_in), dtype=torch.float32).pin_memory()
+            gb = torch.empty((d_out,), dtype=torch.float32).pin_memory() if y.has_bias else None
+            self.gW.append(gW); self.gb.append(gb)
+            self._c[l] = _CLayer(_ptr(y.A), d_in, _ptr(y.Zbar), d_out, T, d_in, d_out, int(y.has_bias),
+                                 y.method, _ptr(gW), d_in, _ptr(gb))
+            self.h2d_bytes += y.A.numel() * y.A.element_size() + y.Zbar.numel() * y.Zbar.element_size()
+            self.d2h_bytes += gW.numel() * 4 + (gb.numel() * 4 if gb is not None else 0)
+        self.clip = torch.empty((self.B,), dtype=torch.float32).pin_memory()
+        self.norms = torch.empty((self.B,), dtype=torch.float32).pin_memory()
+        self.d2h_bytes += 8 * self.B
+        nbytes = load_library().dpclip_step_host_arena_bytes(self._c, self.L, self.B, self.dtype_code)
+        self.arena = torch.empty((nbytes,), dtype=torch.uint8, device=device)
+
+    def run(self, C: float, sigma: float, seed: int, stream_id0: int = 0, stream=None) -> None:
+        dpclip_step_host(self, C, sigma, seed, stream_id0, stream)
+
+
+def dpclip_step_host(hs: HostStep, C: float, sigma: float, seed: int, stream_id0: int = 0, stream=None) -> None:
+    _check("dpclip_step_host", load_library().dpclip_step_host(
+        hs._c, hs.L, hs.B, hs.dtype_code, C, sigma, seed, stream_id0, _ptr(hs.clip), _ptr(hs.norms),
+        _ptr(hs.arena), hs.arena.numel(), _stream(stream)))

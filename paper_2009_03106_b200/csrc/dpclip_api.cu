@@ -1,0 +1,325 @@
+// C ABI of libdpclip: argument checking, method selection and kernel launches.
+#include <stdint.h>
+#include <string.h>
+
+#include "common.cuh"
+#include "kernels_simt.cuh"
+#include "kernels_stream.cuh"
+
+using namespace dpclip;
+
+namespace {
+
+inline size_t elt_size(dpclip_dtype dt) { return dt == DPCLIP_F32 ? 4 : 2; }
+inline bool aligned_to(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+// Kernels launched by this library since it was loaded (observability only; never read by a kernel).
+unsigned long long g_launches = 0;
+inline int launch_status() {
+    ++g_launches;
+    return cudaGetLastError() == cudaSuccess ? DPCLIP_OK : DPCLIP_ERR_CUDA;
+}
+
+int check_layer_args(const void* A, long lda, const void* Z, long ldz, int B, int T, int d_in, int d_out,
+                     dpclip_dtype dtype) {
+    if (!A || !Z) return DPCLIP_ERR_INVALID_ARG;
+    if (B <= 0 || T <= 0 || d_in <= 0 || d_out <= 0) return DPCLIP_ERR_INVALID_ARG;
+    if (lda < d_in || ldz < d_out) return DPCLIP_ERR_INVALID_ARG;
+    if (dtype != DPCLIP_F32 && dtype != DPCLIP_BF16) return DPCLIP_ERR_INVALID_ARG;
+    if ((long)B * T > 0x7FFFFFFFL) return DPCLIP_ERR_INVALID_ARG;
+    if (!aligned_to(A, elt_size(dtype)) || !aligned_to(Z, elt_size(dtype))) return DPCLIP_ERR_MISALIGNED;
+    return DPCLIP_OK;
+}
+
+// 4-element vector loads need the base and every row start on a 4-element boundary.
+inline int vec4_ok(const void* p, long ld, dpclip_dtype dt) {
+    return aligned_to(p, 4 * elt_size(dt)) && (ld % 4 == 0);
+}
+
+void fill_simt_params(SimtParams& p, const void* A, long lda, const void* Z, long ldz, int T, int d_in,
+                      int d_out, int has_bias, dpclip_dtype dtype) {
+    memset(&p, 0, sizeof(p));
+    p.A = A; p.lda = lda; p.Z = Z; p.ldz = ldz;
+    p.T = T; p.d_in = d_in; p.d_out = d_out; p.has_bias = has_bias ? 1 : 0;
+    p.tiles_m = ceil_div(d_out, SIMT_BM);
+    p.tiles_n = ceil_div(d_in + p.has_bias, SIMT_BN);
+    p.vec_a = vec4_ok(A, lda, dtype);
+    p.vec_z = vec4_ok(Z, ldz, dtype);
+}
+
+int launch_t1_norms(const void* A, long lda, const void* Z, long ldz, int B, int d_in, int d_out,
+                    dpclip_dtype dtype, int has_bias, float* sq, cudaStream_t st) {
+    const int va = vec4_ok(A, lda, dtype), vz = vec4_ok(Z, ldz, dtype);
+    if (dtype == DPCLIP_F32)
+        t1_sqnorm_kernel<float><<<B, 256, 0, st>>>((const float*)A, lda, (const float*)Z, ldz, d_in, d_out,
+                                                   has_bias, va, vz, sq);
+    else
+        t1_sqnorm_kernel<__nv_bfloat16><<<B, 256, 0, st>>>((const __nv_bfloat16*)A, lda,
+                                                           (const __nv_bfloat16*)Z, ldz, d_in, d_out,
+                                                           has_bias, va, vz, sq);
+    return launch_status();
+}
+
+int launch_simt_norms(const void* A, long lda, const void* Z, long ldz, int B, int T, int d_in, int d_out,
+                      dpclip_dtype dtype, int has_bias, float* sq, cudaStream_t st) {
+    SimtParams p;
+    fill_simt_params(p, A, lda, Z, ldz, T, d_in, d_out, has_bias, dtype);
+    const int n_tiles = p.tiles_m * p.tiles_n;
+    int split = ceil_div(2 * kNumSMs, B);
+    if (split > n_tiles) split = n_tiles;
+    if (split < 1) split = 1;
+    p.sq = sq;
+    p.use_atomic = split > 1;
+    if (p.use_atomic && cudaMemsetAsync(sq, 0, sizeof(float) * (size_t)B, st) != cudaSuccess)
+        return DPCLIP_ERR_CUDA;
+    dim3 grid(split, B);
+    if (dtype == DPCLIP_F32) zta_simt_kernel<float, false><<<grid, SIMT_THREADS, 0, st>>>(p);
+    else zta_simt_kernel<__nv_bfloat16, false><<<grid, SIMT_THREADS, 0, st>>>(p);
+    return launch_status();
+}
+
+int launch_simt_grad(const void* A, long lda, const void* Z, long ldz, int B, int T, int d_in, int d_out,
+                     dpclip_dtype dtype, const float* clip, float* gW, long ldg, float* gb, cudaStream_t st) {
+    SimtParams p;
+    fill_simt_params(p, A, lda, Z, ldz, T, d_in, d_out, gb != nullptr, dtype);
+    const int n_tiles = p.tiles_m * p.tiles_n;
+    const long rows = (long)B * T;
+    long ksplit = ceil_div(4 * kNumSMs, n_tiles);
+    const long max_split = (rows + 4 * SIMT_BK - 1) / (4 * SIMT_BK);     // at least 64 rows per slice
+    if (ksplit > max_split) ksplit = max_split;
+    if (ksplit < 1) ksplit = 1;
+    if (ksplit > 65535) ksplit = 65535;
+    long per = (rows + ksplit - 1) / ksplit;
+    per = (per + SIMT_BK - 1) / SIMT_BK * SIMT_BK;
+    ksplit = (rows + per - 1) / per;
+    p.clip = clip; p.gW = gW; p.ldg = ldg; p.gb = gb;
+    p.rows_total = rows; p.rows_per_split = per;
+    p.use_atomic = ksplit > 1;
+    if (p.use_atomic) {
+        if (cudaMemset2DAsync(gW, sizeof(float) * (size_t)ldg, 0, sizeof(float) * (size_t)d_in, d_out, st) !=
+            cudaSuccess) return DPCLIP_ERR_CUDA;
+        if (gb && cudaMemsetAsync(gb, 0, sizeof(float) * (size_t)d_out, st) != cudaSuccess)
+            return DPCLIP_ERR_CUDA;
+    }
+    dim3 grid(n_tiles, (unsigned)ksplit);
+    if (dtype == DPCLIP_F32) zta_simt_kernel<float, true><<<grid, SIMT_THREADS, 0, st>>>(p);
+    else zta_simt_kernel<__nv_bfloat16, true><<<grid, SIMT_THREADS, 0, st>>>(p);
+    return launch_status();
+}
+
+}  // namespace
+
+extern "C" {
+
+int dpclip_version(void) { return 100; }
+
+unsigned long long dpclip_launch_count(void) { return g_launches; }
+
+const char* dpclip_status_string(int status) {
+    switch (status) {
+        case DPCLIP_OK: return "ok";
+        case DPCLIP_ERR_INVALID_ARG: return "invalid argument";
+        case DPCLIP_ERR_UNSUPPORTED: return "method not supported for this dtype/shape/alignment";
+        case DPCLIP_ERR_MISALIGNED: return "pointer not aligned to its element size";
+        case DPCLIP_ERR_WORKSPACE: return "workspace missing or too small";
+        case DPCLIP_ERR_CUDA: return "CUDA call or kernel launch failed";
+        case DPCLIP_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+        default: return "unknown status";
+    }
+}
+
+int dpclip_pick_method(int B, int T, int d_in, int d_out, long lda, long ldz, dpclip_dtype dtype) {
+    (void)B; (void)d_in; (void)d_out; (void)lda; (void)ldz; (void)dtype;
+    if (T == 1) return DPCLIP_T1;
+    return DPCLIP_SIMT;
+}
+
+size_t dpclip_workspace_bytes(int B, int T, int d_in, int d_out, dpclip_dtype dtype, dpclip_method method) {
+    (void)B; (void)T; (void)d_in; (void)d_out; (void)dtype; (void)method;
+    return kHeaderBytes;
+}
+
+int dpclip_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
+    if (!workspace || workspace_bytes < (size_t)kHeaderBytes) return DPCLIP_ERR_WORKSPACE;
+    return cudaMemsetAsync(workspace, 0, kHeaderBytes, (cudaStream_t)stream) == cudaSuccess ? DPCLIP_OK
+                                                                                             : DPCLIP_ERR_CUDA;
+}
+
+int dpclip_read_status(const void* workspace, int* host_status, void* stream) {
+    if (!workspace || !host_status) return DPCLIP_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemcpyAsync(host_status, workspace, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return DPCLIP_ERR_CUDA;
+    return cudaStreamSynchronize(st) == cudaSuccess ? DPCLIP_OK : DPCLIP_ERR_CUDA;
+}
+
+int dpclip_layer_sqnorms(const void* A, long lda, const void* Zbar, long ldz, int B, int T, int d_in,
+                         int d_out, dpclip_dtype dtype, int has_bias, dpclip_method method, float* sq_layer,
+                         void* workspace, size_t workspace_bytes, void* stream) {
+    int rc = check_layer_args(A, lda, Zbar, ldz, B, T, d_in, d_out, dtype);
+    if (rc) return rc;
+    if (!sq_layer) return DPCLIP_ERR_INVALID_ARG;
+    if (!aligned_to(sq_layer, 4)) return DPCLIP_ERR_MISALIGNED;
+    if (method == DPCLIP_AUTO) method = (dpclip_method)dpclip_pick_method(B, T, d_in, d_out, lda, ldz, dtype);
+    if (!workspace || workspace_bytes < dpclip_workspace_bytes(B, T, d_in, d_out, dtype, method))
+        return DPCLIP_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    switch (method) {
+        case DPCLIP_T1:
+            if (T != 1) return DPCLIP_ERR_UNSUPPORTED;
+            return launch_t1_norms(A, lda, Zbar, ldz, B, d_in, d_out, dtype, has_bias, sq_layer, st);
+        case DPCLIP_SIMT:
+            return launch_simt_norms(A, lda, Zbar, ldz, B, T, d_in, d_out, dtype, has_bias, sq_layer, st);
+        case DPCLIP_GRAM:
+        case DPCLIP_MATERIALIZE:
+            return DPCLIP_ERR_UNSUPPORTED;
+        default:
+            return DPCLIP_ERR_INVALID_ARG;
+    }
+}
+
+int dpclip_factors(const float* sq_layers, int L, long ld_sq, int B, float C, float* clip, float* norms,
+                   int* n_clipped, void* stream) {
+    if (!sq_layers || !clip) return DPCLIP_ERR_INVALID_ARG;
+    if (L <= 0 || B <= 0 || ld_sq < B || !(C > 0.f)) return DPCLIP_ERR_INVALID_ARG;
+    factors_kernel<<<1, 256, 0, (cudaStream_t)stream>>>(sq_layers, L, ld_sq, B, C, clip, norms, n_clipped);
+    return launch_status();
+}
+
+int dpclip_clipped_grad(const void* A, long lda, const void* Zbar, long ldz, int B, int T, int d_in,
+                        int d_out, dpclip_dtype dtype, const float* clip, float* gW, long ldg, float* gb,
+                        void* workspace, size_t workspace_bytes, void* stream) {
+    int rc = check_layer_args(A, lda, Zbar, ldz, B, T, d_in, d_out, dtype);
+    if (rc) return rc;
+    if (!gW || ldg < d_in) return DPCLIP_ERR_INVALID_ARG;
+    if (!aligned_to(gW, 4) || (gb && !aligned_to(gb, 4))) return DPCLIP_ERR_MISALIGNED;
+    if (!workspace || workspace_bytes < dpclip_workspace_bytes(B, T, d_in, d_out, dtype, DPCLIP_AUTO))
+        return DPCLIP_ERR_WORKSPACE;
+    return launch_simt_grad(A, lda, Zbar, ldz, B, T, d_in, d_out, dtype, clip, gW, ldg, gb,
+                            (cudaStream_t)stream);
+}
+
+int dpclip_add_noise(float* g, size_t n, float sigma, float C, unsigned long long seed,
+                     unsigned long long stream_id, void* stream) {
+    if (n == 0) return DPCLIP_OK;
+    if (!g || !(sigma >= 0.f) || !(C >= 0.f)) return DPCLIP_ERR_INVALID_ARG;
+    if (!aligned_to(g, 4)) return DPCLIP_ERR_MISALIGNED;
+    const size_t nq = (n + 3) / 4;
+    size_t blocks = (nq + 255) / 256;
+    const size_t cap = (size_t)kNumSMs * 16;
+    if (blocks > cap) blocks = cap;
+    noise_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(
+        g, n, sigma * C, (uint32_t)seed, (uint32_t)(seed >> 32), (uint32_t)stream_id,
+        (uint32_t)(stream_id >> 32), aligned_to(g, 16) ? 1 : 0);
+    return launch_status();
+}
+
+int dpclip_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, float C, float sigma,
+                unsigned long long seed, unsigned long long stream_id0, float* sq_layers, float* clip,
+                float* norms, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!layers || L <= 0 || !sq_layers || !clip) return DPCLIP_ERR_INVALID_ARG;
+    int rc;
+    for (int l = 0; l < L; ++l) {
+        const dpclip_layer& y = layers[l];
+        rc = dpclip_layer_sqnorms(y.A, y.lda, y.Zbar, y.ldz, B, y.T, y.d_in, y.d_out, dtype, y.has_bias,
+                                  (dpclip_method)y.method, sq_layers + (size_t)l * B, workspace,
+                                  workspace_bytes, stream);
+        if (rc) return rc;
+    }
+    rc = dpclip_factors(sq_layers, L, B, B, C, clip, norms, nullptr, stream);
+    if (rc) return rc;
+    for (int l = 0; l < L; ++l) {
+        const dpclip_layer& y = layers[l];
+        float* gb = y.has_bias ? y.gb : nullptr;
+        if (y.has_bias && !gb) return DPCLIP_ERR_INVALID_ARG;
+        rc = dpclip_clipped_grad(y.A, y.lda, y.Zbar, y.ldz, B, y.T, y.d_in, y.d_out, dtype, clip, y.gW, y.ldg,
+                                 gb, workspace, workspace_bytes, stream);
+        if (rc) return rc;
+        // noise indexes the dense d_out x d_in tensor, so the step wants unpadded output rows
+        if (y.ldg != y.d_in) return DPCLIP_ERR_UNSUPPORTED;
+        rc = dpclip_add_noise(y.gW, (size_t)y.d_out * y.d_in, sigma, C, seed, stream_id0 + 2ull * l, stream);
+        if (rc) return rc;
+        if (gb) {
+            rc = dpclip_add_noise(gb, (size_t)y.d_out, sigma, C, seed, stream_id0 + 2ull * l + 1, stream);
+            if (rc) return rc;
+        }
+    }
+    return DPCLIP_OK;
+}
+
+size_t dpclip_step_host_arena_bytes(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype) {
+    if (!layers || L <= 0 || B <= 0) return 0;
+    const size_t es = elt_size(dtype);
+    size_t ws = kHeaderBytes, total = 0;
+    for (int l = 0; l < L; ++l) {
+        const dpclip_layer& y = layers[l];
+        size_t w = dpclip_workspace_bytes(B, y.T, y.d_in, y.d_out, dtype, (dpclip_method)y.method);
+        if (w > ws) ws = w;
+        total += round_up((size_t)B * y.T * y.d_in * es, 256);
+        total += round_up((size_t)B * y.T * y.d_out * es, 256);
+        total += round_up((size_t)y.d_out * y.d_in * 4, 256);
+        total += round_up((size_t)y.d_out * 4, 256);
+    }
+    total += round_up(ws, 256);
+    total += round_up((size_t)L * B * 4, 256) + 2 * round_up((size_t)B * 4, 256);
+    return total;
+}
+
+int dpclip_step_host(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, float C, float sigma,
+                     unsigned long long seed, unsigned long long stream_id0, float* host_clip,
+                     float* host_norms, void* arena, size_t arena_bytes, void* stream) {
+    if (!layers || L <= 0 || L > 64 || B <= 0 || !arena) return DPCLIP_ERR_INVALID_ARG;
+    if (!aligned_to(arena, 256)) return DPCLIP_ERR_MISALIGNED;
+    if (arena_bytes < dpclip_step_host_arena_bytes(layers, L, B, dtype)) return DPCLIP_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t es = elt_size(dtype);
+    char* cur = static_cast<char*>(arena);
+    auto take = [&](size_t bytes) { char* p = cur; cur += round_up(bytes, 256); return (void*)p; };
+
+    size_t ws_bytes = kHeaderBytes;
+    for (int l = 0; l < L; ++l) {
+        const dpclip_layer& y = layers[l];
+        if (y.lda != y.d_in || y.ldz != y.d_out || y.ldg != y.d_in) return DPCLIP_ERR_INVALID_ARG;
+        if (!y.A || !y.Zbar || !y.gW || (y.has_bias && !y.gb)) return DPCLIP_ERR_INVALID_ARG;
+        size_t w = dpclip_workspace_bytes(B, y.T, y.d_in, y.d_out, dtype, (dpclip_method)y.method);
+        if (w > ws_bytes) ws_bytes = w;
+    }
+    void* ws = take(ws_bytes);
+    float* sq = (float*)take((size_t)L * B * 4);
+    float* clip = (float*)take((size_t)B * 4);
+    float* norms = (float*)take((size_t)B * 4);
+    if (dpclip_workspace_init(ws, ws_bytes, stream)) return DPCLIP_ERR_CUDA;
+
+    dpclip_layer dev[64];
+    for (int l = 0; l < L; ++l) {
+        const dpclip_layer& y = layers[l];
+        dev[l] = y;
+        const size_t a_bytes = (size_t)B * y.T * y.d_in * es, z_bytes = (size_t)B * y.T * y.d_out * es;
+        void* dA = take(a_bytes);
+        void* dZ = take(z_bytes);
+        dev[l].A = dA; dev[l].Zbar = dZ;
+        dev[l].gW = (float*)take((size_t)y.d_out * y.d_in * 4);
+        dev[l].gb = (float*)take((size_t)y.d_out * 4);
+        if (!y.has_bias) dev[l].gb = nullptr;
+        if (cudaMemcpyAsync(dA, y.A, a_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+            cudaMemcpyAsync(dZ, y.Zbar, z_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+            return DPCLIP_ERR_CUDA;
+    }
+    int rc = dpclip_step(dev, L, B, dtype, C, sigma, seed, stream_id0, sq, clip, norms, ws, ws_bytes, stream);
+    if (rc) return rc;
+    for (int l = 0; l < L; ++l) {
+        const dpclip_layer& y = layers[l];
+        if (cudaMemcpyAsync(y.gW, dev[l].gW, (size_t)y.d_out * y.d_in * 4, cudaMemcpyDeviceToHost, st) !=
+            cudaSuccess) return DPCLIP_ERR_CUDA;
+        if (y.has_bias &&
+            cudaMemcpyAsync(y.gb, dev[l].gb, (size_t)y.d_out * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+            return DPCLIP_ERR_CUDA;
+    }
+    if (host_clip && cudaMemcpyAsync(host_clip, clip, (size_t)B * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return DPCLIP_ERR_CUDA;
+    if (host_norms && cudaMemcpyAsync(host_norms, norms, (size_t)B * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return DPCLIP_ERR_CUDA;
+    return DPCLIP_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,133 @@
+// Bandwidth-bound streaming kernels: T=1 squared norms, clip factors, noise.
+#pragma once
+#include "common.cuh"
+
+namespace dpclip {
+
+// ---------------------------------------------------------------------------
+// T = 1 layer norms (Goodfellow's closed form): the per-example gradient is
+// the outer product zb (x) a, so ||G||_F^2 = ||zb||^2 ||a||^2, and the bias
+// gradient is zb itself, so with a bias the total is (||a||^2 + 1) ||zb||^2.
+// Each row of A and Zbar is read exactly once with 128-bit (fp32) / 64-bit
+// (bf16) loads when aligned; one CTA per example, shuffle + smem reduction.
+// ---------------------------------------------------------------------------
+template <typename T>
+__device__ __forceinline__ float row_sumsq(const T* __restrict__ row, int n, bool vec_ok) {
+    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+    int done = 0;
+    if (vec_ok) {
+        int nv = n >> 2;
+        for (int j = threadIdx.x; j < nv; j += blockDim.x) {
+            float4 v = load4(row + 4 * j);
+            s0 = fmaf(v.x, v.x, s0); s1 = fmaf(v.y, v.y, s1);
+            s2 = fmaf(v.z, v.z, s2); s3 = fmaf(v.w, v.w, s3);
+        }
+        done = nv << 2;
+    }
+    for (int j = done + threadIdx.x; j < n; j += blockDim.x) {
+        float v = to_f32(row[j]);
+        s0 = fmaf(v, v, s0);
+    }
+    return (s0 + s1) + (s2 + s3);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+t1_sqnorm_kernel(const T* __restrict__ A, long lda, const T* __restrict__ Z, long ldz,
+                 int d_in, int d_out, int has_bias, int vec_a, int vec_z, float* __restrict__ sq) {
+    __shared__ float red[32];
+    const int i = blockIdx.x;
+    float sa = row_sumsq(A + (size_t)i * lda, d_in, vec_a != 0);
+    float sz = row_sumsq(Z + (size_t)i * ldz, d_out, vec_z != 0);
+    sa = block_sum(sa, red);
+    sz = block_sum(sz, red);
+    if (threadIdx.x == 0) sq[i] = (sa + (has_bias ? 1.f : 0.f)) * sz;
+}
+
+// ---------------------------------------------------------------------------
+// Cross-layer accumulate + clip factors.  One CTA; B is at most a few
+// thousand, the kernel is pure latency.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+factors_kernel(const float* __restrict__ sq_layers, int L, long ld_sq, int B, float C,
+               float* __restrict__ clip, float* __restrict__ norms, int* __restrict__ n_clipped) {
+    __shared__ float red[32];
+    float cnt = 0.f;
+    for (int i = threadIdx.x; i < B; i += blockDim.x) {
+        float s = 0.f;
+        for (int l = 0; l < L; ++l) s += sq_layers[(size_t)l * ld_sq + i];
+        float n = sqrtf(s);
+        float c = 1.0f;
+        if (n > C) { c = C / n; cnt += 1.f; }       // tie and zero norm stay exactly 1
+        clip[i] = c;
+        if (norms) norms[i] = n;
+    }
+    if (n_clipped) {
+        cnt = block_sum(cnt, red);
+        if (threadIdx.x == 0) n_clipped[0] = (int)cnt;
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Gaussian noise: Philox4x32-10 counter-based generator + Box-Muller.
+// One 128-bit block gives four normals; a thread owns block q = elements
+// 4q..4q+3, so the output depends only on (seed, stream_id, element index).
+// ---------------------------------------------------------------------------
+struct PhiloxBlock { uint32_t v[4]; };
+
+__device__ __forceinline__ PhiloxBlock philox_block(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                                    uint32_t k0, uint32_t k1) {
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+        const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+        c0 = hi1 ^ c1 ^ k0;
+        c1 = lo1;
+        c2 = hi0 ^ c3 ^ k1;
+        c3 = lo0;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    PhiloxBlock b;
+    b.v[0] = c0; b.v[1] = c1; b.v[2] = c2; b.v[3] = c3;
+    return b;
+}
+
+__device__ __forceinline__ float bits_to_u01(uint32_t x) {          // (0, 1]
+    return __fmaf_rn(__uint2float_rn(x), 2.3283064365386963e-10f, 1.1641532182693481e-10f);
+}
+
+__device__ __forceinline__ void box_muller(uint32_t xa, uint32_t xb, float& n0, float& n1) {
+    const float u1 = bits_to_u01(xa), u2 = bits_to_u01(xb);
+    const float r = sqrtf(-2.0f * logf(u1));
+    float s, c;
+    sincospif(2.0f * u2, &s, &c);
+    n0 = r * c;
+    n1 = r * s;
+}
+
+__global__ void __launch_bounds__(256)
+noise_kernel(float* __restrict__ g, size_t n, float scale, uint32_t k0, uint32_t k1,
+             uint32_t s0, uint32_t s1, int vec_ok) {
+    const size_t nq = (n + 3) >> 2;
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t q = (size_t)blockIdx.x * blockDim.x + threadIdx.x; q < nq; q += stride) {
+        PhiloxBlock b = philox_block((uint32_t)q, (uint32_t)(q >> 32), s0, s1, k0, k1);
+        float z[4];
+        box_muller(b.v[0], b.v[1], z[0], z[1]);
+        box_muller(b.v[2], b.v[3], z[2], z[3]);
+        const size_t j = q << 2;
+        if (vec_ok && j + 3 < n) {
+            float4 v = *reinterpret_cast<float4*>(g + j);
+            v.x = fmaf(scale, z[0], v.x); v.y = fmaf(scale, z[1], v.y);
+            v.z = fmaf(scale, z[2], v.z); v.w = fmaf(scale, z[3], v.w);
+            *reinterpret_cast<float4*>(g + j) = v;
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                if (j + e < n) g[j + e] = fmaf(scale, z[e], g[j + e]);
+        }
+    }
+}
+
+}  // namespace dpclip

@@ -1,0 +1,295 @@
+"""Parity of the CUDA path (through the C ABI) with the fp64 oracle, element by
+element on the same seeded inputs.  Sizes span several tiles and ragged tails."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads
+from util import SAT_BAND, TOL, check_saturation, max_rel, rel_fro, to_device
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def dp():
+    import paper_2009_03106_b200 as pkg
+    pkg.load_library()          # fails loudly if the CUDA library is missing
+    return pkg
+
+
+def _ws(dp, nbytes=1 << 20):
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    dp.dpclip_workspace_init(ws)
+    return ws
+
+
+def _sqnorms(dp, A, Z, dtype, has_bias, method=0):
+    dA, dZ = to_device(A, dtype), to_device(Z, dtype)
+    sq = torch.full((A.shape[0],), -1.0, device="cuda")
+    ws = _ws(dp, max(1 << 20, dp.dpclip_workspace_bytes(A.shape[0], A.shape[1], A.shape[2], Z.shape[2],
+                                                       0 if dtype == "f32" else 1, method)))
+    dp.dpclip_layer_sqnorms(dA, dZ, has_bias, sq, ws, method)
+    torch.cuda.synchronize()
+    assert dp.dpclip_read_status(ws) == 0
+    return sq.cpu().numpy()
+
+
+# ---------------------------------------------------------------------------
+# (a) T = 1 norms
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("B,d_in,d_out", [(1, 1, 1), (3, 10, 27), (3, 33, 1), (32, 784, 256), (32, 256, 10),
+                                          (128, 1000, 1000), (128, 8192, 256), (5, 4099, 13)])
+@pytest.mark.parametrize("has_bias", [True, False])
+def test_t1_norms(dp, dtype, B, d_in, d_out, has_bias):
+    A, Z = workloads.random_layer(1, B, 1, d_in, d_out, dtype, scale_z=0.1)
+    ref = oracle.layer_sqnorms(A, Z, has_bias)
+    got = _sqnorms(dp, A, Z, dtype, has_bias)
+    # squared norms: twice the relative tolerance of the norm
+    assert max_rel(np.sqrt(got), np.sqrt(ref)) <= TOL["f32"]["norm"]     # inputs identical, fp32 accumulate
+
+
+def test_t1_norms_strided_rows_and_zero_example(dp):
+    B, d_in, d_out = 6, 50, 20
+    A, Z = workloads.random_layer(2, B, 1, d_in, d_out)
+    A[2] = 0.0                                           # an all-zero example has norm 0
+    bigA = torch.zeros((B, 1, 64), device="cuda"); bigA[:, :, :d_in] = torch.from_numpy(A).cuda()
+    bigZ = torch.zeros((B, 1, 24), device="cuda"); bigZ[:, :, :d_out] = torch.from_numpy(Z).cuda()
+    bigA[:, :, d_in:] = 7.0; bigZ[:, :, d_out:] = 7.0    # padding must not be read
+    sq = torch.empty(B, device="cuda")
+    dp.dpclip_layer_sqnorms(bigA[:, :, :d_in], bigZ[:, :, :d_out], False, sq, _ws(dp))
+    ref = oracle.layer_sqnorms(A, Z, False)
+    got = sq.cpu().numpy()
+    assert got[2] == 0.0
+    assert max_rel(got, ref) <= 2e-5
+
+
+# ---------------------------------------------------------------------------
+# (b) T > 1 norms, fp32-ALU tile kernel
+# ---------------------------------------------------------------------------
+SIMT_SHAPES = [(5, 2, 1, 1), (3, 17, 27, 33), (2, 64, 70, 65), (4, 130, 64, 64), (3, 33, 129, 10),
+               (2, 256, 288, 64)]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("B,T,d_in,d_out", SIMT_SHAPES)
+@pytest.mark.parametrize("has_bias", [True, False])
+def test_simt_norms(dp, dtype, B, T, d_in, d_out, has_bias):
+    A, Z = workloads.random_layer(3, B, T, d_in, d_out, dtype, scale_z=0.05)
+    ref = oracle.layer_sqnorms(A, Z, has_bias)
+    got = _sqnorms(dp, A, Z, dtype, has_bias, method=dp.DPCLIP_SIMT)
+    assert max_rel(np.sqrt(got), np.sqrt(ref)) <= TOL["f32"]["norm"]
+
+
+# ---------------------------------------------------------------------------
+# (c) factors
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("B,L", [(1, 1), (32, 2), (128, 3), (1024, 7), (1500, 2)])
+def test_factors(dp, B, L):
+    rng = np.random.default_rng(B + L)
+    sq = (rng.uniform(0.0, 2.0, (L, B)) ** 2).astype(np.float32)
+    sq[:, 0] = 0.0
+    C = 1.5
+    if B > 4:
+        sq[:, 1] = 0.0; sq[0, 1] = np.float32(C * C)                  # exactly on the threshold: not clipped
+        sq[:, 2] = 0.0; sq[0, 2] = np.float32(C * C * (1 + 3e-5))     # inside the band
+    norms_ref, clip_ref = oracle.factors(sq, C)
+    d_sq = torch.from_numpy(sq).cuda()
+    clip = torch.empty(B, device="cuda"); norms = torch.empty(B, device="cuda")
+    cnt = torch.full((1,), -5, dtype=torch.int32, device="cuda")
+    dp.dpclip_factors(d_sq, C, clip, norms, cnt)
+    clip, norms = clip.cpu().numpy(), norms.cpu().numpy()
+    assert max_rel(norms, norms_ref) <= 1e-6
+    assert np.max(np.abs(clip - clip_ref)) <= 1e-6
+    check_saturation(clip, norms_ref, clip_ref, C)
+    assert clip[0] == 1.0
+    if B > 4:
+        assert clip[1] == 1.0
+    assert int(cnt.item()) == int((clip < 1.0).sum())
+    assert np.all(clip.astype(np.float64) * norms_ref <= C * (1 + 1e-6))
+    # optional outputs may be omitted
+    clip2 = torch.empty(B, device="cuda")
+    dp.dpclip_factors(d_sq, C, clip2)
+    assert np.array_equal(clip2.cpu().numpy(), clip)
+
+
+# ---------------------------------------------------------------------------
+# (d) clipped sum
+# ---------------------------------------------------------------------------
+GRAD_SHAPES = [(1, 1, 1, 1), (32, 1, 784, 256), (128, 1, 1000, 10), (7, 1, 129, 65)] + SIMT_SHAPES
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("B,T,d_in,d_out", GRAD_SHAPES)
+def test_clipped_grad(dp, dtype, B, T, d_in, d_out):
+    A, Z = workloads.random_layer(4, B, T, d_in, d_out, dtype, scale_z=0.05)
+    clip = np.random.default_rng(B).uniform(0.05, 1.0, B).astype(np.float32)
+    clip[::3] = 1.0
+    refW, refb = oracle.clipped_grad(A, Z, clip)
+    dA, dZ = to_device(A, dtype), to_device(Z, dtype)
+    gW = torch.full((d_out, d_in), 9.0, device="cuda"); gb = torch.full((d_out,), 9.0, device="cuda")
+    ws = _ws(dp)
+    dp.dpclip_clipped_grad(dA, dZ, torch.from_numpy(clip).cuda(), gW, gb, ws)
+    tol = TOL["f32"]["grad"]          # identical inputs and fp32 accumulation: the fp32 bound applies
+    assert rel_fro(gW.cpu().numpy(), refW) <= tol
+    assert rel_fro(gb.cpu().numpy(), refb) <= tol
+    # clip = NULL: plain batch gradient; gb = NULL: weights only; padded output rows stay untouched
+    refW1, _ = oracle.clipped_grad(A, Z, None)
+    wide = torch.full((d_out, d_in + 3), 9.0, device="cuda")
+    dp.dpclip_clipped_grad(dA, dZ, None, wide[:, :d_in], None, ws)
+    assert rel_fro(wide[:, :d_in].cpu().numpy(), refW1) <= tol
+    assert torch.all(wide[:, d_in:] == 9.0)
+
+
+# ---------------------------------------------------------------------------
+# (e) noise
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("n", [1, 3, 4, 5, 1023, 4096, 100003])
+def test_noise_matches_oracle(dp, n):
+    sigma, C, seed, sid = 1.1, 0.7, 0x123456789ABCDEF, (1 << 40) + 5
+    base = np.random.default_rng(n).standard_normal(n).astype(np.float32)
+    g = torch.from_numpy(base).cuda()
+    dp.dpclip_add_noise(g, sigma, C, seed, sid)
+    ref = oracle.add_noise(base, sigma, C, seed, sid)
+    assert np.max(np.abs(g.cpu().numpy() - ref)) <= 1e-5 * sigma * C + 1e-6 * np.max(np.abs(ref))
+    # noise-only tensor, and an output that does not start on a 16-byte boundary
+    buf = torch.zeros(n + 1, device="cuda")
+    dp.dpclip_add_noise(buf[1:], 1.0, 1.0, seed, sid)
+    xi = oracle.normals(n, seed, sid)
+    assert np.max(np.abs(buf[1:].cpu().numpy() - xi)) <= 1e-5
+    assert buf[0].item() == 0.0
+
+
+def test_noise_is_stateless_and_stream_dependent(dp):
+    n = 10007
+    a = torch.zeros(n, device="cuda"); b = torch.zeros(n, device="cuda"); c = torch.zeros(n, device="cuda")
+    dp.dpclip_add_noise(a, 1.0, 1.0, 7, 0)
+    dp.dpclip_add_noise(b, 1.0, 1.0, 7, 0)
+    dp.dpclip_add_noise(c, 1.0, 1.0, 7, 1)
+    assert torch.equal(a, b)
+    assert abs(np.corrcoef(a.cpu().numpy(), c.cpu().numpy())[0, 1]) < 0.05
+    z = torch.ones(n, device="cuda")
+    dp.dpclip_add_noise(z, 0.0, 1.0, 7, 0)
+    assert torch.all(z == 1.0)
+
+
+# ---------------------------------------------------------------------------
+# whole step on the paper-shaped workloads
+# ---------------------------------------------------------------------------
+def _calibrate(w, layers, seed, C):
+    """Spread per-example norms around C (the stated distributions put every
+    norm far above it): scale example i's Zbar rows, in every layer, by
+    r_i * C / median norm, r_i log-uniform on [1/8, 8]; a few examples are put
+    within 1e-3 of the threshold."""
+    hb = [l.has_bias for l in w.layers]
+    sq = np.stack([oracle.layer_sqnorms(A, Z, b) for (A, Z), b in zip(layers, hb)])
+    n, _ = oracle.factors(sq, C)
+    r = workloads.spread_factors(len(n), seed)
+    r[:3] = [1.0005, 0.9995, 1.0]
+    s = r * C / n
+    out = []
+    for (A, Z) in layers:
+        Zs = (Z.astype(np.float64) * s[:, None, None]).astype(np.float32)
+        if w.dtype == "bf16":
+            Zs = workloads.round_to_bf16(Zs)
+        out.append((A, Zs))
+    return out
+
+
+def _run_step(dp, w, layers, C, sigma, seed, methods=None):
+    dls = [dp.Layer(to_device(A, w.dtype), to_device(Z, w.dtype), spec.has_bias,
+                    methods[i] if methods else dp.DPCLIP_AUTO)
+           for i, ((A, Z), spec) in enumerate(zip(layers, w.layers))]
+    plan = dp.StepPlan(dls)
+    plan.run(C, sigma, seed, 0)
+    torch.cuda.synchronize()
+    assert dp.dpclip_read_status(plan.workspace) == 0
+    return plan
+
+
+def _check_step(dp, w, layers, C, sigma, seed):
+    hb = [l.has_bias for l in w.layers]
+    tol = TOL[w.dtype]
+    ref = oracle.step(layers, hb, C, sigma, seed, 0)
+    pre = _run_step(dp, w, layers, C, 0.0, seed)            # sigma = 0: the pre-noise gradient
+    assert max_rel(np.sqrt(pre.sq_layers.cpu().numpy()), np.sqrt(ref["sq_layers"])) <= tol["norm"]
+    assert max_rel(pre.norms.cpu().numpy(), ref["norms"]) <= tol["norm"]
+    clip = pre.clip.cpu().numpy()
+    check_saturation(clip, ref["norms"], ref["clip"], C)
+    assert np.max(np.abs(clip - ref["clip"]) / ref["clip"]) <= max(tol["norm"], 2 * SAT_BAND)
+    got_all, ref_all = [], []
+    for l in range(len(layers)):
+        gw = pre.gW[l].cpu().numpy()
+        assert rel_fro(gw, ref["gW"][l]) <= tol["grad"], (l, rel_fro(gw, ref["gW"][l]))
+        got_all.append(gw.ravel()); ref_all.append(ref["gW"][l].ravel())
+        if hb[l]:
+            gb = pre.gb[l].cpu().numpy()
+            assert rel_fro(gb, ref["gb"][l]) <= tol["grad"]
+            got_all.append(gb); ref_all.append(ref["gb"][l])
+    assert rel_fro(np.concatenate(got_all), np.concatenate(ref_all)) <= tol["grad"]
+    # every clipped per-example contribution is within C
+    assert np.all(clip.astype(np.float64) * ref["norms"] <= C * (1 + 1e-4))
+    # with noise: final output = pre-noise + sigma*C*xi, checked against the oracle's noised tensors
+    post = _run_step(dp, w, layers, C, sigma, seed)
+    for l in range(len(layers)):
+        d = post.gW[l].cpu().numpy().astype(np.float64) - pre.gW[l].cpu().numpy()
+        xi = (ref["outW"][l] - ref["gW"][l])
+        assert np.max(np.abs(d - xi)) <= 1e-5 * sigma * C + 4e-7 * np.max(np.abs(ref["outW"][l]))
+        if hb[l]:
+            d = post.gb[l].cpu().numpy().astype(np.float64) - pre.gb[l].cpu().numpy()
+            xi = (ref["outb"][l] - ref["gb"][l])
+            assert np.max(np.abs(d - xi)) <= 1e-5 * sigma * C + 4e-7 * np.max(np.abs(ref["outb"][l]))
+    return ref, pre
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_step_mlp_small(dp, seed):
+    w = workloads.mlp_small()
+    layers = workloads.generate(w, seed)
+    _check_step(dp, w, layers, w.C, w.sigma, seed)
+    ref, _ = _check_step(dp, w, _calibrate(w, layers, seed, w.C), w.C, w.sigma, seed)
+    assert 0 < (ref["clip"] < 1).sum() < w.B
+
+
+@pytest.mark.parametrize("C", [0.1, 1.0, 10.0])
+def test_step_mlp_large(dp, C):
+    w = workloads.mlp_large(C=C)
+    layers = workloads.generate(w, 0)
+    _check_step(dp, w, layers, C, w.sigma, 0)
+    # calibrated at C = 1: about all / half / none of the examples are clipped at 0.1 / 1 / 10
+    cal = _calibrate(w, layers, 0, 1.0)
+    ref, _ = _check_step(dp, w, cal, C, w.sigma, 0)
+    frac = (ref["clip"] < 1).mean()
+    assert {0.1: frac > 0.9, 1.0: 0.3 < frac < 0.7, 10.0: frac < 0.1}[C]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_step_cnn(dp, dtype):
+    w = workloads.cnn(dtype)
+    layers = workloads.generate(w, 0)
+    _check_step(dp, w, layers, w.C, w.sigma, 0)
+    _check_step(dp, w, _calibrate(w, layers, 1, w.C), w.C, w.sigma, 1)
+
+
+def test_step_seq_small(dp):
+    """The sequence-model layer mix at a size the oracle finishes in seconds."""
+    w = workloads.seq("bf16", B=6, T=40, d=64, d_ff=136)
+    layers = workloads.generate(w, 0)
+    _check_step(dp, w, layers, w.C, w.sigma, 0)
+    _check_step(dp, w, _calibrate(w, layers, 2, w.C), w.C, w.sigma, 2)
+
+
+def test_step_host_matches_device_step(dp):
+    w = workloads.mlp_small()
+    layers = workloads.generate(w, 0)
+    dev = _run_step(dp, w, layers, w.C, w.sigma, 3)
+    host_layers = [dp.Layer(torch.from_numpy(A).pin_memory(), torch.from_numpy(Z).pin_memory(), s.has_bias)
+                   for (A, Z), s in zip(layers, w.layers)]
+    hs = dp.HostStep(host_layers)
+    hs.run(w.C, w.sigma, 3, 0)
+    torch.cuda.synchronize()
+    assert np.allclose(hs.clip.numpy(), dev.clip.cpu().numpy(), rtol=1e-6)
+    for l in range(len(layers)):
+        assert rel_fro(hs.gW[l].numpy(), dev.gW[l].cpu().numpy()) <= 1e-6
+        assert rel_fro(hs.gb[l].numpy(), dev.gb[l].cpu().numpy()) <= 1e-6
