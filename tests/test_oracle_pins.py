@@ -12,7 +12,15 @@ import torch.nn.functional as F
 import oracle
 import workloads
 
-torch.set_default_dtype(torch.float64)
+
+
+@pytest.fixture(autouse=True)
+def _fp64_default():
+    """The tiny reference networks are built in fp64; restore the default afterwards."""
+    old = torch.get_default_dtype()
+    torch.set_default_dtype(torch.float64)
+    yield
+    torch.set_default_dtype(old)
 
 
 # ---------------------------------------------------------------------------
