@@ -5,6 +5,9 @@
 #include "common.cuh"
 #include "kernels_simt.cuh"
 #include "kernels_stream.cuh"
+#include "kernels_tc.cuh"
+
+#include <stdlib.h>
 
 using namespace dpclip;
 
@@ -107,6 +110,122 @@ int launch_simt_grad(const void* A, long lda, const void* Z, long ldz, int B, in
     return launch_status();
 }
 
+
+// ---------------------------------------------------------------------------
+// tensor-core paths (bf16): tensor maps + launches
+// ---------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;       // a driver entry point, looked up once; not device state
+    if (!fn) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+// 2-D bf16 matrix [rows][cols] with row stride ld elements; box = box_cols x box_rows, 128-byte swizzle,
+// out-of-range elements read as zero.
+bool make_map_bf16(CUtensorMap* map, const void* base, long rows, long cols, long ld, int box_cols, int box_rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// TMA needs 16-byte aligned bases and row strides.
+inline bool tc_eligible(const void* A, long lda, const void* Z, long ldz, dpclip_dtype dtype) {
+    if (dtype != DPCLIP_BF16) return false;
+    const char* env = getenv("DPCLIP_FORCE_SIMT");
+    if (env && env[0] == '1') return false;
+    return aligned_to(A, 16) && aligned_to(Z, 16) && lda % 8 == 0 && ldz % 8 == 0;
+}
+
+template <typename K>
+bool enable_smem(K kernel, int bytes) {
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
+}
+
+int launch_gram_norms(const void* A, long lda, const void* Z, long ldz, int B, int T, int d_in, int d_out,
+                      int has_bias, float* sq, int* status, cudaStream_t st) {
+    namespace g = tc::gram;
+    const long R = (long)B * T;
+    CUtensorMap ma, mz;
+    if (!make_map_bf16(&ma, A, R, d_in, lda, g::BK, g::BM) || !make_map_bf16(&mz, Z, R, d_out, ldz, g::BK, g::BM))
+        return DPCLIP_ERR_CUDA;
+    g::Params p;
+    memset(&p, 0, sizeof(p));
+    p.R = (int)R; p.T = T; p.d_in = d_in; p.d_out = d_out; p.has_bias = has_bias ? 1 : 0;
+    p.sq = sq; p.status = status;
+    if (T % g::BM == 0) {
+        p.dense_pairs = 1; p.q = T / g::BM; p.ppe = p.q * (p.q + 1) / 2;
+        p.n_items = B * p.ppe;
+    } else {
+        p.dense_pairs = 0;
+        p.kmax = (g::BM % T == 0) ? 1 : (T + g::BM - 1) / g::BM + 1;
+        p.n_items = ceil_div(R, g::BM) * p.kmax;
+    }
+    if (!enable_smem(tc::gram_norm_kernel, g::SMEM_BYTES)) return DPCLIP_ERR_CUDA;
+    if (cudaMemsetAsync(sq, 0, sizeof(float) * (size_t)B, st) != cudaSuccess) return DPCLIP_ERR_CUDA;
+    const int grid = p.n_items < kNumSMs ? p.n_items : kNumSMs;
+    tc::gram_norm_kernel<<<grid, g::THREADS, g::SMEM_BYTES, st>>>(ma, mz, p);
+    return launch_status();
+}
+
+int launch_zta_tc(const void* A, long lda, const void* Z, long ldz, int B, int T, int d_in, int d_out,
+                  bool norm_mode, int has_bias, const float* clip, float* gW, long ldg, float* gb, float* sq,
+                  int* status, cudaStream_t st) {
+    namespace z = tc::zta;
+    const long R = (long)B * T;
+    CUtensorMap ma, mz;
+    if (!make_map_bf16(&ma, A, R, d_in, lda, 64, z::BK) || !make_map_bf16(&mz, Z, R, d_out, ldz, 64, z::BK))
+        return DPCLIP_ERR_CUDA;
+    z::Params p;
+    memset(&p, 0, sizeof(p));
+    p.R = (int)R; p.T = T; p.d_in = d_in; p.d_out = d_out;
+    p.norm_mode = norm_mode ? 1 : 0;
+    p.tiles_m = ceil_div(d_out, z::BM); p.tiles_n = ceil_div(d_in, z::BN);
+    const int tiles = p.tiles_m * p.tiles_n;
+    p.status = status;
+    if (norm_mode) {
+        p.n_items = B * tiles;
+        p.do_bias = has_bias ? 1 : 0;
+        p.sq = sq;
+        if (cudaMemsetAsync(sq, 0, sizeof(float) * (size_t)B, st) != cudaSuccess) return DPCLIP_ERR_CUDA;
+    } else {
+        const int nkb = ceil_div(R, z::BK);
+        int ksplit = (2 * kNumSMs + tiles / 2) / tiles;
+        if (ksplit > nkb) ksplit = nkb;
+        if (ksplit < 1) ksplit = 1;
+        p.kb_per_split = ceil_div(nkb, ksplit);
+        ksplit = ceil_div(nkb, p.kb_per_split);
+        p.n_items = tiles * ksplit;
+        p.clip = clip; p.gW = gW; p.ldg = ldg; p.gb = gb;
+        p.do_bias = gb ? 1 : 0;
+        p.use_atomic = ksplit > 1;
+        p.vec_ok = aligned_to(gW, 16) && ldg % 4 == 0;
+        if (p.use_atomic &&
+            cudaMemset2DAsync(gW, sizeof(float) * (size_t)ldg, 0, sizeof(float) * (size_t)d_in, d_out, st) !=
+                cudaSuccess) return DPCLIP_ERR_CUDA;
+        if (gb && cudaMemsetAsync(gb, 0, sizeof(float) * (size_t)d_out, st) != cudaSuccess) return DPCLIP_ERR_CUDA;
+    }
+    if (!enable_smem(tc::zta_tc_kernel, z::SMEM_BYTES)) return DPCLIP_ERR_CUDA;
+    const int grid = p.n_items < kNumSMs ? p.n_items : kNumSMs;
+    tc::zta_tc_kernel<<<grid, z::THREADS, z::SMEM_BYTES, st>>>(ma, mz, p);
+    return launch_status();
+}
+
 }  // namespace
 
 extern "C" {
@@ -129,8 +248,17 @@ const char* dpclip_status_string(int status) {
 }
 
 int dpclip_pick_method(int B, int T, int d_in, int d_out, long lda, long ldz, dpclip_dtype dtype) {
-    (void)B; (void)d_in; (void)d_out; (void)lda; (void)ldz; (void)dtype;
+    (void)B;
     if (T == 1) return DPCLIP_T1;
+    // alignment of the base pointers is not known here; rows must be 16-byte multiples for TMA
+    if (dtype == DPCLIP_BF16 && lda % 8 == 0 && ldz % 8 == 0) {
+        const char* env = getenv("DPCLIP_FORCE_SIMT");
+        if (!(env && env[0] == '1')) {
+            const double gram = (double)T * (T + 1.0) * ((double)d_in + d_out);      // symmetric Gram blocks
+            const double mat = 2.0 * T * (double)d_in * d_out;                       // one Zb_i^T A_i product
+            return gram <= mat ? DPCLIP_GRAM : DPCLIP_MATERIALIZE;
+        }
+    }
     return DPCLIP_SIMT;
 }
 
@@ -160,7 +288,11 @@ int dpclip_layer_sqnorms(const void* A, long lda, const void* Zbar, long ldz, in
     if (rc) return rc;
     if (!sq_layer) return DPCLIP_ERR_INVALID_ARG;
     if (!aligned_to(sq_layer, 4)) return DPCLIP_ERR_MISALIGNED;
-    if (method == DPCLIP_AUTO) method = (dpclip_method)dpclip_pick_method(B, T, d_in, d_out, lda, ldz, dtype);
+    if (method == DPCLIP_AUTO) {
+        method = (dpclip_method)dpclip_pick_method(B, T, d_in, d_out, lda, ldz, dtype);
+        if ((method == DPCLIP_GRAM || method == DPCLIP_MATERIALIZE) && !tc_eligible(A, lda, Zbar, ldz, dtype))
+            method = DPCLIP_SIMT;
+    }
     if (!workspace || workspace_bytes < dpclip_workspace_bytes(B, T, d_in, d_out, dtype, method))
         return DPCLIP_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
@@ -172,7 +304,13 @@ int dpclip_layer_sqnorms(const void* A, long lda, const void* Zbar, long ldz, in
             return launch_simt_norms(A, lda, Zbar, ldz, B, T, d_in, d_out, dtype, has_bias, sq_layer, st);
         case DPCLIP_GRAM:
         case DPCLIP_MATERIALIZE:
-            return DPCLIP_ERR_UNSUPPORTED;
+            if (dtype != DPCLIP_BF16 || !aligned_to(A, 16) || !aligned_to(Zbar, 16) || lda % 8 || ldz % 8)
+                return DPCLIP_ERR_UNSUPPORTED;
+            if (method == DPCLIP_GRAM)
+                return launch_gram_norms(A, lda, Zbar, ldz, B, T, d_in, d_out, has_bias, sq_layer,
+                                         (int*)workspace, st);
+            return launch_zta_tc(A, lda, Zbar, ldz, B, T, d_in, d_out, true, has_bias, nullptr, nullptr, 0,
+                                 nullptr, sq_layer, (int*)workspace, st);
         default:
             return DPCLIP_ERR_INVALID_ARG;
     }
@@ -195,6 +333,9 @@ int dpclip_clipped_grad(const void* A, long lda, const void* Zbar, long ldz, int
     if (!aligned_to(gW, 4) || (gb && !aligned_to(gb, 4))) return DPCLIP_ERR_MISALIGNED;
     if (!workspace || workspace_bytes < dpclip_workspace_bytes(B, T, d_in, d_out, dtype, DPCLIP_AUTO))
         return DPCLIP_ERR_WORKSPACE;
+    if (tc_eligible(A, lda, Zbar, ldz, dtype))
+        return launch_zta_tc(A, lda, Zbar, ldz, B, T, d_in, d_out, false, 0, clip, gW, ldg, gb, nullptr,
+                             (int*)workspace, (cudaStream_t)stream);
     return launch_simt_grad(A, lda, Zbar, ldz, B, T, d_in, d_out, dtype, clip, gW, ldg, gb,
                             (cudaStream_t)stream);
 }
