@@ -377,26 +377,38 @@ zta_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
                 ok = mbar_wait(&full[stage], phase, abort_flag, p.status);
                 if (!ok) break;
                 uint8_t* zt = smem + stage * STAGE_BYTES;
-                const long row0 = w.row_begin + (long)kb * BK + rsub;
+                // rows of this stage: [blk0, blk0 + 64) (32-bit: B*T < 2^31 is checked on the host)
+                const int blk0 = (int)w.row_begin + kb * BK;
+                const int row_end = (int)w.row_end;
+                const int e_first = blk0 / p.T;
+                const int rem0 = blk0 - e_first * p.T;
+                // fast path: the whole stage lies inside one example and inside the row range
+                const bool uniform = (rem0 + BK <= p.T) && (blk0 + BK <= row_end);
+                float f_uni = 1.f;
+                if (uniform && p.clip) f_uni = __ldg(p.clip + e_first);
+                if (!(uniform && f_uni == 1.f && !bias_here)) {
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const long row = row0 + 8 * i;
-                    float f = 1.f;
-                    if (row >= w.row_end) f = 0.f;                       // rows of another example / past the end
-                    else if (p.clip) f = __ldg(p.clip + row / p.T);
-                    if (f != 1.f || bias_here) {
-                        uint4* ptr = reinterpret_cast<uint4*>(zt + off + i * 1024);
-                        uint4 v = *ptr;
-                        uint32_t wds[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-                        for (int h = 0; h < 4; ++h) {
-                            float lo = __uint_as_float(wds[h] << 16) * f;
-                            float hi = __uint_as_float(wds[h] & 0xFFFF0000u) * f;
-                            cs[2 * h] += lo; cs[2 * h + 1] += hi;
-                            __nv_bfloat162 pk = __floats2bfloat162_rn(lo, hi);
-                            wds[h] = *reinterpret_cast<uint32_t*>(&pk);
+                    for (int i = 0; i < 8; ++i) {
+                        float f = f_uni;
+                        if (!uniform) {
+                            const int rl = rsub + 8 * i;
+                            if (blk0 + rl >= row_end) f = 0.f;           // rows of another example / past the end
+                            else if (p.clip) f = __ldg(p.clip + e_first + (rem0 + rl) / p.T);
                         }
-                        if (f != 1.f) *ptr = make_uint4(wds[0], wds[1], wds[2], wds[3]);
+                        if (f != 1.f || bias_here) {
+                            uint4* ptr = reinterpret_cast<uint4*>(zt + off + i * 1024);
+                            uint4 v = *ptr;
+                            uint32_t wds[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                            for (int h = 0; h < 4; ++h) {
+                                float lo = __uint_as_float(wds[h] << 16) * f;
+                                float hi = __uint_as_float(wds[h] & 0xFFFF0000u) * f;
+                                cs[2 * h] += lo; cs[2 * h + 1] += hi;
+                                __nv_bfloat162 pk = __floats2bfloat162_rn(lo, hi);
+                                wds[h] = *reinterpret_cast<uint32_t*>(&pk);
+                            }
+                            if (f != 1.f) *ptr = make_uint4(wds[0], wds[1], wds[2], wds[3]);
+                        }
                     }
                 }
                 fence_proxy_async_smem();
