@@ -183,9 +183,78 @@ int launch_gram_norms(const void* A, long lda, const void* Z, long ldz, int B, i
     return launch_status();
 }
 
+struct NoiseSpec { float scale; unsigned long long seed, sid_w, sid_b; };
+
+// Largest scratch the split-row clipped sum can ask for: one partial tile per item, at most one
+// wave of 256 x 256 tiles or two waves of 128 x 256 tiles, plus the partial bias sums.
+constexpr size_t kTcScratchBytes = (size_t)kNumSMs * 256 * 256 * 4 + (size_t)2 * kNumSMs * 256 * 4;
+
+// Tile shape: 256 x 256 (MT = 2) cuts the L2->SM traffic per flop by a third but has a single
+// accumulator buffer; it pays once d_out spans at least two 128-row sub-tiles.
+template <int MT>
+int launch_zta_tc_mt(const CUtensorMap& ma, const CUtensorMap& mz, tc::zta::Params p, int B, bool norm_mode,
+                     float* gW, long ldg, float* gb, float* sq, int d_in, int d_out, void* workspace,
+                     size_t workspace_bytes, const NoiseSpec* noise, bool* noise_done, cudaStream_t st) {
+    namespace z = tc::zta;
+    constexpr int BM = z::Cfg<MT>::BM;
+    const long R = p.R;
+    p.tiles_m = ceil_div(d_out, BM); p.tiles_n = ceil_div(d_in, z::BN);
+    const int tiles = p.tiles_m * p.tiles_n;
+    int ksplit = 1;
+    if (norm_mode) {
+        p.n_items = B * tiles;
+        if (cudaMemsetAsync(sq, 0, sizeof(float) * (size_t)B, st) != cudaSuccess) return DPCLIP_ERR_CUDA;
+    } else {
+        const int nkb = ceil_div(R, z::BK);
+        // One wave of equally long items: the kernel is bound by L2->SM traffic, so what matters is that
+        // every SM streams the same number of row blocks.  (MT = 1 has two accumulator buffers and can
+        // overlap the epilogue of one item with the next, so it takes two items per SM when they stay long.)
+        const int per_sm = (MT == 1 && tiles <= kNumSMs && nkb / ((2 * kNumSMs) / tiles) >= 16) ? 2 : 1;
+        ksplit = (per_sm * kNumSMs) / tiles;
+        if (ksplit > nkb) ksplit = nkb;
+        if (ksplit < 1) ksplit = 1;
+        p.kb_per_split = ceil_div(nkb, ksplit);
+        ksplit = ceil_div(nkb, p.kb_per_split);
+        p.n_items = tiles * ksplit;
+        if (ksplit > 1) {
+            const size_t part_bytes = (size_t)p.n_items * BM * z::BN * 4;
+            const size_t bias_bytes = gb ? (size_t)p.n_items * BM * 4 : 0;
+            if (workspace_bytes < kHeaderBytes + part_bytes + bias_bytes) return DPCLIP_ERR_WORKSPACE;
+            p.part = reinterpret_cast<float*>(static_cast<char*>(workspace) + kHeaderBytes);
+            p.bias_part = gb ? p.part + part_bytes / 4 : nullptr;
+        } else if (gb && cudaMemsetAsync(gb, 0, sizeof(float) * (size_t)d_out, st) != cudaSuccess) {
+            return DPCLIP_ERR_CUDA;         // single item per tile: direct stores, bias by red.add
+        }
+    }
+    if (!enable_smem(tc::zta_tc_kernel<MT>, z::SMEM_BYTES)) return DPCLIP_ERR_CUDA;
+    const int grid = p.n_items < kNumSMs ? p.n_items : kNumSMs;
+    tc::zta_tc_kernel<MT><<<grid, z::THREADS, z::SMEM_BYTES, st>>>(ma, mz, p);
+    int rc = launch_status();
+    if (rc || norm_mode || ksplit == 1) return rc;
+
+    tc::ReduceParams r;
+    memset(&r, 0, sizeof(r));
+    r.part = p.part; r.bias_part = p.bias_part;
+    r.n_tiles = tiles; r.tiles_n = p.tiles_n; r.ksplit = ksplit; r.BM = BM;
+    r.d_out = d_out; r.d_in = d_in; r.gW = gW; r.ldg = ldg; r.gb = gb; r.vec_ok = p.vec_ok;
+    if (noise && noise->scale > 0.f && ldg == d_in && d_in % 4 == 0) {
+        r.noise_scale = noise->scale;
+        r.k0 = (uint32_t)noise->seed; r.k1 = (uint32_t)(noise->seed >> 32);
+        r.sw0 = (uint32_t)noise->sid_w; r.sw1 = (uint32_t)(noise->sid_w >> 32);
+        r.sb0 = (uint32_t)noise->sid_b; r.sb1 = (uint32_t)(noise->sid_b >> 32);
+        if (noise_done) *noise_done = true;
+    }
+    const long n_vec = (long)d_out * ((d_in + 3) / 4);
+    long blocks = (n_vec + 255) / 256;
+    if (blocks > 8L * kNumSMs) blocks = 8L * kNumSMs;
+    tc::reduce_partials_kernel<<<(unsigned)blocks, 256, 0, st>>>(r);
+    return launch_status();
+}
+
 int launch_zta_tc(const void* A, long lda, const void* Z, long ldz, int B, int T, int d_in, int d_out,
                   bool norm_mode, int has_bias, const float* clip, float* gW, long ldg, float* gb, float* sq,
-                  int* status, cudaStream_t st) {
+                  void* workspace, size_t workspace_bytes, const NoiseSpec* noise, bool* noise_done,
+                  cudaStream_t st) {
     namespace z = tc::zta;
     const long R = (long)B * T;
     CUtensorMap ma, mz;
@@ -195,35 +264,34 @@ int launch_zta_tc(const void* A, long lda, const void* Z, long ldz, int B, int T
     memset(&p, 0, sizeof(p));
     p.R = (int)R; p.T = T; p.d_in = d_in; p.d_out = d_out;
     p.norm_mode = norm_mode ? 1 : 0;
-    p.tiles_m = ceil_div(d_out, z::BM); p.tiles_n = ceil_div(d_in, z::BN);
-    const int tiles = p.tiles_m * p.tiles_n;
-    p.status = status;
+    p.status = static_cast<int*>(workspace);
     if (norm_mode) {
-        p.n_items = B * tiles;
         p.do_bias = has_bias ? 1 : 0;
         p.sq = sq;
-        if (cudaMemsetAsync(sq, 0, sizeof(float) * (size_t)B, st) != cudaSuccess) return DPCLIP_ERR_CUDA;
     } else {
-        const int nkb = ceil_div(R, z::BK);
-        int ksplit = (2 * kNumSMs + tiles / 2) / tiles;
-        if (ksplit > nkb) ksplit = nkb;
-        if (ksplit < 1) ksplit = 1;
-        p.kb_per_split = ceil_div(nkb, ksplit);
-        ksplit = ceil_div(nkb, p.kb_per_split);
-        p.n_items = tiles * ksplit;
         p.clip = clip; p.gW = gW; p.ldg = ldg; p.gb = gb;
         p.do_bias = gb ? 1 : 0;
-        p.use_atomic = ksplit > 1;
         p.vec_ok = aligned_to(gW, 16) && ldg % 4 == 0;
-        if (p.use_atomic &&
-            cudaMemset2DAsync(gW, sizeof(float) * (size_t)ldg, 0, sizeof(float) * (size_t)d_in, d_out, st) !=
-                cudaSuccess) return DPCLIP_ERR_CUDA;
-        if (gb && cudaMemsetAsync(gb, 0, sizeof(float) * (size_t)d_out, st) != cudaSuccess) return DPCLIP_ERR_CUDA;
     }
-    if (!enable_smem(tc::zta_tc_kernel, z::SMEM_BYTES)) return DPCLIP_ERR_CUDA;
-    const int grid = p.n_items < kNumSMs ? p.n_items : kNumSMs;
-    tc::zta_tc_kernel<<<grid, z::THREADS, z::SMEM_BYTES, st>>>(ma, mz, p);
-    return launch_status();
+    int mt = d_out > 128 ? 2 : 1;
+    const char* env = getenv("DPCLIP_TILE_M");
+    if (env && env[0] == '1') mt = 1;
+    if (env && env[0] == '2') mt = 2;
+    if (mt == 2)
+        return launch_zta_tc_mt<2>(ma, mz, p, B, norm_mode, gW, ldg, gb, sq, d_in, d_out, workspace, workspace_bytes,
+                                   noise, noise_done, st);
+    return launch_zta_tc_mt<1>(ma, mz, p, B, norm_mode, gW, ldg, gb, sq, d_in, d_out, workspace, workspace_bytes,
+                               noise, noise_done, st);
+}
+
+// clipped sum of one layer, optionally with the noise folded into the last pass over the output
+int clipped_grad_impl(const void* A, long lda, const void* Zbar, long ldz, int B, int T, int d_in, int d_out,
+                      dpclip_dtype dtype, const float* clip, float* gW, long ldg, float* gb, void* workspace,
+                      size_t workspace_bytes, const NoiseSpec* noise, bool* noise_done, cudaStream_t st) {
+    if (tc_eligible(A, lda, Zbar, ldz, dtype))
+        return launch_zta_tc(A, lda, Zbar, ldz, B, T, d_in, d_out, false, 0, clip, gW, ldg, gb, nullptr, workspace,
+                             workspace_bytes, noise, noise_done, st);
+    return launch_simt_grad(A, lda, Zbar, ldz, B, T, d_in, d_out, dtype, clip, gW, ldg, gb, st);
 }
 
 }  // namespace
@@ -233,6 +301,12 @@ extern "C" {
 int dpclip_version(void) { return 100; }
 
 unsigned long long dpclip_launch_count(void) { return g_launches; }
+
+#ifdef DPCLIP_TRACE
+int dpclip_trace_copy(unsigned long long* host) {
+    return cudaMemcpyFromSymbol(host, tc::g_trace, sizeof(unsigned long long) * 148 * 4 * 256) == cudaSuccess ? 0 : -5;
+}
+#endif
 
 const char* dpclip_status_string(int status) {
     switch (status) {
@@ -263,8 +337,10 @@ int dpclip_pick_method(int B, int T, int d_in, int d_out, long lda, long ldz, dp
 }
 
 size_t dpclip_workspace_bytes(int B, int T, int d_in, int d_out, dpclip_dtype dtype, dpclip_method method) {
-    (void)B; (void)T; (void)d_in; (void)d_out; (void)dtype; (void)method;
-    return kHeaderBytes;
+    (void)B; (void)T; (void)d_in; (void)d_out; (void)method;
+    // bf16 layers may take the tensor-core clipped sum, which splits the rows over CTAs and keeps one
+    // partial tile per CTA in the workspace; the bound does not depend on the layer's shape
+    return dtype == DPCLIP_BF16 ? kHeaderBytes + kTcScratchBytes : (size_t)kHeaderBytes;
 }
 
 int dpclip_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
@@ -310,7 +386,7 @@ int dpclip_layer_sqnorms(const void* A, long lda, const void* Zbar, long ldz, in
                 return launch_gram_norms(A, lda, Zbar, ldz, B, T, d_in, d_out, has_bias, sq_layer,
                                          (int*)workspace, st);
             return launch_zta_tc(A, lda, Zbar, ldz, B, T, d_in, d_out, true, has_bias, nullptr, nullptr, 0,
-                                 nullptr, sq_layer, (int*)workspace, st);
+                                 nullptr, sq_layer, workspace, workspace_bytes, nullptr, nullptr, st);
         default:
             return DPCLIP_ERR_INVALID_ARG;
     }
@@ -333,11 +409,8 @@ int dpclip_clipped_grad(const void* A, long lda, const void* Zbar, long ldz, int
     if (!aligned_to(gW, 4) || (gb && !aligned_to(gb, 4))) return DPCLIP_ERR_MISALIGNED;
     if (!workspace || workspace_bytes < dpclip_workspace_bytes(B, T, d_in, d_out, dtype, DPCLIP_AUTO))
         return DPCLIP_ERR_WORKSPACE;
-    if (tc_eligible(A, lda, Zbar, ldz, dtype))
-        return launch_zta_tc(A, lda, Zbar, ldz, B, T, d_in, d_out, false, 0, clip, gW, ldg, gb, nullptr,
-                             (int*)workspace, (cudaStream_t)stream);
-    return launch_simt_grad(A, lda, Zbar, ldz, B, T, d_in, d_out, dtype, clip, gW, ldg, gb,
-                            (cudaStream_t)stream);
+    return clipped_grad_impl(A, lda, Zbar, ldz, B, T, d_in, d_out, dtype, clip, gW, ldg, gb, workspace,
+                             workspace_bytes, nullptr, nullptr, (cudaStream_t)stream);
 }
 
 int dpclip_add_noise(float* g, size_t n, float sigma, float C, unsigned long long seed,
@@ -373,16 +446,23 @@ int dpclip_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, fl
         const dpclip_layer& y = layers[l];
         float* gb = y.has_bias ? y.gb : nullptr;
         if (y.has_bias && !gb) return DPCLIP_ERR_INVALID_ARG;
-        rc = dpclip_clipped_grad(y.A, y.lda, y.Zbar, y.ldz, B, y.T, y.d_in, y.d_out, dtype, clip, y.gW, y.ldg,
-                                 gb, workspace, workspace_bytes, stream);
-        if (rc) return rc;
         // noise indexes the dense d_out x d_in tensor, so the step wants unpadded output rows
         if (y.ldg != y.d_in) return DPCLIP_ERR_UNSUPPORTED;
-        rc = dpclip_add_noise(y.gW, (size_t)y.d_out * y.d_in, sigma, C, seed, stream_id0 + 2ull * l, stream);
+        rc = check_layer_args(y.A, y.lda, y.Zbar, y.ldz, B, y.T, y.d_in, y.d_out, dtype);
         if (rc) return rc;
-        if (gb) {
-            rc = dpclip_add_noise(gb, (size_t)y.d_out, sigma, C, seed, stream_id0 + 2ull * l + 1, stream);
+        if (!y.gW) return DPCLIP_ERR_INVALID_ARG;
+        NoiseSpec ns = {sigma * C, seed, stream_id0 + 2ull * l, stream_id0 + 2ull * l + 1};
+        bool noise_done = false;
+        rc = clipped_grad_impl(y.A, y.lda, y.Zbar, y.ldz, B, y.T, y.d_in, y.d_out, dtype, clip, y.gW, y.ldg, gb,
+                               workspace, workspace_bytes, &ns, &noise_done, (cudaStream_t)stream);
+        if (rc) return rc;
+        if (!noise_done) {
+            rc = dpclip_add_noise(y.gW, (size_t)y.d_out * y.d_in, sigma, C, seed, ns.sid_w, stream);
             if (rc) return rc;
+            if (gb) {
+                rc = dpclip_add_noise(gb, (size_t)y.d_out, sigma, C, seed, ns.sid_b, stream);
+                if (rc) return rc;
+            }
         }
     }
     return DPCLIP_OK;

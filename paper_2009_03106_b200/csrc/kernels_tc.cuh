@@ -32,6 +32,14 @@
 namespace dpclip {
 namespace tc {
 
+// Developer-only timeline (compiled in with -DDPCLIP_TRACE; never in the shipped library).
+#ifdef DPCLIP_TRACE
+__device__ unsigned long long g_trace[148][4][256];
+#define DPCLIP_TRACE_AT(role, idx) do { if ((idx) < 256) g_trace[blockIdx.x][role][idx] = global_ns(); } while (0)
+#else
+#define DPCLIP_TRACE_AT(role, idx) do { } while (0)
+#endif
+
 // ===========================================================================
 // Gram kernel
 // ===========================================================================
@@ -224,16 +232,27 @@ gram_norm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 // Zb^T diag(f) A kernel (GRAD and NORM modes)
 // ===========================================================================
 namespace zta {
-constexpr int BM = 128;                        // d_out tile (UMMA M)
 constexpr int BN = 256;                        // d_in tile  (UMMA N)
 constexpr int BK = 64;                         // rows per stage
-constexpr int STAGES = 4;
 constexpr int CHUNK_BYTES = BK * 128;          // one TMA box: 64 rows x 64 bf16 columns
-constexpr int A_BYTES = (BM / 64) * CHUNK_BYTES;   // Zb tile, 16 KB
 constexpr int B_BYTES = (BN / 64) * CHUNK_BYTES;   // A tile, 32 KB
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;     // 48 KB
-constexpr int THREADS = 320;                   // warp 0 TMA, 1 MMA, 2..5 transform, 6..9 epilogue
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
+constexpr int N_TRANSFORM_WARPS = 8, N_EPILOGUE_WARPS = 8;
+constexpr int THREADS = 64 + 32 * (N_TRANSFORM_WARPS + N_EPILOGUE_WARPS);   // warp 0 TMA, warp 1 MMA
+constexpr int OUT_STAGE_BYTES = N_EPILOGUE_WARPS * 4096;          // 32 rows x 32 fp32 per epilogue warp
+constexpr int SMEM_BYTES = 192 * 1024 + 256 + OUT_STAGE_BYTES + 1024;
+
+// MT = number of 128-row sub-tiles of d_out per CTA tile.
+//   MT = 1: 128 x 256 tile, two accumulator buffers in tensor memory (the epilogue of one item
+//           overlaps the main loop of the next), 4 stages of 48 KB.
+//   MT = 2: 256 x 256 tile, one accumulator buffer (all 512 columns), 3 stages of 64 KB; a third
+//           less L2->SM traffic per flop, for layers where that traffic is the limit.
+template <int MT> struct Cfg {
+    static constexpr int BM = 128 * MT;
+    static constexpr int A_BYTES = (BM / 64) * CHUNK_BYTES;
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr int STAGES = MT == 1 ? 4 : 3;
+    static constexpr int NBUF = MT == 1 ? 2 : 1;
+};
 
 struct Params {
     int R, T, d_in, d_out;
@@ -243,38 +262,44 @@ struct Params {
     int kb_per_split;              // GRAD: 64-row blocks per item
     int do_bias;                   // GRAD: gb != NULL; NORM: has_bias
     const float* clip;             // GRAD: [B] or NULL
-    float* gW; long ldg; float* gb; int use_atomic; int vec_ok;
+    float* gW; long ldg; float* gb; int vec_ok;
+    float* part;                   // GRAD with split rows: [n_items][BM][BN] fp32 partial tiles (workspace)
+    float* bias_part;              // GRAD with split rows and a bias: [n_items][BM] partial column sums
     float* sq;                     // NORM
     int* status;
 };
 
-struct Item { int m0, n0, tn; long row_begin, row_end; int nkb; int example; };
+struct Item { int m0, n0, tn; int row_begin, row_end; int nkb; int example; };
 
+template <int MT>
 __device__ __forceinline__ Item decode(const Params& p, int item) {
     Item w;
     const int n_tiles = p.tiles_m * p.tiles_n;
     const int tile = item % n_tiles, outer = item / n_tiles;
-    w.m0 = (tile / p.tiles_n) * BM;
+    w.m0 = (tile / p.tiles_n) * Cfg<MT>::BM;
     w.tn = tile % p.tiles_n;
     w.n0 = w.tn * BN;
     if (p.norm_mode) {
         w.example = outer;
-        w.row_begin = (long)outer * p.T;
+        w.row_begin = outer * p.T;
         w.row_end = w.row_begin + p.T;
     } else {
         w.example = -1;
-        w.row_begin = (long)outer * p.kb_per_split * BK;
-        w.row_end = min(w.row_begin + (long)p.kb_per_split * BK, (long)p.R);
+        w.row_begin = outer * p.kb_per_split * BK;
+        w.row_end = min(w.row_begin + p.kb_per_split * BK, p.R);
     }
-    w.nkb = (int)((w.row_end - w.row_begin + BK - 1) / BK);
+    w.nkb = (w.row_end - w.row_begin + BK - 1) / BK;
     return w;
 }
 }  // namespace zta
 
+template <int MT>
 __global__ void __launch_bounds__(zta::THREADS, 1)
 zta_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_z,
               const zta::Params p) {
     using namespace zta;
+    using C = Cfg<MT>;
+    constexpr int STAGES = C::STAGES, STAGE_BYTES = C::STAGE_BYTES, A_BYTES = C::A_BYTES, NBUF = C::NBUF;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);   // TMA landed
@@ -284,11 +309,16 @@ zta_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
     uint64_t* acc_empty = acc_full + 2;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    float4* out_stage = reinterpret_cast<float4*>(smem + STAGES * STAGE_BYTES + 256);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&ready[s], 4); mbar_init(&empty[s], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); }
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(&full[s], 1); mbar_init(&ready[s], N_TRANSFORM_WARPS);
+            // a stage is released by the MMA commit and, in layers with a bias, by the 8 bias/epilogue warps
+            mbar_init(&empty[s], 1 + (p.do_bias ? N_EPILOGUE_WARPS : 0));
+        }
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], N_EPILOGUE_WARPS); }
         *abort_flag = 0;
         mbar_fence_init();
         tma_prefetch_desc(&map_a);
@@ -305,16 +335,19 @@ zta_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0;
             bool ok = true;
+            int tr = 0;
+            DPCLIP_TRACE_AT(0, 255);
             for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
-                const Item w = decode(p, item);
+                const Item w = decode<MT>(p, item);
                 for (int kb = 0; kb < w.nkb; ++kb) {
                     ok = mbar_wait(&empty[stage], phase ^ 1, abort_flag, p.status);
                     if (!ok) break;
+                    DPCLIP_TRACE_AT(0, tr); ++tr;
                     uint8_t* dst = smem + stage * STAGE_BYTES;
-                    const int y = (int)(w.row_begin + (long)kb * BK);
+                    const int y = w.row_begin + kb * BK;
                     mbar_arrive_expect_tx(&full[stage], STAGE_BYTES);
 #pragma unroll
-                    for (int c = 0; c < BM / 64; ++c)
+                    for (int c = 0; c < C::BM / 64; ++c)
                         tma_load_2d(dst + c * CHUNK_BYTES, &map_z, &full[stage], w.m0 + c * 64, y);
 #pragma unroll
                     for (int c = 0; c < BN / 64; ++c)
@@ -326,19 +359,20 @@ zta_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
     } else if (warp == 1) {
         // ------------------------------------------------ MMA issuer
         if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc_bf16(BM, BN, 1, 1);
+            constexpr uint32_t idesc = make_idesc_bf16(128, BN, 1, 1);
             int stage = 0; uint32_t phase = 0; int it = 0;
             bool ok = true;
+            int tr = 0;
             for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
-                const Item w = decode(p, item);
-                const int buf = it & 1; const uint32_t acc_phase = (it >> 1) & 1;
+                const Item w = decode<MT>(p, item);
+                const int buf = it % NBUF; const uint32_t acc_phase = (it / NBUF) & 1;
                 ok = mbar_wait(&acc_empty[buf], acc_phase ^ 1, abort_flag, p.status);
                 if (!ok) break;
                 tc_fence_after_sync();
-                const uint32_t d_tmem = tmem_base + buf * BN;
                 for (int kb = 0; kb < w.nkb; ++kb) {
                     ok = mbar_wait(&ready[stage], phase, abort_flag, p.status);
                     if (!ok) break;
+                    DPCLIP_TRACE_AT(2, tr); ++tr;
                     tc_fence_after_sync();
                     const uint32_t a_addr = smem_u32(smem + stage * STAGE_BYTES);
                     const uint32_t b_addr = a_addr + A_BYTES;
@@ -346,9 +380,14 @@ zta_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
                     for (int k4 = 0; k4 < BK / 16; ++k4) {
                         // MN-major, 128-byte swizzle: 64-column chunks CHUNK_BYTES apart (leading offset),
                         // 8-row groups 1024 bytes apart (stride offset); 16 rows = 2048 bytes
-                        const uint64_t da = make_smem_desc_sw128(a_addr + k4 * 2048, CHUNK_BYTES, 1024);
                         const uint64_t db = make_smem_desc_sw128(b_addr + k4 * 2048, CHUNK_BYTES, 1024);
-                        mma_bf16_ss(d_tmem, da, db, idesc, (kb == 0 && k4 == 0) ? 0u : 1u);
+#pragma unroll
+                        for (int h = 0; h < MT; ++h) {
+                            const uint64_t da = make_smem_desc_sw128(a_addr + h * 2 * CHUNK_BYTES + k4 * 2048,
+                                                                     CHUNK_BYTES, 1024);
+                            mma_bf16_ss(tmem_base + (buf * MT + h) * BN, da, db, idesc,
+                                        (kb == 0 && k4 == 0) ? 0u : 1u);
+                        }
                     }
                     mma_commit(&empty[stage]);
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
@@ -358,104 +397,172 @@ zta_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
                 ++it;
             }
         }
-    } else if (warp < 6) {
-        // ------------------------------------------------ transform (warps 2..5, 128 threads)
-        // thread t owns the 8 columns [8q, 8q+8) of the Zb tile (q = t / 8) on rows (t % 8) + 8 i
+    } else if (warp < 2 + N_TRANSFORM_WARPS) {
+        // ------------------------------------------------ transform (256 threads)
+        // Within each 128-column half of the Zb tile, thread t owns the 8 columns [8q, 8q+8),
+        // q = t / 16, on rows (t % 16) + 16 i.  Column chunk q sits at 16-byte slot q ^ (row & 7)
+        // of its 128-byte row (the TMA swizzle), which is the same slot for all rows of a thread.
         const int t = threadIdx.x - 64;
-        const int q = t >> 3, rsub = t & 7;
+        const int q = t >> 4, rs = t & 15;
         const int box = q >> 3, lq = q & 7;
-        const uint32_t off = box * CHUNK_BYTES + rsub * 128 + ((lq ^ rsub) << 4);
+        const uint32_t off = box * CHUNK_BYTES + rs * 128 + ((lq ^ (rs & 7)) << 4);
         int stage = 0; uint32_t phase = 0;
         bool ok = true;
+        int tr = 0;
         for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
-            const Item w = decode(p, item);
-            const bool bias_here = p.do_bias && w.tn == 0;
-            float cs[8];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) cs[j] = 0.f;
+            const Item w = decode<MT>(p, item);
             for (int kb = 0; kb < w.nkb; ++kb) {
-                ok = mbar_wait(&full[stage], phase, abort_flag, p.status);
-                if (!ok) break;
-                uint8_t* zt = smem + stage * STAGE_BYTES;
-                // rows of this stage: [blk0, blk0 + 64) (32-bit: B*T < 2^31 is checked on the host)
-                const int blk0 = (int)w.row_begin + kb * BK;
-                const int row_end = (int)w.row_end;
+                // the factors of this stage's rows are fetched BEFORE waiting for the tile, so the
+                // global-load latency overlaps the wait instead of sitting between TMA and MMA
+                const int blk0 = w.row_begin + kb * BK;              // rows [blk0, blk0 + 64)
                 const int e_first = blk0 / p.T;
                 const int rem0 = blk0 - e_first * p.T;
                 // fast path: the whole stage lies inside one example and inside the row range
-                const bool uniform = (rem0 + BK <= p.T) && (blk0 + BK <= row_end);
-                float f_uni = 1.f;
-                if (uniform && p.clip) f_uni = __ldg(p.clip + e_first);
-                if (!(uniform && f_uni == 1.f && !bias_here)) {
+                const bool uniform = (rem0 + BK <= p.T) && (blk0 + BK <= w.row_end);
+                float fr[4];
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        float f = f_uni;
-                        if (!uniform) {
-                            const int rl = rsub + 8 * i;
-                            if (blk0 + rl >= row_end) f = 0.f;           // rows of another example / past the end
-                            else if (p.clip) f = __ldg(p.clip + e_first + (rem0 + rl) / p.T);
-                        }
-                        if (f != 1.f || bias_here) {
-                            uint4* ptr = reinterpret_cast<uint4*>(zt + off + i * 1024);
-                            uint4 v = *ptr;
-                            uint32_t wds[4] = {v.x, v.y, v.z, v.w};
+                for (int i = 0; i < 4; ++i) {
+                    const int rl = uniform ? 0 : rs + 16 * i;
+                    float f = 1.f;
+                    if (blk0 + rl >= w.row_end) f = 0.f;             // rows of another example / past the end
+                    else if (p.clip) f = __ldg(p.clip + e_first + (rem0 + rl) / p.T);
+                    fr[i] = f;
+                }
+                ok = mbar_wait(&full[stage], phase, abort_flag, p.status);
+                if (!ok) break;
+                if (t == 0) { DPCLIP_TRACE_AT(1, tr); ++tr; }
+                uint8_t* zt = smem + stage * STAGE_BYTES;
+                if (!(uniform && fr[0] == 1.f)) {
 #pragma unroll
-                            for (int h = 0; h < 4; ++h) {
-                                float lo = __uint_as_float(wds[h] << 16) * f;
-                                float hi = __uint_as_float(wds[h] & 0xFFFF0000u) * f;
-                                cs[2 * h] += lo; cs[2 * h + 1] += hi;
-                                __nv_bfloat162 pk = __floats2bfloat162_rn(lo, hi);
-                                wds[h] = *reinterpret_cast<uint32_t*>(&pk);
+                    for (int i = 0; i < 4; ++i) {
+                        const float f = fr[i];
+                        if (f != 1.f) {
+                            // packed bf16 path: f = f_hi + f_lo (two bf16); z*f_lo is tiny, so the fused
+                            // multiply-add z*f_hi + (z*f_lo) rounds the product once, like the fp32 path
+                            const __nv_bfloat16 fh = __float2bfloat16_rn(f);
+                            const __nv_bfloat16 fl = __float2bfloat16_rn(f - __bfloat162float(fh));
+                            const __nv_bfloat162 fh2 = __halves2bfloat162(fh, fh), fl2 = __halves2bfloat162(fl, fl);
+#pragma unroll
+                            for (int h = 0; h < MT; ++h) {
+                                uint4* ptr = reinterpret_cast<uint4*>(zt + h * 2 * CHUNK_BYTES + off + i * 2048);
+                                uint4 v = *ptr;
+                                __nv_bfloat162* z2 = reinterpret_cast<__nv_bfloat162*>(&v);
+#pragma unroll
+                                for (int u = 0; u < 4; ++u) z2[u] = __hfma2(z2[u], fh2, __hmul2(z2[u], fl2));
+                                *ptr = v;
                             }
-                            if (f != 1.f) *ptr = make_uint4(wds[0], wds[1], wds[2], wds[3]);
                         }
                     }
                 }
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&ready[stage]);
+                if (t == 0) { DPCLIP_TRACE_AT(1, tr); ++tr; }
                 if (++stage == STAGES) { stage = 0; phase ^= 1; }
             }
             if (!ok) break;
-            if (bias_here) {
-                if (p.norm_mode) {
-                    // complete the column sums over the 8 row-subsets (8 consecutive lanes), then square
-                    float ssq = 0.f;
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        float c = cs[j];
-                        c += __shfl_xor_sync(0xFFFFFFFFu, c, 1);
-                        c += __shfl_xor_sync(0xFFFFFFFFu, c, 2);
-                        c += __shfl_xor_sync(0xFFFFFFFFu, c, 4);
-                        ssq = fmaf(c, c, ssq);
-                    }
-                    if (rsub != 0) ssq = 0.f;
-                    ssq = warp_sum(ssq);
-                    if (lane == 0) atomicAdd(p.sq + w.example, ssq);
-                } else {
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const int m = w.m0 + q * 8 + j;
-                        if (m < p.d_out) atomicAdd(p.gb + m, cs[j]);
-                    }
-                }
-            }
         }
     } else {
-        // ------------------------------------------------ epilogue (warps 6..9)
+        // ------------------------------------------------ epilogue (8 warps)
+        // Warp w may touch tensor-memory lanes 32*(w % 4) .. +31.  Two warps share each lane
+        // quarter: group g = 0/1 takes the two column halves (MT = 1) or the two row halves (MT = 2).
         const int quarter = warp & 3;
-        const int row_local = quarter * 32 + lane;
+        const int g = (warp - (2 + N_TRANSFORM_WARPS)) >> 2;
+        const int ew = warp - (2 + N_TRANSFORM_WARPS);
+        const int h = MT == 2 ? g : 0;
+        const int col_begin = MT == 2 ? 0 : g * (BN / 2);
+        const int col_end = MT == 2 ? BN : col_begin + BN / 2;
+        // While the main loop runs, these warps are otherwise idle: in layers with a bias they take the
+        // column sums of the (already scaled) Zb tile, which is the clipped bias gradient
+        // gb[o] = sum_k f_k zb[k][o].  Same thread -> (column chunk, rows) mapping as the transform.
+        const int bt = threadIdx.x - 32 * (2 + N_TRANSFORM_WARPS);
+        const int bq = bt >> 4, brs = bt & 15;
+        const uint32_t boff = (bq >> 3) * CHUNK_BYTES + brs * 128 + (((bq & 7) ^ (brs & 7)) << 4);
+        int stage = 0; uint32_t phase = 0;
         int it = 0;
-        for (int item = blockIdx.x; item < p.n_items; item += gridDim.x) {
-            const Item w = decode(p, item);
-            const int buf = it & 1; const uint32_t acc_phase = (it >> 1) & 1;
+        bool ok = true;
+        for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
+            const Item w = decode<MT>(p, item);
+            if (p.do_bias) {
+                float cs[MT][8];
+#pragma unroll
+                for (int hh = 0; hh < MT; ++hh)
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) cs[hh][j] = 0.f;
+                for (int kb = 0; kb < w.nkb; ++kb) {
+                    ok = mbar_wait(&ready[stage], phase, abort_flag, p.status);
+                    if (!ok) break;
+                    // GRAD: every n-tile of a row range sees the same Zb rows; stage kb is summed by the
+                    // n-tile with kb % tiles_n == tn, so all items carry an equal share.  NORM: the sums
+                    // must be complete before they are squared, so n-tile 0 takes them all.
+                    const bool mine = p.norm_mode ? w.tn == 0 : (kb % p.tiles_n) == w.tn;
+                    if (mine) {
+                        const uint8_t* zt = smem + stage * STAGE_BYTES;
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+#pragma unroll
+                            for (int hh = 0; hh < MT; ++hh) {
+                                const uint4 v = *reinterpret_cast<const uint4*>(zt + hh * 2 * CHUNK_BYTES + boff + i * 2048);
+                                const uint32_t wds[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                                for (int u = 0; u < 4; ++u) {
+                                    cs[hh][2 * u] += __uint_as_float(wds[u] << 16);
+                                    cs[hh][2 * u + 1] += __uint_as_float(wds[u] & 0xFFFF0000u);
+                                }
+                            }
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&empty[stage]);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                }
+                if (!ok) break;
+                if (p.norm_mode) {
+                    if (w.tn == 0) {
+                        // complete the column sums over the 16 row-subsets (16 consecutive lanes), then square
+                        float ssq = 0.f;
+#pragma unroll
+                        for (int hh = 0; hh < MT; ++hh)
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                float c = cs[hh][j];
+                                c += __shfl_xor_sync(0xFFFFFFFFu, c, 1);
+                                c += __shfl_xor_sync(0xFFFFFFFFu, c, 2);
+                                c += __shfl_xor_sync(0xFFFFFFFFu, c, 4);
+                                c += __shfl_xor_sync(0xFFFFFFFFu, c, 8);
+                                ssq = fmaf(c, c, ssq);
+                            }
+                        if (brs != 0) ssq = 0.f;
+                        ssq = warp_sum(ssq);
+                        if (lane == 0) atomicAdd(p.sq + w.example, ssq);
+                    }
+                } else {
+                    // one value per column: finish the sum over the 16 row-subsets first
+#pragma unroll
+                    for (int hh = 0; hh < MT; ++hh)
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            float c = cs[hh][j];
+                            c += __shfl_xor_sync(0xFFFFFFFFu, c, 1);
+                            c += __shfl_xor_sync(0xFFFFFFFFu, c, 2);
+                            c += __shfl_xor_sync(0xFFFFFFFFu, c, 4);
+                            c += __shfl_xor_sync(0xFFFFFFFFu, c, 8);
+                            if (brs == 0) {
+                                const int ml = hh * 128 + bq * 8 + j;
+                                if (p.bias_part) p.bias_part[(size_t)item * C::BM + ml] = c;
+                                else if (w.m0 + ml < p.d_out) red_add_f32(p.gb + w.m0 + ml, c);
+                            }
+                        }
+                }
+            }
+            const int buf = it % NBUF; const uint32_t acc_phase = (it / NBUF) & 1;
             if (!mbar_wait(&acc_full[buf], acc_phase, abort_flag, p.status)) break;
+            if (threadIdx.x == 64 + 32 * N_TRANSFORM_WARPS) DPCLIP_TRACE_AT(3, 2 * it);
             tc_fence_after_sync();
-            const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * BN;
-            const int m = w.m0 + row_local;
+            const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (buf * MT + h) * BN;
+            const int m_base = w.m0 + h * 128 + quarter * 32;     // first output row of this warp
             float fro = 0.f;
 #pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
+            for (int c0 = col_begin; c0 < col_end; c0 += 32) {
                 uint32_t v[32];
                 tmem_ld_32x32(t_row + c0, v);
                 tmem_ld_wait();
@@ -463,31 +570,49 @@ zta_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
                     // rows/columns beyond d_out/d_in were zero-filled by TMA and add nothing
 #pragma unroll
                     for (int j = 0; j < 32; ++j) { const float x = __uint_as_float(v[j]); fro = fmaf(x, x, fro); }
-                } else if (m < p.d_out) {
-                    const int n = w.n0 + c0;
-                    float* dst = p.gW + (size_t)m * p.ldg + n;
-                    if (p.vec_ok && n + 32 <= p.d_in) {
+                } else {
+                    // Transpose the 32 x 32 block through shared memory so that every store/red
+                    // instruction covers 4 rows x 128 contiguous bytes instead of 32 rows x 16 bytes.
+                    float4* st = out_stage + ew * 256;
 #pragma unroll
-                        for (int j = 0; j < 32; j += 4) {
-                            float4 x = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
-                                                   __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
-                            if (p.use_atomic) atomicAdd(reinterpret_cast<float4*>(dst + j), x);
-                            else *reinterpret_cast<float4*>(dst + j) = x;
-                        }
-                    } else {
+                    for (int j = 0; j < 8; ++j)
+                        st[lane * 8 + (j ^ (lane & 7))] =
+                            make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                        __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+                    __syncwarp();
+                    const int jj = lane & 7;
+                    const int n = w.n0 + c0 + 4 * jj;
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            if (n + j < p.d_in) {
-                                if (p.use_atomic) atomicAdd(dst + j, __uint_as_float(v[j]));
-                                else dst[j] = __uint_as_float(v[j]);
+                    for (int i = 0; i < 8; ++i) {
+                        const int rr = 4 * i + (lane >> 3);
+                        const float4 x = st[rr * 8 + (jj ^ (rr & 7))];
+                        if (p.part) {
+                            // rows split over several items: store the partial tile (dense, no bounds);
+                            // reduce_partials_kernel adds the items of a tile in a fixed order
+                            float* dst = p.part + ((size_t)item * C::BM + (h * 128 + quarter * 32 + rr)) * BN + c0 + 4 * jj;
+                            *reinterpret_cast<float4*>(dst) = x;
+                        } else {
+                            const int mm = m_base + rr;
+                            if (mm < p.d_out) {
+                                float* dst = p.gW + (size_t)mm * p.ldg + n;
+                                if (p.vec_ok && n + 4 <= p.d_in) {
+                                    *reinterpret_cast<float4*>(dst) = x;
+                                } else {
+                                    const float xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+                                    for (int u = 0; u < 4; ++u)
+                                        if (n + u < p.d_in) dst[u] = xs[u];
+                                }
                             }
                         }
                     }
+                    __syncwarp();
                 }
             }
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[buf]);
+            if (threadIdx.x == 64 + 32 * N_TRANSFORM_WARPS) DPCLIP_TRACE_AT(3, 2 * it + 1);
             if (p.norm_mode) {
                 fro = warp_sum(fro);
                 if (lane == 0) atomicAdd(p.sq + w.example, fro);
@@ -503,6 +628,82 @@ zta_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) { tc_fence_after_sync(); tmem_dealloc(tmem_base, 512); }
+}
+
+// ---------------------------------------------------------------------------
+// Second stage of the split-row clipped sum: adds the partial tiles of every
+// output tile in a fixed order (deterministic, no atomics) and writes gW / gb.
+// When noise_scale > 0 the Gaussian noise of element j = m*d_in + n is added in
+// the same pass (requires dense rows and d_in % 4 == 0, so that a float4 of the
+// output is exactly one Philox block).
+// ---------------------------------------------------------------------------
+struct ReduceParams {
+    const float* part; const float* bias_part;
+    int n_tiles, tiles_n, ksplit, BM;
+    int d_out, d_in;
+    float* gW; long ldg; float* gb; int vec_ok;
+    float noise_scale; uint32_t k0, k1, sw0, sw1, sb0, sb1;     // Philox key, weight / bias stream words
+};
+
+}  // namespace tc
+}  // namespace dpclip
+
+#include "kernels_stream.cuh"
+
+namespace dpclip {
+namespace tc {
+
+__global__ void __launch_bounds__(256)
+reduce_partials_kernel(const ReduceParams p) {
+    const int n4 = (p.d_in + 3) >> 2;
+    const long total = (long)p.d_out * n4;
+    const size_t tile_elems = (size_t)p.BM * zta::BN;
+    const size_t ks_stride = (size_t)p.n_tiles * tile_elems;
+    for (long idx = (long)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (long)gridDim.x * blockDim.x) {
+        const int m = (int)(idx / n4), n = (int)(idx % n4) << 2;
+        const int tm = m / p.BM, tn = n / zta::BN;
+        const float* src = p.part + (size_t)(tm * p.tiles_n + tn) * tile_elems + (size_t)(m - tm * p.BM) * zta::BN +
+                           (n - tn * zta::BN);
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int ks = 0; ks < p.ksplit; ++ks) {
+            const float4 v = *reinterpret_cast<const float4*>(src + ks * ks_stride);
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        }
+        if (p.noise_scale > 0.f) {
+            const size_t q = ((size_t)m * p.d_in + n) >> 2;
+            PhiloxBlock b = philox_block((uint32_t)q, (uint32_t)(q >> 32), p.sw0, p.sw1, p.k0, p.k1);
+            float z0, z1, z2, z3;
+            box_muller(b.v[0], b.v[1], z0, z1);
+            box_muller(b.v[2], b.v[3], z2, z3);
+            acc.x = fmaf(p.noise_scale, z0, acc.x); acc.y = fmaf(p.noise_scale, z1, acc.y);
+            acc.z = fmaf(p.noise_scale, z2, acc.z); acc.w = fmaf(p.noise_scale, z3, acc.w);
+        }
+        float* dst = p.gW + (size_t)m * p.ldg + n;
+        if (p.vec_ok && n + 4 <= p.d_in) {
+            *reinterpret_cast<float4*>(dst) = acc;
+        } else {
+            const float xs[4] = {acc.x, acc.y, acc.z, acc.w};
+            for (int u = 0; u < 4; ++u)
+                if (n + u < p.d_in) dst[u] = xs[u];
+        }
+    }
+    if (p.gb) {
+        for (int m = blockIdx.x * blockDim.x + threadIdx.x; m < p.d_out; m += gridDim.x * blockDim.x) {
+            const int tm = m / p.BM;
+            float acc = 0.f;
+            for (int ks = 0; ks < p.ksplit; ++ks)
+                for (int tn = 0; tn < p.tiles_n; ++tn)
+                    acc += p.bias_part[((size_t)ks * p.n_tiles + tm * p.tiles_n + tn) * p.BM + (m - tm * p.BM)];
+            if (p.noise_scale > 0.f) {
+                PhiloxBlock b = philox_block((uint32_t)(m >> 2), 0u, p.sb0, p.sb1, p.k0, p.k1);
+                float z[4];
+                box_muller(b.v[0], b.v[1], z[0], z[1]);
+                box_muller(b.v[2], b.v[3], z[2], z[3]);
+                acc = fmaf(p.noise_scale, z[m & 3], acc);
+            }
+            p.gb[m] = acc;
+        }
+    }
 }
 
 }  // namespace tc
