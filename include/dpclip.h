@@ -100,8 +100,10 @@ int dpclip_factors(const float* sq_layers, int L, long ld_sq, int B, float C,
  *   gW[o][k] = sum_i clip[i] sum_t zb_{i,t}[o] a_{i,t}[k],   gb[o] = sum_i clip[i] sum_t zb_{i,t}[o].
  *   clip  [B] fp32, or NULL for all ones (the plain batch gradient Zbar^T A)
  *   gW    d_out x d_in fp32, row stride ldg, OVERWRITTEN;  gb [d_out] or NULL, OVERWRITTEN
- * When the contraction is split over CTAs the partial sums are combined with
- * fp32 atomic adds, so low-order bits may differ from run to run. */
+ * bf16 layers whose rows are 16-byte multiples take the tensor-core path: rows
+ * are split over CTAs, partial tiles go to the workspace and are added in a
+ * fixed order (bit-reproducible).  Other layers take the fp32-ALU path, which
+ * combines row slices with fp32 atomic adds (low-order bits may vary). */
 int dpclip_clipped_grad(const void* A, long lda, const void* Zbar, long ldz,
                         int B, int T, int d_in, int d_out, dpclip_dtype dtype,
                         const float* clip, float* gW, long ldg, float* gb,
@@ -158,7 +160,9 @@ int dpclip_step_host(const dpclip_layer* layers /* host, host pointers inside */
 size_t dpclip_step_host_arena_bytes(const dpclip_layer* layers /* host */, int L, int B, dpclip_dtype dtype);
 
 /* Bytes of workspace that dpclip_layer_sqnorms / dpclip_clipped_grad need for
- * this shape (always >= 256: the status header). */
+ * this shape: the 256-byte status header, plus, for bf16 layers, room for one
+ * fp32 partial tile per SM of the split-row clipped sum (about 39 MB, a bound
+ * that does not depend on the shape). */
 size_t dpclip_workspace_bytes(int B, int T, int d_in, int d_out, dpclip_dtype dtype, dpclip_method method);
 
 /* Zero the 256-byte status header.  Call once after allocating a workspace. */

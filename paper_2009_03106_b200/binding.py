@@ -244,6 +244,17 @@ class StepPlan:
     def run(self, C: float, sigma: float, seed: int, stream_id0: int = 0, stream=None) -> None:
         dpclip_step(self, C, sigma, seed, stream_id0, stream)
 
+    def capture(self, C: float, sigma: float, seed: int, stream_id0: int = 0):
+        """Record one dpclip_step call into a CUDA graph (the launch-bound small workloads spend most
+        of a step in launch gaps).  Returns the graph; `graph.replay()` re-runs the same kernels on the
+        same buffers with the same (C, sigma, seed, stream ids)."""
+        self.run(C, sigma, seed, stream_id0)          # warm-up outside capture (function attributes, maps)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            self.run(C, sigma, seed, stream_id0)
+        return graph
+
 
 def dpclip_step(plan: StepPlan, C: float, sigma: float, seed: int, stream_id0: int = 0, stream=None) -> None:
     _check("dpclip_step", load_library().dpclip_step(
