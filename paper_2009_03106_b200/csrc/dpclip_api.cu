@@ -6,6 +6,7 @@
 #include "kernels_simt.cuh"
 #include "kernels_stream.cuh"
 #include "kernels_tc.cuh"
+#include "kernels_fused_t1.cuh"
 
 #include <stdlib.h>
 
@@ -132,7 +133,8 @@ EncodeTiledFn encode_tiled_fn() {
 
 // 2-D bf16 matrix [rows][cols] with row stride ld elements; box = box_cols x box_rows, 128-byte swizzle,
 // out-of-range elements read as zero.
-bool make_map_bf16(CUtensorMap* map, const void* base, long rows, long cols, long ld, int box_cols, int box_rows) {
+bool make_map_bf16(CUtensorMap* map, const void* base, long rows, long cols, long ld, int box_cols, int box_rows,
+                   bool swizzle = true) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
     cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
@@ -140,7 +142,8 @@ bool make_map_bf16(CUtensorMap* map, const void* base, long rows, long cols, lon
     cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -169,17 +172,23 @@ int launch_gram_norms(const void* A, long lda, const void* Z, long ldz, int B, i
     p.R = (int)R; p.T = T; p.d_in = d_in; p.d_out = d_out; p.has_bias = has_bias ? 1 : 0;
     p.sq = sq; p.status = status;
     if (T % g::BM == 0) {
-        p.dense_pairs = 1; p.q = T / g::BM; p.ppe = p.q * (p.q + 1) / 2;
-        p.n_items = B * p.ppe;
+        p.dense = 1; p.q = T / g::BM;
+        p.n_groups = B;                       // one example per group
     } else {
-        p.dense_pairs = 0;
-        p.kmax = (g::BM % T == 0) ? 1 : (T + g::BM - 1) / g::BM + 1;
-        p.n_items = ceil_div(R, g::BM) * p.kmax;
+        p.dense = 0;
+        p.n_groups = ceil_div(R, g::BM);      // one 128-row block per group
     }
-    if (!enable_smem(tc::gram_norm_kernel, g::SMEM_BYTES)) return DPCLIP_ERR_CUDA;
     if (cudaMemsetAsync(sq, 0, sizeof(float) * (size_t)B, st) != cudaSuccess) return DPCLIP_ERR_CUDA;
-    const int grid = p.n_items < kNumSMs ? p.n_items : kNumSMs;
-    tc::gram_norm_kernel<<<grid, g::THREADS, g::SMEM_BYTES, st>>>(ma, mz, p);
+    const int grid = p.n_groups < kNumSMs ? p.n_groups : kNumSMs;
+    // every item is on the diagonal when an example spans at most two aligned row blocks
+    const bool diag_only = (T % g::BM == 0 && T <= 2 * g::BM) || (g::BM % T == 0);
+    if (diag_only) {
+        if (!enable_smem(tc::gram_norm_kernel<true>, g::SMEM_BYTES)) return DPCLIP_ERR_CUDA;
+        tc::gram_norm_kernel<true><<<grid, g::THREADS, g::SMEM_BYTES, st>>>(ma, mz, p);
+    } else {
+        if (!enable_smem(tc::gram_norm_kernel<false>, g::SMEM_BYTES)) return DPCLIP_ERR_CUDA;
+        tc::gram_norm_kernel<false><<<grid, g::THREADS, g::SMEM_BYTES, st>>>(ma, mz, p);
+    }
     return launch_status();
 }
 
@@ -292,6 +301,54 @@ int clipped_grad_impl(const void* A, long lda, const void* Zbar, long ldz, int B
         return launch_zta_tc(A, lda, Zbar, ldz, B, T, d_in, d_out, false, 0, clip, gW, ldg, gb, nullptr, workspace,
                              workspace_bytes, noise, noise_done, st);
     return launch_simt_grad(A, lda, Zbar, ldz, B, T, d_in, d_out, dtype, clip, gW, ldg, gb, st);
+}
+
+
+// Whole step in two launches for models made of T = 1 layers only (see kernels_fused_t1.cuh).
+// Returns 1 when the fused path does not apply (the caller then takes the per-layer path).
+int try_fused_t1_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, float C, float sigma,
+                      unsigned long long seed, unsigned long long stream_id0, float* sq, float* clip,
+                      float* norms, cudaStream_t st) {
+    if (L > FUSED_MAX_LAYERS || B > FUSED_MAX_B) return 1;
+    const char* env = getenv("DPCLIP_NO_FUSED_T1");
+    if (env && env[0] == '1') return 1;
+    FusedT1Params p;
+    memset(&p, 0, sizeof(p));
+    int tiles = 0;
+    for (int l = 0; l < L; ++l) {
+        const dpclip_layer& y = layers[l];
+        if (y.T != 1 || y.ldg != y.d_in) return 1;
+        if (y.method != DPCLIP_AUTO && y.method != DPCLIP_T1) return 1;
+        int rc = check_layer_args(y.A, y.lda, y.Zbar, y.ldz, B, 1, y.d_in, y.d_out, dtype);
+        if (rc) return rc;
+        if (!y.gW || (y.has_bias && !y.gb)) return DPCLIP_ERR_INVALID_ARG;
+        if (!aligned_to(y.gW, 16) || (y.gb && !aligned_to(y.gb, 4))) return 1;
+        FusedT1Layer& f = p.layer[l];
+        f.A = y.A; f.lda = y.lda; f.Z = y.Zbar; f.ldz = y.ldz;
+        f.d_in = y.d_in; f.d_out = y.d_out; f.has_bias = y.has_bias ? 1 : 0;
+        f.vec_a = vec4_ok(y.A, y.lda, dtype); f.vec_z = vec4_ok(y.Zbar, y.ldz, dtype);
+        f.gW = y.gW; f.gb = y.has_bias ? y.gb : nullptr;
+        f.tiles_m = ceil_div(y.d_out, SIMT_BM); f.tiles_n = ceil_div(y.d_in + f.has_bias, SIMT_BN);
+        f.tile_begin = tiles;
+        tiles += f.tiles_m * f.tiles_n;
+    }
+    p.L = L; p.B = B; p.total_tiles = tiles;
+    p.C = C; p.noise_scale = sigma * C;
+    p.k0 = (uint32_t)seed; p.k1 = (uint32_t)(seed >> 32); p.stream_id0 = stream_id0;
+    p.sq = sq; p.clip = clip; p.norms = norms;
+    const int rows = L * B;
+    const int grid_n = ceil_div(rows, 4);
+    const int grid_g = tiles < 4 * kNumSMs ? tiles : 4 * kNumSMs;
+    if (dtype == DPCLIP_F32) {
+        t1_all_norms_kernel<float><<<grid_n, 128, 0, st>>>(p);
+        if (launch_status()) return DPCLIP_ERR_CUDA;
+        t1_all_grads_kernel<float><<<grid_g, SIMT_THREADS, 0, st>>>(p);
+    } else {
+        t1_all_norms_kernel<__nv_bfloat16><<<grid_n, 128, 0, st>>>(p);
+        if (launch_status()) return DPCLIP_ERR_CUDA;
+        t1_all_grads_kernel<__nv_bfloat16><<<grid_g, SIMT_THREADS, 0, st>>>(p);
+    }
+    return launch_status();
 }
 
 }  // namespace
@@ -431,8 +488,12 @@ int dpclip_add_noise(float* g, size_t n, float sigma, float C, unsigned long lon
 int dpclip_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, float C, float sigma,
                 unsigned long long seed, unsigned long long stream_id0, float* sq_layers, float* clip,
                 float* norms, void* workspace, size_t workspace_bytes, void* stream) {
-    if (!layers || L <= 0 || !sq_layers || !clip) return DPCLIP_ERR_INVALID_ARG;
-    int rc;
+    if (!layers || L <= 0 || B <= 0 || !sq_layers || !clip) return DPCLIP_ERR_INVALID_ARG;
+    if (!(C > 0.f) || !(sigma >= 0.f)) return DPCLIP_ERR_INVALID_ARG;
+    if (dtype != DPCLIP_F32 && dtype != DPCLIP_BF16) return DPCLIP_ERR_INVALID_ARG;
+    int rc = try_fused_t1_step(layers, L, B, dtype, C, sigma, seed, stream_id0, sq_layers, clip, norms,
+                               (cudaStream_t)stream);
+    if (rc <= 0) return rc;                  // done (0) or argument error (< 0); 1 = take the general path
     for (int l = 0; l < L; ++l) {
         const dpclip_layer& y = layers[l];
         rc = dpclip_layer_sqnorms(y.A, y.lda, y.Zbar, y.ldz, B, y.T, y.d_in, y.d_out, dtype, y.has_bias,

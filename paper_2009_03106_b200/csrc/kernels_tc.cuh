@@ -2,10 +2,12 @@
 //
 //   gram_norm_kernel : per-example squared norms by the Gram identity
 //       ||sum_t zb_t (x) a_t||_F^2 = sum_{t,s} (a_t . a_s)(zb_t . zb_s)
-//     Both Gram factors of a 128 x 128 block of (t, s) pairs are accumulated in
-//     tensor memory (A A^T in columns 0..127, Zb Zb^T in 128..255, fp32) from
-//     K-major operand tiles fetched by TMA; the epilogue multiplies the two
-//     blocks element-wise and reduces, so no Gram matrix reaches HBM.  Rows are
+//     Both Gram factors of a 128 x 256 block of (t, s) pairs (one row block
+//     against two column blocks) are accumulated in tensor memory (A A^T in
+//     columns 0..255, Zb Zb^T in 256..511, fp32) from K-major operand tiles
+//     fetched by TMA; the epilogue multiplies the two blocks element-wise and
+//     reduces, so no Gram matrix reaches HBM.  One CTA walks all blocks of an
+//     example, so re-reads of a tile come from L2.  Rows are
 //     flattened (row = i*T + t), so several short examples share one block and
 //     only same-example (t, s) entries are kept; blocks below the diagonal are
 //     skipped and the strict upper ones counted twice.  The bias term
@@ -46,55 +48,77 @@ __device__ unsigned long long g_trace[148][4][256];
 namespace gram {
 constexpr int BM = 128;                       // rows per block (t and s)
 constexpr int BK = 64;                        // features per stage = one 128-byte swizzle row
-constexpr int STAGES = 4;
-constexpr int TILE_BYTES = BM * BK * 2;       // 16 KB
-constexpr int STAGE_BYTES = 2 * TILE_BYTES;   // row block + column block
-constexpr int THREADS = 192;                  // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int TILE_BYTES = BM * BK * 2;       // 16 KB: 128 rows x 64 features
+// A stage holds the row block's tile and up to two column blocks' tiles.  When every item sits on
+// the diagonal (examples of at most 256 rows, T % 128 == 0) the row block IS the first column block,
+// so stages shrink to two tiles and six of them fit: more bytes in flight per SM, which is what
+// bounds a kernel whose tiles are used once.
+template <bool DIAG_ONLY> struct Cfg {
+    static constexpr int TILES = DIAG_ONLY ? 2 : 3;
+    static constexpr int STAGE_BYTES = TILES * TILE_BYTES;
+    static constexpr int STAGES = DIAG_ONLY ? 6 : 4;
+};
+constexpr int N_EPILOGUE_WARPS = 8;
+constexpr int THREADS = 64 + 32 * N_EPILOGUE_WARPS;   // warp 0 TMA, warp 1 MMA, warps 2..9 epilogue
+constexpr int SMEM_BYTES = 4 * 3 * TILE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;   // = 6 * 2 tiles
 
 struct Params {
     int R, T, d_in, d_out, has_bias;
-    int n_items, dense_pairs, q, ppe, kmax;
+    int n_groups;          // dense (T % 128 == 0): examples; otherwise: 128-row blocks
+    int dense, q;          // q = T / 128 blocks per example in the dense case
     float* sq;
     int* status;
 };
 
-// item -> (row block, column block); false when the item is empty
-__device__ __forceinline__ bool decode(const Params& p, int item, int& rb, int& cb) {
-    if (p.dense_pairs) {                       // T % 128 == 0: q blocks per example, q(q+1)/2 pairs
-        const int e = item / p.ppe;
-        int r = item % p.ppe, j = 0;
-        while (r >= p.q - j) { r -= p.q - j; ++j; }
-        rb = e * p.q + j;
-        cb = rb + r;
+// One unit of MMA work: row block rb against column blocks cb .. cb + ncb - 1 (ncb = 1 or 2).
+struct Sub { int rb, cb, ncb; };
+
+// The sub-items of group g, in a fixed order that every warp role walks identically.
+// Row block rb pairs with column blocks rb .. cb_max(rb) (those that still hold rows of an example
+// that has rows in rb), taken two at a time so that one 128 x 256 MMA covers two of them.
+struct SubIter {
+    int rb, rb_end, cb, cb_max;
+    __device__ __forceinline__ static int cbmax(const Params& p, int rb) {
+        const long last_row = min((long)rb * BM + BM - 1, (long)p.R - 1);
+        const long e_last = last_row / p.T;
+        return (int)(min((e_last + 1) * p.T - 1, (long)p.R - 1) / BM);
+    }
+    __device__ __forceinline__ SubIter(const Params& p, int g) {
+        if (p.dense) { rb = g * p.q; rb_end = rb + p.q; } else { rb = g; rb_end = g + 1; }
+        cb = rb; cb_max = cbmax(p, rb);
+    }
+    __device__ __forceinline__ bool next(const Params& p, Sub& s) {
+        if (rb >= rb_end) return false;
+        s.rb = rb; s.cb = cb; s.ncb = cb + 1 <= cb_max ? 2 : 1;
+        cb += 2;
+        if (cb > cb_max) { ++rb; if (rb < rb_end) { cb = rb; cb_max = cbmax(p, rb); } }
         return true;
     }
-    rb = item / p.kmax;
-    cb = rb + item % p.kmax;
-    const long last_row = min((long)rb * BM + BM - 1, (long)p.R - 1);
-    const long e_last = last_row / p.T;
-    const long cb_max = min((e_last + 1) * p.T - 1, (long)p.R - 1) / BM;
-    return cb <= cb_max;
-}
+};
 }  // namespace gram
 
+template <bool DIAG_ONLY>
 __global__ void __launch_bounds__(gram::THREADS, 1)
 gram_norm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_z,
                  const gram::Params p) {
     using namespace gram;
+    constexpr int STAGES = Cfg<DIAG_ONLY>::STAGES, STAGE_BYTES = Cfg<DIAG_ONLY>::STAGE_BYTES;
+    // offset of the first column block's tile inside a stage (the row block's own tile comes first
+    // only when stages have room for it)
+    constexpr int B_OFF = DIAG_ONLY ? 0 : TILE_BYTES;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
     uint64_t* empty = full + STAGES;
     uint64_t* acc_full = empty + STAGES;
-    uint64_t* acc_empty = acc_full + 2;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+    uint64_t* acc_empty = acc_full + 1;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); }
+        mbar_init(acc_full, 1); mbar_init(acc_empty, N_EPILOGUE_WARPS);
         *abort_flag = 0;
         mbar_fence_init();
         tma_prefetch_desc(&map_a);
@@ -104,7 +128,7 @@ gram_norm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tmem_base = *tmem_slot;      // A A^T in columns 0..255, Zb Zb^T in 256..511
 
     const int nk_a = (p.d_in + BK - 1) / BK, nk_z = (p.d_out + BK - 1) / BK;
 
@@ -112,110 +136,148 @@ gram_norm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         // ------------------------------------------------ TMA producer
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0;
-            for (int item = blockIdx.x; item < p.n_items; item += gridDim.x) {
-                int rb, cb;
-                if (!decode(p, item, rb, cb)) continue;
-                const uint32_t bytes = rb == cb ? TILE_BYTES : STAGE_BYTES;
-                bool ok = true;
-                for (int kb = 0; kb < nk_a + nk_z && ok; ++kb) {
-                    const CUtensorMap* map = kb < nk_a ? &map_a : &map_z;
-                    const int x = (kb < nk_a ? kb : kb - nk_a) * BK;
-                    ok = mbar_wait(&empty[stage], phase ^ 1, abort_flag, p.status);
-                    if (!ok) break;
-                    uint8_t* dst = smem + stage * STAGE_BYTES;
-                    mbar_arrive_expect_tx(&full[stage], bytes);
-                    tma_load_2d(dst, map, &full[stage], x, rb * BM);
-                    if (cb != rb) tma_load_2d(dst + TILE_BYTES, map, &full[stage], x, cb * BM);
-                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+            bool ok = true;
+            int tr = 0;
+            DPCLIP_TRACE_AT(0, 255);
+            for (int g = blockIdx.x; g < p.n_groups && ok; g += gridDim.x) {
+                SubIter it(p, g);
+                Sub s;
+                while (ok && it.next(p, s)) {
+                    const bool diag = s.rb == s.cb;
+                    const uint32_t bytes = TILE_BYTES * (s.ncb + (diag ? 0 : 1));
+                    const int nk = nk_a + nk_z;
+                    for (int kb = 0; kb < nk; ++kb) {
+                        const CUtensorMap* map = kb < nk_a ? &map_a : &map_z;
+                        const int x = (kb < nk_a ? kb : kb - nk_a) * BK;
+                        ok = mbar_wait(&empty[stage], phase ^ 1, abort_flag, p.status);
+                        if (!ok) break;
+                        DPCLIP_TRACE_AT(0, tr); ++tr;
+                        uint8_t* dst = smem + stage * STAGE_BYTES;
+                        mbar_arrive_expect_tx(&full[stage], bytes);
+                        if (!DIAG_ONLY && !diag) tma_load_2d(dst, map, &full[stage], x, s.rb * BM);
+                        tma_load_2d(dst + B_OFF, map, &full[stage], x, s.cb * BM);
+                        if (s.ncb == 2) tma_load_2d(dst + B_OFF + TILE_BYTES, map, &full[stage], x, (s.cb + 1) * BM);
+                        if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                    }
                 }
-                if (!ok) break;
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------ MMA issuer
         if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc_bf16(BM, BM, 0, 0);
-            int stage = 0; uint32_t phase = 0; int it = 0;
-            for (int item = blockIdx.x; item < p.n_items; item += gridDim.x) {
-                int rb, cb;
-                if (!decode(p, item, rb, cb)) continue;
-                const int buf = it & 1; const uint32_t acc_phase = (it >> 1) & 1;
-                bool ok = mbar_wait(&acc_empty[buf], acc_phase ^ 1, abort_flag, p.status);
-                if (!ok) break;
-                tc_fence_after_sync();
-                for (int kb = 0; kb < nk_a + nk_z && ok; ++kb) {
-                    const bool is_a = kb < nk_a;
-                    const uint32_t d_tmem = tmem_base + buf * 256 + (is_a ? 0 : 128);
-                    const bool first = is_a ? kb == 0 : kb == nk_a;
-                    ok = mbar_wait(&full[stage], phase, abort_flag, p.status);
+            int stage = 0; uint32_t phase = 0; uint32_t acc_phase = 0;
+            bool ok = true;
+            int tr = 0;
+            for (int g = blockIdx.x; g < p.n_groups && ok; g += gridDim.x) {
+                SubIter it(p, g);
+                Sub s;
+                while (ok && it.next(p, s)) {
+                    const uint32_t idesc = make_idesc_bf16(BM, BM * s.ncb, 0, 0);
+                    ok = mbar_wait(acc_empty, acc_phase ^ 1, abort_flag, p.status);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    const uint32_t a_addr = smem_u32(smem + stage * STAGE_BYTES);
-                    const uint32_t b_addr = rb == cb ? a_addr : a_addr + TILE_BYTES;
+                    for (int kb = 0; kb < nk_a + nk_z; ++kb) {
+                        const bool is_a = kb < nk_a;
+                        const uint32_t d_tmem = tmem_base + (is_a ? 0 : 256);
+                        const bool first = is_a ? kb == 0 : kb == nk_a;
+                        ok = mbar_wait(&full[stage], phase, abort_flag, p.status);
+                        if (!ok) break;
+                        DPCLIP_TRACE_AT(2, tr); ++tr;
+                        tc_fence_after_sync();
+                        const uint32_t b_addr = smem_u32(smem + stage * STAGE_BYTES) + B_OFF;
+                        const uint32_t a_addr = (DIAG_ONLY || s.rb == s.cb) ? b_addr : b_addr - TILE_BYTES;
 #pragma unroll
-                    for (int k4 = 0; k4 < BK / 16; ++k4) {
-                        // K-major, 128-byte swizzle: 8-row groups 1024 bytes apart; 16 features = 32 bytes
-                        const uint64_t da = make_smem_desc_sw128(a_addr + k4 * 32, 16, 1024);
-                        const uint64_t db = make_smem_desc_sw128(b_addr + k4 * 32, 16, 1024);
-                        mma_bf16_ss(d_tmem, da, db, idesc, (first && k4 == 0) ? 0u : 1u);
+                        for (int k4 = 0; k4 < BK / 16; ++k4) {
+                            // K-major, 128-byte swizzle: 8-row groups 1024 bytes apart; 16 features = 32 bytes.
+                            // The two column blocks are contiguous, so N = 256 simply runs on.
+                            const uint64_t da = make_smem_desc_sw128(a_addr + k4 * 32, 16, 1024);
+                            const uint64_t db = make_smem_desc_sw128(b_addr + k4 * 32, 16, 1024);
+                            mma_bf16_ss(d_tmem, da, db, idesc, (first && k4 == 0) ? 0u : 1u);
+                        }
+                        mma_commit(&empty[stage]);
+                        if (++stage == STAGES) { stage = 0; phase ^= 1; }
                     }
-                    mma_commit(&empty[stage]);
-                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                    if (!ok) break;
+                    mma_commit(acc_full);
+                    acc_phase ^= 1;
                 }
-                if (!ok) break;
-                mma_commit(&acc_full[buf]);
-                ++it;
             }
         }
     } else {
-        // ------------------------------------------------ epilogue (warps 2..5)
-        const int quarter = warp & 3;                       // TMEM lanes 32*quarter .. +31
+        // ------------------------------------------------ epilogue (warps 2..9)
+        // warp w reads tensor-memory lanes 32*(w % 4)..+31; the two warps of a lane quarter take
+        // the two column blocks of the item.
+        const int quarter = warp & 3;
+        const int half = (warp - 2) >> 2;
         const int row_local = quarter * 32 + lane;
-        int it = 0;
-        for (int item = blockIdx.x; item < p.n_items; item += gridDim.x) {
-            int rb, cb;
-            if (!decode(p, item, rb, cb)) continue;
-            const int buf = it & 1; const uint32_t acc_phase = (it >> 1) & 1;
-            if (!mbar_wait(&acc_full[buf], acc_phase, abort_flag, p.status)) break;
-            tc_fence_after_sync();
-            const long r = (long)rb * BM + row_local;
-            const bool valid = r < p.R;
-            const long e = valid ? r / p.T : 0;
-            // columns of this block that belong to the same example as row r
-            long lo = max(e * p.T, (long)cb * BM) - (long)cb * BM;
-            long hi = min(min((e + 1) * p.T, (long)p.R), (long)cb * BM + BM) - (long)cb * BM;
-            if (!valid) { lo = 0; hi = 0; }
-            float s = 0.f, sb = 0.f;
-            const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * 256;
+        uint32_t acc_phase = 0;
+        bool ok = true;
+        int etr = 0;
+        for (int g = blockIdx.x; g < p.n_groups && ok; g += gridDim.x) {
+            SubIter it(p, g);
+            Sub s;
+            while (it.next(p, s)) {
+                ok = mbar_wait(acc_full, acc_phase, abort_flag, p.status);
+                if (!ok) break;
+                if (threadIdx.x == 64) { DPCLIP_TRACE_AT(3, etr); ++etr; }
+                acc_phase ^= 1;
+                tc_fence_after_sync();
+                float val = 0.f;
+                long e = 0;
+                bool valid = false;
+                if (half < s.ncb) {
+                    const int cbk = s.cb + half;                 // this warp's column block
+                    const long r = (long)s.rb * BM + row_local;
+                    valid = r < p.R;
+                    e = valid ? r / p.T : 0;
+                    // columns of the block that belong to the same example as row r
+                    int lo = (int)(max(e * p.T, (long)cbk * BM) - (long)cbk * BM);
+                    int hi = (int)(min(min((e + 1) * p.T, (long)p.R), (long)cbk * BM + BM) - (long)cbk * BM);
+                    if (!valid) { lo = 0; hi = 0; }
+                    float sa = 0.f, sb = 0.f;
+                    const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + half * BM;
 #pragma unroll 1
-            for (int c0 = 0; c0 < BM; c0 += 32) {
-                uint32_t va[32], vz[32];
-                tmem_ld_32x32(t_row + c0, va);
-                tmem_ld_32x32(t_row + 128 + c0, vz);
-                tmem_ld_wait();
+                    for (int c0 = 0; c0 < BM; c0 += 32) {
+                        uint32_t va[32], vz[32];
+                        tmem_ld_32x32(t_row + c0, va);
+                        tmem_ld_32x32(t_row + 256 + c0, vz);
+                        tmem_ld_wait();
+                        if (lo <= c0 && c0 + 32 <= hi) {             // whole chunk inside the example
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const int col = c0 + j;
-                    if (col >= lo && col < hi) {
-                        const float z = __uint_as_float(vz[j]);
-                        s = fmaf(__uint_as_float(va[j]), z, s);
-                        sb += z;
+                            for (int j = 0; j < 32; ++j) {
+                                const float z = __uint_as_float(vz[j]);
+                                sa = fmaf(__uint_as_float(va[j]), z, sa);
+                                sb += z;
+                            }
+                        } else if (c0 < hi && c0 + 32 > lo) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) {
+                                const int col = c0 + j;
+                                if (col >= lo && col < hi) {
+                                    const float z = __uint_as_float(vz[j]);
+                                    sa = fmaf(__uint_as_float(va[j]), z, sa);
+                                    sb += z;
+                                }
+                            }
+                        }
                     }
+                    // blocks above the diagonal stand for their mirror image too
+                    val = (cbk > s.rb ? 2.f : 1.f) * (sa + (p.has_bias ? sb : 0.f));
+                    if (hi <= lo) valid = false;
+                }
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(acc_empty);
+                if (threadIdx.x == 64) { DPCLIP_TRACE_AT(3, etr); ++etr; }
+                const long e0 = __shfl_sync(0xFFFFFFFFu, e, 0);
+                const bool uniform = __all_sync(0xFFFFFFFFu, valid && e == e0);
+                if (uniform) {
+                    val = warp_sum(val);
+                    if (lane == 0) atomicAdd(p.sq + e0, val);
+                } else if (valid) {
+                    atomicAdd(p.sq + e, val);
                 }
             }
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&acc_empty[buf]);
-            float val = (cb > rb ? 2.f : 1.f) * (s + (p.has_bias ? sb : 0.f));
-            const long e0 = __shfl_sync(0xFFFFFFFFu, e, 0);
-            const bool uniform = __all_sync(0xFFFFFFFFu, valid && e == e0);
-            if (uniform) {
-                val = warp_sum(val);
-                if (lane == 0) atomicAdd(p.sq + e0, val);
-            } else if (valid && hi > lo) {
-                atomicAdd(p.sq + e, val);
-            }
-            ++it;
         }
     }
 

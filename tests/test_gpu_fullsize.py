@@ -1,0 +1,128 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times.
+
+The oracle cannot finish these workloads whole, so it is run on sampled
+examples (norms, factors, and the clipped sum restricted to those examples via
+a clip vector that is zero elsewhere -- same shapes, same grid), and the whole
+clipped sum is checked with random bilinear probes u^T G v, which the
+definition gives in O(B T (d_in + d_out)) in fp64."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads
+from util import TOL, max_rel, rel_fro, to_device
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def dp():
+    import paper_2009_03106_b200 as pkg
+    pkg.load_library()
+    return pkg
+
+
+def _probe(A, Z, clip, u, v):
+    """u^T (sum_i c_i Zb_i^T A_i) v from the definition, fp64, chunked over examples."""
+    tot = 0.0
+    for i in range(A.shape[0]):
+        tot += clip[i] * float((Z[i].astype(np.float64) @ u) @ (A[i].astype(np.float64) @ v))
+    return tot
+
+
+def _check_layer_full(dp, A, Z, spec, dtype, sample, ws, probes=4):
+    B = A.shape[0]
+    dA, dZ = to_device(A, dtype), to_device(Z, dtype)
+    tol = TOL[dtype]
+    # norms of sampled examples, every method that applies
+    ref_sq = oracle.layer_sqnorms(A[sample], Z[sample], spec.has_bias)
+    methods = [dp.DPCLIP_AUTO]
+    if dtype == "bf16" and spec.T > 1 and spec.d_in % 8 == 0 and spec.d_out % 8 == 0:
+        methods += [dp.DPCLIP_GRAM, dp.DPCLIP_MATERIALIZE]
+    for m in methods:
+        sq = torch.empty(B, device="cuda")
+        dp.dpclip_layer_sqnorms(dA, dZ, spec.has_bias, sq, ws, m)
+        got = sq.cpu().numpy()
+        assert max_rel(np.sqrt(got[sample]), np.sqrt(ref_sq)) <= tol["norm"], (spec.name, m)
+        assert np.all(np.isfinite(got)) and np.all(got > 0)
+    # clipped sum restricted to the sampled examples: exact comparison with the oracle
+    rng = np.random.default_rng(7)
+    clip = np.zeros(B, np.float32)
+    clip[sample] = rng.uniform(0.2, 1.0, len(sample)).astype(np.float32)
+    clip[sample[0]] = 1.0
+    gW = torch.empty((spec.d_out, spec.d_in), device="cuda")
+    gb = torch.empty((spec.d_out,), device="cuda") if spec.has_bias else None
+    dp.dpclip_clipped_grad(dA, dZ, torch.from_numpy(clip).cuda(), gW, gb, ws)
+    refW, refb = oracle.clipped_grad(A[sample], Z[sample], clip[sample])
+    assert rel_fro(gW.cpu().numpy(), refW) <= tol["grad"], spec.name
+    if gb is not None:
+        assert rel_fro(gb.cpu().numpy(), refb) <= tol["grad"]
+    # whole clipped sum, random probes (E[(u^T E v)^2] = |E|_F^2 for unit Gaussian u, v)
+    full_clip = rng.uniform(0.05, 1.0, B).astype(np.float32)
+    dp.dpclip_clipped_grad(dA, dZ, torch.from_numpy(full_clip).cuda(), gW, gb, ws)
+    G = gW.cpu().numpy().astype(np.float64)
+    errs, mags = [], []
+    for _ in range(probes):
+        u = rng.standard_normal(spec.d_out); v = rng.standard_normal(spec.d_in)
+        want = _probe(A, Z, full_clip.astype(np.float64), u, v)
+        errs.append(u @ G @ v - want); mags.append(want)
+    scale = np.linalg.norm(G)        # |u^T G v| ~ |G|_F for unit Gaussian probes
+    assert np.sqrt(np.mean(np.square(errs))) <= 3 * tol["grad"] * scale, (spec.name, errs, scale)
+    assert dp.dpclip_read_status(ws) == 0
+
+
+def test_sequence_workload_full_size(dp):
+    w = workloads.seq("bf16")
+    layers = workloads.generate(w, seed=0)
+    sample = np.array([0, 17, 63, 64, 127])
+    ws = torch.empty(dp.dpclip_workspace_bytes(w.B, 256, 512, 512, dp.DPCLIP_BF16), dtype=torch.uint8, device="cuda")
+    dp.dpclip_workspace_init(ws)
+    for (A, Z), spec in zip(layers, w.layers):
+        if spec.name in ("attn_k", "attn_v"):          # same shape as attn_q
+            continue
+        _check_layer_full(dp, A, Z, spec, "bf16", sample, ws)
+
+
+def test_sequence_workload_full_step_factors(dp):
+    """Whole dpclip_step at full size: norms and factors of sampled examples."""
+    w = workloads.seq("bf16")
+    layers = workloads.generate(w, seed=1)
+    sample = np.array([3, 40, 101])
+    hb = [s.has_bias for s in w.layers]
+    plan = dp.StepPlan([dp.Layer(to_device(A, "bf16"), to_device(Z, "bf16"), b) for (A, Z), b in zip(layers, hb)])
+    C = 170.0                                           # the stated distributions give norms around 170
+    plan.run(C, 0.0, seed=0)
+    torch.cuda.synchronize()
+    assert dp.dpclip_read_status(plan.workspace) == 0
+    sq = np.stack([oracle.layer_sqnorms(A[sample], Z[sample], b) for (A, Z), b in zip(layers, hb)])
+    n_ref, c_ref = oracle.factors(sq, C)
+    assert max_rel(plan.norms.cpu().numpy()[sample], n_ref) <= TOL["bf16"]["norm"]
+    clip = plan.clip.cpu().numpy()
+    assert np.max(np.abs(clip[sample] - c_ref)) <= 5e-3
+    assert 0 < (clip < 1).sum() < w.B                   # both sides of the threshold occur
+
+
+@pytest.mark.parametrize("B,T,d_in,d_out", [(256, 16, 1024, 1024), (256, 128, 1024, 4096), (64, 2048, 1024, 1024)])
+def test_sweep_points(dp, B, T, d_in, d_out):
+    """Points of the Gram-vs-materialise sweep (both norm forms must agree with the oracle)."""
+    spec = workloads.LayerSpec("dense", T, d_in, d_out, True, "normal")
+    g = torch.Generator(device="cuda").manual_seed(B + T)
+    dA = torch.randn((B, T, d_in), generator=g, device="cuda").to(torch.bfloat16)
+    dZ = (torch.randn((B, T, d_out), generator=g, device="cuda") / (B * T) ** 0.5).to(torch.bfloat16)
+    sample = np.array([0, B // 2, B - 1])
+    A_s = dA[sample].float().cpu().numpy(); Z_s = dZ[sample].float().cpu().numpy()
+    ref_sq = oracle.layer_sqnorms(A_s, Z_s, True)
+    ws = torch.empty(dp.dpclip_workspace_bytes(B, T, d_in, d_out, dp.DPCLIP_BF16), dtype=torch.uint8, device="cuda")
+    dp.dpclip_workspace_init(ws)
+    for m in (dp.DPCLIP_GRAM, dp.DPCLIP_MATERIALIZE):
+        sq = torch.empty(B, device="cuda")
+        dp.dpclip_layer_sqnorms(dA, dZ, True, sq, ws, m)
+        assert max_rel(np.sqrt(sq.cpu().numpy()[sample]), np.sqrt(ref_sq)) <= 2e-5, m
+    clip = np.zeros(B, np.float32); clip[sample] = [1.0, 0.5, 0.25]
+    gW = torch.empty((d_out, d_in), device="cuda"); gb = torch.empty((d_out,), device="cuda")
+    dp.dpclip_clipped_grad(dA, dZ, torch.from_numpy(clip).cuda(), gW, gb, ws)
+    refW, refb = oracle.clipped_grad(A_s, Z_s, clip[sample])
+    assert rel_fro(gW.cpu().numpy(), refW) <= TOL["bf16"]["grad"]
+    assert rel_fro(gb.cpu().numpy(), refb) <= TOL["bf16"]["grad"]
+    assert dp.dpclip_read_status(ws) == 0

@@ -318,6 +318,27 @@ def test_step_mlp_large(dp, C):
     assert {0.1: frac > 0.9, 1.0: 0.3 < frac < 0.7, 10.0: frac < 0.1}[C]
 
 
+def test_step_mlp_per_layer_path(dp, monkeypatch):
+    """The general per-layer path on an all-T=1 model (the fused two-launch path is switched off)."""
+    monkeypatch.setenv("DPCLIP_NO_FUSED_T1", "1")
+    w = workloads.mlp_large(C=1.0)
+    layers = workloads.generate(w, 1)
+    _check_step(dp, w, _calibrate(w, layers, 1, 1.0), 1.0, w.sigma, 1)
+
+
+def test_step_mlp_bf16_and_odd_widths(dp):
+    """Fused T=1 step with bf16 inputs, and with widths that are not multiples of 4 (scalar paths)."""
+    w = workloads.mlp_small("bf16")
+    layers = workloads.generate(w, 0)
+    _check_step(dp, w, _calibrate(w, layers, 0, w.C), w.C, w.sigma, 0)
+    odd = workloads.Workload("mlp_odd", 9, "f32",
+                             (workloads.LayerSpec("fc1", 1, 131, 67, True, "normal"),
+                              workloads.LayerSpec("fc2", 1, 67, 5, False, "relu"),
+                              workloads.LayerSpec("fc3", 1, 5, 1, True, "relu")), 1.0, 0.7, 1.0 / 9)
+    layers = workloads.generate(odd, 3)
+    _check_step(dp, odd, _calibrate(odd, layers, 3, odd.C), odd.C, odd.sigma, 3)
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_step_cnn(dp, dtype):
     w = workloads.cnn(dtype)
