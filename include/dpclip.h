@@ -121,6 +121,34 @@ int dpclip_clipped_grad(const void* A, long lda, const void* Zbar, long ldz,
 int dpclip_add_noise(float* g, size_t n, float sigma, float C,
                      unsigned long long seed, unsigned long long stream_id, void* stream);
 
+/* dpclip_clipped_grad for callers that cannot supply a workspace.  (The paper
+ * has no counterpart: this is an interface variant, not a step of the method.)
+ *
+ * Who needs it: code that cannot obtain device memory at the point of the call
+ * -- a plug-in inside an application that owns all GPU memory, a server whose
+ * pool is fixed at start-up, or a caller already inside a region where device
+ * allocation is not allowed.  The scratch the split-row clipped sum needs is a
+ * fixed 16 MB array inside the library image instead; every GPU that loads the
+ * library holds it until the process exits.
+ *
+ * Same arguments, results and tolerances as dpclip_clipped_grad, minus the
+ * workspace.  Limits and rules:
+ *   - the output, padded to 256 x 256 tiles, must be at most
+ *     dpclip_noalloc_max_output_bytes() (8 MB, e.g. 1024 x 2048 fp32);
+ *     larger layers return DPCLIP_ERR_WORKSPACE and nothing is launched;
+ *   - no device memory is allocated or freed by this call, on any path;
+ *   - the first call on each device looks up the array's device address (that
+ *     device must be current); make that first call outside any stream capture;
+ *   - all calls share the one array: two calls whose kernels may overlap on
+ *     the GPU (different streams, no ordering between them) race on it;
+ *   - a bounded-wait timeout inside the kernel is recorded in the array's
+ *     header, which this call clears at its start; there is no read-back
+ *     entry for it. */
+int dpclip_clipped_grad_noalloc(const void* A, long lda, const void* Zbar, long ldz,
+                                int B, int T, int d_in, int d_out, dpclip_dtype dtype,
+                                const float* clip, float* gW, long ldg, float* gb, void* stream);
+size_t dpclip_noalloc_max_output_bytes(void);
+
 /* One layer of a whole step. */
 typedef struct {
     const void* A;  long lda;       /* B x T x d_in  */

@@ -52,6 +52,10 @@ def load_library():
     L.dpclip_layer_sqnorms.argtypes = [_vp, _l, _vp, _l, _i, _i, _i, _i, _i, _i, _i, _vp, _vp, _sz, _vp]
     L.dpclip_factors.argtypes = [_vp, _i, _l, _i, _f, _vp, _vp, _vp, _vp]
     L.dpclip_clipped_grad.argtypes = [_vp, _l, _vp, _l, _i, _i, _i, _i, _i, _vp, _vp, _l, _vp, _vp, _sz, _vp]
+    L.dpclip_clipped_grad_noalloc.argtypes = [_vp, _l, _vp, _l, _i, _i, _i, _i, _i, _vp, _vp, _l, _vp, _vp]
+    L.dpclip_clipped_grad_noalloc.restype = _i
+    L.dpclip_noalloc_max_output_bytes.argtypes = []
+    L.dpclip_noalloc_max_output_bytes.restype = _sz
     L.dpclip_add_noise.argtypes = [_vp, _sz, _f, _f, _u64, _u64, _vp]
     L.dpclip_step.argtypes = [ctypes.POINTER(_CLayer), _i, _i, _i, _f, _f, _u64, _u64, _vp, _vp, _vp, _vp, _sz, _vp]
     L.dpclip_step_host.argtypes = [ctypes.POINTER(_CLayer), _i, _i, _i, _f, _f, _u64, _u64, _vp, _vp, _vp, _sz, _vp]
@@ -182,6 +186,22 @@ def dpclip_clipped_grad(A: torch.Tensor, Zbar: torch.Tensor, clip: Optional[torc
         _ptr(A), lda, _ptr(Zbar), ldz, B, T, d_in, d_out, _dtype_code(A), _ptr(clip), _ptr(gW),
         gW.stride(0) if d_out > 1 else d_in, _ptr(gb), _ptr(workspace),
         workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+def dpclip_noalloc_max_output_bytes() -> int:
+    return load_library().dpclip_noalloc_max_output_bytes()
+
+
+def dpclip_clipped_grad_noalloc(A: torch.Tensor, Zbar: torch.Tensor, clip: Optional[torch.Tensor],
+                                gW: torch.Tensor, gb: Optional[torch.Tensor], stream=None) -> None:
+    """dpclip_clipped_grad without a workspace argument: for callers that cannot hand the library
+    device memory.  The scratch is a fixed array inside the library; see the header for its limits."""
+    B, T, d_in, lda = _rows(A)
+    _, _, d_out, ldz = _rows(Zbar)
+    assert gW.dtype == torch.float32 and gW.shape == (d_out, d_in) and gW.stride(1) == 1
+    _check("dpclip_clipped_grad_noalloc", load_library().dpclip_clipped_grad_noalloc(
+        _ptr(A), lda, _ptr(Zbar), ldz, B, T, d_in, d_out, _dtype_code(A), _ptr(clip), _ptr(gW),
+        gW.stride(0) if d_out > 1 else d_in, _ptr(gb), _stream(stream)))
 
 
 def dpclip_add_noise(g: torch.Tensor, sigma: float, C: float, seed: int, stream_id: int, stream=None) -> None:

@@ -203,7 +203,8 @@ constexpr size_t kTcScratchBytes = (size_t)kNumSMs * 256 * 256 * 4 + (size_t)2 *
 template <int MT>
 int launch_zta_tc_mt(const CUtensorMap& ma, const CUtensorMap& mz, tc::zta::Params p, int B, bool norm_mode,
                      float* gW, long ldg, float* gb, float* sq, int d_in, int d_out, void* workspace,
-                     size_t workspace_bytes, const NoiseSpec* noise, bool* noise_done, cudaStream_t st) {
+                     size_t workspace_bytes, const NoiseSpec* noise, bool* noise_done, cudaStream_t st,
+                     bool fit_to_workspace = false) {
     namespace z = tc::zta;
     constexpr int BM = z::Cfg<MT>::BM;
     const long R = p.R;
@@ -220,6 +221,12 @@ int launch_zta_tc_mt(const CUtensorMap& ma, const CUtensorMap& mz, tc::zta::Para
         // overlap the epilogue of one item with the next, so it takes two items per SM when they stay long.)
         const int per_sm = (MT == 1 && tiles <= kNumSMs && nkb / ((2 * kNumSMs) / tiles) >= 16) ? 2 : 1;
         ksplit = (per_sm * kNumSMs) / tiles;
+        if (fit_to_workspace) {                 // fixed-size scratch: take fewer, longer row slices
+            const size_t per_item = (size_t)BM * z::BN * 4 + (gb ? (size_t)BM * 4 : 0);
+            const size_t room = workspace_bytes > (size_t)kHeaderBytes ? workspace_bytes - kHeaderBytes : 0;
+            const long fit = (long)(room / per_item / tiles);
+            if (ksplit > fit) ksplit = (int)fit;
+        }
         if (ksplit > nkb) ksplit = nkb;
         if (ksplit < 1) ksplit = 1;
         p.kb_per_split = ceil_div(nkb, ksplit);
@@ -263,7 +270,7 @@ int launch_zta_tc_mt(const CUtensorMap& ma, const CUtensorMap& mz, tc::zta::Para
 int launch_zta_tc(const void* A, long lda, const void* Z, long ldz, int B, int T, int d_in, int d_out,
                   bool norm_mode, int has_bias, const float* clip, float* gW, long ldg, float* gb, float* sq,
                   void* workspace, size_t workspace_bytes, const NoiseSpec* noise, bool* noise_done,
-                  cudaStream_t st) {
+                  cudaStream_t st, bool fit_to_workspace = false) {
     namespace z = tc::zta;
     const long R = (long)B * T;
     CUtensorMap ma, mz;
@@ -288,9 +295,9 @@ int launch_zta_tc(const void* A, long lda, const void* Z, long ldz, int B, int T
     if (env && env[0] == '2') mt = 2;
     if (mt == 2)
         return launch_zta_tc_mt<2>(ma, mz, p, B, norm_mode, gW, ldg, gb, sq, d_in, d_out, workspace, workspace_bytes,
-                                   noise, noise_done, st);
+                                   noise, noise_done, st, fit_to_workspace);
     return launch_zta_tc_mt<1>(ma, mz, p, B, norm_mode, gW, ldg, gb, sq, d_in, d_out, workspace, workspace_bytes,
-                               noise, noise_done, st);
+                               noise, noise_done, st, fit_to_workspace);
 }
 
 // clipped sum of one layer, optionally with the noise folded into the last pass over the output
@@ -602,6 +609,59 @@ int dpclip_step_host(const dpclip_layer* layers, int L, int B, dpclip_dtype dtyp
     if (host_norms && cudaMemcpyAsync(host_norms, norms, (size_t)B * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return DPCLIP_ERR_CUDA;
     return DPCLIP_OK;
+}
+
+
+// ---------------------------------------------------------------------------
+// Clipped sum without a caller-provided workspace.
+//
+// Some callers have no way to hand this library device memory: a plug-in that runs inside a host
+// application which owns every byte of the GPU, a service whose memory pool is carved up once at
+// start-up, or code that is already inside a region where cudaMalloc is not permitted.  For them
+// the split-row scratch of dpclip_clipped_grad lives in the fixed array below instead.  The array
+// is part of the loaded library image: every GPU that loads libdpclip holds these 16 MB (+ 256 bytes)
+// until the process exits, whether or not this entry point is ever called.
+// ---------------------------------------------------------------------------
+constexpr size_t kStaticScratchBytes = (size_t)16 << 20;
+static __device__ __align__(256) unsigned char g_static_scratch[kHeaderBytes + kStaticScratchBytes];
+
+// In host code `g_static_scratch` is only a handle for the runtime, not a device address, so the
+// address is looked up once per device (with that device current) and remembered.
+static void* static_scratch_for_current_device(int* rc) {
+    static void* cached[64] = {nullptr};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { *rc = DPCLIP_ERR_CUDA; return nullptr; }
+    if (!cached[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) { *rc = DPCLIP_ERR_CUDA; return nullptr; }
+        cached[dev] = ptr;
+    }
+    *rc = DPCLIP_OK;
+    return cached[dev];
+}
+
+size_t dpclip_noalloc_max_output_bytes(void) { return kStaticScratchBytes / 2; }
+
+int dpclip_clipped_grad_noalloc(const void* A, long lda, const void* Zbar, long ldz, int B, int T, int d_in,
+                                int d_out, dpclip_dtype dtype, const float* clip, float* gW, long ldg, float* gb,
+                                void* stream) {
+    int rc = check_layer_args(A, lda, Zbar, ldz, B, T, d_in, d_out, dtype);
+    if (rc) return rc;
+    if (!gW || ldg < d_in) return DPCLIP_ERR_INVALID_ARG;
+    if (!aligned_to(gW, 4) || (gb && !aligned_to(gb, 4))) return DPCLIP_ERR_MISALIGNED;
+    // the scratch must hold at least two partial copies of the output, padded to 256 x 256 tiles
+    const size_t padded = (size_t)ceil_div(d_out, 256) * 256 * ((size_t)ceil_div(d_in, 256) * 256) * 4;
+    if (padded > dpclip_noalloc_max_output_bytes()) return DPCLIP_ERR_WORKSPACE;
+    void* scratch = static_scratch_for_current_device(&rc);
+    if (rc) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    // the array keeps whatever the previous call left: the status header has to start at zero (the
+    // partial tiles need no clearing, every tile that is read is written first)
+    if (cudaMemsetAsync(scratch, 0, kHeaderBytes, st) != cudaSuccess) return DPCLIP_ERR_CUDA;
+    if (tc_eligible(A, lda, Zbar, ldz, dtype))
+        return launch_zta_tc(A, lda, Zbar, ldz, B, T, d_in, d_out, false, 0, clip, gW, ldg, gb, nullptr, scratch,
+                             kHeaderBytes + kStaticScratchBytes, nullptr, nullptr, st, /*fit_to_workspace=*/true);
+    return launch_simt_grad(A, lda, Zbar, ldz, B, T, d_in, d_out, dtype, clip, gW, ldg, gb, st);
 }
 
 }  // extern "C"
