@@ -321,6 +321,11 @@ int try_fused_t1_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dty
     if (env && env[0] == '1') return 1;
     FusedT1Params p;
     memset(&p, 0, sizeof(p));
+    // 64 x 64 tiles: several CTAs per SM hide the global-load latency of these short (K = B) products.
+    // The 128 x 128 variant (8 x 8 register tiles, one CTA per SM) measured slower at the MLP sizes
+    // (61 vs 39 us per step on the 784-1000-1000-10, B = 128 model) and is kept for experiments only.
+    int tile = 64;
+    { const char* env = getenv("DPCLIP_T1_TILE"); if (env && atoi(env) == 128) tile = 128; }
     int tiles = 0;
     for (int l = 0; l < L; ++l) {
         const dpclip_layer& y = layers[l];
@@ -335,7 +340,7 @@ int try_fused_t1_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dty
         f.d_in = y.d_in; f.d_out = y.d_out; f.has_bias = y.has_bias ? 1 : 0;
         f.vec_a = vec4_ok(y.A, y.lda, dtype); f.vec_z = vec4_ok(y.Zbar, y.ldz, dtype);
         f.gW = y.gW; f.gb = y.has_bias ? y.gb : nullptr;
-        f.tiles_m = ceil_div(y.d_out, SIMT_BM); f.tiles_n = ceil_div(y.d_in + f.has_bias, SIMT_BN);
+        f.tiles_m = ceil_div(y.d_out, tile); f.tiles_n = ceil_div(y.d_in + f.has_bias, tile);
         f.tile_begin = tiles;
         tiles += f.tiles_m * f.tiles_n;
     }
@@ -344,16 +349,27 @@ int try_fused_t1_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dty
     p.k0 = (uint32_t)seed; p.k1 = (uint32_t)(seed >> 32); p.stream_id0 = stream_id0;
     p.sq = sq; p.clip = clip; p.norms = norms;
     const int rows = L * B;
-    const int grid_n = ceil_div(rows, 4);
+    const int grid_n = rows;
     const int grid_g = tiles < 4 * kNumSMs ? tiles : 4 * kNumSMs;
+    const int smem64 = FusedT1Cfg<64>::SMEM_BYTES, smem128 = FusedT1Cfg<128>::SMEM_BYTES;
     if (dtype == DPCLIP_F32) {
         t1_all_norms_kernel<float><<<grid_n, 128, 0, st>>>(p);
         if (launch_status()) return DPCLIP_ERR_CUDA;
-        t1_all_grads_kernel<float><<<grid_g, SIMT_THREADS, 0, st>>>(p);
+        if (tile == 128) {
+            if (!enable_smem(t1_all_grads_kernel<float, 128>, smem128)) return DPCLIP_ERR_CUDA;
+            t1_all_grads_kernel<float, 128><<<grid_g, SIMT_THREADS, smem128, st>>>(p);
+        } else {
+            t1_all_grads_kernel<float, 64><<<grid_g, SIMT_THREADS, smem64, st>>>(p);
+        }
     } else {
         t1_all_norms_kernel<__nv_bfloat16><<<grid_n, 128, 0, st>>>(p);
         if (launch_status()) return DPCLIP_ERR_CUDA;
-        t1_all_grads_kernel<__nv_bfloat16><<<grid_g, SIMT_THREADS, 0, st>>>(p);
+        if (tile == 128) {
+            if (!enable_smem(t1_all_grads_kernel<__nv_bfloat16, 128>, smem128)) return DPCLIP_ERR_CUDA;
+            t1_all_grads_kernel<__nv_bfloat16, 128><<<grid_g, SIMT_THREADS, smem128, st>>>(p);
+        } else {
+            t1_all_grads_kernel<__nv_bfloat16, 64><<<grid_g, SIMT_THREADS, smem64, st>>>(p);
+        }
     }
     return launch_status();
 }

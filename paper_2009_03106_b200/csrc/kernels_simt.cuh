@@ -94,24 +94,27 @@ zta_simt_kernel(SimtParams p) {
 #pragma unroll
             for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
 
+        float cf = 1.f;
         auto fetch = [&](int slab, float4& zr, float4& ar) {
             const long r = row_begin + (long)slab * SIMT_BK + lk;
             const bool ok = r < row_end;
             zr = simt_load_row4(Z, p.ldz, r, m0 + lc, p.d_out, ok, p.vec_z != 0, false);
             ar = simt_load_row4(A, p.lda, r, n0 + lc, p.d_in, ok, p.vec_a != 0, p.has_bias != 0);
+            cf = 1.f;
             if (GRAD) {
-                if (ok && p.clip) {
-                    const float c = p.clip[r / p.T];
-                    zr.x *= c; zr.y *= c; zr.z *= c; zr.w *= c;
-                }
+                if (ok && p.clip) cf = __ldg(p.clip + r / p.T);
             }
+        };
+        // the loaded values are first touched here, after the FMAs of the current slab
+        auto stash = [&](int buf, const float4& zr, const float4& ar) {
+            *reinterpret_cast<float4*>(&Zs[buf][lk][lc]) = make_float4(zr.x * cf, zr.y * cf, zr.z * cf, zr.w * cf);
+            *reinterpret_cast<float4*>(&As[buf][lk][lc]) = ar;
         };
 
         float4 zr, ar;
         if (n_slabs > 0) {
             fetch(0, zr, ar);
-            *reinterpret_cast<float4*>(&Zs[0][lk][lc]) = zr;
-            *reinterpret_cast<float4*>(&As[0][lk][lc]) = ar;
+            stash(0, zr, ar);
         }
         __syncthreads();
         for (int s = 0; s < n_slabs; ++s) {
@@ -129,10 +132,7 @@ zta_simt_kernel(SimtParams p) {
 #pragma unroll
                     for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(zz[i], aa[j], acc[i][j]);
             }
-            if (more) {
-                *reinterpret_cast<float4*>(&Zs[buf ^ 1][lk][lc]) = zr;
-                *reinterpret_cast<float4*>(&As[buf ^ 1][lk][lc]) = ar;
-            }
+            if (more) stash(buf ^ 1, zr, ar);
             __syncthreads();
         }
 

@@ -727,8 +727,16 @@ reduce_partials_kernel(const ReduceParams p) {
         const float* src = p.part + (size_t)(tm * p.tiles_n + tn) * tile_elems + (size_t)(m - tm * p.BM) * zta::BN +
                            (n - tn * zta::BN);
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int ks = 0; ks < p.ksplit; ++ks) {
-            const float4 v = *reinterpret_cast<const float4*>(src + ks * ks_stride);
+        int ks = 0;
+        for (; ks + 8 <= p.ksplit; ks += 8) {            // eight independent loads in flight, fixed add order
+            float4 v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) v[u] = __ldcs(reinterpret_cast<const float4*>(src + (ks + u) * ks_stride));
+#pragma unroll
+            for (int u = 0; u < 8; ++u) { acc.x += v[u].x; acc.y += v[u].y; acc.z += v[u].z; acc.w += v[u].w; }
+        }
+        for (; ks < p.ksplit; ++ks) {
+            const float4 v = __ldcs(reinterpret_cast<const float4*>(src + ks * ks_stride));
             acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
         }
         if (p.noise_scale > 0.f) {
