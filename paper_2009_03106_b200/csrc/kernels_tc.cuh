@@ -376,9 +376,7 @@ zta_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            mbar_init(&full[s], 1); mbar_init(&ready[s], N_TRANSFORM_WARPS);
-            // a stage is released by the MMA commit and, in layers with a bias, by the 8 bias/epilogue warps
-            mbar_init(&empty[s], 1 + (p.do_bias ? N_EPILOGUE_WARPS : 0));
+            mbar_init(&full[s], 1); mbar_init(&ready[s], N_TRANSFORM_WARPS); mbar_init(&empty[s], 1);
         }
         for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], N_EPILOGUE_WARPS); }
         *abort_flag = 0;
@@ -473,6 +471,13 @@ zta_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
         int tr = 0;
         for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
             const Item w = decode<MT>(p, item);
+            // bias gradient = column sums of the scaled Zb tile; the values pass through these threads'
+            // registers anyway, so the sums cost no extra shared-memory traffic
+            float cs[MT][8];
+#pragma unroll
+            for (int h = 0; h < MT; ++h)
+#pragma unroll
+                for (int j = 0; j < 8; ++j) cs[h][j] = 0.f;
             for (int kb = 0; kb < w.nkb; ++kb) {
                 // the factors of this stage's rows are fetched BEFORE waiting for the tile, so the
                 // global-load latency overlaps the wait instead of sitting between TMA and MMA
@@ -481,6 +486,10 @@ zta_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
                 const int rem0 = blk0 - e_first * p.T;
                 // fast path: the whole stage lies inside one example and inside the row range
                 const bool uniform = (rem0 + BK <= p.T) && (blk0 + BK <= w.row_end);
+                // GRAD: every n-tile of a row range sees the same Zb rows; the bias sums of stage kb are
+                // taken by the n-tile with kb % tiles_n == tn (equal shares).  NORM: the sums must be
+                // complete before they are squared, so n-tile 0 takes them all.
+                const bool bias_here = p.do_bias && (p.norm_mode ? w.tn == 0 : (kb % p.tiles_n) == w.tn);
                 float fr[4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
@@ -494,13 +503,13 @@ zta_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
                 if (!ok) break;
                 if (t == 0) { DPCLIP_TRACE_AT(1, tr); ++tr; }
                 uint8_t* zt = smem + stage * STAGE_BYTES;
-                if (!(uniform && fr[0] == 1.f)) {
+                if (bias_here || !(uniform && fr[0] == 1.f)) {
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         const float f = fr[i];
-                        if (f != 1.f) {
+                        if (f != 1.f || bias_here) {
                             // packed bf16 path: f = f_hi + f_lo (two bf16); z*f_lo is tiny, so the fused
-                            // multiply-add z*f_hi + (z*f_lo) rounds the product once, like the fp32 path
+                            // multiply-add z*f_hi + (z*f_lo) rounds the product once
                             const __nv_bfloat16 fh = __float2bfloat16_rn(f);
                             const __nv_bfloat16 fl = __float2bfloat16_rn(f - __bfloat162float(fh));
                             const __nv_bfloat162 fh2 = __halves2bfloat162(fh, fh), fl2 = __halves2bfloat162(fl, fl);
@@ -508,10 +517,20 @@ zta_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
                             for (int h = 0; h < MT; ++h) {
                                 uint4* ptr = reinterpret_cast<uint4*>(zt + h * 2 * CHUNK_BYTES + off + i * 2048);
                                 uint4 v = *ptr;
-                                __nv_bfloat162* z2 = reinterpret_cast<__nv_bfloat162*>(&v);
+                                if (f != 1.f) {
+                                    __nv_bfloat162* z2 = reinterpret_cast<__nv_bfloat162*>(&v);
 #pragma unroll
-                                for (int u = 0; u < 4; ++u) z2[u] = __hfma2(z2[u], fh2, __hmul2(z2[u], fl2));
-                                *ptr = v;
+                                    for (int u = 0; u < 4; ++u) z2[u] = __hfma2(z2[u], fh2, __hmul2(z2[u], fl2));
+                                    *ptr = v;
+                                }
+                                if (bias_here) {
+                                    const uint32_t wds[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                                    for (int u = 0; u < 4; ++u) {
+                                        cs[h][2 * u] += __uint_as_float(wds[u] << 16);
+                                        cs[h][2 * u + 1] += __uint_as_float(wds[u] & 0xFFFF0000u);
+                                    }
+                                }
                             }
                         }
                     }
@@ -523,6 +542,31 @@ zta_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
                 if (++stage == STAGES) { stage = 0; phase ^= 1; }
             }
             if (!ok) break;
+            if (p.do_bias && !(p.norm_mode && w.tn != 0)) {
+                // finish the column sums over the 16 row-subsets (16 consecutive lanes)
+                float ssq = 0.f;
+#pragma unroll
+                for (int h = 0; h < MT; ++h)
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        float c = cs[h][j];
+                        c += __shfl_xor_sync(0xFFFFFFFFu, c, 1);
+                        c += __shfl_xor_sync(0xFFFFFFFFu, c, 2);
+                        c += __shfl_xor_sync(0xFFFFFFFFu, c, 4);
+                        c += __shfl_xor_sync(0xFFFFFFFFu, c, 8);
+                        ssq = fmaf(c, c, ssq);
+                        if (!p.norm_mode && rs == 0) {
+                            const int ml = h * 128 + q * 8 + j;
+                            if (p.bias_part) p.bias_part[(size_t)item * C::BM + ml] = c;
+                            else if (w.m0 + ml < p.d_out) red_add_f32(p.gb + w.m0 + ml, c);
+                        }
+                    }
+                if (p.norm_mode) {
+                    if (rs != 0) ssq = 0.f;
+                    ssq = warp_sum(ssq);
+                    if (lane == 0) atomicAdd(p.sq + w.example, ssq);
+                }
+            }
         }
     } else {
         // ------------------------------------------------ epilogue (8 warps)
@@ -534,88 +578,9 @@ zta_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
         const int h = MT == 2 ? g : 0;
         const int col_begin = MT == 2 ? 0 : g * (BN / 2);
         const int col_end = MT == 2 ? BN : col_begin + BN / 2;
-        // While the main loop runs, these warps are otherwise idle: in layers with a bias they take the
-        // column sums of the (already scaled) Zb tile, which is the clipped bias gradient
-        // gb[o] = sum_k f_k zb[k][o].  Same thread -> (column chunk, rows) mapping as the transform.
-        const int bt = threadIdx.x - 32 * (2 + N_TRANSFORM_WARPS);
-        const int bq = bt >> 4, brs = bt & 15;
-        const uint32_t boff = (bq >> 3) * CHUNK_BYTES + brs * 128 + (((bq & 7) ^ (brs & 7)) << 4);
-        int stage = 0; uint32_t phase = 0;
         int it = 0;
-        bool ok = true;
-        for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
+        for (int item = blockIdx.x; item < p.n_items; item += gridDim.x) {
             const Item w = decode<MT>(p, item);
-            if (p.do_bias) {
-                float cs[MT][8];
-#pragma unroll
-                for (int hh = 0; hh < MT; ++hh)
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) cs[hh][j] = 0.f;
-                for (int kb = 0; kb < w.nkb; ++kb) {
-                    ok = mbar_wait(&ready[stage], phase, abort_flag, p.status);
-                    if (!ok) break;
-                    // GRAD: every n-tile of a row range sees the same Zb rows; stage kb is summed by the
-                    // n-tile with kb % tiles_n == tn, so all items carry an equal share.  NORM: the sums
-                    // must be complete before they are squared, so n-tile 0 takes them all.
-                    const bool mine = p.norm_mode ? w.tn == 0 : (kb % p.tiles_n) == w.tn;
-                    if (mine) {
-                        const uint8_t* zt = smem + stage * STAGE_BYTES;
-#pragma unroll
-                        for (int i = 0; i < 4; ++i)
-#pragma unroll
-                            for (int hh = 0; hh < MT; ++hh) {
-                                const uint4 v = *reinterpret_cast<const uint4*>(zt + hh * 2 * CHUNK_BYTES + boff + i * 2048);
-                                const uint32_t wds[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-                                for (int u = 0; u < 4; ++u) {
-                                    cs[hh][2 * u] += __uint_as_float(wds[u] << 16);
-                                    cs[hh][2 * u + 1] += __uint_as_float(wds[u] & 0xFFFF0000u);
-                                }
-                            }
-                    }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&empty[stage]);
-                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
-                }
-                if (!ok) break;
-                if (p.norm_mode) {
-                    if (w.tn == 0) {
-                        // complete the column sums over the 16 row-subsets (16 consecutive lanes), then square
-                        float ssq = 0.f;
-#pragma unroll
-                        for (int hh = 0; hh < MT; ++hh)
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) {
-                                float c = cs[hh][j];
-                                c += __shfl_xor_sync(0xFFFFFFFFu, c, 1);
-                                c += __shfl_xor_sync(0xFFFFFFFFu, c, 2);
-                                c += __shfl_xor_sync(0xFFFFFFFFu, c, 4);
-                                c += __shfl_xor_sync(0xFFFFFFFFu, c, 8);
-                                ssq = fmaf(c, c, ssq);
-                            }
-                        if (brs != 0) ssq = 0.f;
-                        ssq = warp_sum(ssq);
-                        if (lane == 0) atomicAdd(p.sq + w.example, ssq);
-                    }
-                } else {
-                    // one value per column: finish the sum over the 16 row-subsets first
-#pragma unroll
-                    for (int hh = 0; hh < MT; ++hh)
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            float c = cs[hh][j];
-                            c += __shfl_xor_sync(0xFFFFFFFFu, c, 1);
-                            c += __shfl_xor_sync(0xFFFFFFFFu, c, 2);
-                            c += __shfl_xor_sync(0xFFFFFFFFu, c, 4);
-                            c += __shfl_xor_sync(0xFFFFFFFFu, c, 8);
-                            if (brs == 0) {
-                                const int ml = hh * 128 + bq * 8 + j;
-                                if (p.bias_part) p.bias_part[(size_t)item * C::BM + ml] = c;
-                                else if (w.m0 + ml < p.d_out) red_add_f32(p.gb + w.m0 + ml, c);
-                            }
-                        }
-                }
-            }
             const int buf = it % NBUF; const uint32_t acc_phase = (it / NBUF) & 1;
             if (!mbar_wait(&acc_full[buf], acc_phase, abort_flag, p.status)) break;
             if (threadIdx.x == 64 + 32 * N_TRANSFORM_WARPS) DPCLIP_TRACE_AT(3, 2 * it);
