@@ -121,6 +121,19 @@ int dpclip_clipped_grad(const void* A, long lda, const void* Zbar, long ldz,
 int dpclip_add_noise(float* g, size_t n, float sigma, float C,
                      unsigned long long seed, unsigned long long stream_id, void* stream);
 
+/* Clipped sum and noise of ONE layer in one call: dpclip_clipped_grad followed by
+ * dpclip_add_noise on gW (stream stream_id_w) and on gb (stream stream_id_b),
+ * with the noise folded into the last pass over the output where the layer's
+ * kernel has one (Algorithm 1, last line: the noised clipped sum is what is
+ * released).  gW has dense rows (row stride d_in).  Same results as the two
+ * separate calls, bit for bit. */
+int dpclip_clipped_grad_noise(const void* A, long lda, const void* Zbar, long ldz,
+                              int B, int T, int d_in, int d_out, dpclip_dtype dtype,
+                              const float* clip, float* gW, float* gb,
+                              float sigma, float C, unsigned long long seed,
+                              unsigned long long stream_id_w, unsigned long long stream_id_b,
+                              void* workspace, size_t workspace_bytes, void* stream);
+
 /* dpclip_clipped_grad for callers that cannot supply a workspace.  (The paper
  * has no counterpart: this is an interface variant, not a step of the method.)
  *

@@ -56,6 +56,9 @@ def load_library():
     L.dpclip_clipped_grad_noalloc.restype = _i
     L.dpclip_noalloc_max_output_bytes.argtypes = []
     L.dpclip_noalloc_max_output_bytes.restype = _sz
+    L.dpclip_clipped_grad_noise.argtypes = [_vp, _l, _vp, _l, _i, _i, _i, _i, _i, _vp, _vp, _vp, _f, _f, _u64, _u64,
+                                            _u64, _vp, _sz, _vp]
+    L.dpclip_clipped_grad_noise.restype = _i
     L.dpclip_add_noise.argtypes = [_vp, _sz, _f, _f, _u64, _u64, _vp]
     L.dpclip_step.argtypes = [ctypes.POINTER(_CLayer), _i, _i, _i, _f, _f, _u64, _u64, _vp, _vp, _vp, _vp, _sz, _vp]
     L.dpclip_step_host.argtypes = [ctypes.POINTER(_CLayer), _i, _i, _i, _f, _f, _u64, _u64, _vp, _vp, _vp, _sz, _vp]
@@ -188,6 +191,18 @@ def dpclip_clipped_grad(A: torch.Tensor, Zbar: torch.Tensor, clip: Optional[torc
         workspace.numel() * workspace.element_size(), _stream(stream)))
 
 
+def dpclip_clipped_grad_noise(A: torch.Tensor, Zbar: torch.Tensor, clip: Optional[torch.Tensor], gW: torch.Tensor,
+                              gb: Optional[torch.Tensor], sigma: float, C: float, seed: int, stream_id_w: int,
+                              stream_id_b: int, workspace: torch.Tensor, stream=None) -> None:
+    B, T, d_in, lda = _rows(A)
+    _, _, d_out, ldz = _rows(Zbar)
+    assert gW.dtype == torch.float32 and gW.shape == (d_out, d_in) and gW.is_contiguous()
+    _check("dpclip_clipped_grad_noise", load_library().dpclip_clipped_grad_noise(
+        _ptr(A), lda, _ptr(Zbar), ldz, B, T, d_in, d_out, _dtype_code(A), _ptr(clip), _ptr(gW), _ptr(gb),
+        sigma, C, seed, stream_id_w, stream_id_b, _ptr(workspace), workspace.numel() * workspace.element_size(),
+        _stream(stream)))
+
+
 def dpclip_noalloc_max_output_bytes() -> int:
     return load_library().dpclip_noalloc_max_output_bytes()
 
@@ -264,15 +279,56 @@ class StepPlan:
     def run(self, C: float, sigma: float, seed: int, stream_id0: int = 0, stream=None) -> None:
         dpclip_step(self, C, sigma, seed, stream_id0, stream)
 
-    def capture(self, C: float, sigma: float, seed: int, stream_id0: int = 0):
-        """Record one dpclip_step call into a CUDA graph (the launch-bound small workloads spend most
-        of a step in launch gaps).  Returns the graph; `graph.replay()` re-runs the same kernels on the
-        same buffers with the same (C, sigma, seed, stream ids)."""
+    def capture(self, C: float, sigma: float, seed: int, stream_id0: int = 0, branches: int = 1):
+        """Record one step into a CUDA graph (the launch-bound small workloads spend most of a step
+        in launch gaps).  Returns the graph; `graph.replay()` re-runs the same kernels on the same
+        buffers with the same (C, sigma, seed, stream ids).
+
+        branches = 1 records one dpclip_step call.  branches > 1 records the same path as per-layer
+        entry-point calls spread over that many streams (layers are independent within the norm
+        stage and within the clipped-sum stage), so the graph has parallel branches and one layer's
+        kernel starts on SMs the previous layer's kernel has already left.  Pure stream plumbing:
+        the arithmetic is the same kernels either way."""
         self.run(C, sigma, seed, stream_id0)          # warm-up outside capture (function attributes, maps)
         torch.cuda.synchronize()
         graph = torch.cuda.CUDAGraph()
+        if branches <= 1:
+            with torch.cuda.graph(graph):
+                self.run(C, sigma, seed, stream_id0)
+            return graph
+        if not hasattr(self, "_branch_ws"):
+            self._branch_ws = [self.workspace] + [torch.empty_like(self.workspace) for _ in range(branches - 1)]
+            for w in self._branch_ws[1:]:
+                dpclip_workspace_init(w)
+            self._streams = [torch.cuda.Stream() for _ in range(branches - 1)]
+            torch.cuda.synchronize()
         with torch.cuda.graph(graph):
-            self.run(C, sigma, seed, stream_id0)
+            main = torch.cuda.current_stream()
+            streams = [main] + self._streams
+
+            def fork():
+                ev = torch.cuda.Event(); ev.record(main)
+                for s in streams[1:]:
+                    s.wait_event(ev)
+
+            def join():
+                for s in streams[1:]:
+                    ev = torch.cuda.Event(); ev.record(s); main.wait_event(ev)
+
+            fork()
+            for l, y in enumerate(self.layers):
+                b = l % branches
+                with torch.cuda.stream(streams[b]):
+                    dpclip_layer_sqnorms(y.A, y.Zbar, y.has_bias, self.sq_layers[l], self._branch_ws[b], y.method)
+            join()
+            dpclip_factors(self.sq_layers, C, self.clip, self.norms)
+            fork()
+            for l, y in enumerate(self.layers):
+                b = l % branches
+                with torch.cuda.stream(streams[b]):
+                    dpclip_clipped_grad_noise(y.A, y.Zbar, self.clip, self.gW[l], self.gb[l], sigma, C, seed,
+                                              stream_id0 + 2 * l, stream_id0 + 2 * l + 1, self._branch_ws[b])
+            join()
         return graph
 
 

@@ -7,6 +7,7 @@
 #include "kernels_stream.cuh"
 #include "kernels_tc.cuh"
 #include "kernels_fused_t1.cuh"
+#include "kernels_narrow.cuh"
 
 #include <stdlib.h>
 
@@ -64,8 +65,40 @@ int launch_t1_norms(const void* A, long lda, const void* Z, long ldz, int B, int
     return launch_status();
 }
 
+// narrow layers (d_in + bias <= 32, d_out <= 64, T > 1): streaming kernel with one lane per column
+inline bool narrow_layer(int T, int d_in, int d_out, int has_bias, long lda, long ldz) {
+    const char* env = getenv("DPCLIP_NO_NARROW");
+    if (env && env[0] == '1') return false;
+    // dense rows: a run of rows is then one contiguous run of memory, which is what the kernel streams
+    return T > 1 && d_in + (has_bias ? 1 : 0) <= 32 && d_out <= 64 && lda == d_in && ldz == d_out;
+}
+
+template <typename T, int MAXM, bool GRAD>
+int launch_narrow_inst(const NarrowParams& p, int grid, cudaStream_t st) {
+    constexpr int smem = NarrowCfg<MAXM>::SMEM_BYTES;
+    if (cudaFuncSetAttribute(narrow_kernel<T, MAXM, GRAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
+        cudaSuccess) return DPCLIP_ERR_CUDA;
+    narrow_kernel<T, MAXM, GRAD><<<grid, NARROW_THREADS, smem, st>>>(p);
+    return launch_status();
+}
+
+template <bool GRAD>
+int launch_narrow(const NarrowParams& p, int grid, int d_out, dpclip_dtype dtype, cudaStream_t st) {
+    if (dtype == DPCLIP_F32)
+        return d_out <= 32 ? launch_narrow_inst<float, 32, GRAD>(p, grid, st) : launch_narrow_inst<float, 64, GRAD>(p, grid, st);
+    return d_out <= 32 ? launch_narrow_inst<__nv_bfloat16, 32, GRAD>(p, grid, st)
+                       : launch_narrow_inst<__nv_bfloat16, 64, GRAD>(p, grid, st);
+}
+
 int launch_simt_norms(const void* A, long lda, const void* Z, long ldz, int B, int T, int d_in, int d_out,
                       dpclip_dtype dtype, int has_bias, float* sq, cudaStream_t st) {
+    if (narrow_layer(T, d_in, d_out, has_bias, lda, ldz)) {
+        NarrowParams q;
+        memset(&q, 0, sizeof(q));
+        q.A = A; q.lda = lda; q.Z = Z; q.ldz = ldz; q.T = T; q.d_in = d_in; q.d_out = d_out;
+        q.has_bias = has_bias ? 1 : 0; q.sq = sq;
+        return launch_narrow<false>(q, B, d_out, dtype, st);
+    }
     SimtParams p;
     fill_simt_params(p, A, lda, Z, ldz, T, d_in, d_out, has_bias, dtype);
     const int n_tiles = p.tiles_m * p.tiles_n;
@@ -84,6 +117,22 @@ int launch_simt_norms(const void* A, long lda, const void* Z, long ldz, int B, i
 
 int launch_simt_grad(const void* A, long lda, const void* Z, long ldz, int B, int T, int d_in, int d_out,
                      dpclip_dtype dtype, const float* clip, float* gW, long ldg, float* gb, cudaStream_t st) {
+    if (narrow_layer(T, d_in, d_out, gb != nullptr, lda, ldz)) {
+        NarrowParams q;
+        memset(&q, 0, sizeof(q));
+        q.A = A; q.lda = lda; q.Z = Z; q.ldz = ldz; q.T = T; q.d_in = d_in; q.d_out = d_out;
+        q.has_bias = gb ? 1 : 0; q.clip = clip; q.gW = gW; q.ldg = ldg; q.gb = gb;
+        q.rows_total = (long)B * T;
+        int grid = 2 * kNumSMs;
+        const long min_rows = 8 * 32;                              // at least one chunk per warp
+        if ((long)grid * min_rows > q.rows_total) grid = (int)((q.rows_total + min_rows - 1) / min_rows);
+        q.rows_per_cta = (q.rows_total + grid - 1) / grid;
+        grid = (int)((q.rows_total + q.rows_per_cta - 1) / q.rows_per_cta);
+        if (cudaMemset2DAsync(gW, sizeof(float) * (size_t)ldg, 0, sizeof(float) * (size_t)d_in, d_out, st) !=
+            cudaSuccess) return DPCLIP_ERR_CUDA;
+        if (gb && cudaMemsetAsync(gb, 0, sizeof(float) * (size_t)d_out, st) != cudaSuccess) return DPCLIP_ERR_CUDA;
+        return launch_narrow<true>(q, grid, d_out, dtype, st);
+    }
     SimtParams p;
     fill_simt_params(p, A, lda, Z, ldz, T, d_in, d_out, gb != nullptr, dtype);
     const int n_tiles = p.tiles_m * p.tiles_n;
@@ -261,7 +310,11 @@ int launch_zta_tc_mt(const CUtensorMap& ma, const CUtensorMap& mz, tc::zta::Para
         if (noise_done) *noise_done = true;
     }
     const long n_vec = (long)d_out * ((d_in + 3) / 4);
-    long blocks = (n_vec + 255) / 256;
+    // widen the per-output lane groups until the grid has about two CTAs per SM (or a full warp per output)
+    int lanes = 1;
+    while (lanes < 32 && lanes * 2 <= ksplit && n_vec * lanes < 2L * kNumSMs * 256) lanes *= 2;
+    r.lanes = lanes;
+    long blocks = (n_vec * lanes + 255) / 256;
     if (blocks > 8L * kNumSMs) blocks = 8L * kNumSMs;
     tc::reduce_partials_kernel<<<(unsigned)blocks, 256, 0, st>>>(r);
     return launch_status();
@@ -491,6 +544,27 @@ int dpclip_clipped_grad(const void* A, long lda, const void* Zbar, long ldz, int
         return DPCLIP_ERR_WORKSPACE;
     return clipped_grad_impl(A, lda, Zbar, ldz, B, T, d_in, d_out, dtype, clip, gW, ldg, gb, workspace,
                              workspace_bytes, nullptr, nullptr, (cudaStream_t)stream);
+}
+
+int dpclip_clipped_grad_noise(const void* A, long lda, const void* Zbar, long ldz, int B, int T, int d_in,
+                              int d_out, dpclip_dtype dtype, const float* clip, float* gW, float* gb, float sigma,
+                              float C, unsigned long long seed, unsigned long long stream_id_w,
+                              unsigned long long stream_id_b, void* workspace, size_t workspace_bytes,
+                              void* stream) {
+    int rc = check_layer_args(A, lda, Zbar, ldz, B, T, d_in, d_out, dtype);
+    if (rc) return rc;
+    if (!gW || !(sigma >= 0.f) || !(C >= 0.f)) return DPCLIP_ERR_INVALID_ARG;
+    if (!aligned_to(gW, 4) || (gb && !aligned_to(gb, 4))) return DPCLIP_ERR_MISALIGNED;
+    if (!workspace || workspace_bytes < dpclip_workspace_bytes(B, T, d_in, d_out, dtype, DPCLIP_AUTO))
+        return DPCLIP_ERR_WORKSPACE;
+    NoiseSpec ns = {sigma * C, seed, stream_id_w, stream_id_b};
+    bool noise_done = false;
+    rc = clipped_grad_impl(A, lda, Zbar, ldz, B, T, d_in, d_out, dtype, clip, gW, d_in, gb, workspace,
+                           workspace_bytes, &ns, &noise_done, (cudaStream_t)stream);
+    if (rc || noise_done) return rc;
+    rc = dpclip_add_noise(gW, (size_t)d_out * d_in, sigma, C, seed, stream_id_w, stream);
+    if (rc || !gb) return rc;
+    return dpclip_add_noise(gb, (size_t)d_out, sigma, C, seed, stream_id_b, stream);
 }
 
 int dpclip_add_noise(float* g, size_t n, float sigma, float C, unsigned long long seed,

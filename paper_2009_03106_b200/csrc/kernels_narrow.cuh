@@ -1,0 +1,187 @@
+// Streaming kernel for narrow layers: d_in (+1 with a bias) <= 32 and d_out <= 64,
+// e.g. the first 3x3 convolution of an RGB network (d_in = 27, T = H*W large).
+//
+// Such a layer is pure streaming (a few hundred flops per row, rows of odd
+// length that neither TMA nor per-row 128-bit loads can fetch), and a 64 x 64
+// tile kernel wastes most of its lanes on it.  Here a lane owns one column n of
+// the product Zb^T [A | 1] (d_out accumulators in registers) and a warp walks
+// the rows in chunks of 32 (16 when d_out > 32).  With dense rows a chunk of A
+// and of Zb is one contiguous run of memory whatever the row length, so the
+// warp fetches it with 128-bit loads (all issued before the previous chunk is
+// computed, i.e. a whole chunk per warp in flight), parks it in shared memory,
+// and then every lane reads its own a[row][n] and the zb row as broadcast
+// 128-bit loads.  The eight warps of a CTA take interleaved chunks; their
+// partial tiles are combined in shared memory at the end.
+//
+//   NORM: one CTA per example; the tile is squared and summed -> sq[i].
+//   GRAD: one CTA per row slice, each row weighted by its example's clip factor
+//         (applied to a[row][n] as it is read); the tile is added to gW / gb
+//         with fp32 atomics.
+#pragma once
+#include "common.cuh"
+
+namespace dpclip {
+
+constexpr int NARROW_THREADS = 256, NARROW_WARPS = NARROW_THREADS / 32;
+
+struct NarrowParams {
+    const void* A; long lda;
+    const void* Z; long ldz;
+    int T, d_in, d_out, has_bias;
+    long rows_total, rows_per_cta;      // GRAD
+    const float* clip; float* gW; long ldg; float* gb;
+    float* sq;                          // NORM
+};
+
+template <int MAXM> struct NarrowCfg {
+    static constexpr int CH = MAXM == 32 ? 32 : 16;                 // rows per warp chunk
+    static constexpr int A_FLOATS = CH * 32, Z_FLOATS = CH * MAXM + 64;   // + slack for reads past short rows
+    static constexpr int SMEM_BYTES = NARROW_WARPS * (A_FLOATS + Z_FLOATS) * 4 + MAXM * 33 * 4 + 128;
+};
+
+// n consecutive elements starting at src -> fp32 in shared memory, by the whole warp.  128-bit loads
+// when src is 16-byte aligned; the loads are issued in `issue`, the values stored in `park`.
+template <typename T, int NV> struct ChunkRegs { uint4 v[NV]; };
+
+template <typename T, int NV>
+__device__ __forceinline__ void chunk_issue(const T* __restrict__ src, int n, int lane, ChunkRegs<T, NV>& r, bool& vec) {
+    constexpr int EPV = 16 / (int)sizeof(T);                        // elements per 128-bit load
+    vec = (reinterpret_cast<uintptr_t>(src) & 15) == 0;
+    if (vec) {
+#pragma unroll
+        for (int u = 0; u < NV; ++u) {
+            const int e = (u * 32 + lane) * EPV;
+            r.v[u] = e + EPV <= n ? __ldg(reinterpret_cast<const uint4*>(src + e)) : make_uint4(0, 0, 0, 0);
+        }
+    }
+}
+
+template <typename T, int NV>
+__device__ __forceinline__ void chunk_park(const T* __restrict__ src, int n, int lane, const ChunkRegs<T, NV>& r,
+                                           bool vec, float* dst) {
+    constexpr int EPV = 16 / (int)sizeof(T);
+    int done = 0;
+    if (vec) {
+#pragma unroll
+        for (int u = 0; u < NV; ++u) {
+            const int e = (u * 32 + lane) * EPV;
+            if (e + EPV <= n) {
+                if (sizeof(T) == 4) {
+                    *reinterpret_cast<uint4*>(dst + e) = r.v[u];
+                } else {
+                    const uint32_t w[4] = {r.v[u].x, r.v[u].y, r.v[u].z, r.v[u].w};
+                    *reinterpret_cast<float4*>(dst + e) =
+                        make_float4(__uint_as_float(w[0] << 16), __uint_as_float(w[0] & 0xFFFF0000u),
+                                    __uint_as_float(w[1] << 16), __uint_as_float(w[1] & 0xFFFF0000u));
+                    *reinterpret_cast<float4*>(dst + e + 4) =
+                        make_float4(__uint_as_float(w[2] << 16), __uint_as_float(w[2] & 0xFFFF0000u),
+                                    __uint_as_float(w[3] << 16), __uint_as_float(w[3] & 0xFFFF0000u));
+                }
+            }
+        }
+        done = (n / EPV) * EPV;
+    }
+    for (int e = done + lane; e < n; e += 32) dst[e] = to_f32(src[e]);      // unaligned chunk, or the tail
+}
+
+template <typename T, int MAXM, bool GRAD>
+__global__ void __launch_bounds__(NARROW_THREADS)
+narrow_kernel(NarrowParams p) {
+    using Cfg = NarrowCfg<MAXM>;
+    constexpr int CH = Cfg::CH;
+    constexpr int EPV = 16 / (int)sizeof(T);
+    constexpr int NVA = (CH * 32 + 32 * EPV - 1) / (32 * EPV), NVZ = (CH * MAXM + 32 * EPV - 1) / (32 * EPV);
+    extern __shared__ __align__(16) float narrow_smem[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    float* As = narrow_smem + warp * (Cfg::A_FLOATS + Cfg::Z_FLOATS);
+    float* Zs = As + Cfg::A_FLOATS;
+    float (*Gs)[33] = reinterpret_cast<float (*)[33]>(narrow_smem + NARROW_WARPS * (Cfg::A_FLOATS + Cfg::Z_FLOATS));
+    __shared__ float red[32];
+
+    const T* __restrict__ A = static_cast<const T*>(p.A);
+    const T* __restrict__ Z = static_cast<const T*>(p.Z);
+    long r0, r1;
+    if (GRAD) { r0 = (long)blockIdx.x * p.rows_per_cta; r1 = min(r0 + p.rows_per_cta, p.rows_total); }
+    else { r0 = (long)blockIdx.x * p.T; r1 = r0 + p.T; }
+
+    for (int i = threadIdx.x; i < MAXM * 33; i += NARROW_THREADS) (&Gs[0][0])[i] = 0.f;
+
+    float G[MAXM];
+#pragma unroll
+    for (int m = 0; m < MAXM; ++m) G[m] = 0.f;
+
+    const bool a_lane = lane < p.d_in, one_lane = p.has_bias && lane == p.d_in;
+    const bool zvec = (p.d_out & 3) == 0;                          // zb rows start on 16-byte boundaries in smem
+    ChunkRegs<T, NVA> ra;
+    ChunkRegs<T, NVZ> rz;
+    bool va = false, vz = false;
+    const long stride = (long)NARROW_WARPS * CH;
+    long base = r0 + (long)warp * CH;
+    auto rows_of = [&](long b) { return (int)min((long)CH, r1 - b); };
+    if (base < r1) {
+        const int nr = rows_of(base);
+        chunk_issue<T, NVA>(A + (size_t)base * p.lda, nr * p.d_in, lane, ra, va);
+        chunk_issue<T, NVZ>(Z + (size_t)base * p.ldz, nr * p.d_out, lane, rz, vz);
+    }
+    for (; base < r1; base += stride) {
+        const int nr = rows_of(base);
+        chunk_park<T, NVA>(A + (size_t)base * p.lda, nr * p.d_in, lane, ra, va, As);
+        chunk_park<T, NVZ>(Z + (size_t)base * p.ldz, nr * p.d_out, lane, rz, vz, Zs);
+        __syncwarp();
+        if (base + stride < r1) {                                  // next chunk's loads fly during this chunk's FMAs
+            const int nn = rows_of(base + stride);
+            chunk_issue<T, NVA>(A + (size_t)(base + stride) * p.lda, nn * p.d_in, lane, ra, va);
+            chunk_issue<T, NVZ>(Z + (size_t)(base + stride) * p.ldz, nn * p.d_out, lane, rz, vz);
+        }
+        int e = GRAD ? (int)(base / p.T) : 0, rem = GRAD ? (int)(base - (long)e * p.T) : 0;
+        float c = 1.f;
+        if (GRAD) { if (p.clip) c = __ldg(p.clip + e); }
+#pragma unroll 4
+        for (int r = 0; r < nr; ++r) {
+            float ar = a_lane ? As[r * p.d_in + lane] : (one_lane ? 1.f : 0.f);
+            if (GRAD) {
+                ar *= c;
+                if (++rem == p.T) { rem = 0; ++e; if (p.clip && base + r + 1 < r1) c = __ldg(p.clip + e); }
+            }
+            const float* zr = Zs + r * p.d_out;
+            if (zvec) {
+#pragma unroll
+                for (int m4 = 0; m4 < MAXM / 4; ++m4) {
+                    const float4 z4 = *reinterpret_cast<const float4*>(zr + 4 * m4);          // broadcast
+                    G[4 * m4 + 0] = fmaf(z4.x, ar, G[4 * m4 + 0]);
+                    G[4 * m4 + 1] = fmaf(z4.y, ar, G[4 * m4 + 1]);
+                    G[4 * m4 + 2] = fmaf(z4.z, ar, G[4 * m4 + 2]);
+                    G[4 * m4 + 3] = fmaf(z4.w, ar, G[4 * m4 + 3]);
+                }
+            } else {
+#pragma unroll
+                for (int m = 0; m < MAXM; ++m) G[m] = fmaf(zr[m], ar, G[m]);
+            }
+        }
+        __syncwarp();
+    }
+
+    __syncthreads();                                               // Gs zeroed by everyone
+#pragma unroll
+    for (int m = 0; m < MAXM; ++m)
+        if (m < p.d_out) atomicAdd(&Gs[m][lane], G[m]);            // entries m >= d_out hold garbage: never used
+    __syncthreads();
+
+    if (GRAD) {
+        for (int i = threadIdx.x; i < p.d_out * 32; i += NARROW_THREADS) {
+            const int m = i >> 5, n = i & 31;
+            if (n < p.d_in) atomicAdd(p.gW + (size_t)m * p.ldg + n, Gs[m][n]);
+            else if (n == p.d_in && p.has_bias && p.gb) atomicAdd(p.gb + m, Gs[m][n]);
+        }
+    } else {
+        float s = 0.f;
+        for (int i = threadIdx.x; i < p.d_out * 32; i += NARROW_THREADS) {
+            const float v = Gs[i >> 5][i & 31];                    // unused columns hold zeros
+            s = fmaf(v, v, s);
+        }
+        s = block_sum(s, red);
+        if (threadIdx.x == 0) p.sq[blockIdx.x] = s;
+    }
+}
+
+}  // namespace dpclip

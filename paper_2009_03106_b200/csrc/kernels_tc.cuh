@@ -669,6 +669,7 @@ struct ReduceParams {
     int n_tiles, tiles_n, ksplit, BM;
     int d_out, d_in;
     float* gW; long ldg; float* gb; int vec_ok;
+    int lanes;                                                  // lanes cooperating on one output float4
     float noise_scale; uint32_t k0, k1, sw0, sw1, sb0, sb1;     // Philox key, weight / bias stream words
 };
 
@@ -686,24 +687,39 @@ reduce_partials_kernel(const ReduceParams p) {
     const long total = (long)p.d_out * n4;
     const size_t tile_elems = (size_t)p.BM * zta::BN;
     const size_t ks_stride = (size_t)p.n_tiles * tile_elems;
-    for (long idx = (long)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (long)gridDim.x * blockDim.x) {
-        const int m = (int)(idx / n4), n = (int)(idx % n4) << 2;
+    // Each output float4 is summed by a group of `lanes` consecutive lanes (a power of two <= 32): small
+    // outputs with many row slices get wide groups, so the kernel always has enough loads in flight.  The
+    // order of the additions depends only on (ksplit, lanes), so the result is reproducible.
+    const int lanes = p.lanes, sub = threadIdx.x & (lanes - 1);
+    const long gid0 = ((long)blockIdx.x * blockDim.x + threadIdx.x) / lanes;
+    const long gstride = ((long)gridDim.x * blockDim.x) / lanes;
+    for (long idx0 = 0; idx0 < total; idx0 += gstride) {          // uniform trip count: shuffles stay converged
+        const long idx = idx0 + gid0;
+        const bool live = idx < total;
+        const int m = live ? (int)(idx / n4) : 0, n = live ? (int)(idx % n4) << 2 : 0;
         const int tm = m / p.BM, tn = n / zta::BN;
         const float* src = p.part + (size_t)(tm * p.tiles_n + tn) * tile_elems + (size_t)(m - tm * p.BM) * zta::BN +
                            (n - tn * zta::BN);
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        int ks = 0;
-        for (; ks + 8 <= p.ksplit; ks += 8) {            // eight independent loads in flight, fixed add order
-            float4 v[8];
+        if (live) {
+            int ks = sub;
+            for (; ks + 3 * lanes < p.ksplit; ks += 4 * lanes) {     // four independent loads in flight
+                float4 v[4];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) v[u] = __ldcs(reinterpret_cast<const float4*>(src + (ks + u) * ks_stride));
+                for (int u = 0; u < 4; ++u) v[u] = __ldcs(reinterpret_cast<const float4*>(src + (ks + u * lanes) * ks_stride));
 #pragma unroll
-            for (int u = 0; u < 8; ++u) { acc.x += v[u].x; acc.y += v[u].y; acc.z += v[u].z; acc.w += v[u].w; }
+                for (int u = 0; u < 4; ++u) { acc.x += v[u].x; acc.y += v[u].y; acc.z += v[u].z; acc.w += v[u].w; }
+            }
+            for (; ks < p.ksplit; ks += lanes) {
+                const float4 v = __ldcs(reinterpret_cast<const float4*>(src + ks * ks_stride));
+                acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+            }
         }
-        for (; ks < p.ksplit; ++ks) {
-            const float4 v = __ldcs(reinterpret_cast<const float4*>(src + ks * ks_stride));
-            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        for (int o = lanes >> 1; o > 0; o >>= 1) {
+            acc.x += __shfl_xor_sync(0xFFFFFFFFu, acc.x, o); acc.y += __shfl_xor_sync(0xFFFFFFFFu, acc.y, o);
+            acc.z += __shfl_xor_sync(0xFFFFFFFFu, acc.z, o); acc.w += __shfl_xor_sync(0xFFFFFFFFu, acc.w, o);
         }
+        if (!live || sub != 0) continue;
         if (p.noise_scale > 0.f) {
             const size_t q = ((size_t)m * p.d_in + n) >> 2;
             PhiloxBlock b = philox_block((uint32_t)q, (uint32_t)(q >> 32), p.sw0, p.sw1, p.k0, p.k1);

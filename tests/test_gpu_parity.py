@@ -196,6 +196,25 @@ def test_clipped_grad(dp, dtype, B, T, d_in, d_out):
     assert dp.dpclip_read_status(ws) == 0
 
 
+@pytest.mark.parametrize("dtype,B,T,d_in,d_out", [("bf16", 8, 256, 512, 256), ("f32", 6, 17, 27, 33),
+                                                  ("bf16", 128, 1, 512, 256)])
+def test_clipped_grad_noise_equals_separate_calls(dp, dtype, B, T, d_in, d_out):
+    A, Z = workloads.random_layer(9, B, T, d_in, d_out, dtype, scale_z=0.05)
+    clip = torch.from_numpy(np.random.default_rng(1).uniform(0.2, 1.0, B).astype(np.float32)).cuda()
+    dA, dZ = to_device(A, dtype), to_device(Z, dtype)
+    ws = _ws(dp)
+    W1 = torch.empty((d_out, d_in), device="cuda"); b1 = torch.empty(d_out, device="cuda")
+    dp.dpclip_clipped_grad(dA, dZ, clip, W1, b1, ws)
+    dp.dpclip_add_noise(W1.view(-1), 0.9, 1.3, 77, 4)
+    dp.dpclip_add_noise(b1, 0.9, 1.3, 77, 5)
+    W2 = torch.empty((d_out, d_in), device="cuda"); b2 = torch.empty(d_out, device="cuda")
+    dp.dpclip_clipped_grad_noise(dA, dZ, clip, W2, b2, 0.9, 1.3, 77, 4, 5, ws)
+    if dtype == "bf16":       # deterministic tensor-core path: identical bits
+        assert torch.equal(W1, W2) and torch.equal(b1, b2)
+    else:                     # fp32-ALU path combines row slices with atomics
+        assert rel_fro(W2.cpu().numpy(), W1.cpu().numpy()) <= 1e-6
+
+
 # ---------------------------------------------------------------------------
 # (e) noise
 # ---------------------------------------------------------------------------
