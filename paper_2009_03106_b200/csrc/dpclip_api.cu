@@ -310,11 +310,11 @@ int launch_zta_tc_mt(const CUtensorMap& ma, const CUtensorMap& mz, tc::zta::Para
         if (noise_done) *noise_done = true;
     }
     const long n_vec = (long)d_out * ((d_in + 3) / 4);
-    // widen the per-output lane groups until the grid has about two CTAs per SM (or a full warp per output)
+    // split the row slices over up to 8 thread rows per CTA until the grid has about two CTAs per SM
     int lanes = 1;
-    while (lanes < 32 && lanes * 2 <= ksplit && n_vec * lanes < 2L * kNumSMs * 256) lanes *= 2;
+    while (lanes < 8 && lanes * 2 <= ksplit && n_vec * lanes < 2L * kNumSMs * 256) lanes *= 2;
     r.lanes = lanes;
-    long blocks = (n_vec * lanes + 255) / 256;
+    long blocks = (n_vec + (256 / lanes) - 1) / (256 / lanes);
     if (blocks > 8L * kNumSMs) blocks = 8L * kNumSMs;
     tc::reduce_partials_kernel<<<(unsigned)blocks, 256, 0, st>>>(r);
     return launch_status();

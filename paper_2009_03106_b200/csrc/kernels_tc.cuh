@@ -669,7 +669,7 @@ struct ReduceParams {
     int n_tiles, tiles_n, ksplit, BM;
     int d_out, d_in;
     float* gW; long ldg; float* gb; int vec_ok;
-    int lanes;                                                  // lanes cooperating on one output float4
+    int lanes;                                                  // thread rows of a CTA sharing the row slices (1..8)
     float noise_scale; uint32_t k0, k1, sw0, sw1, sb0, sb1;     // Philox key, weight / bias stream words
 };
 
@@ -683,18 +683,19 @@ namespace tc {
 
 __global__ void __launch_bounds__(256)
 reduce_partials_kernel(const ReduceParams p) {
+    __shared__ float4 part_s[256];
     const int n4 = (p.d_in + 3) >> 2;
     const long total = (long)p.d_out * n4;
     const size_t tile_elems = (size_t)p.BM * zta::BN;
     const size_t ks_stride = (size_t)p.n_tiles * tile_elems;
-    // Each output float4 is summed by a group of `lanes` consecutive lanes (a power of two <= 32): small
-    // outputs with many row slices get wide groups, so the kernel always has enough loads in flight.  The
-    // order of the additions depends only on (ksplit, lanes), so the result is reproducible.
-    const int lanes = p.lanes, sub = threadIdx.x & (lanes - 1);
-    const long gid0 = ((long)blockIdx.x * blockDim.x + threadIdx.x) / lanes;
-    const long gstride = ((long)gridDim.x * blockDim.x) / lanes;
-    for (long idx0 = 0; idx0 < total; idx0 += gstride) {          // uniform trip count: shuffles stay converged
-        const long idx = idx0 + gid0;
+    // The 256 threads of a CTA form `groups` rows of 256 / groups threads: a row covers consecutive
+    // output float4s (coalesced loads) and takes every groups-th row slice; the rows' sums are then
+    // combined through shared memory in a fixed order.  Small outputs with many slices get many groups,
+    // so the kernel always has enough loads in flight, and the result is reproducible.
+    const int groups = p.lanes, width = 256 / groups;
+    const int gy = threadIdx.x / width, gx = threadIdx.x - gy * width;
+    for (long idx0 = (long)blockIdx.x * width; idx0 < total; idx0 += (long)gridDim.x * width) {
+        const long idx = idx0 + gx;
         const bool live = idx < total;
         const int m = live ? (int)(idx / n4) : 0, n = live ? (int)(idx % n4) << 2 : 0;
         const int tm = m / p.BM, tn = n / zta::BN;
@@ -702,24 +703,30 @@ reduce_partials_kernel(const ReduceParams p) {
                            (n - tn * zta::BN);
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         if (live) {
-            int ks = sub;
-            for (; ks + 3 * lanes < p.ksplit; ks += 4 * lanes) {     // four independent loads in flight
+            int ks = gy;
+            for (; ks + 3 * groups < p.ksplit; ks += 4 * groups) {  // four independent loads in flight
                 float4 v[4];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) v[u] = __ldcs(reinterpret_cast<const float4*>(src + (ks + u * lanes) * ks_stride));
+                for (int u = 0; u < 4; ++u) v[u] = __ldcs(reinterpret_cast<const float4*>(src + (ks + u * groups) * ks_stride));
 #pragma unroll
                 for (int u = 0; u < 4; ++u) { acc.x += v[u].x; acc.y += v[u].y; acc.z += v[u].z; acc.w += v[u].w; }
             }
-            for (; ks < p.ksplit; ks += lanes) {
+            for (; ks < p.ksplit; ks += groups) {
                 const float4 v = __ldcs(reinterpret_cast<const float4*>(src + ks * ks_stride));
                 acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
             }
         }
-        for (int o = lanes >> 1; o > 0; o >>= 1) {
-            acc.x += __shfl_xor_sync(0xFFFFFFFFu, acc.x, o); acc.y += __shfl_xor_sync(0xFFFFFFFFu, acc.y, o);
-            acc.z += __shfl_xor_sync(0xFFFFFFFFu, acc.z, o); acc.w += __shfl_xor_sync(0xFFFFFFFFu, acc.w, o);
+        if (groups > 1) {
+            __syncthreads();
+            part_s[threadIdx.x] = acc;
+            __syncthreads();
+            if (gy == 0)
+                for (int g = 1; g < groups; ++g) {
+                    const float4 v = part_s[g * width + gx];
+                    acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+                }
         }
-        if (!live || sub != 0) continue;
+        if (!live || gy != 0) continue;
         if (p.noise_scale > 0.f) {
             const size_t q = ((size_t)m * p.d_in + n) >> 2;
             PhiloxBlock b = philox_block((uint32_t)q, (uint32_t)(q >> 32), p.sw0, p.sw1, p.k0, p.k1);
@@ -739,12 +746,18 @@ reduce_partials_kernel(const ReduceParams p) {
         }
     }
     if (p.gb) {
-        for (int m = blockIdx.x * blockDim.x + threadIdx.x; m < p.d_out; m += gridDim.x * blockDim.x) {
+        // bias: one warp per output, lanes over the (row slice, n-tile) partial sums, fixed-order combine
+        const int lane = threadIdx.x & 31;
+        const int n_part = p.ksplit * p.tiles_n;
+        for (int m = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; m < p.d_out; m += (gridDim.x * blockDim.x) >> 5) {
             const int tm = m / p.BM;
             float acc = 0.f;
-            for (int ks = 0; ks < p.ksplit; ++ks)
-                for (int tn = 0; tn < p.tiles_n; ++tn)
-                    acc += p.bias_part[((size_t)ks * p.n_tiles + tm * p.tiles_n + tn) * p.BM + (m - tm * p.BM)];
+            for (int j = lane; j < n_part; j += 32) {
+                const int ks = j / p.tiles_n, tn = j - ks * p.tiles_n;
+                acc += p.bias_part[((size_t)ks * p.n_tiles + tm * p.tiles_n + tn) * p.BM + (m - tm * p.BM)];
+            }
+            acc = warp_sum(acc);
+            if (lane != 0) continue;
             if (p.noise_scale > 0.f) {
                 PhiloxBlock b = philox_block((uint32_t)(m >> 2), 0u, p.sb0, p.sb1, p.k0, p.k1);
                 float z[4];
