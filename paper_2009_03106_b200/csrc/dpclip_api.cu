@@ -123,8 +123,8 @@ int launch_simt_grad(const void* A, long lda, const void* Z, long ldz, int B, in
         q.A = A; q.lda = lda; q.Z = Z; q.ldz = ldz; q.T = T; q.d_in = d_in; q.d_out = d_out;
         q.has_bias = gb ? 1 : 0; q.clip = clip; q.gW = gW; q.ldg = ldg; q.gb = gb;
         q.rows_total = (long)B * T;
-        int grid = 2 * kNumSMs;
-        const long min_rows = 8 * 32;                              // at least one chunk per warp
+        int grid = kNumSMs;                                        // one wave: the kernel holds a whole SM
+        const long min_rows = NARROW_WARPS * 32;                   // at least one chunk per warp
         if ((long)grid * min_rows > q.rows_total) grid = (int)((q.rows_total + min_rows - 1) / min_rows);
         q.rows_per_cta = (q.rows_total + grid - 1) / grid;
         grid = (int)((q.rows_total + q.rows_per_cta - 1) / q.rows_per_cta);

@@ -10,7 +10,7 @@
 // warp fetches it with 128-bit loads (all issued before the previous chunk is
 // computed, i.e. a whole chunk per warp in flight), parks it in shared memory,
 // and then every lane reads its own a[row][n] and the zb row as broadcast
-// 128-bit loads.  The eight warps of a CTA take interleaved chunks; their
+// 128-bit loads.  The sixteen warps of a CTA take interleaved chunks; their
 // partial tiles are combined in shared memory at the end.
 //
 //   NORM: one CTA per example; the tile is squared and summed -> sq[i].
@@ -22,7 +22,7 @@
 
 namespace dpclip {
 
-constexpr int NARROW_THREADS = 256, NARROW_WARPS = NARROW_THREADS / 32;
+constexpr int NARROW_THREADS = 512, NARROW_WARPS = NARROW_THREADS / 32;   // 16 warps: one CTA per SM, latency hidden by warps
 
 struct NarrowParams {
     const void* A; long lda;
