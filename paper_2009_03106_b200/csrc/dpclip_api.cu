@@ -6,6 +6,7 @@
 #include "kernels_simt.cuh"
 #include "kernels_stream.cuh"
 #include "kernels_tc.cuh"
+#include "kernels_tf32.cuh"
 #include "kernels_fused_t1.cuh"
 #include "kernels_narrow.cuh"
 
@@ -247,6 +248,33 @@ struct NoiseSpec { float scale; unsigned long long seed, sid_w, sid_b; };
 // wave of 256 x 256 tiles or two waves of 128 x 256 tiles, plus the partial bias sums.
 constexpr size_t kTcScratchBytes = (size_t)kNumSMs * 256 * 256 * 4 + (size_t)2 * kNumSMs * 256 * 4;
 
+// second stage of a split-row clipped sum: fixed-order sum of the partial tiles (+ optional noise)
+int launch_reduce_partials(const tc::zta::Params& p, int tiles, int ksplit, int BM, int BN, int d_in, int d_out,
+                           float* gW, long ldg, float* gb, const NoiseSpec* noise, bool* noise_done,
+                           cudaStream_t st) {
+    tc::ReduceParams r;
+    memset(&r, 0, sizeof(r));
+    r.part = p.part; r.bias_part = p.bias_part;
+    r.n_tiles = tiles; r.tiles_n = p.tiles_n; r.ksplit = ksplit; r.BM = BM; r.BN = BN;
+    r.d_out = d_out; r.d_in = d_in; r.gW = gW; r.ldg = ldg; r.gb = gb; r.vec_ok = p.vec_ok;
+    if (noise && noise->scale > 0.f && ldg == d_in && d_in % 4 == 0) {
+        r.noise_scale = noise->scale;
+        r.k0 = (uint32_t)noise->seed; r.k1 = (uint32_t)(noise->seed >> 32);
+        r.sw0 = (uint32_t)noise->sid_w; r.sw1 = (uint32_t)(noise->sid_w >> 32);
+        r.sb0 = (uint32_t)noise->sid_b; r.sb1 = (uint32_t)(noise->sid_b >> 32);
+        if (noise_done) *noise_done = true;
+    }
+    const long n_vec = (long)d_out * ((d_in + 3) / 4);
+    // split the row slices over up to 8 thread rows per CTA until the grid has about two CTAs per SM
+    int lanes = 1;
+    while (lanes < 8 && lanes * 2 <= ksplit && n_vec * lanes < 2L * kNumSMs * 256) lanes *= 2;
+    r.lanes = lanes;
+    long blocks = (n_vec + (256 / lanes) - 1) / (256 / lanes);
+    if (blocks > 8L * kNumSMs) blocks = 8L * kNumSMs;
+    tc::reduce_partials_kernel<<<(unsigned)blocks, 256, 0, st>>>(r);
+    return launch_status();
+}
+
 // Tile shape: 256 x 256 (MT = 2) cuts the L2->SM traffic per flop by a third but has a single
 // accumulator buffer; it pays once d_out spans at least two 128-row sub-tiles.
 template <int MT>
@@ -297,27 +325,7 @@ int launch_zta_tc_mt(const CUtensorMap& ma, const CUtensorMap& mz, tc::zta::Para
     int rc = launch_status();
     if (rc || norm_mode || ksplit == 1) return rc;
 
-    tc::ReduceParams r;
-    memset(&r, 0, sizeof(r));
-    r.part = p.part; r.bias_part = p.bias_part;
-    r.n_tiles = tiles; r.tiles_n = p.tiles_n; r.ksplit = ksplit; r.BM = BM;
-    r.d_out = d_out; r.d_in = d_in; r.gW = gW; r.ldg = ldg; r.gb = gb; r.vec_ok = p.vec_ok;
-    if (noise && noise->scale > 0.f && ldg == d_in && d_in % 4 == 0) {
-        r.noise_scale = noise->scale;
-        r.k0 = (uint32_t)noise->seed; r.k1 = (uint32_t)(noise->seed >> 32);
-        r.sw0 = (uint32_t)noise->sid_w; r.sw1 = (uint32_t)(noise->sid_w >> 32);
-        r.sb0 = (uint32_t)noise->sid_b; r.sb1 = (uint32_t)(noise->sid_b >> 32);
-        if (noise_done) *noise_done = true;
-    }
-    const long n_vec = (long)d_out * ((d_in + 3) / 4);
-    // split the row slices over up to 8 thread rows per CTA until the grid has about two CTAs per SM
-    int lanes = 1;
-    while (lanes < 8 && lanes * 2 <= ksplit && n_vec * lanes < 2L * kNumSMs * 256) lanes *= 2;
-    r.lanes = lanes;
-    long blocks = (n_vec + (256 / lanes) - 1) / (256 / lanes);
-    if (blocks > 8L * kNumSMs) blocks = 8L * kNumSMs;
-    tc::reduce_partials_kernel<<<(unsigned)blocks, 256, 0, st>>>(r);
-    return launch_status();
+    return launch_reduce_partials(p, tiles, ksplit, BM, z::BN, d_in, d_out, gW, ldg, gb, noise, noise_done, st);
 }
 
 int launch_zta_tc(const void* A, long lda, const void* Z, long ldz, int B, int T, int d_in, int d_out,
@@ -353,6 +361,82 @@ int launch_zta_tc(const void* A, long lda, const void* Z, long ldz, int B, int T
                                noise, noise_done, st, fit_to_workspace);
 }
 
+// fp32 layers on the tensor cores (error-compensated tf32): TMA needs 16-byte aligned bases and rows
+inline bool tf32_eligible(const void* A, long lda, const void* Z, long ldz, int B, int T, int d_in, int d_out,
+                          dpclip_dtype dtype) {
+    if (dtype != DPCLIP_F32) return false;
+    const char* env = getenv("DPCLIP_FORCE_SIMT");
+    if (env && env[0] == '1') return false;
+    if (!(aligned_to(A, 16) && aligned_to(Z, 16) && lda % 4 == 0 && ldz % 4 == 0)) return false;
+    // worth it once there is real contraction work; tiny layers stay on the fp32-ALU kernels
+    return (double)B * T * d_in * d_out >= 32.0 * 1024 * 1024;
+}
+
+bool make_map_f32(CUtensorMap* map, const void* base, long rows, long cols, long ld, int box_cols, int box_rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * 4};
+    cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int launch_zta_tf32(const void* A, long lda, const void* Z, long ldz, int B, int T, int d_in, int d_out,
+                    bool norm_mode, int has_bias, const float* clip, float* gW, long ldg, float* gb, float* sq,
+                    void* workspace, size_t workspace_bytes, const NoiseSpec* noise, bool* noise_done,
+                    cudaStream_t st) {
+    namespace t = tc::t32;
+    const long R = (long)B * T;
+    CUtensorMap ma, mz;
+    if (!make_map_f32(&ma, A, R, d_in, lda, 32, t::BK) || !make_map_f32(&mz, Z, R, d_out, ldz, 32, t::BK))
+        return DPCLIP_ERR_CUDA;
+    tc::zta::Params p;
+    memset(&p, 0, sizeof(p));
+    p.R = (int)R; p.T = T; p.d_in = d_in; p.d_out = d_out;
+    p.norm_mode = norm_mode ? 1 : 0;
+    p.status = static_cast<int*>(workspace);
+    p.tiles_m = ceil_div(d_out, t::BM); p.tiles_n = ceil_div(d_in, t::BN);
+    const int tiles = p.tiles_m * p.tiles_n;
+    int ksplit = 1;
+    if (norm_mode) {
+        p.do_bias = has_bias ? 1 : 0;
+        p.sq = sq;
+        p.n_items = B * tiles;
+        if (cudaMemsetAsync(sq, 0, sizeof(float) * (size_t)B, st) != cudaSuccess) return DPCLIP_ERR_CUDA;
+    } else {
+        p.clip = clip; p.gW = gW; p.ldg = ldg; p.gb = gb;
+        p.do_bias = gb ? 1 : 0;
+        p.vec_ok = aligned_to(gW, 16) && ldg % 4 == 0;
+        const int nkb = ceil_div(R, t::BK);
+        // two accumulator buffers: two items per SM when they stay long enough, else one wave
+        const int per_sm = (tiles <= kNumSMs && nkb / ((2 * kNumSMs) / tiles) >= 16) ? 2 : 1;
+        ksplit = (per_sm * kNumSMs) / tiles;
+        if (ksplit > nkb) ksplit = nkb;
+        if (ksplit < 1) ksplit = 1;
+        p.kb_per_split = ceil_div(nkb, ksplit);
+        ksplit = ceil_div(nkb, p.kb_per_split);
+        p.n_items = tiles * ksplit;
+        if (ksplit > 1) {
+            const size_t part_bytes = (size_t)p.n_items * t::BM * t::BN * 4;
+            const size_t bias_bytes = gb ? (size_t)p.n_items * t::BM * 4 : 0;
+            if (workspace_bytes < kHeaderBytes + part_bytes + bias_bytes) return DPCLIP_ERR_WORKSPACE;
+            p.part = reinterpret_cast<float*>(static_cast<char*>(workspace) + kHeaderBytes);
+            p.bias_part = gb ? p.part + part_bytes / 4 : nullptr;
+        } else if (gb && cudaMemsetAsync(gb, 0, sizeof(float) * (size_t)d_out, st) != cudaSuccess) {
+            return DPCLIP_ERR_CUDA;
+        }
+    }
+    if (!enable_smem(tc::zta_tf32_kernel, t::SMEM_BYTES)) return DPCLIP_ERR_CUDA;
+    const int grid = p.n_items < kNumSMs ? p.n_items : kNumSMs;
+    tc::zta_tf32_kernel<<<grid, t::THREADS, t::SMEM_BYTES, st>>>(ma, mz, p);
+    int rc = launch_status();
+    if (rc || norm_mode || ksplit == 1) return rc;
+    return launch_reduce_partials(p, tiles, ksplit, t::BM, t::BN, d_in, d_out, gW, ldg, gb, noise, noise_done, st);
+}
+
 // clipped sum of one layer, optionally with the noise folded into the last pass over the output
 int clipped_grad_impl(const void* A, long lda, const void* Zbar, long ldz, int B, int T, int d_in, int d_out,
                       dpclip_dtype dtype, const float* clip, float* gW, long ldg, float* gb, void* workspace,
@@ -360,6 +444,9 @@ int clipped_grad_impl(const void* A, long lda, const void* Zbar, long ldz, int B
     if (tc_eligible(A, lda, Zbar, ldz, dtype))
         return launch_zta_tc(A, lda, Zbar, ldz, B, T, d_in, d_out, false, 0, clip, gW, ldg, gb, nullptr, workspace,
                              workspace_bytes, noise, noise_done, st);
+    if (tf32_eligible(A, lda, Zbar, ldz, B, T, d_in, d_out, dtype) && !narrow_layer(T, d_in, d_out, gb != nullptr, lda, ldz))
+        return launch_zta_tf32(A, lda, Zbar, ldz, B, T, d_in, d_out, false, 0, clip, gW, ldg, gb, nullptr, workspace,
+                               workspace_bytes, noise, noise_done, st);
     return launch_simt_grad(A, lda, Zbar, ldz, B, T, d_in, d_out, dtype, clip, gW, ldg, gb, st);
 }
 
@@ -466,14 +553,24 @@ int dpclip_pick_method(int B, int T, int d_in, int d_out, long lda, long ldz, dp
             return gram <= mat ? DPCLIP_GRAM : DPCLIP_MATERIALIZE;
         }
     }
+    // fp32: materialised tiles on the tensor cores (error-compensated tf32) once the layer is large
+    // enough and its rows are 16-byte multiples; narrow and small layers stay on the fp32 ALUs
+    if (dtype == DPCLIP_F32 && lda % 4 == 0 && ldz % 4 == 0 && !narrow_layer(T, d_in, d_out, 1, lda, ldz) &&
+        (double)B * T * d_in * d_out >= 32.0 * 1024 * 1024) {
+        const char* env = getenv("DPCLIP_FORCE_SIMT");
+        if (!(env && env[0] == '1')) return DPCLIP_MATERIALIZE;
+    }
     return DPCLIP_SIMT;
 }
 
 size_t dpclip_workspace_bytes(int B, int T, int d_in, int d_out, dpclip_dtype dtype, dpclip_method method) {
-    (void)B; (void)T; (void)d_in; (void)d_out; (void)method;
-    // bf16 layers may take the tensor-core clipped sum, which splits the rows over CTAs and keeps one
-    // partial tile per CTA in the workspace; the bound does not depend on the layer's shape
-    return dtype == DPCLIP_BF16 ? kHeaderBytes + kTcScratchBytes : (size_t)kHeaderBytes;
+    (void)method;
+    // Layers that may take a tensor-core clipped sum (all bf16 layers; fp32 layers above the size where
+    // the tf32 path is used) split their rows over CTAs and keep one partial tile per CTA in the
+    // workspace; the bound does not depend on the layer's shape.
+    if (dtype == DPCLIP_BF16) return kHeaderBytes + kTcScratchBytes;
+    if ((double)B * T * d_in * d_out >= 32.0 * 1024 * 1024) return kHeaderBytes + kTcScratchBytes;
+    return (size_t)kHeaderBytes;
 }
 
 int dpclip_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
@@ -499,7 +596,10 @@ int dpclip_layer_sqnorms(const void* A, long lda, const void* Zbar, long ldz, in
     if (!aligned_to(sq_layer, 4)) return DPCLIP_ERR_MISALIGNED;
     if (method == DPCLIP_AUTO) {
         method = (dpclip_method)dpclip_pick_method(B, T, d_in, d_out, lda, ldz, dtype);
-        if ((method == DPCLIP_GRAM || method == DPCLIP_MATERIALIZE) && !tc_eligible(A, lda, Zbar, ldz, dtype))
+        if (dtype == DPCLIP_BF16 && (method == DPCLIP_GRAM || method == DPCLIP_MATERIALIZE) &&
+            !tc_eligible(A, lda, Zbar, ldz, dtype))
+            method = DPCLIP_SIMT;
+        if (dtype == DPCLIP_F32 && method == DPCLIP_MATERIALIZE && !tf32_eligible(A, lda, Zbar, ldz, B, T, d_in, d_out, dtype))
             method = DPCLIP_SIMT;
     }
     if (!workspace || workspace_bytes < dpclip_workspace_bytes(B, T, d_in, d_out, dtype, method))
@@ -513,7 +613,13 @@ int dpclip_layer_sqnorms(const void* A, long lda, const void* Zbar, long ldz, in
             return launch_simt_norms(A, lda, Zbar, ldz, B, T, d_in, d_out, dtype, has_bias, sq_layer, st);
         case DPCLIP_GRAM:
         case DPCLIP_MATERIALIZE:
-            if (dtype != DPCLIP_BF16 || !aligned_to(A, 16) || !aligned_to(Zbar, 16) || lda % 8 || ldz % 8)
+            if (dtype == DPCLIP_F32) {                    // fp32: materialised tiles via error-compensated tf32
+                if (method != DPCLIP_MATERIALIZE || !aligned_to(A, 16) || !aligned_to(Zbar, 16) || lda % 4 || ldz % 4)
+                    return DPCLIP_ERR_UNSUPPORTED;
+                return launch_zta_tf32(A, lda, Zbar, ldz, B, T, d_in, d_out, true, has_bias, nullptr, nullptr, 0,
+                                       nullptr, sq_layer, workspace, workspace_bytes, nullptr, nullptr, st);
+            }
+            if (!aligned_to(A, 16) || !aligned_to(Zbar, 16) || lda % 8 || ldz % 8)
                 return DPCLIP_ERR_UNSUPPORTED;
             if (method == DPCLIP_GRAM)
                 return launch_gram_norms(A, lda, Zbar, ldz, B, T, d_in, d_out, has_bias, sq_layer,

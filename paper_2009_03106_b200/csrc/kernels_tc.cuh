@@ -666,7 +666,7 @@ zta_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
 // ---------------------------------------------------------------------------
 struct ReduceParams {
     const float* part; const float* bias_part;
-    int n_tiles, tiles_n, ksplit, BM;
+    int n_tiles, tiles_n, ksplit, BM, BN;                       // partial tiles are BM x BN fp32
     int d_out, d_in;
     float* gW; long ldg; float* gb; int vec_ok;
     int lanes;                                                  // thread rows of a CTA sharing the row slices (1..8)
@@ -686,7 +686,7 @@ reduce_partials_kernel(const ReduceParams p) {
     __shared__ float4 part_s[256];
     const int n4 = (p.d_in + 3) >> 2;
     const long total = (long)p.d_out * n4;
-    const size_t tile_elems = (size_t)p.BM * zta::BN;
+    const size_t tile_elems = (size_t)p.BM * p.BN;
     const size_t ks_stride = (size_t)p.n_tiles * tile_elems;
     // The 256 threads of a CTA form `groups` rows of 256 / groups threads: a row covers consecutive
     // output float4s (coalesced loads) and takes every groups-th row slice; the rows' sums are then
@@ -698,9 +698,9 @@ reduce_partials_kernel(const ReduceParams p) {
         const long idx = idx0 + gx;
         const bool live = idx < total;
         const int m = live ? (int)(idx / n4) : 0, n = live ? (int)(idx % n4) << 2 : 0;
-        const int tm = m / p.BM, tn = n / zta::BN;
-        const float* src = p.part + (size_t)(tm * p.tiles_n + tn) * tile_elems + (size_t)(m - tm * p.BM) * zta::BN +
-                           (n - tn * zta::BN);
+        const int tm = m / p.BM, tn = n / p.BN;
+        const float* src = p.part + (size_t)(tm * p.tiles_n + tn) * tile_elems + (size_t)(m - tm * p.BM) * p.BN +
+                           (n - tn * p.BN);
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         if (live) {
             int ks = gy;

@@ -133,6 +133,40 @@ def test_tensor_core_clipped_grad(dp, B, T, d_in, d_out):
 
 
 # ---------------------------------------------------------------------------
+# fp32 layers on the tensor cores (error-compensated tf32): still inside the fp32 tolerance
+# ---------------------------------------------------------------------------
+# (1, 16384, ...) is one long accumulation: 512 stages, drained to registers every few stages
+TF32_SHAPES = [(8, 256, 288, 64), (6, 200, 264, 136), (2, 2048, 128, 128), (16, 64, 576, 128), (40, 33, 100, 260),
+               (1, 16384, 128, 128)]
+
+
+@pytest.mark.parametrize("B,T,d_in,d_out", TF32_SHAPES)
+@pytest.mark.parametrize("has_bias", [True, False])
+def test_tf32_norms(dp, B, T, d_in, d_out, has_bias):
+    A, Z = workloads.random_layer(11, B, T, d_in, d_out, "f32", scale_z=0.05)
+    ref = oracle.layer_sqnorms(A, Z, has_bias)
+    got = _sqnorms(dp, A, Z, "f32", has_bias, method=dp.DPCLIP_MATERIALIZE)
+    assert max_rel(np.sqrt(got), np.sqrt(ref)) <= TOL["f32"]["norm"], max_rel(np.sqrt(got), np.sqrt(ref))
+    assert dp.dpclip_pick_method(B, T, d_in, d_out, d_in, d_out, dp.DPCLIP_F32) == dp.DPCLIP_MATERIALIZE
+
+
+@pytest.mark.parametrize("B,T,d_in,d_out", TF32_SHAPES + [(128, 1, 8192, 256)])
+def test_tf32_clipped_grad(dp, B, T, d_in, d_out):
+    A, Z = workloads.random_layer(12, B, T, d_in, d_out, "f32", scale_z=0.05)
+    clip = np.random.default_rng(B).uniform(0.05, 1.0, B).astype(np.float32)
+    clip[::2] = 1.0
+    refW, refb = oracle.clipped_grad(A, Z, clip)
+    dA, dZ = to_device(A, "f32"), to_device(Z, "f32")
+    gW = torch.full((d_out, d_in), 9.0, device="cuda"); gb = torch.full((d_out,), 9.0, device="cuda")
+    ws = _ws(dp)
+    dp.dpclip_clipped_grad(dA, dZ, torch.from_numpy(clip).cuda(), gW, gb, ws)
+    assert dp.dpclip_read_status(ws) == 0
+    e = rel_fro(gW.cpu().numpy(), refW)
+    assert e <= TOL["f32"]["grad"], e
+    assert rel_fro(gb.cpu().numpy(), refb) <= TOL["f32"]["grad"]
+
+
+# ---------------------------------------------------------------------------
 # (c) factors
 # ---------------------------------------------------------------------------
 @pytest.mark.parametrize("B,L", [(1, 1), (32, 2), (128, 3), (1024, 7), (1500, 2)])
