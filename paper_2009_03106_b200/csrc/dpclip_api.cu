@@ -6,6 +6,7 @@
 #include "kernels_simt.cuh"
 #include "kernels_stream.cuh"
 #include "kernels_tc.cuh"
+#include "kernels_fused_t1_tf32.cuh"
 #include "kernels_tf32.cuh"
 #include "kernels_fused_t1.cuh"
 #include "kernels_narrow.cuh"
@@ -453,9 +454,44 @@ int clipped_grad_impl(const void* A, long lda, const void* Zbar, long ldz, int B
 
 // Whole step in two launches for models made of T = 1 layers only (see kernels_fused_t1.cuh).
 // Returns 1 when the fused path does not apply (the caller then takes the per-layer path).
+// Second launch of the fused step on the tensor cores (fp32 models).  Every layer must either be addressable
+// by TMA (16-byte aligned base and row stride); the zb of a thin layer (at most 16 outputs) need not be.  Returns 1 when the model
+// does not qualify, so that the caller falls back to the fp32-ALU kernel.
+int launch_fused_t1_tf32(const FusedT1Params& base, void* workspace, size_t workspace_bytes, cudaStream_t st) {
+    namespace f = tc::f1;
+    { const char* env = getenv("DPCLIP_NO_T1_TF32"); if (env && env[0] == '1') return 1; }
+    if (!workspace || workspace_bytes < kHeaderBytes) return 1;
+    static_assert(sizeof(f::Params) <= 4096, "kernel parameter space");
+    f::Params q;
+    memset(&q, 0, sizeof(q));
+    q.base = base;
+    q.status = static_cast<int*>(workspace);
+    int items = 0, tc_layers = 0;
+    for (int l = 0; l < base.L; ++l) {
+        const FusedT1Layer& y = base.layer[l];
+        const bool a_ok = aligned_to(y.A, 16) && y.lda % 4 == 0;
+        const bool z_ok = aligned_to(y.Z, 16) && y.ldz % 4 == 0;
+        const bool thin = y.d_out <= f::THIN_MAX_OUT;
+        if (!a_ok || !(z_ok || thin)) return 1;
+        q.item_begin[l] = items;
+        q.thin[l] = thin ? 1 : 0;
+        if (!make_map_f32(&q.map_a[l], y.A, base.B, y.d_in, y.lda, 32, f::BK)) return DPCLIP_ERR_CUDA;
+        if (!thin && !make_map_f32(&q.map_z[l], y.Z, base.B, y.d_out, y.ldz, 32, f::BK)) return DPCLIP_ERR_CUDA;
+        q.tiles_n[l] = ceil_div(y.d_in, f::BN);
+        items += ceil_div(y.d_out, f::BM) * q.tiles_n[l];
+        if (!thin) ++tc_layers;
+    }
+    if (!tc_layers) return 1;
+    q.total_items = items;
+    if (!enable_smem(tc::t1_all_grads_tf32_kernel, f::SMEM_BYTES)) return DPCLIP_ERR_CUDA;
+    const int grid = items < kNumSMs ? items : kNumSMs;
+    tc::t1_all_grads_tf32_kernel<<<grid, f::THREADS, f::SMEM_BYTES, st>>>(q);
+    return launch_status();
+}
+
 int try_fused_t1_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, float C, float sigma,
                       unsigned long long seed, unsigned long long stream_id0, float* sq, float* clip,
-                      float* norms, cudaStream_t st) {
+                      float* norms, void* workspace, size_t workspace_bytes, cudaStream_t st) {
     if (L > FUSED_MAX_LAYERS || B > FUSED_MAX_B) return 1;
     const char* env = getenv("DPCLIP_NO_FUSED_T1");
     if (env && env[0] == '1') return 1;
@@ -495,6 +531,8 @@ int try_fused_t1_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dty
     if (dtype == DPCLIP_F32) {
         t1_all_norms_kernel<float><<<grid_n, 128, 0, st>>>(p);
         if (launch_status()) return DPCLIP_ERR_CUDA;
+        const int rc = launch_fused_t1_tf32(p, workspace, workspace_bytes, st);
+        if (rc <= 0) return rc;
         if (tile == 128) {
             if (!enable_smem(t1_all_grads_kernel<float, 128>, smem128)) return DPCLIP_ERR_CUDA;
             t1_all_grads_kernel<float, 128><<<grid_g, SIMT_THREADS, smem128, st>>>(p);
@@ -694,8 +732,8 @@ int dpclip_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, fl
     if (!layers || L <= 0 || B <= 0 || !sq_layers || !clip) return DPCLIP_ERR_INVALID_ARG;
     if (!(C > 0.f) || !(sigma >= 0.f)) return DPCLIP_ERR_INVALID_ARG;
     if (dtype != DPCLIP_F32 && dtype != DPCLIP_BF16) return DPCLIP_ERR_INVALID_ARG;
-    int rc = try_fused_t1_step(layers, L, B, dtype, C, sigma, seed, stream_id0, sq_layers, clip, norms,
-                               (cudaStream_t)stream);
+    int rc = try_fused_t1_step(layers, L, B, dtype, C, sigma, seed, stream_id0, sq_layers, clip, norms, workspace,
+                               workspace_bytes, (cudaStream_t)stream);
     if (rc <= 0) return rc;                  // done (0) or argument error (< 0); 1 = take the general path
     for (int l = 0; l < L; ++l) {
         const dpclip_layer& y = layers[l];

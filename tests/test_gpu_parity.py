@@ -392,6 +392,43 @@ def test_step_mlp_bf16_and_odd_widths(dp):
     _check_step(dp, odd, _calibrate(odd, layers, 3, odd.C), odd.C, odd.sigma, 3)
 
 
+def test_step_mlp_tensor_core_edges(dp):
+    """Fused T=1 step on the tensor cores (fp32, rows TMA can address): a batch that is not a multiple of
+    the 32-row stage and spans two accumulation windows, ragged tiles, a layer without bias, a thin head."""
+    w = workloads.Workload("mlp_tc_edges", 200, "f32",
+                           (workloads.LayerSpec("fc1", 1, 132, 260, True, "normal"),
+                            workloads.LayerSpec("fc2", 1, 260, 36, False, "relu"),
+                            workloads.LayerSpec("fc3", 1, 36, 16, True, "relu"),
+                            workloads.LayerSpec("fc4", 1, 16, 3, True, "relu")), 1.0, 0.9, 1.0 / 200)
+    layers = workloads.generate(w, 5)
+    _check_step(dp, w, _calibrate(w, layers, 5, w.C), w.C, w.sigma, 5)
+
+
+def test_step_mlp_fp32_alu_kernel(dp, monkeypatch):
+    """The fp32-ALU second launch of the fused step (what models the tensor-core launch rejects fall back to)."""
+    monkeypatch.setenv("DPCLIP_NO_T1_TF32", "1")
+    w = workloads.mlp_small()
+    layers = workloads.generate(w, 4)
+    _check_step(dp, w, _calibrate(w, layers, 4, w.C), w.C, w.sigma, 4)
+
+
+def test_step_mlp_padded_rows(dp):
+    """Input rows padded to a 16-byte stride with a width that is not a multiple of 4: tensor-core launch,
+    element-wise noise and store paths."""
+    B, d_in, d_out, C, sigma, seed = 70, 130, 72, 1.0, 0.8, 11
+    A, Z = workloads.random_layer(21, B, 1, d_in, d_out, "f32", scale_z=0.05)
+    hb = [True]
+    ref = oracle.step([(A, Z)], hb, C, sigma, seed, 0)
+    Ap = torch.zeros(B, 1, 132, device="cuda"); Ap[:, :, :d_in] = torch.from_numpy(A).cuda()
+    plan = dp.StepPlan([dp.Layer(Ap[:, :, :d_in], to_device(Z, "f32"), True)])
+    plan.run(C, sigma, seed, 0)
+    torch.cuda.synchronize()
+    assert dp.dpclip_read_status(plan.workspace) == 0
+    assert max_rel(plan.norms.cpu().numpy(), ref["norms"]) <= TOL["f32"]["norm"]
+    assert rel_fro(plan.gW[0].cpu().numpy(), ref["outW"][0]) <= TOL["f32"]["grad"]
+    assert rel_fro(plan.gb[0].cpu().numpy(), ref["outb"][0]) <= TOL["f32"]["grad"]
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_step_cnn(dp, dtype):
     w = workloads.cnn(dtype)
