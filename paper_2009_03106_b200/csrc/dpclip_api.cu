@@ -22,6 +22,7 @@ inline bool aligned_to(const void* p, size_t a) { return (reinterpret_cast<uintp
 inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // Kernels launched by this library since it was loaded (observability only; never read by a kernel).
 unsigned long long g_launches = 0;
+constexpr int kGridCounterOffset = 64;   // workspace header: status word at 0, grid-barrier counter here
 inline int launch_status() {
     ++g_launches;
     return cudaGetLastError() == cudaSuccess ? DPCLIP_OK : DPCLIP_ERR_CUDA;
@@ -457,7 +458,8 @@ int clipped_grad_impl(const void* A, long lda, const void* Zbar, long ldz, int B
 // Second launch of the fused step on the tensor cores (fp32 models).  Every layer must either be addressable
 // by TMA (16-byte aligned base and row stride); the zb of a thin layer (at most 16 outputs) need not be.  Returns 1 when the model
 // does not qualify, so that the caller falls back to the fp32-ALU kernel.
-int launch_fused_t1_tf32(const FusedT1Params& base, void* workspace, size_t workspace_bytes, cudaStream_t st) {
+int launch_fused_t1_tf32(const FusedT1Params& base, bool one_launch, void* workspace, size_t workspace_bytes,
+                         cudaStream_t st) {
     namespace f = tc::f1;
     { const char* env = getenv("DPCLIP_NO_T1_TF32"); if (env && env[0] == '1') return 1; }
     if (!workspace || workspace_bytes < kHeaderBytes) return 1;
@@ -483,9 +485,25 @@ int launch_fused_t1_tf32(const FusedT1Params& base, void* workspace, size_t work
     }
     if (!tc_layers) return 1;
     q.total_items = items;
-    if (!enable_smem(tc::t1_all_grads_tf32_kernel, f::SMEM_BYTES)) return DPCLIP_ERR_CUDA;
     const int grid = items < kNumSMs ? items : kNumSMs;
-    tc::t1_all_grads_tf32_kernel<<<grid, f::THREADS, f::SMEM_BYTES, st>>>(q);
+    if (one_launch) {
+        // the whole step as one cooperative launch (its CTAs meet at a grid-wide barrier)
+        q.grid_counter = reinterpret_cast<unsigned int*>(static_cast<char*>(workspace) + kGridCounterOffset);
+        if (!enable_smem(tc::t1_all_grads_tf32_kernel<true>, f::SMEM_BYTES)) return DPCLIP_ERR_CUDA;
+        cudaLaunchConfig_t cfg;
+        memset(&cfg, 0, sizeof(cfg));
+        cfg.gridDim = dim3(grid); cfg.blockDim = dim3(f::THREADS); cfg.dynamicSmemBytes = f::SMEM_BYTES; cfg.stream = st;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeCooperative; attr.val.cooperative = 1;
+        cfg.attrs = &attr; cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, tc::t1_all_grads_tf32_kernel<true>, q) != cudaSuccess) {
+            cudaGetLastError();
+            return 1;                       // cannot be made resident at once: take the two-launch form
+        }
+        return launch_status();
+    }
+    if (!enable_smem(tc::t1_all_grads_tf32_kernel<false>, f::SMEM_BYTES)) return DPCLIP_ERR_CUDA;
+    tc::t1_all_grads_tf32_kernel<false><<<grid, f::THREADS, f::SMEM_BYTES, st>>>(q);
     return launch_status();
 }
 
@@ -529,9 +547,15 @@ int try_fused_t1_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dty
     const int grid_g = tiles < 4 * kNumSMs ? tiles : 4 * kNumSMs;
     const int smem64 = FusedT1Cfg<64>::SMEM_BYTES, smem128 = FusedT1Cfg<128>::SMEM_BYTES;
     if (dtype == DPCLIP_F32) {
+        bool one = true;
+        { const char* env = getenv("DPCLIP_T1_ONE_LAUNCH"); if (env && env[0] == '0') one = false; }
+        if (one) {
+            const int rc = launch_fused_t1_tf32(p, true, workspace, workspace_bytes, st);
+            if (rc <= 0) return rc;
+        }
         t1_all_norms_kernel<float><<<grid_n, 128, 0, st>>>(p);
         if (launch_status()) return DPCLIP_ERR_CUDA;
-        const int rc = launch_fused_t1_tf32(p, workspace, workspace_bytes, st);
+        const int rc = launch_fused_t1_tf32(p, false, workspace, workspace_bytes, st);
         if (rc <= 0) return rc;
         if (tile == 128) {
             if (!enable_smem(t1_all_grads_kernel<float, 128>, smem128)) return DPCLIP_ERR_CUDA;

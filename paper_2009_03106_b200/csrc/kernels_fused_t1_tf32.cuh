@@ -4,9 +4,9 @@
 // norms, clipped sums of ALL layers, Philox noise added before the single
 // store of each output), but the products run as error-compensated tf32 on
 // tcgen05: per layer, 128 x 128 output tiles with K = B rows, operands brought
-// by TMA as 32-row stages, split into a tf32 high part and an fp32 low part by
-// the transform warps (which also apply diag(c) to the zb rows and take the
-// bias column sums), three MMAs per K = 8 step.
+// by TMA as 32-row stages and split on chip into a tf32 high part and an fp32
+// low part (the transform warps take the zb tile: diag(c), low plane, bias
+// column sums; the epilogue warps take the A tile), three MMAs per K = 8 step.
 //
 // The tensor core reads an fp32 word as tf32 by ignoring its low 13 mantissa
 // bits, so the high part needs no copy of its own: the (scaled) operand stays
@@ -57,6 +57,7 @@ struct Params {
     int tiles_n[FUSED_MAX_LAYERS];
     int total_items;
     int* status;
+    unsigned int* grid_counter;          // one-launch form: arrivals at the grid-wide barrier (self-resetting)
 };
 
 struct Item { int l, thin, m0, n0, tn; };
@@ -79,8 +80,79 @@ __device__ __forceinline__ float philox_normal(size_t e, unsigned long long sid,
     box_muller(b.v[e & 2], b.v[(e & 2) + 1], za, zb);
     return (e & 1) ? zb : za;
 }
+// Sums of squares of two rows (one of A, one of Zb), taken by one warp.  All loads of a pass (up to
+// eight 128-bit loads per lane and row) are issued before the first value is used: the rows are short and
+// the time is load latency.  Partial sums are returned per lane (warp_sum them).
+__device__ __forceinline__ void warp_rows_sumsq(const float* __restrict__ ra, int na, bool vec_a,
+                                                const float* __restrict__ rz, int nz, bool vec_z, int lane,
+                                                float& sa, float& sz) {
+    sa = 0.f; sz = 0.f;
+    const int nva = vec_a ? na >> 2 : 0, nvz = vec_z ? nz >> 2 : 0;
+    const int passes = (max(nva, nvz) + 255) >> 8;
+    for (int ps = 0; ps < passes; ++ps) {
+        float4 va[8], vz[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int j = (ps << 8) + (u << 5) + lane;
+            va[u] = j < nva ? *reinterpret_cast<const float4*>(ra + 4 * j) : make_float4(0.f, 0.f, 0.f, 0.f);
+            vz[u] = j < nvz ? *reinterpret_cast<const float4*>(rz + 4 * j) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            sa += (va[u].x * va[u].x + va[u].y * va[u].y) + (va[u].z * va[u].z + va[u].w * va[u].w);
+            sz += (vz[u].x * vz[u].x + vz[u].y * vz[u].y) + (vz[u].z * vz[u].z + vz[u].w * vz[u].w);
+        }
+    }
+    // tails, and rows that cannot take 128-bit loads
+    for (int j0 = nva << 2; j0 < na; j0 += 128) {
+        float v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) { const int j = j0 + (u << 5) + lane; v[u] = j < na ? ra[j] : 0.f; }
+        sa += (v[0] * v[0] + v[1] * v[1]) + (v[2] * v[2] + v[3] * v[3]);
+    }
+    for (int j0 = nvz << 2; j0 < nz; j0 += 128) {
+        float v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) { const int j = j0 + (u << 5) + lane; v[u] = j < nz ? rz[j] : 0.f; }
+        sz += (v[0] * v[0] + v[1] * v[1]) + (v[2] * v[2] + v[3] * v[3]);
+    }
+}
+
+__device__ __forceinline__ void named_barrier_sync(int id, int threads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
+// Grid-wide barrier of a cooperative launch (all CTAs resident).  Every CTA adds one to the counter on
+// arrival and one more when it leaves the kernel; the counter wraps to zero at 2 * gridDim.x, so each
+// launch finds it at zero.  The wait is bounded like every other wait here.
+__device__ __forceinline__ bool grid_barrier_arrive_and_wait(unsigned int* ctr, volatile int* abort_flag,
+                                                             int* status_word) {
+    __threadfence();
+    atomicInc(ctr, 2u * gridDim.x - 1u);
+    const uint64_t t0 = global_ns();
+    uint32_t spins = 0;
+    while (true) {
+        uint32_t v;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ctr) : "memory");
+        if (v >= gridDim.x) return true;
+        if ((++spins & 0x3F) == 0) {
+            if (*abort_flag) return false;
+            if (global_ns() - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                if (status_word) atomicExch(status_word, (int)DPCLIP_ERR_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
 }  // namespace f1
 
+// ONE_LAUNCH = false: second launch of the step (layer norms already in p.sq).
+// ONE_LAUNCH = true : the whole step in one cooperative launch.  TMA and the noise generator start at
+//                     once (neither depends on the factors); meanwhile the transform warps take the layer
+//                     norms of the rows dealt to this CTA, meet the other CTAs at a grid-wide barrier,
+//                     rebuild the factors and only then start on the staged tiles.
+template <bool ONE_LAUNCH>
 __global__ void __launch_bounds__(f1::THREADS, 1)
 t1_all_grads_tf32_kernel(const __grid_constant__ f1::Params q) {
     using namespace f1;
@@ -88,7 +160,7 @@ t1_all_grads_tf32_kernel(const __grid_constant__ f1::Params q) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);   // TMA landed
-    uint64_t* ready = full + STAGES;                                             // low planes written
+    uint64_t* ready = full + STAGES;                                             // low planes written (all 16 warps)
     uint64_t* empty = ready + STAGES;                                            // MMA done with the stage
     uint64_t* acc_full = empty + STAGES;
     uint64_t* acc_empty = acc_full + 2;
@@ -101,7 +173,7 @@ t1_all_grads_tf32_kernel(const __grid_constant__ f1::Params q) {
     if (threadIdx.x == 0) {
         DPCLIP_TRACE_AT(0, 255);
         for (int s = 0; s < STAGES; ++s) {
-            mbar_init(&full[s], 1); mbar_init(&ready[s], N_TRANSFORM_WARPS); mbar_init(&empty[s], 1);
+            mbar_init(&full[s], 1); mbar_init(&ready[s], N_TRANSFORM_WARPS + N_EPILOGUE_WARPS); mbar_init(&empty[s], 1);
         }
         for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], N_EPILOGUE_WARPS); }
         *abort_flag = 0;
@@ -113,6 +185,7 @@ t1_all_grads_tf32_kernel(const __grid_constant__ f1::Params q) {
     }
     if (warp == 1) { tmem_alloc(tmem_slot, 256); tmem_relinquish(); }
     // factors, rebuilt by every CTA from the layer norms (L * B floats, L2-resident)
+    if (!ONE_LAUNCH)
     for (int i = threadIdx.x; i < p.B; i += THREADS) {
         float s = 0.f;
         for (int l = 0; l < p.L; ++l) s += p.sq[(size_t)l * p.B + i];
@@ -129,6 +202,10 @@ t1_all_grads_tf32_kernel(const __grid_constant__ f1::Params q) {
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer
+        // one-launch form: the tiles are not needed before the factors exist, so the tile loads start when
+        // the norm phase has its rows (its few loads then do not queue behind megabytes of tile traffic,
+        // and the tile loads hit L2)
+        if (ONE_LAUNCH) named_barrier_sync(2, 32 + 32 * N_TRANSFORM_WARPS);
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0;
             bool ok = true;
@@ -211,6 +288,7 @@ t1_all_grads_tf32_kernel(const __grid_constant__ f1::Params q) {
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) { tc_fence_after_sync(); tmem_dealloc(tmem_base, 256); }
+    if (ONE_LAUNCH && threadIdx.x == 0) atomicInc(q.grid_counter, 2u * gridDim.x - 1u);   // leave: see the barrier
 }
 
 }  // namespace tc

@@ -97,13 +97,30 @@ __device__ __forceinline__ float bits_to_u01(uint32_t x) {          // (0, 1]
     return __fmaf_rn(__uint2float_rn(x), 2.3283064365386963e-10f, 1.1641532182693481e-10f);
 }
 
+// Box-Muller pair from two 32-bit draws.  The generator costs more issue slots than anything else in the
+// small fused steps, so it uses the hardware approximations where their error stays well inside the
+// 1e-5 absolute budget of a standard normal (every kernel shares this one function, so all launch
+// forms give the same bits):
+//   ln u1 : lg2.approx (relative error 2^-22 below 1/2, absolute 2^-22 above); within 2^-7 of 1, where an
+//           absolute error would dominate the small radius, the series -w - w^2/2 - w^3/3 - w^4/4, w = 1 - u1
+//   sqrt  : sqrt.approx (about 1 ulp)
+//   angle : 2 pi (u2 - 1/2) lies in (-pi, pi], where sin/cos.approx are good to 2^-20.9 absolute;
+//           cos(2 pi u2) = -cos(2 pi (u2 - 1/2)), likewise for sin
 __device__ __forceinline__ void box_muller(uint32_t xa, uint32_t xb, float& n0, float& n1) {
     const float u1 = bits_to_u01(xa), u2 = bits_to_u01(xb);
-    const float r = sqrtf(-2.0f * logf(u1));
+    float l2;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(l2) : "f"(u1));
+    const float w = 1.0f - u1;                                  // exact for u1 >= 1/2
+    const float series = -w * fmaf(w, fmaf(w, fmaf(w, 0.25f, 0.333333343f), 0.5f), 1.0f);
+    const float ln = w < 0.0078125f ? series : l2 * 0.693147182f;
+    float r;
+    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(-2.0f * ln));
+    const float th = 6.28318548f * (u2 - 0.5f);
     float s, c;
-    sincospif(2.0f * u2, &s, &c);
-    n0 = r * c;
-    n1 = r * s;
+    asm("sin.approx.ftz.f32 %0, %1;" : "=f"(s) : "f"(th));
+    asm("cos.approx.ftz.f32 %0, %1;" : "=f"(c) : "f"(th));
+    n0 = -r * c;
+    n1 = -r * s;
 }
 
 __global__ void __launch_bounds__(256)
