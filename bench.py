@@ -233,7 +233,8 @@ def kernel_breakdown(torch, dp, w, plan, steps, flush, C, sigma):
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures
 # summarised under profiles/ (same workload, same launch configuration); None where not captured
 NCU_TRAFFIC_BYTES = {
-    ("mlp_784_1000_1000_10_b128", "t1_all_grads_kernel"): 2.54e6,     # profiles/fused_t1_mlp_784_1000_1000_10_b128.txt
+    ("mlp_784_1000_1000_10_b128", "t1_all_grads_tf32_kernel"): 2.55e6,   # profiles/fused_t1_mlp_784_1000_1000_10_b128.txt
+    ("mlp_784_1000_1000_10_b128", "t1_all_grads_kernel"): 2.54e6,
     ("seq_b128_t256_d512_bf16", "grad[ffn_in]"): 171.7e6,             # profiles/tc_kernels_seq_b128_t256.txt
     ("seq_b128_t256_d512_bf16", "grad[lstm_gates]"): 171.7e6,
     ("seq_b128_t256_d512_bf16", "grad[ffn_out]"): 171.7e6,

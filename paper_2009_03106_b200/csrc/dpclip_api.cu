@@ -740,6 +740,7 @@ int dpclip_add_noise(float* g, size_t n, float sigma, float C, unsigned long lon
     if (n == 0) return DPCLIP_OK;
     if (!g || !(sigma >= 0.f) || !(C >= 0.f)) return DPCLIP_ERR_INVALID_ARG;
     if (!aligned_to(g, 4)) return DPCLIP_ERR_MISALIGNED;
+    if (sigma * C == 0.f) return DPCLIP_OK;          // nothing to add: no launch
     const size_t nq = (n + 3) / 4;
     size_t blocks = (nq + 255) / 256;
     const size_t cap = (size_t)kNumSMs * 16;

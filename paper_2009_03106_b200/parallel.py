@@ -7,8 +7,9 @@ the flat gradient buffer (NCCL over NVLink on GPUs), and the noise is added
 after the reduction, once, with the same (seed, stream) on every rank so that
 all ranks hold the same released gradient.
 
-`ops` is the set of entry points to call; it defaults to the CUDA binding.
-Tests on CPU ranks (gloo) pass their own object with the same four methods.
+`ops` is the set of entry points to call; it defaults to the CUDA binding
+(whose whole-step call covers everything before the reduction).  Tests on CPU
+ranks (gloo) pass their own object with the four per-stage methods.
 """
 from __future__ import annotations
 
@@ -18,11 +19,17 @@ import torch.distributed as dist
 def sharded_step(plan, C: float, sigma: float, seed: int, stream_id0: int = 0, group=None, ops=None) -> None:
     if ops is None:
         from . import binding as ops
-    for l, y in enumerate(plan.layers):
-        ops.dpclip_layer_sqnorms(y.A, y.Zbar, y.has_bias, plan.sq_layers[l], plan.workspace, y.method)
-    ops.dpclip_factors(plan.sq_layers, C, plan.clip, plan.norms)
-    for l, y in enumerate(plan.layers):
-        ops.dpclip_clipped_grad(y.A, y.Zbar, plan.clip, plan.gW[l], plan.gb[l], plan.workspace)
+    whole = getattr(ops, "dpclip_step", None)
+    if whole is not None:
+        # norms -> factors -> clipped sums of this rank's examples in one library call (sigma = 0: the noise
+        # belongs after the reduction); all-T=1 models take the one-launch fused kernel this way
+        whole(plan, C, 0.0, seed, stream_id0)
+    else:
+        for l, y in enumerate(plan.layers):
+            ops.dpclip_layer_sqnorms(y.A, y.Zbar, y.has_bias, plan.sq_layers[l], plan.workspace, y.method)
+        ops.dpclip_factors(plan.sq_layers, C, plan.clip, plan.norms)
+        for l, y in enumerate(plan.layers):
+            ops.dpclip_clipped_grad(y.A, y.Zbar, plan.clip, plan.gW[l], plan.gb[l], plan.workspace)
     if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
         dist.all_reduce(plan.flat, op=dist.ReduceOp.SUM, group=group)
     for l in range(len(plan.layers)):

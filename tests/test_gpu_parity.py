@@ -445,6 +445,23 @@ def test_step_seq_small(dp):
     _check_step(dp, w, _calibrate(w, layers, 2, w.C), w.C, w.sigma, 2)
 
 
+def test_sharded_step_single_rank_equals_step(dp):
+    """The data-parallel wrapper on one rank (no process group): whole-step call without noise, then the
+    noise launches, must give what one dpclip_step call gives."""
+    from paper_2009_03106_b200 import parallel
+    for w, seed in ((workloads.mlp_small(), 3), (workloads.seq("bf16", B=5, T=40, d=64, d_ff=136), 4)):
+        layers = workloads.generate(w, seed)
+        ref = _run_step(dp, w, layers, w.C, w.sigma, seed)
+        dls = [dp.Layer(to_device(A, w.dtype), to_device(Z, w.dtype), spec.has_bias)
+               for (A, Z), spec in zip(layers, w.layers)]
+        plan = dp.StepPlan(dls)
+        parallel.sharded_step(plan, w.C, w.sigma, seed, 0)
+        torch.cuda.synchronize()
+        assert dp.dpclip_read_status(plan.workspace) == 0
+        assert torch.equal(plan.clip, ref.clip)
+        assert rel_fro(plan.flat.cpu().numpy(), ref.flat.cpu().numpy()) <= 1e-6
+
+
 def test_step_host_matches_device_step(dp):
     w = workloads.mlp_small()
     layers = workloads.generate(w, 0)
