@@ -1,9 +1,10 @@
 // Tensor-core path for fp32 layers: Zb^T diag(f) A with error-compensated tf32.
 //
 // fp32 inputs must come out within 1e-5, which plain tf32 (10-bit mantissa)
-// cannot give.  Each operand x is split on chip into hi = x rounded to 10
-// mantissa bits (exactly a tf32 number) and lo = x - hi (exact in fp32,
-// at most 2^-10 |x|), and the product is taken as hi*hi + hi*lo + lo*hi with
+// cannot give.  Each operand x is split on chip into hi = x truncated to 10
+// mantissa bits (what the tensor core reads of the fp32 word itself, so the
+// high part needs no copy) and lo = x - hi (exact in fp32, below 2^-10 |x|,
+// written to a second plane), and the product is taken as hi*hi + hi*lo + lo*hi with
 // fp32 accumulation in tensor memory; the dropped lo*lo term and the tf32
 // rounding of lo are both about 2^-20 relative.  Three kind::tf32 MMAs replace
 // one fp32-ALU tile product at several times its speed.
@@ -17,9 +18,10 @@
 // Structure as zta_tc_kernel (same Params, same GRAD / NORM modes, same
 // split-row partial tiles): 128 x 128 output tile, 32-row stages; TMA brings
 // the raw fp32 tiles (MN-major, 32-column boxes of 128-byte rows, 32-byte swizzle atoms), the
-// transform warps apply the per-row factor to Zb, write hi in place and lo to a
-// second plane (and take the bias column sums on the way), one thread issues
-// the twelve MMAs of a stage, eight epilogue warps drain the accumulator.
+// transform warps apply the per-row factor to Zb in place and write its low
+// plane (taking the bias column sums on the way), the epilogue warps write the
+// low plane of A, one thread issues the twelve MMAs of a stage, and the
+// epilogue warps drain the accumulator.
 #pragma once
 #include "kernels_tc.cuh"
 
@@ -38,10 +40,6 @@ constexpr int THREADS = 64 + 32 * (N_TRANSFORM_WARPS + N_EPILOGUE_WARPS);
 constexpr int OUT_STAGE_BYTES = N_EPILOGUE_WARPS * 4096;
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 256 + OUT_STAGE_BYTES + 1024;
 constexpr uint32_t TF32_MASK = 0xFFFFE000u;           // keeps sign, exponent and 10 mantissa bits
-
-// x rounded to the nearest tf32 number (ties away from zero in magnitude); the low part x - hi is then
-// at most 2^-11 |x| with either sign, so what the tensor core drops of it does not add up one-sidedly.
-__device__ __forceinline__ uint32_t tf32_hi(uint32_t x) { return (x + 0x1000u) & TF32_MASK; }
 
 __device__ __forceinline__ zta::Item decode(const zta::Params& p, int item) {
     zta::Item w;
@@ -83,7 +81,7 @@ zta_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            mbar_init(&full[s], 1); mbar_init(&ready[s], N_TRANSFORM_WARPS); mbar_init(&empty[s], 1);
+            mbar_init(&full[s], 1); mbar_init(&ready[s], N_TRANSFORM_WARPS + N_EPILOGUE_WARPS); mbar_init(&empty[s], 1);
         }
         for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], N_EPILOGUE_WARPS); }
         *abort_flag = 0;
