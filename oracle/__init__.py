@@ -50,6 +50,12 @@ def lib():
             L.oracle_clipped_grad.argtypes = [_dp, _dp] + [ctypes.c_int] * 4 + [_dp, _dp, _dp]
             L.oracle_clipped_grad.restype = ctypes.c_int
             u32p = ctypes.POINTER(ctypes.c_uint32)
+            L.oracle_elementwise_example_grad.argtypes = [_dp, _dp, ctypes.c_int, ctypes.c_int, _dp, _dp]
+            L.oracle_elementwise_example_grad.restype = None
+            L.oracle_elementwise_sqnorms.argtypes = [_dp, _dp] + [ctypes.c_int] * 4 + [_dp]
+            L.oracle_elementwise_sqnorms.restype = ctypes.c_int
+            L.oracle_elementwise_clipped_grad.argtypes = [_dp, _dp] + [ctypes.c_int] * 3 + [_dp, _dp, _dp]
+            L.oracle_elementwise_clipped_grad.restype = ctypes.c_int
             L.oracle_philox4x32_10.argtypes = [u32p, u32p, u32p]
             L.oracle_philox4x32_10.restype = None
             L.oracle_normals.argtypes = [ctypes.c_size_t, ctypes.c_uint64, ctypes.c_uint64, _dp]
@@ -114,6 +120,41 @@ def clipped_grad(A, Z, clip: Optional[np.ndarray]) -> Tuple[np.ndarray, np.ndarr
     if lib().oracle_clipped_grad(_p(A), _p(Z), B, T, d_in, d_out, cp, _p(gW), _p(gb)):
         raise MemoryError
     return gW, gb
+
+
+def elementwise_example_grad(H_i, Z_i) -> Tuple[np.ndarray, np.ndarray]:
+    """H_i, Z_i: (T, d) -> (ggamma_i (d,), gbeta_i (d,)) of a LayerNorm-style gain/shift pair."""
+    H_i, Z_i = _f64(H_i), _f64(Z_i)
+    T, d = H_i.shape
+    assert Z_i.shape == (T, d)
+    gg = np.empty(d); gs = np.empty(d)
+    lib().oracle_elementwise_example_grad(_p(H_i), _p(Z_i), T, d, _p(gg), _p(gs))
+    return gg, gs
+
+
+def elementwise_sqnorms(H, Z, has_shift: bool) -> np.ndarray:
+    """H, Z: (B, T, d) -> squared per-example norms (B,) of the gain (and shift) gradients."""
+    H, Z = _f64(H), _f64(Z)
+    B, T, d = H.shape
+    assert Z.shape == (B, T, d)
+    sq = np.empty(B)
+    if lib().oracle_elementwise_sqnorms(_p(H), _p(Z), B, T, d, int(has_shift), _p(sq)):
+        raise MemoryError
+    return sq
+
+
+def elementwise_clipped_grad(H, Z, clip: Optional[np.ndarray]) -> Tuple[np.ndarray, np.ndarray]:
+    """-> (g_scale (d,), g_shift (d,)), the clipped sums before noise."""
+    H, Z = _f64(H), _f64(Z)
+    B, T, d = H.shape
+    g_scale = np.empty(d); g_shift = np.empty(d)
+    cp = None
+    if clip is not None:
+        clip = _f64(clip); assert clip.shape == (B,)
+        cp = _p(clip)
+    if lib().oracle_elementwise_clipped_grad(_p(H), _p(Z), B, T, d, cp, _p(g_scale), _p(g_shift)):
+        raise MemoryError
+    return g_scale, g_shift
 
 
 def philox4x32_10(ctr: Sequence[int], key: Sequence[int]) -> List[int]:

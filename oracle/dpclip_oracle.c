@@ -14,6 +14,7 @@
  *   convolution          G = deltaZ . im2col(X)               Algorithm 3
  *   recurrent / LSTM     dL/dW = sum_t dL/dz(t) (outer) h(t-1), dL/db = sum_t dL/dz(t)   Algorithm 4
  *   attention projection dL/dW^Q = (dL/dQ)^T Q_prev           Sec. "Multi-head attention"
+ *   LayerNorm gain/shift dL/dgamma = dL/dh (.) hbar, dL/dbeta = dL/dh   Sec. "LayerNorm Layers" and its Algorithm
  *
  * All of these are one formula once the layer input is given as A (T rows of
  * d_in) and the back-propagated signal as Zbar (T rows of d_out):
@@ -123,6 +124,57 @@ int oracle_clipped_grad(const double* A, const double* Z, int B, int T, int d_in
         for (int o = 0; o < d_out; ++o) gb_out[o] += c * gb[o];
     }
     free(G); free(gb);
+    return 0;
+}
+
+/* ------------------------------------------- element-wise parameter layers */
+
+/* LayerNorm-style layer h = gamma (.) hbar + beta (Sec. "LayerNorm Layers"): for one position the
+ * per-example gradients are dL/dgamma = dL/dh (.) hbar and dL/dbeta = dL/dh (the section's Algorithm is
+ * the product Z (.) H).  gamma and beta are shared by the T positions of an example, so, as for every
+ * shared parameter, the per-position terms are summed BEFORE the norm is taken:
+ *     ggamma_i = sum_t zbar_{i,t} (.) hbar_{i,t},   gbeta_i = sum_t zbar_{i,t}.
+ * H: T x d normalised inputs, Z: T x d back-propagated signals; gg[d], gs[d] OVERWRITTEN. */
+void oracle_elementwise_example_grad(const double* H, const double* Z, int T, int d, double* gg, double* gs)
+{
+    for (int j = 0; j < d; ++j) { gg[j] = 0.0; gs[j] = 0.0; }
+    for (int t = 0; t < T; ++t)
+        for (int j = 0; j < d; ++j) {
+            gg[j] += Z[(size_t)t * d + j] * H[(size_t)t * d + j];
+            gs[j] += Z[(size_t)t * d + j];
+        }
+}
+
+/* Squared per-example norms of such a layer: ||ggamma_i||^2 (+ ||gbeta_i||^2 with a shift).  sq[B]. */
+int oracle_elementwise_sqnorms(const double* H, const double* Z, int B, int T, int d, int has_shift, double* sq)
+{
+    double* gg = (double*)malloc(sizeof(double) * (size_t)d);
+    double* gs = (double*)malloc(sizeof(double) * (size_t)d);
+    if (!gg || !gs) { free(gg); free(gs); return -1; }
+    for (int i = 0; i < B; ++i) {
+        oracle_elementwise_example_grad(H + (size_t)i * T * d, Z + (size_t)i * T * d, T, d, gg, gs);
+        double s = sum_squares(gg, (size_t)d);
+        if (has_shift) s += sum_squares(gs, (size_t)d);
+        sq[i] = s;
+    }
+    free(gg); free(gs);
+    return 0;
+}
+
+/* Clipped sums: g_scale = sum_i clip[i] ggamma_i, g_shift = sum_i clip[i] gbeta_i (clip NULL = ones). */
+int oracle_elementwise_clipped_grad(const double* H, const double* Z, int B, int T, int d, const double* clip,
+                                    double* g_scale, double* g_shift)
+{
+    double* gg = (double*)malloc(sizeof(double) * (size_t)d);
+    double* gs = (double*)malloc(sizeof(double) * (size_t)d);
+    if (!gg || !gs) { free(gg); free(gs); return -1; }
+    for (int j = 0; j < d; ++j) { g_scale[j] = 0.0; g_shift[j] = 0.0; }
+    for (int i = 0; i < B; ++i) {
+        oracle_elementwise_example_grad(H + (size_t)i * T * d, Z + (size_t)i * T * d, T, d, gg, gs);
+        double c = clip ? clip[i] : 1.0;
+        for (int j = 0; j < d; ++j) { g_scale[j] += c * gg[j]; g_shift[j] += c * gs[j]; }
+    }
+    free(gg); free(gs);
     return 0;
 }
 

@@ -296,3 +296,74 @@ def test_every_clipped_example_is_within_C_on_a_workload():
     # clipped sum of B examples has norm at most B*C
     tot = np.sqrt(sum((g ** 2).sum() for g in res["gW"]) + sum((g ** 2).sum() for g in res["gb"]))
     assert tot <= w.B * w.C * (1 + 1e-9)
+
+
+# ---------------------------------------------------------------------------
+# element-wise parameter layers (LayerNorm gain and shift)
+# ---------------------------------------------------------------------------
+def test_layernorm_per_example_gradient_matches_autograd():
+    """A LayerNorm inside a small sequence network: the per-example gradients of its gain and shift,
+    taken by one backward pass per example, equal sum_t zbar (.) hbar and sum_t zbar."""
+    B, S, d = 3, 5, 6
+    g = torch.Generator().manual_seed(21)
+    X = torch.randn(B, S, d, generator=g)
+    W = torch.randn(d, d, generator=g)
+    gamma = torch.randn(d, generator=g, requires_grad=True)
+    beta = torch.randn(d, generator=g, requires_grad=True)
+    U = torch.tanh(X @ W.T)
+    mu = U.mean(dim=-1, keepdim=True)
+    var = ((U - mu) ** 2).mean(dim=-1, keepdim=True)
+    Hbar = (U - mu) / torch.sqrt(var + 1e-5)                   # normalised input: what the caller supplies
+    Hout = gamma * Hbar + beta
+    # the library routine must agree with this hand-written forward pass
+    np.testing.assert_allclose(Hout.detach().numpy(),
+                               F.layer_norm(U, (d,), gamma, beta, 1e-5).detach().numpy(), rtol=1e-12, atol=1e-12)
+    losses = (torch.sin(Hout) * torch.arange(1, S + 1).view(1, S, 1)).sum(dim=(1, 2))
+    for i in range(B):
+        gg_ref, gs_ref = torch.autograd.grad(losses[i], (gamma, beta), retain_graph=True)
+        (zbar,) = torch.autograd.grad(losses[i], (Hout,), retain_graph=True)
+        gg, gs = oracle.elementwise_example_grad(Hbar[i].detach().numpy(), zbar[i].numpy())
+        np.testing.assert_allclose(gg, gg_ref.numpy(), rtol=1e-11, atol=1e-13)
+        np.testing.assert_allclose(gs, gs_ref.numpy(), rtol=1e-11, atol=1e-13)
+
+
+def test_elementwise_layer_is_the_diagonal_of_the_dense_layer():
+    """h = gamma (.) hbar is a dense layer whose weight is diag(gamma): its gradient is the diagonal of
+    the dense per-example gradient, which the autograd pins above already fix."""
+    rng = np.random.default_rng(5)
+    B, T, d = 4, 7, 9
+    H = rng.standard_normal((B, T, d)); Z = rng.standard_normal((B, T, d))
+    sq = oracle.elementwise_sqnorms(H, Z, True)
+    sq_noshift = oracle.elementwise_sqnorms(H, Z, False)
+    for i in range(B):
+        G, gb = oracle.example_grad(H[i], Z[i])
+        gg, gs = oracle.elementwise_example_grad(H[i], Z[i])
+        np.testing.assert_allclose(gg, np.diag(G), rtol=1e-13, atol=1e-14)
+        np.testing.assert_allclose(gs, gb, rtol=1e-13, atol=1e-14)
+        np.testing.assert_allclose(sq[i], (np.diag(G) ** 2).sum() + (gb ** 2).sum(), rtol=1e-13)
+        np.testing.assert_allclose(sq_noshift[i], (np.diag(G) ** 2).sum(), rtol=1e-13)
+    # T = 1: the section's Algorithm, G = Z (.) H row by row
+    H1, Z1 = H[:, :1], Z[:, :1]
+    np.testing.assert_allclose(oracle.elementwise_sqnorms(H1, Z1, False), ((Z1 * H1) ** 2).sum(axis=(1, 2)), rtol=1e-13)
+
+
+def test_elementwise_clipped_sum_limits_and_linearity():
+    rng = np.random.default_rng(6)
+    B, T, d = 5, 3, 8
+    H = rng.standard_normal((B, T, d)); Z = rng.standard_normal((B, T, d))
+    g1, s1 = oracle.elementwise_clipped_grad(H, Z, None)                    # all factors one
+    np.testing.assert_allclose(g1, np.einsum("btj,btj->j", Z, H), rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(s1, Z.sum(axis=(0, 1)), rtol=1e-12, atol=1e-13)
+    c = rng.uniform(0.1, 1.0, B)
+    gc, sc = oracle.elementwise_clipped_grad(H, Z, c)
+    np.testing.assert_allclose(gc, np.einsum("i,itj,itj->j", c, Z, H), rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(sc, np.einsum("i,itj->j", c, Z), rtol=1e-12, atol=1e-13)
+    acc_g = np.zeros(d)
+    for i in range(B):                                                      # linear in the factors
+        e = np.zeros(B); e[i] = 1.0
+        acc_g += c[i] * oracle.elementwise_clipped_grad(H, Z, e)[0]
+    np.testing.assert_allclose(acc_g, gc, rtol=1e-12, atol=1e-13)
+    # permuting the positions of an example (jointly in H and Z) changes nothing
+    perm = rng.permutation(T)
+    np.testing.assert_allclose(oracle.elementwise_sqnorms(H[:, perm], Z[:, perm], True),
+                               oracle.elementwise_sqnorms(H, Z, True), rtol=1e-12)
