@@ -353,6 +353,24 @@ def bench_workload(torch, dp, w, steps, warmup, flush, peaks, with_e2e=True):
     return res
 
 
+def bench_elementwise(torch, dp, B, T, d, dtype, steps, flush, peaks):
+    """LayerNorm gain/shift parameters (element-wise layers): the two streaming kernels, each timed alone
+    with CUDA events, L2 flushed between launches.  Algorithmic bytes = Hbar and Zbar once per kernel."""
+    H, Z = workloads.layernorm_pair(0, B, T, d, dtype, var_z=1.0 / (B * T))
+    dH, dZ = to_dev(H, dtype, torch), to_dev(Z, dtype, torch)
+    clip = torch.rand(B, device="cuda") * 0.9 + 0.1
+    sq = torch.empty(B, device="cuda"); g = torch.empty(d, device="cuda"); sh = torch.empty(d, device="cuda")
+    nbytes = 2 * B * T * d * (4 if dtype == "f32" else 2)
+    out = dict(workload=f"layernorm_b{B}_t{T}_d{d}_{dtype}", algorithmic_bytes=nbytes)
+    for name, fn in (("norm", lambda: dp.dpclip_elementwise_sqnorms(dH, dZ, True, sq)),
+                     ("grad", lambda: dp.dpclip_elementwise_clipped_grad(dH, dZ, clip, g, sh))):
+        ms = float(np.median(time_steps(torch, fn, steps, 3, flush)))
+        ach = nbytes / (ms * 1e-3) / 1e9
+        out[name] = dict(ms=ms, roofline=dict(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s",
+                                              frac=ach / peaks["hbm_gbs"], traffic=None, peak_source=peaks["source"]))
+    return out
+
+
 # ---------------------------------------------------------------------------
 # CPU oracle legs
 # ---------------------------------------------------------------------------
@@ -503,6 +521,10 @@ def main():
                                 timing=("rotating sets, one graph of all timed steps" if r.get("rotating") else "flush + events per step"),
                                 step_roofline_frac=r["step_roofline_us"] / (ms * 1e3), roofline=r["roofline"],
                                 breakdown_us=r["breakdown"])
+        if args.others:
+            for shape in ((128, 256, 512, "bf16"), (512, 512, 1024, "bf16")):
+                r = bench_elementwise(torch, dp, *shape, min(args.steps, 20), flush, peaks)
+                others[r["workload"]] = r
         line["workloads"] = others
         if not args.no_cpu_baseline:
             line["cpu_baseline"], _, _ = oracle_sample(w)

@@ -109,6 +109,28 @@ int dpclip_clipped_grad(const void* A, long lda, const void* Zbar, long ldz,
                         const float* clip, float* gW, long ldg, float* gb,
                         void* workspace, size_t workspace_bytes, void* stream);
 
+/* Element-wise parameter layers h = gamma (.) hbar + beta (Sec. "LayerNorm Layers" and its
+ * Algorithm, G = Z (.) H): per example the gradients are
+ *   ggamma_i = sum_t zb_{i,t} (.) hbar_{i,t}   and   gbeta_i = sum_t zb_{i,t},
+ * the sum over the T positions that share gamma and beta being taken before the norm.
+ *   Hbar, Zbar  device, [B*T][ld] row-major, dtype `dtype`: the NORMALISED layer input and the
+ *               back-propagated signal of the layer output (the caller normalises; the library
+ *               never sees mean or variance)
+ *   sq_layer    [B] fp32, OVERWRITTEN with ||ggamma_i||^2 (+ ||gbeta_i||^2 when has_shift): one
+ *               more row of the [L][B] array that dpclip_factors sums
+ *   clip        [B] or NULL (all ones)
+ *   g_scale     [d] fp32, OVERWRITTEN with sum_i clip[i] ggamma_i
+ *   g_shift     [d] fp32 or NULL, OVERWRITTEN with sum_i clip[i] gbeta_i
+ * Noise is added with dpclip_add_noise on g_scale / g_shift.  No workspace; partial sums of a
+ * column are combined with fp32 atomics, so the last bits depend on the order of arrival.
+ * Errors as for dpclip_layer_sqnorms. */
+int dpclip_elementwise_sqnorms(const void* Hbar, long ldh, const void* Zbar, long ldz,
+                               int B, int T, int d, dpclip_dtype dtype, int has_shift,
+                               float* sq_layer, void* stream);
+int dpclip_elementwise_clipped_grad(const void* Hbar, long ldh, const void* Zbar, long ldz,
+                                    int B, int T, int d, dpclip_dtype dtype,
+                                    const float* clip, float* g_scale, float* g_shift, void* stream);
+
 /* Gaussian mechanism: g[j] += sigma * C * xi_j for j in [0, n), xi_j ~ N(0,1).
  * The paper names no generator.  This library uses Philox4x32-10 with key =
  * (seed lo, seed hi) and counter = (q lo, q hi, stream_id lo, stream_id hi),

@@ -60,6 +60,10 @@ def load_library():
                                             _u64, _vp, _sz, _vp]
     L.dpclip_clipped_grad_noise.restype = _i
     L.dpclip_add_noise.argtypes = [_vp, _sz, _f, _f, _u64, _u64, _vp]
+    L.dpclip_elementwise_sqnorms.argtypes = [_vp, _l, _vp, _l, _i, _i, _i, _i, _i, _vp, _vp]
+    L.dpclip_elementwise_sqnorms.restype = _i
+    L.dpclip_elementwise_clipped_grad.argtypes = [_vp, _l, _vp, _l, _i, _i, _i, _i, _vp, _vp, _vp, _vp]
+    L.dpclip_elementwise_clipped_grad.restype = _i
     L.dpclip_step.argtypes = [ctypes.POINTER(_CLayer), _i, _i, _i, _f, _f, _u64, _u64, _vp, _vp, _vp, _vp, _sz, _vp]
     L.dpclip_step_host.argtypes = [ctypes.POINTER(_CLayer), _i, _i, _i, _f, _f, _u64, _u64, _vp, _vp, _vp, _sz, _vp]
     L.dpclip_step_host_arena_bytes.argtypes = [ctypes.POINTER(_CLayer), _i, _i, _i]
@@ -223,6 +227,29 @@ def dpclip_add_noise(g: torch.Tensor, sigma: float, C: float, seed: int, stream_
     assert g.dtype == torch.float32 and g.is_contiguous()
     _check("dpclip_add_noise", load_library().dpclip_add_noise(_ptr(g), g.numel(), sigma, C, seed, stream_id,
                                                                _stream(stream)))
+
+
+def dpclip_elementwise_sqnorms(Hbar: torch.Tensor, Zbar: torch.Tensor, has_shift: bool, sq_layer: torch.Tensor,
+                               stream=None) -> None:
+    B, T, d, ldh = _rows(Hbar)
+    B2, T2, d2, ldz = _rows(Zbar)
+    assert (B, T, d) == (B2, T2, d2) and Hbar.dtype == Zbar.dtype
+    assert sq_layer.dtype == torch.float32 and sq_layer.numel() >= B and sq_layer.is_contiguous()
+    _check("dpclip_elementwise_sqnorms", load_library().dpclip_elementwise_sqnorms(
+        _ptr(Hbar), ldh, _ptr(Zbar), ldz, B, T, d, _dtype_code(Hbar), int(has_shift), _ptr(sq_layer), _stream(stream)))
+
+
+def dpclip_elementwise_clipped_grad(Hbar: torch.Tensor, Zbar: torch.Tensor, clip: Optional[torch.Tensor],
+                                    g_scale: torch.Tensor, g_shift: Optional[torch.Tensor], stream=None) -> None:
+    B, T, d, ldh = _rows(Hbar)
+    B2, T2, d2, ldz = _rows(Zbar)
+    assert (B, T, d) == (B2, T2, d2) and Hbar.dtype == Zbar.dtype
+    assert g_scale.dtype == torch.float32 and g_scale.numel() == d and g_scale.is_contiguous()
+    assert g_shift is None or (g_shift.dtype == torch.float32 and g_shift.numel() == d and g_shift.is_contiguous())
+    assert clip is None or (clip.dtype == torch.float32 and clip.numel() >= B and clip.is_contiguous())
+    _check("dpclip_elementwise_clipped_grad", load_library().dpclip_elementwise_clipped_grad(
+        _ptr(Hbar), ldh, _ptr(Zbar), ldz, B, T, d, _dtype_code(Hbar), _ptr(clip) if clip is not None else None,
+        _ptr(g_scale), _ptr(g_shift) if g_shift is not None else None, _stream(stream)))
 
 
 # ----------------------------------------------------------------------------

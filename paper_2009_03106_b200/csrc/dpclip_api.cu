@@ -10,6 +10,7 @@
 #include "kernels_tf32.cuh"
 #include "kernels_fused_t1.cuh"
 #include "kernels_narrow.cuh"
+#include "kernels_elementwise.cuh"
 
 #include <stdlib.h>
 
@@ -733,6 +734,51 @@ int dpclip_clipped_grad_noise(const void* A, long lda, const void* Zbar, long ld
     rc = dpclip_add_noise(gW, (size_t)d_out * d_in, sigma, C, seed, stream_id_w, stream);
     if (rc || !gb) return rc;
     return dpclip_add_noise(gb, (size_t)d_out, sigma, C, seed, stream_id_b, stream);
+}
+
+int dpclip_elementwise_sqnorms(const void* Hbar, long ldh, const void* Zbar, long ldz, int B, int T, int d,
+                               dpclip_dtype dtype, int has_shift, float* sq_layer, void* stream) {
+    int rc = check_layer_args(Hbar, ldh, Zbar, ldz, B, T, d, d, dtype);
+    if (rc) return rc;
+    if (!sq_layer) return DPCLIP_ERR_INVALID_ARG;
+    if (B > 65535) return DPCLIP_ERR_UNSUPPORTED;
+    cudaStream_t st = (cudaStream_t)stream;
+    const bool vec = vec4_ok(Hbar, ldh, dtype) && vec4_ok(Zbar, ldz, dtype) && d % 4 == 0;
+    const int v = vec ? 4 : 1;
+    const int cg = (long)ceil_div(d, 64 * v) * B >= 4L * kNumSMs ? 64 : 32;
+    const dim3 grid(ceil_div(d, cg * v), B);
+    const int use_atomic = grid.x > 1;
+    if (use_atomic && cudaMemsetAsync(sq_layer, 0, sizeof(float) * (size_t)B, st) != cudaSuccess) return DPCLIP_ERR_CUDA;
+    if (dtype == DPCLIP_F32) launch_ew_norm<float>(vec, cg, grid, st, Hbar, ldh, Zbar, ldz, T, d, has_shift, sq_layer, use_atomic);
+    else launch_ew_norm<__nv_bfloat16>(vec, cg, grid, st, Hbar, ldh, Zbar, ldz, T, d, has_shift, sq_layer, use_atomic);
+    return launch_status();
+}
+
+int dpclip_elementwise_clipped_grad(const void* Hbar, long ldh, const void* Zbar, long ldz, int B, int T, int d,
+                                    dpclip_dtype dtype, const float* clip, float* g_scale, float* g_shift,
+                                    void* stream) {
+    int rc = check_layer_args(Hbar, ldh, Zbar, ldz, B, T, d, d, dtype);
+    if (rc) return rc;
+    if (!g_scale) return DPCLIP_ERR_INVALID_ARG;
+    if (!aligned_to(g_scale, 4) || (g_shift && !aligned_to(g_shift, 4))) return DPCLIP_ERR_MISALIGNED;
+    cudaStream_t st = (cudaStream_t)stream;
+    const bool vec = vec4_ok(Hbar, ldh, dtype) && vec4_ok(Zbar, ldz, dtype) && d % 4 == 0;
+    const int v = vec ? 4 : 1;
+    const long R = (long)B * T;
+    const int cg = 64;
+    const int col_blocks = ceil_div(d, cg * v);
+    // about four CTAs per SM in all, and at least 64 rows per CTA
+    long slices = (4L * kNumSMs + col_blocks - 1) / col_blocks;
+    if (slices > (R + 63) / 64) slices = (R + 63) / 64;
+    if (slices < 1) slices = 1;
+    if (slices > 65535) slices = 65535;
+    const long rows_per_cta = (R + slices - 1) / slices;
+    const dim3 grid(col_blocks, (unsigned)ceil_div(R, rows_per_cta));
+    if (cudaMemsetAsync(g_scale, 0, sizeof(float) * (size_t)d, st) != cudaSuccess) return DPCLIP_ERR_CUDA;
+    if (g_shift && cudaMemsetAsync(g_shift, 0, sizeof(float) * (size_t)d, st) != cudaSuccess) return DPCLIP_ERR_CUDA;
+    if (dtype == DPCLIP_F32) launch_ew_grad<float>(vec, cg, grid, st, Hbar, ldh, Zbar, ldz, R, rows_per_cta, T, d, clip, g_scale, g_shift);
+    else launch_ew_grad<__nv_bfloat16>(vec, cg, grid, st, Hbar, ldh, Zbar, ldz, R, rows_per_cta, T, d, clip, g_scale, g_shift);
+    return launch_status();
 }
 
 int dpclip_add_noise(float* g, size_t n, float sigma, float C, unsigned long long seed,

@@ -167,6 +167,96 @@ def test_tf32_clipped_grad(dp, B, T, d_in, d_out):
 
 
 # ---------------------------------------------------------------------------
+# element-wise parameter layers (LayerNorm gain / shift)
+# ---------------------------------------------------------------------------
+EW_SHAPES = [(1, 1, 1), (3, 1, 10), (5, 7, 33), (4, 40, 64), (6, 37, 260), (128, 1, 1000), (16, 256, 512), (3, 300, 1028)]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("B,T,d", EW_SHAPES)
+def test_elementwise_norms_and_clipped_sums(dp, B, T, d, dtype):
+    H, Z = workloads.layernorm_pair(31, B, T, d, dtype, var_z=0.01)
+    tol = TOL[dtype]
+    dH, dZ = to_device(H, dtype), to_device(Z, dtype)
+    for has_shift in (True, False):
+        ref = oracle.elementwise_sqnorms(H, Z, has_shift)
+        sq = torch.full((B,), -1.0, device="cuda")
+        dp.dpclip_elementwise_sqnorms(dH, dZ, has_shift, sq)
+        got = sq.cpu().numpy()
+        assert max_rel(np.sqrt(got), np.sqrt(ref)) <= tol["norm"], max_rel(np.sqrt(got), np.sqrt(ref))
+    clip = np.random.default_rng(B + d).uniform(0.05, 1.0, B).astype(np.float32)
+    clip[::2] = 1.0
+    for c in (clip, None):
+        ref_g, ref_s = oracle.elementwise_clipped_grad(H, Z, c)
+        g_scale = torch.full((d,), 7.0, device="cuda"); g_shift = torch.full((d,), 7.0, device="cuda")
+        dp.dpclip_elementwise_clipped_grad(dH, dZ, None if c is None else torch.from_numpy(c).cuda(), g_scale, g_shift)
+        assert rel_fro(g_scale.cpu().numpy(), ref_g) <= tol["grad"], rel_fro(g_scale.cpu().numpy(), ref_g)
+        assert rel_fro(g_shift.cpu().numpy(), ref_s) <= tol["grad"]
+    only = torch.full((d,), 7.0, device="cuda")
+    dp.dpclip_elementwise_clipped_grad(dH, dZ, torch.from_numpy(clip).cuda(), only, None)     # no shift parameter
+    assert rel_fro(only.cpu().numpy(), oracle.elementwise_clipped_grad(H, Z, clip)[0]) <= tol["grad"]
+
+
+def test_elementwise_padded_rows(dp):
+    """Row stride larger than the width, and a width that is not a multiple of 4 (scalar path)."""
+    B, T, d, ld = 5, 9, 30, 32
+    H, Z = workloads.layernorm_pair(32, B, T, d, "f32", var_z=0.01)
+    Hp = torch.full((B, T, ld), float("nan"), device="cuda"); Zp = torch.full((B, T, ld), float("nan"), device="cuda")
+    Hp[:, :, :d] = torch.from_numpy(H).cuda(); Zp[:, :, :d] = torch.from_numpy(Z).cuda()
+    sq = torch.empty(B, device="cuda")
+    dp.dpclip_elementwise_sqnorms(Hp[:, :, :d], Zp[:, :, :d], True, sq)
+    assert max_rel(np.sqrt(sq.cpu().numpy()), np.sqrt(oracle.elementwise_sqnorms(H, Z, True))) <= TOL["f32"]["norm"]
+    g = torch.empty(d, device="cuda"); s = torch.empty(d, device="cuda")
+    dp.dpclip_elementwise_clipped_grad(Hp[:, :, :d], Zp[:, :, :d], None, g, s)
+    rg, rs = oracle.elementwise_clipped_grad(H, Z, None)
+    assert rel_fro(g.cpu().numpy(), rg) <= TOL["f32"]["grad"] and rel_fro(s.cpu().numpy(), rs) <= TOL["f32"]["grad"]
+
+
+def test_transformer_block_with_layernorms(dp):
+    """Dense layers and LayerNorm parameters of one block clipped together: per-layer norm rows from both
+    kinds of entry points, one factor computation, clipped sums and noise per tensor."""
+    B, T, d, dff, C, sigma, seed = 6, 24, 64, 136, 1.0, 0.7, 9
+    w = workloads.seq("bf16", B=B, T=T, d=d, d_ff=dff)
+    dense = workloads.generate(w, 3)
+    lns = [workloads.layernorm_pair(40 + k, B, T, d, "bf16", var_z=1.0 / (B * T)) for k in range(2)]
+    hb = [s.has_bias for s in w.layers]
+    sq_ref = [oracle.layer_sqnorms(A, Z, b) for (A, Z), b in zip(dense, hb)] + [oracle.elementwise_sqnorms(H, Z, True) for H, Z in lns]
+    # spread the norms around C as the calibrated workloads do
+    n0, _ = oracle.factors(np.stack(sq_ref), C)
+    r = workloads.spread_factors(B, 1) * C / n0
+    scale = lambda Z: workloads.round_to_bf16((Z.astype(np.float64) * r[:, None, None]).astype(np.float32))   # noqa: E731
+    dense = [(A, scale(Z)) for A, Z in dense]
+    lns = [(H, scale(Z)) for H, Z in lns]
+    sq_ref = np.stack([oracle.layer_sqnorms(A, Z, b) for (A, Z), b in zip(dense, hb)] +
+                      [oracle.elementwise_sqnorms(H, Z, True) for H, Z in lns])
+    norms_ref, clip_ref = oracle.factors(sq_ref, C)
+    L = len(dense) + len(lns)
+    sq = torch.empty(L, B, device="cuda"); ws = _ws(dp)
+    dd = [(to_device(A, "bf16"), to_device(Z, "bf16")) for A, Z in dense]
+    dl = [(to_device(H, "bf16"), to_device(Z, "bf16")) for H, Z in lns]
+    for l, ((A, Z), b) in enumerate(zip(dd, hb)):
+        dp.dpclip_layer_sqnorms(A, Z, b, sq[l], ws)
+    for k, (H, Z) in enumerate(dl):
+        dp.dpclip_elementwise_sqnorms(H, Z, True, sq[len(dd) + k])
+    clip = torch.empty(B, device="cuda"); norms = torch.empty(B, device="cuda")
+    dp.dpclip_factors(sq, C, clip, norms)
+    assert max_rel(norms.cpu().numpy(), norms_ref) <= TOL["bf16"]["norm"]
+    check_saturation(clip.cpu().numpy(), norms_ref, clip_ref, C)
+    assert 0 < int((clip < 1).sum()) < B
+    for k, ((H, Z), (Hn, Zn)) in enumerate(zip(dl, lns)):
+        g = torch.empty(d, device="cuda"); s = torch.empty(d, device="cuda")
+        dp.dpclip_elementwise_clipped_grad(H, Z, clip, g, s)
+        rg, rs = oracle.elementwise_clipped_grad(Hn, Zn, clip_ref)
+        assert rel_fro(g.cpu().numpy(), rg) <= TOL["bf16"]["grad"] and rel_fro(s.cpu().numpy(), rs) <= TOL["bf16"]["grad"]
+        pre = g.clone()
+        sid = 2 * (len(dd) + k)
+        dp.dpclip_add_noise(g, sigma, C, seed, sid)
+        xi = oracle.normals(d, seed, sid)
+        assert np.max(np.abs((g - pre).cpu().numpy() - sigma * C * xi)) <= 1e-5 * sigma * C + 1e-6
+    assert dp.dpclip_read_status(ws) == 0
+
+
+# ---------------------------------------------------------------------------
 # (c) factors
 # ---------------------------------------------------------------------------
 @pytest.mark.parametrize("B,L", [(1, 1), (32, 2), (128, 3), (1024, 7), (1500, 2)])

@@ -235,3 +235,17 @@ def random_layer(rng_seed: int, B: int, T: int, d_in: int, d_out: int, dtype: st
     if dtype == "bf16":
         A, Z = round_to_bf16(A), round_to_bf16(Z)
     return A, Z
+
+
+def layernorm_pair(rng_seed: int, B: int, T: int, d: int, dtype: str = "f32", var_z: float = 1.0
+                   ) -> Tuple[np.ndarray, np.ndarray]:
+    """Inputs of an element-wise gain/shift layer: Hbar (B, T, d) with every row normalised to zero mean
+    and unit variance (what a LayerNorm hands to its gain), Zbar ~ N(0, var_z)."""
+    rng = np.random.default_rng([rng_seed, B, T, d, 0x1A7E2])
+    X = rng.standard_normal((B, T, d), dtype=np.float32)
+    X -= X.mean(axis=-1, keepdims=True)
+    X /= np.sqrt((X * X).mean(axis=-1, keepdims=True) + np.float32(1e-5))
+    Z = rng.standard_normal((B, T, d), dtype=np.float32) * np.float32(np.sqrt(var_z))
+    if dtype == "bf16":
+        X, Z = round_to_bf16(X), round_to_bf16(Z)
+    return np.ascontiguousarray(X), np.ascontiguousarray(Z)
