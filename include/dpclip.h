@@ -214,7 +214,13 @@ int dpclip_step(const dpclip_layer* layers /* host */, int L, int B, dpclip_dtyp
  * buffer of at least dpclip_step_host_arena_bytes() bytes that stages inputs,
  * outputs and the workspace.  host_clip [B] and host_norms [B] (either may be
  * NULL) receive the factors.  All copies and kernels are enqueued on `stream`;
- * the results are valid after the caller synchronises it. */
+ * the results are valid after the caller synchronises it.
+ * Copies are merged when the host tensors of a direction are carved out of one
+ * buffer in arena order, each on the next 256-byte boundary: inputs as
+ * A_0, Zbar_0, A_1, Zbar_1, ... give ONE host-to-device copy; results as gW_0,
+ * gb_0 (its d_out*4-byte slot is kept even without a bias), gW_1, ..., clip,
+ * norms give ONE device-to-host copy.  Any other placement is copied tensor by
+ * tensor. */
 int dpclip_step_host(const dpclip_layer* layers /* host, host pointers inside */, int L, int B,
                      dpclip_dtype dtype, float C, float sigma,
                      unsigned long long seed, unsigned long long stream_id0,

@@ -370,7 +370,11 @@ class HostStep:
     copied to the device, the path runs, outputs are copied back, all inside
     one dpclip_step_host call enqueued on the current stream."""
 
-    def __init__(self, host_layers: Sequence[Layer], device="cuda"):
+    def __init__(self, host_layers: Sequence[Layer], device="cuda", pack_inputs: bool = False):
+        """Results always live in one pinned buffer carved up in the library's arena order, so they come
+        back in one copy.  pack_inputs=True also copies the given host tensors, once, into one pinned
+        buffer in arena order (`self.layers` then holds views of it for the caller to refill every step),
+        so the inputs go up in one copy too."""
         self.layers = list(host_layers)
         self.L = len(self.layers)
         self.B = self.layers[0].A.shape[0]
@@ -379,19 +383,38 @@ class HostStep:
         self.gW, self.gb = [], []
         self.h2d_bytes = 0
         self.d2h_bytes = 0
-        for l, y in enumerate(self.layers):
+        up = lambda n: (n + 255) // 256 * 256                                   # noqa: E731
+        shapes = []
+        for y in self.layers:
             assert not y.A.is_cuda and y.A.is_contiguous() and y.Zbar.is_contiguous()
             B, T, d_in, _ = _rows(y.A)
             _, _, d_out, _ = _rows(y.Zbar)
-            gW = torch.empty((d_out, d_in), dtype=torch.float32).pin_memory()
-            gb = torch.empty((d_out,), dtype=torch.float32).pin_memory() if y.has_bias else None
+            shapes.append((T, d_in, d_out))
+        es = self.layers[0].A.element_size()
+        if pack_inputs:
+            total = sum(up(self.B * T * d_in * es) + up(self.B * T * d_out * es) for T, d_in, d_out in shapes)
+            self._in_flat = torch.empty((total,), dtype=torch.uint8).pin_memory()
+            off, packed = 0, []
+            for y, (T, d_in, d_out) in zip(self.layers, shapes):
+                na, nz = self.B * T * d_in * es, self.B * T * d_out * es
+                a = self._in_flat[off:off + na].view(y.A.dtype).view(y.A.shape); off += up(na)
+                z = self._in_flat[off:off + nz].view(y.Zbar.dtype).view(y.Zbar.shape); off += up(nz)
+                a.copy_(y.A); z.copy_(y.Zbar)
+                packed.append(Layer(a, z, y.has_bias, y.method))
+            self.layers = packed
+        total = sum(up(d_out * d_in * 4) + up(d_out * 4) for _, d_in, d_out in shapes) + 2 * up(self.B * 4)
+        self._out_flat = torch.empty((total,), dtype=torch.uint8).pin_memory()
+        off = 0
+        for l, (y, (T, d_in, d_out)) in enumerate(zip(self.layers, shapes)):
+            gW = self._out_flat[off:off + d_out * d_in * 4].view(torch.float32).view(d_out, d_in); off += up(d_out * d_in * 4)
+            gb = self._out_flat[off:off + d_out * 4].view(torch.float32) if y.has_bias else None; off += up(d_out * 4)
             self.gW.append(gW); self.gb.append(gb)
             self._c[l] = _CLayer(_ptr(y.A), d_in, _ptr(y.Zbar), d_out, T, d_in, d_out, int(y.has_bias),
                                  y.method, _ptr(gW), d_in, _ptr(gb))
             self.h2d_bytes += y.A.numel() * y.A.element_size() + y.Zbar.numel() * y.Zbar.element_size()
             self.d2h_bytes += gW.numel() * 4 + (gb.numel() * 4 if gb is not None else 0)
-        self.clip = torch.empty((self.B,), dtype=torch.float32).pin_memory()
-        self.norms = torch.empty((self.B,), dtype=torch.float32).pin_memory()
+        self.clip = self._out_flat[off:off + self.B * 4].view(torch.float32); off += up(self.B * 4)
+        self.norms = self._out_flat[off:off + self.B * 4].view(torch.float32); off += up(self.B * 4)
         self.d2h_bytes += 8 * self.B
         nbytes = load_library().dpclip_step_host_arena_bytes(self._c, self.L, self.B, self.dtype_code)
         self.arena = torch.empty((nbytes,), dtype=torch.uint8, device=device)

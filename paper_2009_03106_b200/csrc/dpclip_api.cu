@@ -880,27 +880,61 @@ int dpclip_step_host(const dpclip_layer* layers, int L, int B, dpclip_dtype dtyp
     }
     void* ws = take(ws_bytes);
     float* sq = (float*)take((size_t)L * B * 4);
-    float* clip = (float*)take((size_t)B * 4);
-    float* norms = (float*)take((size_t)B * 4);
     if (dpclip_workspace_init(ws, ws_bytes, stream)) return DPCLIP_ERR_CUDA;
 
+    // Arena: [workspace][sq][A_0][Zb_0][A_1][Zb_1]...[gW_0][gb_0][gW_1]...[clip][norms], every tensor on
+    // the next 256-byte boundary.  When the host tensors of a direction sit back to back in the same
+    // order with the same padding (one pinned buffer carved up this way), that direction is ONE copy.
     dpclip_layer dev[64];
+    char* in_begin = cur;
+    bool in_packed = true;
+    const char* h_in0 = static_cast<const char*>(layers[0].A);
     for (int l = 0; l < L; ++l) {
         const dpclip_layer& y = layers[l];
         dev[l] = y;
         const size_t a_bytes = (size_t)B * y.T * y.d_in * es, z_bytes = (size_t)B * y.T * y.d_out * es;
-        void* dA = take(a_bytes);
-        void* dZ = take(z_bytes);
-        dev[l].A = dA; dev[l].Zbar = dZ;
+        dev[l].A = take(a_bytes);
+        dev[l].Zbar = take(z_bytes);
+        in_packed = in_packed && static_cast<const char*>(y.A) - h_in0 == static_cast<const char*>(dev[l].A) - in_begin &&
+                    static_cast<const char*>(y.Zbar) - h_in0 == static_cast<const char*>(dev[l].Zbar) - in_begin;
+    }
+    const size_t in_bytes = (size_t)(cur - in_begin);
+    char* out_begin = cur;
+    bool out_packed = true;
+    const char* h_out0 = reinterpret_cast<const char*>(layers[0].gW);
+    for (int l = 0; l < L; ++l) {
+        const dpclip_layer& y = layers[l];
         dev[l].gW = (float*)take((size_t)y.d_out * y.d_in * 4);
         dev[l].gb = (float*)take((size_t)y.d_out * 4);
+        out_packed = out_packed && reinterpret_cast<const char*>(y.gW) - h_out0 == reinterpret_cast<const char*>(dev[l].gW) - out_begin &&
+                     (!y.has_bias || reinterpret_cast<const char*>(y.gb) - h_out0 == reinterpret_cast<const char*>(dev[l].gb) - out_begin);
         if (!y.has_bias) dev[l].gb = nullptr;
-        if (cudaMemcpyAsync(dA, y.A, a_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-            cudaMemcpyAsync(dZ, y.Zbar, z_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
-            return DPCLIP_ERR_CUDA;
+    }
+    float* clip = (float*)take((size_t)B * 4);
+    float* norms = (float*)take((size_t)B * 4);
+    out_packed = out_packed && host_clip && host_norms &&
+                 reinterpret_cast<const char*>(host_clip) - h_out0 == reinterpret_cast<const char*>(clip) - out_begin &&
+                 reinterpret_cast<const char*>(host_norms) - h_out0 == reinterpret_cast<const char*>(norms) - out_begin;
+    const size_t out_bytes = (size_t)(cur - out_begin);
+
+    if (in_packed) {
+        if (cudaMemcpyAsync(in_begin, h_in0, in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return DPCLIP_ERR_CUDA;
+    } else {
+        for (int l = 0; l < L; ++l) {
+            const dpclip_layer& y = layers[l];
+            const size_t a_bytes = (size_t)B * y.T * y.d_in * es, z_bytes = (size_t)B * y.T * y.d_out * es;
+            if (cudaMemcpyAsync(const_cast<void*>(dev[l].A), y.A, a_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+                cudaMemcpyAsync(const_cast<void*>(dev[l].Zbar), y.Zbar, z_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+                return DPCLIP_ERR_CUDA;
+        }
     }
     int rc = dpclip_step(dev, L, B, dtype, C, sigma, seed, stream_id0, sq, clip, norms, ws, ws_bytes, stream);
     if (rc) return rc;
+    if (out_packed) {
+        if (cudaMemcpyAsync(const_cast<char*>(h_out0), out_begin, out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+            return DPCLIP_ERR_CUDA;
+        return DPCLIP_OK;
+    }
     for (int l = 0; l < L; ++l) {
         const dpclip_layer& y = layers[l];
         if (cudaMemcpyAsync(y.gW, dev[l].gW, (size_t)y.d_out * y.d_in * 4, cudaMemcpyDeviceToHost, st) !=

@@ -564,4 +564,12 @@ def test_step_host_matches_device_step(dp):
     assert np.allclose(hs.clip.numpy(), dev.clip.cpu().numpy(), rtol=1e-6)
     for l in range(len(layers)):
         assert rel_fro(hs.gW[l].numpy(), dev.gW[l].cpu().numpy()) <= 1e-6
+    # inputs packed into one pinned buffer (one copy per direction): same results
+    hp = dp.HostStep(host_layers, pack_inputs=True)
+    hp.run(w.C, w.sigma, 3, 0)
+    torch.cuda.synchronize()
+    assert np.array_equal(hp.clip.numpy(), hs.clip.numpy()) and np.array_equal(hp.norms.numpy(), hs.norms.numpy())
+    for l in range(len(layers)):
+        assert np.array_equal(hp.gW[l].numpy(), hs.gW[l].numpy())
+        assert np.array_equal(hp.gb[l].numpy(), hs.gb[l].numpy())
         assert rel_fro(hs.gb[l].numpy(), dev.gb[l].cpu().numpy()) <= 1e-6
