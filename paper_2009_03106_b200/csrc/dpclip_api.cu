@@ -508,6 +508,64 @@ int launch_fused_t1_tf32(const FusedT1Params& base, bool one_launch, void* works
     return launch_status();
 }
 
+// One T = 1 layer of the caller's model as the fused kernels see it.  Returns 0, 1 (the layer does not
+// qualify for the fused kernels) or a negative argument error.
+int fill_fused_t1_layer(FusedT1Layer& f, const dpclip_layer& y, int index, int B, dpclip_dtype dtype, int tile,
+                        int& tiles) {
+    if (y.T != 1 || y.ldg != y.d_in) return 1;
+    if (y.method != DPCLIP_AUTO && y.method != DPCLIP_T1) return 1;
+    int rc = check_layer_args(y.A, y.lda, y.Zbar, y.ldz, B, 1, y.d_in, y.d_out, dtype);
+    if (rc) return rc;
+    if (!y.gW || (y.has_bias && !y.gb)) return DPCLIP_ERR_INVALID_ARG;
+    if (!aligned_to(y.gW, 16) || (y.gb && !aligned_to(y.gb, 4))) return 1;
+    f.A = y.A; f.lda = y.lda; f.Z = y.Zbar; f.ldz = y.ldz;
+    f.d_in = y.d_in; f.d_out = y.d_out; f.has_bias = y.has_bias ? 1 : 0;
+    f.vec_a = vec4_ok(y.A, y.lda, dtype); f.vec_z = vec4_ok(y.Zbar, y.ldz, dtype);
+    f.gW = y.gW; f.gb = y.has_bias ? y.gb : nullptr;
+    f.tiles_m = ceil_div(y.d_out, tile); f.tiles_n = ceil_div(y.d_in + f.has_bias, tile);
+    f.tile_begin = tiles;
+    f.index = index;
+    tiles += f.tiles_m * f.tiles_n;
+    return 0;
+}
+
+// The T = 1 layers of a model that also has T > 1 layers (fp32): their norms in one launch (into their rows
+// of sq), and, once the factors of the whole model exist, their clipped sums with noise in one tensor-core
+// launch.  `group` lists the layers' positions in the model.  prepare returns 0 when the group qualifies.
+struct T1Group {
+    FusedT1Params p;
+    bool active = false;
+};
+
+int prepare_t1_group(T1Group& g, const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, float C, float sigma,
+                     unsigned long long seed, unsigned long long stream_id0, float* sq, float* clip) {
+    g.active = false;
+    if (dtype != DPCLIP_F32 || B > FUSED_MAX_B) return 0;
+    { const char* env = getenv("DPCLIP_NO_FUSED_T1"); if (env && env[0] == '1') return 0; }
+    { const char* env = getenv("DPCLIP_NO_T1_TF32"); if (env && env[0] == '1') return 0; }
+    memset(&g.p, 0, sizeof(g.p));
+    int n = 0, tiles = 0;
+    for (int l = 0; l < L; ++l) {
+        if (layers[l].T != 1) continue;
+        if (n == FUSED_MAX_LAYERS) return 0;
+        const int rc = fill_fused_t1_layer(g.p.layer[n], layers[l], l, B, dtype, 64, tiles);
+        if (rc < 0) return rc;
+        if (rc) return 0;
+        const FusedT1Layer& y = g.p.layer[n];
+        const bool a_ok = aligned_to(y.A, 16) && y.lda % 4 == 0;
+        const bool z_ok = aligned_to(y.Z, 16) && y.ldz % 4 == 0;
+        if (!a_ok || !(z_ok || y.d_out <= tc::f1::THIN_MAX_OUT)) return 0;
+        ++n;
+    }
+    if (n == 0 || n == L) return 0;
+    g.p.L = n; g.p.B = B; g.p.total_tiles = tiles;
+    g.p.C = C; g.p.noise_scale = sigma * C;
+    g.p.k0 = (uint32_t)seed; g.p.k1 = (uint32_t)(seed >> 32); g.p.stream_id0 = stream_id0;
+    g.p.sq = sq; g.p.clip = clip; g.p.norms = nullptr; g.p.clip_in = clip;
+    g.active = true;
+    return 0;
+}
+
 int try_fused_t1_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, float C, float sigma,
                       unsigned long long seed, unsigned long long stream_id0, float* sq, float* clip,
                       float* norms, void* workspace, size_t workspace_bytes, cudaStream_t st) {
@@ -516,28 +574,14 @@ int try_fused_t1_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dty
     if (env && env[0] == '1') return 1;
     FusedT1Params p;
     memset(&p, 0, sizeof(p));
-    // 64 x 64 tiles: several CTAs per SM hide the global-load latency of these short (K = B) products.
-    // The 128 x 128 variant (8 x 8 register tiles, one CTA per SM) measured slower at the MLP sizes
-    // (61 vs 39 us per step on the 784-1000-1000-10, B = 128 model) and is kept for experiments only.
-    int tile = 64;
-    { const char* env = getenv("DPCLIP_T1_TILE"); if (env && atoi(env) == 128) tile = 128; }
+    // fp32-ALU form: 64 x 64 tiles, several CTAs per SM hide the global-load latency of these short (K = B)
+    // products (128 x 128 register tiles, one CTA per SM, measured slower: 61 vs 39 us per step on the
+    // 784-1000-1000-10, B = 128 model).
+    const int tile = 64;
     int tiles = 0;
     for (int l = 0; l < L; ++l) {
-        const dpclip_layer& y = layers[l];
-        if (y.T != 1 || y.ldg != y.d_in) return 1;
-        if (y.method != DPCLIP_AUTO && y.method != DPCLIP_T1) return 1;
-        int rc = check_layer_args(y.A, y.lda, y.Zbar, y.ldz, B, 1, y.d_in, y.d_out, dtype);
+        const int rc = fill_fused_t1_layer(p.layer[l], layers[l], l, B, dtype, tile, tiles);
         if (rc) return rc;
-        if (!y.gW || (y.has_bias && !y.gb)) return DPCLIP_ERR_INVALID_ARG;
-        if (!aligned_to(y.gW, 16) || (y.gb && !aligned_to(y.gb, 4))) return 1;
-        FusedT1Layer& f = p.layer[l];
-        f.A = y.A; f.lda = y.lda; f.Z = y.Zbar; f.ldz = y.ldz;
-        f.d_in = y.d_in; f.d_out = y.d_out; f.has_bias = y.has_bias ? 1 : 0;
-        f.vec_a = vec4_ok(y.A, y.lda, dtype); f.vec_z = vec4_ok(y.Zbar, y.ldz, dtype);
-        f.gW = y.gW; f.gb = y.has_bias ? y.gb : nullptr;
-        f.tiles_m = ceil_div(y.d_out, tile); f.tiles_n = ceil_div(y.d_in + f.has_bias, tile);
-        f.tile_begin = tiles;
-        tiles += f.tiles_m * f.tiles_n;
     }
     p.L = L; p.B = B; p.total_tiles = tiles;
     p.C = C; p.noise_scale = sigma * C;
@@ -546,7 +590,7 @@ int try_fused_t1_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dty
     const int rows = L * B;
     const int grid_n = rows;
     const int grid_g = tiles < 4 * kNumSMs ? tiles : 4 * kNumSMs;
-    const int smem64 = FusedT1Cfg<64>::SMEM_BYTES, smem128 = FusedT1Cfg<128>::SMEM_BYTES;
+    const int smem64 = FusedT1Cfg<64>::SMEM_BYTES;
     if (dtype == DPCLIP_F32) {
         bool one = true;
         { const char* env = getenv("DPCLIP_T1_ONE_LAUNCH"); if (env && env[0] == '0') one = false; }
@@ -558,21 +602,11 @@ int try_fused_t1_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dty
         if (launch_status()) return DPCLIP_ERR_CUDA;
         const int rc = launch_fused_t1_tf32(p, false, workspace, workspace_bytes, st);
         if (rc <= 0) return rc;
-        if (tile == 128) {
-            if (!enable_smem(t1_all_grads_kernel<float, 128>, smem128)) return DPCLIP_ERR_CUDA;
-            t1_all_grads_kernel<float, 128><<<grid_g, SIMT_THREADS, smem128, st>>>(p);
-        } else {
-            t1_all_grads_kernel<float, 64><<<grid_g, SIMT_THREADS, smem64, st>>>(p);
-        }
+        t1_all_grads_kernel<float, 64><<<grid_g, SIMT_THREADS, smem64, st>>>(p);
     } else {
         t1_all_norms_kernel<__nv_bfloat16><<<grid_n, 128, 0, st>>>(p);
         if (launch_status()) return DPCLIP_ERR_CUDA;
-        if (tile == 128) {
-            if (!enable_smem(t1_all_grads_kernel<__nv_bfloat16, 128>, smem128)) return DPCLIP_ERR_CUDA;
-            t1_all_grads_kernel<__nv_bfloat16, 128><<<grid_g, SIMT_THREADS, smem128, st>>>(p);
-        } else {
-            t1_all_grads_kernel<__nv_bfloat16, 64><<<grid_g, SIMT_THREADS, smem64, st>>>(p);
-        }
+        t1_all_grads_kernel<__nv_bfloat16, 64><<<grid_g, SIMT_THREADS, smem64, st>>>(p);
     }
     return launch_status();
 }
@@ -806,8 +840,17 @@ int dpclip_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, fl
     int rc = try_fused_t1_step(layers, L, B, dtype, C, sigma, seed, stream_id0, sq_layers, clip, norms, workspace,
                                workspace_bytes, (cudaStream_t)stream);
     if (rc <= 0) return rc;                  // done (0) or argument error (< 0); 1 = take the general path
+    T1Group t1;
+    rc = prepare_t1_group(t1, layers, L, B, dtype, C, sigma, seed, stream_id0, sq_layers, clip);
+    if (rc) return rc;
+    if (t1.active && (!workspace || workspace_bytes < (size_t)kHeaderBytes)) t1.active = false;
+    if (t1.active) {
+        t1_all_norms_kernel<float><<<t1.p.L * B, 128, 0, (cudaStream_t)stream>>>(t1.p);
+        if (launch_status()) return DPCLIP_ERR_CUDA;
+    }
     for (int l = 0; l < L; ++l) {
         const dpclip_layer& y = layers[l];
+        if (t1.active && y.T == 1) continue;
         rc = dpclip_layer_sqnorms(y.A, y.lda, y.Zbar, y.ldz, B, y.T, y.d_in, y.d_out, dtype, y.has_bias,
                                   (dpclip_method)y.method, sq_layers + (size_t)l * B, workspace,
                                   workspace_bytes, stream);
@@ -815,8 +858,14 @@ int dpclip_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, fl
     }
     rc = dpclip_factors(sq_layers, L, B, B, C, clip, norms, nullptr, stream);
     if (rc) return rc;
+    if (t1.active) {
+        rc = launch_fused_t1_tf32(t1.p, false, workspace, workspace_bytes, (cudaStream_t)stream);
+        if (rc < 0) return rc;
+        if (rc > 0) return DPCLIP_ERR_UNSUPPORTED;           // prepare_t1_group checked the same conditions
+    }
     for (int l = 0; l < L; ++l) {
         const dpclip_layer& y = layers[l];
+        if (t1.active && y.T == 1) continue;
         float* gb = y.has_bias ? y.gb : nullptr;
         if (y.has_bias && !gb) return DPCLIP_ERR_INVALID_ARG;
         // noise indexes the dense d_out x d_in tensor, so the step wants unpadded output rows

@@ -29,6 +29,7 @@ struct FusedT1Layer {
     int vec_a, vec_z;
     float* gW; float* gb;          // dense rows (ldg == d_in)
     int tiles_m, tiles_n, tile_begin;
+    int index;                     // position of the layer in the caller's model: row of sq, noise stream ids
 };
 
 struct FusedT1Params {
@@ -38,6 +39,7 @@ struct FusedT1Params {
     uint32_t k0, k1;               // Philox key
     unsigned long long stream_id0;
     float* sq; float* clip; float* norms;
+    const float* clip_in;          // factors already known (T = 1 layers of a mixed model): sq is not summed
 };
 
 // one CTA of 128 threads per (layer, example): every thread has at most a few independent 128-bit
@@ -54,7 +56,7 @@ t1_all_norms_kernel(const __grid_constant__ FusedT1Params p) {
     float sz = row_sumsq(z, y.d_out, y.vec_z != 0);
     sa = block_sum(sa, red);
     sz = block_sum(sz, red);
-    if (threadIdx.x == 0) p.sq[(size_t)l * p.B + i] = (sa + (y.has_bias ? 1.f : 0.f)) * sz;
+    if (threadIdx.x == 0) p.sq[(size_t)y.index * p.B + i] = (sa + (y.has_bias ? 1.f : 0.f)) * sz;
 }
 
 // One row of four consecutive outputs (m, n .. n+3) of layer y: add the noise, store once.
@@ -62,7 +64,7 @@ t1_all_norms_kernel(const __grid_constant__ FusedT1Params p) {
 __device__ __forceinline__ void fused_t1_emit4(const FusedT1Params& p, const FusedT1Layer& y, int l, int m, int n,
                                                float (&out)[4]) {
     if (m >= y.d_out || n > y.d_in) return;
-    const unsigned long long sid_w = p.stream_id0 + 2ull * l, sid_b = sid_w + 1;
+    const unsigned long long sid_w = p.stream_id0 + 2ull * y.index, sid_b = sid_w + 1;
     const bool row4 = (y.d_in & 3) == 0 && n + 4 <= y.d_in;       // four in-range columns = one Philox block
     if (p.noise_scale > 0.f) {
         const size_t j0 = (size_t)m * y.d_in + n;
@@ -129,6 +131,7 @@ t1_all_grads_kernel(const __grid_constant__ FusedT1Params p) {
     const int tid = threadIdx.x;
     // factors, rebuilt by every CTA (cheaper than a third launch or a grid barrier)
     for (int i = tid; i < p.B; i += SIMT_THREADS) {
+        if (p.clip_in) { clip_s[i] = p.clip_in[i]; continue; }
         float s = 0.f;
         for (int l = 0; l < p.L; ++l) s += p.sq[(size_t)l * p.B + i];
         const float n = sqrtf(s);

@@ -187,6 +187,7 @@ t1_all_grads_tf32_kernel(const __grid_constant__ f1::Params q) {
     // factors, rebuilt by every CTA from the layer norms (L * B floats, L2-resident)
     if (!ONE_LAUNCH)
     for (int i = threadIdx.x; i < p.B; i += THREADS) {
+        if (p.clip_in) { clip_s[i] = p.clip_in[i]; continue; }
         float s = 0.f;
         for (int l = 0; l < p.L; ++l) s += p.sq[(size_t)l * p.B + i];
         const float n = sqrtf(s);

@@ -492,6 +492,13 @@ def test_step_mlp_tensor_core_edges(dp):
                             workloads.LayerSpec("fc4", 1, 16, 3, True, "relu")), 1.0, 0.9, 1.0 / 200)
     layers = workloads.generate(w, 5)
     _check_step(dp, w, _calibrate(w, layers, 5, w.C), w.C, w.sigma, 5)
+    # more output tiles (13 x 12 + 1 x 13 = 169) than SMs: every CTA of the one-launch kernel walks several
+    # items, so the stage ring, the two accumulator buffers and the noise drawing carry over between items
+    big = workloads.Workload("mlp_tc_many_tiles", 48, "f32",
+                             (workloads.LayerSpec("fc1", 1, 1536, 1664, True, "normal"),
+                              workloads.LayerSpec("fc2", 1, 1664, 12, True, "relu")), 1.0, 0.9, 1.0 / 48)
+    layers = workloads.generate(big, 6)
+    _check_step(dp, big, _calibrate(big, layers, 6, big.C), big.C, big.sigma, 6)
 
 
 def test_step_mlp_fp32_alu_kernel(dp, monkeypatch):
