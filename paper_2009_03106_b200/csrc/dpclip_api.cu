@@ -119,8 +119,12 @@ int launch_simt_norms(const void* A, long lda, const void* Z, long ldz, int B, i
     return launch_status();
 }
 
+struct NoiseSpec { float scale; unsigned long long seed, sid_w, sid_b; };
+
 int launch_simt_grad(const void* A, long lda, const void* Z, long ldz, int B, int T, int d_in, int d_out,
-                     dpclip_dtype dtype, const float* clip, float* gW, long ldg, float* gb, cudaStream_t st) {
+                     dpclip_dtype dtype, const float* clip, float* gW, long ldg, float* gb, cudaStream_t st,
+                     void* workspace = nullptr, size_t workspace_bytes = 0, const NoiseSpec* noise = nullptr,
+                     bool* noise_done = nullptr) {
     if (narrow_layer(T, d_in, d_out, gb != nullptr, lda, ldz)) {
         NarrowParams q;
         memset(&q, 0, sizeof(q));
@@ -132,6 +136,26 @@ int launch_simt_grad(const void* A, long lda, const void* Z, long ldz, int B, in
         if ((long)grid * min_rows > q.rows_total) grid = (int)((q.rows_total + min_rows - 1) / min_rows);
         q.rows_per_cta = (q.rows_total + grid - 1) / grid;
         grid = (int)((q.rows_total + q.rows_per_cta - 1) / q.rows_per_cta);
+        const int maxm = d_out <= 32 ? 32 : 64;
+        const size_t part_bytes = (size_t)grid * maxm * 32 * 4;
+        if (workspace && workspace_bytes >= (size_t)kHeaderBytes + part_bytes && grid > 1) {
+            // partial tile per CTA, then a fixed-order reduce that also adds the noise
+            q.part = reinterpret_cast<float*>(static_cast<char*>(workspace) + kHeaderBytes);
+            int rc = launch_narrow<true>(q, grid, d_out, dtype, st);
+            if (rc) return rc;
+            NarrowReduceParams r;
+            memset(&r, 0, sizeof(r));
+            r.part = q.part; r.n_parts = grid; r.maxm = maxm; r.d_out = d_out; r.d_in = d_in; r.has_bias = gb ? 1 : 0;
+            r.gW = gW; r.ldg = ldg; r.gb = gb;
+            if (noise && noise->scale > 0.f && ldg == d_in) {
+                r.noise_scale = noise->scale;
+                r.k0 = (uint32_t)noise->seed; r.k1 = (uint32_t)(noise->seed >> 32);
+                r.sid_w = noise->sid_w; r.sid_b = noise->sid_b;
+                if (noise_done) *noise_done = true;
+            }
+            narrow_reduce_kernel<<<d_out, 256, 0, st>>>(r);
+            return launch_status();
+        }
         if (cudaMemset2DAsync(gW, sizeof(float) * (size_t)ldg, 0, sizeof(float) * (size_t)d_in, d_out, st) !=
             cudaSuccess) return DPCLIP_ERR_CUDA;
         if (gb && cudaMemsetAsync(gb, 0, sizeof(float) * (size_t)d_out, st) != cudaSuccess) return DPCLIP_ERR_CUDA;
@@ -244,8 +268,6 @@ int launch_gram_norms(const void* A, long lda, const void* Z, long ldz, int B, i
     }
     return launch_status();
 }
-
-struct NoiseSpec { float scale; unsigned long long seed, sid_w, sid_b; };
 
 // Largest scratch the split-row clipped sum can ask for: one partial tile per item, at most one
 // wave of 256 x 256 tiles or two waves of 128 x 256 tiles, plus the partial bias sums.
@@ -450,7 +472,8 @@ int clipped_grad_impl(const void* A, long lda, const void* Zbar, long ldz, int B
     if (tf32_eligible(A, lda, Zbar, ldz, B, T, d_in, d_out, dtype) && !narrow_layer(T, d_in, d_out, gb != nullptr, lda, ldz))
         return launch_zta_tf32(A, lda, Zbar, ldz, B, T, d_in, d_out, false, 0, clip, gW, ldg, gb, nullptr, workspace,
                                workspace_bytes, noise, noise_done, st);
-    return launch_simt_grad(A, lda, Zbar, ldz, B, T, d_in, d_out, dtype, clip, gW, ldg, gb, st);
+    return launch_simt_grad(A, lda, Zbar, ldz, B, T, d_in, d_out, dtype, clip, gW, ldg, gb, st, workspace,
+                            workspace_bytes, noise, noise_done);
 }
 
 

@@ -15,10 +15,13 @@
 //
 //   NORM: one CTA per example; the tile is squared and summed -> sq[i].
 //   GRAD: one CTA per row slice, each row weighted by its example's clip factor
-//         (applied to a[row][n] as it is read); the tile is added to gW / gb
-//         with fp32 atomics.
+//         (applied to a[row][n] as it is read); the CTA's tile goes to a partial
+//         buffer and narrow_reduce_kernel sums the partials in a fixed order and
+//         adds the noise (148 CTAs adding onto the same thousand addresses with
+//         atomics serialise; without a workspace the atomics remain the fallback).
 #pragma once
 #include "common.cuh"
+#include "kernels_stream.cuh"
 
 namespace dpclip {
 
@@ -31,6 +34,7 @@ struct NarrowParams {
     long rows_total, rows_per_cta;      // GRAD
     const float* clip; float* gW; long ldg; float* gb;
     float* sq;                          // NORM
+    float* part;                        // GRAD: per-CTA partial tiles [grid][MAXM][32] instead of atomics (or NULL)
 };
 
 template <int MAXM> struct NarrowCfg {
@@ -167,7 +171,10 @@ narrow_kernel(NarrowParams p) {
         if (m < p.d_out) atomicAdd(&Gs[m][lane], G[m]);            // entries m >= d_out hold garbage: never used
     __syncthreads();
 
-    if (GRAD) {
+    if (GRAD && p.part) {
+        float* mine = p.part + (size_t)blockIdx.x * MAXM * 32;
+        for (int i = threadIdx.x; i < MAXM * 32; i += NARROW_THREADS) mine[i] = Gs[i >> 5][i & 31];
+    } else if (GRAD) {
         for (int i = threadIdx.x; i < p.d_out * 32; i += NARROW_THREADS) {
             const int m = i >> 5, n = i & 31;
             if (n < p.d_in) atomicAdd(p.gW + (size_t)m * p.ldg + n, Gs[m][n]);
@@ -182,6 +189,49 @@ narrow_kernel(NarrowParams p) {
         s = block_sum(s, red);
         if (threadIdx.x == 0) p.sq[blockIdx.x] = s;
     }
+}
+
+// Second stage of the narrow clipped sum: out[m][n] = sum over the CTAs' partial tiles, + noise.
+// One CTA per output row m: 32 columns x 8 groups of partials, combined through shared memory.
+struct NarrowReduceParams {
+    const float* part; int n_parts, maxm;
+    int d_out, d_in, has_bias;
+    float* gW; long ldg; float* gb;
+    float noise_scale; uint32_t k0, k1; unsigned long long sid_w, sid_b;
+};
+
+__global__ void __launch_bounds__(256)
+narrow_reduce_kernel(const NarrowReduceParams p) {
+    __shared__ float comb[8][32];
+    const int m = blockIdx.x, n = threadIdx.x & 31, g = threadIdx.x >> 5;
+    const size_t stride = (size_t)p.maxm * 32;
+    const float* src = p.part + (size_t)m * 32 + n;
+    float acc = 0.f;
+    int ks = g;
+    for (; ks + 24 < p.n_parts; ks += 32) {                          // four independent loads in flight
+        float v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) v[u] = __ldcs(src + (size_t)(ks + 8 * u) * stride);
+        acc += (v[0] + v[1]) + (v[2] + v[3]);
+    }
+    for (; ks < p.n_parts; ks += 8) acc += __ldcs(src + (size_t)ks * stride);
+    comb[g][n] = acc;
+    __syncthreads();
+    if (g != 0) return;
+#pragma unroll
+    for (int j = 1; j < 8; ++j) acc += comb[j][n];
+    const bool is_bias = n == p.d_in && p.has_bias;
+    if (n >= p.d_in && !is_bias) return;
+    if (p.noise_scale > 0.f) {
+        const size_t e = is_bias ? (size_t)m : (size_t)m * p.d_in + n;
+        const unsigned long long sid = is_bias ? p.sid_b : p.sid_w;
+        const size_t q = e >> 2;
+        PhiloxBlock b = philox_block((uint32_t)q, (uint32_t)(q >> 32), (uint32_t)sid, (uint32_t)(sid >> 32), p.k0, p.k1);
+        float za, zb;
+        box_muller(b.v[e & 2], b.v[(e & 2) + 1], za, zb);
+        acc = fmaf(p.noise_scale, (e & 1) ? zb : za, acc);
+    }
+    if (is_bias) p.gb[m] = acc; else p.gW[(size_t)m * p.ldg + n] = acc;
 }
 
 }  // namespace dpclip
