@@ -25,7 +25,11 @@
  *   - `stream` is a cudaStream_t passed as void* (NULL = legacy default stream).
  *     Calls only enqueue work; they never synchronise the stream.
  *   - The caller owns every buffer, including the workspace.  The library
- *     allocates no device memory and keeps no state between calls.
+ *     allocates no device memory and keeps no state between calls.  A
+ *     workspace holds scratch (partial tiles) and, in its header, a status
+ *     word and the grid-barrier counter of the one-launch T = 1 step: calls
+ *     that may run at the same time (different streams) need workspaces of
+ *     their own; calls ordered on one stream can share one.
  *   - Layout: A is B x T x d_in with row stride `lda` ELEMENTS (>= d_in), rows
  *     of one example contiguous (example i starts at row i*T); Zbar likewise
  *     with `ldz`.  Outputs are fp32; gW is d_out x d_in row-major with row
@@ -202,7 +206,11 @@ typedef struct {
  *   sq_layers  [L][B] fp32 scratch/outputs, clip [B], norms [B] or NULL
  *   workspace  >= the largest dpclip_workspace_bytes() over the layers
  * Output rows must be dense (ldg == d_in; UNSUPPORTED otherwise) because the
- * noise is indexed by the element's position in the dense tensor. */
+ * noise is indexed by the element's position in the dense tensor.
+ * A model whose layers all have T = 1 runs as ONE cooperative launch when it
+ * is fp32 with 16-byte-multiple input rows (norms, a grid-wide barrier with a
+ * bounded wait, factors, clipped sums on the tensor cores, noise), else as two
+ * launches; other models run layer by layer, their T = 1 layers together. */
 int dpclip_step(const dpclip_layer* layers /* host */, int L, int B, dpclip_dtype dtype,
                 float C, float sigma, unsigned long long seed, unsigned long long stream_id0,
                 float* sq_layers, float* clip, float* norms,
