@@ -134,7 +134,9 @@ int launch_simt_grad(const void* A, long lda, const void* Z, long ldz, int B, in
         int grid = kNumSMs;                                        // one wave: the kernel holds a whole SM
         const long min_rows = NARROW_WARPS * 32;                   // at least one chunk per warp
         if ((long)grid * min_rows > q.rows_total) grid = (int)((q.rows_total + min_rows - 1) / min_rows);
-        q.rows_per_cta = (q.rows_total + grid - 1) / grid;
+        // whole 32-row chunks per CTA: every chunk of a dense layer then starts on a 16-byte boundary whatever
+        // the row length, and takes the 128-bit load path (a slice starting mid-chunk falls back to scalar loads)
+        q.rows_per_cta = ((q.rows_total + grid - 1) / grid + 31) / 32 * 32;
         grid = (int)((q.rows_total + q.rows_per_cta - 1) / q.rows_per_cta);
         const int maxm = d_out <= 32 ? 32 : 64;
         const size_t part_bytes = (size_t)grid * maxm * 32 * 4;
