@@ -216,6 +216,22 @@ int dpclip_step(const dpclip_layer* layers /* host */, int L, int B, dpclip_dtyp
                 float* sq_layers, float* clip, float* norms,
                 void* workspace, size_t workspace_bytes, void* stream);
 
+/* The T = 1 layers of a descriptor array taken together (layers with T > 1 are skipped): their
+ * squared norms in one launch, written to THEIR rows of sq_layers [L][B]; and, given the factors
+ * of the whole model, their clipped sums with the noise (streams stream_id0 + 2l, + 2l + 1 for
+ * layer l of the array) in one tensor-core launch.  This is what dpclip_step does for the T = 1
+ * layers of a mixed model; the two calls let a caller that spreads the layers of a model over
+ * several streams do the same.  fp32 only, input rows 16-byte multiples (the zb rows of a layer
+ * with at most 16 outputs excepted), dense output rows: DPCLIP_ERR_UNSUPPORTED otherwise, and
+ * nothing is launched. */
+int dpclip_t1_layers_supported(const dpclip_layer* layers /* host */, int L, int B, dpclip_dtype dtype); /* 1 or 0 */
+int dpclip_t1_layers_sqnorms(const dpclip_layer* layers /* host */, int L, int B, dpclip_dtype dtype,
+                             float* sq_layers, void* stream);
+int dpclip_t1_layers_clipped_grad_noise(const dpclip_layer* layers /* host */, int L, int B, dpclip_dtype dtype,
+                                        const float* clip, float C, float sigma,
+                                        unsigned long long seed, unsigned long long stream_id0,
+                                        void* workspace, size_t workspace_bytes, void* stream);
+
 /* Same, for callers whose tensors live in HOST memory (pinned memory makes the
  * copies asynchronous).  `layers[l].A/Zbar/gW/gb` are HOST pointers with dense
  * rows (lda = d_in, ldz = d_out, ldg = d_in are required).  `arena` is a device

@@ -60,6 +60,13 @@ def load_library():
                                             _u64, _vp, _sz, _vp]
     L.dpclip_clipped_grad_noise.restype = _i
     L.dpclip_add_noise.argtypes = [_vp, _sz, _f, _f, _u64, _u64, _vp]
+    L.dpclip_t1_layers_supported.argtypes = [ctypes.POINTER(_CLayer), _i, _i, _i]
+    L.dpclip_t1_layers_supported.restype = _i
+    L.dpclip_t1_layers_sqnorms.argtypes = [ctypes.POINTER(_CLayer), _i, _i, _i, _vp, _vp]
+    L.dpclip_t1_layers_sqnorms.restype = _i
+    L.dpclip_t1_layers_clipped_grad_noise.argtypes = [ctypes.POINTER(_CLayer), _i, _i, _i, _vp, _f, _f, _u64, _u64,
+                                                      _vp, _sz, _vp]
+    L.dpclip_t1_layers_clipped_grad_noise.restype = _i
     L.dpclip_elementwise_sqnorms.argtypes = [_vp, _l, _vp, _l, _i, _i, _i, _i, _i, _vp, _vp]
     L.dpclip_elementwise_sqnorms.restype = _i
     L.dpclip_elementwise_clipped_grad.argtypes = [_vp, _l, _vp, _l, _i, _i, _i, _i, _vp, _vp, _vp, _vp]
@@ -342,21 +349,49 @@ class StepPlan:
                 for s in streams[1:]:
                     ev = torch.cuda.Event(); ev.record(s); main.wait_event(ev)
 
+            # the T = 1 layers of a mixed model go together (one launch per stage) when the library takes them
+            t1_together = any(y.A.shape[1] == 1 for y in self.layers) and dpclip_t1_layers_supported(self)
+            rest = [(l, y) for l, y in enumerate(self.layers) if not (t1_together and y.A.shape[1] == 1)]
+            last = streams[-1]
             fork()
-            for l, y in enumerate(self.layers):
-                b = l % branches
+            if t1_together:
+                with torch.cuda.stream(last):
+                    dpclip_t1_layers_sqnorms(self)
+            for k, (l, y) in enumerate(rest):
+                b = k % branches
                 with torch.cuda.stream(streams[b]):
                     dpclip_layer_sqnorms(y.A, y.Zbar, y.has_bias, self.sq_layers[l], self._branch_ws[b], y.method)
             join()
             dpclip_factors(self.sq_layers, C, self.clip, self.norms)
             fork()
-            for l, y in enumerate(self.layers):
-                b = l % branches
+            if t1_together:
+                with torch.cuda.stream(last):
+                    dpclip_t1_layers_clipped_grad_noise(self, C, sigma, seed, stream_id0, self._branch_ws[-1])
+            for k, (l, y) in enumerate(rest):
+                b = k % branches
                 with torch.cuda.stream(streams[b]):
                     dpclip_clipped_grad_noise(y.A, y.Zbar, self.clip, self.gW[l], self.gb[l], sigma, C, seed,
                                               stream_id0 + 2 * l, stream_id0 + 2 * l + 1, self._branch_ws[b])
             join()
         return graph
+
+
+def dpclip_t1_layers_sqnorms(plan: StepPlan, stream=None) -> None:
+    _check("dpclip_t1_layers_sqnorms", load_library().dpclip_t1_layers_sqnorms(
+        plan._c, plan.L, plan.B, plan.dtype_code, _ptr(plan.sq_layers), _stream(stream)))
+
+
+def dpclip_t1_layers_clipped_grad_noise(plan: StepPlan, C: float, sigma: float, seed: int, stream_id0: int = 0,
+                                        workspace: Optional[torch.Tensor] = None, stream=None) -> None:
+    ws = plan.workspace if workspace is None else workspace
+    _check("dpclip_t1_layers_clipped_grad_noise", load_library().dpclip_t1_layers_clipped_grad_noise(
+        plan._c, plan.L, plan.B, plan.dtype_code, _ptr(plan.clip), C, sigma, seed, stream_id0, _ptr(ws), ws.numel(),
+        _stream(stream)))
+
+
+def dpclip_t1_layers_supported(plan: StepPlan) -> bool:
+    """Whether the library takes the plan's T = 1 layers together (nothing is launched)."""
+    return bool(load_library().dpclip_t1_layers_supported(plan._c, plan.L, plan.B, plan.dtype_code))
 
 
 def dpclip_step(plan: StepPlan, C: float, sigma: float, seed: int, stream_id0: int = 0, stream=None) -> None:

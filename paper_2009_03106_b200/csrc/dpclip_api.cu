@@ -563,7 +563,8 @@ struct T1Group {
 };
 
 int prepare_t1_group(T1Group& g, const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, float C, float sigma,
-                     unsigned long long seed, unsigned long long stream_id0, float* sq, float* clip) {
+                     unsigned long long seed, unsigned long long stream_id0, float* sq, const float* clip,
+                     bool mixed_only = true) {
     g.active = false;
     if (dtype != DPCLIP_F32 || B > FUSED_MAX_B) return 0;
     { const char* env = getenv("DPCLIP_NO_FUSED_T1"); if (env && env[0] == '1') return 0; }
@@ -582,11 +583,11 @@ int prepare_t1_group(T1Group& g, const dpclip_layer* layers, int L, int B, dpcli
         if (!a_ok || !(z_ok || y.d_out <= tc::f1::THIN_MAX_OUT)) return 0;
         ++n;
     }
-    if (n == 0 || n == L) return 0;
+    if (n == 0 || (mixed_only && n == L)) return 0;
     g.p.L = n; g.p.B = B; g.p.total_tiles = tiles;
     g.p.C = C; g.p.noise_scale = sigma * C;
     g.p.k0 = (uint32_t)seed; g.p.k1 = (uint32_t)(seed >> 32); g.p.stream_id0 = stream_id0;
-    g.p.sq = sq; g.p.clip = clip; g.p.norms = nullptr; g.p.clip_in = clip;
+    g.p.sq = sq; g.p.clip = nullptr; g.p.norms = nullptr; g.p.clip_in = clip;
     g.active = true;
     return 0;
 }
@@ -793,6 +794,39 @@ int dpclip_clipped_grad_noise(const void* A, long lda, const void* Zbar, long ld
     rc = dpclip_add_noise(gW, (size_t)d_out * d_in, sigma, C, seed, stream_id_w, stream);
     if (rc || !gb) return rc;
     return dpclip_add_noise(gb, (size_t)d_out, sigma, C, seed, stream_id_b, stream);
+}
+
+int dpclip_t1_layers_supported(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype) {
+    if (!layers || L <= 0 || B <= 0) return 0;
+    T1Group g;
+    if (prepare_t1_group(g, layers, L, B, dtype, 1.f, 0.f, 0, 0, nullptr, nullptr, /*mixed_only=*/false)) return 0;
+    return g.active ? 1 : 0;
+}
+
+int dpclip_t1_layers_sqnorms(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, float* sq_layers,
+                             void* stream) {
+    if (!layers || L <= 0 || B <= 0 || !sq_layers) return DPCLIP_ERR_INVALID_ARG;
+    T1Group g;
+    int rc = prepare_t1_group(g, layers, L, B, dtype, 1.f, 0.f, 0, 0, sq_layers, nullptr, /*mixed_only=*/false);
+    if (rc) return rc;
+    if (!g.active) return DPCLIP_ERR_UNSUPPORTED;
+    t1_all_norms_kernel<float><<<g.p.L * B, 128, 0, (cudaStream_t)stream>>>(g.p);
+    return launch_status();
+}
+
+int dpclip_t1_layers_clipped_grad_noise(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype,
+                                        const float* clip, float C, float sigma, unsigned long long seed,
+                                        unsigned long long stream_id0, void* workspace, size_t workspace_bytes,
+                                        void* stream) {
+    if (!layers || L <= 0 || B <= 0 || !clip) return DPCLIP_ERR_INVALID_ARG;
+    if (!(C > 0.f) || !(sigma >= 0.f)) return DPCLIP_ERR_INVALID_ARG;
+    if (!workspace || workspace_bytes < (size_t)kHeaderBytes) return DPCLIP_ERR_WORKSPACE;
+    T1Group g;
+    int rc = prepare_t1_group(g, layers, L, B, dtype, C, sigma, seed, stream_id0, nullptr, clip, /*mixed_only=*/false);
+    if (rc) return rc;
+    if (!g.active) return DPCLIP_ERR_UNSUPPORTED;
+    rc = launch_fused_t1_tf32(g.p, false, workspace, workspace_bytes, (cudaStream_t)stream);
+    return rc > 0 ? DPCLIP_ERR_UNSUPPORTED : rc;
 }
 
 int dpclip_elementwise_sqnorms(const void* Hbar, long ldh, const void* Zbar, long ldz, int B, int T, int d,
