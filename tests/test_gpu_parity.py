@@ -542,6 +542,35 @@ def test_step_seq_small(dp):
     _check_step(dp, w, _calibrate(w, layers, 2, w.C), w.C, w.sigma, 2)
 
 
+def test_per_layer_clipping_through_the_same_entry_points(dp):
+    """Per-layer clipping (each layer's gradient clipped to C / sqrt(L) on its own, the variant the paper's
+    per-layer norms make possible): the rows of sq stay separate, so it is dpclip_factors on one row at a
+    time and a clipped sum per layer with that layer's factors."""
+    w = workloads.seq("bf16", B=6, T=24, d=64, d_ff=136)
+    layers = workloads.generate(w, 8)
+    L, C = len(layers), 0.05
+    Cl = C / np.sqrt(L)
+    ws = _ws(dp)
+    total_sq = np.zeros(w.B)
+    for (A, Z), spec in zip(layers, w.layers):
+        sq_ref = oracle.layer_sqnorms(A, Z, spec.has_bias)
+        n_ref, c_ref = oracle.factors(sq_ref[None, :], Cl)
+        gW_ref, gb_ref = oracle.clipped_grad(A, Z, c_ref)
+        dA, dZ = to_device(A, "bf16"), to_device(Z, "bf16")
+        sq = torch.empty(1, w.B, device="cuda"); clip = torch.empty(w.B, device="cuda")
+        dp.dpclip_layer_sqnorms(dA, dZ, spec.has_bias, sq[0], ws)
+        dp.dpclip_factors(sq, Cl, clip)
+        check_saturation(clip.cpu().numpy(), n_ref, c_ref, Cl)
+        gW = torch.empty(spec.d_out, spec.d_in, device="cuda")
+        gb = torch.empty(spec.d_out, device="cuda") if spec.has_bias else None
+        dp.dpclip_clipped_grad(dA, dZ, clip, gW, gb, ws)
+        assert rel_fro(gW.cpu().numpy(), gW_ref) <= TOL["bf16"]["grad"]
+        total_sq += (c_ref ** 2) * sq_ref
+    # every example's clipped gradient over all layers is then within C
+    assert np.all(np.sqrt(total_sq) <= C * (1 + 1e-6))
+    assert dp.dpclip_read_status(ws) == 0
+
+
 def test_sharded_step_single_rank_equals_step(dp):
     """The data-parallel wrapper on one rank (no process group): whole-step call without noise, then the
     noise launches, must give what one dpclip_step call gives."""
