@@ -450,33 +450,44 @@ def run_sweep(args):
     rows = []
     print(f"{'B':>5} {'T':>5} {'d_in':>5} {'d_out':>5} | {'gram us':>9} {'mat us':>9} {'faster':>7} {'flop rule':>9} "
           f"{'auto':>6} | {'clipped sum us':>14} {'TFLOP/s':>8}")
-    for B in (256, 1024):
-        for T in (16, 128, 512, 2048):
-            for d_in, d_out in ((1024, 1024), (1024, 4096), (4096, 1024)):
-                if 2 * B * T * (d_in + d_out) > 12e9:
-                    continue                                                    # keep the device footprint bounded
-                g = torch.Generator(device="cuda").manual_seed(B * 7919 + T)
-                A = torch.randn(B, T, d_in, device="cuda", generator=g).to(torch.bfloat16)
-                Z = (torch.randn(B, T, d_out, device="cuda", generator=g) * (B * T) ** -0.5).to(torch.bfloat16)
-                sq = torch.empty(B, device="cuda"); clip = torch.rand(B, device="cuda", generator=g) * 0.9 + 0.1
-                gW = torch.empty(d_out, d_in, device="cuda"); gb = torch.empty(d_out, device="cuda")
-                n = max(3, min(args.steps, 10))
-                t = {}
-                for name, m in (("gram", dp.DPCLIP_GRAM), ("mat", dp.DPCLIP_MATERIALIZE)):
-                    t[name] = float(np.median(time_steps(torch, lambda: dp.dpclip_layer_sqnorms(A, Z, True, sq, ws, m), n, 3, flush)))
-                t["grad"] = float(np.median(time_steps(torch, lambda: dp.dpclip_clipped_grad(A, Z, clip, gW, gb, ws), n, 3, flush)))
-                assert dp.dpclip_read_status(ws) == 0
-                rule = "gram" if T * (T + 1) * (d_in + d_out) <= 2 * T * d_in * d_out else "mat"
-                auto = {dp.DPCLIP_GRAM: "gram", dp.DPCLIP_MATERIALIZE: "mat"}.get(
-                    dp.dpclip_pick_method(B, T, d_in, d_out, d_in, d_out, dp.DPCLIP_BF16), "other")
-                tf = 2.0 * B * T * d_in * d_out / (t["grad"] * 1e-3) / 1e12
-                rows.append(dict(B=B, T=T, d_in=d_in, d_out=d_out, gram_ms=t["gram"], materialize_ms=t["mat"],
-                                 faster="gram" if t["gram"] <= t["mat"] else "mat", flop_rule=rule, auto=auto,
-                                 clipped_sum_ms=t["grad"], clipped_sum_tflops=tf))
-                print(f"{B:5d} {T:5d} {d_in:5d} {d_out:5d} | {t['gram'] * 1e3:9.1f} {t['mat'] * 1e3:9.1f} {rows[-1]['faster']:>7} "
-                      f"{rule:>9} {auto:>6} | {t['grad'] * 1e3:14.1f} {tf:8.0f}", flush=True)
-                del A, Z
-    print(json.dumps(dict(sweep="norm_method_crossover", dtype="bf16", peaks=peaks, points=rows)))
+    if args.points:
+        grid_points = [tuple(int(v) for v in pt.split(",")) for pt in args.points.split(";") if pt]
+    else:
+        grid_points = [(B, T, d_in, d_out) for B in (256, 1024) for T in (16, 128, 512, 2048)
+                       for d_in, d_out in ((1024, 1024), (1024, 4096), (4096, 1024))]
+    for B, T, d_in, d_out in grid_points:
+        if 2 * B * T * (d_in + d_out) > 12e9:
+            continue                                                    # keep the device footprint bounded
+        g = torch.Generator(device="cuda").manual_seed(B * 7919 + T)
+        A = torch.randn(B, T, d_in, device="cuda", generator=g).to(torch.bfloat16)
+        Z = (torch.randn(B, T, d_out, device="cuda", generator=g) * (B * T) ** -0.5).to(torch.bfloat16)
+        sq = torch.empty(B, device="cuda"); clip = torch.rand(B, device="cuda", generator=g) * 0.9 + 0.1
+        gW = torch.empty(d_out, d_in, device="cuda"); gb = torch.empty(d_out, device="cuda")
+        n = max(3, min(args.steps, 10))
+        t = {}
+        for name, m in (("gram", dp.DPCLIP_GRAM), ("mat", dp.DPCLIP_MATERIALIZE)):
+            t[name] = float(np.median(time_steps(torch, lambda: dp.dpclip_layer_sqnorms(A, Z, True, sq, ws, m), n, 3, flush)))
+        t["grad"] = float(np.median(time_steps(torch, lambda: dp.dpclip_clipped_grad(A, Z, clip, gW, gb, ws), n, 3, flush)))
+        assert dp.dpclip_read_status(ws) == 0
+        rule = "gram" if T * (T + 1) * (d_in + d_out) <= 2 * T * d_in * d_out else "mat"
+        auto = {dp.DPCLIP_GRAM: "gram", dp.DPCLIP_MATERIALIZE: "mat"}.get(
+            dp.dpclip_pick_method(B, T, d_in, d_out, d_in, d_out, dp.DPCLIP_BF16), "other")
+        tf = 2.0 * B * T * d_in * d_out / (t["grad"] * 1e-3) / 1e12
+        rows.append(dict(B=B, T=T, d_in=d_in, d_out=d_out, gram_ms=t["gram"], materialize_ms=t["mat"],
+                         faster="gram" if t["gram"] <= t["mat"] else "mat", flop_rule=rule, auto=auto,
+                         clipped_sum_ms=t["grad"], clipped_sum_tflops=tf))
+        print(f"{B:5d} {T:5d} {d_in:5d} {d_out:5d} | {t['gram'] * 1e3:9.1f} {t['mat'] * 1e3:9.1f} {rows[-1]['faster']:>7} "
+              f"{rule:>9} {auto:>6} | {t['grad'] * 1e3:14.1f} {tf:8.0f}", flush=True)
+        del A, Z
+    noise = None
+    if args.noise_n:
+        # the noise kernel alone at a size where it is bandwidth-bound (8 bytes per element: read + write)
+        g = torch.zeros(args.noise_n, device="cuda")
+        ms = float(np.median(time_steps(torch, lambda: dp.dpclip_add_noise(g, 1.0, 1.0, 1, 0), 5, 3, flush)))
+        noise = dict(n=args.noise_n, ms=ms, gbs=8.0 * args.noise_n / (ms * 1e-3) / 1e9)
+        print(f"noise n={args.noise_n}: {ms * 1e3:.1f} us  {noise['gbs']:.0f} GB/s "
+              f"({noise['gbs'] / peaks['hbm_gbs']:.2f} of the {peaks['source']} copy bandwidth)")
+    print(json.dumps(dict(sweep="norm_method_crossover", dtype="bf16", peaks=peaks, points=rows, noise=noise)))
 
 
 # ---------------------------------------------------------------------------
@@ -490,6 +501,8 @@ def main():
     ap.add_argument("--others", default="cfg1,cfg3_f32,cfg3_bf16,cfg4",
                     help="further workloads reported under 'workloads' (N=1 only; '' for none)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--points", default="", help="with --sweep: only these points, 'B,T,d_in,d_out;B,T,d_in,d_out;...'")
+    ap.add_argument("--noise-n", type=int, default=0, help="with --sweep: also time dpclip_add_noise on this many elements")
     ap.add_argument("--sweep", action="store_true",
                     help="instead of the benchmark line: Gram-vs-materialise sweep of the T > 1 norm (1 GPU)")
     args = ap.parse_args()
