@@ -281,10 +281,18 @@ def roofline_for(w, breakdown, peaks):
     nbytes, flops = layer_work(w, spec, kind)
     ms = breakdown[key]
     t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9)
-    # bf16 layers whose rows are 16-byte multiples run on the tcgen05 kernels
-    tc_layer = w.dtype == "bf16" and spec.d_in % 8 == 0 and spec.d_out % 8 == 0
-    on_tensor = kind in ("norm_gram", "norm_mat") or (kind == "grad" and tc_layer)
-    alu_peak = (peaks["bf16_tflops"] if on_tensor else FFMA_PEAK_TFLOPS) * 1e12
+    # bf16 layers whose rows are 16-byte multiples run on the tcgen05 kernels; so do fp32 layers above 2^25
+    # multiply-adds whose rows are 16-byte multiples (three tf32 MMAs per product), unless they are narrow
+    # enough for the streaming kernel
+    narrow = spec.T > 1 and spec.d_in + (1 if spec.has_bias else 0) <= 32 and spec.d_out <= 64
+    tc_bf16 = w.dtype == "bf16" and spec.d_in % 8 == 0 and spec.d_out % 8 == 0
+    tc_f32 = (w.dtype == "f32" and spec.d_in % 4 == 0 and spec.d_out % 4 == 0 and not narrow and
+              float(w.B) * spec.T * spec.d_in * spec.d_out >= 2 ** 25)
+    on_tensor = (kind in ("norm_gram", "norm_mat") or (kind == "grad" and (tc_bf16 or tc_f32))) and not narrow
+    if on_tensor and w.dtype == "f32":
+        alu_peak = peaks["bf16_tflops"] * TF32X3_PER_BF16 * 1e12
+    else:
+        alu_peak = (peaks["bf16_tflops"] if on_tensor else FFMA_PEAK_TFLOPS) * 1e12
     t_alu = flops / alu_peak
     total = sum(breakdown.values())
     if t_hbm >= t_alu:
