@@ -216,6 +216,13 @@ int dpclip_step(const dpclip_layer* layers /* host */, int L, int B, dpclip_dtyp
                 float* sq_layers, float* clip, float* norms,
                 void* workspace, size_t workspace_bytes, void* stream);
 
+/* Noise on every released tensor of a model in one launch: weights of layer l on noise stream
+ * stream_id0 + 2l, its bias on + 2l + 1, exactly as dpclip_step numbers them (dense output rows
+ * required).  For callers that add the noise after their own reduction over ranks.
+ * sigma * C == 0 launches nothing. */
+int dpclip_step_noise(const dpclip_layer* layers /* host */, int L, float C, float sigma,
+                      unsigned long long seed, unsigned long long stream_id0, void* stream);
+
 /* The T = 1 layers of a descriptor array taken together (layers with T > 1 are skipped): their
  * squared norms in one launch, written to THEIR rows of sq_layers [L][B]; and, given the factors
  * of the whole model, their clipped sums with the noise (streams stream_id0 + 2l, + 2l + 1 for

@@ -60,6 +60,8 @@ def load_library():
                                             _u64, _vp, _sz, _vp]
     L.dpclip_clipped_grad_noise.restype = _i
     L.dpclip_add_noise.argtypes = [_vp, _sz, _f, _f, _u64, _u64, _vp]
+    L.dpclip_step_noise.argtypes = [ctypes.POINTER(_CLayer), _i, _f, _f, _u64, _u64, _vp]
+    L.dpclip_step_noise.restype = _i
     L.dpclip_t1_layers_supported.argtypes = [ctypes.POINTER(_CLayer), _i, _i, _i]
     L.dpclip_t1_layers_supported.restype = _i
     L.dpclip_t1_layers_sqnorms.argtypes = [ctypes.POINTER(_CLayer), _i, _i, _i, _vp, _vp]
@@ -374,6 +376,11 @@ class StepPlan:
                                               stream_id0 + 2 * l, stream_id0 + 2 * l + 1, self._branch_ws[b])
             join()
         return graph
+
+
+def dpclip_step_noise(plan: StepPlan, C: float, sigma: float, seed: int, stream_id0: int = 0, stream=None) -> None:
+    _check("dpclip_step_noise", load_library().dpclip_step_noise(plan._c, plan.L, C, sigma, seed, stream_id0,
+                                                                 _stream(stream)))
 
 
 def dpclip_t1_layers_sqnorms(plan: StepPlan, stream=None) -> None:

@@ -796,6 +796,40 @@ int dpclip_clipped_grad_noise(const void* A, long lda, const void* Zbar, long ld
     return dpclip_add_noise(gb, (size_t)d_out, sigma, C, seed, stream_id_b, stream);
 }
 
+int dpclip_step_noise(const dpclip_layer* layers, int L, float C, float sigma, unsigned long long seed,
+                      unsigned long long stream_id0, void* stream) {
+    if (!layers || L <= 0 || !(C >= 0.f) || !(sigma >= 0.f)) return DPCLIP_ERR_INVALID_ARG;
+    if (sigma * C == 0.f) return DPCLIP_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    for (int l0 = 0; l0 < L; l0 += NOISE_BATCH_MAX / 2) {          // at most 64 layers (128 tensors) per launch
+        NoiseBatchParams p;
+        memset(&p, 0, sizeof(p));
+        p.scale = sigma * C; p.k0 = (uint32_t)seed; p.k1 = (uint32_t)(seed >> 32);
+        int blocks = 0;
+        const int l1 = l0 + NOISE_BATCH_MAX / 2 < L ? l0 + NOISE_BATCH_MAX / 2 : L;
+        for (int l = l0; l < l1; ++l) {
+            const dpclip_layer& y = layers[l];
+            if (!y.gW || y.d_in <= 0 || y.d_out <= 0) return DPCLIP_ERR_INVALID_ARG;
+            if (y.ldg != y.d_in) return DPCLIP_ERR_UNSUPPORTED;      // noise indexes the dense tensor
+            if (y.has_bias && !y.gb) return DPCLIP_ERR_INVALID_ARG;
+            if (!aligned_to(y.gW, 4) || (y.gb && !aligned_to(y.gb, 4))) return DPCLIP_ERR_MISALIGNED;
+            auto add = [&](float* g, size_t n, unsigned long long sid) {
+                const size_t nq = (n + 3) / 4;
+                size_t b = (nq + 255) / 256;
+                if (b > (size_t)kNumSMs * 4) b = (size_t)kNumSMs * 4;
+                p.g[p.count] = g; p.n[p.count] = n; p.sid[p.count] = sid; p.blk_begin[p.count] = blocks;
+                blocks += (int)b; ++p.count;
+            };
+            add(y.gW, (size_t)y.d_out * y.d_in, stream_id0 + 2ull * l);
+            if (y.has_bias) add(y.gb, (size_t)y.d_out, stream_id0 + 2ull * l + 1);
+        }
+        p.blk_begin[p.count] = blocks;
+        noise_batch_kernel<<<blocks, 256, 0, st>>>(p);
+        if (launch_status()) return DPCLIP_ERR_CUDA;
+    }
+    return DPCLIP_OK;
+}
+
 int dpclip_t1_layers_supported(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype) {
     if (!layers || L <= 0 || B <= 0) return 0;
     T1Group g;

@@ -147,4 +147,44 @@ noise_kernel(float* __restrict__ g, size_t n, float scale, uint32_t k0, uint32_t
     }
 }
 
+// Noise on every released tensor of a model in ONE launch (the weights and the bias of layer l are
+// tensors 2l and 2l + 1, with their own noise streams).  Blocks are dealt to tensors by a prefix table.
+constexpr int NOISE_BATCH_MAX = 128;
+struct NoiseBatchParams {
+    float* g[NOISE_BATCH_MAX];
+    unsigned long long n[NOISE_BATCH_MAX];
+    unsigned long long sid[NOISE_BATCH_MAX];
+    int blk_begin[NOISE_BATCH_MAX + 1];          // first block of tensor k; blk_begin[count] = grid size
+    int count;
+    float scale; uint32_t k0, k1;
+};
+
+__global__ void __launch_bounds__(256)
+noise_batch_kernel(const __grid_constant__ NoiseBatchParams p) {
+    int k = 0;
+    while (k + 1 < p.count && (int)blockIdx.x >= p.blk_begin[k + 1]) ++k;
+    float* __restrict__ g = p.g[k];
+    const size_t n = p.n[k], nq = (n + 3) >> 2;
+    const uint32_t s0 = (uint32_t)p.sid[k], s1 = (uint32_t)(p.sid[k] >> 32);
+    const bool vec_ok = (reinterpret_cast<uintptr_t>(g) & 15) == 0;
+    const size_t stride = (size_t)(p.blk_begin[k + 1] - p.blk_begin[k]) * blockDim.x;
+    for (size_t q = (size_t)(blockIdx.x - p.blk_begin[k]) * blockDim.x + threadIdx.x; q < nq; q += stride) {
+        PhiloxBlock b = philox_block((uint32_t)q, (uint32_t)(q >> 32), s0, s1, p.k0, p.k1);
+        float z[4];
+        box_muller(b.v[0], b.v[1], z[0], z[1]);
+        box_muller(b.v[2], b.v[3], z[2], z[3]);
+        const size_t j = q << 2;
+        if (vec_ok && j + 3 < n) {
+            float4 v = *reinterpret_cast<float4*>(g + j);
+            v.x = fmaf(p.scale, z[0], v.x); v.y = fmaf(p.scale, z[1], v.y);
+            v.z = fmaf(p.scale, z[2], v.z); v.w = fmaf(p.scale, z[3], v.w);
+            *reinterpret_cast<float4*>(g + j) = v;
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                if (j + e < n) g[j + e] = fmaf(p.scale, z[e], g[j + e]);
+        }
+    }
+}
+
 }  // namespace dpclip

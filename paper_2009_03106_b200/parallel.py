@@ -32,6 +32,10 @@ def sharded_step(plan, C: float, sigma: float, seed: int, stream_id0: int = 0, g
             ops.dpclip_clipped_grad(y.A, y.Zbar, plan.clip, plan.gW[l], plan.gb[l], plan.workspace)
     if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
         dist.all_reduce(plan.flat, op=dist.ReduceOp.SUM, group=group)
+    all_noise = getattr(ops, "dpclip_step_noise", None)
+    if all_noise is not None:
+        all_noise(plan, C, sigma, seed, stream_id0)               # every tensor's noise in one launch
+        return
     for l in range(len(plan.layers)):
         ops.dpclip_add_noise(plan.gW[l].view(-1), sigma, C, seed, stream_id0 + 2 * l)
         if plan.gb[l] is not None:

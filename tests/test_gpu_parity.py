@@ -358,6 +358,23 @@ def test_noise_matches_oracle(dp, n):
     assert buf[0].item() == 0.0
 
 
+def test_step_noise_equals_per_tensor_noise(dp):
+    """One launch for all tensors of a model gives bit for bit what one dpclip_add_noise call per tensor gives."""
+    w = workloads.cnn("f32")
+    layers = workloads.generate(w, 0, examples=2)
+    mk = lambda: dp.StepPlan([dp.Layer(to_device(A, "f32"), to_device(Z, "f32"), s.has_bias)     # noqa: E731
+                              for (A, Z), s in zip(layers, w.layers)])
+    a, b = mk(), mk()
+    dp.dpclip_step_noise(a, 0.7, 1.3, 99, 6)
+    for l in range(len(layers)):
+        dp.dpclip_add_noise(b.gW[l].view(-1), 1.3, 0.7, 99, 6 + 2 * l)
+        dp.dpclip_add_noise(b.gb[l], 1.3, 0.7, 99, 6 + 2 * l + 1)
+    torch.cuda.synchronize()
+    for l in range(len(layers)):
+        assert torch.equal(a.gW[l], b.gW[l]) and torch.equal(a.gb[l], b.gb[l])
+        assert float(a.gW[l].abs().max()) > 0
+
+
 def test_noise_is_stateless_and_stream_dependent(dp):
     n = 10007
     a = torch.zeros(n, device="cuda"); b = torch.zeros(n, device="cuda"); c = torch.zeros(n, device="cuda")
