@@ -86,8 +86,34 @@ int launch_narrow_inst(const NarrowParams& p, int grid, cudaStream_t st) {
     return launch_status();
 }
 
+template <int MAXM, int WARPS, bool GRAD>
+int launch_narrow_ring_inst(const NarrowParams& p, int grid, cudaStream_t st) {
+    constexpr int smem = NarrowRingCfg<MAXM, WARPS>::SMEM_BYTES;
+    if (cudaFuncSetAttribute(narrow_ring_kernel<MAXM, WARPS, GRAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
+        cudaSuccess) return DPCLIP_ERR_CUDA;
+    narrow_ring_kernel<MAXM, WARPS, GRAD><<<grid, 32 * WARPS, smem, st>>>(p);
+    return launch_status();
+}
+
+// fp32 with every 16-row chunk starting on a 16-byte boundary (in A and in Zb): the cp.async ring form
+inline bool narrow_ring_ok(const NarrowParams& p, dpclip_dtype dtype, bool grad) {
+    const char* env = getenv("DPCLIP_NO_NARROW_RING");
+    if (env && env[0] == '1') return false;
+    if (dtype != DPCLIP_F32 || !aligned_to(p.A, 16) || !aligned_to(p.Z, 16)) return false;
+    // chunk starts are multiples of 16 rows from the slice start: 16 * d * 4 bytes is always a multiple of 16;
+    // the slice start itself is a multiple of 32 rows (GRAD) or of T rows (NORM)
+    if (!grad && (((long)p.T * p.d_in) % 4 != 0 || ((long)p.T * p.d_out) % 4 != 0)) return false;
+    return true;
+}
+
 template <bool GRAD>
 int launch_narrow(const NarrowParams& p, int grid, int d_out, dpclip_dtype dtype, cudaStream_t st) {
+    if (narrow_ring_ok(p, dtype, GRAD)) {
+        // two 8-warp CTAs per SM when there are CTAs enough for that, else one 16-warp CTA
+        if (grid > kNumSMs)
+            return d_out <= 32 ? launch_narrow_ring_inst<32, 8, GRAD>(p, grid, st) : launch_narrow_ring_inst<64, 8, GRAD>(p, grid, st);
+        return d_out <= 32 ? launch_narrow_ring_inst<32, 16, GRAD>(p, grid, st) : launch_narrow_ring_inst<64, 16, GRAD>(p, grid, st);
+    }
     if (dtype == DPCLIP_F32)
         return d_out <= 32 ? launch_narrow_inst<float, 32, GRAD>(p, grid, st) : launch_narrow_inst<float, 64, GRAD>(p, grid, st);
     return d_out <= 32 ? launch_narrow_inst<__nv_bfloat16, 32, GRAD>(p, grid, st)
@@ -131,7 +157,8 @@ int launch_simt_grad(const void* A, long lda, const void* Z, long ldz, int B, in
         q.A = A; q.lda = lda; q.Z = Z; q.ldz = ldz; q.T = T; q.d_in = d_in; q.d_out = d_out;
         q.has_bias = gb ? 1 : 0; q.clip = clip; q.gW = gW; q.ldg = ldg; q.gb = gb;
         q.rows_total = (long)B * T;
-        int grid = kNumSMs;                                        // one wave: the kernel holds a whole SM
+        // one wave: a CTA of the register-staged kernel holds a whole SM; the cp.async form runs two per SM
+        int grid = narrow_ring_ok(q, dtype, true) ? 2 * kNumSMs : kNumSMs;
         const long min_rows = NARROW_WARPS * 32;                   // at least one chunk per warp
         if ((long)grid * min_rows > q.rows_total) grid = (int)((q.rows_total + min_rows - 1) / min_rows);
         // whole 32-row chunks per CTA: every chunk of a dense layer then starts on a 16-byte boundary whatever

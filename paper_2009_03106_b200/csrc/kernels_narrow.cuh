@@ -191,6 +191,178 @@ narrow_kernel(NarrowParams p) {
     }
 }
 
+// ---------------------------------------------------------------------------
+// fp32 inputs whose chunks start on 16-byte boundaries: the same computation with the chunks copied
+// by cp.async straight into a per-warp ring of shared-memory slots (16 rows per chunk, three slots;
+// two when d_out > 32).  No staging registers, so several chunks per warp are in flight from the
+// first instruction on and the inner loop has registers to keep two rows' operands outstanding (the
+// register-staged kernel above stalls on its shared-memory loads for lack of them).
+// ---------------------------------------------------------------------------
+template <int MAXM, int WARPS_> struct NarrowRingCfg {
+    static constexpr int CH = 16;
+    // 8 warps: half an SM's shared memory, two CTAs per SM (one computes while the other starts up or winds
+    // down); 16 warps: one CTA per SM, for launches with fewer CTAs than SMs (one example per CTA, small B)
+    static constexpr int WARPS = WARPS_, THREADS = 32 * WARPS;
+    static constexpr int SLOTS = MAXM == 32 ? 3 : 2;
+    static constexpr int A_FLOATS = CH * 32, Z_FLOATS = CH * MAXM + 64;      // + slack for reads past short rows
+    static constexpr int SLOT_FLOATS = A_FLOATS + Z_FLOATS;
+    static constexpr int SMEM_BYTES = WARPS * SLOTS * SLOT_FLOATS * 4 + MAXM * 33 * 4 + 128;
+};
+
+__device__ __forceinline__ void cp_async_16(float* smem_dst, const float* gmem_src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)),
+                 "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// n floats (n % 4 == 0 is copied by cp.async; a remainder of up to 3 floats by plain loads)
+__device__ __forceinline__ void ring_issue(float* dst, const float* __restrict__ src, int n, int lane) {
+    const int nv = n >> 2;
+    for (int v = lane; v < nv; v += 32) cp_async_16(dst + 4 * v, src + 4 * v);
+    if (lane < (n & 3)) dst[(nv << 2) + lane] = src[(nv << 2) + lane];
+}
+
+template <int MAXM, int WARPS, bool GRAD>
+__global__ void __launch_bounds__(32 * WARPS, 16 / WARPS)
+narrow_ring_kernel(NarrowParams p) {
+    using Cfg = NarrowRingCfg<MAXM, WARPS>;
+    constexpr int CH = Cfg::CH, SLOTS = Cfg::SLOTS;
+    extern __shared__ __align__(16) float narrow_smem[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    float* ring = narrow_smem + warp * SLOTS * Cfg::SLOT_FLOATS;
+    float (*Gs)[33] = reinterpret_cast<float (*)[33]>(narrow_smem + Cfg::WARPS * SLOTS * Cfg::SLOT_FLOATS);
+    __shared__ float red[32];
+
+    const float* __restrict__ A = static_cast<const float*>(p.A);
+    const float* __restrict__ Z = static_cast<const float*>(p.Z);
+    long r0, r1;
+    if (GRAD) { r0 = (long)blockIdx.x * p.rows_per_cta; r1 = min(r0 + p.rows_per_cta, p.rows_total); }
+    else { r0 = (long)blockIdx.x * p.T; r1 = r0 + p.T; }
+
+    const long stride = (long)Cfg::WARPS * CH;
+    const long first = r0 + (long)warp * CH;
+    auto rows_of = [&](long b) { return b < r1 ? (int)min((long)CH, r1 - b) : 0; };
+    auto issue = [&](long b, int slot) {
+        const int nr = rows_of(b);
+        if (nr > 0) {
+            float* dst = ring + slot * Cfg::SLOT_FLOATS;
+            ring_issue(dst, A + (size_t)b * p.lda, nr * p.d_in, lane);
+            ring_issue(dst + Cfg::A_FLOATS, Z + (size_t)b * p.ldz, nr * p.d_out, lane);
+        }
+        cp_async_commit();                                        // one group per chunk, empty or not
+    };
+#pragma unroll
+    for (int s = 0; s < SLOTS; ++s) issue(first + s * stride, s);
+
+    for (int i = threadIdx.x; i < MAXM * 33; i += Cfg::THREADS) (&Gs[0][0])[i] = 0.f;
+
+    // Lane (mi, ni) = (lane / 4, lane % 4) owns the MR x 8 block of the tile at rows MR * mi, columns 8 * ni,
+    // and the bias sums of its rows.  Per input row: its zb values with one or two 128-bit loads, its eight
+    // a values with scalar loads (four distinct addresses per instruction): about 12 cycles of the shared-
+    // memory pipe, where one column per lane with the zb row broadcast to all lanes costs 33 (a 128-bit
+    // load takes four cycles even when every lane reads the same address) and bound the kernel.  Blocks that
+    // hang over the tile (columns >= d_in, rows >= d_out) accumulate whatever lies behind the row and are
+    // dropped at the end.
+    constexpr int MR = MAXM / 8;
+    const int mi = lane >> 2, ni = lane & 3;
+    float G[MR][8], gs[MR];
+#pragma unroll
+    for (int i = 0; i < MR; ++i) {
+        gs[i] = 0.f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) G[i][j] = 0.f;
+    }
+    const bool zvec = (p.d_out & 3) == 0;
+
+    int slot = 0;
+    for (long base = first; base < r1; base += stride) {
+        cp_async_wait<SLOTS - 1>();                                // this chunk has landed (later ones may be in flight)
+        __syncwarp();
+        const int nr = rows_of(base);
+        const float* As = ring + slot * Cfg::SLOT_FLOATS;
+        const float* Zs = As + Cfg::A_FLOATS;
+        int e = GRAD ? (int)(base / p.T) : 0, rem = GRAD ? (int)(base - (long)e * p.T) : 0;
+        float c = 1.f;
+        if (GRAD) { if (p.clip) c = __ldg(p.clip + e); }
+        // two rows' operands are kept outstanding: while row r is multiplied, row r + 1 is already loaded
+        // into the other register set (ping-pong), so the FMAs never wait for shared memory
+        auto load_row = [&](int r, float (&z)[MR], float (&a)[8]) {
+            const float* zr = Zs + r * p.d_out + MR * mi;
+            if (zvec) {
+#pragma unroll
+                for (int i = 0; i < MR; i += 4) {
+                    const float4 z4 = *reinterpret_cast<const float4*>(zr + i);
+                    z[i] = z4.x; z[i + 1] = z4.y; z[i + 2] = z4.z; z[i + 3] = z4.w;
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < MR; ++i) z[i] = zr[i];
+            }
+            const float* ar = As + r * p.d_in + 8 * ni;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) a[j] = ar[j];
+        };
+        auto fma_row = [&](int r, float (&z)[MR], const float (&a)[8]) {
+            if (GRAD) {
+#pragma unroll
+                for (int i = 0; i < MR; ++i) z[i] *= c;
+                if (++rem == p.T) { rem = 0; ++e; if (p.clip && base + r + 1 < r1) c = __ldg(p.clip + e); }
+            }
+#pragma unroll
+            for (int i = 0; i < MR; ++i) {
+                gs[i] += z[i];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) G[i][j] = fmaf(z[i], a[j], G[i][j]);
+            }
+        };
+        float z0[MR], z1[MR], a0[8], a1[8];
+        if (nr > 0) load_row(0, z0, a0);
+#pragma unroll 1
+        for (int r = 0; r < nr; r += 2) {
+            if (r + 1 < nr) load_row(r + 1, z1, a1);
+            fma_row(r, z0, a0);
+            if (r + 2 < nr) load_row(r + 2, z0, a0);
+            if (r + 1 < nr) fma_row(r + 1, z1, a1);
+        }
+        __syncwarp();                                              // everyone is done with the slot
+        issue(base + SLOTS * stride, slot);
+        if (++slot == SLOTS) slot = 0;
+    }
+    cp_async_wait<0>();
+
+    __syncthreads();                                               // Gs zeroed by everyone
+#pragma unroll
+    for (int i = 0; i < MR; ++i) {
+        const int m = MR * mi + i;
+        if (m >= p.d_out) continue;
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            if (8 * ni + j < p.d_in) atomicAdd(&Gs[m][8 * ni + j], G[i][j]);
+        if (ni == 0 && p.has_bias) atomicAdd(&Gs[m][p.d_in], gs[i]);          // the all-ones column of [A | 1]
+    }
+    __syncthreads();
+
+    if (GRAD && p.part) {
+        float* mine = p.part + (size_t)blockIdx.x * MAXM * 32;
+        for (int i = threadIdx.x; i < MAXM * 32; i += Cfg::THREADS) mine[i] = Gs[i >> 5][i & 31];
+    } else if (GRAD) {
+        for (int i = threadIdx.x; i < p.d_out * 32; i += Cfg::THREADS) {
+            const int m = i >> 5, n = i & 31;
+            if (n < p.d_in) atomicAdd(p.gW + (size_t)m * p.ldg + n, Gs[m][n]);
+            else if (n == p.d_in && p.has_bias && p.gb) atomicAdd(p.gb + m, Gs[m][n]);
+        }
+    } else {
+        float s = 0.f;
+        for (int i = threadIdx.x; i < p.d_out * 32; i += Cfg::THREADS) {
+            const float v = Gs[i >> 5][i & 31];                    // unused columns hold zeros
+            s = fmaf(v, v, s);
+        }
+        s = block_sum(s, red);
+        if (threadIdx.x == 0) p.sq[blockIdx.x] = s;
+    }
+}
+
 // Second stage of the narrow clipped sum: out[m][n] = sum over the CTAs' partial tiles, + noise.
 // One CTA per output row m: 32 columns x 8 groups of partials, combined through shared memory.
 struct NarrowReduceParams {

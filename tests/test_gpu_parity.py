@@ -518,6 +518,22 @@ def test_step_mlp_tensor_core_edges(dp):
     _check_step(dp, big, _calibrate(big, layers, 6, big.C), big.C, big.sigma, 6)
 
 
+def test_narrow_layer_register_staged_form(dp, monkeypatch):
+    """fp32 narrow layers normally take the cp.async ring kernel; the register-staged kernel (what bf16 and
+    unaligned layers use) must give the same norms and clipped sums on the same fp32 input."""
+    monkeypatch.setenv("DPCLIP_NO_NARROW_RING", "1")
+    B, T, d_in, d_out = 5, 200, 27, 32
+    A, Z = workloads.random_layer(33, B, T, d_in, d_out, "f32", scale_z=0.05)
+    ref = oracle.layer_sqnorms(A, Z, True)
+    got = _sqnorms(dp, A, Z, "f32", True)
+    assert max_rel(np.sqrt(got), np.sqrt(ref)) <= TOL["f32"]["norm"]
+    clip = np.random.default_rng(1).uniform(0.1, 1.0, B).astype(np.float32)
+    refW, refb = oracle.clipped_grad(A, Z, clip)
+    gW = torch.empty(d_out, d_in, device="cuda"); gb = torch.empty(d_out, device="cuda")
+    dp.dpclip_clipped_grad(to_device(A, "f32"), to_device(Z, "f32"), torch.from_numpy(clip).cuda(), gW, gb, _ws(dp))
+    assert rel_fro(gW.cpu().numpy(), refW) <= TOL["f32"]["grad"] and rel_fro(gb.cpu().numpy(), refb) <= TOL["f32"]["grad"]
+
+
 def test_step_mlp_fp32_alu_kernel(dp, monkeypatch):
     """The fp32-ALU second launch of the fused step (what models the tensor-core launch rejects fall back to)."""
     monkeypatch.setenv("DPCLIP_NO_T1_TF32", "1")
