@@ -56,6 +56,12 @@ def lib():
             L.oracle_elementwise_sqnorms.restype = ctypes.c_int
             L.oracle_elementwise_clipped_grad.argtypes = [_dp, _dp] + [ctypes.c_int] * 3 + [_dp, _dp, _dp]
             L.oracle_elementwise_clipped_grad.restype = ctypes.c_int
+            L.oracle_dp_sgd_step.argtypes = [_dp, _dp, ctypes.c_size_t, ctypes.c_double, ctypes.c_double, ctypes.c_double,
+                                             ctypes.c_uint64, ctypes.c_uint64, ctypes.c_double]
+            L.oracle_dp_sgd_step.restype = ctypes.c_int
+            L.oracle_dp_adam_step.argtypes = [_dp, _dp, _dp, _dp, ctypes.c_size_t] + [ctypes.c_double] * 3 + \
+                                             [ctypes.c_uint64, ctypes.c_uint64] + [ctypes.c_double] * 4 + [ctypes.c_int]
+            L.oracle_dp_adam_step.restype = ctypes.c_int
             L.oracle_philox4x32_10.argtypes = [u32p, u32p, u32p]
             L.oracle_philox4x32_10.restype = None
             L.oracle_normals.argtypes = [ctypes.c_size_t, ctypes.c_uint64, ctypes.c_uint64, _dp]
@@ -177,6 +183,26 @@ def add_noise(g, sigma: float, C: float, seed: int, stream_id: int) -> np.ndarra
     if lib().oracle_add_noise(_p(flat), flat.size, float(sigma), float(C), seed, stream_id):
         raise MemoryError
     return out
+
+
+def dp_sgd_step(theta, gsum, inv_tau: float, C: float, sigma: float, seed: int, stream_id: int, lr: float) -> np.ndarray:
+    """theta - lr * (gsum + sigma C xi) / tau (Algorithm 1's update); returns the new parameters."""
+    th = _f64(theta).copy().reshape(-1); g = _f64(gsum).reshape(-1)
+    if lib().oracle_dp_sgd_step(_p(th), _p(g), th.size, inv_tau, C, sigma, seed, stream_id, lr):
+        raise MemoryError
+    return th.reshape(np.shape(theta))
+
+
+def dp_adam_step(theta, m, v, gsum, inv_tau: float, C: float, sigma: float, seed: int, stream_id: int, lr: float,
+                 beta1: float, beta2: float, eps: float, t: int):
+    """One step of the private Adam; returns (theta, m, v) after the step."""
+    th = _f64(theta).copy().reshape(-1); mm = _f64(m).copy().reshape(-1); vv = _f64(v).copy().reshape(-1)
+    g = _f64(gsum).reshape(-1)
+    if lib().oracle_dp_adam_step(_p(th), _p(mm), _p(vv), _p(g), th.size, inv_tau, C, sigma, seed, stream_id, lr,
+                                 beta1, beta2, eps, t):
+        raise MemoryError
+    sh = np.shape(theta)
+    return th.reshape(sh), mm.reshape(sh), vv.reshape(sh)
 
 
 def step(layers, has_bias: Sequence[bool], C: float, sigma: float, seed: int, stream_id0: int = 0):

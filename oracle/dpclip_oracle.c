@@ -242,3 +242,43 @@ int oracle_add_noise(double* g, size_t n, double sigma, double C, uint64_t seed,
     free(xi);
     return 0;
 }
+
+/* -------------------------------------------------------- parameter updates */
+
+/* The update of Algorithm 1's last line, theta <- theta - eta * (noise + (1/tau) * clipped sum), with the
+ * noise read as in the rest of this file: N(0, sigma^2 C^2) on the SUM, so the noisy mean gradient is
+ *     g[j] = (gsum[j] + sigma * C * xi_j) / tau.
+ * inv_tau = 1/tau.  theta[n] is updated in place. */
+int oracle_dp_sgd_step(double* theta, const double* gsum, size_t n, double inv_tau, double C, double sigma,
+                       uint64_t seed, uint64_t stream_id, double lr)
+{
+    double* xi = (double*)malloc(sizeof(double) * (n ? n : 1));
+    if (!xi) return -1;
+    oracle_normals(n, seed, stream_id, xi);
+    for (size_t j = 0; j < n; ++j) theta[j] -= lr * (gsum[j] + sigma * C * xi[j]) * inv_tau;
+    free(xi);
+    return 0;
+}
+
+/* The private Adam of the experiments (Sec. "Experiments": the non-private Adam of Kingma & Ba fed with the
+ * noisy clipped gradient; step size 0.001, beta1 = 0.9, beta2 = 0.999 there).  With g as above and t the
+ * 1-based step count:
+ *     m <- beta1 m + (1 - beta1) g,   v <- beta2 v + (1 - beta2) g^2,
+ *     theta <- theta - lr * (m / (1 - beta1^t)) / (sqrt(v / (1 - beta2^t)) + eps). */
+int oracle_dp_adam_step(double* theta, double* m, double* v, const double* gsum, size_t n, double inv_tau, double C,
+                        double sigma, uint64_t seed, uint64_t stream_id, double lr, double beta1, double beta2,
+                        double eps, int t)
+{
+    double* xi = (double*)malloc(sizeof(double) * (n ? n : 1));
+    if (!xi) return -1;
+    oracle_normals(n, seed, stream_id, xi);
+    const double c1 = 1.0 - pow(beta1, (double)t), c2 = 1.0 - pow(beta2, (double)t);
+    for (size_t j = 0; j < n; ++j) {
+        const double g = (gsum[j] + sigma * C * xi[j]) * inv_tau;
+        m[j] = beta1 * m[j] + (1.0 - beta1) * g;
+        v[j] = beta2 * v[j] + (1.0 - beta2) * g * g;
+        theta[j] -= lr * (m[j] / c1) / (sqrt(v[j] / c2) + eps);
+    }
+    free(xi);
+    return 0;
+}

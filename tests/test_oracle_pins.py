@@ -367,3 +367,35 @@ def test_elementwise_clipped_sum_limits_and_linearity():
     perm = rng.permutation(T)
     np.testing.assert_allclose(oracle.elementwise_sqnorms(H[:, perm], Z[:, perm], True),
                                oracle.elementwise_sqnorms(H, Z, True), rtol=1e-12)
+
+
+# ---------------------------------------------------------------------------
+# parameter updates (Algorithm 1's last line; the private Adam of the experiments)
+# ---------------------------------------------------------------------------
+def test_dp_updates_match_library_optimizers():
+    """Fed with the same noisy mean gradient, the oracle's SGD and Adam steps must be the library's."""
+    rng = np.random.default_rng(9)
+    n, tau, C, sigma, lr = 37, 16, 1.3, 0.7, 1e-3
+    theta0 = rng.standard_normal(n)
+    for opt_name in ("sgd", "adam"):
+        p = torch.tensor(theta0.copy(), requires_grad=True)
+        opt = torch.optim.SGD([p], lr=lr) if opt_name == "sgd" else torch.optim.Adam([p], lr=lr, betas=(0.9, 0.999), eps=1e-8)
+        th = theta0.copy(); m = np.zeros(n); v = np.zeros(n)
+        for t in range(1, 5):
+            gsum = rng.standard_normal(n) * 3.0
+            g = (gsum + sigma * C * oracle.normals(n, 5, 100 + t)) / tau        # the noisy mean gradient
+            p.grad = torch.tensor(g)
+            opt.step()
+            if opt_name == "sgd":
+                th = oracle.dp_sgd_step(th, gsum, 1.0 / tau, C, sigma, 5, 100 + t, lr)
+            else:
+                th, m, v = oracle.dp_adam_step(th, m, v, gsum, 1.0 / tau, C, sigma, 5, 100 + t, lr, 0.9, 0.999, 1e-8, t)
+                st = opt.state[p]
+                np.testing.assert_allclose(m, st["exp_avg"].numpy(), rtol=1e-12, atol=1e-15)
+                np.testing.assert_allclose(v, st["exp_avg_sq"].numpy(), rtol=1e-12, atol=1e-18)
+            np.testing.assert_allclose(th, p.detach().numpy(), rtol=1e-11, atol=1e-14)
+
+
+def test_dp_sgd_step_without_noise_is_plain_descent():
+    th = oracle.dp_sgd_step(np.ones(5), np.arange(5.0), 0.25, 1.0, 0.0, 1, 2, 0.1)
+    np.testing.assert_allclose(th, 1.0 - 0.1 * 0.25 * np.arange(5.0), rtol=1e-15)
