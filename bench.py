@@ -495,6 +495,16 @@ def run_sweep(args):
         noise = dict(n=args.noise_n, ms=ms, gbs=8.0 * args.noise_n / (ms * 1e-3) / 1e9)
         print(f"noise n={args.noise_n}: {ms * 1e3:.1f} us  {noise['gbs']:.0f} GB/s "
               f"({noise['gbs'] / peaks['hbm_gbs']:.2f} of the {peaks['source']} copy bandwidth)")
+        # parameter updates with the noise folded in: SGD 12 bytes per parameter (gsum, theta in; theta out),
+        # Adam 28 (gsum, theta, m, v in; theta, m, v out)
+        th = torch.zeros(args.noise_n, device="cuda"); m = torch.zeros_like(th); v = torch.zeros_like(th)
+        for name, nbytes, fn in (("dp_sgd_step", 12.0, lambda: dp.dpclip_dp_sgd_step(th, g, 1 / 128, 1.0, 1.0, 1, 0, 1e-3)),
+                                 ("dp_adam_step", 28.0, lambda: dp.dpclip_dp_adam_step(th, m, v, g, 1 / 128, 1.0, 1.0, 1, 0, 1e-3,
+                                                                                       0.9, 0.999, 1e-8, 1))):
+            ms = float(np.median(time_steps(torch, fn, 5, 3, flush)))
+            gbs = nbytes * args.noise_n / (ms * 1e-3) / 1e9
+            noise[name] = dict(ms=ms, gbs=gbs)
+            print(f"{name} n={args.noise_n}: {ms * 1e3:.1f} us  {gbs:.0f} GB/s ({gbs / peaks['hbm_gbs']:.2f} of the copy bandwidth)")
     print(json.dumps(dict(sweep="norm_method_crossover", dtype="bf16", peaks=peaks, points=rows, noise=noise)))
 
 

@@ -216,6 +216,23 @@ int dpclip_step(const dpclip_layer* layers /* host */, int L, int B, dpclip_dtyp
                 float* sq_layers, float* clip, float* norms,
                 void* workspace, size_t workspace_bytes, void* stream);
 
+/* Parameter updates with the noise folded in (one pass over the parameters instead of a noise pass and
+ * an optimiser pass).  gsum is the PRE-noise clipped sum of one tensor (run the step with sigma = 0);
+ * the noisy mean gradient is g[j] = (gsum[j] + sigma * C * xi_j) * inv_tau with xi as in dpclip_add_noise
+ * for the same (seed, stream_id), inv_tau = 1 / batch size.
+ *   dpclip_dp_sgd_step : theta -= lr * g                                  (Algorithm 1, last line)
+ *   dpclip_dp_adam_step: m = beta1 m + (1 - beta1) g, v = beta2 v + (1 - beta2) g^2,
+ *                        theta -= lr * (m / (1 - beta1^step)) / (sqrt(v / (1 - beta2^step)) + eps),
+ *                        step counted from 1 (the private Adam of Sec. "Experiments": lr 0.001,
+ *                        beta1 0.9, beta2 0.999 there).
+ * theta, m, v [n] fp32 updated in place; gsum [n] fp32 read only.  Errors: INVALID_ARG (null pointer,
+ * negative sigma or C, inv_tau <= 0, step < 1, beta outside [0, 1)), MISALIGNED. */
+int dpclip_dp_sgd_step(float* theta, const float* gsum, size_t n, float inv_tau, float C, float sigma,
+                       unsigned long long seed, unsigned long long stream_id, float lr, void* stream);
+int dpclip_dp_adam_step(float* theta, float* m, float* v, const float* gsum, size_t n, float inv_tau,
+                        float C, float sigma, unsigned long long seed, unsigned long long stream_id,
+                        float lr, float beta1, float beta2, float eps, int step, void* stream);
+
 /* Noise on every released tensor of a model in one launch: weights of layer l on noise stream
  * stream_id0 + 2l, its bias on + 2l + 1, exactly as dpclip_step numbers them (dense output rows
  * required).  For callers that add the noise after their own reduction over ranks.

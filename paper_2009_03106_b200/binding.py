@@ -60,6 +60,10 @@ def load_library():
                                             _u64, _vp, _sz, _vp]
     L.dpclip_clipped_grad_noise.restype = _i
     L.dpclip_add_noise.argtypes = [_vp, _sz, _f, _f, _u64, _u64, _vp]
+    L.dpclip_dp_sgd_step.argtypes = [_vp, _vp, _sz, _f, _f, _f, _u64, _u64, _f, _vp]
+    L.dpclip_dp_sgd_step.restype = _i
+    L.dpclip_dp_adam_step.argtypes = [_vp, _vp, _vp, _vp, _sz, _f, _f, _f, _u64, _u64, _f, _f, _f, _f, _i, _vp]
+    L.dpclip_dp_adam_step.restype = _i
     L.dpclip_step_noise.argtypes = [ctypes.POINTER(_CLayer), _i, _f, _f, _u64, _u64, _vp]
     L.dpclip_step_noise.restype = _i
     L.dpclip_t1_layers_supported.argtypes = [ctypes.POINTER(_CLayer), _i, _i, _i]
@@ -376,6 +380,24 @@ class StepPlan:
                                               stream_id0 + 2 * l, stream_id0 + 2 * l + 1, self._branch_ws[b])
             join()
         return graph
+
+
+def dpclip_dp_sgd_step(theta: torch.Tensor, gsum: torch.Tensor, inv_tau: float, C: float, sigma: float, seed: int,
+                       stream_id: int, lr: float, stream=None) -> None:
+    assert theta.dtype == gsum.dtype == torch.float32 and theta.is_contiguous() and gsum.is_contiguous()
+    assert theta.numel() == gsum.numel()
+    _check("dpclip_dp_sgd_step", load_library().dpclip_dp_sgd_step(
+        _ptr(theta), _ptr(gsum), theta.numel(), inv_tau, C, sigma, seed, stream_id, lr, _stream(stream)))
+
+
+def dpclip_dp_adam_step(theta: torch.Tensor, m: torch.Tensor, v: torch.Tensor, gsum: torch.Tensor, inv_tau: float,
+                        C: float, sigma: float, seed: int, stream_id: int, lr: float, beta1: float, beta2: float,
+                        eps: float, step: int, stream=None) -> None:
+    for t in (theta, m, v, gsum):
+        assert t.dtype == torch.float32 and t.is_contiguous() and t.numel() == theta.numel()
+    _check("dpclip_dp_adam_step", load_library().dpclip_dp_adam_step(
+        _ptr(theta), _ptr(m), _ptr(v), _ptr(gsum), theta.numel(), inv_tau, C, sigma, seed, stream_id, lr, beta1, beta2,
+        eps, step, _stream(stream)))
 
 
 def dpclip_step_noise(plan: StepPlan, C: float, sigma: float, seed: int, stream_id0: int = 0, stream=None) -> None:

@@ -3,6 +3,8 @@
 #include <string.h>
 
 #include "common.cuh"
+#include <math.h>
+
 #include "kernels_simt.cuh"
 #include "kernels_stream.cuh"
 #include "kernels_tc.cuh"
@@ -821,6 +823,47 @@ int dpclip_clipped_grad_noise(const void* A, long lda, const void* Zbar, long ld
     rc = dpclip_add_noise(gW, (size_t)d_out * d_in, sigma, C, seed, stream_id_w, stream);
     if (rc || !gb) return rc;
     return dpclip_add_noise(gb, (size_t)d_out, sigma, C, seed, stream_id_b, stream);
+}
+
+static int launch_dp_update(bool adam, float* theta, float* m, float* v, const float* gsum, size_t n, float inv_tau,
+                            float C, float sigma, unsigned long long seed, unsigned long long stream_id, float lr,
+                            float beta1, float beta2, float eps, int step, void* stream) {
+    if (n == 0) return DPCLIP_OK;
+    if (!theta || !gsum || (adam && (!m || !v))) return DPCLIP_ERR_INVALID_ARG;
+    if (!(sigma >= 0.f) || !(C >= 0.f) || !(inv_tau > 0.f)) return DPCLIP_ERR_INVALID_ARG;
+    if (adam && (step < 1 || !(beta1 >= 0.f && beta1 < 1.f) || !(beta2 >= 0.f && beta2 < 1.f))) return DPCLIP_ERR_INVALID_ARG;
+    if (!aligned_to(theta, 4) || !aligned_to(gsum, 4) || (adam && (!aligned_to(m, 4) || !aligned_to(v, 4))))
+        return DPCLIP_ERR_MISALIGNED;
+    UpdateParams p;
+    memset(&p, 0, sizeof(p));
+    p.theta = theta; p.m = m; p.v = v; p.gsum = gsum; p.n = n;
+    p.inv_tau = inv_tau; p.scale = sigma * C; p.lr = lr; p.beta1 = beta1; p.beta2 = beta2; p.eps = eps;
+    if (adam) {
+        p.inv_c1 = (float)(1.0 / (1.0 - pow((double)beta1, (double)step)));
+        p.inv_c2 = (float)(1.0 / (1.0 - pow((double)beta2, (double)step)));
+    }
+    p.k0 = (uint32_t)seed; p.k1 = (uint32_t)(seed >> 32); p.s0 = (uint32_t)stream_id; p.s1 = (uint32_t)(stream_id >> 32);
+    p.vec_ok = aligned_to(theta, 16) && aligned_to(gsum, 16) && (!adam || (aligned_to(m, 16) && aligned_to(v, 16)));
+    const size_t nq = (n + 3) / 4;
+    size_t blocks = (nq + 255) / 256;
+    const size_t cap = (size_t)kNumSMs * 16;
+    if (blocks > cap) blocks = cap;
+    if (adam) dp_update_kernel<true><<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(p);
+    else dp_update_kernel<false><<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(p);
+    return launch_status();
+}
+
+int dpclip_dp_sgd_step(float* theta, const float* gsum, size_t n, float inv_tau, float C, float sigma,
+                       unsigned long long seed, unsigned long long stream_id, float lr, void* stream) {
+    return launch_dp_update(false, theta, nullptr, nullptr, gsum, n, inv_tau, C, sigma, seed, stream_id, lr, 0.f, 0.f,
+                            0.f, 1, stream);
+}
+
+int dpclip_dp_adam_step(float* theta, float* m, float* v, const float* gsum, size_t n, float inv_tau, float C,
+                        float sigma, unsigned long long seed, unsigned long long stream_id, float lr, float beta1,
+                        float beta2, float eps, int step, void* stream) {
+    return launch_dp_update(true, theta, m, v, gsum, n, inv_tau, C, sigma, seed, stream_id, lr, beta1, beta2, eps,
+                            step, stream);
 }
 
 int dpclip_step_noise(const dpclip_layer* layers, int L, float C, float sigma, unsigned long long seed,

@@ -147,6 +147,74 @@ noise_kernel(float* __restrict__ g, size_t n, float scale, uint32_t k0, uint32_t
     }
 }
 
+// ---------------------------------------------------------------------------
+// Parameter updates with the noise folded in (one pass over the parameters instead of a noise pass
+// followed by an optimiser pass).  g = (gsum + scale * xi) * inv_tau is the noisy mean gradient of
+// Algorithm 1's last line; ADAM = false applies theta -= lr * g, ADAM = true the Adam rule with bias
+// corrections c1 = 1 - beta1^t, c2 = 1 - beta2^t computed on the host.
+// ---------------------------------------------------------------------------
+struct UpdateParams {
+    float* theta; float* m; float* v; const float* gsum; size_t n;
+    float inv_tau, scale, lr, beta1, beta2, eps, inv_c1, inv_c2;
+    uint32_t k0, k1, s0, s1;
+    int vec_ok;
+};
+
+template <bool ADAM>
+__global__ void __launch_bounds__(256)
+dp_update_kernel(const UpdateParams p) {
+    const size_t nq = (p.n + 3) >> 2;
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t q = (size_t)blockIdx.x * blockDim.x + threadIdx.x; q < nq; q += stride) {
+        const size_t j = q << 2;
+        const bool full = p.vec_ok && j + 3 < p.n;
+        float g[4], th[4], mm[4], vv[4];
+        if (full) {
+            const float4 a = *reinterpret_cast<const float4*>(p.gsum + j), b = *reinterpret_cast<const float4*>(p.theta + j);
+            g[0] = a.x; g[1] = a.y; g[2] = a.z; g[3] = a.w; th[0] = b.x; th[1] = b.y; th[2] = b.z; th[3] = b.w;
+            if (ADAM) {
+                const float4 c = *reinterpret_cast<const float4*>(p.m + j), d = *reinterpret_cast<const float4*>(p.v + j);
+                mm[0] = c.x; mm[1] = c.y; mm[2] = c.z; mm[3] = c.w; vv[0] = d.x; vv[1] = d.y; vv[2] = d.z; vv[3] = d.w;
+            }
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const bool in = j + e < p.n;
+                g[e] = in ? p.gsum[j + e] : 0.f; th[e] = in ? p.theta[j + e] : 0.f;
+                if (ADAM) { mm[e] = in ? p.m[j + e] : 0.f; vv[e] = in ? p.v[j + e] : 0.f; }
+            }
+        }
+        float z[4] = {0.f, 0.f, 0.f, 0.f};
+        if (p.scale > 0.f) {
+            PhiloxBlock b = philox_block((uint32_t)q, (uint32_t)(q >> 32), p.s0, p.s1, p.k0, p.k1);
+            box_muller(b.v[0], b.v[1], z[0], z[1]);
+            box_muller(b.v[2], b.v[3], z[2], z[3]);
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float gn = fmaf(p.scale, z[e], g[e]) * p.inv_tau;
+            if (ADAM) {
+                mm[e] = fmaf(p.beta1, mm[e], (1.f - p.beta1) * gn);
+                vv[e] = fmaf(p.beta2, vv[e], (1.f - p.beta2) * gn * gn);
+                th[e] -= p.lr * (mm[e] * p.inv_c1) / (sqrtf(vv[e] * p.inv_c2) + p.eps);
+            } else {
+                th[e] = fmaf(-p.lr, gn, th[e]);
+            }
+        }
+        if (full) {
+            *reinterpret_cast<float4*>(p.theta + j) = make_float4(th[0], th[1], th[2], th[3]);
+            if (ADAM) {
+                *reinterpret_cast<float4*>(p.m + j) = make_float4(mm[0], mm[1], mm[2], mm[3]);
+                *reinterpret_cast<float4*>(p.v + j) = make_float4(vv[0], vv[1], vv[2], vv[3]);
+            }
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                if (j + e < p.n) { p.theta[j + e] = th[e]; if (ADAM) { p.m[j + e] = mm[e]; p.v[j + e] = vv[e]; } }
+        }
+    }
+}
+
 // Noise on every released tensor of a model in ONE launch (the weights and the bias of layer l are
 // tensors 2l and 2l + 1, with their own noise streams).  Blocks are dealt to tensors by a prefix table.
 constexpr int NOISE_BATCH_MAX = 128;

@@ -375,6 +375,41 @@ def test_step_noise_equals_per_tensor_noise(dp):
         assert float(a.gW[l].abs().max()) > 0
 
 
+@pytest.mark.parametrize("n", [1, 5, 4096, 100003])
+def test_dp_sgd_and_adam_steps(dp, n):
+    """Parameter updates with the noise folded in (Algorithm 1's last line; the private Adam of the
+    experiments) against the oracle, over several steps so that the moments carry over."""
+    rng = np.random.default_rng(n)
+    # both sides start from the same (fp32-representable) hyper-parameters: 1 - 0.999 differs by 1.3e-5 between
+    # the fp32 and the fp64 reading of 0.999
+    tau, C, sigma, lr, b1, b2, eps = (128, 1.0, float(np.float32(1.1)), float(np.float32(1e-3)), float(np.float32(0.9)),
+                                      float(np.float32(0.999)), float(np.float32(1e-8)))
+    th0 = rng.standard_normal(n).astype(np.float32)
+    # SGD
+    gsum = (rng.standard_normal(n) * 5).astype(np.float32)
+    th = torch.from_numpy(th0.copy()).cuda()
+    dp.dpclip_dp_sgd_step(th, torch.from_numpy(gsum).cuda(), 1.0 / tau, C, sigma, 7, 11, 0.05)
+    ref = oracle.dp_sgd_step(th0, gsum, 1.0 / tau, C, sigma, 7, 11, 0.05)
+    assert np.max(np.abs(th.cpu().numpy() - ref)) <= 1e-5 * 0.05 + 2e-7 * np.max(np.abs(ref))
+    # Adam, 3 steps
+    th = torch.from_numpy(th0.copy()).cuda(); m = torch.zeros(n, device="cuda"); v = torch.zeros(n, device="cuda")
+    rth, rm, rv = th0.astype(np.float64), np.zeros(n), np.zeros(n)
+    for t in range(1, 4):
+        gsum = (rng.standard_normal(n) * 5).astype(np.float32)
+        dp.dpclip_dp_adam_step(th, m, v, torch.from_numpy(gsum).cuda(), 1.0 / tau, C, sigma, 7, 20 + t, lr, b1, b2, eps, t)
+        rth, rm, rv = oracle.dp_adam_step(rth, rm, rv, gsum, 1.0 / tau, C, sigma, 7, 20 + t, lr, b1, b2, eps, t)
+        # the moments are sums of terms of either sign: the error scales with the terms (|g| ~ 5 / tau), not with
+        # what is left of them
+        gs = 5.0 / tau
+        assert np.max(np.abs(m.cpu().numpy() - rm)) <= 1e-5 * np.max(np.abs(rm)) + 1e-6 * gs
+        assert np.max(np.abs(v.cpu().numpy() - rv)) <= 1e-5 * np.max(np.abs(rv)) + 1e-6 * gs * gs
+        assert np.max(np.abs(th.cpu().numpy() - rth)) <= 1e-4 * lr + 2e-7 * np.max(np.abs(rth))
+    # sigma = 0 draws nothing: plain optimiser
+    th = torch.ones(n, device="cuda"); g = torch.full((n,), 2.0, device="cuda")
+    dp.dpclip_dp_sgd_step(th, g, 0.5, 1.0, 0.0, 1, 1, 0.1)
+    assert torch.allclose(th, torch.full((n,), 0.9, device="cuda"), rtol=1e-6)
+
+
 def test_noise_is_stateless_and_stream_dependent(dp):
     n = 10007
     a = torch.zeros(n, device="cuda"); b = torch.zeros(n, device="cuda"); c = torch.zeros(n, device="cuda")
