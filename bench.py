@@ -392,6 +392,34 @@ def bench_elementwise(torch, dp, B, T, d, dtype, steps, flush, peaks):
     return out
 
 
+def bench_conv_implicit(torch, dp, name, B, C, H, W, k, pad, d_out, dtype, steps, flush, peaks):
+    """A convolution layer straight from its feature map (implicit im2col, fp32-ALU tiles), next to the same
+    layer through the patch-matrix entry points.  Algorithmic bytes: feature map + Zbar once per kernel."""
+    X, Z = workloads.conv_inputs(0, B, C, H, W, k, pad, 1, d_out, dtype, var_z=1.0 / B)
+    A = workloads.im2col(X, k, pad)
+    dX, dZ, dA = to_dev(X, dtype, torch), to_dev(Z, dtype, torch), to_dev(A, dtype, torch)
+    T, d_in = Z.shape[1], C * k * k
+    clip = torch.rand(B, device="cuda") * 0.9 + 0.1
+    sq = torch.empty(B, device="cuda"); gW = torch.empty(d_out, d_in, device="cuda"); gb = torch.empty(d_out, device="cuda")
+    ws = torch.empty(dp.dpclip_workspace_bytes(B, T, d_in, d_out, dp.DPCLIP_BF16), dtype=torch.uint8, device="cuda")
+    dp.dpclip_workspace_init(ws)
+    es = 4 if dtype == "f32" else 2
+    nbytes = (X.size + Z.size) * es
+    flops = 2.0 * B * T * d_in * d_out
+    out = dict(workload=name, algorithmic_bytes=int(nbytes), patch_matrix_bytes=int((A.size + Z.size) * es))
+    for kind, fn, ref in (("norm", lambda: dp.dpclip_conv_sqnorms(dX, dZ, k, k, 1, pad, True, sq),
+                           lambda: dp.dpclip_layer_sqnorms(dA, dZ, True, sq, ws)),
+                          ("grad", lambda: dp.dpclip_conv_clipped_grad(dX, dZ, k, k, 1, pad, clip, gW, gb),
+                           lambda: dp.dpclip_clipped_grad(dA, dZ, clip, gW, gb, ws))):
+        ms = float(np.median(time_steps(torch, fn, steps, 3, flush)))
+        ms_ref = float(np.median(time_steps(torch, ref, steps, 3, flush)))
+        ach = flops / (ms * 1e-3) / 1e12
+        out[kind] = dict(ms=ms, patch_matrix_path_ms=ms_ref,
+                         roofline=dict(bound="alu", achieved=ach, peak=FFMA_PEAK_TFLOPS, unit="TFLOP/s",
+                                       frac=ach / FFMA_PEAK_TFLOPS, traffic=None, peak_source="derived"))
+    return out
+
+
 # ---------------------------------------------------------------------------
 # CPU oracle legs
 # ---------------------------------------------------------------------------
@@ -623,6 +651,9 @@ def main():
             for shape in ((128, 256, 512, "bf16"), (512, 512, 1024, "bf16")):
                 r = bench_elementwise(torch, dp, *shape, min(args.steps, 20), flush, peaks)
                 others[r["workload"]] = r
+            r = bench_conv_implicit(torch, dp, "conv2_implicit_im2col_b128_f32", 128, 32, 16, 16, 3, 1, 64, "f32",
+                                    min(args.steps, 20), flush, peaks)
+            others[r["workload"]] = r
         line["workloads"] = others
         if not args.no_cpu_baseline:
             line["cpu_baseline"], _, _ = oracle_sample(w)

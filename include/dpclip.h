@@ -216,6 +216,26 @@ int dpclip_step(const dpclip_layer* layers /* host */, int L, int B, dpclip_dtyp
                 float* sq_layers, float* clip, float* norms,
                 void* workspace, size_t workspace_bytes, void* stream);
 
+/* Convolution layers given by their INPUT feature map (implicit im2col).  Algorithm 3 unfolds the input into
+ * the patch matrix (kh * kw copies of every pixel) and reshapes dL/dZ to [tau, c_out, T]; here element
+ * (row (i, t), column (c, ky, kx)) of that matrix is read straight from
+ *   X[i][c][y' * stride - pad + ky][x' * stride - pad + kx]   (zero outside the map), t = y' * W' + x',
+ * so the unfolded copy never exists, and dL/dZ can be passed as it comes out of back-propagation.
+ *   X       device, [B][C][H][W] contiguous, dtype `dtype`
+ *   Zbar    device, [B][T][d_out] (z_channel_major = 0) or [B][d_out][T] (= 1, i.e. [B][c_out][H'][W']),
+ *           T = H' * W', H' = (H + 2 pad - kh) / stride + 1, likewise W'
+ *   sq_layer, clip, gW, gb  as for dpclip_layer_sqnorms / dpclip_clipped_grad; gW is [d_out][C*kh*kw] with
+ *           columns ordered (c, ky, kx), c slowest: a convolution weight [c_out][c_in][kh][kw] flattened
+ * Square or rectangular kernels, any stride and zero padding; dilation 1.  fp32-ALU tiles (64 x 64), fp32
+ * accumulation; partial sums of split rows are combined with fp32 atomics.  No workspace.  Noise is added
+ * with dpclip_add_noise.  Errors as for dpclip_layer_sqnorms. */
+typedef struct { int C, H, W, kh, kw, stride, pad; } dpclip_conv;
+int dpclip_conv_sqnorms(const void* X, const void* Zbar, int z_channel_major, int B, const dpclip_conv* geom,
+                        int d_out, dpclip_dtype dtype, int has_bias, float* sq_layer, void* stream);
+int dpclip_conv_clipped_grad(const void* X, const void* Zbar, int z_channel_major, int B, const dpclip_conv* geom,
+                             int d_out, dpclip_dtype dtype, const float* clip, float* gW, long ldg, float* gb,
+                             void* stream);
+
 /* Parameter updates with the noise folded in (one pass over the parameters instead of a noise pass and
  * an optimiser pass).  gsum is the PRE-noise clipped sum of one tensor (run the step with sigma = 0);
  * the noisy mean gradient is g[j] = (gsum[j] + sigma * C * xi_j) * inv_tau with xi as in dpclip_add_noise

@@ -30,6 +30,11 @@ class DpclipError(RuntimeError):
         super().__init__(f"{fn} failed: {status} ({dpclip_status_string(status)})")
 
 
+class _CConv(ctypes.Structure):
+    _fields_ = [("C", ctypes.c_int), ("H", ctypes.c_int), ("W", ctypes.c_int), ("kh", ctypes.c_int),
+                ("kw", ctypes.c_int), ("stride", ctypes.c_int), ("pad", ctypes.c_int)]
+
+
 class _CLayer(ctypes.Structure):
     _fields_ = [("A", _vp), ("lda", _l), ("Zbar", _vp), ("ldz", _l),
                 ("T", _i), ("d_in", _i), ("d_out", _i), ("has_bias", _i), ("method", _i),
@@ -60,6 +65,10 @@ def load_library():
                                             _u64, _vp, _sz, _vp]
     L.dpclip_clipped_grad_noise.restype = _i
     L.dpclip_add_noise.argtypes = [_vp, _sz, _f, _f, _u64, _u64, _vp]
+    L.dpclip_conv_sqnorms.argtypes = [_vp, _vp, _i, _i, ctypes.POINTER(_CConv), _i, _i, _i, _vp, _vp]
+    L.dpclip_conv_sqnorms.restype = _i
+    L.dpclip_conv_clipped_grad.argtypes = [_vp, _vp, _i, _i, ctypes.POINTER(_CConv), _i, _i, _vp, _vp, _l, _vp, _vp]
+    L.dpclip_conv_clipped_grad.restype = _i
     L.dpclip_dp_sgd_step.argtypes = [_vp, _vp, _sz, _f, _f, _f, _u64, _u64, _f, _vp]
     L.dpclip_dp_sgd_step.restype = _i
     L.dpclip_dp_adam_step.argtypes = [_vp, _vp, _vp, _vp, _sz, _f, _f, _f, _u64, _u64, _f, _f, _f, _f, _i, _vp]
@@ -380,6 +389,41 @@ class StepPlan:
                                               stream_id0 + 2 * l, stream_id0 + 2 * l + 1, self._branch_ws[b])
             join()
         return graph
+
+
+def _conv_args(X: torch.Tensor, Zbar: torch.Tensor, kh: int, kw: int, stride: int, pad: int, z_channel_major: bool):
+    assert X.dim() == 4 and X.is_contiguous() and Zbar.is_contiguous() and X.dtype == Zbar.dtype
+    B, C, H, W = X.shape
+    Ho, Wo = (H + 2 * pad - kh) // stride + 1, (W + 2 * pad - kw) // stride + 1
+    if z_channel_major:
+        d_out = Zbar.shape[1]
+        assert Zbar.numel() == B * d_out * Ho * Wo
+    else:
+        d_out = Zbar.shape[-1]
+        assert Zbar.numel() == B * Ho * Wo * d_out
+    return B, d_out, _CConv(C, H, W, kh, kw, stride, pad)
+
+
+def dpclip_conv_sqnorms(X: torch.Tensor, Zbar: torch.Tensor, kh: int, kw: int, stride: int, pad: int, has_bias: bool,
+                        sq_layer: torch.Tensor, z_channel_major: bool = False, stream=None) -> None:
+    B, d_out, geom = _conv_args(X, Zbar, kh, kw, stride, pad, z_channel_major)
+    assert sq_layer.dtype == torch.float32 and sq_layer.numel() >= B and sq_layer.is_contiguous()
+    _check("dpclip_conv_sqnorms", load_library().dpclip_conv_sqnorms(
+        _ptr(X), _ptr(Zbar), int(z_channel_major), B, ctypes.byref(geom), d_out, _dtype_code(X), int(has_bias),
+        _ptr(sq_layer), _stream(stream)))
+
+
+def dpclip_conv_clipped_grad(X: torch.Tensor, Zbar: torch.Tensor, kh: int, kw: int, stride: int, pad: int,
+                             clip: Optional[torch.Tensor], gW: torch.Tensor, gb: Optional[torch.Tensor],
+                             z_channel_major: bool = False, stream=None) -> None:
+    B, d_out, geom = _conv_args(X, Zbar, kh, kw, stride, pad, z_channel_major)
+    d_in = X.shape[1] * kh * kw
+    assert gW.dtype == torch.float32 and gW.shape == (d_out, d_in) and gW.stride(1) == 1
+    assert gb is None or (gb.dtype == torch.float32 and gb.numel() == d_out and gb.is_contiguous())
+    _check("dpclip_conv_clipped_grad", load_library().dpclip_conv_clipped_grad(
+        _ptr(X), _ptr(Zbar), int(z_channel_major), B, ctypes.byref(geom), d_out, _dtype_code(X),
+        _ptr(clip) if clip is not None else None, _ptr(gW), gW.stride(0), _ptr(gb) if gb is not None else None,
+        _stream(stream)))
 
 
 def dpclip_dp_sgd_step(theta: torch.Tensor, gsum: torch.Tensor, inv_tau: float, C: float, sigma: float, seed: int,

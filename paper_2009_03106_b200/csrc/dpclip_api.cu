@@ -866,6 +866,83 @@ int dpclip_dp_adam_step(float* theta, float* m, float* v, const float* gsum, siz
                             step, stream);
 }
 
+// Convolution layers given by their input feature map (implicit im2col).
+static int conv_setup(SimtParams& p, const void* X, const void* Zbar, int z_channel_major, int B, const dpclip_conv* g,
+                      int d_out, dpclip_dtype dtype, int has_bias, int* T_out) {
+    if (!X || !Zbar || !g) return DPCLIP_ERR_INVALID_ARG;
+    if (B <= 0 || d_out <= 0 || g->C <= 0 || g->H <= 0 || g->W <= 0 || g->kh <= 0 || g->kw <= 0 || g->stride <= 0 ||
+        g->pad < 0) return DPCLIP_ERR_INVALID_ARG;
+    if (dtype != DPCLIP_F32 && dtype != DPCLIP_BF16) return DPCLIP_ERR_INVALID_ARG;
+    if (g->H + 2 * g->pad < g->kh || g->W + 2 * g->pad < g->kw) return DPCLIP_ERR_INVALID_ARG;
+    if (!aligned_to(X, elt_size(dtype)) || !aligned_to(Zbar, elt_size(dtype))) return DPCLIP_ERR_MISALIGNED;
+    const int Ho = (g->H + 2 * g->pad - g->kh) / g->stride + 1, Wo = (g->W + 2 * g->pad - g->kw) / g->stride + 1;
+    const long T = (long)Ho * Wo, d_in = (long)g->C * g->kh * g->kw;
+    if (T * B > 0x7FFFFFFFL || d_in > 0x7FFFFFFFL || (long)g->C * g->H * g->W > 0x7FFFFFFFL) return DPCLIP_ERR_INVALID_ARG;
+    fill_simt_params(p, X, d_in, Zbar, d_out, (int)T, (int)d_in, d_out, has_bias, dtype);
+    p.vec_a = 0;
+    p.vec_z = z_channel_major ? 0 : vec4_ok(Zbar, d_out, dtype);
+    p.cC = g->C; p.cH = g->H; p.cW = g->W; p.kh = g->kh; p.kw = g->kw; p.stride = g->stride; p.pad = g->pad;
+    p.Wo = Wo; p.z_cm = z_channel_major ? 1 : 0;
+    *T_out = (int)T;
+    return DPCLIP_OK;
+}
+
+int dpclip_conv_sqnorms(const void* X, const void* Zbar, int z_channel_major, int B, const dpclip_conv* geom,
+                        int d_out, dpclip_dtype dtype, int has_bias, float* sq_layer, void* stream) {
+    SimtParams p;
+    int T = 0;
+    int rc = conv_setup(p, X, Zbar, z_channel_major, B, geom, d_out, dtype, has_bias, &T);
+    if (rc) return rc;
+    if (!sq_layer) return DPCLIP_ERR_INVALID_ARG;
+    if (B > 65535) return DPCLIP_ERR_UNSUPPORTED;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int n_tiles = p.tiles_m * p.tiles_n;
+    int split = ceil_div(2 * kNumSMs, B);
+    if (split > n_tiles) split = n_tiles;
+    if (split < 1) split = 1;
+    p.sq = sq_layer;
+    p.use_atomic = split > 1;
+    if (p.use_atomic && cudaMemsetAsync(sq_layer, 0, sizeof(float) * (size_t)B, st) != cudaSuccess) return DPCLIP_ERR_CUDA;
+    dim3 grid(split, B);
+    if (dtype == DPCLIP_F32) zta_simt_kernel<float, false, true><<<grid, SIMT_THREADS, 0, st>>>(p);
+    else zta_simt_kernel<__nv_bfloat16, false, true><<<grid, SIMT_THREADS, 0, st>>>(p);
+    return launch_status();
+}
+
+int dpclip_conv_clipped_grad(const void* X, const void* Zbar, int z_channel_major, int B, const dpclip_conv* geom,
+                             int d_out, dpclip_dtype dtype, const float* clip, float* gW, long ldg, float* gb,
+                             void* stream) {
+    SimtParams p;
+    int T = 0;
+    int rc = conv_setup(p, X, Zbar, z_channel_major, B, geom, d_out, dtype, gb != nullptr, &T);
+    if (rc) return rc;
+    if (!gW || ldg < p.d_in) return DPCLIP_ERR_INVALID_ARG;
+    if (!aligned_to(gW, 4) || (gb && !aligned_to(gb, 4))) return DPCLIP_ERR_MISALIGNED;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int n_tiles = p.tiles_m * p.tiles_n;
+    const long rows = (long)B * T;
+    long ksplit = ceil_div(4 * kNumSMs, n_tiles);
+    const long max_split = (rows + 4 * SIMT_BK - 1) / (4 * SIMT_BK);
+    if (ksplit > max_split) ksplit = max_split;
+    if (ksplit < 1) ksplit = 1;
+    if (ksplit > 65535) ksplit = 65535;
+    long per = (rows + ksplit - 1) / ksplit;
+    per = (per + SIMT_BK - 1) / SIMT_BK * SIMT_BK;
+    ksplit = (rows + per - 1) / per;
+    p.clip = clip; p.gW = gW; p.ldg = ldg; p.gb = gb;
+    p.rows_total = rows; p.rows_per_split = per;
+    p.use_atomic = ksplit > 1;
+    if (p.use_atomic) {
+        if (cudaMemset2DAsync(gW, sizeof(float) * (size_t)ldg, 0, sizeof(float) * (size_t)p.d_in, d_out, st) != cudaSuccess)
+            return DPCLIP_ERR_CUDA;
+        if (gb && cudaMemsetAsync(gb, 0, sizeof(float) * (size_t)d_out, st) != cudaSuccess) return DPCLIP_ERR_CUDA;
+    }
+    dim3 grid(n_tiles, (unsigned)ksplit);
+    if (dtype == DPCLIP_F32) zta_simt_kernel<float, true, true><<<grid, SIMT_THREADS, 0, st>>>(p);
+    else zta_simt_kernel<__nv_bfloat16, true, true><<<grid, SIMT_THREADS, 0, st>>>(p);
+    return launch_status();
+}
+
 int dpclip_step_noise(const dpclip_layer* layers, int L, float C, float sigma, unsigned long long seed,
                       unsigned long long stream_id0, void* stream) {
     if (!layers || L <= 0 || !(C >= 0.f) || !(sigma >= 0.f)) return DPCLIP_ERR_INVALID_ARG;

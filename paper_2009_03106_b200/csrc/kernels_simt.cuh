@@ -39,6 +39,9 @@ struct SimtParams {
     // GRAD
     const float* clip; float* gW; long ldg; float* gb;
     long rows_total; long rows_per_split;
+    // CONV (implicit im2col): A is the feature map [B][C][H][W]; row (i, y', x') and column (c, ky, kx) of the
+    // patch matrix are gathered on the fly; Z may be channel-major [B][d_out][T]
+    int cC, cH, cW, kh, kw, stride, pad, Wo, z_cm;
 };
 
 template <typename T>
@@ -57,7 +60,11 @@ __device__ __forceinline__ float4 simt_load_row4(const T* __restrict__ base, lon
     return make_float4(e[0], e[1], e[2], e[3]);
 }
 
-template <typename T, bool GRAD>
+// CONV = true: the layer is a convolution given by its INPUT feature map (Algorithm 3 builds the patch
+// matrix with unfold; here element (row (i, t), column (c, ky, kx)) is read straight from
+// X[i][c][y' * stride - pad + ky][x' * stride - pad + kx], zero outside the map, so the kh * kw-fold copy of
+// the input never exists), and optionally by dL/dZ in its native [B][c_out][T] layout.
+template <typename T, bool GRAD, bool CONV = false>
 __global__ void __launch_bounds__(SIMT_THREADS)
 zta_simt_kernel(SimtParams p) {
     __shared__ __align__(16) float Zs[2][SIMT_BK][SIMT_BM];
@@ -95,11 +102,53 @@ zta_simt_kernel(SimtParams p) {
             for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
 
         float cf = 1.f;
+        // CONV: this thread's four patch columns, fixed for the tile: offset inside an example's map and tap
+        int coff[4], cky[4], ckx[4];
+        if (CONV) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int n = n0 + lc + j, kk = p.kh * p.kw;
+                const int c = n / kk, rem = n - c * kk;
+                cky[j] = rem / p.kw; ckx[j] = rem - cky[j] * p.kw;
+                coff[j] = (c * p.cH + cky[j]) * p.cW + ckx[j];
+            }
+        }
         auto fetch = [&](int slab, float4& zr, float4& ar) {
             const long r = row_begin + (long)slab * SIMT_BK + lk;
             const bool ok = r < row_end;
+            if (CONV) {
+                const int ri = (int)r;                                // B * T < 2^31 (checked by the launcher)
+                const int i = ri / p.T, t = ri - i * p.T;
+                const int yo = t / p.Wo, xo = t - yo * p.Wo;
+                const int y0 = yo * p.stride - p.pad, x0 = xo * p.stride - p.pad;
+                const T* xi = A + (size_t)i * p.cC * p.cH * p.cW + (y0 * p.cW + x0);
+                float e[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int n = n0 + lc + j;
+                    const int y = y0 + cky[j], x = x0 + ckx[j];
+                    float v = 0.f;
+                    if (ok) {
+                        if (n < p.d_in) { if (y >= 0 && y < p.cH && x >= 0 && x < p.cW) v = to_f32(xi[coff[j]]); }
+                        else if (n == p.d_in && p.has_bias) v = 1.f;
+                    }
+                    e[j] = v;
+                }
+                ar = make_float4(e[0], e[1], e[2], e[3]);
+                if (p.z_cm) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const int m = m0 + lc + j;
+                        e[j] = (ok && m < p.d_out) ? to_f32(Z[((size_t)i * p.d_out + m) * p.T + t]) : 0.f;
+                    }
+                    zr = make_float4(e[0], e[1], e[2], e[3]);
+                } else {
+                    zr = simt_load_row4(Z, p.ldz, r, m0 + lc, p.d_out, ok, p.vec_z != 0, false);
+                }
+            } else {
             zr = simt_load_row4(Z, p.ldz, r, m0 + lc, p.d_out, ok, p.vec_z != 0, false);
             ar = simt_load_row4(A, p.lda, r, n0 + lc, p.d_in, ok, p.vec_a != 0, p.has_bias != 0);
+            }
             cf = 1.f;
             if (GRAD) {
                 if (ok && p.clip) cf = __ldg(p.clip + r / p.T);

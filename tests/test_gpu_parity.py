@@ -257,6 +257,40 @@ def test_transformer_block_with_layernorms(dp):
 
 
 # ---------------------------------------------------------------------------
+# convolution layers given by their input feature map (implicit im2col)
+# ---------------------------------------------------------------------------
+CONV_CASES = [  # B, C, H, W, k, pad, stride, d_out
+    (3, 3, 8, 8, 3, 1, 1, 5), (2, 4, 9, 7, (3, 2), 1, 2, 70), (4, 32, 16, 16, 3, 1, 1, 64), (2, 5, 6, 6, 1, 0, 1, 3),
+    (2, 2, 11, 10, 5, 2, 3, 9), (3, 8, 4, 4, 4, 0, 1, 6),
+]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("case", CONV_CASES)
+def test_conv_implicit_im2col(dp, case, dtype):
+    """Norms and clipped sums straight from the feature map equal the oracle's on the unfolded patch matrix,
+    with dL/dZ in either layout."""
+    B, C, H, W, k, pad, stride, d_out = case
+    kh, kw = (k, k) if isinstance(k, int) else k
+    X, Z = workloads.conv_inputs(17, B, C, H, W, k, pad, stride, d_out, dtype, var_z=0.01)
+    A = workloads.im2col(X, k, pad, stride)                      # what Algorithm 3 would build
+    tol = TOL[dtype]
+    dX, dZ = to_device(X, dtype), to_device(Z, dtype)
+    dZcm = dZ.transpose(1, 2).contiguous()                        # [B][d_out][T], the layout of dL/dZ itself
+    clip = np.random.default_rng(B).uniform(0.1, 1.0, B).astype(np.float32)
+    refW, refb = oracle.clipped_grad(A, Z, clip)
+    for cm, z in ((False, dZ), (True, dZcm)):
+        for has_bias in (True, False):
+            ref = oracle.layer_sqnorms(A, Z, has_bias)
+            sq = torch.full((B,), -1.0, device="cuda")
+            dp.dpclip_conv_sqnorms(dX, z, kh, kw, stride, pad, has_bias, sq, z_channel_major=cm)
+            assert max_rel(np.sqrt(sq.cpu().numpy()), np.sqrt(ref)) <= tol["norm"]
+        gW = torch.full((d_out, C * kh * kw), 3.0, device="cuda"); gb = torch.full((d_out,), 3.0, device="cuda")
+        dp.dpclip_conv_clipped_grad(dX, z, kh, kw, stride, pad, torch.from_numpy(clip).cuda(), gW, gb, z_channel_major=cm)
+        assert rel_fro(gW.cpu().numpy(), refW) <= tol["grad"] and rel_fro(gb.cpu().numpy(), refb) <= tol["grad"]
+
+
+# ---------------------------------------------------------------------------
 # (c) factors
 # ---------------------------------------------------------------------------
 @pytest.mark.parametrize("B,L", [(1, 1), (32, 2), (128, 3), (1024, 7), (1500, 2)])

@@ -117,6 +117,11 @@ def test_im2col_generator_matches_library_unfold():
     ours = workloads.im2col(fmap, 3, 1)
     ref = F.unfold(torch.from_numpy(fmap).double(), 3, padding=1).transpose(1, 2).numpy()
     np.testing.assert_array_equal(ours.astype(np.float64), ref)
+    # strides, rectangular kernels, no padding
+    for k, pad, stride in ((2, 0, 2), ((3, 2), 1, 1), ((1, 3), 2, 2), (5, 2, 3)):
+        ours = workloads.im2col(fmap, k, pad, stride)
+        ref = F.unfold(torch.from_numpy(fmap).double(), k, padding=pad, stride=stride).transpose(1, 2).numpy()
+        np.testing.assert_array_equal(ours.astype(np.float64), ref)
 
 
 def test_recurrent_per_example_gradient_matches_autograd():

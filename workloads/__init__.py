@@ -164,23 +164,38 @@ def to_bf16_bits(x: np.ndarray) -> np.ndarray:
 # --------------------------------------------------------------------------
 # generators
 # --------------------------------------------------------------------------
-def im2col(fmap: np.ndarray, k: int, pad: int) -> np.ndarray:
-    """(B, C, H, W) -> (B, H*W, C*k*k) patch matrix for a stride-1 k x k
-    convolution with zero padding `pad` (output H x W when pad = (k-1)/2).
-    Column order is (c, ky, kx) with c slowest, matching a convolution
-    weight flattened from [c_out, c_in, k, k]."""
+def im2col(fmap: np.ndarray, k, pad: int, stride: int = 1) -> np.ndarray:
+    """(B, C, H, W) -> (B, H'*W', C*kh*kw) patch matrix of a kh x kw convolution (k = int or (kh, kw)) with
+    zero padding `pad` and stride `stride`; H' = (H + 2 pad - kh) / stride + 1.  Column order is
+    (c, ky, kx) with c slowest, matching a convolution weight flattened from [c_out, c_in, kh, kw]."""
+    kh, kw = (k, k) if isinstance(k, int) else k
     B, C, H, W = fmap.shape
-    Ho, Wo = H + 2 * pad - k + 1, W + 2 * pad - k + 1
+    Ho, Wo = (H + 2 * pad - kh) // stride + 1, (W + 2 * pad - kw) // stride + 1
     padded = np.zeros((B, C, H + 2 * pad, W + 2 * pad), dtype=fmap.dtype)
     padded[:, :, pad:pad + H, pad:pad + W] = fmap
-    out = np.empty((B, Ho * Wo, C * k * k), dtype=fmap.dtype)
+    out = np.empty((B, Ho * Wo, C * kh * kw), dtype=fmap.dtype)
     col = 0
     for c in range(C):
-        for ky in range(k):
-            for kx in range(k):
-                out[:, :, col] = padded[:, c, ky:ky + Ho, kx:kx + Wo].reshape(B, Ho * Wo)
+        for ky in range(kh):
+            for kx in range(kw):
+                out[:, :, col] = padded[:, c, ky:ky + (Ho - 1) * stride + 1:stride,
+                                        kx:kx + (Wo - 1) * stride + 1:stride].reshape(B, Ho * Wo)
                 col += 1
     return out
+
+
+def conv_inputs(rng_seed: int, B: int, C: int, H: int, W: int, k, pad: int, stride: int, d_out: int,
+                dtype: str = "f32", var_z: float = 1.0) -> Tuple[np.ndarray, np.ndarray]:
+    """Inputs of a convolution layer as back-propagation has them: the feature map X (B, C, H, W), ReLU of
+    N(0,1), and Zbar (B, T, d_out) ~ N(0, var_z), T = H' W'."""
+    kh, kw = (k, k) if isinstance(k, int) else k
+    rng = np.random.default_rng([rng_seed, B, C, H, W, kh, kw, pad, stride, d_out])
+    X = np.maximum(rng.standard_normal((B, C, H, W), dtype=np.float32), 0.0)
+    Ho, Wo = (H + 2 * pad - kh) // stride + 1, (W + 2 * pad - kw) // stride + 1
+    Z = rng.standard_normal((B, Ho * Wo, d_out), dtype=np.float32) * np.float32(np.sqrt(var_z))
+    if dtype == "bf16":
+        X, Z = round_to_bf16(X), round_to_bf16(Z)
+    return np.ascontiguousarray(X), np.ascontiguousarray(Z)
 
 
 def _draw_A(rng: np.random.Generator, B: int, spec: LayerSpec) -> np.ndarray:
