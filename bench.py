@@ -407,9 +407,9 @@ def bench_conv_implicit(torch, dp, name, B, C, H, W, k, pad, d_out, dtype, steps
     nbytes = (X.size + Z.size) * es
     flops = 2.0 * B * T * d_in * d_out
     out = dict(workload=name, algorithmic_bytes=int(nbytes), patch_matrix_bytes=int((A.size + Z.size) * es))
-    for kind, fn, ref in (("norm", lambda: dp.dpclip_conv_sqnorms(dX, dZ, k, k, 1, pad, True, sq),
+    for kind, fn, ref in (("norm", lambda: dp.dpclip_conv_sqnorms(dX, dZ, k, k, 1, pad, True, sq, workspace=ws),
                            lambda: dp.dpclip_layer_sqnorms(dA, dZ, True, sq, ws)),
-                          ("grad", lambda: dp.dpclip_conv_clipped_grad(dX, dZ, k, k, 1, pad, clip, gW, gb),
+                          ("grad", lambda: dp.dpclip_conv_clipped_grad(dX, dZ, k, k, 1, pad, clip, gW, gb, workspace=ws),
                            lambda: dp.dpclip_clipped_grad(dA, dZ, clip, gW, gb, ws))):
         ms = float(np.median(time_steps(torch, fn, steps, 3, flush)))
         ms_ref = float(np.median(time_steps(torch, ref, steps, 3, flush)))

@@ -226,15 +226,19 @@ int dpclip_step(const dpclip_layer* layers /* host */, int L, int B, dpclip_dtyp
  *           T = H' * W', H' = (H + 2 pad - kh) / stride + 1, likewise W'
  *   sq_layer, clip, gW, gb  as for dpclip_layer_sqnorms / dpclip_clipped_grad; gW is [d_out][C*kh*kw] with
  *           columns ordered (c, ky, kx), c slowest: a convolution weight [c_out][c_in][kh][kw] flattened
- * Square or rectangular kernels, any stride and zero padding; dilation 1.  fp32-ALU tiles (64 x 64), fp32
- * accumulation; partial sums of split rows are combined with fp32 atomics.  No workspace.  Noise is added
- * with dpclip_add_noise.  Errors as for dpclip_layer_sqnorms. */
+ * Square or rectangular kernels, any stride and zero padding; dilation 1.  fp32 layers with dL/dZ as
+ * [B][T][d_out] (rows 16-byte multiples) above 2^25 multiply-adds run on the tensor cores (error-
+ * compensated tf32, the patch rows gathered by the warps that prepare the operand planes) and need a
+ * workspace of dpclip_workspace_bytes(B, T, C*kh*kw, d_out, ...) bytes; everything else, and any call
+ * with workspace == NULL, runs on fp32-ALU tiles (64 x 64) and combines the partial sums of split rows
+ * with fp32 atomics.  Noise is added with dpclip_add_noise.  Errors as for dpclip_layer_sqnorms. */
 typedef struct { int C, H, W, kh, kw, stride, pad; } dpclip_conv;
 int dpclip_conv_sqnorms(const void* X, const void* Zbar, int z_channel_major, int B, const dpclip_conv* geom,
-                        int d_out, dpclip_dtype dtype, int has_bias, float* sq_layer, void* stream);
+                        int d_out, dpclip_dtype dtype, int has_bias, float* sq_layer,
+                        void* workspace, size_t workspace_bytes, void* stream);
 int dpclip_conv_clipped_grad(const void* X, const void* Zbar, int z_channel_major, int B, const dpclip_conv* geom,
                              int d_out, dpclip_dtype dtype, const float* clip, float* gW, long ldg, float* gb,
-                             void* stream);
+                             void* workspace, size_t workspace_bytes, void* stream);
 
 /* Parameter updates with the noise folded in (one pass over the parameters instead of a noise pass and
  * an optimiser pass).  gsum is the PRE-noise clipped sum of one tensor (run the step with sigma = 0);

@@ -65,9 +65,9 @@ def load_library():
                                             _u64, _vp, _sz, _vp]
     L.dpclip_clipped_grad_noise.restype = _i
     L.dpclip_add_noise.argtypes = [_vp, _sz, _f, _f, _u64, _u64, _vp]
-    L.dpclip_conv_sqnorms.argtypes = [_vp, _vp, _i, _i, ctypes.POINTER(_CConv), _i, _i, _i, _vp, _vp]
+    L.dpclip_conv_sqnorms.argtypes = [_vp, _vp, _i, _i, ctypes.POINTER(_CConv), _i, _i, _i, _vp, _vp, _sz, _vp]
     L.dpclip_conv_sqnorms.restype = _i
-    L.dpclip_conv_clipped_grad.argtypes = [_vp, _vp, _i, _i, ctypes.POINTER(_CConv), _i, _i, _vp, _vp, _l, _vp, _vp]
+    L.dpclip_conv_clipped_grad.argtypes = [_vp, _vp, _i, _i, ctypes.POINTER(_CConv), _i, _i, _vp, _vp, _l, _vp, _vp, _sz, _vp]
     L.dpclip_conv_clipped_grad.restype = _i
     L.dpclip_dp_sgd_step.argtypes = [_vp, _vp, _sz, _f, _f, _f, _u64, _u64, _f, _vp]
     L.dpclip_dp_sgd_step.restype = _i
@@ -405,17 +405,20 @@ def _conv_args(X: torch.Tensor, Zbar: torch.Tensor, kh: int, kw: int, stride: in
 
 
 def dpclip_conv_sqnorms(X: torch.Tensor, Zbar: torch.Tensor, kh: int, kw: int, stride: int, pad: int, has_bias: bool,
-                        sq_layer: torch.Tensor, z_channel_major: bool = False, stream=None) -> None:
+                        sq_layer: torch.Tensor, z_channel_major: bool = False,
+                        workspace: Optional[torch.Tensor] = None, stream=None) -> None:
     B, d_out, geom = _conv_args(X, Zbar, kh, kw, stride, pad, z_channel_major)
     assert sq_layer.dtype == torch.float32 and sq_layer.numel() >= B and sq_layer.is_contiguous()
     _check("dpclip_conv_sqnorms", load_library().dpclip_conv_sqnorms(
         _ptr(X), _ptr(Zbar), int(z_channel_major), B, ctypes.byref(geom), d_out, _dtype_code(X), int(has_bias),
-        _ptr(sq_layer), _stream(stream)))
+        _ptr(sq_layer), _ptr(workspace) if workspace is not None else None,
+        workspace.numel() if workspace is not None else 0, _stream(stream)))
 
 
 def dpclip_conv_clipped_grad(X: torch.Tensor, Zbar: torch.Tensor, kh: int, kw: int, stride: int, pad: int,
                              clip: Optional[torch.Tensor], gW: torch.Tensor, gb: Optional[torch.Tensor],
-                             z_channel_major: bool = False, stream=None) -> None:
+                             z_channel_major: bool = False, workspace: Optional[torch.Tensor] = None,
+                             stream=None) -> None:
     B, d_out, geom = _conv_args(X, Zbar, kh, kw, stride, pad, z_channel_major)
     d_in = X.shape[1] * kh * kw
     assert gW.dtype == torch.float32 and gW.shape == (d_out, d_in) and gW.stride(1) == 1
@@ -423,6 +426,7 @@ def dpclip_conv_clipped_grad(X: torch.Tensor, Zbar: torch.Tensor, kh: int, kw: i
     _check("dpclip_conv_clipped_grad", load_library().dpclip_conv_clipped_grad(
         _ptr(X), _ptr(Zbar), int(z_channel_major), B, ctypes.byref(geom), d_out, _dtype_code(X),
         _ptr(clip) if clip is not None else None, _ptr(gW), gW.stride(0), _ptr(gb) if gb is not None else None,
+        _ptr(workspace) if workspace is not None else None, workspace.numel() if workspace is not None else 0,
         _stream(stream)))
 
 

@@ -443,12 +443,13 @@ bool make_map_f32(CUtensorMap* map, const void* base, long rows, long cols, long
 int launch_zta_tf32(const void* A, long lda, const void* Z, long ldz, int B, int T, int d_in, int d_out,
                     bool norm_mode, int has_bias, const float* clip, float* gW, long ldg, float* gb, float* sq,
                     void* workspace, size_t workspace_bytes, const NoiseSpec* noise, bool* noise_done,
-                    cudaStream_t st) {
+                    cudaStream_t st, const tc::ConvGather* conv = nullptr) {
     namespace t = tc::t32;
     const long R = (long)B * T;
     CUtensorMap ma, mz;
-    if (!make_map_f32(&ma, A, R, d_in, lda, 32, t::BK) || !make_map_f32(&mz, Z, R, d_out, ldz, 32, t::BK))
-        return DPCLIP_ERR_CUDA;
+    if (!make_map_f32(&mz, Z, R, d_out, ldz, 32, t::BK)) return DPCLIP_ERR_CUDA;
+    if (conv) ma = mz;                                       // A is gathered from the feature map: no tensor map for it
+    else if (!make_map_f32(&ma, A, R, d_in, lda, 32, t::BK)) return DPCLIP_ERR_CUDA;
     tc::zta::Params p;
     memset(&p, 0, sizeof(p));
     p.R = (int)R; p.T = T; p.d_in = d_in; p.d_out = d_out;
@@ -485,9 +486,16 @@ int launch_zta_tf32(const void* A, long lda, const void* Z, long ldz, int B, int
             return DPCLIP_ERR_CUDA;
         }
     }
-    if (!enable_smem(tc::zta_tf32_kernel, t::SMEM_BYTES)) return DPCLIP_ERR_CUDA;
     const int grid = p.n_items < kNumSMs ? p.n_items : kNumSMs;
-    tc::zta_tf32_kernel<<<grid, t::THREADS, t::SMEM_BYTES, st>>>(ma, mz, p);
+    if (conv) {
+        if (!enable_smem(tc::zta_tf32_kernel<true>, t::SMEM_BYTES)) return DPCLIP_ERR_CUDA;
+        tc::zta_tf32_kernel<true><<<grid, t::THREADS, t::SMEM_BYTES, st>>>(ma, mz, p, *conv);
+    } else {
+        tc::ConvGather none;
+        memset(&none, 0, sizeof(none));
+        if (!enable_smem(tc::zta_tf32_kernel<false>, t::SMEM_BYTES)) return DPCLIP_ERR_CUDA;
+        tc::zta_tf32_kernel<false><<<grid, t::THREADS, t::SMEM_BYTES, st>>>(ma, mz, p, none);
+    }
     int rc = launch_status();
     if (rc || norm_mode || ksplit == 1) return rc;
     return launch_reduce_partials(p, tiles, ksplit, t::BM, t::BN, d_in, d_out, gW, ldg, gb, noise, noise_done, st);
@@ -887,8 +895,22 @@ static int conv_setup(SimtParams& p, const void* X, const void* Zbar, int z_chan
     return DPCLIP_OK;
 }
 
+// fp32, dL/dZ as [B][T][d_out] with 16-byte rows, enough work: the tensor-core kernel with the A operand gathered
+static bool conv_tf32_ok(const SimtParams& p, const void* X, const void* Zbar, int z_channel_major, int B, int T,
+                         dpclip_dtype dtype, const void* workspace, size_t workspace_bytes, tc::ConvGather* cg) {
+    { const char* env = getenv("DPCLIP_FORCE_SIMT"); if (env && env[0] == '1') return false; }
+    if (dtype != DPCLIP_F32 || z_channel_major || !workspace || workspace_bytes < (size_t)kHeaderBytes) return false;
+    if (!aligned_to(Zbar, 16) || p.d_out % 4 != 0 || p.kh > 255 || p.kw > 255) return false;
+    if ((double)B * T * p.d_in * p.d_out < 32.0 * 1024 * 1024) return false;
+    cg->X = static_cast<const float*>(X);
+    cg->C = p.cC; cg->H = p.cH; cg->W = p.cW; cg->kh = p.kh; cg->kw = p.kw; cg->stride = p.stride; cg->pad = p.pad;
+    cg->Wo = p.Wo;
+    return true;
+}
+
 int dpclip_conv_sqnorms(const void* X, const void* Zbar, int z_channel_major, int B, const dpclip_conv* geom,
-                        int d_out, dpclip_dtype dtype, int has_bias, float* sq_layer, void* stream) {
+                        int d_out, dpclip_dtype dtype, int has_bias, float* sq_layer, void* workspace,
+                        size_t workspace_bytes, void* stream) {
     SimtParams p;
     int T = 0;
     int rc = conv_setup(p, X, Zbar, z_channel_major, B, geom, d_out, dtype, has_bias, &T);
@@ -896,6 +918,10 @@ int dpclip_conv_sqnorms(const void* X, const void* Zbar, int z_channel_major, in
     if (!sq_layer) return DPCLIP_ERR_INVALID_ARG;
     if (B > 65535) return DPCLIP_ERR_UNSUPPORTED;
     cudaStream_t st = (cudaStream_t)stream;
+    tc::ConvGather cg;
+    if (conv_tf32_ok(p, X, Zbar, z_channel_major, B, T, dtype, workspace, workspace_bytes, &cg))
+        return launch_zta_tf32(nullptr, p.d_in, Zbar, d_out, B, T, p.d_in, d_out, true, has_bias, nullptr, nullptr, 0,
+                               nullptr, sq_layer, workspace, workspace_bytes, nullptr, nullptr, st, &cg);
     const int n_tiles = p.tiles_m * p.tiles_n;
     int split = ceil_div(2 * kNumSMs, B);
     if (split > n_tiles) split = n_tiles;
@@ -911,7 +937,7 @@ int dpclip_conv_sqnorms(const void* X, const void* Zbar, int z_channel_major, in
 
 int dpclip_conv_clipped_grad(const void* X, const void* Zbar, int z_channel_major, int B, const dpclip_conv* geom,
                              int d_out, dpclip_dtype dtype, const float* clip, float* gW, long ldg, float* gb,
-                             void* stream) {
+                             void* workspace, size_t workspace_bytes, void* stream) {
     SimtParams p;
     int T = 0;
     int rc = conv_setup(p, X, Zbar, z_channel_major, B, geom, d_out, dtype, gb != nullptr, &T);
@@ -919,6 +945,11 @@ int dpclip_conv_clipped_grad(const void* X, const void* Zbar, int z_channel_majo
     if (!gW || ldg < p.d_in) return DPCLIP_ERR_INVALID_ARG;
     if (!aligned_to(gW, 4) || (gb && !aligned_to(gb, 4))) return DPCLIP_ERR_MISALIGNED;
     cudaStream_t st = (cudaStream_t)stream;
+    tc::ConvGather cg;
+    if (conv_tf32_ok(p, X, Zbar, z_channel_major, B, T, dtype, workspace, workspace_bytes, &cg) &&
+        workspace_bytes >= (size_t)kHeaderBytes + kTcScratchBytes)
+        return launch_zta_tf32(nullptr, p.d_in, Zbar, d_out, B, T, p.d_in, d_out, false, 0, clip, gW, ldg, gb, nullptr,
+                               workspace, workspace_bytes, nullptr, nullptr, st, &cg);
     const int n_tiles = p.tiles_m * p.tiles_n;
     const long rows = (long)B * T;
     long ksplit = ceil_div(4 * kNumSMs, n_tiles);

@@ -62,9 +62,19 @@ __device__ __forceinline__ zta::Item decode(const zta::Params& p, int item) {
 }
 }  // namespace t32
 
+// CONV = true: the layer is a convolution given by its input feature map X [B][C][H][W] (implicit im2col).
+// No TMA for the A operand: the transform warps gather element (row (i, t), column (c, ky, kx)) of the
+// patch matrix from X[i][c][y' stride - pad + ky][x' stride - pad + kx] (zero outside the map) with plain
+// loads, one stage ahead, and write both of its planes in the layout TMA would have produced.
+struct ConvGather {
+    const float* X;
+    int C, H, W, kh, kw, stride, pad, Wo;
+};
+
+template <bool CONV>
 __global__ void __launch_bounds__(t32::THREADS, 1)
 zta_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_z,
-                const zta::Params p) {
+                const zta::Params p, const ConvGather cg) {
     using namespace t32;
     using zta::Item;
     extern __shared__ uint8_t smem_raw[];
@@ -81,7 +91,8 @@ zta_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            mbar_init(&full[s], 1); mbar_init(&ready[s], N_TRANSFORM_WARPS + N_EPILOGUE_WARPS); mbar_init(&empty[s], 1);
+            mbar_init(&full[s], 1); mbar_init(&ready[s], CONV ? N_TRANSFORM_WARPS : N_TRANSFORM_WARPS + N_EPILOGUE_WARPS);
+            mbar_init(&empty[s], 1);
         }
         for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], N_EPILOGUE_WARPS); }
         *abort_flag = 0;
@@ -107,13 +118,15 @@ zta_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     if (!ok) break;
                     uint8_t* dst = smem + stage * STAGE_BYTES;
                     const int y = w.row_begin + kb * BK;
-                    mbar_arrive_expect_tx(&full[stage], 2 * TILE_BYTES);
+                    mbar_arrive_expect_tx(&full[stage], CONV ? TILE_BYTES : 2 * TILE_BYTES);
 #pragma unroll
                     for (int c = 0; c < 4; ++c)
                         tma_load_2d(dst + OFF_Z + c * CHUNK_BYTES, &map_z, &full[stage], w.m0 + c * 32, y);
+                    if (!CONV) {
 #pragma unroll
-                    for (int c = 0; c < 4; ++c)
-                        tma_load_2d(dst + OFF_A + c * CHUNK_BYTES, &map_a, &full[stage], w.n0 + c * 32, y);
+                        for (int c = 0; c < 4; ++c)
+                            tma_load_2d(dst + OFF_A + c * CHUNK_BYTES, &map_a, &full[stage], w.n0 + c * 32, y);
+                    }
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
             }

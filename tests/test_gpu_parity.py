@@ -262,6 +262,8 @@ def test_transformer_block_with_layernorms(dp):
 CONV_CASES = [  # B, C, H, W, k, pad, stride, d_out
     (3, 3, 8, 8, 3, 1, 1, 5), (2, 4, 9, 7, (3, 2), 1, 2, 70), (4, 32, 16, 16, 3, 1, 1, 64), (2, 5, 6, 6, 1, 0, 1, 3),
     (2, 2, 11, 10, 5, 2, 3, 9), (3, 8, 4, 4, 4, 0, 1, 6),
+    # large enough for the tensor-core form (fp32, dL/dZ row-major): ragged tiles, stride, rectangular kernel
+    (8, 32, 16, 16, 3, 1, 1, 64), (64, 16, 20, 18, (3, 2), 1, 2, 72), (3, 40, 30, 30, 3, 0, 1, 132),
 ]
 
 
@@ -279,15 +281,22 @@ def test_conv_implicit_im2col(dp, case, dtype):
     dZcm = dZ.transpose(1, 2).contiguous()                        # [B][d_out][T], the layout of dL/dZ itself
     clip = np.random.default_rng(B).uniform(0.1, 1.0, B).astype(np.float32)
     refW, refb = oracle.clipped_grad(A, Z, clip)
-    for cm, z in ((False, dZ), (True, dZcm)):
+    ws = _ws(dp)
+    # with a workspace the library may take the tensor-core form; without one it stays on the fp32-ALU tiles
+    for cm, z, w in ((False, dZ, ws), (False, dZ, None), (True, dZcm, ws)):
         for has_bias in (True, False):
             ref = oracle.layer_sqnorms(A, Z, has_bias)
             sq = torch.full((B,), -1.0, device="cuda")
-            dp.dpclip_conv_sqnorms(dX, z, kh, kw, stride, pad, has_bias, sq, z_channel_major=cm)
-            assert max_rel(np.sqrt(sq.cpu().numpy()), np.sqrt(ref)) <= tol["norm"]
+            dp.dpclip_conv_sqnorms(dX, z, kh, kw, stride, pad, has_bias, sq, z_channel_major=cm, workspace=w)
+            assert max_rel(np.sqrt(sq.cpu().numpy()), np.sqrt(ref)) <= tol["norm"], (cm, w is None, has_bias)
         gW = torch.full((d_out, C * kh * kw), 3.0, device="cuda"); gb = torch.full((d_out,), 3.0, device="cuda")
-        dp.dpclip_conv_clipped_grad(dX, z, kh, kw, stride, pad, torch.from_numpy(clip).cuda(), gW, gb, z_channel_major=cm)
+        dp.dpclip_conv_clipped_grad(dX, z, kh, kw, stride, pad, torch.from_numpy(clip).cuda(), gW, gb,
+                                    z_channel_major=cm, workspace=w)
         assert rel_fro(gW.cpu().numpy(), refW) <= tol["grad"] and rel_fro(gb.cpu().numpy(), refb) <= tol["grad"]
+        gW.fill_(3.0)
+        dp.dpclip_conv_clipped_grad(dX, z, kh, kw, stride, pad, None, gW, None, z_channel_major=cm, workspace=w)
+        assert rel_fro(gW.cpu().numpy(), oracle.clipped_grad(A, Z, None)[0]) <= tol["grad"]
+    assert dp.dpclip_read_status(ws) == 0
 
 
 # ---------------------------------------------------------------------------
