@@ -413,10 +413,19 @@ def bench_conv_implicit(torch, dp, name, B, C, H, W, k, pad, d_out, dtype, steps
                            lambda: dp.dpclip_clipped_grad(dA, dZ, clip, gW, gb, ws))):
         ms = float(np.median(time_steps(torch, fn, steps, 3, flush)))
         ms_ref = float(np.median(time_steps(torch, ref, steps, 3, flush)))
-        ach = flops / (ms * 1e-3) / 1e12
-        out[kind] = dict(ms=ms, patch_matrix_path_ms=ms_ref,
-                         roofline=dict(bound="alu", achieved=ach, peak=FFMA_PEAK_TFLOPS, unit="TFLOP/s",
-                                       frac=ach / FFMA_PEAK_TFLOPS, traffic=None, peak_source="derived"))
+        # fp32 layers of this size take the tensor-core form (three tf32 MMAs per product); the binding roof is the
+        # larger of bytes / HBM and flops / (3 x tf32)
+        peak_tf = peaks["bf16_tflops"] * TF32X3_PER_BF16 if dtype == "f32" else FFMA_PEAK_TFLOPS
+        t_hbm, t_mma = nbytes / (peaks["hbm_gbs"] * 1e9), flops / (peak_tf * 1e12)
+        if t_hbm >= t_mma:
+            ach = nbytes / (ms * 1e-3) / 1e9
+            roof = dict(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s", frac=ach / peaks["hbm_gbs"])
+        else:
+            ach = flops / (ms * 1e-3) / 1e12
+            roof = dict(bound="tensor" if dtype == "f32" else "alu", achieved=ach, peak=peak_tf, unit="TFLOP/s",
+                        frac=ach / peak_tf)
+        roof.update(traffic=None, peak_source=peaks["source"])
+        out[kind] = dict(ms=ms, patch_matrix_path_ms=ms_ref, roofline=roof)
     return out
 
 
