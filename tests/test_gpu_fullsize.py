@@ -172,3 +172,31 @@ def test_multi_branch_graph_matches_eager_step(dp):
             assert rel_fro(plan.gW[l].cpu().numpy(), eager.gW[l].cpu().numpy()) <= 2e-6
             if plan.gb[l] is not None:
                 assert rel_fro(plan.gb[l].cpu().numpy(), eager.gb[l].cpu().numpy()) <= 2e-6
+
+
+def test_one_launch_step_repeats_bit_for_bit(dp):
+    """The one-launch step crosses a grid-wide barrier whose counter lives in the workspace and resets itself:
+    thousands of back-to-back launches, and launches from two streams at once (own workspaces), must keep
+    giving the same bits and leave the status word clean."""
+    w = workloads.mlp_large()
+    layers = workloads.generate(w, 0)
+    mk = lambda: dp.StepPlan([dp.Layer(to_device(A, w.dtype), to_device(Z, w.dtype), s.has_bias)     # noqa: E731
+                              for (A, Z), s in zip(layers, w.layers)])
+    a, b = mk(), mk()
+    a.run(w.C, w.sigma, 1)
+    torch.cuda.synchronize()
+    ref, ref_clip = a.flat.clone(), a.clip.clone()
+    for it in range(3000):
+        a.run(w.C, w.sigma, 1)
+        if it % 500 == 0:
+            assert torch.equal(a.flat, ref) and torch.equal(a.clip, ref_clip)
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    for it in range(500):
+        with torch.cuda.stream(s1):
+            a.run(w.C, w.sigma, 1)
+        with torch.cuda.stream(s2):
+            b.run(w.C, w.sigma, 1)
+    torch.cuda.synchronize()
+    assert torch.equal(a.flat, ref) and torch.equal(b.flat, ref)
+    assert dp.dpclip_read_status(a.workspace) == 0 and dp.dpclip_read_status(b.workspace) == 0
