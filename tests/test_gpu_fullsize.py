@@ -200,3 +200,26 @@ def test_one_launch_step_repeats_bit_for_bit(dp):
     torch.cuda.synchronize()
     assert torch.equal(a.flat, ref) and torch.equal(b.flat, ref)
     assert dp.dpclip_read_status(a.workspace) == 0 and dp.dpclip_read_status(b.workspace) == 0
+
+
+def test_grid_barrier_timeout_is_reported_and_recoverable(dp):
+    """A grid barrier that cannot complete (its counter in the workspace header is corrupted before the launch,
+    so one arrival is lost) must run into its bounded wait: the kernel returns, the status word says TIMEOUT,
+    the context stays usable, and after dpclip_workspace_init the same plan gives the right answer again."""
+    w = workloads.mlp_small()
+    layers = workloads.generate(w, 0)
+    plan = dp.StepPlan([dp.Layer(to_device(A, w.dtype), to_device(Z, w.dtype), s.has_bias)
+                        for (A, Z), s in zip(layers, w.layers)])
+    plan.run(w.C, w.sigma, 1)
+    torch.cuda.synchronize()
+    good = plan.flat.clone()
+    plan.workspace[64:68].view(torch.int32).fill_(0x7FFFFFFF)      # the barrier counter: the first arrival wraps it to 0
+    plan.run(w.C, w.sigma, 1)
+    torch.cuda.synchronize()                                         # returns after the two-second wait limit
+    assert dp.dpclip_read_status(plan.workspace) == -6               # DPCLIP_ERR_TIMEOUT
+    dp.dpclip_workspace_init(plan.workspace)
+    plan.flat.zero_()
+    plan.run(w.C, w.sigma, 1)
+    torch.cuda.synchronize()
+    assert dp.dpclip_read_status(plan.workspace) == 0
+    assert torch.equal(plan.flat, good)
