@@ -245,16 +245,21 @@ TF32X3_PER_BF16 = (1.1 / 2.25) / 3.0      # nominal tf32 : bf16 dense ratio, thr
 
 
 def roofline_fused_t1(w, step_ms, peaks):
-    """All-T=1 models run inside one dpclip_step call.  fp32 models whose rows TMA can address take the
-    one-launch tensor-core kernel (t1_all_grads_tf32_kernel<true>: norms, factors, clipped sums as
-    error-compensated tf32, noise); others take two launches (t1_all_norms_kernel + t1_all_grads_kernel on
-    the fp32 ALUs).  The kernel time is taken as the whole step's device time, which can only understate it.
-    The contraction peak for fp32-by-3xtf32 is the measured bf16 peak x the nominal tf32:bf16 ratio / 3."""
+    """All-T=1 models run inside one dpclip_step call.  Models whose rows TMA can address take the
+    one-launch tensor-core kernel (t1_all_grads_tf32_kernel<true, T>: norms, factors, clipped sums, noise;
+    fp32 as error-compensated tf32, bf16 as one kind::f16 instruction per 16 rows); others take two launches
+    (t1_all_norms_kernel + t1_all_grads_kernel on the fp32 ALUs).  The kernel time is taken as the whole
+    step's device time, which can only understate it.  The contraction peak for fp32-by-3xtf32 is the
+    measured bf16 peak x the nominal tf32:bf16 ratio / 3; for bf16 it is the measured bf16 peak."""
     flops = sum(2.0 * w.B * s.d_in * s.d_out for s in w.layers)
     nbytes = w.input_bytes() + 4 * w.n_params
-    on_tensor = w.dtype == "f32" and all(s.d_in % 4 == 0 and (s.d_out % 4 == 0 or s.d_out <= 16) for s in w.layers)
+    quantum = 4 if w.dtype == "f32" else 8
+    on_tensor = all(s.d_in % quantum == 0 and (s.d_out % quantum == 0 or s.d_out <= 16) for s in w.layers)
     kernel = "t1_all_grads_tf32_kernel" if on_tensor else "t1_all_grads_kernel"
-    peak_tf = peaks["bf16_tflops"] * TF32X3_PER_BF16 if on_tensor else FFMA_PEAK_TFLOPS
+    if on_tensor:
+        peak_tf = peaks["bf16_tflops"] * (TF32X3_PER_BF16 if w.dtype == "f32" else 1.0)
+    else:
+        peak_tf = FFMA_PEAK_TFLOPS
     t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9)
     t_alu = flops / (peak_tf * 1e12)
     if t_hbm >= t_alu:
@@ -553,7 +558,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="cfg2")
     ap.add_argument("--impl", default="dpclip", choices=["dpclip", "reference"])
-    ap.add_argument("--others", default="cfg1,cfg3_f32,cfg3_bf16,cfg4",
+    ap.add_argument("--others", default="cfg1,cfg2_bf16,cfg3_f32,cfg3_bf16,cfg4",
                     help="further workloads reported under 'workloads' (N=1 only; '' for none)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--points", default="", help="with --sweep: only these points, 'B,T,d_in,d_out;B,T,d_in,d_out;...'")

@@ -521,8 +521,37 @@ int clipped_grad_impl(const void* A, long lda, const void* Zbar, long ldz, int B
 // Second launch of the fused step on the tensor cores (fp32 models).  Every layer must either be addressable
 // by TMA (16-byte aligned base and row stride); the zb of a thin layer (at most 16 outputs) need not be.  Returns 1 when the model
 // does not qualify, so that the caller falls back to the fp32-ALU kernel.
-int launch_fused_t1_tf32(const FusedT1Params& base, bool one_launch, void* workspace, size_t workspace_bytes,
-                         cudaStream_t st) {
+// Alignment that TMA asks of one operand of the fused tensor-core kernels (16-byte base and row stride).
+inline bool t1_tma_ok(const void* ptr, long ld, dpclip_dtype dtype) {
+    return aligned_to(ptr, 16) && ld % (dtype == DPCLIP_BF16 ? 8 : 4) == 0;
+}
+
+template <typename T>
+int launch_fused_t1_tc(tc::f1::Params& q, bool one_launch, int grid, void* workspace, cudaStream_t st) {
+    namespace f = tc::f1;
+    if (one_launch) {
+        // the whole step as one cooperative launch (its CTAs meet at a grid-wide barrier)
+        q.grid_counter = reinterpret_cast<unsigned int*>(static_cast<char*>(workspace) + kGridCounterOffset);
+        if (!enable_smem(tc::t1_all_grads_tf32_kernel<true, T>, f::SMEM_BYTES)) return DPCLIP_ERR_CUDA;
+        cudaLaunchConfig_t cfg;
+        memset(&cfg, 0, sizeof(cfg));
+        cfg.gridDim = dim3(grid); cfg.blockDim = dim3(f::THREADS); cfg.dynamicSmemBytes = f::SMEM_BYTES; cfg.stream = st;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeCooperative; attr.val.cooperative = 1;
+        cfg.attrs = &attr; cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, tc::t1_all_grads_tf32_kernel<true, T>, q) != cudaSuccess) {
+            cudaGetLastError();
+            return 1;                       // cannot be made resident at once: take the two-launch form
+        }
+        return launch_status();
+    }
+    if (!enable_smem(tc::t1_all_grads_tf32_kernel<false, T>, f::SMEM_BYTES)) return DPCLIP_ERR_CUDA;
+    tc::t1_all_grads_tf32_kernel<false, T><<<grid, f::THREADS, f::SMEM_BYTES, st>>>(q);
+    return launch_status();
+}
+
+int launch_fused_t1_tf32(const FusedT1Params& base, bool one_launch, dpclip_dtype dtype, void* workspace,
+                         size_t workspace_bytes, cudaStream_t st) {
     namespace f = tc::f1;
     { const char* env = getenv("DPCLIP_NO_T1_TF32"); if (env && env[0] == '1') return 1; }
     if (!workspace || workspace_bytes < kHeaderBytes) return 1;
@@ -531,17 +560,21 @@ int launch_fused_t1_tf32(const FusedT1Params& base, bool one_launch, void* works
     memset(&q, 0, sizeof(q));
     q.base = base;
     q.status = static_cast<int*>(workspace);
+    const bool bf16 = dtype == DPCLIP_BF16;
     int items = 0, tc_layers = 0;
     for (int l = 0; l < base.L; ++l) {
         const FusedT1Layer& y = base.layer[l];
-        const bool a_ok = aligned_to(y.A, 16) && y.lda % 4 == 0;
-        const bool z_ok = aligned_to(y.Z, 16) && y.ldz % 4 == 0;
         const bool thin = y.d_out <= f::THIN_MAX_OUT;
-        if (!a_ok || !(z_ok || thin)) return 1;
+        if (!t1_tma_ok(y.A, y.lda, dtype) || !(t1_tma_ok(y.Z, y.ldz, dtype) || thin)) return 1;
         q.item_begin[l] = items;
         q.thin[l] = thin ? 1 : 0;
-        if (!make_map_f32(&q.map_a[l], y.A, base.B, y.d_in, y.lda, 32, f::BK)) return DPCLIP_ERR_CUDA;
-        if (!thin && !make_map_f32(&q.map_z[l], y.Z, base.B, y.d_out, y.ldz, 32, f::BK)) return DPCLIP_ERR_CUDA;
+        if (bf16) {
+            if (!make_map_bf16(&q.map_a[l], y.A, base.B, y.d_in, y.lda, 64, f::BK)) return DPCLIP_ERR_CUDA;
+            if (!thin && !make_map_bf16(&q.map_z[l], y.Z, base.B, y.d_out, y.ldz, 64, f::BK)) return DPCLIP_ERR_CUDA;
+        } else {
+            if (!make_map_f32(&q.map_a[l], y.A, base.B, y.d_in, y.lda, 32, f::BK)) return DPCLIP_ERR_CUDA;
+            if (!thin && !make_map_f32(&q.map_z[l], y.Z, base.B, y.d_out, y.ldz, 32, f::BK)) return DPCLIP_ERR_CUDA;
+        }
         q.tiles_n[l] = ceil_div(y.d_in, f::BN);
         items += ceil_div(y.d_out, f::BM) * q.tiles_n[l];
         if (!thin) ++tc_layers;
@@ -549,25 +582,8 @@ int launch_fused_t1_tf32(const FusedT1Params& base, bool one_launch, void* works
     if (!tc_layers) return 1;
     q.total_items = items;
     const int grid = items < kNumSMs ? items : kNumSMs;
-    if (one_launch) {
-        // the whole step as one cooperative launch (its CTAs meet at a grid-wide barrier)
-        q.grid_counter = reinterpret_cast<unsigned int*>(static_cast<char*>(workspace) + kGridCounterOffset);
-        if (!enable_smem(tc::t1_all_grads_tf32_kernel<true>, f::SMEM_BYTES)) return DPCLIP_ERR_CUDA;
-        cudaLaunchConfig_t cfg;
-        memset(&cfg, 0, sizeof(cfg));
-        cfg.gridDim = dim3(grid); cfg.blockDim = dim3(f::THREADS); cfg.dynamicSmemBytes = f::SMEM_BYTES; cfg.stream = st;
-        cudaLaunchAttribute attr;
-        attr.id = cudaLaunchAttributeCooperative; attr.val.cooperative = 1;
-        cfg.attrs = &attr; cfg.numAttrs = 1;
-        if (cudaLaunchKernelEx(&cfg, tc::t1_all_grads_tf32_kernel<true>, q) != cudaSuccess) {
-            cudaGetLastError();
-            return 1;                       // cannot be made resident at once: take the two-launch form
-        }
-        return launch_status();
-    }
-    if (!enable_smem(tc::t1_all_grads_tf32_kernel<false>, f::SMEM_BYTES)) return DPCLIP_ERR_CUDA;
-    tc::t1_all_grads_tf32_kernel<false><<<grid, f::THREADS, f::SMEM_BYTES, st>>>(q);
-    return launch_status();
+    return bf16 ? launch_fused_t1_tc<__nv_bfloat16>(q, one_launch, grid, workspace, st)
+                : launch_fused_t1_tc<float>(q, one_launch, grid, workspace, st);
 }
 
 // One T = 1 layer of the caller's model as the fused kernels see it.  Returns 0, 1 (the layer does not
@@ -603,11 +619,11 @@ int prepare_t1_group(T1Group& g, const dpclip_layer* layers, int L, int B, dpcli
                      unsigned long long seed, unsigned long long stream_id0, float* sq, const float* clip,
                      bool mixed_only = true) {
     g.active = false;
-    if (dtype != DPCLIP_F32 || B > FUSED_MAX_B) return 0;
+    if (B > FUSED_MAX_B) return 0;
     { const char* env = getenv("DPCLIP_NO_FUSED_T1"); if (env && env[0] == '1') return 0; }
     { const char* env = getenv("DPCLIP_NO_T1_TF32"); if (env && env[0] == '1') return 0; }
     memset(&g.p, 0, sizeof(g.p));
-    int n = 0, tiles = 0;
+    int n = 0, tiles = 0, wide = 0;
     for (int l = 0; l < L; ++l) {
         if (layers[l].T != 1) continue;
         if (n == FUSED_MAX_LAYERS) return 0;
@@ -615,12 +631,12 @@ int prepare_t1_group(T1Group& g, const dpclip_layer* layers, int L, int B, dpcli
         if (rc < 0) return rc;
         if (rc) return 0;
         const FusedT1Layer& y = g.p.layer[n];
-        const bool a_ok = aligned_to(y.A, 16) && y.lda % 4 == 0;
-        const bool z_ok = aligned_to(y.Z, 16) && y.ldz % 4 == 0;
-        if (!a_ok || !(z_ok || y.d_out <= tc::f1::THIN_MAX_OUT)) return 0;
+        if (!t1_tma_ok(y.A, y.lda, dtype) || !(t1_tma_ok(y.Z, y.ldz, dtype) || y.d_out <= tc::f1::THIN_MAX_OUT))
+            return 0;
+        if (y.d_out > tc::f1::THIN_MAX_OUT) ++wide;
         ++n;
     }
-    if (n == 0 || (mixed_only && n == L)) return 0;
+    if (n == 0 || wide == 0 || (mixed_only && n == L)) return 0;    // the kernel wants one tensor-core layer
     g.p.L = n; g.p.B = B; g.p.total_tiles = tiles;
     g.p.C = C; g.p.noise_scale = sigma * C;
     g.p.k0 = (uint32_t)seed; g.p.k1 = (uint32_t)(seed >> 32); g.p.stream_id0 = stream_id0;
@@ -654,23 +670,19 @@ int try_fused_t1_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dty
     const int grid_n = rows;
     const int grid_g = tiles < 4 * kNumSMs ? tiles : 4 * kNumSMs;
     const int smem64 = FusedT1Cfg<64>::SMEM_BYTES;
-    if (dtype == DPCLIP_F32) {
-        bool one = true;
-        { const char* env = getenv("DPCLIP_T1_ONE_LAUNCH"); if (env && env[0] == '0') one = false; }
-        if (one) {
-            const int rc = launch_fused_t1_tf32(p, true, workspace, workspace_bytes, st);
-            if (rc <= 0) return rc;
-        }
-        t1_all_norms_kernel<float><<<grid_n, 128, 0, st>>>(p);
-        if (launch_status()) return DPCLIP_ERR_CUDA;
-        const int rc = launch_fused_t1_tf32(p, false, workspace, workspace_bytes, st);
+    bool one = true;
+    { const char* env = getenv("DPCLIP_T1_ONE_LAUNCH"); if (env && env[0] == '0') one = false; }
+    if (one) {
+        const int rc = launch_fused_t1_tf32(p, true, dtype, workspace, workspace_bytes, st);
         if (rc <= 0) return rc;
-        t1_all_grads_kernel<float, 64><<<grid_g, SIMT_THREADS, smem64, st>>>(p);
-    } else {
-        t1_all_norms_kernel<__nv_bfloat16><<<grid_n, 128, 0, st>>>(p);
-        if (launch_status()) return DPCLIP_ERR_CUDA;
-        t1_all_grads_kernel<__nv_bfloat16, 64><<<grid_g, SIMT_THREADS, smem64, st>>>(p);
     }
+    if (dtype == DPCLIP_F32) t1_all_norms_kernel<float><<<grid_n, 128, 0, st>>>(p);
+    else t1_all_norms_kernel<__nv_bfloat16><<<grid_n, 128, 0, st>>>(p);
+    if (launch_status()) return DPCLIP_ERR_CUDA;
+    const int rc = launch_fused_t1_tf32(p, false, dtype, workspace, workspace_bytes, st);
+    if (rc <= 0) return rc;
+    if (dtype == DPCLIP_F32) t1_all_grads_kernel<float, 64><<<grid_g, SIMT_THREADS, smem64, st>>>(p);
+    else t1_all_grads_kernel<__nv_bfloat16, 64><<<grid_g, SIMT_THREADS, smem64, st>>>(p);
     return launch_status();
 }
 
@@ -1022,7 +1034,8 @@ int dpclip_t1_layers_sqnorms(const dpclip_layer* layers, int L, int B, dpclip_dt
     int rc = prepare_t1_group(g, layers, L, B, dtype, 1.f, 0.f, 0, 0, sq_layers, nullptr, /*mixed_only=*/false);
     if (rc) return rc;
     if (!g.active) return DPCLIP_ERR_UNSUPPORTED;
-    t1_all_norms_kernel<float><<<g.p.L * B, 128, 0, (cudaStream_t)stream>>>(g.p);
+    if (dtype == DPCLIP_F32) t1_all_norms_kernel<float><<<g.p.L * B, 128, 0, (cudaStream_t)stream>>>(g.p);
+    else t1_all_norms_kernel<__nv_bfloat16><<<g.p.L * B, 128, 0, (cudaStream_t)stream>>>(g.p);
     return launch_status();
 }
 
@@ -1037,7 +1050,7 @@ int dpclip_t1_layers_clipped_grad_noise(const dpclip_layer* layers, int L, int B
     int rc = prepare_t1_group(g, layers, L, B, dtype, C, sigma, seed, stream_id0, nullptr, clip, /*mixed_only=*/false);
     if (rc) return rc;
     if (!g.active) return DPCLIP_ERR_UNSUPPORTED;
-    rc = launch_fused_t1_tf32(g.p, false, workspace, workspace_bytes, (cudaStream_t)stream);
+    rc = launch_fused_t1_tf32(g.p, false, dtype, workspace, workspace_bytes, (cudaStream_t)stream);
     return rc > 0 ? DPCLIP_ERR_UNSUPPORTED : rc;
 }
 
@@ -1116,7 +1129,8 @@ int dpclip_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, fl
     if (rc) return rc;
     if (t1.active && (!workspace || workspace_bytes < (size_t)kHeaderBytes)) t1.active = false;
     if (t1.active) {
-        t1_all_norms_kernel<float><<<t1.p.L * B, 128, 0, (cudaStream_t)stream>>>(t1.p);
+        if (dtype == DPCLIP_F32) t1_all_norms_kernel<float><<<t1.p.L * B, 128, 0, (cudaStream_t)stream>>>(t1.p);
+        else t1_all_norms_kernel<__nv_bfloat16><<<t1.p.L * B, 128, 0, (cudaStream_t)stream>>>(t1.p);
         if (launch_status()) return DPCLIP_ERR_CUDA;
     }
     for (int l = 0; l < L; ++l) {
@@ -1130,7 +1144,7 @@ int dpclip_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, fl
     rc = dpclip_factors(sq_layers, L, B, B, C, clip, norms, nullptr, stream);
     if (rc) return rc;
     if (t1.active) {
-        rc = launch_fused_t1_tf32(t1.p, false, workspace, workspace_bytes, (cudaStream_t)stream);
+        rc = launch_fused_t1_tf32(t1.p, false, dtype, workspace, workspace_bytes, (cudaStream_t)stream);
         if (rc < 0) return rc;
         if (rc > 0) return DPCLIP_ERR_UNSUPPORTED;           // prepare_t1_group checked the same conditions
     }

@@ -83,37 +83,50 @@ __device__ __forceinline__ float philox_normal(size_t e, unsigned long long sid,
 // Sums of squares of two rows (one of A, one of Zb), taken by one warp.  All loads of a pass (up to
 // eight 128-bit loads per lane and row) are issued before the first value is used: the rows are short and
 // the time is load latency.  Partial sums are returned per lane (warp_sum them).
-__device__ __forceinline__ void warp_rows_sumsq(const float* __restrict__ ra, int na, bool vec_a,
-                                                const float* __restrict__ rz, int nz, bool vec_z, int lane,
+// Four consecutive elements as loaded (conversion is left to the consumer, so that a batch of predicated
+// loads stays a batch of plain load instructions).
+__device__ __forceinline__ float4 load_raw4(const float* p) { return *reinterpret_cast<const float4*>(p); }
+__device__ __forceinline__ uint2 load_raw4(const __nv_bfloat16* p) { return *reinterpret_cast<const uint2*>(p); }
+__device__ __forceinline__ float sumsq_raw4(float4 v) { return (v.x * v.x + v.y * v.y) + (v.z * v.z + v.w * v.w); }
+__device__ __forceinline__ float sumsq_raw4(uint2 r) {
+    const float x = __uint_as_float(r.x << 16), y = __uint_as_float(r.x & 0xFFFF0000u);
+    const float z = __uint_as_float(r.y << 16), w = __uint_as_float(r.y & 0xFFFF0000u);
+    return (x * x + y * y) + (z * z + w * w);
+}
+template <typename T> struct Raw4 { using type = float4; };
+template <> struct Raw4<__nv_bfloat16> { using type = uint2; };
+
+template <typename T>
+__device__ __forceinline__ void warp_rows_sumsq(const T* __restrict__ ra, int na, bool vec_a,
+                                                const T* __restrict__ rz, int nz, bool vec_z, int lane,
                                                 float& sa, float& sz) {
+    using R = typename Raw4<T>::type;
     sa = 0.f; sz = 0.f;
     const int nva = vec_a ? na >> 2 : 0, nvz = vec_z ? nz >> 2 : 0;
     const int passes = (max(nva, nvz) + 255) >> 8;
     for (int ps = 0; ps < passes; ++ps) {
-        float4 va[8], vz[8];
+        R va[8], vz[8];
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
             const int j = (ps << 8) + (u << 5) + lane;
-            va[u] = j < nva ? *reinterpret_cast<const float4*>(ra + 4 * j) : make_float4(0.f, 0.f, 0.f, 0.f);
-            vz[u] = j < nvz ? *reinterpret_cast<const float4*>(rz + 4 * j) : make_float4(0.f, 0.f, 0.f, 0.f);
+            va[u] = R{}; vz[u] = R{};
+            if (j < nva) va[u] = load_raw4(ra + 4 * j);
+            if (j < nvz) vz[u] = load_raw4(rz + 4 * j);
         }
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            sa += (va[u].x * va[u].x + va[u].y * va[u].y) + (va[u].z * va[u].z + va[u].w * va[u].w);
-            sz += (vz[u].x * vz[u].x + vz[u].y * vz[u].y) + (vz[u].z * vz[u].z + vz[u].w * vz[u].w);
-        }
+        for (int u = 0; u < 8; ++u) { sa += sumsq_raw4(va[u]); sz += sumsq_raw4(vz[u]); }
     }
-    // tails, and rows that cannot take 128-bit loads
+    // tails, and rows that cannot take vector loads
     for (int j0 = nva << 2; j0 < na; j0 += 128) {
         float v[4];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) { const int j = j0 + (u << 5) + lane; v[u] = j < na ? ra[j] : 0.f; }
+        for (int u = 0; u < 4; ++u) { const int j = j0 + (u << 5) + lane; v[u] = j < na ? to_f32(ra[j]) : 0.f; }
         sa += (v[0] * v[0] + v[1] * v[1]) + (v[2] * v[2] + v[3] * v[3]);
     }
     for (int j0 = nvz << 2; j0 < nz; j0 += 128) {
         float v[4];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) { const int j = j0 + (u << 5) + lane; v[u] = j < nz ? rz[j] : 0.f; }
+        for (int u = 0; u < 4; ++u) { const int j = j0 + (u << 5) + lane; v[u] = j < nz ? to_f32(rz[j]) : 0.f; }
         sz += (v[0] * v[0] + v[1] * v[1]) + (v[2] * v[2] + v[3] * v[3]);
     }
 }
@@ -152,10 +165,15 @@ __device__ __forceinline__ bool grid_barrier_arrive_and_wait(unsigned int* ctr, 
 //                     once (neither depends on the factors); meanwhile the transform warps take the layer
 //                     norms of the rows dealt to this CTA, meet the other CTAs at a grid-wide barrier,
 //                     rebuild the factors and only then start on the staged tiles.
-template <bool ONE_LAUNCH>
+// T = float: error-compensated tf32 as described above.  T = __nv_bfloat16: the same pipeline with one
+// kind::f16 MMA per K = 16 step and no low planes (products of bf16 inputs are exact in fp32; the only
+// rounding is that of c * zb back to bf16); a stage holds 32 rows as two 64-column boxes per operand.
+template <bool ONE_LAUNCH, typename T = float>
 __global__ void __launch_bounds__(f1::THREADS, 1)
 t1_all_grads_tf32_kernel(const __grid_constant__ f1::Params q) {
     using namespace f1;
+    constexpr bool BF16 = sizeof(T) == 2;
+    constexpr int BOXES = BF16 ? 2 : 4, BOX_COLS = BF16 ? 64 : 32;          // TMA boxes per 128-column tile
     const FusedT1Params& p = q.base;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -173,7 +191,8 @@ t1_all_grads_tf32_kernel(const __grid_constant__ f1::Params q) {
     if (threadIdx.x == 0) {
         DPCLIP_TRACE_AT(0, 255);
         for (int s = 0; s < STAGES; ++s) {
-            mbar_init(&full[s], 1); mbar_init(&ready[s], N_TRANSFORM_WARPS + N_EPILOGUE_WARPS); mbar_init(&empty[s], 1);
+            mbar_init(&full[s], 1); mbar_init(&ready[s], BF16 ? N_TRANSFORM_WARPS : N_TRANSFORM_WARPS + N_EPILOGUE_WARPS);
+            mbar_init(&empty[s], 1);
         }
         for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], N_EPILOGUE_WARPS); }
         *abort_flag = 0;
@@ -221,15 +240,15 @@ t1_all_grads_tf32_kernel(const __grid_constant__ f1::Params q) {
                     if (!ok) break;
                     uint8_t* dst = smem + stage * STAGE_BYTES;
                     DPCLIP_TRACE_AT(0, tr); ++tr;
-                    mbar_arrive_expect_tx(&full[stage], w.thin ? TILE_BYTES : 2 * TILE_BYTES);
+                    mbar_arrive_expect_tx(&full[stage], (w.thin ? 1 : 2) * BOXES * CHUNK_BYTES);
                     if (!w.thin) {
 #pragma unroll
-                        for (int c = 0; c < 4; ++c)
-                            tma_load_2d(dst + OFF_Z + c * CHUNK_BYTES, mz, &full[stage], w.m0 + c * 32, kb * BK);
+                        for (int c = 0; c < BOXES; ++c)
+                            tma_load_2d(dst + OFF_Z + c * CHUNK_BYTES, mz, &full[stage], w.m0 + c * BOX_COLS, kb * BK);
                     }
 #pragma unroll
-                    for (int c = 0; c < 4; ++c)
-                        tma_load_2d(dst + OFF_A + c * CHUNK_BYTES, ma, &full[stage], w.n0 + c * 32, kb * BK);
+                    for (int c = 0; c < BOXES; ++c)
+                        tma_load_2d(dst + OFF_A + c * CHUNK_BYTES, ma, &full[stage], w.n0 + c * BOX_COLS, kb * BK);
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
             }
@@ -237,7 +256,7 @@ t1_all_grads_tf32_kernel(const __grid_constant__ f1::Params q) {
     } else if (warp == 1) {
         // ------------------------------------------------ MMA issuer
         if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc_tf32(BM, BN, 1, 1);
+            constexpr uint32_t idesc = BF16 ? make_idesc_bf16(BM, BN, 1, 1) : make_idesc_tf32(BM, BN, 1, 1);
             int stage = 0; uint32_t phase = 0; int it = 0;
             bool ok = true;
             [[maybe_unused]] int tr = 0;
@@ -259,6 +278,16 @@ t1_all_grads_tf32_kernel(const __grid_constant__ f1::Params q) {
                     tc_fence_after_sync();
                     DPCLIP_TRACE_AT(2, tr); ++tr;
                     const uint32_t base = smem_u32(smem + stage * STAGE_BYTES);
+                    if (BF16) {
+#pragma unroll
+                        for (int k16 = 0; k16 < BK / 16; ++k16) {
+                            // MN-major bf16, 128-byte swizzle: 64-column chunks CHUNK_BYTES apart, 8-row groups
+                            // 1024 bytes apart, 16 rows per K = 16 instruction
+                            const uint64_t dz = make_smem_desc_sw128(base + OFF_Z + k16 * 2048, CHUNK_BYTES, 1024);
+                            const uint64_t da = make_smem_desc_sw128(base + OFF_A + k16 * 2048, CHUNK_BYTES, 1024);
+                            mma_bf16_ss(d_tmem, dz, da, idesc, (window_start && k16 == 0) ? 0u : 1u);
+                        }
+                    } else
 #pragma unroll
                     for (int k8 = 0; k8 < BK / 8; ++k8) {
                         // the raw planes double as the high parts (the low 13 bits are not read)
@@ -277,7 +306,11 @@ t1_all_grads_tf32_kernel(const __grid_constant__ f1::Params q) {
             }
         }
     } else if (warp < 2 + N_TRANSFORM_WARPS) {
+        if constexpr (BF16) {
+#include "kernels_fused_t1_bf16_transform.inc"
+        } else {
 #include "kernels_fused_t1_tf32_transform.inc"
+        }
     } else {
 #include "kernels_fused_t1_tf32_epilogue.inc"
     }

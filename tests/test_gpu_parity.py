@@ -596,6 +596,30 @@ def test_step_mlp_tensor_core_edges(dp):
     _check_step(dp, big, _calibrate(big, layers, 6, big.C), big.C, big.sigma, 6)
 
 
+def test_step_mlp_bf16_tensor_core(dp, monkeypatch):
+    """Fused T=1 step on the tensor cores with bf16 inputs (one kind::f16 instruction per 16 rows, no low
+    planes): the paper-shaped MLPs, ragged tiles with a bias-free layer and a thin head, more tiles than SMs,
+    and the two-launch form."""
+    for w, seed in ((workloads.mlp_small("bf16"), 2), (workloads.mlp_large("bf16", C=1.0), 3)):
+        layers = workloads.generate(w, seed)
+        _check_step(dp, w, _calibrate(w, layers, seed, w.C), w.C, w.sigma, seed)
+    edges = workloads.Workload("mlp_tc_edges_bf16", 200, "bf16",
+                               (workloads.LayerSpec("fc1", 1, 136, 264, True, "normal"),
+                                workloads.LayerSpec("fc2", 1, 264, 40, False, "relu"),
+                                workloads.LayerSpec("fc3", 1, 40, 16, True, "relu"),
+                                workloads.LayerSpec("fc4", 1, 16, 3, True, "relu")), 1.0, 0.9, 1.0 / 200)
+    layers = workloads.generate(edges, 5)
+    _check_step(dp, edges, _calibrate(edges, layers, 5, edges.C), edges.C, edges.sigma, 5)
+    big = workloads.Workload("mlp_tc_many_tiles_bf16", 48, "bf16",
+                             (workloads.LayerSpec("fc1", 1, 1536, 1664, True, "normal"),
+                              workloads.LayerSpec("fc2", 1, 1664, 12, True, "relu")), 1.0, 0.9, 1.0 / 48)
+    layers = workloads.generate(big, 6)
+    _check_step(dp, big, _calibrate(big, layers, 6, big.C), big.C, big.sigma, 6)
+    monkeypatch.setenv("DPCLIP_T1_ONE_LAUNCH", "0")
+    layers = workloads.generate(edges, 7)
+    _check_step(dp, edges, _calibrate(edges, layers, 7, edges.C), edges.C, edges.sigma, 7)
+
+
 def test_narrow_layer_register_staged_form(dp, monkeypatch):
     """fp32 narrow layers normally take the cp.async ring kernel; the register-staged kernel (what bf16 and
     unaligned layers use) must give the same norms and clipped sums on the same fp32 input."""

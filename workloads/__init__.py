@@ -71,7 +71,7 @@ def _dense(name, d_in, d_out, a_dist, bias=True):
 def mlp_small(dtype="f32") -> Workload:
     """MLP 784->256->10, B=32 (two dense layers + biases)."""
     B = 32
-    return Workload("mlp_784_256_10_b32", B, dtype,
+    return Workload("mlp_784_256_10_b32" + ("" if dtype == "f32" else "_" + dtype), B, dtype,
                     (_dense("fc1", 784, 256, "normal"), _dense("fc2", 256, 10, "relu")),
                     C=1.0, sigma=1.1, zbar_var=1.0 / B)
 
@@ -79,7 +79,7 @@ def mlp_small(dtype="f32") -> Workload:
 def mlp_large(dtype="f32", C=1.0) -> Workload:
     """MLP 784->1000->1000->10, B=128 (three dense layers + biases)."""
     B = 128
-    return Workload("mlp_784_1000_1000_10_b128", B, dtype,
+    return Workload("mlp_784_1000_1000_10_b128" + ("" if dtype == "f32" else "_" + dtype), B, dtype,
                     (_dense("fc1", 784, 1000, "normal"), _dense("fc2", 1000, 1000, "relu"),
                      _dense("fc3", 1000, 10, "relu")),
                     C=C, sigma=1.1, zbar_var=1.0 / B)
@@ -136,6 +136,7 @@ def by_name(name: str) -> Workload:
     table = {
         "cfg1": lambda: mlp_small("f32"),
         "cfg2": lambda: mlp_large("f32", 1.0),
+        "cfg2_bf16": lambda: mlp_large("bf16", 1.0),
         "cfg3_f32": lambda: cnn("f32"),
         "cfg3_bf16": lambda: cnn("bf16"),
         "cfg4": lambda: seq("bf16"),
