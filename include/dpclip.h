@@ -207,9 +207,10 @@ typedef struct {
  *   workspace  >= the largest dpclip_workspace_bytes() over the layers
  * Output rows must be dense (ldg == d_in; UNSUPPORTED otherwise) because the
  * noise is indexed by the element's position in the dense tensor.
- * A model whose layers all have T = 1 runs as ONE cooperative launch when it
- * is fp32 with 16-byte-multiple input rows (norms, a grid-wide barrier with a
- * bounded wait, factors, clipped sums on the tensor cores, noise), else as two
+ * A model whose layers all have T = 1 runs as ONE cooperative launch when its
+ * input rows are 16-byte multiples (4 fp32 / 8 bf16 elements; the zb rows of
+ * a layer with at most 16 outputs excepted): norms, a grid-wide barrier with a
+ * bounded wait, factors, clipped sums on the tensor cores, noise; else as two
  * launches; other models run layer by layer, their T = 1 layers together. */
 int dpclip_step(const dpclip_layer* layers /* host */, int L, int B, dpclip_dtype dtype,
                 float C, float sigma, unsigned long long seed, unsigned long long stream_id0,
@@ -269,9 +270,9 @@ int dpclip_step_noise(const dpclip_layer* layers /* host */, int L, float C, flo
  * of the whole model, their clipped sums with the noise (streams stream_id0 + 2l, + 2l + 1 for
  * layer l of the array) in one tensor-core launch.  This is what dpclip_step does for the T = 1
  * layers of a mixed model; the two calls let a caller that spreads the layers of a model over
- * several streams do the same.  fp32 only, input rows 16-byte multiples (the zb rows of a layer
- * with at most 16 outputs excepted), dense output rows: DPCLIP_ERR_UNSUPPORTED otherwise, and
- * nothing is launched. */
+ * several streams do the same.  Input rows must be 16-byte multiples (the zb rows of a layer
+ * with at most 16 outputs excepted), output rows dense, and at least one of the layers must have
+ * more than 16 outputs: DPCLIP_ERR_UNSUPPORTED otherwise, and nothing is launched. */
 int dpclip_t1_layers_supported(const dpclip_layer* layers /* host */, int L, int B, dpclip_dtype dtype); /* 1 or 0 */
 int dpclip_t1_layers_sqnorms(const dpclip_layer* layers /* host */, int L, int B, dpclip_dtype dtype,
                              float* sq_layers, void* stream);
@@ -279,6 +280,37 @@ int dpclip_t1_layers_clipped_grad_noise(const dpclip_layer* layers /* host */, i
                                         const float* clip, float C, float sigma,
                                         unsigned long long seed, unsigned long long stream_id0,
                                         void* workspace, size_t workspace_bytes, void* stream);
+
+/* The layers of a descriptor array whose norms go by the Gram identity (Section "Extension to
+ * recurrent layers" and the attention section: sum over (t, s) of (a_t . a_s)(zb_t . zb_s)), taken
+ * together: bf16 layers with T > 1 whose method is DPCLIP_GRAM, or DPCLIP_AUTO resolving to it,
+ * and whose rows TMA can address, run in ONE launch per eight layers of a kind (the kinds:
+ * T = 256; other T with at most two 128-row blocks per example; longer examples).  Their squared norms go to
+ * THEIR rows of sq_layers [L][B].  taken (host, [L], may be NULL) is set to 1 for every layer
+ * that was handled and to 0 for the others, which the caller passes to dpclip_layer_sqnorms as
+ * before; fewer than two candidates, fp32 input or no workspace: nothing is launched and
+ * nothing is taken.  With a small batch (one example per SM) a single layer's launch is a chain
+ * of exposed latencies; a queue of items per CTA hides them.  The workspace is used for its
+ * status header only. */
+int dpclip_gram_layers_sqnorms(const dpclip_layer* layers /* host */, int L, int B, dpclip_dtype dtype,
+                               float* sq_layers, int* taken /* host, out */,
+                               void* workspace, size_t workspace_bytes, void* stream);
+
+/* Clipped sums with noise (Eq. 1 applied to the sum over examples of c_i Zbar_i^T A_i, Algorithm 1's
+ * last two steps) of layers that have ONE shape, taken together: bf16 layers with T > 1, equal
+ * (T, d_in, d_out), rows TMA can address, dense output rows and d_in a multiple of 4 run as one
+ * tensor-core launch plus one reduce launch per group of two to eight layers (e.g. the four
+ * attention projections of a Transformer block).  Results and noise streams are those of
+ * dpclip_step: layer l of the array draws from streams stream_id0 + 2l (weights) and + 2l + 1
+ * (bias).  taken (host, [L], required) is set to 1 for the layers that were handled; the caller
+ * runs dpclip_clipped_grad_noise on the others.  Nothing qualifies: nothing is launched.  The
+ * launches share `workspace` (one set of partial tiles for the whole group): run them on the
+ * stream that owns it. */
+int dpclip_same_shape_layers_clipped_grad_noise(const dpclip_layer* layers /* host */, int L, int B,
+                                                dpclip_dtype dtype, const float* clip, float C, float sigma,
+                                                unsigned long long seed, unsigned long long stream_id0,
+                                                int* taken /* host, out */,
+                                                void* workspace, size_t workspace_bytes, void* stream);
 
 /* Same, for callers whose tensors live in HOST memory (pinned memory makes the
  * copies asynchronous).  `layers[l].A/Zbar/gW/gb` are HOST pointers with dense

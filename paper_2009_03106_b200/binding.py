@@ -79,6 +79,13 @@ def load_library():
     L.dpclip_t1_layers_supported.restype = _i
     L.dpclip_t1_layers_sqnorms.argtypes = [ctypes.POINTER(_CLayer), _i, _i, _i, _vp, _vp]
     L.dpclip_t1_layers_sqnorms.restype = _i
+    L.dpclip_gram_layers_sqnorms.argtypes = [ctypes.POINTER(_CLayer), _i, _i, _i, _vp, ctypes.POINTER(ctypes.c_int),
+                                             _vp, ctypes.c_size_t, _vp]
+    L.dpclip_gram_layers_sqnorms.restype = _i
+    L.dpclip_same_shape_layers_clipped_grad_noise.argtypes = [
+        ctypes.POINTER(_CLayer), _i, _i, _i, _vp, ctypes.c_float, ctypes.c_float, ctypes.c_ulonglong,
+        ctypes.c_ulonglong, ctypes.POINTER(ctypes.c_int), _vp, ctypes.c_size_t, _vp]
+    L.dpclip_same_shape_layers_clipped_grad_noise.restype = _i
     L.dpclip_t1_layers_clipped_grad_noise.argtypes = [ctypes.POINTER(_CLayer), _i, _i, _i, _vp, _f, _f, _u64, _u64,
                                                       _vp, _sz, _vp]
     L.dpclip_t1_layers_clipped_grad_noise.restype = _i
@@ -366,14 +373,17 @@ class StepPlan:
 
             # the T = 1 layers of a mixed model go together (one launch per stage) when the library takes them
             t1_together = any(y.A.shape[1] == 1 for y in self.layers) and dpclip_t1_layers_supported(self)
-            rest = [(l, y) for l, y in enumerate(self.layers) if not (t1_together and y.A.shape[1] == 1)]
             last = streams[-1]
             fork()
+            # layers whose norms go by the Gram identity share one launch (on the first branch)
+            taken = dpclip_gram_layers_sqnorms(self, self._branch_ws[0])
+            rest = [(l, y) for l, y in enumerate(self.layers) if not (t1_together and y.A.shape[1] == 1)]
             if t1_together:
                 with torch.cuda.stream(last):
                     dpclip_t1_layers_sqnorms(self)
-            for k, (l, y) in enumerate(rest):
-                b = k % branches
+            rest_norms = [(l, y) for l, y in rest if not taken[l]]
+            for k, (l, y) in enumerate(rest_norms):
+                b = (k + (1 if any(taken) else 0)) % branches
                 with torch.cuda.stream(streams[b]):
                     dpclip_layer_sqnorms(y.A, y.Zbar, y.has_bias, self.sq_layers[l], self._branch_ws[b], y.method)
             join()
@@ -382,8 +392,11 @@ class StepPlan:
             if t1_together:
                 with torch.cuda.stream(last):
                     dpclip_t1_layers_clipped_grad_noise(self, C, sigma, seed, stream_id0, self._branch_ws[-1])
+            # layers of one shape share a launch (first branch)
+            grouped = dpclip_same_shape_layers_clipped_grad_noise(self, C, sigma, seed, stream_id0, self._branch_ws[0])
+            rest = [(l, y) for l, y in rest if not grouped[l]]
             for k, (l, y) in enumerate(rest):
-                b = k % branches
+                b = (k + (1 if any(grouped) else 0)) % branches
                 with torch.cuda.stream(streams[b]):
                     dpclip_clipped_grad_noise(y.A, y.Zbar, self.clip, self.gW[l], self.gb[l], sigma, C, seed,
                                               stream_id0 + 2 * l, stream_id0 + 2 * l + 1, self._branch_ws[b])
@@ -464,6 +477,27 @@ def dpclip_t1_layers_clipped_grad_noise(plan: StepPlan, C: float, sigma: float, 
     _check("dpclip_t1_layers_clipped_grad_noise", load_library().dpclip_t1_layers_clipped_grad_noise(
         plan._c, plan.L, plan.B, plan.dtype_code, _ptr(plan.clip), C, sigma, seed, stream_id0, _ptr(ws), ws.numel(),
         _stream(stream)))
+
+
+def dpclip_gram_layers_sqnorms(plan: StepPlan, workspace: Optional[torch.Tensor] = None, stream=None) -> List[bool]:
+    """Norms of the plan's Gram-method layers in one launch; returns which layers were taken."""
+    ws = plan.workspace if workspace is None else workspace
+    taken = (ctypes.c_int * plan.L)()
+    _check("dpclip_gram_layers_sqnorms", load_library().dpclip_gram_layers_sqnorms(
+        plan._c, plan.L, plan.B, plan.dtype_code, _ptr(plan.sq_layers), taken, _ptr(ws), ws.numel(), _stream(stream)))
+    return [bool(t) for t in taken]
+
+
+def dpclip_same_shape_layers_clipped_grad_noise(plan: StepPlan, C: float, sigma: float, seed: int, stream_id0: int = 0,
+                                                workspace: Optional[torch.Tensor] = None, stream=None) -> List[bool]:
+    """Clipped sums + noise of the plan's same-shape layer groups, one launch per group; returns which
+    layers were taken."""
+    ws = plan.workspace if workspace is None else workspace
+    taken = (ctypes.c_int * plan.L)()
+    _check("dpclip_same_shape_layers_clipped_grad_noise", load_library().dpclip_same_shape_layers_clipped_grad_noise(
+        plan._c, plan.L, plan.B, plan.dtype_code, _ptr(plan.clip), C, sigma, seed, stream_id0, taken, _ptr(ws),
+        ws.numel(), _stream(stream)))
+    return [bool(t) for t in taken]
 
 
 def dpclip_t1_layers_supported(plan: StepPlan) -> bool:

@@ -268,36 +268,104 @@ bool enable_smem(K kernel, int bytes) {
     return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
 }
 
-int launch_gram_norms(const void* A, long lda, const void* Z, long ldz, int B, int T, int d_in, int d_out,
-                      int has_bias, float* sq, int* status, cudaStream_t st) {
+// One layer of a Gram-norm launch.
+struct GramLayer {
+    const void* A; long lda; const void* Z; long ldz;
+    int B, T, d_in, d_out, has_bias;
+    float* sq;
+};
+
+// every item is on the diagonal when an example spans at most two aligned row blocks
+inline bool gram_diag_only(int T) {
     namespace g = tc::gram;
-    const long R = (long)B * T;
-    CUtensorMap ma, mz;
-    if (!make_map_bf16(&ma, A, R, d_in, lda, g::BK, g::BM) || !make_map_bf16(&mz, Z, R, d_out, ldz, g::BK, g::BM))
-        return DPCLIP_ERR_CUDA;
-    g::Params p;
-    memset(&p, 0, sizeof(p));
-    p.R = (int)R; p.T = T; p.d_in = d_in; p.d_out = d_out; p.has_bias = has_bias ? 1 : 0;
-    p.sq = sq; p.status = status;
-    if (T % g::BM == 0) {
-        p.dense = 1; p.q = T / g::BM;
-        p.n_groups = B;                       // one example per group
-    } else {
-        p.dense = 0;
-        p.n_groups = ceil_div(R, g::BM);      // one 128-row block per group
+    return (T % g::BM == 0 && T <= 2 * g::BM) || (g::BM % T == 0);
+}
+
+// Which Gram kernel a layer takes; layers of one class can share a launch.
+//   0: examples of exactly two row blocks (their own kernel: one HBM pass per example)
+//   1: other layers whose items all sit on the diagonal (stages of two tiles, six of them)
+//   2: the rest
+inline int gram_class(int T) {
+    { const char* env = getenv("DPCLIP_NO_GRAM_Q2"); if (env && env[0] == '1') return gram_diag_only(T) ? 1 : 2; }
+    if (T == 2 * tc::gram::BM) return 0;
+    return gram_diag_only(T) ? 1 : 2;
+}
+
+// Norms of up to gram::MAX_LAYERS layers by the Gram identity in ONE launch.  All layers must agree on
+// gram_class(T).  Layers go in descending order of bytes per group, so that the round-robin deal
+// leaves the small items for the end of every CTA's queue.
+int launch_gram_group(const GramLayer* ls, int n, int* status, cudaStream_t st) {
+    namespace g = tc::gram;
+    if (n <= 0 || n > g::MAX_LAYERS) return DPCLIP_ERR_INVALID_ARG;
+    int order[g::MAX_LAYERS];
+    for (int i = 0; i < n; ++i) order[i] = i;
+    auto cost = [&](int i) {
+        const long rows = ls[i].T % g::BM == 0 ? ls[i].T : g::BM;
+        return rows * (long)(ls[i].d_in + ls[i].d_out);
+    };
+    for (int i = 1; i < n; ++i)                       // insertion sort, stable
+        for (int j = i; j > 0 && cost(order[j]) > cost(order[j - 1]); --j) { const int t = order[j]; order[j] = order[j - 1]; order[j - 1] = t; }
+    static_assert(sizeof(g::Launch) <= 4096, "kernel parameter space");
+    g::Launch q;
+    memset(&q, 0, sizeof(q));
+    q.L = n; q.status = status;
+    const int cls = gram_class(ls[0].T);
+    int groups = 0;
+    for (int k = 0; k < n; ++k) {
+        const GramLayer& y = ls[order[k]];
+        if (gram_class(y.T) != cls) return DPCLIP_ERR_INVALID_ARG;
+        const long R = (long)y.B * y.T;
+        if (!make_map_bf16(&q.map_a[k], y.A, R, y.d_in, y.lda, g::BK, g::BM) ||
+            !make_map_bf16(&q.map_z[k], y.Z, R, y.d_out, y.ldz, g::BK, g::BM))
+            return DPCLIP_ERR_CUDA;
+        g::Params& p = q.layer[k];
+        p.R = (int)R; p.T = y.T; p.d_in = y.d_in; p.d_out = y.d_out; p.has_bias = y.has_bias ? 1 : 0;
+        p.sq = y.sq;
+        if (y.T % g::BM == 0) {
+            p.dense = 1; p.q = y.T / g::BM;
+            p.n_groups = y.B;                     // one example per group
+        } else {
+            p.dense = 0;
+            p.n_groups = ceil_div(R, g::BM);      // one 128-row block per group
+        }
+        q.group_begin[k] = groups;
+        groups += p.n_groups;
     }
-    if (cudaMemsetAsync(sq, 0, sizeof(float) * (size_t)B, st) != cudaSuccess) return DPCLIP_ERR_CUDA;
-    const int grid = p.n_groups < kNumSMs ? p.n_groups : kNumSMs;
-    // every item is on the diagonal when an example spans at most two aligned row blocks
-    const bool diag_only = (T % g::BM == 0 && T <= 2 * g::BM) || (g::BM % T == 0);
-    if (diag_only) {
+    // the kernel accumulates with atomics: clear the rows, adjacent rows of sq in one memset
+    {
+        int by_ptr[g::MAX_LAYERS];
+        for (int i = 0; i < n; ++i) by_ptr[i] = i;
+        for (int i = 1; i < n; ++i)
+            for (int j = i; j > 0 && ls[by_ptr[j]].sq < ls[by_ptr[j - 1]].sq; --j) { const int t = by_ptr[j]; by_ptr[j] = by_ptr[j - 1]; by_ptr[j - 1] = t; }
+        for (int i = 0; i < n;) {
+            float* begin = ls[by_ptr[i]].sq;
+            float* end = begin + ls[by_ptr[i]].B;
+            int j = i + 1;
+            while (j < n && ls[by_ptr[j]].sq == end) { end += ls[by_ptr[j]].B; ++j; }
+            if (cudaMemsetAsync(begin, 0, sizeof(float) * (size_t)(end - begin), st) != cudaSuccess) return DPCLIP_ERR_CUDA;
+            i = j;
+        }
+    }
+    q.group_begin[n] = groups;
+    q.total_groups = groups;
+    const int grid = groups < kNumSMs ? groups : kNumSMs;
+    if (cls == 0) {
+        if (!enable_smem(tc::gram_norm_q2_kernel, g::SMEM_BYTES)) return DPCLIP_ERR_CUDA;
+        tc::gram_norm_q2_kernel<<<grid, g::THREADS, g::SMEM_BYTES, st>>>(q);
+    } else if (cls == 1) {
         if (!enable_smem(tc::gram_norm_kernel<true>, g::SMEM_BYTES)) return DPCLIP_ERR_CUDA;
-        tc::gram_norm_kernel<true><<<grid, g::THREADS, g::SMEM_BYTES, st>>>(ma, mz, p);
+        tc::gram_norm_kernel<true><<<grid, g::THREADS, g::SMEM_BYTES, st>>>(q);
     } else {
         if (!enable_smem(tc::gram_norm_kernel<false>, g::SMEM_BYTES)) return DPCLIP_ERR_CUDA;
-        tc::gram_norm_kernel<false><<<grid, g::THREADS, g::SMEM_BYTES, st>>>(ma, mz, p);
+        tc::gram_norm_kernel<false><<<grid, g::THREADS, g::SMEM_BYTES, st>>>(q);
     }
     return launch_status();
+}
+
+int launch_gram_norms(const void* A, long lda, const void* Z, long ldz, int B, int T, int d_in, int d_out,
+                      int has_bias, float* sq, int* status, cudaStream_t st) {
+    const GramLayer y = {A, lda, Z, ldz, B, T, d_in, d_out, has_bias, sq};
+    return launch_gram_group(&y, 1, status, st);
 }
 
 // Largest scratch the split-row clipped sum can ask for: one partial tile per item, at most one
@@ -305,11 +373,26 @@ int launch_gram_norms(const void* A, long lda, const void* Z, long ldz, int B, i
 constexpr size_t kTcScratchBytes = (size_t)kNumSMs * 256 * 256 * 4 + (size_t)2 * kNumSMs * 256 * 4;
 
 // second stage of a split-row clipped sum: fixed-order sum of the partial tiles (+ optional noise)
+// Layers of one shape that share a clipped-sum launch (n == 0: a single layer).
+struct GradGroup {
+    int n;
+    float* gW[tc::zta::MAX_LAYERS]; float* gb[tc::zta::MAX_LAYERS];
+    unsigned long long sid_w[tc::zta::MAX_LAYERS], sid_b[tc::zta::MAX_LAYERS];
+};
+
 int launch_reduce_partials(const tc::zta::Params& p, int tiles, int ksplit, int BM, int BN, int d_in, int d_out,
                            float* gW, long ldg, float* gb, const NoiseSpec* noise, bool* noise_done,
-                           cudaStream_t st) {
+                           cudaStream_t st, const GradGroup* grp = nullptr) {
     tc::ReduceParams r;
     memset(&r, 0, sizeof(r));
+    if (grp && grp->n > 0) {
+        r.n_layers = grp->n; r.tiles_layer = tiles / grp->n;
+        for (int l = 0; l < grp->n; ++l) {
+            r.gW_l[l] = grp->gW[l]; r.gb_l[l] = grp->gb[l];
+            r.sw0_l[l] = (uint32_t)grp->sid_w[l]; r.sw1_l[l] = (uint32_t)(grp->sid_w[l] >> 32);
+            r.sb0_l[l] = (uint32_t)grp->sid_b[l]; r.sb1_l[l] = (uint32_t)(grp->sid_b[l] >> 32);
+        }
+    }
     r.part = p.part; r.bias_part = p.bias_part;
     r.n_tiles = tiles; r.tiles_n = p.tiles_n; r.ksplit = ksplit; r.BM = BM; r.BN = BN;
     r.d_out = d_out; r.d_in = d_in; r.gW = gW; r.ldg = ldg; r.gb = gb; r.vec_ok = p.vec_ok;
@@ -327,21 +410,23 @@ int launch_reduce_partials(const tc::zta::Params& p, int tiles, int ksplit, int 
     r.lanes = lanes;
     long blocks = (n_vec + (256 / lanes) - 1) / (256 / lanes);
     if (blocks > 8L * kNumSMs) blocks = 8L * kNumSMs;
-    tc::reduce_partials_kernel<<<(unsigned)blocks, 256, 0, st>>>(r);
+    tc::reduce_partials_kernel<<<dim3((unsigned)blocks, r.n_layers > 0 ? r.n_layers : 1), 256, 0, st>>>(r);
     return launch_status();
 }
 
 // Tile shape: 256 x 256 (MT = 2) cuts the L2->SM traffic per flop by a third but has a single
 // accumulator buffer; it pays once d_out spans at least two 128-row sub-tiles.
 template <int MT>
-int launch_zta_tc_mt(const CUtensorMap& ma, const CUtensorMap& mz, tc::zta::Params p, int B, bool norm_mode,
+int launch_zta_tc_mt(const tc::zta::Maps& maps, tc::zta::Params p, int B, bool norm_mode,
                      float* gW, long ldg, float* gb, float* sq, int d_in, int d_out, void* workspace,
                      size_t workspace_bytes, const NoiseSpec* noise, bool* noise_done, cudaStream_t st,
-                     bool fit_to_workspace = false) {
+                     bool fit_to_workspace = false, const GradGroup* grp = nullptr) {
     namespace z = tc::zta;
     constexpr int BM = z::Cfg<MT>::BM;
     const long R = p.R;
-    p.tiles_m = ceil_div(d_out, BM); p.tiles_n = ceil_div(d_in, z::BN);
+    p.tiles_m_layer = ceil_div(d_out, BM);
+    p.tiles_m = p.tiles_m_layer * (grp && grp->n > 0 ? grp->n : 1);
+    p.tiles_n = ceil_div(d_in, z::BN);
     const int tiles = p.tiles_m * p.tiles_n;
     int ksplit = 1;
     if (norm_mode) {
@@ -365,6 +450,7 @@ int launch_zta_tc_mt(const CUtensorMap& ma, const CUtensorMap& mz, tc::zta::Para
         p.kb_per_split = ceil_div(nkb, ksplit);
         ksplit = ceil_div(nkb, p.kb_per_split);
         p.n_items = tiles * ksplit;
+        if (grp && grp->n > 0 && ksplit == 1) return 1;        // a group's outputs go through the partial tiles
         if (ksplit > 1) {
             const size_t part_bytes = (size_t)p.n_items * BM * z::BN * 4;
             const size_t bias_bytes = gb ? (size_t)p.n_items * BM * 4 : 0;
@@ -377,11 +463,11 @@ int launch_zta_tc_mt(const CUtensorMap& ma, const CUtensorMap& mz, tc::zta::Para
     }
     if (!enable_smem(tc::zta_tc_kernel<MT>, z::SMEM_BYTES)) return DPCLIP_ERR_CUDA;
     const int grid = p.n_items < kNumSMs ? p.n_items : kNumSMs;
-    tc::zta_tc_kernel<MT><<<grid, z::THREADS, z::SMEM_BYTES, st>>>(ma, mz, p);
+    tc::zta_tc_kernel<MT><<<grid, z::THREADS, z::SMEM_BYTES, st>>>(maps, p);
     int rc = launch_status();
     if (rc || norm_mode || ksplit == 1) return rc;
 
-    return launch_reduce_partials(p, tiles, ksplit, BM, z::BN, d_in, d_out, gW, ldg, gb, noise, noise_done, st);
+    return launch_reduce_partials(p, tiles, ksplit, BM, z::BN, d_in, d_out, gW, ldg, gb, noise, noise_done, st, grp);
 }
 
 int launch_zta_tc(const void* A, long lda, const void* Z, long ldz, int B, int T, int d_in, int d_out,
@@ -390,8 +476,8 @@ int launch_zta_tc(const void* A, long lda, const void* Z, long ldz, int B, int T
                   cudaStream_t st, bool fit_to_workspace = false) {
     namespace z = tc::zta;
     const long R = (long)B * T;
-    CUtensorMap ma, mz;
-    if (!make_map_bf16(&ma, A, R, d_in, lda, 64, z::BK) || !make_map_bf16(&mz, Z, R, d_out, ldz, 64, z::BK))
+    z::Maps maps;
+    if (!make_map_bf16(&maps.a[0], A, R, d_in, lda, 64, z::BK) || !make_map_bf16(&maps.z[0], Z, R, d_out, ldz, 64, z::BK))
         return DPCLIP_ERR_CUDA;
     z::Params p;
     memset(&p, 0, sizeof(p));
@@ -411,10 +497,56 @@ int launch_zta_tc(const void* A, long lda, const void* Z, long ldz, int B, int T
     if (env && env[0] == '1') mt = 1;
     if (env && env[0] == '2') mt = 2;
     if (mt == 2)
-        return launch_zta_tc_mt<2>(ma, mz, p, B, norm_mode, gW, ldg, gb, sq, d_in, d_out, workspace, workspace_bytes,
+        return launch_zta_tc_mt<2>(maps, p, B, norm_mode, gW, ldg, gb, sq, d_in, d_out, workspace, workspace_bytes,
                                    noise, noise_done, st, fit_to_workspace);
-    return launch_zta_tc_mt<1>(ma, mz, p, B, norm_mode, gW, ldg, gb, sq, d_in, d_out, workspace, workspace_bytes,
+    return launch_zta_tc_mt<1>(maps, p, B, norm_mode, gW, ldg, gb, sq, d_in, d_out, workspace, workspace_bytes,
                                noise, noise_done, st, fit_to_workspace);
+}
+
+// Clipped sums (+ noise) of n layers of ONE shape in one tensor-core launch and one reduce launch.
+// Returns 1 when the group does not qualify (the caller then goes layer by layer).
+int launch_zta_tc_group(const dpclip_layer* const* ls, const int* index, int n, int B, const float* clip,
+                        float noise_scale, unsigned long long seed, unsigned long long stream_id0,
+                        void* workspace, size_t workspace_bytes, cudaStream_t st) {
+    namespace z = tc::zta;
+    if (n < 2 || n > z::MAX_LAYERS) return 1;
+    const dpclip_layer& y0 = *ls[0];
+    const long R = (long)B * y0.T;
+    z::Maps maps;
+    GradGroup grp;
+    memset(&grp, 0, sizeof(grp));
+    grp.n = n;
+    float* any_gb = nullptr;
+    bool vec_ok = true;
+    for (int l = 0; l < n; ++l) {
+        const dpclip_layer& y = *ls[l];
+        if (!make_map_bf16(&maps.a[l], y.A, R, y.d_in, y.lda, 64, z::BK) ||
+            !make_map_bf16(&maps.z[l], y.Zbar, R, y.d_out, y.ldz, 64, z::BK))
+            return DPCLIP_ERR_CUDA;
+        grp.gW[l] = y.gW; grp.gb[l] = y.has_bias ? y.gb : nullptr;
+        grp.sid_w[l] = stream_id0 + 2ull * index[l]; grp.sid_b[l] = grp.sid_w[l] + 1;
+        if (grp.gb[l]) any_gb = grp.gb[l];
+        vec_ok = vec_ok && aligned_to(y.gW, 16);
+    }
+    z::Params p;
+    memset(&p, 0, sizeof(p));
+    p.R = (int)R; p.T = y0.T; p.d_in = y0.d_in; p.d_out = y0.d_out;
+    p.status = static_cast<int*>(workspace);
+    p.clip = clip; p.gW = y0.gW; p.ldg = y0.d_in; p.gb = any_gb;
+    p.do_bias = any_gb ? 1 : 0;
+    p.vec_ok = vec_ok && y0.d_in % 4 == 0;
+    const NoiseSpec ns = {noise_scale, seed, 0, 0};             // the streams come from the group
+    bool noise_done = false;
+    int rc;
+    if (y0.d_out > 128)
+        rc = launch_zta_tc_mt<2>(maps, p, B, false, y0.gW, y0.d_in, any_gb, nullptr, y0.d_in, y0.d_out, workspace,
+                                 workspace_bytes, &ns, &noise_done, st, false, &grp);
+    else
+        rc = launch_zta_tc_mt<1>(maps, p, B, false, y0.gW, y0.d_in, any_gb, nullptr, y0.d_in, y0.d_out, workspace,
+                                 workspace_bytes, &ns, &noise_done, st, false, &grp);
+    if (rc) return rc;
+    if (noise_scale > 0.f && !noise_done) return DPCLIP_ERR_UNSUPPORTED;     // the caller checked d_in % 4
+    return DPCLIP_OK;
 }
 
 // fp32 layers on the tensor cores (error-compensated tf32): TMA needs 16-byte aligned bases and rows
@@ -803,6 +935,86 @@ int dpclip_layer_sqnorms(const void* A, long lda, const void* Zbar, long ldz, in
     }
 }
 
+int dpclip_gram_layers_sqnorms(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, float* sq_layers,
+                               int* taken, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!layers || L <= 0 || B <= 0 || !sq_layers) return DPCLIP_ERR_INVALID_ARG;
+    if (taken) for (int l = 0; l < L; ++l) taken[l] = 0;
+    if (dtype != DPCLIP_BF16 || !workspace || workspace_bytes < (size_t)kHeaderBytes) return DPCLIP_OK;
+    { const char* env = getenv("DPCLIP_NO_GRAM_GROUP"); if (env && env[0] == '1') return DPCLIP_OK; }
+    namespace g = tc::gram;
+    for (int cls = 0; cls < 3; ++cls) {                    // one launch per kernel class (see gram_class)
+        GramLayer batch[g::MAX_LAYERS];
+        int idx[g::MAX_LAYERS];
+        int n = 0;
+        auto flush = [&]() -> int {
+            // a single layer gains nothing from this entry point: leave it to the per-layer call
+            if (n >= 2) {
+                const int rc = launch_gram_group(batch, n, (int*)workspace, (cudaStream_t)stream);
+                if (rc) return rc;
+                if (taken) for (int i = 0; i < n; ++i) taken[idx[i]] = 1;
+            }
+            n = 0;
+            return DPCLIP_OK;
+        };
+        for (int l = 0; l < L; ++l) {
+            const dpclip_layer& y = layers[l];
+            if (y.T <= 1 || gram_class(y.T) != cls) continue;
+            if (check_layer_args(y.A, y.lda, y.Zbar, y.ldz, B, y.T, y.d_in, y.d_out, dtype)) continue;
+            if (!tc_eligible(y.A, y.lda, y.Zbar, y.ldz, dtype)) continue;
+            int method = y.method;
+            if (method == DPCLIP_AUTO) method = dpclip_pick_method(B, y.T, y.d_in, y.d_out, y.lda, y.ldz, dtype);
+            if (method != DPCLIP_GRAM) continue;
+            batch[n] = {y.A, y.lda, y.Zbar, y.ldz, B, y.T, y.d_in, y.d_out, y.has_bias ? 1 : 0, sq_layers + (size_t)l * B};
+            idx[n] = l;
+            if (++n == g::MAX_LAYERS) { const int rc = flush(); if (rc) return rc; }
+        }
+        const int rc = flush();
+        if (rc) return rc;
+    }
+    return DPCLIP_OK;
+}
+
+int dpclip_same_shape_layers_clipped_grad_noise(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype,
+                                                const float* clip, float C, float sigma, unsigned long long seed,
+                                                unsigned long long stream_id0, int* taken, void* workspace,
+                                                size_t workspace_bytes, void* stream) {
+    if (!layers || L <= 0 || B <= 0) return DPCLIP_ERR_INVALID_ARG;
+    if (!(C >= 0.f) || !(sigma >= 0.f)) return DPCLIP_ERR_INVALID_ARG;
+    if (taken) for (int l = 0; l < L; ++l) taken[l] = 0;
+    if (dtype != DPCLIP_BF16 || !workspace || workspace_bytes < (size_t)kHeaderBytes) return DPCLIP_OK;
+    { const char* env = getenv("DPCLIP_NO_GRAD_GROUP"); if (env && env[0] == '1') return DPCLIP_OK; }
+    namespace z = tc::zta;
+    constexpr int kMaxTracked = 256;
+    if (L > kMaxTracked) return DPCLIP_OK;
+    bool done[kMaxTracked] = {false};
+    auto candidate = [&](const dpclip_layer& y) {
+        if (y.T <= 1 || !y.gW || y.ldg != y.d_in || y.d_in % 4 != 0 || (y.has_bias && !y.gb)) return false;
+        if (check_layer_args(y.A, y.lda, y.Zbar, y.ldz, B, y.T, y.d_in, y.d_out, dtype)) return false;
+        if (!aligned_to(y.gW, 4) || (y.has_bias && !aligned_to(y.gb, 4))) return false;
+        return tc_eligible(y.A, y.lda, y.Zbar, y.ldz, dtype);
+    };
+    for (int l0 = 0; l0 < L; ++l0) {
+        if (done[l0] || !candidate(layers[l0])) continue;
+        const dpclip_layer* grp[z::MAX_LAYERS];
+        int idx[z::MAX_LAYERS];
+        int n = 0;
+        for (int l = l0; l < L && n < z::MAX_LAYERS; ++l) {
+            const dpclip_layer& y = layers[l];
+            if (done[l] || y.T != layers[l0].T || y.d_in != layers[l0].d_in || y.d_out != layers[l0].d_out) continue;
+            if (!candidate(y)) continue;
+            grp[n] = &y; idx[n] = l; ++n;
+        }
+        for (int i = 0; i < n; ++i) done[idx[i]] = true;
+        if (n < 2) continue;
+        const int rc = launch_zta_tc_group(grp, idx, n, B, clip, sigma * C, seed, stream_id0, workspace, workspace_bytes,
+                                           (cudaStream_t)stream);
+        if (rc < 0) return rc;
+        if (rc == 0 && taken) for (int i = 0; i < n; ++i) taken[idx[i]] = 1;
+        if (rc == 0 && !taken) return DPCLIP_ERR_INVALID_ARG;     // without `taken` the caller cannot know
+    }
+    return DPCLIP_OK;
+}
+
 int dpclip_factors(const float* sq_layers, int L, long ld_sq, int B, float C, float* clip, float* norms,
                    int* n_clipped, void* stream) {
     if (!sq_layers || !clip) return DPCLIP_ERR_INVALID_ARG;
@@ -1133,9 +1345,16 @@ int dpclip_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, fl
         else t1_all_norms_kernel<__nv_bfloat16><<<t1.p.L * B, 128, 0, (cudaStream_t)stream>>>(t1.p);
         if (launch_status()) return DPCLIP_ERR_CUDA;
     }
+    int in_gram_group[64];
+    const bool track = L <= 64;
+    if (track) {
+        rc = dpclip_gram_layers_sqnorms(layers, L, B, dtype, sq_layers, in_gram_group, workspace, workspace_bytes, stream);
+        if (rc) return rc;
+    }
     for (int l = 0; l < L; ++l) {
         const dpclip_layer& y = layers[l];
         if (t1.active && y.T == 1) continue;
+        if (track && in_gram_group[l]) continue;
         rc = dpclip_layer_sqnorms(y.A, y.lda, y.Zbar, y.ldz, B, y.T, y.d_in, y.d_out, dtype, y.has_bias,
                                   (dpclip_method)y.method, sq_layers + (size_t)l * B, workspace,
                                   workspace_bytes, stream);
@@ -1148,9 +1367,16 @@ int dpclip_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, fl
         if (rc < 0) return rc;
         if (rc > 0) return DPCLIP_ERR_UNSUPPORTED;           // prepare_t1_group checked the same conditions
     }
+    int in_grad_group[64];
+    if (track) {
+        rc = dpclip_same_shape_layers_clipped_grad_noise(layers, L, B, dtype, clip, C, sigma, seed, stream_id0,
+                                                         in_grad_group, workspace, workspace_bytes, stream);
+        if (rc) return rc;
+    }
     for (int l = 0; l < L; ++l) {
         const dpclip_layer& y = layers[l];
         if (t1.active && y.T == 1) continue;
+        if (track && in_grad_group[l]) continue;
         float* gb = y.has_bias ? y.gb : nullptr;
         if (y.has_bias && !gb) return DPCLIP_ERR_INVALID_ARG;
         // noise indexes the dense d_out x d_in tensor, so the step wants unpadded output rows

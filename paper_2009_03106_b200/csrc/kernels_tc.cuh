@@ -62,13 +62,34 @@ constexpr int N_EPILOGUE_WARPS = 8;
 constexpr int THREADS = 64 + 32 * N_EPILOGUE_WARPS;   // warp 0 TMA, warp 1 MMA, warps 2..9 epilogue
 constexpr int SMEM_BYTES = 4 * 3 * TILE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;   // = 6 * 2 tiles
 
-struct Params {
+constexpr int MAX_LAYERS = 8;                 // layers one launch can take
+
+struct Params {            // one layer
     int R, T, d_in, d_out, has_bias;
     int n_groups;          // dense (T % 128 == 0): examples; otherwise: 128-row blocks
     int dense, q;          // q = T / 128 blocks per example in the dense case
     float* sq;
+};
+
+// One launch: the groups of up to MAX_LAYERS layers, dealt to the CTAs in one sequence (layer 0's groups
+// first).  With one example per CTA a single layer of a small batch is a latency chain (set-up, first
+// load, the second row block and both epilogues are all exposed); several layers in one launch give every
+// CTA a queue of items, so loads of the next item run under the MMAs and epilogues of the current one.
+struct Launch {
+    CUtensorMap map_a[MAX_LAYERS], map_z[MAX_LAYERS];
+    Params layer[MAX_LAYERS];
+    int group_begin[MAX_LAYERS + 1];
+    int L, total_groups;
     int* status;
 };
+
+// layer of group g (group_begin is ascending; L is small)
+__device__ __forceinline__ int layer_of(const Launch& q, int g) {
+    int l = 0;
+#pragma unroll 1
+    while (l + 1 < q.L && g >= q.group_begin[l + 1]) ++l;
+    return l;
+}
 
 // One unit of MMA work: row block rb against column blocks cb .. cb + ncb - 1 (ncb = 1 or 2).
 struct Sub { int rb, cb, ncb; };
@@ -76,22 +97,29 @@ struct Sub { int rb, cb, ncb; };
 // The sub-items of group g, in a fixed order that every warp role walks identically.
 // Row block rb pairs with column blocks rb .. cb_max(rb) (those that still hold rows of an example
 // that has rows in rb), taken two at a time so that one 128 x 256 MMA covers two of them.
+// In the dense case the row blocks of an example are walked from the LAST to the first: row block rb needs
+// the column blocks rb .. q-1, so every pass then fetches exactly one block that has not been read before
+// (its own) and re-reads the others from L2.  Walking upwards, the first pass streams the whole example
+// from HBM and the later ones run out of L2; CTAs that start together then alternate in lockstep between
+// a phase that saturates HBM and one that leaves it idle (measured: 23 us per 512 KB example instead of the
+// 12.5 us its bytes take).
 struct SubIter {
-    int rb, rb_end, cb, cb_max;
+    int rb, rb_first, rb_last, cb, cb_max;
     __device__ __forceinline__ static int cbmax(const Params& p, int rb) {
         const long last_row = min((long)rb * BM + BM - 1, (long)p.R - 1);
         const long e_last = last_row / p.T;
         return (int)(min((e_last + 1) * p.T - 1, (long)p.R - 1) / BM);
     }
     __device__ __forceinline__ SubIter(const Params& p, int g) {
-        if (p.dense) { rb = g * p.q; rb_end = rb + p.q; } else { rb = g; rb_end = g + 1; }
+        if (p.dense) { rb_first = g * p.q; rb_last = rb_first + p.q - 1; } else { rb_first = g; rb_last = g; }
+        rb = rb_last;
         cb = rb; cb_max = cbmax(p, rb);
     }
     __device__ __forceinline__ bool next(const Params& p, Sub& s) {
-        if (rb >= rb_end) return false;
+        if (rb < rb_first) return false;
         s.rb = rb; s.cb = cb; s.ncb = cb + 1 <= cb_max ? 2 : 1;
         cb += 2;
-        if (cb > cb_max) { ++rb; if (rb < rb_end) { cb = rb; cb_max = cbmax(p, rb); } }
+        if (cb > cb_max) { --rb; if (rb >= rb_first) { cb = rb; cb_max = cbmax(p, rb); } }
         return true;
     }
 };
@@ -99,8 +127,7 @@ struct SubIter {
 
 template <bool DIAG_ONLY>
 __global__ void __launch_bounds__(gram::THREADS, 1)
-gram_norm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_z,
-                 const gram::Params p) {
+gram_norm_kernel(const __grid_constant__ gram::Launch q) {
     using namespace gram;
     constexpr int STAGES = Cfg<DIAG_ONLY>::STAGES, STAGE_BYTES = Cfg<DIAG_ONLY>::STAGE_BYTES;
     // offset of the first column block's tile inside a stage (the row block's own tile comes first
@@ -121,16 +148,13 @@ gram_norm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         mbar_init(acc_full, 1); mbar_init(acc_empty, N_EPILOGUE_WARPS);
         *abort_flag = 0;
         mbar_fence_init();
-        tma_prefetch_desc(&map_a);
-        tma_prefetch_desc(&map_z);
+        for (int l = 0; l < q.L; ++l) { tma_prefetch_desc(&q.map_a[l]); tma_prefetch_desc(&q.map_z[l]); }
     }
     if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;      // A A^T in columns 0..255, Zb Zb^T in 256..511
-
-    const int nk_a = (p.d_in + BK - 1) / BK, nk_z = (p.d_out + BK - 1) / BK;
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer
@@ -139,17 +163,20 @@ gram_norm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             bool ok = true;
             int tr = 0;
             DPCLIP_TRACE_AT(0, 255);
-            for (int g = blockIdx.x; g < p.n_groups && ok; g += gridDim.x) {
-                SubIter it(p, g);
+            for (int g = blockIdx.x; g < q.total_groups && ok; g += gridDim.x) {
+                const int l = layer_of(q, g);
+                const Params& p = q.layer[l];
+                const int nk_a = (p.d_in + BK - 1) / BK, nk_z = (p.d_out + BK - 1) / BK;
+                SubIter it(p, g - q.group_begin[l]);
                 Sub s;
                 while (ok && it.next(p, s)) {
                     const bool diag = s.rb == s.cb;
                     const uint32_t bytes = TILE_BYTES * (s.ncb + (diag ? 0 : 1));
                     const int nk = nk_a + nk_z;
                     for (int kb = 0; kb < nk; ++kb) {
-                        const CUtensorMap* map = kb < nk_a ? &map_a : &map_z;
+                        const CUtensorMap* map = kb < nk_a ? &q.map_a[l] : &q.map_z[l];
                         const int x = (kb < nk_a ? kb : kb - nk_a) * BK;
-                        ok = mbar_wait(&empty[stage], phase ^ 1, abort_flag, p.status);
+                        ok = mbar_wait(&empty[stage], phase ^ 1, abort_flag, q.status);
                         if (!ok) break;
                         DPCLIP_TRACE_AT(0, tr); ++tr;
                         uint8_t* dst = smem + stage * STAGE_BYTES;
@@ -168,19 +195,22 @@ gram_norm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             int stage = 0; uint32_t phase = 0; uint32_t acc_phase = 0;
             bool ok = true;
             int tr = 0;
-            for (int g = blockIdx.x; g < p.n_groups && ok; g += gridDim.x) {
-                SubIter it(p, g);
+            for (int g = blockIdx.x; g < q.total_groups && ok; g += gridDim.x) {
+                const int l = layer_of(q, g);
+                const Params& p = q.layer[l];
+                const int nk_a = (p.d_in + BK - 1) / BK, nk_z = (p.d_out + BK - 1) / BK;
+                SubIter it(p, g - q.group_begin[l]);
                 Sub s;
                 while (ok && it.next(p, s)) {
                     const uint32_t idesc = make_idesc_bf16(BM, BM * s.ncb, 0, 0);
-                    ok = mbar_wait(acc_empty, acc_phase ^ 1, abort_flag, p.status);
+                    ok = mbar_wait(acc_empty, acc_phase ^ 1, abort_flag, q.status);
                     if (!ok) break;
                     tc_fence_after_sync();
                     for (int kb = 0; kb < nk_a + nk_z; ++kb) {
                         const bool is_a = kb < nk_a;
                         const uint32_t d_tmem = tmem_base + (is_a ? 0 : 256);
                         const bool first = is_a ? kb == 0 : kb == nk_a;
-                        ok = mbar_wait(&full[stage], phase, abort_flag, p.status);
+                        ok = mbar_wait(&full[stage], phase, abort_flag, q.status);
                         if (!ok) break;
                         DPCLIP_TRACE_AT(2, tr); ++tr;
                         tc_fence_after_sync();
@@ -213,11 +243,13 @@ gram_norm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         uint32_t acc_phase = 0;
         bool ok = true;
         int etr = 0;
-        for (int g = blockIdx.x; g < p.n_groups && ok; g += gridDim.x) {
-            SubIter it(p, g);
+        for (int g = blockIdx.x; g < q.total_groups && ok; g += gridDim.x) {
+            const int l = layer_of(q, g);
+            const Params& p = q.layer[l];
+            SubIter it(p, g - q.group_begin[l]);
             Sub s;
             while (it.next(p, s)) {
-                ok = mbar_wait(acc_full, acc_phase, abort_flag, p.status);
+                ok = mbar_wait(acc_full, acc_phase, abort_flag, q.status);
                 if (!ok) break;
                 if (threadIdx.x == 64) { DPCLIP_TRACE_AT(3, etr); ++etr; }
                 acc_phase ^= 1;
@@ -290,6 +322,197 @@ gram_norm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     if (warp == 1) { tc_fence_after_sync(); tmem_dealloc(tmem_base, 512); }
 }
 
+// ---------------------------------------------------------------------------
+// Gram kernel for examples of exactly two 128-row blocks (T = 256), every layer of the launch.
+//
+// The generic kernel walks such an example as two passes (row block 1 against itself, then row block 0
+// against both), and the second pass re-reads half of the example.  With one example per SM in flight, 148
+// examples' worth of other data passes through L2 between the two reads, so for wide layers the re-read
+// comes from HBM again (measured: 1.5x the algorithmic DRAM traffic).  Here each K-chunk of the WIDER
+// operand X is fetched once and feeds both its products at once:
+//     P1  X rows 0..255  ->  G^X_0  = X_0 [X_0; X_1]^T  (tensor-memory columns   0..255)
+//                            G^X_11 = X_1 X_1^T         (columns 256..383)
+//     P2  Y rows 128..255 -> G^Y_11                     (columns 384..511)   epilogue E1: <G^X_11, G^Y_11>
+//     P3  Y rows 0..255  ->  G^Y_0                      (columns 256..511)   epilogue E0: <G^X_0, G^Y_0>,
+//                                                                            block (0,1) counted twice
+// Only the narrower operand's second half is read twice, a few hundred KB apart (an L2 hit).  All 512
+// columns are in use, so E1 must finish before P3 starts and E0 before the next example's P1.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(gram::THREADS, 1)
+gram_norm_q2_kernel(const __grid_constant__ gram::Launch q) {
+    using namespace gram;
+    constexpr int STAGES = 6, STAGE_BYTES = 2 * TILE_BYTES;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
+    uint64_t* empty = full + STAGES;
+    uint64_t* acc_full = empty + STAGES;
+    uint64_t* acc_empty = acc_full + 1;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 1);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        mbar_init(acc_full, 1); mbar_init(acc_empty, N_EPILOGUE_WARPS);
+        *abort_flag = 0;
+        mbar_fence_init();
+        for (int l = 0; l < q.L; ++l) { tma_prefetch_desc(&q.map_a[l]); tma_prefetch_desc(&q.map_z[l]); }
+    }
+    if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int stage = 0; uint32_t phase = 0;
+            bool ok = true;
+            for (int g = blockIdx.x; g < q.total_groups && ok; g += gridDim.x) {
+                const int l = layer_of(q, g);
+                const Params& p = q.layer[l];
+                const bool x_is_z = p.d_out > p.d_in;
+                const CUtensorMap* map_x = x_is_z ? &q.map_z[l] : &q.map_a[l];
+                const CUtensorMap* map_y = x_is_z ? &q.map_a[l] : &q.map_z[l];
+                const int nk_x = ((x_is_z ? p.d_out : p.d_in) + BK - 1) / BK;
+                const int nk_y = ((x_is_z ? p.d_in : p.d_out) + BK - 1) / BK;
+                const int r0 = (g - q.group_begin[l]) * 2 * BM;
+                for (int kb = 0; kb < nk_x + 2 * nk_y && ok; ++kb) {
+                    // P1: both blocks of X; P2: block 1 of Y; P3: both blocks of Y
+                    const bool p1 = kb < nk_x, p2 = !p1 && kb < nk_x + nk_y;
+                    const CUtensorMap* map = p1 ? map_x : map_y;
+                    const int x = (p1 ? kb : (p2 ? kb - nk_x : kb - nk_x - nk_y)) * BK;
+                    ok = mbar_wait(&empty[stage], phase ^ 1, abort_flag, q.status);
+                    if (!ok) break;
+                    uint8_t* dst = smem + stage * STAGE_BYTES;
+                    mbar_arrive_expect_tx(&full[stage], p2 ? TILE_BYTES : 2 * TILE_BYTES);
+                    if (p2) {
+                        tma_load_2d(dst, map, &full[stage], x, r0 + BM);
+                    } else {
+                        tma_load_2d(dst, map, &full[stage], x, r0);
+                        tma_load_2d(dst + TILE_BYTES, map, &full[stage], x, r0 + BM);
+                    }
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc256 = make_idesc_bf16(BM, 2 * BM, 0, 0), idesc128 = make_idesc_bf16(BM, BM, 0, 0);
+            int stage = 0; uint32_t phase = 0; uint32_t acc_phase = 0;
+            bool ok = true;
+            for (int g = blockIdx.x; g < q.total_groups && ok; g += gridDim.x) {
+                const int l = layer_of(q, g);
+                const Params& p = q.layer[l];
+                const bool x_is_z = p.d_out > p.d_in;
+                const int nk_x = ((x_is_z ? p.d_out : p.d_in) + BK - 1) / BK;
+                const int nk_y = ((x_is_z ? p.d_in : p.d_out) + BK - 1) / BK;
+                // the previous example's last epilogue has read every column
+                ok = mbar_wait(acc_empty, acc_phase ^ 1, abort_flag, q.status);
+                if (!ok) break;
+                tc_fence_after_sync();
+                for (int kb = 0; kb < nk_x + 2 * nk_y; ++kb) {
+                    const bool p1 = kb < nk_x, p2 = !p1 && kb < nk_x + nk_y;
+                    if (kb == nk_x + nk_y) {
+                        // P2 is complete: hand G^X_11, G^Y_11 to the epilogue and wait until it has read them
+                        // (P3 overwrites their columns)
+                        mma_commit(acc_full);
+                        acc_phase ^= 1;
+                        ok = mbar_wait(acc_empty, acc_phase ^ 1, abort_flag, q.status);
+                        if (!ok) break;
+                        tc_fence_after_sync();
+                    }
+                    ok = mbar_wait(&full[stage], phase, abort_flag, q.status);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const uint32_t t0 = smem_u32(smem + stage * STAGE_BYTES), t1 = t0 + TILE_BYTES;
+                    const bool first = p1 ? kb == 0 : (p2 ? kb == nk_x : kb == nk_x + nk_y);
+#pragma unroll
+                    for (int k4 = 0; k4 < BK / 16; ++k4) {
+                        // K-major, 128-byte swizzle: 8-row groups 1024 bytes apart; 16 features = 32 bytes.
+                        // The two row blocks of a stage are contiguous, so N = 256 simply runs on.
+                        const uint32_t acc = (first && k4 == 0) ? 0u : 1u;
+                        const uint64_t d0 = make_smem_desc_sw128(t0 + k4 * 32, 16, 1024);
+                        if (p1) {
+                            const uint64_t d1 = make_smem_desc_sw128(t1 + k4 * 32, 16, 1024);
+                            mma_bf16_ss(tmem_base, d0, d0, idesc256, acc);               // G^X_0
+                            mma_bf16_ss(tmem_base + 256, d1, d1, idesc128, acc);         // G^X_11
+                        } else if (p2) {
+                            mma_bf16_ss(tmem_base + 384, d0, d0, idesc128, acc);         // G^Y_11 (the stage holds block 1)
+                        } else {
+                            mma_bf16_ss(tmem_base + 256, d0, d0, idesc256, acc);         // G^Y_0
+                        }
+                    }
+                    mma_commit(&empty[stage]);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                }
+                if (!ok) break;
+                mma_commit(acc_full);
+                acc_phase ^= 1;
+            }
+        }
+    } else {
+        // ------------------------------------------------ epilogue (warps 2..9)
+        // warp w reads tensor-memory lanes 32*(w % 4)..+31; the two warps of a lane quarter split the columns
+        const int quarter = warp & 3;
+        const int half = (warp - 2) >> 2;
+        uint32_t acc_phase = 0;
+        bool ok = true;
+        const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16);
+        for (int g = blockIdx.x; g < q.total_groups && ok; g += gridDim.x) {
+            const int l = layer_of(q, g);
+            const Params& p = q.layer[l];
+            const bool x_is_z = p.d_out > p.d_in;
+            const int e = g - q.group_begin[l];
+            float val = 0.f;
+#pragma unroll 1
+            for (int pass = 0; pass < 2; ++pass) {
+                // pass 0 = E1: 128 columns of G^X_11 (at 256) and G^Y_11 (at 384), 64 per warp;
+                // pass 1 = E0: 256 columns of G^X_0 (at 0) and G^Y_0 (at 256), 128 per warp
+                ok = mbar_wait(acc_full, acc_phase, abort_flag, q.status);
+                if (!ok) break;
+                acc_phase ^= 1;
+                tc_fence_after_sync();
+                const int width = pass == 0 ? 64 : 128;
+                const uint32_t cx = (pass == 0 ? 256 : 0) + half * width, cy = (pass == 0 ? 384 : 256) + half * width;
+                float sa = 0.f, sb = 0.f;
+#pragma unroll 1
+                for (int c0 = 0; c0 < width; c0 += 32) {
+                    uint32_t vx[32], vy[32];
+                    tmem_ld_32x32(t_row + cx + c0, vx);
+                    tmem_ld_32x32(t_row + cy + c0, vy);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const float x = __uint_as_float(vx[j]), y = __uint_as_float(vy[j]);
+                        sa = fmaf(x, y, sa);
+                        sb += x_is_z ? x : y;                   // entries of Zb Zb^T: the bias term
+                    }
+                }
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(acc_empty);
+                // block (0,1) stands for its mirror image (1,0) too
+                val += ((pass == 1 && half == 1) ? 2.f : 1.f) * (sa + (p.has_bias ? sb : 0.f));
+            }
+            if (!ok) break;
+            val = warp_sum(val);
+            if (lane == 0) atomicAdd(p.sq + e, val);
+        }
+    }
+
+    // ---------------------------------------------------- teardown
+    if (*abort_flag) {                                      // let copies in flight land before the CTA exits
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) { tc_fence_after_sync(); tmem_dealloc(tmem_base, 512); }
+}
+
 // ===========================================================================
 // Zb^T diag(f) A kernel (GRAD and NORM modes)
 // ===========================================================================
@@ -319,7 +542,8 @@ template <int MT> struct Cfg {
 struct Params {
     int R, T, d_in, d_out;
     int norm_mode;                 // 0 = GRAD, 1 = NORM
-    int tiles_m, tiles_n;
+    int tiles_m, tiles_n;          // tiles_m counts the d_out tiles of ALL layers of the launch (layer-major)
+    int tiles_m_layer;             // d_out tiles of one layer (= tiles_m for a single layer)
     int n_items;
     int kb_per_split;              // GRAD: 64-row blocks per item
     int do_bias;                   // GRAD: gb != NULL; NORM: has_bias
@@ -331,14 +555,23 @@ struct Params {
     int* status;
 };
 
-struct Item { int m0, n0, tn; int row_begin, row_end; int nkb; int example; };
+// Several layers of ONE shape (same R, T, d_in, d_out: e.g. the four attention projections) can share a
+// GRAD launch: their d_out tiles are stacked, every item knows its layer and takes that layer's tensor
+// maps, and the partial tiles of all layers go to one scratch area.  A layer of this size alone gives each
+// CTA 14 stages, a third of which is pipeline fill and epilogue; four of them give 57.
+constexpr int MAX_LAYERS = 8;
+struct Maps { CUtensorMap a[MAX_LAYERS], z[MAX_LAYERS]; };
+
+struct Item { int m0, n0, tn; int row_begin, row_end; int nkb; int example; int layer; };
 
 template <int MT>
 __device__ __forceinline__ Item decode(const Params& p, int item) {
     Item w;
     const int n_tiles = p.tiles_m * p.tiles_n;
     const int tile = item % n_tiles, outer = item / n_tiles;
-    w.m0 = (tile / p.tiles_n) * Cfg<MT>::BM;
+    const int tm = tile / p.tiles_n;
+    w.layer = tm / p.tiles_m_layer;
+    w.m0 = (tm - w.layer * p.tiles_m_layer) * Cfg<MT>::BM;
     w.tn = tile % p.tiles_n;
     w.n0 = w.tn * BN;
     if (p.norm_mode) {
@@ -357,8 +590,7 @@ __device__ __forceinline__ Item decode(const Params& p, int item) {
 
 template <int MT>
 __global__ void __launch_bounds__(zta::THREADS, 1)
-zta_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_z,
-              const zta::Params p) {
+zta_tc_kernel(const __grid_constant__ zta::Maps maps, const zta::Params p) {
     using namespace zta;
     using C = Cfg<MT>;
     constexpr int STAGES = C::STAGES, STAGE_BYTES = C::STAGE_BYTES, A_BYTES = C::A_BYTES, NBUF = C::NBUF;
@@ -381,8 +613,8 @@ zta_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
         for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], N_EPILOGUE_WARPS); }
         *abort_flag = 0;
         mbar_fence_init();
-        tma_prefetch_desc(&map_a);
-        tma_prefetch_desc(&map_z);
+        const int n_layers = p.tiles_m / p.tiles_m_layer;
+        for (int l = 0; l < n_layers; ++l) { tma_prefetch_desc(&maps.a[l]); tma_prefetch_desc(&maps.z[l]); }
     }
     if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
     tc_fence_before_sync();
@@ -399,6 +631,8 @@ zta_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
             DPCLIP_TRACE_AT(0, 255);
             for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
                 const Item w = decode<MT>(p, item);
+                const CUtensorMap* map_a = &maps.a[w.layer];
+                const CUtensorMap* map_z = &maps.z[w.layer];
                 for (int kb = 0; kb < w.nkb; ++kb) {
                     ok = mbar_wait(&empty[stage], phase ^ 1, abort_flag, p.status);
                     if (!ok) break;
@@ -408,10 +642,10 @@ zta_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
                     mbar_arrive_expect_tx(&full[stage], STAGE_BYTES);
 #pragma unroll
                     for (int c = 0; c < C::BM / 64; ++c)
-                        tma_load_2d(dst + c * CHUNK_BYTES, &map_z, &full[stage], w.m0 + c * 64, y);
+                        tma_load_2d(dst + c * CHUNK_BYTES, map_z, &full[stage], w.m0 + c * 64, y);
 #pragma unroll
                     for (int c = 0; c < BN / 64; ++c)
-                        tma_load_2d(dst + A_BYTES + c * CHUNK_BYTES, &map_a, &full[stage], w.n0 + c * 64, y);
+                        tma_load_2d(dst + A_BYTES + c * CHUNK_BYTES, map_a, &full[stage], w.n0 + c * 64, y);
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
             }
@@ -671,6 +905,12 @@ struct ReduceParams {
     float* gW; long ldg; float* gb; int vec_ok;
     int lanes;                                                  // thread rows of a CTA sharing the row slices (1..8)
     float noise_scale; uint32_t k0, k1, sw0, sw1, sb0, sb1;     // Philox key, weight / bias stream words
+    // Layers of one shape that shared a GRAD launch: blockIdx.y = layer; layer y's tiles start at tile
+    // y * tiles_layer of every row slice, and its outputs and noise streams come from the arrays (n_layers
+    // == 0: a single layer described by the scalar fields above).
+    int n_layers, tiles_layer;
+    float* gW_l[zta::MAX_LAYERS]; float* gb_l[zta::MAX_LAYERS];
+    uint32_t sw0_l[zta::MAX_LAYERS], sw1_l[zta::MAX_LAYERS], sb0_l[zta::MAX_LAYERS], sb1_l[zta::MAX_LAYERS];
 };
 
 }  // namespace tc
@@ -682,8 +922,16 @@ namespace dpclip {
 namespace tc {
 
 __global__ void __launch_bounds__(256)
-reduce_partials_kernel(const ReduceParams p) {
+reduce_partials_kernel(const ReduceParams q) {
     __shared__ float4 part_s[256];
+    ReduceParams p = q;
+    if (q.n_layers > 0) {
+        const int y = blockIdx.y;
+        p.part = q.part + (size_t)y * q.tiles_layer * q.BM * q.BN;
+        if (q.bias_part) p.bias_part = q.bias_part + (size_t)y * q.tiles_layer * q.BM;
+        p.gW = q.gW_l[y]; p.gb = q.gb_l[y];
+        p.sw0 = q.sw0_l[y]; p.sw1 = q.sw1_l[y]; p.sb0 = q.sb0_l[y]; p.sb1 = q.sb1_l[y];
+    }
     const int n4 = (p.d_in + 3) >> 2;
     const long total = (long)p.d_out * n4;
     const size_t tile_elems = (size_t)p.BM * p.BN;

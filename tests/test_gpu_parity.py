@@ -677,6 +677,63 @@ def test_step_seq_small(dp):
     _check_step(dp, w, _calibrate(w, layers, 2, w.C), w.C, w.sigma, 2)
 
 
+def test_gram_layers_in_one_launch(dp):
+    """Gram-identity norms of several layers in one launch: examples of one, two and three 128-row blocks,
+    examples that share a block, ragged lengths, with and without bias, more layers than one launch takes;
+    every row of sq equals the oracle's, layers the entry point does not take are reported as such."""
+    B = 3
+    shapes = [(256, 64, 136, True), (128, 72, 64, False), (64, 64, 64, True), (256, 136, 64, False),   # two-block and shorter examples
+              (100, 64, 72, True), (384, 64, 64, False), (40, 136, 64, True)]                            # the rest
+    shapes += [(64, 64, 8 * k, bool(k & 1)) for k in range(1, 9)]          # 10 layers of one-or-two-block examples: two launches
+    data = [workloads.random_layer(50 + i, B, T, d_in, d_out, "bf16", scale_z=0.05) for i, (T, d_in, d_out, _) in enumerate(shapes)]
+    layers = [dp.Layer(to_device(A, "bf16"), to_device(Z, "bf16"), hb, dp.DPCLIP_GRAM) for (A, Z), (_, _, _, hb) in zip(data, shapes)]
+    # a T = 1 layer, an fp32-ALU layer (rows TMA cannot address) and a lone layer of its class are left alone
+    A1, Z1 = workloads.random_layer(90, B, 1, 64, 64, "bf16", scale_z=0.05)
+    A2, Z2 = workloads.random_layer(91, B, 24, 27, 64, "bf16", scale_z=0.05)
+    layers += [dp.Layer(to_device(A1, "bf16"), to_device(Z1, "bf16"), True),
+               dp.Layer(to_device(A2, "bf16"), to_device(Z2, "bf16"), True, dp.DPCLIP_GRAM)]
+    plan = dp.StepPlan(layers)
+    plan.sq_layers.fill_(float("nan"))
+    taken = dp.dpclip_gram_layers_sqnorms(plan)
+    torch.cuda.synchronize()
+    assert dp.dpclip_read_status(plan.workspace) == 0
+    assert taken == [True] * len(shapes) + [False, False]
+    sq = plan.sq_layers.cpu().numpy()
+    for l, ((A, Z), (_, _, _, hb)) in enumerate(zip(data, shapes)):
+        ref = oracle.layer_sqnorms(A, Z, hb)
+        assert max_rel(np.sqrt(sq[l]), np.sqrt(ref)) <= TOL["bf16"]["norm"], (l, shapes[l])
+    assert np.isnan(sq[len(shapes):]).all()
+    # one candidate only: nothing is taken
+    lone = dp.StepPlan(layers[:1])
+    assert dp.dpclip_gram_layers_sqnorms(lone) == [False]
+
+
+def test_step_same_shape_layers_share_launches(dp, monkeypatch):
+    """Layers of one shape go through one clipped-sum launch (stacked d_out tiles, one set of partial tiles,
+    one reduce with every layer's own noise streams): 256-row and 128-row tile forms, ragged d_out, layers
+    with and without bias in one group, a group next to single layers; and the same model layer by layer."""
+    L = workloads.LayerSpec
+    w = workloads.Workload("same_shape_groups", 5, "bf16",
+                           (L("a1", 48, 72, 136, True, "normal"), L("b1", 48, 136, 72, False, "normal"),
+                            L("a2", 48, 72, 136, False, "normal"), L("c", 48, 64, 64, True, "normal"),
+                            L("a3", 48, 72, 136, True, "relu"), L("b2", 48, 136, 72, False, "relu"),
+                            L("head", 1, 136, 24, True, "relu")), 1.0, 0.8, 1.0 / (5 * 48))
+    layers = workloads.generate(w, 3)
+    cal = _calibrate(w, layers, 3, w.C)
+    _check_step(dp, w, cal, w.C, w.sigma, 3)
+    plan = _run_step(dp, w, cal, w.C, w.sigma, 3)
+    taken = dp.dpclip_same_shape_layers_clipped_grad_noise(plan, w.C, w.sigma, 3, 0)
+    torch.cuda.synchronize()
+    assert taken == [True, True, True, False, True, True, False]
+    monkeypatch.setenv("DPCLIP_NO_GRAD_GROUP", "1")
+    monkeypatch.setenv("DPCLIP_NO_GRAM_GROUP", "1")
+    single = _run_step(dp, w, cal, w.C, w.sigma, 3)
+    for l in range(len(layers)):
+        a, b = plan.gW[l].cpu().numpy(), single.gW[l].cpu().numpy()
+        assert rel_fro(a, b) <= 1e-5            # same products, another summation order
+    _check_step(dp, w, cal, w.C, w.sigma, 3)
+
+
 def test_per_layer_clipping_through_the_same_entry_points(dp):
     """Per-layer clipping (each layer's gradient clipped to C / sqrt(L) on its own, the variant the paper's
     per-layer norms make possible): the rows of sq stay separate, so it is dpclip_factors on one row at a
