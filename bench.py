@@ -208,20 +208,38 @@ def kernel_breakdown(torch, dp, w, plan, steps, flush, C, sigma):
         s.record(); fn(); e.record()
         acc.setdefault(key, []).append((s, e))
 
+    # what dpclip_step does: layers whose norms go by the Gram identity share a launch, and so do the clipped
+    # sums of layers of one shape; the grouped calls report which layers they took
+    taken_n = taken_g = [False] * len(w.layers)
     for it in range(steps + 1):
         flush()
+        box = {}
+        timed(("norm_gram_group", -2), lambda: box.update(t=dp.dpclip_gram_layers_sqnorms(plan)))
+        taken_n = box["t"]
         for l, (y, spec) in enumerate(zip(plan.layers, w.layers)):
+            if taken_n[l]:
+                continue
             m = dp.dpclip_pick_method(w.B, spec.T, spec.d_in, spec.d_out, None, None, plan.dtype_code)
             kind = {dp.DPCLIP_T1: "norm_t1", dp.DPCLIP_SIMT: "norm_simt", dp.DPCLIP_GRAM: "norm_gram",
                     dp.DPCLIP_MATERIALIZE: "norm_mat"}[m]
             timed((kind, l), lambda: dp.dpclip_layer_sqnorms(y.A, y.Zbar, spec.has_bias, plan.sq_layers[l],
                                                              plan.workspace))
         timed(("factors", -1), lambda: dp.dpclip_factors(plan.sq_layers, C, plan.clip, plan.norms))
+        timed(("grad_group", -3), lambda: box.update(g=dp.dpclip_same_shape_layers_clipped_grad_noise(plan, C, sigma, 1, 0)))
+        taken_g = box["g"]
         for l, (y, spec) in enumerate(zip(plan.layers, w.layers)):
+            if taken_g[l]:
+                continue
             timed(("grad", l), lambda: dp.dpclip_clipped_grad(y.A, y.Zbar, plan.clip, plan.gW[l], plan.gb[l],
                                                               plan.workspace))
             timed(("noise", l), lambda: (dp.dpclip_add_noise(plan.gW[l], sigma, C, 1, 2 * l),
                                          plan.gb[l] is not None and dp.dpclip_add_noise(plan.gb[l], sigma, C, 1, 2 * l + 1)))
+    if not any(taken_n):
+        acc.pop(("norm_gram_group", -2))
+    if not any(taken_g):
+        acc.pop(("grad_group", -3))
+    kernel_breakdown.groups = {"norm_gram_group": [l for l, t in enumerate(taken_n) if t],
+                               "grad_group": [l for l, t in enumerate(taken_g) if t]}
     torch.cuda.synchronize()
     out = {}
     for key, evs in acc.items():
@@ -230,14 +248,19 @@ def kernel_breakdown(torch, dp, w, plan, steps, flush, C, sigma):
     return out
 
 
+kernel_breakdown.groups = {}          # members of the grouped launches of the last breakdown
+
+
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures
 # summarised under profiles/ (same workload, same launch configuration); None where not captured
 NCU_TRAFFIC_BYTES = {
     ("mlp_784_1000_1000_10_b128", "t1_all_grads_tf32_kernel"): 2.55e6,   # profiles/fused_t1_mlp_784_1000_1000_10_b128.txt
     ("mlp_784_1000_1000_10_b128", "t1_all_grads_kernel"): 2.54e6,
-    ("seq_b128_t256_d512_bf16", "grad[ffn_in]"): 171.7e6,             # profiles/tc_kernels_seq_b128_t256.txt
-    ("seq_b128_t256_d512_bf16", "grad[lstm_gates]"): 171.7e6,
-    ("seq_b128_t256_d512_bf16", "grad[ffn_out]"): 171.7e6,
+    ("seq_b128_t256_d512_bf16", "norm_gram_group"): 775.3e6,          # profiles/tc_kernels_seq_b128_t256.txt
+    ("seq_b128_t256_d512_bf16", "grad_group"): 272.7e6,
+    ("seq_b128_t256_d512_bf16", "grad[ffn_in]"): 171.1e6,
+    ("seq_b128_t256_d512_bf16", "grad[lstm_gates]"): 171.1e6,
+    ("seq_b128_t256_d512_bf16", "grad[ffn_out]"): 171.1e6,
 }
 
 
@@ -277,11 +300,44 @@ def roofline_fused_t1(w, step_ms, peaks):
     return r
 
 
+def entry_name(w, key):
+    """Layer name(s) of a breakdown entry."""
+    kind, l = key
+    if kind in kernel_breakdown.groups:
+        return "+".join(w.layers[i].name for i in kernel_breakdown.groups[kind])
+    return w.layers[l].name if l >= 0 else "all"
+
+
+def roofline_group(w, key, breakdown, peaks):
+    """Roofline of a launch that several layers share (bf16, tensor cores): work = the member layers' sum."""
+    kind = key[0]
+    base = "norm_gram" if kind == "norm_gram_group" else "grad"
+    members = kernel_breakdown.groups[kind]
+    nbytes = sum(layer_work(w, w.layers[i], base)[0] for i in members)
+    flops = sum(layer_work(w, w.layers[i], base)[1] for i in members)
+    ms = breakdown[key]
+    t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9)
+    t_alu = flops / (peaks["bf16_tflops"] * 1e12)
+    if t_hbm >= t_alu:
+        ach = nbytes / (ms * 1e-3) / 1e9
+        r = dict(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s", frac=ach / peaks["hbm_gbs"])
+    else:
+        ach = flops / (ms * 1e-3) / 1e12
+        r = dict(bound="tensor", achieved=ach, peak=peaks["bf16_tflops"], unit="TFLOP/s", frac=ach / peaks["bf16_tflops"])
+    name = f"{kind}[{entry_name(w, key)}]"
+    r.update(traffic=NCU_TRAFFIC_BYTES.get((w.name, kind)), kernel=name, kernel_ms=ms,
+             share_of_step=ms / sum(breakdown.values()), algorithmic_bytes=nbytes, algorithmic_flops=flops,
+             peak_source=peaks["source"])
+    return r
+
+
 def roofline_for(w, breakdown, peaks):
     """Roofline of the launch that takes the largest share of the step."""
     cands = {k: v for k, v in breakdown.items() if k[0] not in ("factors",)}
     key = max(cands, key=cands.get)
     kind, l = key
+    if kind in kernel_breakdown.groups:
+        return roofline_group(w, key, breakdown, peaks)
     spec = w.layers[l]
     nbytes, flops = layer_work(w, spec, kind)
     ms = breakdown[key]
@@ -336,8 +392,7 @@ def bench_workload(torch, dp, w, steps, warmup, flush, peaks, with_e2e=True):
     res = dict(times_ms=times, warm_ms=float(np.median(warm)), eager_ms=float(np.median(eager)),
                single_graph_ms=float(np.mean(single)), rotating=rotating,
                launches_per_step=int(launches_per_step),
-               breakdown={f"{k[0]}[{w.layers[k[1]].name if k[1] >= 0 else 'all'}]": round(v * 1e3, 2)
-                          for k, v in bd.items()},
+               breakdown={f"{k[0]}[{entry_name(w, k)}]": round(v * 1e3, 2) for k, v in bd.items()},
                roofline=(roofline_fused_t1(w, float(np.mean(times)), peaks) if branches == 1
                          else roofline_for(w, bd, peaks)))
     # whole-step lower bound: max(total algorithmic bytes / HBM, total flops / the engine used)
@@ -559,13 +614,15 @@ def main():
     ap.add_argument("--workload", default="cfg2")
     ap.add_argument("--impl", default="dpclip", choices=["dpclip", "reference"])
     ap.add_argument("--others", default="cfg1,cfg2_bf16,cfg3_f32,cfg3_bf16,cfg4",
-                    help="further workloads reported under 'workloads' (N=1 only; '' for none)")
+                    help="further workloads reported under 'workloads' (N=1 only; 'none' for none)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--points", default="", help="with --sweep: only these points, 'B,T,d_in,d_out;B,T,d_in,d_out;...'")
     ap.add_argument("--noise-n", type=int, default=0, help="with --sweep: also time dpclip_add_noise on this many elements")
     ap.add_argument("--sweep", action="store_true",
                     help="instead of the benchmark line: Gram-vs-materialise sweep of the T > 1 norm (1 GPU)")
     args = ap.parse_args()
+    if args.others == "none":
+        args.others = ""
     args.warmup = max(args.warmup, 3) if args.impl == "dpclip" else args.warmup
     if args.impl == "reference":
         return run_reference(args)

@@ -27,9 +27,11 @@
  *   - The caller owns every buffer, including the workspace.  The library
  *     allocates no device memory and keeps no state between calls.  A
  *     workspace holds scratch (partial tiles) and, in its header, a status
- *     word and the grid-barrier counter of the one-launch T = 1 step: calls
- *     that may run at the same time (different streams) need workspaces of
- *     their own; calls ordered on one stream can share one.
+ *     word, the grid-barrier counter of the one-launch T = 1 step and the
+ *     item counter of the Gram kernel for T = 256 (both return to zero by
+ *     themselves when a launch completes): calls that may run at the same
+ *     time (different streams) need workspaces of their own; calls ordered
+ *     on one stream can share one.
  *   - Layout: A is B x T x d_in with row stride `lda` ELEMENTS (>= d_in), rows
  *     of one example contiguous (example i starts at row i*T); Zbar likewise
  *     with `ldz`.  Outputs are fp32; gW is d_out x d_in row-major with row

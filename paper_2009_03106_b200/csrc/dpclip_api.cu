@@ -26,6 +26,7 @@ inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // Kernels launched by this library since it was loaded (observability only; never read by a kernel).
 unsigned long long g_launches = 0;
 constexpr int kGridCounterOffset = 64;   // workspace header: status word at 0, grid-barrier counter here
+constexpr int kWorkCounterOffset = 128;  // item counter of the dynamically scheduled Gram kernel (wraps to zero by itself)
 inline int launch_status() {
     ++g_launches;
     return cudaGetLastError() == cudaSuccess ? DPCLIP_OK : DPCLIP_ERR_CUDA;
@@ -350,6 +351,7 @@ int launch_gram_group(const GramLayer* ls, int n, int* status, cudaStream_t st) 
     q.total_groups = groups;
     const int grid = groups < kNumSMs ? groups : kNumSMs;
     if (cls == 0) {
+        q.work_counter = reinterpret_cast<unsigned int*>(reinterpret_cast<char*>(status) + kWorkCounterOffset);
         if (!enable_smem(tc::gram_norm_q2_kernel, g::SMEM_BYTES)) return DPCLIP_ERR_CUDA;
         tc::gram_norm_q2_kernel<<<grid, g::THREADS, g::SMEM_BYTES, st>>>(q);
     } else if (cls == 1) {
@@ -1006,6 +1008,18 @@ int dpclip_same_shape_layers_clipped_grad_noise(const dpclip_layer* layers, int 
         }
         for (int i = 0; i < n; ++i) done[idx[i]] = true;
         if (n < 2) continue;
+        {
+            // Sharing a launch pays when a layer alone leaves every CTA a short row slice (pipeline fill and
+            // epilogue then weigh heavily); layers that already give long slices keep their own launches,
+            // whose one-wave split uses the SMs more evenly (measured on two 512 -> 2048 layers at
+            // B*T = 32768: 174 us together on 128 CTAs, 2 x 80 us apart on 144).
+            const dpclip_layer& y = layers[l0];
+            const int bm = y.d_out > 128 ? 256 : 128;
+            const int tiles = ceil_div(y.d_out, bm) * ceil_div(y.d_in, z::BN);
+            const long nkb = ceil_div((long)B * y.T, (long)z::BK);
+            const int ksplit = tiles < kNumSMs ? kNumSMs / tiles : 1;
+            if (nkb / ksplit >= 32) continue;
+        }
         const int rc = launch_zta_tc_group(grp, idx, n, B, clip, sigma * C, seed, stream_id0, workspace, workspace_bytes,
                                            (cudaStream_t)stream);
         if (rc < 0) return rc;

@@ -81,6 +81,7 @@ struct Launch {
     int group_begin[MAX_LAYERS + 1];
     int L, total_groups;
     int* status;
+    unsigned int* work_counter;    // gram_norm_q2_kernel: items are handed out in order from this counter
 };
 
 // layer of group g (group_begin is ascending; L is small)
@@ -342,19 +343,24 @@ __global__ void __launch_bounds__(gram::THREADS, 1)
 gram_norm_q2_kernel(const __grid_constant__ gram::Launch q) {
     using namespace gram;
     constexpr int STAGES = 6, STAGE_BYTES = 2 * TILE_BYTES;
+    constexpr int SCHED = 4;                               // depth of the item queue
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
     uint64_t* empty = full + STAGES;
     uint64_t* acc_full = empty + STAGES;
     uint64_t* acc_empty = acc_full + 1;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 1);
+    uint64_t* sched_full = acc_empty + 1;                  // item queue: producer -> MMA issuer and epilogue warps
+    uint64_t* sched_empty = sched_full + SCHED;
+    volatile int* sched_item = reinterpret_cast<volatile int*>(sched_empty + SCHED);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(const_cast<int*>(sched_item) + SCHED);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
         mbar_init(acc_full, 1); mbar_init(acc_empty, N_EPILOGUE_WARPS);
+        for (int s = 0; s < SCHED; ++s) { mbar_init(&sched_full[s], 1); mbar_init(&sched_empty[s], 1 + N_EPILOGUE_WARPS); }
         *abort_flag = 0;
         mbar_fence_init();
         for (int l = 0; l < q.L; ++l) { tma_prefetch_desc(&q.map_a[l]); tma_prefetch_desc(&q.map_z[l]); }
@@ -369,8 +375,26 @@ gram_norm_q2_kernel(const __grid_constant__ gram::Launch q) {
         // ------------------------------------------------ TMA producer
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0;
+            int slot = 0; uint32_t sphase = 0;
             bool ok = true;
-            for (int g = blockIdx.x; g < q.total_groups && ok; g += gridDim.x) {
+            [[maybe_unused]] int tr = 0;
+            DPCLIP_TRACE_AT(0, 255);
+            // Items (layer-major, widest layers first) are taken in order from a counter shared by the CTAs,
+            // so a CTA that drew wide examples simply draws fewer of them.  Every CTA draws until it sees a
+            // value past the end, exactly once: after total + grid draws the counter has wrapped to zero,
+            // ready for the next launch.  The next item is drawn before the loads of the current one are
+            // issued, and published to the other roles through a small queue in shared memory.
+            const unsigned int wrap = (unsigned int)q.total_groups + gridDim.x - 1;
+            int g_next = (int)atomicInc(q.work_counter, wrap);
+            while (ok) {
+                const int g = g_next < q.total_groups ? g_next : -1;
+                if (g >= 0) g_next = (int)atomicInc(q.work_counter, wrap);
+                ok = mbar_wait(&sched_empty[slot], sphase ^ 1, abort_flag, q.status);
+                if (!ok) break;
+                sched_item[slot] = g;
+                mbar_arrive(&sched_full[slot]);
+                if (++slot == SCHED) { slot = 0; sphase ^= 1; }
+                if (g < 0) break;
                 const int l = layer_of(q, g);
                 const Params& p = q.layer[l];
                 const bool x_is_z = p.d_out > p.d_in;
@@ -386,6 +410,7 @@ gram_norm_q2_kernel(const __grid_constant__ gram::Launch q) {
                     const int x = (p1 ? kb : (p2 ? kb - nk_x : kb - nk_x - nk_y)) * BK;
                     ok = mbar_wait(&empty[stage], phase ^ 1, abort_flag, q.status);
                     if (!ok) break;
+                    DPCLIP_TRACE_AT(0, tr); ++tr;
                     uint8_t* dst = smem + stage * STAGE_BYTES;
                     mbar_arrive_expect_tx(&full[stage], p2 ? TILE_BYTES : 2 * TILE_BYTES);
                     if (p2) {
@@ -403,8 +428,16 @@ gram_norm_q2_kernel(const __grid_constant__ gram::Launch q) {
         if (lane == 0) {
             constexpr uint32_t idesc256 = make_idesc_bf16(BM, 2 * BM, 0, 0), idesc128 = make_idesc_bf16(BM, BM, 0, 0);
             int stage = 0; uint32_t phase = 0; uint32_t acc_phase = 0;
+            int slot = 0; uint32_t sphase = 0;
             bool ok = true;
-            for (int g = blockIdx.x; g < q.total_groups && ok; g += gridDim.x) {
+            [[maybe_unused]] int tr = 0;
+            while (ok) {
+                ok = mbar_wait(&sched_full[slot], sphase, abort_flag, q.status);
+                if (!ok) break;
+                const int g = sched_item[slot];
+                mbar_arrive(&sched_empty[slot]);
+                if (++slot == SCHED) { slot = 0; sphase ^= 1; }
+                if (g < 0) break;
                 const int l = layer_of(q, g);
                 const Params& p = q.layer[l];
                 const bool x_is_z = p.d_out > p.d_in;
@@ -427,6 +460,7 @@ gram_norm_q2_kernel(const __grid_constant__ gram::Launch q) {
                     }
                     ok = mbar_wait(&full[stage], phase, abort_flag, q.status);
                     if (!ok) break;
+                    DPCLIP_TRACE_AT(2, tr); ++tr;
                     tc_fence_after_sync();
                     const uint32_t t0 = smem_u32(smem + stage * STAGE_BYTES), t1 = t0 + TILE_BYTES;
                     const bool first = p1 ? kb == 0 : (p2 ? kb == nk_x : kb == nk_x + nk_y);
@@ -460,9 +494,18 @@ gram_norm_q2_kernel(const __grid_constant__ gram::Launch q) {
         const int quarter = warp & 3;
         const int half = (warp - 2) >> 2;
         uint32_t acc_phase = 0;
+        int slot = 0; uint32_t sphase = 0;
         bool ok = true;
+        [[maybe_unused]] int etr = 0;
         const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16);
-        for (int g = blockIdx.x; g < q.total_groups && ok; g += gridDim.x) {
+        while (ok) {
+            ok = mbar_wait(&sched_full[slot], sphase, abort_flag, q.status);
+            if (!ok) break;
+            const int g = sched_item[slot];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sched_empty[slot]);
+            if (++slot == SCHED) { slot = 0; sphase ^= 1; }
+            if (g < 0) break;
             const int l = layer_of(q, g);
             const Params& p = q.layer[l];
             const bool x_is_z = p.d_out > p.d_in;
@@ -474,6 +517,7 @@ gram_norm_q2_kernel(const __grid_constant__ gram::Launch q) {
                 // pass 1 = E0: 256 columns of G^X_0 (at 0) and G^Y_0 (at 256), 128 per warp
                 ok = mbar_wait(acc_full, acc_phase, abort_flag, q.status);
                 if (!ok) break;
+                if (threadIdx.x == 64) { DPCLIP_TRACE_AT(3, etr); ++etr; }
                 acc_phase ^= 1;
                 tc_fence_after_sync();
                 const int width = pass == 0 ? 64 : 128;
@@ -495,6 +539,7 @@ gram_norm_q2_kernel(const __grid_constant__ gram::Launch q) {
                 tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(acc_empty);
+                if (threadIdx.x == 64) { DPCLIP_TRACE_AT(3, etr); ++etr; }
                 // block (0,1) stands for its mirror image (1,0) too
                 val += ((pass == 1 && half == 1) ? 2.f : 1.f) * (sa + (p.has_bias ? sb : 0.f));
             }
