@@ -12,6 +12,7 @@
 #include "kernels_tf32.cuh"
 #include "kernels_fused_t1.cuh"
 #include "kernels_narrow.cuh"
+#include "kernels_narrow_tc.cuh"
 #include "kernels_elementwise.cuh"
 
 #include <stdlib.h>
@@ -109,6 +110,34 @@ inline bool narrow_ring_ok(const NarrowParams& p, dpclip_dtype dtype, bool grad)
     return true;
 }
 
+// bf16 narrow layers on the tensor cores (needs the status word of a workspace for its bounded waits)
+inline bool narrow_tc_ok(const NarrowParams& p, dpclip_dtype dtype, const int* status) {
+    const char* env = getenv("DPCLIP_NO_NARROW_TC");
+    if (env && env[0] == '1') return false;
+    return dtype == DPCLIP_BF16 && status != nullptr;
+}
+
+template <bool GRAD>
+int launch_narrow_tc(const NarrowParams& p, int grid, int n_items, int* status, cudaStream_t st) {
+    namespace n = tc::ntc;
+    n::Params q;
+    memset(&q, 0, sizeof(q));
+    q.A = static_cast<const __nv_bfloat16*>(p.A); q.Z = static_cast<const __nv_bfloat16*>(p.Z);
+    q.T = p.T; q.d_in = p.d_in; q.d_out = p.d_out; q.has_bias = p.has_bias;
+    q.n_items = n_items; q.rows_total = p.rows_total; q.rows_per_cta = p.rows_per_cta;
+    // 32-row blocks of dense rows are 64 * d bytes: block starts stay 16-byte aligned when the item starts are
+    const bool bases = aligned_to(p.A, 16) && aligned_to(p.Z, 16);
+    q.vec = bases && (GRAD || (((long)p.T * p.d_in) % 8 == 0 && ((long)p.T * p.d_out) % 8 == 0));
+    q.clip = p.clip; q.sq = p.sq; q.part = p.part; q.part_m = p.d_out <= 32 ? 32 : 64;
+    q.status = status;
+    if (!GRAD && p.d_out > 32 && cudaMemsetAsync(p.sq, 0, sizeof(float) * (size_t)n_items, st) != cudaSuccess)
+        return DPCLIP_ERR_CUDA;
+    if (cudaFuncSetAttribute(tc::narrow_tc_kernel<GRAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, n::SMEM_BYTES) !=
+        cudaSuccess) return DPCLIP_ERR_CUDA;
+    tc::narrow_tc_kernel<GRAD><<<grid, n::THREADS, n::SMEM_BYTES, st>>>(q);
+    return launch_status();
+}
+
 template <bool GRAD>
 int launch_narrow(const NarrowParams& p, int grid, int d_out, dpclip_dtype dtype, cudaStream_t st) {
     if (narrow_ring_ok(p, dtype, GRAD)) {
@@ -124,12 +153,14 @@ int launch_narrow(const NarrowParams& p, int grid, int d_out, dpclip_dtype dtype
 }
 
 int launch_simt_norms(const void* A, long lda, const void* Z, long ldz, int B, int T, int d_in, int d_out,
-                      dpclip_dtype dtype, int has_bias, float* sq, cudaStream_t st) {
+                      dpclip_dtype dtype, int has_bias, float* sq, cudaStream_t st, int* status = nullptr) {
     if (narrow_layer(T, d_in, d_out, has_bias, lda, ldz)) {
         NarrowParams q;
         memset(&q, 0, sizeof(q));
         q.A = A; q.lda = lda; q.Z = Z; q.ldz = ldz; q.T = T; q.d_in = d_in; q.d_out = d_out;
         q.has_bias = has_bias ? 1 : 0; q.sq = sq;
+        if (narrow_tc_ok(q, dtype, status))
+            return launch_narrow_tc<false>(q, B < kNumSMs ? B : kNumSMs, B, status, st);
         return launch_narrow<false>(q, B, d_out, dtype, st);
     }
     SimtParams p;
@@ -160,8 +191,10 @@ int launch_simt_grad(const void* A, long lda, const void* Z, long ldz, int B, in
         q.A = A; q.lda = lda; q.Z = Z; q.ldz = ldz; q.T = T; q.d_in = d_in; q.d_out = d_out;
         q.has_bias = gb ? 1 : 0; q.clip = clip; q.gW = gW; q.ldg = ldg; q.gb = gb;
         q.rows_total = (long)B * T;
+        int* status = (workspace && workspace_bytes >= (size_t)kHeaderBytes) ? static_cast<int*>(workspace) : nullptr;
+        const bool on_tc = narrow_tc_ok(q, dtype, status);
         // one wave: a CTA of the register-staged kernel holds a whole SM; the cp.async form runs two per SM
-        int grid = narrow_ring_ok(q, dtype, true) ? 2 * kNumSMs : kNumSMs;
+        int grid = (!on_tc && narrow_ring_ok(q, dtype, true)) ? 2 * kNumSMs : kNumSMs;
         const long min_rows = NARROW_WARPS * 32;                   // at least one chunk per warp
         if ((long)grid * min_rows > q.rows_total) grid = (int)((q.rows_total + min_rows - 1) / min_rows);
         // whole 32-row chunks per CTA: every chunk of a dense layer then starts on a 16-byte boundary whatever
@@ -173,7 +206,7 @@ int launch_simt_grad(const void* A, long lda, const void* Z, long ldz, int B, in
         if (workspace && workspace_bytes >= (size_t)kHeaderBytes + part_bytes && grid > 1) {
             // partial tile per CTA, then a fixed-order reduce that also adds the noise
             q.part = reinterpret_cast<float*>(static_cast<char*>(workspace) + kHeaderBytes);
-            int rc = launch_narrow<true>(q, grid, d_out, dtype, st);
+            int rc = on_tc ? launch_narrow_tc<true>(q, grid, 1, status, st) : launch_narrow<true>(q, grid, d_out, dtype, st);
             if (rc) return rc;
             NarrowReduceParams r;
             memset(&r, 0, sizeof(r));
@@ -916,7 +949,8 @@ int dpclip_layer_sqnorms(const void* A, long lda, const void* Zbar, long ldz, in
             if (T != 1) return DPCLIP_ERR_UNSUPPORTED;
             return launch_t1_norms(A, lda, Zbar, ldz, B, d_in, d_out, dtype, has_bias, sq_layer, st);
         case DPCLIP_SIMT:
-            return launch_simt_norms(A, lda, Zbar, ldz, B, T, d_in, d_out, dtype, has_bias, sq_layer, st);
+            return launch_simt_norms(A, lda, Zbar, ldz, B, T, d_in, d_out, dtype, has_bias, sq_layer, st,
+                                     static_cast<int*>(workspace));
         case DPCLIP_GRAM:
         case DPCLIP_MATERIALIZE:
             if (dtype == DPCLIP_F32) {                    // fp32: materialised tiles via error-compensated tf32

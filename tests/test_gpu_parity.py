@@ -350,7 +350,8 @@ def test_clipped_grad(dp, dtype, B, T, d_in, d_out):
     dp.dpclip_clipped_grad(dA, dZ, torch.from_numpy(clip).cuda(), gW, gb, ws)
     # identical inputs and fp32 accumulation: the fp32 bound applies, except on the tensor-core path,
     # which rounds clip*zbar to bf16 in shared memory (bf16 rows that are 16-byte multiples take it)
-    on_tc = dtype == "bf16" and d_in % 8 == 0 and d_out % 8 == 0
+    narrow = T > 1 and d_in + 1 <= 32 and d_out <= 64
+    on_tc = dtype == "bf16" and ((d_in % 8 == 0 and d_out % 8 == 0) or narrow)
     tol = TOL["bf16"]["grad"] if on_tc else TOL["f32"]["grad"]
     assert rel_fro(gW.cpu().numpy(), refW) <= tol
     assert rel_fro(gb.cpu().numpy(), refb) <= tol
@@ -618,6 +619,42 @@ def test_step_mlp_bf16_tensor_core(dp, monkeypatch):
     monkeypatch.setenv("DPCLIP_T1_ONE_LAUNCH", "0")
     layers = workloads.generate(edges, 7)
     _check_step(dp, edges, _calibrate(edges, layers, 7, edges.C), edges.C, edges.sigma, 7)
+
+
+NARROW_TC_SHAPES = [(128, 1024, 27, 32),      # the first convolution of the CNN: aligned 32-row blocks, vector loads
+                    (3, 100, 27, 32),         # item starts off the 16-byte grid: element-wise loads
+                    (5, 72, 27, 32),          # aligned, a ragged last block (72 = 2 * 32 + 8)
+                    (300, 64, 24, 64),        # more examples than SMs (several items per CTA), both lane quarters
+                    (4, 40, 31, 40), (2, 33, 5, 3), (7, 2, 1, 1)]
+
+
+@pytest.mark.parametrize("B,T,d_in,d_out", NARROW_TC_SHAPES)
+@pytest.mark.parametrize("has_bias", [True, False])
+def test_narrow_layers_tensor_core(dp, B, T, d_in, d_out, has_bias):
+    """bf16 narrow layers: blocks of rows scattered into the operand layout by the fill warps, contraction on
+    the tensor cores.  Norms see exact products; the clipped sum rounds c * zb once to bf16."""
+    A, Z = workloads.random_layer(60, B, T, d_in, d_out, "bf16", scale_z=0.05)
+    n = min(B, 12)                                            # the oracle materialises every example: sample
+    idx = np.unique(np.concatenate([np.arange(min(n, B)), np.arange(max(0, B - 3), B), [B // 2]]))
+    ref = oracle.layer_sqnorms(A[idx], Z[idx], has_bias)
+    got = _sqnorms(dp, A, Z, "bf16", has_bias)
+    assert max_rel(np.sqrt(got[idx]), np.sqrt(ref)) <= TOL["f32"]["norm"]
+    clip = np.random.default_rng(B).uniform(0.05, 1.0, B).astype(np.float32)
+    clip[::3] = 1.0
+    refW, refb = oracle.clipped_grad(A, Z, clip)
+    gW = torch.full((d_out, d_in), 9.0, device="cuda")
+    gb = torch.full((d_out,), 9.0, device="cuda") if has_bias else None
+    ws = _ws(dp)
+    dp.dpclip_clipped_grad(to_device(A, "bf16"), to_device(Z, "bf16"), torch.from_numpy(clip).cuda(), gW, gb, ws)
+    torch.cuda.synchronize()
+    assert dp.dpclip_read_status(ws) == 0
+    assert rel_fro(gW.cpu().numpy(), refW) <= TOL["bf16"]["grad"]
+    if has_bias:
+        assert rel_fro(gb.cpu().numpy(), refb) <= TOL["bf16"]["grad"]
+    # no factors: exact products, fp32 accumulation
+    refW1, _ = oracle.clipped_grad(A, Z, None)
+    dp.dpclip_clipped_grad(to_device(A, "bf16"), to_device(Z, "bf16"), None, gW, gb, ws)
+    assert rel_fro(gW.cpu().numpy(), refW1) <= 2e-5
 
 
 def test_narrow_layer_register_staged_form(dp, monkeypatch):
