@@ -110,11 +110,15 @@ inline bool narrow_ring_ok(const NarrowParams& p, dpclip_dtype dtype, bool grad)
     return true;
 }
 
-// bf16 narrow layers on the tensor cores (needs the status word of a workspace for its bounded waits)
+// bf16 narrow layers on the tensor cores: needs the status word of a workspace for its bounded waits, and
+// items (examples, row slices) that start and end on 16-byte boundaries in both inputs, which the bulk copies
+// into shared memory ask for
 inline bool narrow_tc_ok(const NarrowParams& p, dpclip_dtype dtype, const int* status) {
     const char* env = getenv("DPCLIP_NO_NARROW_TC");
     if (env && env[0] == '1') return false;
-    return dtype == DPCLIP_BF16 && status != nullptr;
+    if (dtype != DPCLIP_BF16 || status == nullptr) return false;
+    if (!aligned_to(p.A, 16) || !aligned_to(p.Z, 16)) return false;
+    return ((long)p.T * p.d_in) % 8 == 0 && ((long)p.T * p.d_out) % 8 == 0;
 }
 
 template <bool GRAD>
@@ -125,9 +129,6 @@ int launch_narrow_tc(const NarrowParams& p, int grid, int n_items, int* status, 
     q.A = static_cast<const __nv_bfloat16*>(p.A); q.Z = static_cast<const __nv_bfloat16*>(p.Z);
     q.T = p.T; q.d_in = p.d_in; q.d_out = p.d_out; q.has_bias = p.has_bias;
     q.n_items = n_items; q.rows_total = p.rows_total; q.rows_per_cta = p.rows_per_cta;
-    // 32-row blocks of dense rows are 64 * d bytes: block starts stay 16-byte aligned when the item starts are
-    const bool bases = aligned_to(p.A, 16) && aligned_to(p.Z, 16);
-    q.vec = bases && (GRAD || (((long)p.T * p.d_in) % 8 == 0 && ((long)p.T * p.d_out) % 8 == 0));
     q.clip = p.clip; q.sq = p.sq; q.part = p.part; q.part_m = p.d_out <= 32 ? 32 : 64;
     q.status = status;
     if (!GRAD && p.d_out > 32 && cudaMemsetAsync(p.sq, 0, sizeof(float) * (size_t)n_items, st) != cudaSuccess)

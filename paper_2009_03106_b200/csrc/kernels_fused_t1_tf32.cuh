@@ -176,7 +176,7 @@ t1_all_grads_tf32_kernel(const __grid_constant__ f1::Params q) {
     constexpr int BOXES = BF16 ? 2 : 4, BOX_COLS = BF16 ? 64 : 32;          // TMA boxes per 128-column tile
     const FusedT1Params& p = q.base;
     extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);   // 1024-byte aligned; an offset from the array keeps the accesses in the shared state space
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);   // TMA landed
     uint64_t* ready = full + STAGES;                                             // low planes written (all 16 warps)
     uint64_t* empty = ready + STAGES;                                            // MMA done with the stage

@@ -78,7 +78,7 @@ zta_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     using namespace t32;
     using zta::Item;
     extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);   // 1024-byte aligned; an offset from the array keeps the accesses in the shared state space
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);   // TMA landed
     uint64_t* ready = full + STAGES;                                             // hi/lo planes written
     uint64_t* empty = ready + STAGES;                                            // MMA done with the stage

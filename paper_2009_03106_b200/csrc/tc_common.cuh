@@ -51,7 +51,11 @@ constexpr uint64_t kWaitLimitNs = 2000000000ull;
 
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
                                           int* status_word) {
-    if (mbar_try_wait(bar, parity)) return true;
+    // Fast path without the clock: reading %globaltimer is slow (it shows as a long-scoreboard stall of
+    // several hundred nanoseconds), and try_wait itself already blocks for a while before it gives up.
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = global_ns();
     uint32_t spins = 0;
     while (true) {
