@@ -223,3 +223,53 @@ def test_grid_barrier_timeout_is_reported_and_recoverable(dp):
     torch.cuda.synchronize()
     assert dp.dpclip_read_status(plan.workspace) == 0
     assert torch.equal(plan.flat, good)
+
+
+def test_grouped_launches_repeat_over_thousands_of_calls(dp):
+    """The Gram kernel for two-block examples draws its items from a counter in the workspace header that must be
+    back at zero after every launch (it wraps after total + grid draws), and the narrow tensor-core kernel
+    re-arms its rings per launch: two thousand back-to-back launches of each give the first launch's result every
+    time (the sums are combined by atomics, so equal up to fp32 rounding order), and the status word stays clear."""
+    w = workloads.seq("bf16", B=40, T=256, d=64, d_ff=136)
+    data = workloads.generate(w, 3)
+    layers = [dp.Layer(to_device(A, "bf16"), to_device(Z, "bf16"), s.has_bias, dp.DPCLIP_GRAM)
+              for (A, Z), s in zip(data, w.layers)]
+    plan = dp.StepPlan(layers)
+    taken = dp.dpclip_gram_layers_sqnorms(plan)
+    assert all(taken)
+    torch.cuda.synchronize()
+    first = plan.sq_layers.clone()
+    sample = [0, 17, 39]
+    for l, ((A, Z), s) in enumerate(zip(data, w.layers)):
+        ref = oracle.layer_sqnorms(A[sample], Z[sample], s.has_bias)
+        assert max_rel(np.sqrt(first[l].cpu().numpy()[sample]), np.sqrt(ref)) <= TOL["bf16"]["norm"]
+    worst = torch.zeros((), device="cuda")
+    for it in range(2000):
+        dp.dpclip_gram_layers_sqnorms(plan)
+        if it % 100 == 99:
+            worst = torch.maximum(worst, ((plan.sq_layers - first).abs() / first).max())
+    torch.cuda.synchronize()
+    assert dp.dpclip_read_status(plan.workspace) == 0
+    assert float(worst) <= 1e-5
+    # narrow tensor-core kernel: norms (several items per CTA) and clipped sum, 2000 launches each
+    B, T, d_in, d_out = 200, 128, 27, 32
+    A, Z = workloads.random_layer(71, B, T, d_in, d_out, "bf16", scale_z=0.05)
+    dA, dZ = to_device(A, "bf16"), to_device(Z, "bf16")
+    ws = torch.empty(max(1 << 20, dp.dpclip_workspace_bytes(B, T, d_in, d_out, 1, 0)), dtype=torch.uint8, device="cuda")
+    dp.dpclip_workspace_init(ws)
+    sq = torch.empty(B, device="cuda"); gW = torch.empty(d_out, d_in, device="cuda"); gb = torch.empty(d_out, device="cuda")
+    clip = torch.rand(B, device="cuda") * 0.9 + 0.1
+    dp.dpclip_layer_sqnorms(dA, dZ, True, sq, ws); dp.dpclip_clipped_grad(dA, dZ, clip, gW, gb, ws)
+    torch.cuda.synchronize()
+    sq0, gW0, gb0 = sq.clone(), gW.clone(), gb.clone()
+    ref = oracle.layer_sqnorms(A[:4], Z[:4], True)
+    assert max_rel(np.sqrt(sq0.cpu().numpy()[:4]), np.sqrt(ref)) <= TOL["bf16"]["norm"]
+    same = torch.ones((), dtype=torch.bool, device="cuda")
+    for it in range(2000):
+        dp.dpclip_layer_sqnorms(dA, dZ, True, sq, ws)
+        dp.dpclip_clipped_grad(dA, dZ, clip, gW, gb, ws)
+        if it % 100 == 99:
+            same &= torch.equal(sq, sq0) & torch.equal(gW, gW0) & torch.equal(gb, gb0)
+    torch.cuda.synchronize()
+    assert dp.dpclip_read_status(ws) == 0
+    assert bool(same)                       # no atomics on this path: bit for bit
