@@ -13,6 +13,7 @@
 #include "kernels_fused_t1.cuh"
 #include "kernels_narrow.cuh"
 #include "kernels_narrow_tc.cuh"
+#include "kernels_conv_tc.cuh"
 #include "kernels_elementwise.cuh"
 
 #include <stdlib.h>
@@ -1181,6 +1182,80 @@ static bool conv_tf32_ok(const SimtParams& p, const void* X, const void* Zbar, i
     return true;
 }
 
+// bf16 convolution layers on the tensor cores (implicit im2col): see kernels_conv_tc.cuh for the restrictions
+static bool conv_tc_ok(const SimtParams& p, const void* X, const void* Zbar, int z_channel_major, int B, int T,
+                       dpclip_dtype dtype, const void* workspace, size_t workspace_bytes) {
+    { const char* env = getenv("DPCLIP_FORCE_SIMT"); if (env && env[0] == '1') return false; }
+    { const char* env = getenv("DPCLIP_NO_CONV_TC"); if (env && env[0] == '1') return false; }
+    if (dtype != DPCLIP_BF16 || z_channel_major || !workspace || workspace_bytes < (size_t)kHeaderBytes) return false;
+    if (p.stride != 1 || !(p.Wo == 8 || p.Wo == 16 || p.Wo == 32 || p.Wo == 64) || T % 64 != 0) return false;
+    if (p.d_out % 8 != 0 || p.d_out > 128) return false;
+    const long x_elems = (long)p.cC * p.cH * p.cW;
+    if (x_elems * 2 > tc::ctc::X_BYTES || x_elems % 8 != 0) return false;
+    return aligned_to(X, 16) && aligned_to(Zbar, 16);
+}
+
+extern "C++" {
+template <bool GRAD>
+static int launch_conv_tc(const SimtParams& sp, const void* X, const void* Zbar, int B, int T, int has_bias,
+                          const float* clip, float* sq, float* gW, long ldg, float* gb, void* workspace,
+                          size_t workspace_bytes, cudaStream_t st) {
+    namespace c = tc::ctc;
+    CUtensorMap mz;
+    if (!make_map_bf16(&mz, Zbar, (long)B * T, sp.d_out, sp.d_out, 64, c::BK)) return DPCLIP_ERR_CUDA;
+    c::Params p;
+    memset(&p, 0, sizeof(p));
+    p.X = static_cast<const __nv_bfloat16*>(X);
+    p.B = B; p.C = sp.cC; p.H = sp.cH; p.W = sp.cW; p.kh = sp.kh; p.kw = sp.kw; p.pad = sp.pad;
+    p.Wo = sp.Wo; p.Ho = T / sp.Wo;
+    p.wo_shift = sp.Wo == 8 ? 3 : sp.Wo == 16 ? 4 : sp.Wo == 32 ? 5 : 6;
+    p.T = T; p.d_in = sp.d_in; p.d_out = sp.d_out; p.has_bias = has_bias ? 1 : 0;
+    p.tiles_n = ceil_div(sp.d_in + p.has_bias, c::BN);
+    p.status = static_cast<int*>(workspace);
+    int slices = 1;
+    if (GRAD) {
+        // one wave: as many slices of examples as there are SMs per block of patch columns
+        slices = kNumSMs / p.tiles_n;
+        if (slices > B) slices = B;
+        if (slices < 1) slices = 1;
+        p.ex_per_item = ceil_div(B, slices);
+        slices = ceil_div(B, p.ex_per_item);
+        p.n_items = slices * p.tiles_n;
+        const size_t part_bytes = (size_t)p.n_items * 128 * c::BN * 4;
+        if (workspace_bytes < (size_t)kHeaderBytes + part_bytes) return 1;        // the caller takes the fp32-ALU kernel
+        p.part = reinterpret_cast<float*>(static_cast<char*>(workspace) + kHeaderBytes);
+        p.clip = clip;
+    } else {
+        p.ex_per_item = 1;
+        p.n_items = B * p.tiles_n;
+        p.sq = sq;
+        if (cudaMemsetAsync(sq, 0, sizeof(float) * (size_t)B, st) != cudaSuccess) return DPCLIP_ERR_CUDA;
+    }
+    if (!enable_smem(tc::conv_tc_kernel<GRAD>, c::SMEM_BYTES)) return DPCLIP_ERR_CUDA;
+    const int grid = p.n_items < kNumSMs ? p.n_items : kNumSMs;
+    tc::conv_tc_kernel<GRAD><<<grid, c::THREADS, c::SMEM_BYTES, st>>>(mz, p);
+    int rc = launch_status();
+    if (rc || !GRAD) return rc;
+    // fixed-order sum of the slices' tiles; the bias sums are column d_in of the tiles
+    tc::zta::Params zp;
+    memset(&zp, 0, sizeof(zp));
+    zp.part = p.part; zp.tiles_n = p.tiles_n; zp.vec_ok = aligned_to(gW, 16) && ldg % 4 == 0;
+    tc::ReduceParams r;
+    memset(&r, 0, sizeof(r));
+    r.part = p.part; r.n_tiles = p.tiles_n; r.tiles_n = p.tiles_n; r.ksplit = slices; r.BM = 128; r.BN = c::BN;
+    r.d_out = sp.d_out; r.d_in = sp.d_in; r.gW = gW; r.ldg = ldg; r.gb = gb; r.vec_ok = zp.vec_ok;
+    r.bias_col = 1;
+    const long n_vec = (long)sp.d_out * ((sp.d_in + 3) / 4);
+    int lanes = 1;
+    while (lanes < 8 && lanes * 2 <= slices && n_vec * lanes < 2L * kNumSMs * 256) lanes *= 2;
+    r.lanes = lanes;
+    long blocks = (n_vec + (256 / lanes) - 1) / (256 / lanes);
+    if (blocks > 8L * kNumSMs) blocks = 8L * kNumSMs;
+    tc::reduce_partials_kernel<<<(unsigned)blocks, 256, 0, st>>>(r);
+    return launch_status();
+}
+}  // extern "C++"
+
 int dpclip_conv_sqnorms(const void* X, const void* Zbar, int z_channel_major, int B, const dpclip_conv* geom,
                         int d_out, dpclip_dtype dtype, int has_bias, float* sq_layer, void* workspace,
                         size_t workspace_bytes, void* stream) {
@@ -1192,6 +1267,9 @@ int dpclip_conv_sqnorms(const void* X, const void* Zbar, int z_channel_major, in
     if (B > 65535) return DPCLIP_ERR_UNSUPPORTED;
     cudaStream_t st = (cudaStream_t)stream;
     tc::ConvGather cg;
+    if (conv_tc_ok(p, X, Zbar, z_channel_major, B, T, dtype, workspace, workspace_bytes))
+        return launch_conv_tc<false>(p, X, Zbar, B, T, has_bias, nullptr, sq_layer, nullptr, 0, nullptr, workspace,
+                                     workspace_bytes, st);
     if (conv_tf32_ok(p, X, Zbar, z_channel_major, B, T, dtype, workspace, workspace_bytes, &cg))
         return launch_zta_tf32(nullptr, p.d_in, Zbar, d_out, B, T, p.d_in, d_out, true, has_bias, nullptr, nullptr, 0,
                                nullptr, sq_layer, workspace, workspace_bytes, nullptr, nullptr, st, &cg);
@@ -1219,6 +1297,10 @@ int dpclip_conv_clipped_grad(const void* X, const void* Zbar, int z_channel_majo
     if (!aligned_to(gW, 4) || (gb && !aligned_to(gb, 4))) return DPCLIP_ERR_MISALIGNED;
     cudaStream_t st = (cudaStream_t)stream;
     tc::ConvGather cg;
+    if (conv_tc_ok(p, X, Zbar, z_channel_major, B, T, dtype, workspace, workspace_bytes)) {
+        rc = launch_conv_tc<true>(p, X, Zbar, B, T, gb != nullptr, clip, nullptr, gW, ldg, gb, workspace, workspace_bytes, st);
+        if (rc <= 0) return rc;
+    }
     if (conv_tf32_ok(p, X, Zbar, z_channel_major, B, T, dtype, workspace, workspace_bytes, &cg) &&
         workspace_bytes >= (size_t)kHeaderBytes + kTcScratchBytes)
         return launch_zta_tf32(nullptr, p.d_in, Zbar, d_out, B, T, p.d_in, d_out, false, 0, clip, gW, ldg, gb, nullptr,

@@ -954,6 +954,7 @@ struct ReduceParams {
     // y * tiles_layer of every row slice, and its outputs and noise streams come from the arrays (n_layers
     // == 0: a single layer described by the scalar fields above).
     int n_layers, tiles_layer;
+    int bias_col;                                               // 1: the bias sums are column d_in of the tiles (no bias_part)
     float* gW_l[zta::MAX_LAYERS]; float* gb_l[zta::MAX_LAYERS];
     uint32_t sw0_l[zta::MAX_LAYERS], sw1_l[zta::MAX_LAYERS], sb0_l[zta::MAX_LAYERS], sb1_l[zta::MAX_LAYERS];
 };
@@ -1045,9 +1046,16 @@ reduce_partials_kernel(const ReduceParams q) {
         for (int m = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; m < p.d_out; m += (gridDim.x * blockDim.x) >> 5) {
             const int tm = m / p.BM;
             float acc = 0.f;
-            for (int j = lane; j < n_part; j += 32) {
-                const int ks = j / p.tiles_n, tn = j - ks * p.tiles_n;
-                acc += p.bias_part[((size_t)ks * p.n_tiles + tm * p.tiles_n + tn) * p.BM + (m - tm * p.BM)];
+            if (p.bias_col) {
+                // the tiles were built from [A | 1]: the sums sit in column d_in of the tile that holds it
+                const int tn = p.d_in / p.BN, cb = p.d_in - tn * p.BN;
+                for (int ks = lane; ks < p.ksplit; ks += 32)
+                    acc += p.part[(((size_t)ks * p.n_tiles + tm * p.tiles_n + tn) * p.BM + (m - tm * p.BM)) * p.BN + cb];
+            } else {
+                for (int j = lane; j < n_part; j += 32) {
+                    const int ks = j / p.tiles_n, tn = j - ks * p.tiles_n;
+                    acc += p.bias_part[((size_t)ks * p.n_tiles + tm * p.tiles_n + tn) * p.BM + (m - tm * p.BM)];
+                }
             }
             acc = warp_sum(acc);
             if (lane != 0) continue;

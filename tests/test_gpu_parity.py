@@ -264,6 +264,11 @@ CONV_CASES = [  # B, C, H, W, k, pad, stride, d_out
     (2, 2, 11, 10, 5, 2, 3, 9), (3, 8, 4, 4, 4, 0, 1, 6),
     # large enough for the tensor-core form (fp32, dL/dZ row-major): ragged tiles, stride, rectangular kernel
     (8, 32, 16, 16, 3, 1, 1, 64), (64, 16, 20, 18, (3, 2), 1, 2, 72), (3, 40, 30, 30, 3, 0, 1, 132),
+    # shapes the bf16 tensor-core form takes (stride 1, output width 8 .. 64, T % 64 == 0, d_out % 8 == 0, <= 128): three
+    # blocks of patch columns with both Zb chunks, more examples than SMs, a rectangular kernel without padding, a 5 x 5
+    # kernel with a ragged d_out, a 32 x 32 map
+    (5, 64, 8, 8, 3, 1, 1, 128), (160, 4, 8, 8, 3, 1, 1, 16), (3, 6, 10, 8, (3, 1), 0, 1, 24), (2, 8, 16, 16, 5, 2, 1, 40),
+    (2, 3, 32, 32, 3, 1, 1, 32),
 ]
 
 
