@@ -453,7 +453,7 @@ def bench_elementwise(torch, dp, B, T, d, dtype, steps, flush, peaks):
 
 
 def bench_conv_implicit(torch, dp, name, B, C, H, W, k, pad, d_out, dtype, steps, flush, peaks):
-    """A convolution layer straight from its feature map (implicit im2col, fp32-ALU tiles), next to the same
+    """A convolution layer straight from its feature map (implicit im2col on the tensor cores), next to the same
     layer through the patch-matrix entry points.  Algorithmic bytes: feature map + Zbar once per kernel."""
     X, Z = workloads.conv_inputs(0, B, C, H, W, k, pad, 1, d_out, dtype, var_z=1.0 / B)
     A = workloads.im2col(X, k, pad)
@@ -473,17 +473,16 @@ def bench_conv_implicit(torch, dp, name, B, C, H, W, k, pad, d_out, dtype, steps
                            lambda: dp.dpclip_clipped_grad(dA, dZ, clip, gW, gb, ws))):
         ms = float(np.median(time_steps(torch, fn, steps, 3, flush)))
         ms_ref = float(np.median(time_steps(torch, ref, steps, 3, flush)))
-        # fp32 layers of this size take the tensor-core form (three tf32 MMAs per product); the binding roof is the
-        # larger of bytes / HBM and flops / (3 x tf32)
-        peak_tf = peaks["bf16_tflops"] * TF32X3_PER_BF16 if dtype == "f32" else FFMA_PEAK_TFLOPS
+        # layers of this size take the tensor-core forms (fp32: three tf32 MMAs per product); the binding roof is the
+        # larger of bytes / HBM and flops / the tensor peak of the form
+        peak_tf = peaks["bf16_tflops"] * (TF32X3_PER_BF16 if dtype == "f32" else 1.0)
         t_hbm, t_mma = nbytes / (peaks["hbm_gbs"] * 1e9), flops / (peak_tf * 1e12)
         if t_hbm >= t_mma:
             ach = nbytes / (ms * 1e-3) / 1e9
             roof = dict(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s", frac=ach / peaks["hbm_gbs"])
         else:
             ach = flops / (ms * 1e-3) / 1e12
-            roof = dict(bound="tensor" if dtype == "f32" else "alu", achieved=ach, peak=peak_tf, unit="TFLOP/s",
-                        frac=ach / peak_tf)
+            roof = dict(bound="tensor", achieved=ach, peak=peak_tf, unit="TFLOP/s", frac=ach / peak_tf)
         roof.update(traffic=None, peak_source=peaks["source"])
         out[kind] = dict(ms=ms, patch_matrix_path_ms=ms_ref, roofline=roof)
     return out
@@ -722,9 +721,10 @@ def main():
             for shape in ((128, 256, 512, "bf16"), (512, 512, 1024, "bf16")):
                 r = bench_elementwise(torch, dp, *shape, min(args.steps, 20), flush, peaks)
                 others[r["workload"]] = r
-            r = bench_conv_implicit(torch, dp, "conv2_implicit_im2col_b128_f32", 128, 32, 16, 16, 3, 1, 64, "f32",
-                                    min(args.steps, 20), flush, peaks)
-            others[r["workload"]] = r
+            for cdt in ("f32", "bf16"):
+                r = bench_conv_implicit(torch, dp, "conv2_implicit_im2col_b128_" + cdt, 128, 32, 16, 16, 3, 1, 64, cdt,
+                                        min(args.steps, 20), flush, peaks)
+                others[r["workload"]] = r
         line["workloads"] = others
         if not args.no_cpu_baseline:
             line["cpu_baseline"], _, _ = oracle_sample(w)

@@ -31,8 +31,9 @@ constexpr int P_BYTES = BN * 128;                // patch tile: 256 N-rows x 64 
 constexpr int STAGE_BYTES = Z_BYTES + P_BYTES;   // 48 KB
 constexpr int STAGES = 3;
 constexpr int X_BYTES = 32 * 1024;               // raw feature map of one example (two buffers)
-constexpr int PATCH_WARPS = 8, SCALE_WARPS = 4, EPI_WARPS = 4;
-constexpr int THREADS = 32 * (2 + EPI_WARPS + PATCH_WARPS + SCALE_WARPS);   // warp 0 copies, 1 MMA, 2..5 epilogue, 6..13 patches, 14..17 scale
+constexpr int PATCH_WARPS = 16, SCALE_WARPS = 4, EPI_WARPS = 4;   // the converter is bound by the latency of its
+                                                                  // dependent integer chains: four warps per scheduler
+constexpr int THREADS = 32 * (2 + EPI_WARPS + PATCH_WARPS + SCALE_WARPS);   // warp 0 copies, 1 MMA, 2..5 epilogue, 6..21 patches, 22..25 scale
 constexpr int TAB_BYTES = 2 * BN * 8;             // patch-column tables of two items in flight
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 2 * X_BYTES + TAB_BYTES + 256 + 1024;
 
@@ -62,6 +63,22 @@ __device__ __forceinline__ uint4 shifted8(const uint4& cur, const uint4& nb, int
     const uint32_t sh = (uint32_t)half * 16u;
     return make_uint4(__funnelshift_r(w0, w1, sh), __funnelshift_r(w1, w2, sh), __funnelshift_r(w2, w3, sh),
                       __funnelshift_r(w3, w4, sh));
+}
+// The same for a dx that is uniform across the warp: a plain switch.
+__device__ __forceinline__ uint4 shifted8u(const uint4& prev, const uint4& cur, const uint4& next, int dx) {
+    switch (dx) {
+        case -3: return make_uint4(__funnelshift_r(prev.z, prev.w, 16), __funnelshift_r(prev.w, cur.x, 16),
+                                   __funnelshift_r(cur.x, cur.y, 16), __funnelshift_r(cur.y, cur.z, 16));
+        case -2: return make_uint4(prev.w, cur.x, cur.y, cur.z);
+        case -1: return make_uint4(__funnelshift_r(prev.w, cur.x, 16), __funnelshift_r(cur.x, cur.y, 16),
+                                   __funnelshift_r(cur.y, cur.z, 16), __funnelshift_r(cur.z, cur.w, 16));
+        case 1:  return make_uint4(__funnelshift_r(cur.x, cur.y, 16), __funnelshift_r(cur.y, cur.z, 16),
+                                   __funnelshift_r(cur.z, cur.w, 16), __funnelshift_r(cur.w, next.x, 16));
+        case 2:  return make_uint4(cur.y, cur.z, cur.w, next.x);
+        case 3:  return make_uint4(__funnelshift_r(cur.y, cur.z, 16), __funnelshift_r(cur.z, cur.w, 16),
+                                   __funnelshift_r(cur.w, next.x, 16), __funnelshift_r(next.x, next.y, 16));
+        default: return cur;
+    }
 }
 }  // namespace ctc
 
@@ -229,33 +246,59 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_z, const ctc::Params p) {
             }
         }
     } else if (warp < 2 + EPI_WARPS + PATCH_WARPS) {
-        // ------------------------------------------------ patch tiles.  Thread = (K-unit u = t % 8, N-row group t / 8): in
-        // each of eight passes the eight lanes of a group fill the eight 16-byte units of ONE N-row (128
-        // contiguous bytes of the tile), reading eight neighbouring 16-byte runs of the feature map; four N-rows
-        // (mostly one channel) per warp and pass.  (With thread = N-row the lanes of a warp sat a whole channel
-        // apart in the feature map, the 2-byte loads hit the same banks four at a time, and the shared-memory
-        // pipe bounded the kernel: 1.25 us per stage.)
-        const int t = threadIdx.x - 32 * (2 + EPI_WARPS);      // 0 .. 255
-        const int u = t & 7, nq = t >> 3;
-        const int khw = p.kh * p.kw;
+        // ------------------------------------------------ patch tiles.  The k_w patch columns (c, ky, 0 .. k_w - 1) read
+        // the same input row shifted by one pixel each, so a thread takes one such GROUP of columns and one
+        // K-unit u (eight consecutive t = one output row y', eight neighbouring x'): it loads the aligned 16-byte
+        // vector of the row and its two neighbours once, and every column of the group is a funnel shift of
+        // them (zeros at the edge of the map), stored as the 16-byte unit u of that column's N-row.  Lanes =
+        // (u = t % 8, group t / 8): the eight u of a group read 128 contiguous bytes and write 128 contiguous
+        // bytes per column.  Per unit ~10 instructions; with one thread per unit and column the converter
+        // needed ~45 and bounded the kernel (issue slots: 0.6 us per stage before a single load).
+        const int t = threadIdx.x - 32 * (2 + EPI_WARPS);      // 0 .. 511
+        constexpr int GQ = 4 * PATCH_WARPS;                    // groups per pass
+        const int u = t & 7, gq = t >> 3;
         const bool vec_rows = (p.W & 7) == 0 && p.pad <= 3 && p.kw - 1 - p.pad <= 3;
+        const bool fast3 = vec_rows && p.kw == 3 && p.pad == 1;
         int g = 0, xe = 0, it = 0;
         bool ok = true;
         for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x, ++it) {
             int e0, ne, j; decode(item, e0, ne, j);
-            // The item's patch columns, decoded once: thread t writes the entry of column t.  Two tables (item
-            // parity): nobody can still be reading the one written here, because the table of the item before this
-            // one was complete only after every warp had finished the item before that.
+            const int n0 = j * BN;                                         // first patch column of the block
+            const int n_real = min(BN, p.d_in - n0);                       // real columns in the block (> 0)
+            const int n_rows = (min(BN, p.d_in + p.has_bias - n0) + 31) & ~31;     // N-rows the MMAs read
+            const int rg0 = n0 / p.kw;                                     // first group that overlaps the block
+            const int n_groups = (n0 + n_real - 1) / p.kw - rg0 + 1;
+            // The item's groups, decoded once: thread t writes the entry of group t.  Two tables (item parity):
+            // nobody can still be reading the one written here, because the table of the item before this one
+            // was complete only after every warp had finished the item before that.
             int2* tab = col_tab + (it & 1) * BN;
             {
-                const int ng = j * BN + t;
-                const int c = ng / khw, kr = ng - c * khw, ky = kr / p.kw, kx = kr - ky * p.kw;
-                const int kind = ng < p.d_in ? 1 : ((p.has_bias && ng == p.d_in) ? 2 : 0);   // 0: zero column, 2: all ones
-                tab[t] = make_int2(c * p.H * p.W, ((ky - p.pad) & 0xFF) | (((kx - p.pad) & 0xFF) << 8) | (kind << 16));
+                if (t < n_groups) {
+                    const int rg = rg0 + t, c = rg / p.kh, ky = rg - c * p.kh;
+                    tab[t] = make_int2(c * p.H * p.W, ky - p.pad);
+                }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&tab_full[it & 1]);
                 ok = mbar_wait(&tab_full[it & 1], (it >> 1) & 1, abort_flag, p.status);
                 if (!ok) break;
+            }
+            // 3 x 3 kernels with one pixel of padding (the common case): everything that does not depend on the
+            // stage is worked out here, for the at most two groups a thread owns (86 groups per block of 256
+            // columns, 64 groups per pass): byte offset of the channel, ky - pad, and for each of the three columns
+            // whether it lies in this block and where its 16-byte unit goes in the tile.
+            int f_coff[2] = {0, 0}, f_dy[2] = {0, 0};
+            uint32_t f_soff[2][3];
+            bool f_ok[2][3];
+#pragma unroll
+            for (int gs = 0; gs < 2; ++gs) {
+                const int gi = gq + GQ * gs, rg = rg0 + gi, c = rg / p.kh;
+                f_coff[gs] = c * p.H * p.W * 2; f_dy[gs] = rg - c * p.kh - p.pad;
+#pragma unroll
+                for (int kx = 0; kx < 3; ++kx) {
+                    const int n = rg * 3 + kx - n0;
+                    f_ok[gs][kx] = fast3 && gi < n_groups && (unsigned)n < (unsigned)n_real;
+                    f_soff[gs][kx] = (uint32_t)(n * 128) + (((uint32_t)u ^ (uint32_t)(n & 7)) << 4);
+                }
             }
             for (int e = e0; e < e0 + ne && ok; ++e, ++xe) {
                 const int b = xe & 1;
@@ -269,49 +312,67 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_z, const ctc::Params p) {
                     if (!ok) break;
                     if (t == 0) DPCLIP_TRACE_AT(1, 2 * g);
                     uint8_t* pt = smem + s * STAGE_BYTES + Z_BYTES;
-                    // eight consecutive t = one output row y', eight neighbouring x'
                     const int t0 = kb * BK + 8 * u;
                     const int yb = t0 >> p.wo_shift, xb = t0 & (p.Wo - 1);
-                    if (vec_rows) {
-                        // rows of the map are 16-byte multiples: a unit is the aligned vector at xb, shifted by dx
-                        // elements into its neighbour (zeros at the edge of the map)
-                        const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
-#pragma unroll 4
-                        for (int i = 0; i < 8; ++i) {
-                            const int n = 32 * i + nq;
-                            const int2 col = tab[n];
-                            const int dy = (int)(signed char)(col.y & 0xFF), dx = (int)(signed char)((col.y >> 8) & 0xFF);
-                            const int y = yb + dy;
-                            const bool live = (col.y >> 16) == 1 && (unsigned)y < (unsigned)p.H;
-                            const uint4* rowv = reinterpret_cast<const uint4*>(xs + col.x + y * p.W) + (xb >> 3);
-                            const bool need = live && ((dx < 0 && xb > 0) || (dx > 0 && xb + 8 < p.W));
+                    const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+                    if (fast3) {
+                        const uint8_t* xb_ptr = reinterpret_cast<const uint8_t*>(xs) + (xb >> 3) * 16;
+                        const bool has_prev = xb > 0, has_next = xb + 8 < p.W;
+#pragma unroll
+                        for (int gs = 0; gs < 2; ++gs) {
+                            if (!(f_ok[gs][0] || f_ok[gs][1] || f_ok[gs][2])) continue;
+                            const int y = yb + f_dy[gs];
+                            const bool live = (unsigned)y < (unsigned)p.H;
+                            const uint4* rowv = reinterpret_cast<const uint4*>(xb_ptr + f_coff[gs] + y * p.W * 2);
                             const uint4 cur = live ? rowv[0] : zero;
-                            const uint4 nb = need ? rowv[dx < 0 ? -1 : 1] : zero;
-                            uint4 w = shifted8(cur, nb, dx);
-                            if ((col.y >> 16) == 2) w = make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);   // bf16 1.0
-                            *reinterpret_cast<uint4*>(pt + n * 128 + (((uint32_t)u ^ (uint32_t)(n & 7)) << 4)) = w;
+                            const uint4 prev = (live && has_prev) ? rowv[-1] : zero;
+                            const uint4 next = (live && has_next) ? rowv[1] : zero;
+                            if (f_ok[gs][0])
+                                *reinterpret_cast<uint4*>(pt + f_soff[gs][0]) =
+                                    make_uint4(__funnelshift_r(prev.w, cur.x, 16), __funnelshift_r(cur.x, cur.y, 16),
+                                               __funnelshift_r(cur.y, cur.z, 16), __funnelshift_r(cur.z, cur.w, 16));
+                            if (f_ok[gs][1]) *reinterpret_cast<uint4*>(pt + f_soff[gs][1]) = cur;
+                            if (f_ok[gs][2])
+                                *reinterpret_cast<uint4*>(pt + f_soff[gs][2]) =
+                                    make_uint4(__funnelshift_r(cur.x, cur.y, 16), __funnelshift_r(cur.y, cur.z, 16),
+                                               __funnelshift_r(cur.z, cur.w, 16), __funnelshift_r(cur.w, next.x, 16));
                         }
-                    } else {
-#pragma unroll 2
-                        for (int i = 0; i < 8; ++i) {
-                            const int n = 32 * i + nq;
-                            const int2 col = tab[n];
-                            const int dy = (int)(signed char)(col.y & 0xFF), dx = (int)(signed char)((col.y >> 8) & 0xFF);
-                            const int kind = col.y >> 16;
-                            const int y = yb + dy;
-                            uint4 w = make_uint4(0u, 0u, 0u, 0u);
-                            if (kind == 1 && (unsigned)y < (unsigned)p.H) {
-                                const unsigned short* row = xs + col.x + y * p.W;
+                    } else
+                    for (int gi = gq; gi < n_groups; gi += GQ) {
+                        const int2 grp = tab[gi];
+                        const int y = yb + grp.y;
+                        const bool live = (unsigned)y < (unsigned)p.H;
+                        const unsigned short* row = xs + grp.x + y * p.W;
+                        uint4 cur = zero, prev = zero, next = zero;
+                        if (vec_rows && live) {
+                            const uint4* rowv = reinterpret_cast<const uint4*>(row) + (xb >> 3);
+                            cur = rowv[0];
+                            if (xb > 0) prev = rowv[-1];
+                            if (xb + 8 < p.W) next = rowv[1];
+                        }
+                        int n = (rg0 + gi) * p.kw - n0;                    // N-row of the group's first column
+#pragma unroll 1
+                        for (int kx = 0; kx < p.kw; ++kx, ++n) {
+                            if ((unsigned)n >= (unsigned)n_real) continue;   // column of a neighbouring block
+                            const int dx = kx - p.pad;
+                            uint4 w = zero;
+                            if (vec_rows) {
+                                w = shifted8u(prev, cur, next, dx);
+                            } else if (live) {
                                 const int x0 = xb + dx;
                                 uint32_t v[8];
 #pragma unroll
                                 for (int q = 0; q < 8; ++q) v[q] = (unsigned)(x0 + q) < (unsigned)p.W ? (uint32_t)row[x0 + q] : 0u;
                                 w = make_uint4(v[0] | (v[1] << 16), v[2] | (v[3] << 16), v[4] | (v[5] << 16), v[6] | (v[7] << 16));
-                            } else if (kind == 2) {
-                                w = make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);      // bf16 1.0
                             }
                             *reinterpret_cast<uint4*>(pt + n * 128 + (((uint32_t)u ^ (uint32_t)(n & 7)) << 4)) = w;
                         }
+                    }
+                    // the all-ones bias column and the zero rows up to the next multiple of 32
+                    for (int r = n_real + gq; r < n_rows; r += GQ) {
+                        const bool ones = p.has_bias && n0 + r == p.d_in;
+                        const uint32_t v = ones ? 0x3F803F80u : 0u;            // bf16 1.0 twice
+                        *reinterpret_cast<uint4*>(pt + r * 128 + (((uint32_t)u ^ (uint32_t)(r & 7)) << 4)) = make_uint4(v, v, v, v);
                     }
                     fence_proxy_async_smem();
                     __syncwarp();
