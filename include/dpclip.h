@@ -232,8 +232,8 @@ int dpclip_step(const dpclip_layer* layers /* host */, int L, int B, dpclip_dtyp
  * Square or rectangular kernels, any stride and zero padding; dilation 1.  fp32 layers with dL/dZ as
  * [B][T][d_out] (rows 16-byte multiples) above 2^25 multiply-adds run on the tensor cores (error-
  * compensated tf32, the patch rows gathered by the warps that prepare the operand planes) and need a
- * workspace of dpclip_workspace_bytes(B, T, C*kh*kw, d_out, ...) bytes.  bf16 layers with dL/dZ as
- * [B][T][d_out] also run on the tensor cores when the stride is 1, the output width is 8, 16, 32 or 64, T is a
+ * workspace of dpclip_workspace_bytes(B, T, C*kh*kw, d_out, ...) bytes.  bf16 layers (dL/dZ in either
+ * layout) also run on the tensor cores when the stride is 1, the output width is 8, 16, 32 or 64, T is a
  * multiple of 64, d_out a multiple of 8 and at most 128, a feature map (C*H*W) at most 32 KB and a multiple of
  * 16 bytes, X and Zbar 16-byte aligned, and a workspace is given (its header for the norms; the partial tiles
  * for the clipped sum): the feature map of an example is copied to shared memory once and the patch tiles are

@@ -1187,7 +1187,7 @@ static bool conv_tc_ok(const SimtParams& p, const void* X, const void* Zbar, int
                        dpclip_dtype dtype, const void* workspace, size_t workspace_bytes) {
     { const char* env = getenv("DPCLIP_FORCE_SIMT"); if (env && env[0] == '1') return false; }
     { const char* env = getenv("DPCLIP_NO_CONV_TC"); if (env && env[0] == '1') return false; }
-    if (dtype != DPCLIP_BF16 || z_channel_major || !workspace || workspace_bytes < (size_t)kHeaderBytes) return false;
+    if (dtype != DPCLIP_BF16 || !workspace || workspace_bytes < (size_t)kHeaderBytes) return false;
     if (p.stride != 1 || !(p.Wo == 8 || p.Wo == 16 || p.Wo == 32 || p.Wo == 64) || T % 64 != 0) return false;
     if (p.d_out % 8 != 0 || p.d_out > 128) return false;
     const long x_elems = (long)p.cC * p.cH * p.cW;
@@ -1202,9 +1202,12 @@ static int launch_conv_tc(const SimtParams& sp, const void* X, const void* Zbar,
                           size_t workspace_bytes, cudaStream_t st) {
     namespace c = tc::ctc;
     CUtensorMap mz;
-    if (!make_map_bf16(&mz, Zbar, (long)B * T, sp.d_out, sp.d_out, 64, c::BK)) return DPCLIP_ERR_CUDA;
+    // dL/dZ as [B][T][d_out]: boxes of 64 rows t x 64 columns; as [B][d_out][T]: one box of d_out rows x 64 t
+    if (sp.z_cm ? !make_map_bf16(&mz, Zbar, (long)B * sp.d_out, T, T, c::BK, sp.d_out)
+                : !make_map_bf16(&mz, Zbar, (long)B * T, sp.d_out, sp.d_out, 64, c::BK)) return DPCLIP_ERR_CUDA;
     c::Params p;
     memset(&p, 0, sizeof(p));
+    p.z_cm = sp.z_cm;
     p.X = static_cast<const __nv_bfloat16*>(X);
     p.B = B; p.C = sp.cC; p.H = sp.cH; p.W = sp.cW; p.kh = sp.kh; p.kw = sp.kw; p.pad = sp.pad;
     p.Wo = sp.Wo; p.Ho = T / sp.Wo;

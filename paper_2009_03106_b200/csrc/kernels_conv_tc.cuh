@@ -15,6 +15,7 @@
 //   NORM: item = (example, block of 256 patch columns); the epilogue squares and sums the block -> sq[i] (atomics).
 //   GRAD: item = (slice of examples, block of 256 patch columns); the tile goes to the partial buffer that
 //         reduce_partials_kernel sums (the bias gradient is column d_in of the last block).
+// Zb may be [B][T][d_out] or [B][d_out][T] (then its tiles are K-major too).
 // Restrictions (checked on the host; anything else takes the fp32-ALU kernel): stride 1, output width 8, 16, 32
 // or 64, T a multiple of 64, d_out a multiple of 8 and at most 128, feature map at most 32 KB per example.
 // Every wait is bounded; on a timeout the CTA sets the status word and unwinds.
@@ -41,6 +42,7 @@ struct Params {
     const __nv_bfloat16* X;            // [B][C][H][W]
     int B, C, H, W, kh, kw, pad, Ho, Wo, wo_shift;
     int T, d_in, d_out, has_bias;
+    int z_cm;                          // Zb is [B][d_out][T] (the layout of dL/dZ itself): its tiles are K-major
     int tiles_n;                       // blocks of 256 patch columns (d_in + bias columns in all)
     int n_items;                       // NORM: B * tiles_n; GRAD: slices * tiles_n
     int ex_per_item;                   // GRAD: examples per slice (NORM: 1)
@@ -155,9 +157,16 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_z, const ctc::Params p) {
                         ok = mbar_wait(&empty[s], ((g / STAGES) & 1) ^ 1, abort_flag, p.status);
                         if (!ok) break;
                         uint8_t* zt = smem + s * STAGE_BYTES;
-                        mbar_arrive_expect_tx(&zfull[s], (uint32_t)(z_chunks * BK * 128));
-                        for (int c = 0; c < z_chunks; ++c)
-                            tma_load_2d(zt + c * (BK * 128), &map_z, &zfull[s], c * 64, e * p.T + kb * BK);
+                        if (p.z_cm) {
+                            // [d_out rows][64 t]: one box, 128 bytes per row (rows past d_out keep stale values: they
+                            // only feed accumulator rows nobody reads)
+                            mbar_arrive_expect_tx(&zfull[s], (uint32_t)(p.d_out * 128));
+                            tma_load_2d(zt, &map_z, &zfull[s], kb * BK, e * p.d_out);
+                        } else {
+                            mbar_arrive_expect_tx(&zfull[s], (uint32_t)(z_chunks * BK * 128));
+                            for (int c = 0; c < z_chunks; ++c)
+                                tma_load_2d(zt + c * (BK * 128), &map_z, &zfull[s], c * 64, e * p.T + kb * BK);
+                        }
                     }
                 }
             }
@@ -173,7 +182,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_z, const ctc::Params p) {
                 const int n_cols = min(BN, p.d_in + p.has_bias - j * BN);
                 // N in steps of 32: the epilogue reads the accumulator 32 columns at a time, and patch rows past the
                 // last real column are zero
-                const uint32_t idesc = make_idesc_bf16(128, (n_cols + 31) & ~31, 1, 0);
+                const uint32_t idesc = make_idesc_bf16(128, (n_cols + 31) & ~31, p.z_cm ? 0 : 1, 0);
                 const int buf = it & 1;
                 ok = mbar_wait(&acc_empty[buf], ((it >> 1) & 1) ^ 1, abort_flag, p.status);
                 if (!ok) break;
@@ -191,7 +200,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_z, const ctc::Params p) {
                         // Zb: MN-major, 64-column chunks BK * 128 bytes apart (stride 0 when only one holds data:
                         // the M rows 64..127 then re-read it and are never used); 16 rows = 2048 bytes.
                         // patches: K-major, 8-row groups 1024 bytes apart; 16 contraction elements = 32 bytes.
-                        const uint64_t dz = make_smem_desc_sw128(zb + k16 * 2048, z_chunks > 1 ? BK * 128 : 0, 1024);
+                        const uint64_t dz = p.z_cm ? make_smem_desc_sw128(zb + k16 * 32, 16, 1024)      // K-major rows of 64 t
+                                                   : make_smem_desc_sw128(zb + k16 * 2048, z_chunks > 1 ? BK * 128 : 0, 1024);
                         const uint64_t dp = make_smem_desc_sw128(pb + k16 * 32, 16, 1024);
                         mma_bf16_ss(tmem_base + buf * BN, dz, dp, idesc, (kk == 0 && k16 == 0) ? 0u : 1u);
                     }
@@ -403,7 +413,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_z, const ctc::Params p) {
                     if (!ok) break;
                     if (f != 1.0f) {
                         uint4* zt = reinterpret_cast<uint4*>(smem + s * STAGE_BYTES);
-                        const int units = z_chunks * BK * 8;           // 16-byte units of the chunks that hold data
+                        const int units = p.z_cm ? p.d_out * 8 : z_chunks * BK * 8;   // 16-byte units that hold data
                         for (int i = t; i < units; i += 32 * SCALE_WARPS) {
                             uint4 v = zt[i];
                             __nv_bfloat162* z2 = reinterpret_cast<__nv_bfloat162*>(&v);
