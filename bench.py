@@ -485,6 +485,11 @@ def bench_conv_implicit(torch, dp, name, B, C, H, W, k, pad, d_out, dtype, steps
             roof = dict(bound="tensor", achieved=ach, peak=peak_tf, unit="TFLOP/s", frac=ach / peak_tf)
         roof.update(traffic=None, peak_source=peaks["source"])
         out[kind] = dict(ms=ms, patch_matrix_path_ms=ms_ref, roofline=roof)
+    # dL/dZ as back-propagation produces it, [B][c_out][T] (the patch-matrix path would first have to transpose it)
+    dZcm = dZ.transpose(1, 2).contiguous()
+    out["norm_channel_major_ms"] = float(np.median(time_steps(
+        torch, lambda: dp.dpclip_conv_sqnorms(dX, dZcm, k, k, 1, pad, True, sq, z_channel_major=True, workspace=ws),
+        steps, 3, flush)))
     return out
 
 
