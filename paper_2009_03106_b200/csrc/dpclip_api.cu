@@ -14,6 +14,7 @@
 #include "kernels_narrow.cuh"
 #include "kernels_narrow_tc.cuh"
 #include "kernels_conv_tc.cuh"
+#include "kernels_narrow_pack.cuh"
 #include "kernels_elementwise.cuh"
 
 #include <stdlib.h>
@@ -140,6 +141,46 @@ int launch_narrow_tc(const NarrowParams& p, int grid, int n_items, int* status, 
     return launch_status();
 }
 
+// Narrow layers with d_out <= 32 on the tensor cores, four row groups per instruction (either dtype): the same
+// conditions as narrow_tc_ok, on 16-byte multiples of the element size
+inline bool narrow_pack_ok(const NarrowParams& p, dpclip_dtype dtype, const int* status) {
+    const char* env = getenv("DPCLIP_NO_NARROW_TC");
+    if (env && env[0] == '1') return false;
+    { const char* e2 = getenv("DPCLIP_NO_NARROW_PACK"); if (e2 && e2[0] == '1') return false; }
+    if (status == nullptr || p.d_out > 32 || p.d_in + p.has_bias > 32) return false;
+    if (dtype == DPCLIP_BF16) {
+        // bf16 has few instructions to save (one per 16 rows), and four partial tiles per CTA cost the reduce more
+        // than the packing gains: measured 15.7 / 21.5 us against 14.9 / 18.1 us for the unpacked kernel on the
+        // first convolution of the CNN.  Kept selectable for measurements.
+        const char* e3 = getenv("DPCLIP_NARROW_PACK_BF16");
+        if (!(e3 && e3[0] == '1')) return false;
+    }
+    if (!aligned_to(p.A, 16) || !aligned_to(p.Z, 16)) return false;
+    const long es = elt_size(dtype);
+    return ((long)p.T * p.d_in * es) % 16 == 0 && ((long)p.T * p.d_out * es) % 16 == 0;
+}
+
+template <typename T, bool GRAD>
+int launch_narrow_pack_inst(const tc::npk::Params& q, int grid, cudaStream_t st) {
+    using Cfg = tc::npk::Cfg<T>;
+    if (cudaFuncSetAttribute(tc::narrow_pack_kernel<T, GRAD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             Cfg::SMEM_BYTES) != cudaSuccess) return DPCLIP_ERR_CUDA;
+    tc::narrow_pack_kernel<T, GRAD><<<grid, tc::npk::THREADS, Cfg::SMEM_BYTES, st>>>(q);
+    return launch_status();
+}
+
+template <bool GRAD>
+int launch_narrow_pack(const NarrowParams& p, int grid, int n_items, dpclip_dtype dtype, int* status, cudaStream_t st) {
+    tc::npk::Params q;
+    memset(&q, 0, sizeof(q));
+    q.A = p.A; q.Z = p.Z; q.T = p.T; q.d_in = p.d_in; q.d_out = p.d_out; q.has_bias = p.has_bias;
+    q.n_items = n_items; q.rows_total = p.rows_total; q.rows_per_cta = p.rows_per_cta;
+    q.clip = p.clip; q.sq = p.sq; q.part = p.part; q.status = status;
+    if (!GRAD && cudaMemsetAsync(p.sq, 0, sizeof(float) * (size_t)n_items, st) != cudaSuccess) return DPCLIP_ERR_CUDA;
+    return dtype == DPCLIP_F32 ? launch_narrow_pack_inst<float, GRAD>(q, grid, st)
+                               : launch_narrow_pack_inst<__nv_bfloat16, GRAD>(q, grid, st);
+}
+
 template <bool GRAD>
 int launch_narrow(const NarrowParams& p, int grid, int d_out, dpclip_dtype dtype, cudaStream_t st) {
     if (narrow_ring_ok(p, dtype, GRAD)) {
@@ -161,6 +202,8 @@ int launch_simt_norms(const void* A, long lda, const void* Z, long ldz, int B, i
         memset(&q, 0, sizeof(q));
         q.A = A; q.lda = lda; q.Z = Z; q.ldz = ldz; q.T = T; q.d_in = d_in; q.d_out = d_out;
         q.has_bias = has_bias ? 1 : 0; q.sq = sq;
+        if (narrow_pack_ok(q, dtype, status))
+            return launch_narrow_pack<false>(q, B < kNumSMs ? B : kNumSMs, B, dtype, status, st);
         if (narrow_tc_ok(q, dtype, status))
             return launch_narrow_tc<false>(q, B < kNumSMs ? B : kNumSMs, B, status, st);
         return launch_narrow<false>(q, B, d_out, dtype, st);
@@ -194,7 +237,8 @@ int launch_simt_grad(const void* A, long lda, const void* Z, long ldz, int B, in
         q.has_bias = gb ? 1 : 0; q.clip = clip; q.gW = gW; q.ldg = ldg; q.gb = gb;
         q.rows_total = (long)B * T;
         int* status = (workspace && workspace_bytes >= (size_t)kHeaderBytes) ? static_cast<int*>(workspace) : nullptr;
-        const bool on_tc = narrow_tc_ok(q, dtype, status);
+        const bool on_pack = narrow_pack_ok(q, dtype, status);
+        const bool on_tc = on_pack || narrow_tc_ok(q, dtype, status);
         // one wave: a CTA of the register-staged kernel holds a whole SM; the cp.async form runs two per SM
         int grid = (!on_tc && narrow_ring_ok(q, dtype, true)) ? 2 * kNumSMs : kNumSMs;
         const long min_rows = NARROW_WARPS * 32;                   // at least one chunk per warp
@@ -204,15 +248,18 @@ int launch_simt_grad(const void* A, long lda, const void* Z, long ldz, int B, in
         q.rows_per_cta = ((q.rows_total + grid - 1) / grid + 31) / 32 * 32;
         grid = (int)((q.rows_total + q.rows_per_cta - 1) / q.rows_per_cta);
         const int maxm = d_out <= 32 ? 32 : 64;
-        const size_t part_bytes = (size_t)grid * maxm * 32 * 4;
+        const int parts_per_cta = on_pack ? 4 : 1;                 // the packed kernel leaves its four diagonal blocks
+        const size_t part_bytes = (size_t)grid * parts_per_cta * maxm * 32 * 4;
         if (workspace && workspace_bytes >= (size_t)kHeaderBytes + part_bytes && grid > 1) {
             // partial tile per CTA, then a fixed-order reduce that also adds the noise
             q.part = reinterpret_cast<float*>(static_cast<char*>(workspace) + kHeaderBytes);
-            int rc = on_tc ? launch_narrow_tc<true>(q, grid, 1, status, st) : launch_narrow<true>(q, grid, d_out, dtype, st);
+            int rc = on_pack ? launch_narrow_pack<true>(q, grid, 1, dtype, status, st)
+                   : on_tc   ? launch_narrow_tc<true>(q, grid, 1, status, st)
+                             : launch_narrow<true>(q, grid, d_out, dtype, st);
             if (rc) return rc;
             NarrowReduceParams r;
             memset(&r, 0, sizeof(r));
-            r.part = q.part; r.n_parts = grid; r.maxm = maxm; r.d_out = d_out; r.d_in = d_in; r.has_bias = gb ? 1 : 0;
+            r.part = q.part; r.n_parts = grid * parts_per_cta; r.maxm = maxm; r.d_out = d_out; r.d_in = d_in; r.has_bias = gb ? 1 : 0;
             r.gW = gW; r.ldg = ldg; r.gb = gb;
             if (noise && noise->scale > 0.f && ldg == d_in) {
                 r.noise_scale = noise->scale;

@@ -633,16 +633,18 @@ NARROW_TC_SHAPES = [(128, 1024, 27, 32),      # the first convolution of the CNN
                     (4, 40, 31, 40), (2, 33, 5, 3), (7, 2, 1, 1)]
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
 @pytest.mark.parametrize("B,T,d_in,d_out", NARROW_TC_SHAPES)
 @pytest.mark.parametrize("has_bias", [True, False])
-def test_narrow_layers_tensor_core(dp, B, T, d_in, d_out, has_bias):
-    """bf16 narrow layers: blocks of rows scattered into the operand layout by the fill warps, contraction on
-    the tensor cores.  Norms see exact products; the clipped sum rounds c * zb once to bf16."""
-    A, Z = workloads.random_layer(60, B, T, d_in, d_out, "bf16", scale_z=0.05)
+def test_narrow_layers_tensor_core(dp, B, T, d_in, d_out, has_bias, dtype):
+    """Narrow layers on the tensor cores: raw chunks re-arranged into operand tiles in shared memory, four 16-row
+    groups per instruction for d_out <= 32 (bf16 and fp32 as error-compensated tf32), one group for bf16 up to 64
+    outputs.  Norms see exact products; the bf16 clipped sum rounds c * zb once to bf16."""
+    A, Z = workloads.random_layer(60, B, T, d_in, d_out, dtype, scale_z=0.05)
     n = min(B, 12)                                            # the oracle materialises every example: sample
     idx = np.unique(np.concatenate([np.arange(min(n, B)), np.arange(max(0, B - 3), B), [B // 2]]))
     ref = oracle.layer_sqnorms(A[idx], Z[idx], has_bias)
-    got = _sqnorms(dp, A, Z, "bf16", has_bias)
+    got = _sqnorms(dp, A, Z, dtype, has_bias)
     assert max_rel(np.sqrt(got[idx]), np.sqrt(ref)) <= TOL["f32"]["norm"]
     clip = np.random.default_rng(B).uniform(0.05, 1.0, B).astype(np.float32)
     clip[::3] = 1.0
@@ -650,16 +652,32 @@ def test_narrow_layers_tensor_core(dp, B, T, d_in, d_out, has_bias):
     gW = torch.full((d_out, d_in), 9.0, device="cuda")
     gb = torch.full((d_out,), 9.0, device="cuda") if has_bias else None
     ws = _ws(dp)
-    dp.dpclip_clipped_grad(to_device(A, "bf16"), to_device(Z, "bf16"), torch.from_numpy(clip).cuda(), gW, gb, ws)
+    dp.dpclip_clipped_grad(to_device(A, dtype), to_device(Z, dtype), torch.from_numpy(clip).cuda(), gW, gb, ws)
     torch.cuda.synchronize()
     assert dp.dpclip_read_status(ws) == 0
-    assert rel_fro(gW.cpu().numpy(), refW) <= TOL["bf16"]["grad"]
+    assert rel_fro(gW.cpu().numpy(), refW) <= TOL[dtype]["grad"]
     if has_bias:
-        assert rel_fro(gb.cpu().numpy(), refb) <= TOL["bf16"]["grad"]
+        assert rel_fro(gb.cpu().numpy(), refb) <= TOL[dtype]["grad"]
     # no factors: exact products, fp32 accumulation
     refW1, _ = oracle.clipped_grad(A, Z, None)
-    dp.dpclip_clipped_grad(to_device(A, "bf16"), to_device(Z, "bf16"), None, gW, gb, ws)
+    dp.dpclip_clipped_grad(to_device(A, dtype), to_device(Z, dtype), None, gW, gb, ws)
     assert rel_fro(gW.cpu().numpy(), refW1) <= 2e-5
+
+
+def test_narrow_packed_kernel_bf16(dp, monkeypatch):
+    """The four-groups-per-instruction kernel with bf16 operands (fp32 layers take it by default, bf16 layers
+    only on request)."""
+    monkeypatch.setenv("DPCLIP_NARROW_PACK_BF16", "1")
+    B, T, d_in, d_out = 150, 136, 27, 32
+    A, Z = workloads.random_layer(61, B, T, d_in, d_out, "bf16", scale_z=0.05)
+    idx = np.array([0, 1, 74, 149])
+    got = _sqnorms(dp, A, Z, "bf16", True)
+    assert max_rel(np.sqrt(got[idx]), np.sqrt(oracle.layer_sqnorms(A[idx], Z[idx], True))) <= TOL["f32"]["norm"]
+    clip = np.random.default_rng(3).uniform(0.05, 1.0, B).astype(np.float32)
+    refW, refb = oracle.clipped_grad(A, Z, clip)
+    gW = torch.empty(d_out, d_in, device="cuda"); gb = torch.empty(d_out, device="cuda")
+    dp.dpclip_clipped_grad(to_device(A, "bf16"), to_device(Z, "bf16"), torch.from_numpy(clip).cuda(), gW, gb, _ws(dp))
+    assert rel_fro(gW.cpu().numpy(), refW) <= TOL["bf16"]["grad"] and rel_fro(gb.cpu().numpy(), refb) <= TOL["bf16"]["grad"]
 
 
 def test_narrow_layer_register_staged_form(dp, monkeypatch):
