@@ -97,6 +97,7 @@ narrow_pack_kernel(const npk::Params p) {
     const int n_raw = min(MAX_RAW, RAW_BYTES / chunk_bytes) / STAGES * STAGES;      // a multiple of the teams: see below
 
     if (threadIdx.x == 0) {
+        DPCLIP_TRACE_AT(0, 254);
         for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], TEAM); mbar_init(&empty[s], 1); }
         for (int s = 0; s < MAX_RAW; ++s) { mbar_init(&raw_full[s], 1); mbar_init(&raw_empty[s], TEAM); }
         for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], EPI_WARPS); }
@@ -164,6 +165,8 @@ narrow_pack_kernel(const npk::Params p) {
             constexpr uint32_t idesc = F32 ? make_idesc_tf32(128, 128, 1, 1) : make_idesc_bf16(128, 128, 1, 1);
             int stage = 0; uint32_t phase = 0; int it = 0;
             bool ok = true;
+            [[maybe_unused]] int tr = 0;
+            DPCLIP_TRACE_AT(0, 255);
             for (int item = item0; item < n_items && ok; item += item_step, ++it) {
                 long r0, r1; item_rows(item, r0, r1);
                 const int nkb = (int)((r1 - r0 + BK - 1) / BK);
@@ -175,6 +178,7 @@ narrow_pack_kernel(const npk::Params p) {
                 for (int kb = 0; kb < nkb; ++kb) {
                     ok = mbar_wait(&full[stage], phase, abort_flag, p.status);
                     if (!ok) break;
+                    DPCLIP_TRACE_AT(2, tr); ++tr;
                     tc_fence_after_sync();
                     const uint32_t base = smem_u32(smem + stage * STAGE_BYTES);
                     if (F32) {
@@ -211,6 +215,7 @@ narrow_pack_kernel(const npk::Params p) {
         for (int item = item0; item < n_items; item += item_step, ++it) {
             const int buf = it & 1;
             if (!mbar_wait(&acc_full[buf], (it >> 1) & 1, abort_flag, p.status)) break;
+            if (threadIdx.x == 64) DPCLIP_TRACE_AT(3, it);
             tc_fence_after_sync();
             uint32_t v[32];
             tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + buf * 128 + q * 32, v);
@@ -280,6 +285,7 @@ narrow_pack_kernel(const npk::Params p) {
                 if (ok) ok = mbar_wait(&empty[f], my_phase ^ 1, abort_flag, p.status);
                 if (!ok) break;
                 my_phase ^= 1;
+                if (cw == 0 && lane == 0) DPCLIP_TRACE_AT(1, 2 * (gs / STAGES));
                 const uint8_t* ra = raw + rslot * chunk_bytes;
                 const uint8_t* rz = ra + a_chunk;
                 // ---- [A|1]: lane = column c; the 16 rows of group grp go to tile column 32 grp + c, K-rows 0 .. 15.
@@ -375,6 +381,7 @@ narrow_pack_kernel(const npk::Params p) {
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) { mbar_arrive(&full[f]); mbar_arrive(&raw_empty[rslot]); }
+                if (cw == 0 && lane == 0) DPCLIP_TRACE_AT(1, 2 * (gs / STAGES) + 1);
             }
             seq += nkb;
         }
