@@ -149,9 +149,9 @@ inline bool narrow_pack_ok(const NarrowParams& p, dpclip_dtype dtype, const int*
     { const char* e2 = getenv("DPCLIP_NO_NARROW_PACK"); if (e2 && e2[0] == '1') return false; }
     if (status == nullptr || p.d_out > 32 || p.d_in + p.has_bias > 32) return false;
     if (dtype == DPCLIP_BF16) {
-        // bf16 has few instructions to save (one per 16 rows), and four partial tiles per CTA cost the reduce more
-        // than the packing gains: measured 15.7 / 21.5 us against 14.9 / 18.1 us for the unpacked kernel on the
-        // first convolution of the CNN.  Kept selectable for measurements.
+        // bf16 has few instructions to save (one per 16 rows) and pays for the extra pass through shared memory in
+        // the epilogue: measured 16.4 / 18.0 us against 15.2 / 17.9 us for the unpacked kernel on the first
+        // convolution of the CNN.  Kept selectable for measurements.
         const char* e3 = getenv("DPCLIP_NARROW_PACK_BF16");
         if (!(e3 && e3[0] == '1')) return false;
     }
@@ -248,7 +248,7 @@ int launch_simt_grad(const void* A, long lda, const void* Z, long ldz, int B, in
         q.rows_per_cta = ((q.rows_total + grid - 1) / grid + 31) / 32 * 32;
         grid = (int)((q.rows_total + q.rows_per_cta - 1) / q.rows_per_cta);
         const int maxm = d_out <= 32 ? 32 : 64;
-        const int parts_per_cta = on_pack ? 4 : 1;                 // the packed kernel leaves its four diagonal blocks
+        const int parts_per_cta = 1;
         const size_t part_bytes = (size_t)grid * parts_per_cta * maxm * 32 * 4;
         if (workspace && workspace_bytes >= (size_t)kHeaderBytes + part_bytes && grid > 1) {
             // partial tile per CTA, then a fixed-order reduce that also adds the noise

@@ -17,9 +17,9 @@
 // chunks, teams of converter warps re-arrange them into the operand tiles of their own stage slot (fp32: raw
 // value = high part, since the tensor core ignores the low 13 mantissa bits; low part into its own plane),
 // one thread issues the MMAs, four epilogue warps.
-//   NORM: item = example; the four blocks are added through shared memory, squared, summed -> sq[i] (atomics).
-//   GRAD: one row slice per CTA, zb scaled by the clip factor during the conversion (bf16: one rounding; fp32:
-//         exact to fp32); each diagonal block is written as a partial tile of its own for narrow_reduce_kernel.
+//   The four blocks are added through shared memory.  NORM: item = example; the sum is squared and summed -> sq[i]
+//   (atomics).  GRAD: one row slice per CTA, zb scaled by the clip factor during the conversion (bf16: one rounding;
+//   fp32: exact to fp32); the sum is the CTA's partial tile for narrow_reduce_kernel.
 // Needs 16-byte aligned inputs and T * d_in, T * d_out multiples of 16 bytes' worth of elements.  Every wait is
 // bounded; on a timeout the CTA sets the status word and unwinds.
 #pragma once
@@ -52,7 +52,7 @@ struct Params {
     long rows_total, rows_per_cta;     // GRAD: one slice per CTA (rows_per_cta a multiple of 32)
     const float* clip;                 // GRAD: [B] or NULL
     float* sq;                         // NORM: [B], pre-zeroed
-    float* part;                       // GRAD: [4 * grid][32][32] partial tiles (one per CTA and diagonal block)
+    float* part;                       // GRAD: [grid][32][32] partial tiles
     int* status;
 };
 
@@ -223,30 +223,25 @@ narrow_pack_kernel(const npk::Params p) {
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[buf]);
-            if (GRAD) {
-                float4* dst = reinterpret_cast<float4*>(p.part + (((size_t)blockIdx.x * 4 + q) * 32 + lane) * 32);
+            // the four blocks meet in shared memory; warp q then takes rows 8 q .. 8 q + 7 of their sum
+            if (!mbar_wait(red_empty, (it & 1) ^ 1, abort_flag, p.status)) break;
+            float* mine = red + (q * 32 + lane) * 33;
 #pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    dst[j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
-                                         __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
-            } else {
-                // the four blocks meet in shared memory; warp q then squares and sums rows 8 q .. 8 q + 7 of their sum
-                if (!mbar_wait(red_empty, (it & 1) ^ 1, abort_flag, p.status)) break;
-                float* mine = red + (q * 32 + lane) * 33;
+            for (int j = 0; j < 32; ++j) mine[j] = __uint_as_float(v[j]);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(red_full);
+            if (!mbar_wait(red_full, it & 1, abort_flag, p.status)) break;
+            float s = 0.f;
 #pragma unroll
-                for (int j = 0; j < 32; ++j) mine[j] = __uint_as_float(v[j]);
-                __syncwarp();
-                if (lane == 0) mbar_arrive(red_full);
-                if (!mbar_wait(red_full, it & 1, abort_flag, p.status)) break;
-                float s = 0.f;
-#pragma unroll
-                for (int m = 8 * q; m < 8 * q + 8; ++m) {
-                    const float x = (red[(0 * 32 + m) * 33 + lane] + red[(1 * 32 + m) * 33 + lane]) +
-                                    (red[(2 * 32 + m) * 33 + lane] + red[(3 * 32 + m) * 33 + lane]);
-                    s = fmaf(x, x, s);
-                }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(red_empty);
+            for (int m = 8 * q; m < 8 * q + 8; ++m) {
+                const float x = (red[(0 * 32 + m) * 33 + lane] + red[(1 * 32 + m) * 33 + lane]) +
+                                (red[(2 * 32 + m) * 33 + lane] + red[(3 * 32 + m) * 33 + lane]);
+                if (GRAD) p.part[((size_t)blockIdx.x * 32 + m) * 32 + lane] = x;      // the CTA's partial tile
+                else s = fmaf(x, x, s);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(red_empty);
+            if (!GRAD) {
                 s = warp_sum(s);
                 if (lane == 0) atomicAdd(p.sq + item, s);
             }
