@@ -517,7 +517,7 @@ int launch_zta_tc_mt(const tc::zta::Maps& maps, tc::zta::Params p, int B, bool n
         p.n_items = B * tiles;
         if (cudaMemsetAsync(sq, 0, sizeof(float) * (size_t)B, st) != cudaSuccess) return DPCLIP_ERR_CUDA;
     } else {
-        const int nkb = ceil_div(R, z::BK);
+        const int nkb = ceil_div(R, z::Cfg<MT>::BK);
         // One wave of equally long items: the kernel is bound by L2->SM traffic, so what matters is that
         // every SM streams the same number of row blocks.  (MT = 1 has two accumulator buffers and can
         // overlap the epilogue of one item with the next, so it takes two items per SM when they stay long.)
@@ -560,8 +560,13 @@ int launch_zta_tc(const void* A, long lda, const void* Z, long ldz, int B, int T
                   cudaStream_t st, bool fit_to_workspace = false) {
     namespace z = tc::zta;
     const long R = (long)B * T;
+    int mt = d_out > 128 ? 2 : 1;
+    const char* env = getenv("DPCLIP_TILE_M");
+    if (env && env[0] == '1') mt = 1;
+    if (env && env[0] == '2') mt = 2;
+    const int bk = mt == 2 ? z::Cfg<2>::BK : z::Cfg<1>::BK;           // rows of a TMA box = rows of a stage
     z::Maps maps;
-    if (!make_map_bf16(&maps.a[0], A, R, d_in, lda, 64, z::BK) || !make_map_bf16(&maps.z[0], Z, R, d_out, ldz, 64, z::BK))
+    if (!make_map_bf16(&maps.a[0], A, R, d_in, lda, 64, bk) || !make_map_bf16(&maps.z[0], Z, R, d_out, ldz, 64, bk))
         return DPCLIP_ERR_CUDA;
     z::Params p;
     memset(&p, 0, sizeof(p));
@@ -576,10 +581,6 @@ int launch_zta_tc(const void* A, long lda, const void* Z, long ldz, int B, int T
         p.do_bias = gb ? 1 : 0;
         p.vec_ok = aligned_to(gW, 16) && ldg % 4 == 0;
     }
-    int mt = d_out > 128 ? 2 : 1;
-    const char* env = getenv("DPCLIP_TILE_M");
-    if (env && env[0] == '1') mt = 1;
-    if (env && env[0] == '2') mt = 2;
     if (mt == 2)
         return launch_zta_tc_mt<2>(maps, p, B, norm_mode, gW, ldg, gb, sq, d_in, d_out, workspace, workspace_bytes,
                                    noise, noise_done, st, fit_to_workspace);
@@ -596,6 +597,7 @@ int launch_zta_tc_group(const dpclip_layer* const* ls, const int* index, int n, 
     if (n < 2 || n > z::MAX_LAYERS) return 1;
     const dpclip_layer& y0 = *ls[0];
     const long R = (long)B * y0.T;
+    const int bk = y0.d_out > 128 ? z::Cfg<2>::BK : z::Cfg<1>::BK;
     z::Maps maps;
     GradGroup grp;
     memset(&grp, 0, sizeof(grp));
@@ -604,8 +606,8 @@ int launch_zta_tc_group(const dpclip_layer* const* ls, const int* index, int n, 
     bool vec_ok = true;
     for (int l = 0; l < n; ++l) {
         const dpclip_layer& y = *ls[l];
-        if (!make_map_bf16(&maps.a[l], y.A, R, y.d_in, y.lda, 64, z::BK) ||
-            !make_map_bf16(&maps.z[l], y.Zbar, R, y.d_out, y.ldz, 64, z::BK))
+        if (!make_map_bf16(&maps.a[l], y.A, R, y.d_in, y.lda, 64, bk) ||
+            !make_map_bf16(&maps.z[l], y.Zbar, R, y.d_out, y.ldz, 64, bk))
             return DPCLIP_ERR_CUDA;
         grp.gW[l] = y.gW; grp.gb[l] = y.has_bias ? y.gb : nullptr;
         grp.sid_w[l] = stream_id0 + 2ull * index[l]; grp.sid_b[l] = grp.sid_w[l] + 1;
@@ -1099,7 +1101,7 @@ int dpclip_same_shape_layers_clipped_grad_noise(const dpclip_layer* layers, int 
             const dpclip_layer& y = layers[l0];
             const int bm = y.d_out > 128 ? 256 : 128;
             const int tiles = ceil_div(y.d_out, bm) * ceil_div(y.d_in, z::BN);
-            const long nkb = ceil_div((long)B * y.T, (long)z::BK);
+            const long nkb = ceil_div((long)B * y.T, 64L);          // 64-row blocks
             const int ksplit = tiles < kNumSMs ? kNumSMs / tiles : 1;
             if (nkb / ksplit >= 32) continue;
         }

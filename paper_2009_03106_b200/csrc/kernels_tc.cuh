@@ -563,9 +563,6 @@ gram_norm_q2_kernel(const __grid_constant__ gram::Launch q) {
 // ===========================================================================
 namespace zta {
 constexpr int BN = 256;                        // d_in tile  (UMMA N)
-constexpr int BK = 64;                         // rows per stage
-constexpr int CHUNK_BYTES = BK * 128;          // one TMA box: 64 rows x 64 bf16 columns
-constexpr int B_BYTES = (BN / 64) * CHUNK_BYTES;   // A tile, 32 KB
 constexpr int N_TRANSFORM_WARPS = 8, N_EPILOGUE_WARPS = 8;
 constexpr int THREADS = 64 + 32 * (N_TRANSFORM_WARPS + N_EPILOGUE_WARPS);   // warp 0 TMA, warp 1 MMA
 constexpr int OUT_STAGE_BYTES = N_EPILOGUE_WARPS * 4096;          // 32 rows x 32 fp32 per epilogue warp
@@ -576,11 +573,16 @@ constexpr int SMEM_BYTES = 192 * 1024 + 256 + OUT_STAGE_BYTES + 1024;
 //           overlaps the main loop of the next), 4 stages of 48 KB.
 //   MT = 2: 256 x 256 tile, one accumulator buffer (all 512 columns), 3 stages of 64 KB; a third
 //           less L2->SM traffic per flop, for layers where that traffic is the limit.
+// Stages are 64 rows: with 32-row stages (twice as many slots) the large tile ran 10-15 % slower, the
+// per-stage cost of the transform warps (barrier round trips, proxy fence) weighing twice.
 template <int MT> struct Cfg {
     static constexpr int BM = 128 * MT;
-    static constexpr int A_BYTES = (BM / 64) * CHUNK_BYTES;
+    static constexpr int BK = 64;                                 // rows per stage
+    static constexpr int CHUNK_BYTES = BK * 128;                  // one TMA box: BK rows x 64 bf16 columns
+    static constexpr int A_BYTES = (BM / 64) * CHUNK_BYTES;       // Zb tile
+    static constexpr int B_BYTES = (BN / 64) * CHUNK_BYTES;       // A tile
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int STAGES = MT == 1 ? 4 : 3;
+    static constexpr int STAGES = (192 * 1024) / STAGE_BYTES;
     static constexpr int NBUF = MT == 1 ? 2 : 1;
 };
 
@@ -590,7 +592,7 @@ struct Params {
     int tiles_m, tiles_n;          // tiles_m counts the d_out tiles of ALL layers of the launch (layer-major)
     int tiles_m_layer;             // d_out tiles of one layer (= tiles_m for a single layer)
     int n_items;
-    int kb_per_split;              // GRAD: 64-row blocks per item
+    int kb_per_split;              // GRAD: stages (blocks of Cfg::BK rows) per item
     int do_bias;                   // GRAD: gb != NULL; NORM: has_bias
     const float* clip;             // GRAD: [B] or NULL
     float* gW; long ldg; float* gb; int vec_ok;
@@ -625,10 +627,10 @@ __device__ __forceinline__ Item decode(const Params& p, int item) {
         w.row_end = w.row_begin + p.T;
     } else {
         w.example = -1;
-        w.row_begin = outer * p.kb_per_split * BK;
-        w.row_end = min(w.row_begin + p.kb_per_split * BK, p.R);
+        w.row_begin = outer * p.kb_per_split * Cfg<MT>::BK;
+        w.row_end = min(w.row_begin + p.kb_per_split * Cfg<MT>::BK, p.R);
     }
-    w.nkb = (w.row_end - w.row_begin + BK - 1) / BK;
+    w.nkb = (w.row_end - w.row_begin + Cfg<MT>::BK - 1) / Cfg<MT>::BK;
     return w;
 }
 }  // namespace zta
@@ -639,6 +641,7 @@ zta_tc_kernel(const __grid_constant__ zta::Maps maps, const zta::Params p) {
     using namespace zta;
     using C = Cfg<MT>;
     constexpr int STAGES = C::STAGES, STAGE_BYTES = C::STAGE_BYTES, A_BYTES = C::A_BYTES, NBUF = C::NBUF;
+    constexpr int BK = C::BK, CHUNK_BYTES = C::CHUNK_BYTES;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);   // 1024-byte aligned; an offset from the array keeps the accesses in the shared state space
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);   // TMA landed
@@ -760,7 +763,7 @@ zta_tc_kernel(const __grid_constant__ zta::Maps maps, const zta::Params p) {
             for (int kb = 0; kb < w.nkb; ++kb) {
                 // the factors of this stage's rows are fetched BEFORE waiting for the tile, so the
                 // global-load latency overlaps the wait instead of sitting between TMA and MMA
-                const int blk0 = w.row_begin + kb * BK;              // rows [blk0, blk0 + 64)
+                const int blk0 = w.row_begin + kb * BK;              // rows [blk0, blk0 + BK)
                 const int e_first = blk0 / p.T;
                 const int rem0 = blk0 - e_first * p.T;
                 // fast path: the whole stage lies inside one example and inside the row range
@@ -769,9 +772,10 @@ zta_tc_kernel(const __grid_constant__ zta::Maps maps, const zta::Params p) {
                 // taken by the n-tile with kb % tiles_n == tn (equal shares).  NORM: the sums must be
                 // complete before they are squared, so n-tile 0 takes them all.
                 const bool bias_here = p.do_bias && (p.norm_mode ? w.tn == 0 : (kb % p.tiles_n) == w.tn);
-                float fr[4];
+                constexpr int NR = BK / 16;                          // rows per thread and sub-tile
+                float fr[NR];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
+                for (int i = 0; i < NR; ++i) {
                     const int rl = uniform ? 0 : rs + 16 * i;
                     float f = 1.f;
                     if (blk0 + rl >= w.row_end) f = 0.f;             // rows of another example / past the end
@@ -782,34 +786,62 @@ zta_tc_kernel(const __grid_constant__ zta::Maps maps, const zta::Params p) {
                 if (!ok) break;
                 if (t == 0) { DPCLIP_TRACE_AT(1, tr); ++tr; }
                 uint8_t* zt = smem + stage * STAGE_BYTES;
-                if (bias_here || !(uniform && fr[0] == 1.f)) {
+                // packed bf16 scaling: f = f_hi + f_lo (two bf16); z*f_lo is tiny, so the fused
+                // multiply-add z*f_hi + (z*f_lo) rounds the product once
+                auto scale8 = [](uint4& v, float f) {
+                    const __nv_bfloat16 fh = __float2bfloat16_rn(f);
+                    const __nv_bfloat16 fl = __float2bfloat16_rn(f - __bfloat162float(fh));
+                    const __nv_bfloat162 fh2 = __halves2bfloat162(fh, fh), fl2 = __halves2bfloat162(fl, fl);
+                    __nv_bfloat162* z2 = reinterpret_cast<__nv_bfloat162*>(&v);
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
+                    for (int u = 0; u < 4; ++u) z2[u] = __hfma2(z2[u], fh2, __hmul2(z2[u], fl2));
+                };
+                auto add8 = [](float* c, const uint4& v) {
+                    const uint32_t wds[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        c[2 * u] += __uint_as_float(wds[u] << 16);
+                        c[2 * u + 1] += __uint_as_float(wds[u] & 0xFFFF0000u);
+                    }
+                };
+                if (uniform) {
+                    // one factor for the whole stage: all loads are issued before the first store, so the
+                    // stage costs one shared-memory round trip instead of one per row
+                    const float f = fr[0];
+                    if (f != 1.f || bias_here) {
+                        uint4 v[MT][NR];
+#pragma unroll
+                        for (int h = 0; h < MT; ++h)
+#pragma unroll
+                            for (int i = 0; i < NR; ++i)
+                                v[h][i] = *reinterpret_cast<const uint4*>(zt + h * 2 * CHUNK_BYTES + off + i * 2048);
+                        if (f != 1.f) {
+#pragma unroll
+                            for (int h = 0; h < MT; ++h)
+#pragma unroll
+                                for (int i = 0; i < NR; ++i) {
+                                    scale8(v[h][i], f);
+                                    *reinterpret_cast<uint4*>(zt + h * 2 * CHUNK_BYTES + off + i * 2048) = v[h][i];
+                                }
+                        }
+                        if (bias_here) {
+#pragma unroll
+                            for (int h = 0; h < MT; ++h)
+#pragma unroll
+                                for (int i = 0; i < NR; ++i) add8(cs[h], v[h][i]);
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < NR; ++i) {
                         const float f = fr[i];
                         if (f != 1.f || bias_here) {
-                            // packed bf16 path: f = f_hi + f_lo (two bf16); z*f_lo is tiny, so the fused
-                            // multiply-add z*f_hi + (z*f_lo) rounds the product once
-                            const __nv_bfloat16 fh = __float2bfloat16_rn(f);
-                            const __nv_bfloat16 fl = __float2bfloat16_rn(f - __bfloat162float(fh));
-                            const __nv_bfloat162 fh2 = __halves2bfloat162(fh, fh), fl2 = __halves2bfloat162(fl, fl);
 #pragma unroll
                             for (int h = 0; h < MT; ++h) {
                                 uint4* ptr = reinterpret_cast<uint4*>(zt + h * 2 * CHUNK_BYTES + off + i * 2048);
                                 uint4 v = *ptr;
-                                if (f != 1.f) {
-                                    __nv_bfloat162* z2 = reinterpret_cast<__nv_bfloat162*>(&v);
-#pragma unroll
-                                    for (int u = 0; u < 4; ++u) z2[u] = __hfma2(z2[u], fh2, __hmul2(z2[u], fl2));
-                                    *ptr = v;
-                                }
-                                if (bias_here) {
-                                    const uint32_t wds[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-                                    for (int u = 0; u < 4; ++u) {
-                                        cs[h][2 * u] += __uint_as_float(wds[u] << 16);
-                                        cs[h][2 * u + 1] += __uint_as_float(wds[u] & 0xFFFF0000u);
-                                    }
-                                }
+                                if (f != 1.f) { scale8(v, f); *ptr = v; }
+                                if (bias_here) add8(cs[h], v);
                             }
                         }
                     }
