@@ -47,10 +47,16 @@ __device__ __forceinline__ void ew_accumulate(const T* __restrict__ H, long ldh,
     for (int u = 0; u < VEC; ++u) { gg[u] = 0.f; gs[u] = 0.f; }
     constexpr int UNR = sizeof(T) == 2 ? 8 : 4;
     long r = r0 + rg;
-    // example of row r and the row's position in it, advanced without divisions
-    long e = WEIGHTED ? r / rows_per_example : 0;
-    long rem = WEIGHTED ? r - e * rows_per_example : 0;
-    auto advance = [&](int by) { rem += by; while (rem >= rows_per_example) { rem -= rows_per_example; ++e; } };
+    // example of row r and the row's position in it, advanced without divisions (and without a loop when an
+    // example has at least RG rows: one predicated step)
+    int e = WEIGHTED ? (int)(r / rows_per_example) : 0;
+    int rem = WEIGHTED ? (int)(r - (long)e * rows_per_example) : 0;
+    const bool one_step = rows_per_example >= RG;
+    auto advance = [&](int by) {
+        rem += by;
+        if (one_step) { const bool over = rem >= rows_per_example; rem -= over ? rows_per_example : 0; e += over ? 1 : 0; }
+        else while (rem >= rows_per_example) { rem -= rows_per_example; ++e; }
+    };
     for (; r + (UNR - 1) * RG < r1; r += UNR * RG) {
         EwRaw<T, VEC> h[UNR], z[UNR];
         float w[UNR];
@@ -59,7 +65,21 @@ __device__ __forceinline__ void ew_accumulate(const T* __restrict__ H, long ldh,
             const long rr = r + k * RG;
             ew_load(H + (size_t)rr * ldh + c0, h[k]);
             ew_load(Z + (size_t)rr * ldz + c0, z[k]);
-            if (WEIGHTED) { w[k] = __ldg(clip + e); advance(RG); } else w[k] = 1.f;
+            w[k] = 1.f;
+        }
+        if (WEIGHTED) {
+            // the rows of a batch are the same for the whole warp; when they lie in one example (the usual
+            // case) one factor load serves the batch instead of one per row
+            if (rem + (UNR - 1) * RG < rows_per_example) {
+                const float w0 = __ldg(clip + e);
+#pragma unroll
+                for (int k = 0; k < UNR; ++k) w[k] = w0;
+                rem += UNR * RG;                                   // < 2 * rows_per_example here
+                if (rem >= rows_per_example) { rem -= rows_per_example; ++e; }
+            } else {
+#pragma unroll
+                for (int k = 0; k < UNR; ++k) { w[k] = __ldg(clip + e); advance(RG); }
+            }
         }
 #pragma unroll
         for (int k = 0; k < UNR; ++k) {
