@@ -554,8 +554,6 @@ def run_sweep(args):
     peaks = measured_peaks()
     flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     flush = lambda: flush_buf.fill_(1)                                           # noqa: E731
-    ws = torch.empty(dp.dpclip_workspace_bytes(1, 2, 1024, 1024, dp.DPCLIP_BF16), dtype=torch.uint8, device="cuda")
-    dp.dpclip_workspace_init(ws)
     rows = []
     print(f"{'B':>5} {'T':>5} {'d_in':>5} {'d_out':>5} | {'gram us':>9} {'mat us':>9} {'faster':>7} {'flop rule':>9} "
           f"{'auto':>6} | {'clipped sum us':>14} {'TFLOP/s':>8}")
@@ -567,6 +565,8 @@ def run_sweep(args):
     for B, T, d_in, d_out in grid_points:
         if 2 * B * T * (d_in + d_out) > 12e9:
             continue                                                    # keep the device footprint bounded
+        ws = torch.empty(dp.dpclip_workspace_bytes(B, T, d_in, d_out, dp.DPCLIP_BF16), dtype=torch.uint8, device="cuda")
+        dp.dpclip_workspace_init(ws)
         g = torch.Generator(device="cuda").manual_seed(B * 7919 + T)
         A = torch.randn(B, T, d_in, device="cuda", generator=g).to(torch.bfloat16)
         Z = (torch.randn(B, T, d_out, device="cuda", generator=g) * (B * T) ** -0.5).to(torch.bfloat16)

@@ -340,8 +340,12 @@ size_t dpclip_step_host_arena_bytes(const dpclip_layer* layers /* host */, int L
 
 /* Bytes of workspace that dpclip_layer_sqnorms / dpclip_clipped_grad need for
  * this shape: the 256-byte status header, plus, for bf16 layers, room for one
- * fp32 partial tile per SM of the split-row clipped sum (about 39 MB, a bound
- * that does not depend on the shape). */
+ * fp32 partial tile per SM of the split-row clipped sum (about 39 MB).  Long
+ * bf16 layers whose 256 x 256 output tiles do not fill one wave of SMs (64
+ * tiles: 128 of 148) are cut into more, shorter row slices that do; the query
+ * then reports one partial tile per slice (up to a few hundred MB).  A smaller
+ * workspace of at least the 39 MB form is accepted: the layer then runs as one
+ * wave. */
 size_t dpclip_workspace_bytes(int B, int T, int d_in, int d_out, dpclip_dtype dtype, dpclip_method method);
 
 /* Zero the 256-byte status header.  Call once after allocating a workspace. */

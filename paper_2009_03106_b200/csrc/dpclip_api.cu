@@ -456,6 +456,36 @@ int launch_gram_norms(const void* A, long lda, const void* Z, long ldz, int B, i
 // wave of 256 x 256 tiles or two waves of 128 x 256 tiles, plus the partial bias sums.
 constexpr size_t kTcScratchBytes = (size_t)kNumSMs * 256 * 256 * 4 + (size_t)2 * kNumSMs * 256 * 4;
 
+// Row split of the bf16 tensor-core clipped sum: how many row slices each output tile is cut into.
+//   one wave  : floor(per_sm * SMs / tiles) slices -- every CTA one item (two for the small tile when they
+//               stay long); its partial tiles fit the fixed scratch above.
+//   preferred : when one wave would leave more than 5 % of the SMs idle (64 tiles of 256 x 256: 128 of 148)
+//               and the row ranges stay long (>= 192 stages of 64 rows, so that pipeline fill and epilogue
+//               stay below 4 % of an item), the smallest split whose items fill whole waves to >= 97 %; it
+//               needs one partial tile per item, which the workspace query reports for the layer.
+struct ZtaSplit { int one_wave, preferred; };
+inline ZtaSplit zta_pick_split(long nkb, int tiles, int per_sm) {
+    ZtaSplit r;
+    long base = ((long)per_sm * kNumSMs) / tiles;
+    if (base > nkb) base = nkb;
+    if (base < 1) base = 1;
+    r.one_wave = r.preferred = (int)base;
+    auto fill = [&](long ks) {
+        const long items = (long)tiles * ks, waves = (items + kNumSMs - 1) / kNumSMs;
+        return (double)items / (double)(waves * kNumSMs);
+    };
+    double best = fill(base);
+    if (per_sm != 1 || best >= 0.95) return r;
+    for (long ks = base + 1; ks <= 64 * base && nkb / ks >= 192; ++ks) {
+        const double f = fill(ks);
+        if (f > best + 0.01) { best = f; r.preferred = (int)ks; if (f >= 0.97) break; }
+    }
+    return r;
+}
+inline size_t zta_scratch_bytes(int tiles, int ksplit, int BM, bool bias) {
+    return (size_t)tiles * ksplit * ((size_t)BM * 256 * 4 + (bias ? (size_t)BM * 4 : 0));
+}
+
 // second stage of a split-row clipped sum: fixed-order sum of the partial tiles (+ optional noise)
 // Layers of one shape that share a clipped-sum launch (n == 0: a single layer).
 struct GradGroup {
@@ -522,7 +552,12 @@ int launch_zta_tc_mt(const tc::zta::Maps& maps, tc::zta::Params p, int B, bool n
         // every SM streams the same number of row blocks.  (MT = 1 has two accumulator buffers and can
         // overlap the epilogue of one item with the next, so it takes two items per SM when they stay long.)
         const int per_sm = (MT == 1 && tiles <= kNumSMs && nkb / ((2 * kNumSMs) / tiles) >= 16) ? 2 : 1;
-        ksplit = (per_sm * kNumSMs) / tiles;
+        const ZtaSplit split = zta_pick_split(nkb, tiles, per_sm);
+        // the preferred split when the workspace holds its partial tiles, else one wave
+        ksplit = split.one_wave;
+        if (split.preferred != split.one_wave && !fit_to_workspace &&
+            workspace_bytes >= kHeaderBytes + zta_scratch_bytes(tiles, split.preferred, BM, gb != nullptr))
+            ksplit = split.preferred;
         if (fit_to_workspace) {                 // fixed-size scratch: take fewer, longer row slices
             const size_t per_item = (size_t)BM * z::BN * 4 + (gb ? (size_t)BM * 4 : 0);
             const size_t room = workspace_bytes > (size_t)kHeaderBytes ? workspace_bytes - kHeaderBytes : 0;
@@ -953,12 +988,29 @@ int dpclip_pick_method(int B, int T, int d_in, int d_out, long lda, long ldz, dp
     return DPCLIP_SIMT;
 }
 
+// The least workspace an entry point accepts for a layer (the public query may ask for more: see there).
+static size_t workspace_floor(int B, int T, int d_in, int d_out, dpclip_dtype dtype) {
+    if (dtype == DPCLIP_BF16) return kHeaderBytes + kTcScratchBytes;
+    if ((double)B * T * d_in * d_out >= 32.0 * 1024 * 1024) return kHeaderBytes + kTcScratchBytes;
+    return (size_t)kHeaderBytes;
+}
+
 size_t dpclip_workspace_bytes(int B, int T, int d_in, int d_out, dpclip_dtype dtype, dpclip_method method) {
     (void)method;
     // Layers that may take a tensor-core clipped sum (all bf16 layers; fp32 layers above the size where
     // the tf32 path is used) split their rows over CTAs and keep one partial tile per CTA in the
     // workspace; the bound does not depend on the layer's shape.
-    if (dtype == DPCLIP_BF16) return kHeaderBytes + kTcScratchBytes;
+    if (dtype == DPCLIP_BF16) {
+        // ... except for long layers whose tiles do not fill one wave of SMs: room for their preferred split
+        size_t need = kTcScratchBytes;
+        if (d_out > 128 && B > 0 && T > 0 && d_in > 0) {
+            const int tiles = ceil_div(d_out, 256) * ceil_div(d_in, 256);
+            const ZtaSplit split = zta_pick_split(ceil_div((long)B * T, 64L), tiles, 1);
+            const size_t pref = zta_scratch_bytes(tiles, split.preferred, 256, true);
+            if (split.preferred != split.one_wave && pref > need) need = pref;
+        }
+        return kHeaderBytes + need;
+    }
     if ((double)B * T * d_in * d_out >= 32.0 * 1024 * 1024) return kHeaderBytes + kTcScratchBytes;
     return (size_t)kHeaderBytes;
 }
@@ -992,7 +1044,7 @@ int dpclip_layer_sqnorms(const void* A, long lda, const void* Zbar, long ldz, in
         if (dtype == DPCLIP_F32 && method == DPCLIP_MATERIALIZE && !tf32_eligible(A, lda, Zbar, ldz, B, T, d_in, d_out, dtype))
             method = DPCLIP_SIMT;
     }
-    if (!workspace || workspace_bytes < dpclip_workspace_bytes(B, T, d_in, d_out, dtype, method))
+    if (!workspace || workspace_bytes < workspace_floor(B, T, d_in, d_out, dtype))
         return DPCLIP_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     switch (method) {
@@ -1129,7 +1181,7 @@ int dpclip_clipped_grad(const void* A, long lda, const void* Zbar, long ldz, int
     if (rc) return rc;
     if (!gW || ldg < d_in) return DPCLIP_ERR_INVALID_ARG;
     if (!aligned_to(gW, 4) || (gb && !aligned_to(gb, 4))) return DPCLIP_ERR_MISALIGNED;
-    if (!workspace || workspace_bytes < dpclip_workspace_bytes(B, T, d_in, d_out, dtype, DPCLIP_AUTO))
+    if (!workspace || workspace_bytes < workspace_floor(B, T, d_in, d_out, dtype))
         return DPCLIP_ERR_WORKSPACE;
     return clipped_grad_impl(A, lda, Zbar, ldz, B, T, d_in, d_out, dtype, clip, gW, ldg, gb, workspace,
                              workspace_bytes, nullptr, nullptr, (cudaStream_t)stream);
@@ -1144,7 +1196,7 @@ int dpclip_clipped_grad_noise(const void* A, long lda, const void* Zbar, long ld
     if (rc) return rc;
     if (!gW || !(sigma >= 0.f) || !(C >= 0.f)) return DPCLIP_ERR_INVALID_ARG;
     if (!aligned_to(gW, 4) || (gb && !aligned_to(gb, 4))) return DPCLIP_ERR_MISALIGNED;
-    if (!workspace || workspace_bytes < dpclip_workspace_bytes(B, T, d_in, d_out, dtype, DPCLIP_AUTO))
+    if (!workspace || workspace_bytes < workspace_floor(B, T, d_in, d_out, dtype))
         return DPCLIP_ERR_WORKSPACE;
     NoiseSpec ns = {sigma * C, seed, stream_id_w, stream_id_b};
     bool noise_done = false;
