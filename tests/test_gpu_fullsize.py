@@ -103,7 +103,8 @@ def test_sequence_workload_full_step_factors(dp):
     assert 0 < (clip < 1).sum() < w.B                   # both sides of the threshold occur
 
 
-@pytest.mark.parametrize("B,T,d_in,d_out", [(256, 16, 1024, 1024), (256, 128, 1024, 4096), (64, 2048, 1024, 1024)])
+@pytest.mark.parametrize("B,T,d_in,d_out", [(256, 16, 1024, 1024), (256, 128, 1024, 4096), (64, 2048, 1024, 1024),
+                                            (256, 512, 1024, 4096)])
 def test_sweep_points(dp, B, T, d_in, d_out):
     """Points of the Gram-vs-materialise sweep (both norm forms must agree with the oracle)."""
     spec = workloads.LayerSpec("dense", T, d_in, d_out, True, "normal")
@@ -126,6 +127,17 @@ def test_sweep_points(dp, B, T, d_in, d_out):
     assert rel_fro(gW.cpu().numpy(), refW) <= TOL["bf16"]["grad"]
     assert rel_fro(gb.cpu().numpy(), refb) <= TOL["bf16"]["grad"]
     assert dp.dpclip_read_status(ws) == 0
+    # The last point has 64 output tiles and long row ranges: with the queried workspace it is cut into several
+    # waves of row slices; the smallest workspace the entry point accepts makes it run as one wave.  Same sums.
+    floor = dp.dpclip_workspace_bytes(1, 1, 1, 1, dp.DPCLIP_BF16)
+    if ws.numel() > floor:
+        ws2 = torch.empty(floor, dtype=torch.uint8, device="cuda")
+        dp.dpclip_workspace_init(ws2)
+        gW2 = torch.empty_like(gW); gb2 = torch.empty_like(gb)
+        dp.dpclip_clipped_grad(dA, dZ, torch.from_numpy(clip).cuda(), gW2, gb2, ws2)
+        assert rel_fro(gW2.cpu().numpy(), gW.cpu().numpy()) <= 1e-6
+        assert rel_fro(gb2.cpu().numpy(), gb.cpu().numpy()) <= 1e-6
+        assert dp.dpclip_read_status(ws2) == 0
 
 
 def test_mlp_large_graph_replay_full_size(dp):
