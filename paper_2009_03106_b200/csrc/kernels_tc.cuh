@@ -832,17 +832,33 @@ zta_tc_kernel(const __grid_constant__ zta::Maps maps, const zta::Params p) {
                         }
                     }
                 } else {
+                    // a factor per row (short examples, the ends of a row range): the same order -- all loads,
+                    // then the rows that need it rewritten -- at the price of loading rows whose factor is 1
+                    bool any = bias_here;
 #pragma unroll
-                    for (int i = 0; i < NR; ++i) {
-                        const float f = fr[i];
-                        if (f != 1.f || bias_here) {
+                    for (int i = 0; i < NR; ++i) any = any || fr[i] != 1.f;
+                    if (any) {
+                        uint4 v[MT][NR];
 #pragma unroll
-                            for (int h = 0; h < MT; ++h) {
-                                uint4* ptr = reinterpret_cast<uint4*>(zt + h * 2 * CHUNK_BYTES + off + i * 2048);
-                                uint4 v = *ptr;
-                                if (f != 1.f) { scale8(v, f); *ptr = v; }
-                                if (bias_here) add8(cs[h], v);
+                        for (int h = 0; h < MT; ++h)
+#pragma unroll
+                            for (int i = 0; i < NR; ++i)
+                                v[h][i] = *reinterpret_cast<const uint4*>(zt + h * 2 * CHUNK_BYTES + off + i * 2048);
+#pragma unroll
+                        for (int i = 0; i < NR; ++i) {
+                            if (fr[i] != 1.f) {
+#pragma unroll
+                                for (int h = 0; h < MT; ++h) {
+                                    scale8(v[h][i], fr[i]);
+                                    *reinterpret_cast<uint4*>(zt + h * 2 * CHUNK_BYTES + off + i * 2048) = v[h][i];
+                                }
                             }
+                        }
+                        if (bias_here) {
+#pragma unroll
+                            for (int h = 0; h < MT; ++h)
+#pragma unroll
+                                for (int i = 0; i < NR; ++i) add8(cs[h], v[h][i]);
                         }
                     }
                 }
