@@ -247,6 +247,36 @@ int dpclip_conv_clipped_grad(const void* X, const void* Zbar, int z_channel_majo
                              int d_out, dpclip_dtype dtype, const float* clip, float* gW, long ldg, float* gb,
                              void* workspace, size_t workspace_bytes, void* stream);
 
+/* The whole path over a model whose layers are not all dense products: Algorithm 1 with the per-layer
+ * gradients of Sec. "Fully-connected", "Convolutional" and "LayerNorm" layers in one call.
+ *   kind DPCLIP_KIND_DENSE       `layer` as in dpclip_step.
+ *   kind DPCLIP_KIND_ELEMENTWISE gain/shift of a normalisation layer: layer.A = hbar [B][T][d] (lda),
+ *                                layer.Zbar = dL/dh [B][T][d] (ldz), d_in = d_out = d, has_bias = the layer
+ *                                has a shift, gW = the gain's gradient [d], gb = the shift's [d]; ldg, method
+ *                                unused.
+ *   kind DPCLIP_KIND_CONV        convolution given by its input feature map: layer.A = X [B][C][H][W] dense,
+ *                                layer.Zbar = dL/dZ ([B][Ho*Wo][d_out], or [B][d_out][Ho*Wo] when
+ *                                z_channel_major), `conv` the geometry, gW [d_out][C*kh*kw] with ldg =
+ *                                C*kh*kw, gb [d_out]; lda, ldz, T, d_in, method unused.
+ * Row l of sq_layers [L][B] and the noise streams stream_id0 + 2l (gW) and + 2l + 1 (gb) belong to layer l
+ * whatever its kind; factors and norms are over all L layers.  Dense layers take the same launches as in
+ * dpclip_step (a model of dense layers only IS dpclip_step); the other kinds run through their per-layer
+ * entry points followed by dpclip_add_noise.  workspace >= dpclip_model_workspace_bytes().  L <= 256.
+ * Errors as for the per-layer entry points; INVALID_ARG for an unknown kind or d_in != d_out in an
+ * element-wise layer; UNSUPPORTED for padded output rows. */
+typedef enum { DPCLIP_KIND_DENSE = 0, DPCLIP_KIND_ELEMENTWISE = 1, DPCLIP_KIND_CONV = 2 } dpclip_layer_kind;
+typedef struct {
+    int kind;                       /* dpclip_layer_kind */
+    dpclip_layer layer;
+    dpclip_conv conv;               /* kind CONV */
+    int z_channel_major;            /* kind CONV */
+} dpclip_model_layer;
+int dpclip_model_step(const dpclip_model_layer* layers /* host */, int L, int B, dpclip_dtype dtype,
+                      float C, float sigma, unsigned long long seed, unsigned long long stream_id0,
+                      float* sq_layers, float* clip, float* norms,
+                      void* workspace, size_t workspace_bytes, void* stream);
+size_t dpclip_model_workspace_bytes(const dpclip_model_layer* layers /* host */, int L, int B, dpclip_dtype dtype);
+
 /* Parameter updates with the noise folded in (one pass over the parameters instead of a noise pass and
  * an optimiser pass).  gsum is the PRE-noise clipped sum of one tensor (run the step with sigma = 0);
  * the noisy mean gradient is g[j] = (gsum[j] + sigma * C * xi_j) * inv_tau with xi as in dpclip_add_noise

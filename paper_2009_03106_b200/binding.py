@@ -41,6 +41,10 @@ class _CLayer(ctypes.Structure):
                 ("gW", _vp), ("ldg", _l), ("gb", _vp)]
 
 
+class _CModelLayer(ctypes.Structure):
+    _fields_ = [("kind", _i), ("layer", _CLayer), ("conv", _CConv), ("z_channel_major", _i)]
+
+
 def library_path() -> str:
     return _LIB_PATH
 
@@ -97,6 +101,11 @@ def load_library():
     L.dpclip_step_host.argtypes = [ctypes.POINTER(_CLayer), _i, _i, _i, _f, _f, _u64, _u64, _vp, _vp, _vp, _sz, _vp]
     L.dpclip_step_host_arena_bytes.argtypes = [ctypes.POINTER(_CLayer), _i, _i, _i]
     L.dpclip_step_host_arena_bytes.restype = _sz
+    L.dpclip_model_step.argtypes = [ctypes.POINTER(_CModelLayer), _i, _i, _i, _f, _f, _u64, _u64, _vp, _vp, _vp, _vp,
+                                    _sz, _vp]
+    L.dpclip_model_step.restype = _i
+    L.dpclip_model_workspace_bytes.argtypes = [ctypes.POINTER(_CModelLayer), _i, _i, _i]
+    L.dpclip_model_workspace_bytes.restype = _sz
     L.dpclip_workspace_bytes.argtypes = [_i, _i, _i, _i, _i, _i]
     L.dpclip_workspace_bytes.restype = _sz
     L.dpclip_workspace_init.argtypes = [_vp, _sz, _vp]
@@ -507,6 +516,99 @@ def dpclip_t1_layers_supported(plan: StepPlan) -> bool:
 
 def dpclip_step(plan: StepPlan, C: float, sigma: float, seed: int, stream_id0: int = 0, stream=None) -> None:
     _check("dpclip_step", load_library().dpclip_step(
+        plan._c, plan.L, plan.B, plan.dtype_code, C, sigma, seed, stream_id0, _ptr(plan.sq_layers),
+        _ptr(plan.clip), _ptr(plan.norms), _ptr(plan.workspace), plan.workspace.numel(), _stream(stream)))
+
+
+DPCLIP_KIND_DENSE, DPCLIP_KIND_ELEMENTWISE, DPCLIP_KIND_CONV = 0, 1, 2
+
+
+@dataclass
+class ModelLayer:
+    """One layer of a model for dpclip_model_step.
+    dense:        A (B, T, d_in), Zbar (B, T, d_out)
+    element-wise: A = hbar (B, T, d), Zbar (B, T, d); has_bias = the layer has a shift
+    conv:         A = X (B, C, H, W), Zbar (B, Ho*Wo, d_out) or, z_channel_major, (B, d_out, Ho*Wo);
+                  conv = (kh, kw, stride, pad)"""
+    kind: int
+    A: torch.Tensor
+    Zbar: torch.Tensor
+    has_bias: bool = True
+    method: int = DPCLIP_AUTO
+    conv: Optional[tuple] = None
+    z_channel_major: bool = False
+
+
+class ModelPlan:
+    """Buffers and the C descriptor array of a model with dense, element-wise and convolution layers.
+    Holds no arithmetic: `run` is one dpclip_model_step call.  gW[l] is (d_out, d_in) for dense and
+    convolution layers (d_in = C*kh*kw) and (d,) for element-wise layers; all live in `flat`."""
+
+    def __init__(self, layers: Sequence[ModelLayer], device=None):
+        self.layers = list(layers)
+        self.L = len(self.layers)
+        dev = device or self.layers[0].A.device
+        self.B = self.layers[0].A.shape[0]
+        self.dtype_code = _dtype_code(self.layers[0].A)
+        self._c = (_CModelLayer * self.L)()
+        shapes, total = [], 0
+        for y in self.layers:
+            assert y.A.shape[0] == self.B and _dtype_code(y.A) == self.dtype_code and y.A.dtype == y.Zbar.dtype
+            if y.kind == DPCLIP_KIND_DENSE:
+                w_shape, nb = (y.Zbar.shape[-1], y.A.shape[-1]), y.Zbar.shape[-1]
+            elif y.kind == DPCLIP_KIND_ELEMENTWISE:
+                assert y.A.shape == y.Zbar.shape
+                w_shape, nb = (y.A.shape[-1],), y.A.shape[-1]
+            elif y.kind == DPCLIP_KIND_CONV:
+                kh, kw, stride, pad = y.conv
+                _, d_out, _ = _conv_args(y.A, y.Zbar, kh, kw, stride, pad, y.z_channel_major)
+                w_shape, nb = (d_out, y.A.shape[1] * kh * kw), d_out
+            else:
+                raise ValueError(f"unknown layer kind {y.kind}")
+            nw = 1
+            for v in w_shape:
+                nw *= v
+            ow = total; total += -(-nw // 64) * 64
+            ob = total; total += (-(-nb // 64) * 64) if y.has_bias else 0
+            shapes.append((w_shape, nw, ow, nb, ob))
+        self.flat = torch.zeros((total,), dtype=torch.float32, device=dev)
+        self.gW: List[torch.Tensor] = []
+        self.gb: List[Optional[torch.Tensor]] = []
+        for l, (y, (w_shape, nw, ow, nb, ob)) in enumerate(zip(self.layers, shapes)):
+            gW = self.flat[ow:ow + nw].view(*w_shape)
+            gb = self.flat[ob:ob + nb] if y.has_bias else None
+            self.gW.append(gW); self.gb.append(gb)
+            c = self._c[l]
+            c.kind = y.kind
+            if y.kind == DPCLIP_KIND_CONV:
+                kh, kw, stride, pad = y.conv
+                _, d_out, geom = _conv_args(y.A, y.Zbar, kh, kw, stride, pad, y.z_channel_major)
+                c.conv = geom
+                c.z_channel_major = int(y.z_channel_major)
+                c.layer = _CLayer(_ptr(y.A), 0, _ptr(y.Zbar), 0, 0, w_shape[1], d_out, int(y.has_bias), y.method,
+                                  _ptr(gW), w_shape[1], _ptr(gb))
+            else:
+                B, T, d_in, lda = _rows(y.A)
+                _, _, d_out, ldz = _rows(y.Zbar)
+                c.layer = _CLayer(_ptr(y.A), lda, _ptr(y.Zbar), ldz, T, d_in, d_out, int(y.has_bias), y.method,
+                                  _ptr(gW), d_in, _ptr(gb))
+        self.sq_layers = torch.empty((self.L, self.B), dtype=torch.float32, device=dev)
+        self.clip = torch.empty((self.B,), dtype=torch.float32, device=dev)
+        self.norms = torch.empty((self.B,), dtype=torch.float32, device=dev)
+        ws = dpclip_model_workspace_bytes(self)
+        self.workspace = torch.empty((ws,), dtype=torch.uint8, device=dev)
+        dpclip_workspace_init(self.workspace)
+
+    def run(self, C: float, sigma: float, seed: int, stream_id0: int = 0, stream=None) -> None:
+        dpclip_model_step(self, C, sigma, seed, stream_id0, stream)
+
+
+def dpclip_model_workspace_bytes(plan: ModelPlan) -> int:
+    return load_library().dpclip_model_workspace_bytes(plan._c, plan.L, plan.B, plan.dtype_code)
+
+
+def dpclip_model_step(plan: ModelPlan, C: float, sigma: float, seed: int, stream_id0: int = 0, stream=None) -> None:
+    _check("dpclip_model_step", load_library().dpclip_model_step(
         plan._c, plan.L, plan.B, plan.dtype_code, C, sigma, seed, stream_id0, _ptr(plan.sq_layers),
         _ptr(plan.clip), _ptr(plan.norms), _ptr(plan.workspace), plan.workspace.numel(), _stream(stream)))
 

@@ -1563,15 +1563,59 @@ int dpclip_add_noise(float* g, size_t n, float sigma, float C, unsigned long lon
     return launch_status();
 }
 
-int dpclip_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, float C, float sigma,
-                unsigned long long seed, unsigned long long stream_id0, float* sq_layers, float* clip,
-                float* norms, void* workspace, size_t workspace_bytes, void* stream) {
-    if (!layers || L <= 0 || B <= 0 || !sq_layers || !clip) return DPCLIP_ERR_INVALID_ARG;
-    if (!(C > 0.f) || !(sigma >= 0.f)) return DPCLIP_ERR_INVALID_ARG;
-    if (dtype != DPCLIP_F32 && dtype != DPCLIP_BF16) return DPCLIP_ERR_INVALID_ARG;
-    int rc = try_fused_t1_step(layers, L, B, dtype, C, sigma, seed, stream_id0, sq_layers, clip, norms, workspace,
-                               workspace_bytes, (cudaStream_t)stream);
-    if (rc <= 0) return rc;                  // done (0) or argument error (< 0); 1 = take the general path
+// Norms / clipped sum + noise of a layer that is not a dense product (element-wise parameters, convolution
+// given by its feature map): the per-layer entry points, with the layer's row of sq and its noise streams.
+static int other_kind_sqnorms(const dpclip_model_layer& m, int B, dpclip_dtype dtype, float* sq_row, void* workspace,
+                              size_t workspace_bytes, void* stream) {
+    const dpclip_layer& y = m.layer;
+    if (m.kind == DPCLIP_KIND_ELEMENTWISE) {
+        if (y.d_in != y.d_out) return DPCLIP_ERR_INVALID_ARG;
+        return dpclip_elementwise_sqnorms(y.A, y.lda, y.Zbar, y.ldz, B, y.T, y.d_in, dtype, y.has_bias, sq_row, stream);
+    }
+    if (m.kind == DPCLIP_KIND_CONV)
+        return dpclip_conv_sqnorms(y.A, y.Zbar, m.z_channel_major, B, &m.conv, y.d_out, dtype, y.has_bias, sq_row,
+                                   workspace, workspace_bytes, stream);
+    return DPCLIP_ERR_INVALID_ARG;
+}
+
+static int other_kind_clipped_grad_noise(const dpclip_model_layer& m, int B, dpclip_dtype dtype, const float* clip,
+                                         float C, float sigma, unsigned long long seed, unsigned long long sid_w,
+                                         unsigned long long sid_b, void* workspace, size_t workspace_bytes,
+                                         void* stream) {
+    const dpclip_layer& y = m.layer;
+    float* gb = y.has_bias ? y.gb : nullptr;
+    if (!y.gW || (y.has_bias && !gb)) return DPCLIP_ERR_INVALID_ARG;
+    size_t n_w = 0;
+    int rc;
+    if (m.kind == DPCLIP_KIND_ELEMENTWISE) {
+        if (y.d_in != y.d_out) return DPCLIP_ERR_INVALID_ARG;
+        rc = dpclip_elementwise_clipped_grad(y.A, y.lda, y.Zbar, y.ldz, B, y.T, y.d_in, dtype, clip, y.gW, gb, stream);
+        n_w = (size_t)y.d_in;
+    } else if (m.kind == DPCLIP_KIND_CONV) {
+        const long d_in = (long)m.conv.C * m.conv.kh * m.conv.kw;
+        if (y.ldg != d_in) return DPCLIP_ERR_UNSUPPORTED;        // noise indexes the dense tensor
+        rc = dpclip_conv_clipped_grad(y.A, y.Zbar, m.z_channel_major, B, &m.conv, y.d_out, dtype, clip, y.gW, y.ldg, gb,
+                                      workspace, workspace_bytes, stream);
+        n_w = (size_t)y.d_out * (size_t)d_in;
+    } else {
+        return DPCLIP_ERR_INVALID_ARG;
+    }
+    if (rc) return rc;
+    rc = dpclip_add_noise(y.gW, n_w, sigma, C, seed, sid_w, stream);
+    if (rc) return rc;
+    if (gb) rc = dpclip_add_noise(gb, m.kind == DPCLIP_KIND_ELEMENTWISE ? (size_t)y.d_in : (size_t)y.d_out, sigma, C,
+                                  seed, sid_b, stream);
+    return rc;
+}
+
+// The path layer by layer (with the launches that several layers share).  `other`, when given, is the model's
+// own descriptor array: entries of a kind other than dense have a placeholder with T = 0 in `layers`, which
+// every grouping rule below passes over, and go through the two functions above.
+static int step_general(const dpclip_layer* layers, const dpclip_model_layer* other, int L, int B, dpclip_dtype dtype,
+                        float C, float sigma, unsigned long long seed, unsigned long long stream_id0,
+                        float* sq_layers, float* clip, float* norms, void* workspace, size_t workspace_bytes,
+                        void* stream) {
+    int rc;
     T1Group t1;
     rc = prepare_t1_group(t1, layers, L, B, dtype, C, sigma, seed, stream_id0, sq_layers, clip);
     if (rc) return rc;
@@ -1589,6 +1633,11 @@ int dpclip_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, fl
     }
     for (int l = 0; l < L; ++l) {
         const dpclip_layer& y = layers[l];
+        if (other && other[l].kind != DPCLIP_KIND_DENSE) {
+            rc = other_kind_sqnorms(other[l], B, dtype, sq_layers + (size_t)l * B, workspace, workspace_bytes, stream);
+            if (rc) return rc;
+            continue;
+        }
         if (t1.active && y.T == 1) continue;
         if (track && in_gram_group[l]) continue;
         rc = dpclip_layer_sqnorms(y.A, y.lda, y.Zbar, y.ldz, B, y.T, y.d_in, y.d_out, dtype, y.has_bias,
@@ -1611,6 +1660,12 @@ int dpclip_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, fl
     }
     for (int l = 0; l < L; ++l) {
         const dpclip_layer& y = layers[l];
+        if (other && other[l].kind != DPCLIP_KIND_DENSE) {
+            rc = other_kind_clipped_grad_noise(other[l], B, dtype, clip, C, sigma, seed, stream_id0 + 2ull * l,
+                                               stream_id0 + 2ull * l + 1, workspace, workspace_bytes, stream);
+            if (rc) return rc;
+            continue;
+        }
         if (t1.active && y.T == 1) continue;
         if (track && in_grad_group[l]) continue;
         float* gb = y.has_bias ? y.gb : nullptr;
@@ -1635,6 +1690,63 @@ int dpclip_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, fl
         }
     }
     return DPCLIP_OK;
+}
+
+int dpclip_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, float C, float sigma,
+                unsigned long long seed, unsigned long long stream_id0, float* sq_layers, float* clip,
+                float* norms, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!layers || L <= 0 || B <= 0 || !sq_layers || !clip) return DPCLIP_ERR_INVALID_ARG;
+    if (!(C > 0.f) || !(sigma >= 0.f)) return DPCLIP_ERR_INVALID_ARG;
+    if (dtype != DPCLIP_F32 && dtype != DPCLIP_BF16) return DPCLIP_ERR_INVALID_ARG;
+    const int rc = try_fused_t1_step(layers, L, B, dtype, C, sigma, seed, stream_id0, sq_layers, clip, norms, workspace,
+                                     workspace_bytes, (cudaStream_t)stream);
+    if (rc <= 0) return rc;                  // done (0) or argument error (< 0); 1 = take the general path
+    return step_general(layers, nullptr, L, B, dtype, C, sigma, seed, stream_id0, sq_layers, clip, norms, workspace,
+                        workspace_bytes, stream);
+}
+
+static int conv_out_positions(const dpclip_conv& g) {
+    if (g.stride <= 0 || g.kh <= 0 || g.kw <= 0) return 0;
+    const int Ho = (g.H + 2 * g.pad - g.kh) / g.stride + 1, Wo = (g.W + 2 * g.pad - g.kw) / g.stride + 1;
+    return Ho > 0 && Wo > 0 ? Ho * Wo : 0;
+}
+
+size_t dpclip_model_workspace_bytes(const dpclip_model_layer* layers, int L, int B, dpclip_dtype dtype) {
+    size_t ws = kHeaderBytes;
+    if (!layers || L <= 0 || B <= 0) return ws;
+    for (int l = 0; l < L; ++l) {
+        const dpclip_layer& y = layers[l].layer;
+        size_t w = kHeaderBytes;
+        if (layers[l].kind == DPCLIP_KIND_DENSE)
+            w = dpclip_workspace_bytes(B, y.T, y.d_in, y.d_out, dtype, (dpclip_method)y.method);
+        else if (layers[l].kind == DPCLIP_KIND_CONV)
+            w = dpclip_workspace_bytes(B, conv_out_positions(layers[l].conv),
+                                       layers[l].conv.C * layers[l].conv.kh * layers[l].conv.kw, y.d_out, dtype, DPCLIP_AUTO);
+        if (w > ws) ws = w;
+    }
+    return ws;
+}
+
+int dpclip_model_step(const dpclip_model_layer* layers, int L, int B, dpclip_dtype dtype, float C, float sigma,
+                      unsigned long long seed, unsigned long long stream_id0, float* sq_layers, float* clip,
+                      float* norms, void* workspace, size_t workspace_bytes, void* stream) {
+    constexpr int kMaxLayers = 256;
+    if (!layers || L <= 0 || L > kMaxLayers || B <= 0 || !sq_layers || !clip) return DPCLIP_ERR_INVALID_ARG;
+    if (!(C > 0.f) || !(sigma >= 0.f)) return DPCLIP_ERR_INVALID_ARG;
+    if (dtype != DPCLIP_F32 && dtype != DPCLIP_BF16) return DPCLIP_ERR_INVALID_ARG;
+    dpclip_layer dense[kMaxLayers];
+    bool all_dense = true;
+    for (int l = 0; l < L; ++l) {
+        if (layers[l].kind == DPCLIP_KIND_DENSE) { dense[l] = layers[l].layer; continue; }
+        if (layers[l].kind != DPCLIP_KIND_ELEMENTWISE && layers[l].kind != DPCLIP_KIND_CONV) return DPCLIP_ERR_INVALID_ARG;
+        memset(&dense[l], 0, sizeof(dense[l]));             // T = 0: no grouping rule takes it
+        all_dense = false;
+    }
+    if (all_dense)
+        return dpclip_step(dense, L, B, dtype, C, sigma, seed, stream_id0, sq_layers, clip, norms, workspace,
+                           workspace_bytes, stream);
+    return step_general(dense, layers, L, B, dtype, C, sigma, seed, stream_id0, sq_layers, clip, norms, workspace,
+                        workspace_bytes, stream);
 }
 
 size_t dpclip_step_host_arena_bytes(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype) {

@@ -304,6 +304,68 @@ def test_conv_implicit_im2col(dp, case, dtype):
     assert dp.dpclip_read_status(ws) == 0
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_model_step_mixed_layer_kinds(dp, dtype):
+    """One dpclip_model_step call over a convolution given by its feature map (channel-major dL/dZ), a
+    LayerNorm's gain and shift, a sequence layer and a T = 1 head: row l of the norms, the factors over all
+    layers, clipped sums and the noise streams 2l / 2l + 1 equal the oracle's, layer kind by layer kind."""
+    B, C, sigma, seed, sid0 = 7, 1.0, 0.6, 21, 4
+    cin, H, W, k, pad, stride, cout = 3, 8, 8, 3, 1, 1, 16
+    X, Zc = workloads.conv_inputs(5, B, cin, H, W, k, pad, stride, cout, dtype, var_z=0.02)
+    Ac = workloads.im2col(X, k, pad, stride)
+    Hn, Zn = workloads.layernorm_pair(6, B, 12, 48, dtype, var_z=0.01)
+    rng = np.random.default_rng(8)
+    rnd = (lambda a: workloads.round_to_bf16(a.astype(np.float32))) if dtype == "bf16" else (lambda a: a.astype(np.float32))
+    As, Zs = rnd(rng.standard_normal((B, 12, 48))), rnd(rng.standard_normal((B, 12, 40)) * 0.1)
+    A1, Z1 = rnd(rng.standard_normal((B, 1, 40))), rnd(rng.standard_normal((B, 1, 10)) * 0.5)
+    sq_ref = np.stack([oracle.layer_sqnorms(Ac, Zc, True), oracle.elementwise_sqnorms(Hn, Zn, True),
+                       oracle.layer_sqnorms(As, Zs, True), oracle.layer_sqnorms(A1, Z1, False)])
+    # rescale dL/dZ per example so that the norms straddle C (both sides of the threshold occur)
+    n0, _ = oracle.factors(sq_ref, C)
+    r = (workloads.spread_factors(B, 1) * C / n0)
+    sc = lambda Z: rnd(Z.astype(np.float64) * r.reshape((B,) + (1,) * (Z.ndim - 1)))          # noqa: E731
+    Zc, Zn, Zs, Z1 = sc(Zc), sc(Zn), sc(Zs), sc(Z1)
+    sq_ref = np.stack([oracle.layer_sqnorms(Ac, Zc, True), oracle.elementwise_sqnorms(Hn, Zn, True),
+                       oracle.layer_sqnorms(As, Zs, True), oracle.layer_sqnorms(A1, Z1, False)])
+    norms_ref, clip_ref = oracle.factors(sq_ref, C)
+    assert 0 < (clip_ref < 1).sum() < B
+    ref = [oracle.clipped_grad(Ac, Zc, clip_ref), oracle.elementwise_clipped_grad(Hn, Zn, clip_ref),
+           oracle.clipped_grad(As, Zs, clip_ref), (oracle.clipped_grad(A1, Z1, clip_ref)[0], None)]
+    dZc = to_device(Zc, dtype).transpose(1, 2).contiguous()          # [B][d_out][T]
+    plan = dp.ModelPlan([
+        dp.ModelLayer(dp.DPCLIP_KIND_CONV, to_device(X, dtype), dZc, True, conv=(k, k, stride, pad), z_channel_major=True),
+        dp.ModelLayer(dp.DPCLIP_KIND_ELEMENTWISE, to_device(Hn, dtype), to_device(Zn, dtype), True),
+        dp.ModelLayer(dp.DPCLIP_KIND_DENSE, to_device(As, dtype), to_device(Zs, dtype), True),
+        dp.ModelLayer(dp.DPCLIP_KIND_DENSE, to_device(A1, dtype), to_device(Z1, dtype), False)])
+    tol = TOL[dtype]
+    for sg in (0.0, sigma):
+        plan.flat.fill_(float("nan"))
+        plan.run(C, sg, seed, sid0)
+        torch.cuda.synchronize()
+        assert dp.dpclip_read_status(plan.workspace) == 0
+        assert max_rel(np.sqrt(plan.sq_layers.cpu().numpy()), np.sqrt(sq_ref)) <= tol["norm"]
+        assert max_rel(plan.norms.cpu().numpy(), norms_ref) <= tol["norm"]
+        check_saturation(plan.clip.cpu().numpy(), norms_ref, clip_ref, C)
+        for l, (rW, rb) in enumerate(ref):
+            eW = oracle.add_noise(rW.reshape(-1), sg, C, seed, sid0 + 2 * l).reshape(rW.shape)
+            assert plan.gW[l].shape == rW.shape
+            assert rel_fro(plan.gW[l].cpu().numpy(), eW) <= tol["grad"], (sg, l)
+            if rb is not None:
+                eb = oracle.add_noise(rb, sg, C, seed, sid0 + 2 * l + 1)
+                assert rel_fro(plan.gb[l].cpu().numpy(), eb) <= tol["grad"], (sg, l)
+            else:
+                assert plan.gb[l] is None
+    # a model of dense layers only is dpclip_step
+    dense = [dp.ModelLayer(dp.DPCLIP_KIND_DENSE, to_device(As, dtype), to_device(Zs, dtype), True),
+             dp.ModelLayer(dp.DPCLIP_KIND_DENSE, to_device(A1, dtype), to_device(Z1, dtype), False)]
+    mp = dp.ModelPlan(dense); mp.run(C, sigma, seed, sid0)
+    sp = dp.StepPlan([dp.Layer(y.A, y.Zbar, y.has_bias) for y in dense]); sp.run(C, sigma, seed, sid0)
+    torch.cuda.synchronize()
+    assert torch.equal(mp.clip, sp.clip)
+    for l in range(2):
+        assert torch.equal(mp.gW[l], sp.gW[l])
+
+
 # ---------------------------------------------------------------------------
 # (c) factors
 # ---------------------------------------------------------------------------
