@@ -452,6 +452,32 @@ def bench_elementwise(torch, dp, B, T, d, dtype, steps, flush, peaks):
     return out
 
 
+def bench_model_block(torch, dp, steps, flush):
+    """One Transformer block through dpclip_model_step (one call, one stream, replayed as a CUDA graph): LayerNorm
+    gain/shift, four bias-free d -> d attention projections, LayerNorm, d -> d_ff and d_ff -> d layers;
+    B = 128, T = 256, d = 512, d_ff = 2048, bf16."""
+    import dataclasses
+    w = workloads.seq("bf16")
+    w = dataclasses.replace(w, layers=w.layers[:6])
+    dense = workloads.generate(w, 0)
+    lns = [workloads.layernorm_pair(50 + k, w.B, 256, 512, "bf16", var_z=w.zbar_var) for k in range(2)]
+    mk = lambda kind, A, Z, b: dp.ModelLayer(kind, to_dev(A, "bf16", torch), to_dev(Z, "bf16", torch), b)   # noqa: E731
+    d = [mk(dp.DPCLIP_KIND_DENSE, A, Z, s.has_bias) for (A, Z), s in zip(dense, w.layers)]
+    n = [mk(dp.DPCLIP_KIND_ELEMENTWISE, H, Z, True) for H, Z in lns]
+    plan = dp.ModelPlan([n[0]] + d[:4] + [n[1]] + d[4:])
+    plan.run(w.C, w.sigma, 1)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        plan.run(w.C, w.sigma, 1)
+    ms = float(np.mean(time_steps(torch, graph.replay, steps, 3, flush)))
+    assert dp.dpclip_read_status(plan.workspace) == 0
+    nbytes = sum(2 * 2 * y.A.numel() + 2 * 2 * y.Zbar.numel() for y in plan.layers) + 4 * plan.flat.numel()
+    return dict(workload="transformer_block_b128_t256_d512_bf16", entry="dpclip_model_step", layers=plan.L,
+                ms_per_step=ms, value=w.B / (ms * 1e-3), algorithmic_bytes=nbytes,
+                clipped_fraction=float((plan.clip < 1).float().mean().item()))
+
+
 def bench_conv_implicit(torch, dp, name, B, C, H, W, k, pad, d_out, dtype, steps, flush, peaks):
     """A convolution layer straight from its feature map (implicit im2col on the tensor cores), next to the same
     layer through the patch-matrix entry points.  Algorithmic bytes: feature map + Zbar once per kernel."""
@@ -731,6 +757,8 @@ def main():
             for shape in ((128, 256, 512, "bf16"), (512, 512, 1024, "bf16")):
                 r = bench_elementwise(torch, dp, *shape, min(args.steps, 20), flush, peaks)
                 others[r["workload"]] = r
+            r = bench_model_block(torch, dp, min(args.steps, 20), flush)
+            others[r["workload"]] = r
             for cdt in ("f32", "bf16"):
                 r = bench_conv_implicit(torch, dp, "conv2_implicit_im2col_b128_" + cdt, 128, 32, 16, 16, 3, 1, 64, cdt,
                                         min(args.steps, 20), flush, peaks)
