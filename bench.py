@@ -470,11 +470,14 @@ def bench_model_block(torch, dp, steps, flush):
     graph = torch.cuda.CUDAGraph()
     with torch.cuda.graph(graph):
         plan.run(w.C, w.sigma, 1)
-    ms = float(np.mean(time_steps(torch, graph.replay, steps, 3, flush)))
+    one_stream_ms = float(np.mean(time_steps(torch, graph.replay, steps, 3, flush)))
+    graph4 = plan.capture(w.C, w.sigma, 1, branches=4)
+    ms = float(np.mean(time_steps(torch, graph4.replay, steps, 3, flush)))
     assert dp.dpclip_read_status(plan.workspace) == 0
     nbytes = sum(2 * 2 * y.A.numel() + 2 * 2 * y.Zbar.numel() for y in plan.layers) + 4 * plan.flat.numel()
     return dict(workload="transformer_block_b128_t256_d512_bf16", entry="dpclip_model_step", layers=plan.L,
-                ms_per_step=ms, value=w.B / (ms * 1e-3), algorithmic_bytes=nbytes,
+                ms_per_step=ms, one_stream_ms_per_step=one_stream_ms, value=w.B / (ms * 1e-3), algorithmic_bytes=nbytes,
+                timing="graph of per-layer calls on four streams; one_stream = the single dpclip_model_step call as a graph",
                 clipped_fraction=float((plan.clip < 1).float().mean().item()))
 
 

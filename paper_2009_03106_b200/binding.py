@@ -9,6 +9,7 @@ from __future__ import annotations
 import ctypes
 import os
 from dataclasses import dataclass
+from types import SimpleNamespace
 from typing import List, Optional, Sequence
 
 import torch
@@ -344,6 +345,23 @@ class StepPlan:
     def run(self, C: float, sigma: float, seed: int, stream_id0: int = 0, stream=None) -> None:
         dpclip_step(self, C, sigma, seed, stream_id0, stream)
 
+    # what `capture` needs to know about a layer (ModelPlan answers differently for the other layer kinds)
+    def _grouping(self):
+        """The object the several-layers-per-launch entry points take (dense descriptors, one per layer)."""
+        return self
+
+    def _is_t1(self, l: int) -> bool:
+        return self.layers[l].A.shape[1] == 1
+
+    def _norm(self, l: int, ws: torch.Tensor) -> None:
+        y = self.layers[l]
+        dpclip_layer_sqnorms(y.A, y.Zbar, y.has_bias, self.sq_layers[l], ws, y.method)
+
+    def _grad(self, l: int, ws: torch.Tensor, C: float, sigma: float, seed: int, stream_id0: int) -> None:
+        y = self.layers[l]
+        dpclip_clipped_grad_noise(y.A, y.Zbar, self.clip, self.gW[l], self.gb[l], sigma, C, seed,
+                                  stream_id0 + 2 * l, stream_id0 + 2 * l + 1, ws)
+
     def capture(self, C: float, sigma: float, seed: int, stream_id0: int = 0, branches: int = 1):
         """Record one step into a CUDA graph (the launch-bound small workloads spend most of a step
         in launch gaps).  Returns the graph; `graph.replay()` re-runs the same kernels on the same
@@ -381,34 +399,34 @@ class StepPlan:
                     ev = torch.cuda.Event(); ev.record(s); main.wait_event(ev)
 
             # the T = 1 layers of a mixed model go together (one launch per stage) when the library takes them
-            t1_together = any(y.A.shape[1] == 1 for y in self.layers) and dpclip_t1_layers_supported(self)
+            grp = self._grouping()
+            t1_together = any(self._is_t1(l) for l in range(self.L)) and dpclip_t1_layers_supported(grp)
             last = streams[-1]
             fork()
             # layers whose norms go by the Gram identity share one launch (on the first branch)
-            taken = dpclip_gram_layers_sqnorms(self, self._branch_ws[0])
-            rest = [(l, y) for l, y in enumerate(self.layers) if not (t1_together and y.A.shape[1] == 1)]
+            taken = dpclip_gram_layers_sqnorms(grp, self._branch_ws[0])
+            rest = [l for l in range(self.L) if not (t1_together and self._is_t1(l))]
             if t1_together:
                 with torch.cuda.stream(last):
-                    dpclip_t1_layers_sqnorms(self)
-            rest_norms = [(l, y) for l, y in rest if not taken[l]]
-            for k, (l, y) in enumerate(rest_norms):
+                    dpclip_t1_layers_sqnorms(grp)
+            rest_norms = [l for l in rest if not taken[l]]
+            for k, l in enumerate(rest_norms):
                 b = (k + (1 if any(taken) else 0)) % branches
                 with torch.cuda.stream(streams[b]):
-                    dpclip_layer_sqnorms(y.A, y.Zbar, y.has_bias, self.sq_layers[l], self._branch_ws[b], y.method)
+                    self._norm(l, self._branch_ws[b])
             join()
             dpclip_factors(self.sq_layers, C, self.clip, self.norms)
             fork()
             if t1_together:
                 with torch.cuda.stream(last):
-                    dpclip_t1_layers_clipped_grad_noise(self, C, sigma, seed, stream_id0, self._branch_ws[-1])
+                    dpclip_t1_layers_clipped_grad_noise(grp, C, sigma, seed, stream_id0, self._branch_ws[-1])
             # layers of one shape share a launch (first branch)
-            grouped = dpclip_same_shape_layers_clipped_grad_noise(self, C, sigma, seed, stream_id0, self._branch_ws[0])
-            rest = [(l, y) for l, y in rest if not grouped[l]]
-            for k, (l, y) in enumerate(rest):
+            grouped = dpclip_same_shape_layers_clipped_grad_noise(grp, C, sigma, seed, stream_id0, self._branch_ws[0])
+            rest = [l for l in rest if not grouped[l]]
+            for k, l in enumerate(rest):
                 b = (k + (1 if any(grouped) else 0)) % branches
                 with torch.cuda.stream(streams[b]):
-                    dpclip_clipped_grad_noise(y.A, y.Zbar, self.clip, self.gW[l], self.gb[l], sigma, C, seed,
-                                              stream_id0 + 2 * l, stream_id0 + 2 * l + 1, self._branch_ws[b])
+                    self._grad(l, self._branch_ws[b], C, sigma, seed, stream_id0)
             join()
         return graph
 
@@ -539,10 +557,11 @@ class ModelLayer:
     z_channel_major: bool = False
 
 
-class ModelPlan:
+class ModelPlan(StepPlan):
     """Buffers and the C descriptor array of a model with dense, element-wise and convolution layers.
-    Holds no arithmetic: `run` is one dpclip_model_step call.  gW[l] is (d_out, d_in) for dense and
-    convolution layers (d_in = C*kh*kw) and (d,) for element-wise layers; all live in `flat`."""
+    Holds no arithmetic: `run` is one dpclip_model_step call; `capture` with several branches records the same
+    path as per-layer entry-point calls (dense layers with the launches they share).  gW[l] is (d_out, d_in)
+    for dense and convolution layers (d_in = C*kh*kw) and (d,) for element-wise layers; all live in `flat`."""
 
     def __init__(self, layers: Sequence[ModelLayer], device=None):
         self.layers = list(layers)
@@ -601,6 +620,49 @@ class ModelPlan:
 
     def run(self, C: float, sigma: float, seed: int, stream_id0: int = 0, stream=None) -> None:
         dpclip_model_step(self, C, sigma, seed, stream_id0, stream)
+
+    def _grouping(self):
+        # dense descriptors at their positions in the model; the other kinds as T = 0 entries, which none of
+        # the several-layers-per-launch entry points takes
+        if not hasattr(self, "_dense"):
+            arr = (_CLayer * self.L)()
+            for l, y in enumerate(self.layers):
+                if y.kind == DPCLIP_KIND_DENSE:
+                    arr[l] = self._c[l].layer
+            self._dense = SimpleNamespace(_c=arr, L=self.L, B=self.B, dtype_code=self.dtype_code,
+                                          sq_layers=self.sq_layers, clip=self.clip, norms=self.norms,
+                                          workspace=self.workspace)
+        return self._dense
+
+    def _is_t1(self, l: int) -> bool:
+        y = self.layers[l]
+        return y.kind == DPCLIP_KIND_DENSE and y.A.shape[1] == 1
+
+    def _norm(self, l: int, ws: torch.Tensor) -> None:
+        y = self.layers[l]
+        if y.kind == DPCLIP_KIND_ELEMENTWISE:
+            dpclip_elementwise_sqnorms(y.A, y.Zbar, y.has_bias, self.sq_layers[l])
+        elif y.kind == DPCLIP_KIND_CONV:
+            kh, kw, stride, pad = y.conv
+            dpclip_conv_sqnorms(y.A, y.Zbar, kh, kw, stride, pad, y.has_bias, self.sq_layers[l], y.z_channel_major, ws)
+        else:
+            dpclip_layer_sqnorms(y.A, y.Zbar, y.has_bias, self.sq_layers[l], ws, y.method)
+
+    def _grad(self, l: int, ws: torch.Tensor, C: float, sigma: float, seed: int, stream_id0: int) -> None:
+        y = self.layers[l]
+        if y.kind == DPCLIP_KIND_DENSE:
+            dpclip_clipped_grad_noise(y.A, y.Zbar, self.clip, self.gW[l], self.gb[l], sigma, C, seed,
+                                      stream_id0 + 2 * l, stream_id0 + 2 * l + 1, ws)
+            return
+        if y.kind == DPCLIP_KIND_ELEMENTWISE:
+            dpclip_elementwise_clipped_grad(y.A, y.Zbar, self.clip, self.gW[l], self.gb[l])
+        else:
+            kh, kw, stride, pad = y.conv
+            dpclip_conv_clipped_grad(y.A, y.Zbar, kh, kw, stride, pad, self.clip, self.gW[l], self.gb[l],
+                                     y.z_channel_major, ws)
+        dpclip_add_noise(self.gW[l], sigma, C, seed, stream_id0 + 2 * l)
+        if self.gb[l] is not None:
+            dpclip_add_noise(self.gb[l], sigma, C, seed, stream_id0 + 2 * l + 1)
 
 
 def dpclip_model_workspace_bytes(plan: ModelPlan) -> int:

@@ -355,6 +355,16 @@ def test_model_step_mixed_layer_kinds(dp, dtype):
                 assert rel_fro(plan.gb[l].cpu().numpy(), eb) <= tol["grad"], (sg, l)
             else:
                 assert plan.gb[l] is None
+    # the same path recorded as per-layer calls on three streams
+    eager = [t.clone() for t in plan.gW] + [plan.clip.clone()]
+    graph = plan.capture(C, sigma, seed, sid0, branches=3)
+    plan.flat.fill_(float("nan")); plan.clip.fill_(float("nan"))
+    graph.replay(); graph.replay()
+    torch.cuda.synchronize()
+    assert dp.dpclip_read_status(plan.workspace) == 0
+    assert np.allclose(plan.clip.cpu().numpy(), eager[-1].cpu().numpy(), rtol=2e-6, atol=0)
+    for l in range(plan.L):
+        assert rel_fro(plan.gW[l].cpu().numpy(), eager[l].cpu().numpy()) <= 2e-6, l
     # a model of dense layers only is dpclip_step
     dense = [dp.ModelLayer(dp.DPCLIP_KIND_DENSE, to_device(As, dtype), to_device(Zs, dtype), True),
              dp.ModelLayer(dp.DPCLIP_KIND_DENSE, to_device(A1, dtype), to_device(Z1, dtype), False)]
