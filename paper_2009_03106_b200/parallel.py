@@ -20,10 +20,11 @@ def sharded_step(plan, C: float, sigma: float, seed: int, stream_id0: int = 0, g
     if ops is None:
         from . import binding as ops
     whole = getattr(ops, "dpclip_step", None)
+    mixed = any(getattr(y, "kind", 0) != 0 for y in plan.layers)      # LayerNorm / feature-map convolution layers
     if whole is not None:
         # norms -> factors -> clipped sums of this rank's examples in one library call (sigma = 0: the noise
         # belongs after the reduction); all-T=1 models take the one-launch fused kernel this way
-        whole(plan, C, 0.0, seed, stream_id0)
+        (ops.dpclip_model_step if mixed else whole)(plan, C, 0.0, seed, stream_id0)
     else:
         for l, y in enumerate(plan.layers):
             ops.dpclip_layer_sqnorms(y.A, y.Zbar, y.has_bias, plan.sq_layers[l], plan.workspace, y.method)
@@ -33,7 +34,7 @@ def sharded_step(plan, C: float, sigma: float, seed: int, stream_id0: int = 0, g
     if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
         dist.all_reduce(plan.flat, op=dist.ReduceOp.SUM, group=group)
     all_noise = getattr(ops, "dpclip_step_noise", None)
-    if all_noise is not None:
+    if all_noise is not None and not mixed:
         all_noise(plan, C, sigma, seed, stream_id0)               # every tensor's noise in one launch
         return
     for l in range(len(plan.layers)):

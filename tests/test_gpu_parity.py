@@ -365,6 +365,13 @@ def test_model_step_mixed_layer_kinds(dp, dtype):
     assert np.allclose(plan.clip.cpu().numpy(), eager[-1].cpu().numpy(), rtol=2e-6, atol=0)
     for l in range(plan.L):
         assert rel_fro(plan.gW[l].cpu().numpy(), eager[l].cpu().numpy()) <= 2e-6, l
+    # the data-parallel wrapper on one rank: the model step without noise, then the noise per tensor
+    from paper_2009_03106_b200 import parallel
+    plan.flat.fill_(float("nan"))
+    parallel.sharded_step(plan, C, sigma, seed, sid0)
+    torch.cuda.synchronize()
+    for l in range(plan.L):
+        assert rel_fro(plan.gW[l].cpu().numpy(), eager[l].cpu().numpy()) <= 2e-6, l
     # a model of dense layers only is dpclip_step
     dense = [dp.ModelLayer(dp.DPCLIP_KIND_DENSE, to_device(As, dtype), to_device(Zs, dtype), True),
              dp.ModelLayer(dp.DPCLIP_KIND_DENSE, to_device(A1, dtype), to_device(Z1, dtype), False)]
