@@ -481,6 +481,34 @@ def bench_model_block(torch, dp, steps, flush):
                 clipped_fraction=float((plan.clip < 1).float().mean().item()))
 
 
+def bench_model_cnn(torch, dp, dtype, steps, flush):
+    """The CNN of the cnn_32x32x3 workloads with its convolutions given by their feature maps and dL/dZ in the
+    channel-major layout it has in a framework (no patch matrices anywhere), dense 8192 -> 256 -> 10 on top:
+    ModelPlan, graph of per-layer calls on four streams.  B = 128."""
+    B = 128
+    convs = [(3, 32, 32, 32), (32, 16, 16, 64), (64, 8, 8, 128)]
+    layers = []
+    for i, (cin, H, W, cout) in enumerate(convs):
+        X, Z = workloads.conv_inputs(60 + i, B, cin, H, W, 3, 1, 1, cout, dtype, var_z=1.0 / B)
+        dZ = to_dev(Z, dtype, torch).transpose(1, 2).contiguous()
+        layers.append(dp.ModelLayer(dp.DPCLIP_KIND_CONV, to_dev(X, dtype, torch), dZ, True, conv=(3, 3, 1, 1),
+                                    z_channel_major=True))
+    rng = np.random.default_rng(63)
+    for d_in, d_out in ((8192, 256), (256, 10)):
+        A = np.maximum(rng.standard_normal((B, 1, d_in)), 0).astype(np.float32)
+        Z = (rng.standard_normal((B, 1, d_out)) / np.sqrt(B)).astype(np.float32)
+        layers.append(dp.ModelLayer(dp.DPCLIP_KIND_DENSE, to_dev(A, dtype, torch), to_dev(Z, dtype, torch), True))
+    plan = dp.ModelPlan(layers)
+    graph = plan.capture(1.0, 1.0, 1, branches=4)
+    ms = float(np.mean(time_steps(torch, graph.replay, steps, 3, flush)))
+    assert dp.dpclip_read_status(plan.workspace) == 0
+    es = 4 if dtype == "f32" else 2
+    nbytes = sum(2 * es * (y.A.numel() + y.Zbar.numel()) for y in plan.layers) + 4 * plan.flat.numel()
+    return dict(workload=f"cnn_feature_maps_b128_{dtype}", entry="ModelPlan.capture (per-layer calls, four streams)",
+                layers=plan.L, ms_per_step=ms, value=B / (ms * 1e-3), algorithmic_bytes=nbytes,
+                clipped_fraction=float((plan.clip < 1).float().mean().item()))
+
+
 def bench_conv_implicit(torch, dp, name, B, C, H, W, k, pad, d_out, dtype, steps, flush, peaks):
     """A convolution layer straight from its feature map (implicit im2col on the tensor cores), next to the same
     layer through the patch-matrix entry points.  Algorithmic bytes: feature map + Zbar once per kernel."""
@@ -762,6 +790,9 @@ def main():
                 others[r["workload"]] = r
             r = bench_model_block(torch, dp, min(args.steps, 20), flush)
             others[r["workload"]] = r
+            for cdt in ("f32", "bf16"):
+                r = bench_model_cnn(torch, dp, cdt, min(args.steps, 20), flush)
+                others[r["workload"]] = r
             for cdt in ("f32", "bf16"):
                 r = bench_conv_implicit(torch, dp, "conv2_implicit_im2col_b128_" + cdt, 128, 32, 16, 16, 3, 1, 64, cdt,
                                         min(args.steps, 20), flush, peaks)

@@ -246,6 +246,11 @@ int dpclip_conv_sqnorms(const void* X, const void* Zbar, int z_channel_major, in
 int dpclip_conv_clipped_grad(const void* X, const void* Zbar, int z_channel_major, int B, const dpclip_conv* geom,
                              int d_out, dpclip_dtype dtype, const float* clip, float* gW, long ldg, float* gb,
                              void* workspace, size_t workspace_bytes, void* stream);
+/* Workspace for the two calls above: dpclip_workspace_bytes() of the layer's patch-matrix shape, plus, for
+ * fp32 layers with dL/dZ channel-major that are large enough for the tensor cores, B*T*d_out*4 bytes for a
+ * [B][T][d_out] copy of dL/dZ (written by a transpose kernel at the start of each call; with less workspace
+ * the call still works and reads dL/dZ in place on the fp32-ALU kernel). */
+size_t dpclip_conv_workspace_bytes(int B, const dpclip_conv* geom, int d_out, dpclip_dtype dtype, int z_channel_major);
 
 /* The whole path over a model whose layers are not all dense products: Algorithm 1 with the per-layer
  * gradients of Sec. "Fully-connected", "Convolutional" and "LayerNorm" layers in one call.

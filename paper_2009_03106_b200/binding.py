@@ -74,6 +74,8 @@ def load_library():
     L.dpclip_conv_sqnorms.restype = _i
     L.dpclip_conv_clipped_grad.argtypes = [_vp, _vp, _i, _i, ctypes.POINTER(_CConv), _i, _i, _vp, _vp, _l, _vp, _vp, _sz, _vp]
     L.dpclip_conv_clipped_grad.restype = _i
+    L.dpclip_conv_workspace_bytes.argtypes = [_i, ctypes.POINTER(_CConv), _i, _i, _i]
+    L.dpclip_conv_workspace_bytes.restype = _sz
     L.dpclip_dp_sgd_step.argtypes = [_vp, _vp, _sz, _f, _f, _f, _u64, _u64, _f, _vp]
     L.dpclip_dp_sgd_step.restype = _i
     L.dpclip_dp_adam_step.argtypes = [_vp, _vp, _vp, _vp, _sz, _f, _f, _f, _u64, _u64, _f, _f, _f, _f, _i, _vp]
@@ -442,6 +444,12 @@ def _conv_args(X: torch.Tensor, Zbar: torch.Tensor, kh: int, kw: int, stride: in
         d_out = Zbar.shape[-1]
         assert Zbar.numel() == B * Ho * Wo * d_out
     return B, d_out, _CConv(C, H, W, kh, kw, stride, pad)
+
+
+def dpclip_conv_workspace_bytes(X: torch.Tensor, Zbar: torch.Tensor, kh: int, kw: int, stride: int, pad: int,
+                                z_channel_major: bool = False) -> int:
+    B, d_out, geom = _conv_args(X, Zbar, kh, kw, stride, pad, z_channel_major)
+    return load_library().dpclip_conv_workspace_bytes(B, ctypes.byref(geom), d_out, _dtype_code(X), int(z_channel_major))
 
 
 def dpclip_conv_sqnorms(X: torch.Tensor, Zbar: torch.Tensor, kh: int, kw: int, stride: int, pad: int, has_bias: bool,

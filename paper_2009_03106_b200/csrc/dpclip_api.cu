@@ -1360,6 +1360,68 @@ static int launch_conv_tc(const SimtParams& sp, const void* X, const void* Zbar,
 }
 }  // extern "C++"
 
+// fp32 dL/dZ in the channel-major layout [B][d_out][T]: the tf32 tensor-core kernel reads [row][feature]
+// tiles, so the tensor is rewritten once per call as [B][T][d_out] behind the partial-tile scratch when the
+// workspace has room for it (dpclip_conv_workspace_bytes); otherwise the fp32-ALU kernel reads it in place.
+// Returns the pointer to use and clears *channel_major when it did.
+static const void* conv_f32_rows_of_channel_major(const SimtParams& p, const void* Zbar, int* channel_major, int B, int T,
+                                                  dpclip_dtype dtype, void* workspace, size_t workspace_bytes,
+                                                  cudaStream_t st, int* rc) {
+    *rc = DPCLIP_OK;
+    if (dtype != DPCLIP_F32 || !*channel_major || !workspace || B > 65535) return Zbar;
+    { const char* env = getenv("DPCLIP_FORCE_SIMT"); if (env && env[0] == '1') return Zbar; }
+    if (p.d_out % 4 != 0 || p.kh > 255 || p.kw > 255) return Zbar;
+    if ((double)B * T * p.d_in * p.d_out < 32.0 * 1024 * 1024) return Zbar;           // stays on the fp32-ALU tiles
+    const size_t z_bytes = (size_t)B * T * p.d_out * 4;
+    if (workspace_bytes < (size_t)kHeaderBytes + kTcScratchBytes + z_bytes) return Zbar;
+    float* rows = reinterpret_cast<float*>(static_cast<char*>(workspace) + kHeaderBytes + kTcScratchBytes);
+    const dim3 grid(ceil_div(T, 32), ceil_div(p.d_out, 32), B);
+    channel_major_to_rows_kernel<<<grid, 256, 0, st>>>(static_cast<const float*>(Zbar), rows, p.d_out, T);
+    if (launch_status()) { *rc = DPCLIP_ERR_CUDA; return Zbar; }
+    *channel_major = 0;
+    return rows;
+}
+
+// fp32 first layers with at most 32 patch columns and 32 outputs: write the patch matrix out behind the scratch
+// areas above and hand it to the dense entry points (packed narrow tensor-core kernel).  Needs dL/dZ as rows.
+// Returns the patch matrix, or NULL when the layer does not qualify or the workspace has no room.
+static const float* conv_f32_narrow_patches(const SimtParams& p, const void* X, const void* z_rows, int z_cm, int B, int T,
+                                            dpclip_dtype dtype, int has_bias, void* workspace, size_t workspace_bytes,
+                                            cudaStream_t st, int* rc) {
+    *rc = DPCLIP_OK;
+    if (dtype != DPCLIP_F32 || z_cm || !workspace || p.d_out > 32 || p.d_in + (has_bias ? 1 : 0) > 32) return nullptr;
+    { const char* env = getenv("DPCLIP_FORCE_SIMT"); if (env && env[0] == '1') return nullptr; }
+    { const char* env = getenv("DPCLIP_NO_CONV_PATCHES"); if (env && env[0] == '1') return nullptr; }
+    if ((double)B * T * p.d_in * p.d_out < 32.0 * 1024 * 1024) return nullptr;
+    if (((long)T * p.d_in * 4) % 16 != 0 || ((long)T * p.d_out * 4) % 16 != 0 || !aligned_to(z_rows, 16)) return nullptr;
+    const size_t z_bytes = round_up((size_t)B * T * p.d_out * 4, 256), a_bytes = (size_t)B * T * p.d_in * 4;
+    if (workspace_bytes < (size_t)kHeaderBytes + kTcScratchBytes + z_bytes + a_bytes) return nullptr;
+    float* patches = reinterpret_cast<float*>(static_cast<char*>(workspace) + kHeaderBytes + kTcScratchBytes + z_bytes);
+    const long rows = (long)B * T;
+    if (rows > 0x7FFFFFFFL - 64) return nullptr;
+    im2col_f32_kernel<<<(unsigned)((rows + 63) / 64), 256, 0, st>>>(static_cast<const float*>(X), patches, (int)rows, T,
+                                                                    p.d_in, p.cC, p.cH, p.cW, p.kh, p.kw, p.stride, p.pad,
+                                                                    p.Wo);
+    if (launch_status()) { *rc = DPCLIP_ERR_CUDA; return nullptr; }
+    return patches;
+}
+
+size_t dpclip_conv_workspace_bytes(int B, const dpclip_conv* geom, int d_out, dpclip_dtype dtype, int z_channel_major) {
+    if (!geom || B <= 0 || d_out <= 0 || geom->stride <= 0) return kHeaderBytes;
+    const int Ho = (geom->H + 2 * geom->pad - geom->kh) / geom->stride + 1;
+    const int Wo = (geom->W + 2 * geom->pad - geom->kw) / geom->stride + 1;
+    if (Ho <= 0 || Wo <= 0) return kHeaderBytes;
+    const int T = Ho * Wo;
+    size_t w = dpclip_workspace_bytes(B, T, geom->C * geom->kh * geom->kw, d_out, dtype, DPCLIP_AUTO);
+    if (dtype == DPCLIP_F32 && w >= (size_t)kHeaderBytes + kTcScratchBytes) {
+        const int d_in = geom->C * geom->kh * geom->kw;
+        const bool narrow = d_out <= 32 && d_in + 1 <= 32;
+        if (z_channel_major || narrow) w += round_up((size_t)B * T * d_out * 4, 256);   // the row-major copy of dL/dZ
+        if (narrow) w += (size_t)B * T * d_in * 4;                                       // the patch matrix
+    }
+    return w;
+}
+
 int dpclip_conv_sqnorms(const void* X, const void* Zbar, int z_channel_major, int B, const dpclip_conv* geom,
                         int d_out, dpclip_dtype dtype, int has_bias, float* sq_layer, void* workspace,
                         size_t workspace_bytes, void* stream) {
@@ -1374,8 +1436,16 @@ int dpclip_conv_sqnorms(const void* X, const void* Zbar, int z_channel_major, in
     if (conv_tc_ok(p, X, Zbar, z_channel_major, B, T, dtype, workspace, workspace_bytes))
         return launch_conv_tc<false>(p, X, Zbar, B, T, has_bias, nullptr, sq_layer, nullptr, 0, nullptr, workspace,
                                      workspace_bytes, st);
-    if (conv_tf32_ok(p, X, Zbar, z_channel_major, B, T, dtype, workspace, workspace_bytes, &cg))
-        return launch_zta_tf32(nullptr, p.d_in, Zbar, d_out, B, T, p.d_in, d_out, true, has_bias, nullptr, nullptr, 0,
+    int z_cm = z_channel_major;
+    const void* z_rows = conv_f32_rows_of_channel_major(p, Zbar, &z_cm, B, T, dtype, workspace, workspace_bytes, st, &rc);
+    if (rc) return rc;
+    if (const float* patches = conv_f32_narrow_patches(p, X, z_rows, z_cm, B, T, dtype, has_bias, workspace, workspace_bytes,
+                                                       st, &rc))
+        return dpclip_layer_sqnorms(patches, p.d_in, z_rows, d_out, B, T, p.d_in, d_out, dtype, has_bias, DPCLIP_AUTO,
+                                    sq_layer, workspace, (size_t)kHeaderBytes + kTcScratchBytes, stream);
+    if (rc) return rc;
+    if (conv_tf32_ok(p, X, z_rows, z_cm, B, T, dtype, workspace, workspace_bytes, &cg))
+        return launch_zta_tf32(nullptr, p.d_in, z_rows, d_out, B, T, p.d_in, d_out, true, has_bias, nullptr, nullptr, 0,
                                nullptr, sq_layer, workspace, workspace_bytes, nullptr, nullptr, st, &cg);
     const int n_tiles = p.tiles_m * p.tiles_n;
     int split = ceil_div(2 * kNumSMs, B);
@@ -1405,9 +1475,17 @@ int dpclip_conv_clipped_grad(const void* X, const void* Zbar, int z_channel_majo
         rc = launch_conv_tc<true>(p, X, Zbar, B, T, gb != nullptr, clip, nullptr, gW, ldg, gb, workspace, workspace_bytes, st);
         if (rc <= 0) return rc;
     }
-    if (conv_tf32_ok(p, X, Zbar, z_channel_major, B, T, dtype, workspace, workspace_bytes, &cg) &&
+    int z_cm = z_channel_major;
+    const void* z_rows = conv_f32_rows_of_channel_major(p, Zbar, &z_cm, B, T, dtype, workspace, workspace_bytes, st, &rc);
+    if (rc) return rc;
+    if (const float* patches = conv_f32_narrow_patches(p, X, z_rows, z_cm, B, T, dtype, gb != nullptr, workspace,
+                                                       workspace_bytes, st, &rc))
+        return dpclip_clipped_grad(patches, p.d_in, z_rows, d_out, B, T, p.d_in, d_out, dtype, clip, gW, ldg, gb, workspace,
+                                   (size_t)kHeaderBytes + kTcScratchBytes, stream);
+    if (rc) return rc;
+    if (conv_tf32_ok(p, X, z_rows, z_cm, B, T, dtype, workspace, workspace_bytes, &cg) &&
         workspace_bytes >= (size_t)kHeaderBytes + kTcScratchBytes)
-        return launch_zta_tf32(nullptr, p.d_in, Zbar, d_out, B, T, p.d_in, d_out, false, 0, clip, gW, ldg, gb, nullptr,
+        return launch_zta_tf32(nullptr, p.d_in, z_rows, d_out, B, T, p.d_in, d_out, false, 0, clip, gW, ldg, gb, nullptr,
                                workspace, workspace_bytes, nullptr, nullptr, st, &cg);
     const int n_tiles = p.tiles_m * p.tiles_n;
     const long rows = (long)B * T;
@@ -1705,12 +1783,6 @@ int dpclip_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, fl
                         workspace_bytes, stream);
 }
 
-static int conv_out_positions(const dpclip_conv& g) {
-    if (g.stride <= 0 || g.kh <= 0 || g.kw <= 0) return 0;
-    const int Ho = (g.H + 2 * g.pad - g.kh) / g.stride + 1, Wo = (g.W + 2 * g.pad - g.kw) / g.stride + 1;
-    return Ho > 0 && Wo > 0 ? Ho * Wo : 0;
-}
-
 size_t dpclip_model_workspace_bytes(const dpclip_model_layer* layers, int L, int B, dpclip_dtype dtype) {
     size_t ws = kHeaderBytes;
     if (!layers || L <= 0 || B <= 0) return ws;
@@ -1720,8 +1792,7 @@ size_t dpclip_model_workspace_bytes(const dpclip_model_layer* layers, int L, int
         if (layers[l].kind == DPCLIP_KIND_DENSE)
             w = dpclip_workspace_bytes(B, y.T, y.d_in, y.d_out, dtype, (dpclip_method)y.method);
         else if (layers[l].kind == DPCLIP_KIND_CONV)
-            w = dpclip_workspace_bytes(B, conv_out_positions(layers[l].conv),
-                                       layers[l].conv.C * layers[l].conv.kh * layers[l].conv.kw, y.d_out, dtype, DPCLIP_AUTO);
+            w = dpclip_conv_workspace_bytes(B, &layers[l].conv, y.d_out, dtype, layers[l].z_channel_major);
         if (w > ws) ws = w;
     }
     return ws;

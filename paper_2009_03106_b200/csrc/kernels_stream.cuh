@@ -255,4 +255,51 @@ noise_batch_kernel(const __grid_constant__ NoiseBatchParams p) {
     }
 }
 
+// Patch matrix of a convolution written out, [B*T][C*kh*kw] fp32 with columns in (c, ky, kx) order and zeros
+// for the padding (Sec. "Convolutional Layers": the unfolded input).  Only for first layers whose patch rows are
+// at most 32 columns: there the packed narrow tensor-core kernel on the patch matrix beats the implicit forms,
+// and the matrix is a few MB.  CTA = 64 rows; lane = patch column (its (c, ky, kx) worked out once), warp w takes
+// rows w, w + 8, ...: a warp writes one row's d_in consecutive floats, rows back to back.
+__global__ void __launch_bounds__(256)
+im2col_f32_kernel(const float* __restrict__ X, float* __restrict__ P, int rows, int T, int d_in, int C, int H, int W,
+                  int kh, int kw, int stride, int pad, int Wo) {
+    const int n = threadIdx.x & 31, w = threadIdx.x >> 5;
+    if (n >= d_in) return;
+    const int c = n / (kh * kw), r = n - c * kh * kw, ky = r / kw, kx = r - ky * kw;
+    const int row0 = blockIdx.x * 64;
+#pragma unroll 4
+    for (int i = 0; i < 8; ++i) {
+        const int row = row0 + w + 8 * i;
+        if (row >= rows) break;
+        const int b = row / T, t = row - b * T;
+        const int yo = t / Wo, xo = t - yo * Wo;
+        const int y = yo * stride - pad + ky, x = xo * stride - pad + kx;
+        float v = 0.f;
+        if (y >= 0 && y < H && x >= 0 && x < W) v = __ldg(X + (((size_t)b * C + c) * H + y) * W + x);
+        P[(size_t)row * d_in + n] = v;
+    }
+}
+
+// dL/dZ of a convolution as a framework holds it, [B][d_out][T] (channel-major), rewritten as [B][T][d_out]
+// for the kernels that read [row][feature] tiles: 32 x 32 tiles through shared memory, reads and writes
+// both 128-byte coalesced.  grid = (ceil(T / 32), ceil(d_out / 32), B), 256 threads.
+__global__ void __launch_bounds__(256)
+channel_major_to_rows_kernel(const float* __restrict__ src, float* __restrict__ dst, int d_out, int T) {
+    __shared__ float tile[32][33];
+    const size_t base = (size_t)blockIdx.z * d_out * T;
+    const int t0 = blockIdx.x * 32, m0 = blockIdx.y * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int m = m0 + ty + 8 * i, t = t0 + tx;
+        if (m < d_out && t < T) tile[ty + 8 * i][tx] = src[base + (size_t)m * T + t];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int t = t0 + ty + 8 * i, m = m0 + tx;
+        if (t < T && m < d_out) dst[base + (size_t)t * d_out + m] = tile[tx][ty + 8 * i];
+    }
+}
+
 }  // namespace dpclip

@@ -269,6 +269,8 @@ CONV_CASES = [  # B, C, H, W, k, pad, stride, d_out
     # kernel with a ragged d_out, a 32 x 32 map
     (5, 64, 8, 8, 3, 1, 1, 128), (160, 4, 8, 8, 3, 1, 1, 16), (3, 6, 10, 8, (3, 1), 0, 1, 24), (2, 8, 16, 16, 5, 2, 1, 40),
     (2, 3, 32, 32, 3, 1, 1, 32),
+    # a first layer (27 patch columns, 32 outputs) large enough for the explicit-patch-matrix route in fp32
+    (40, 3, 32, 32, 3, 1, 1, 32),
 ]
 
 
@@ -288,7 +290,14 @@ def test_conv_implicit_im2col(dp, case, dtype):
     refW, refb = oracle.clipped_grad(A, Z, clip)
     ws = _ws(dp)
     # with a workspace the library may take the tensor-core form; without one it stays on the fp32-ALU tiles
-    for cm, z, w in ((False, dZ, ws), (False, dZ, None), (True, dZcm, ws)):
+    # channel-major fp32 layers reach the tensor cores through a row-major copy of dL/dZ in the workspace when it
+    # has the room the conv query asks for
+    ws_cm = torch.empty(dp.dpclip_conv_workspace_bytes(dX, dZcm, kh, kw, stride, pad, True), dtype=torch.uint8, device="cuda")
+    dp.dpclip_workspace_init(ws_cm)
+    variants = [(False, dZ, ws), (False, dZ, None), (True, dZcm, ws)]
+    if ws_cm.numel() > ws.numel():
+        variants.append((True, dZcm, ws_cm))
+    for cm, z, w in variants:
         for has_bias in (True, False):
             ref = oracle.layer_sqnorms(A, Z, has_bias)
             sq = torch.full((B,), -1.0, device="cuda")
