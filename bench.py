@@ -518,7 +518,9 @@ def bench_conv_implicit(torch, dp, name, B, C, H, W, k, pad, d_out, dtype, steps
     T, d_in = Z.shape[1], C * k * k
     clip = torch.rand(B, device="cuda") * 0.9 + 0.1
     sq = torch.empty(B, device="cuda"); gW = torch.empty(d_out, d_in, device="cuda"); gb = torch.empty(d_out, device="cuda")
-    ws = torch.empty(dp.dpclip_workspace_bytes(B, T, d_in, d_out, dp.DPCLIP_BF16), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(max(dp.dpclip_workspace_bytes(B, T, d_in, d_out, dp.DPCLIP_BF16),
+                         dp.dpclip_conv_workspace_bytes(dX, dZ.transpose(1, 2).contiguous(), k, k, 1, pad, True)),
+                     dtype=torch.uint8, device="cuda")
     dp.dpclip_workspace_init(ws)
     es = 4 if dtype == "f32" else 2
     nbytes = (X.size + Z.size) * es
