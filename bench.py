@@ -481,6 +481,26 @@ def bench_model_block(torch, dp, steps, flush):
                 clipped_fraction=float((plan.clip < 1).float().mean().item()))
 
 
+def bench_per_layer(torch, dp, steps, flush):
+    """Per-layer clipping (every layer to C / sqrt(L)) over the layers of the sequence workload: one
+    dpclip_step_per_layer call replayed as a graph on one stream."""
+    w = workloads.seq("bf16")
+    data = workloads.generate(w, 0)
+    plan = dp.StepPlan([dp.Layer(to_dev(A, "bf16", torch), to_dev(Z, "bf16", torch), s.has_bias)
+                        for (A, Z), s in zip(data, w.layers)])
+    Cl = [w.C / np.sqrt(plan.L)] * plan.L
+    clip = torch.empty(plan.L, plan.B, device="cuda")
+    dp.dpclip_step_per_layer(plan, Cl, w.sigma, 1, clip_layers=clip)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        dp.dpclip_step_per_layer(plan, Cl, w.sigma, 1, clip_layers=clip)
+    ms = float(np.mean(time_steps(torch, graph.replay, steps, 3, flush)))
+    assert dp.dpclip_read_status(plan.workspace) == 0
+    return dict(workload="per_layer_clipping_" + w.name, entry="dpclip_step_per_layer", layers=plan.L, ms_per_step=ms,
+                value=w.B / (ms * 1e-3), clipped_fraction=float((clip < 1).float().mean().item()))
+
+
 def bench_model_cnn(torch, dp, dtype, steps, flush):
     """The CNN of the cnn_32x32x3 workloads with its convolutions given by their feature maps and dL/dZ in the
     channel-major layout it has in a framework (no patch matrices anywhere), dense 8192 -> 256 -> 10 on top:
@@ -791,6 +811,8 @@ def main():
                 r = bench_elementwise(torch, dp, *shape, min(args.steps, 20), flush, peaks)
                 others[r["workload"]] = r
             r = bench_model_block(torch, dp, min(args.steps, 20), flush)
+            others[r["workload"]] = r
+            r = bench_per_layer(torch, dp, min(args.steps, 20), flush)
             others[r["workload"]] = r
             for cdt in ("f32", "bf16"):
                 r = bench_model_cnn(torch, dp, cdt, min(args.steps, 20), flush)

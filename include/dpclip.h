@@ -252,6 +252,21 @@ int dpclip_conv_clipped_grad(const void* X, const void* Zbar, int z_channel_majo
  * the call still works and reads dL/dZ in place on the fp32-ALU kernel). */
 size_t dpclip_conv_workspace_bytes(int B, const dpclip_conv* geom, int d_out, dpclip_dtype dtype, int z_channel_major);
 
+/* Per-layer clipping: every layer's per-example gradient is clipped to its own threshold C_layer[l] (for
+ * instance C / sqrt(L), so that the concatenated gradient stays within C), the variant that per-layer norms
+ * make possible (Sec. "Related Work", per-layer clipping).  For each layer in turn: squared norms -> factors
+ * from that row alone -> clipped sum -> noise N(0, sigma^2 * sum_l C_layer[l]^2) on every coordinate (the
+ * sensitivity of the concatenated clipped gradient), streams stream_id0 + 2l / + 2l + 1 as in dpclip_step.
+ *   C_layer       host [L], each > 0
+ *   sq_layers     [L][B], clip_layers [L][B] (row l = layer l's factors), norms_layers [L][B] or NULL
+ * No layer waits for another layer's norm, and a layer's clipped sum follows its own norm pass while its
+ * inputs are still in L2.  Errors as for dpclip_step. */
+int dpclip_step_per_layer(const dpclip_layer* layers /* host */, int L, int B, dpclip_dtype dtype,
+                          const float* C_layer /* host */, float sigma,
+                          unsigned long long seed, unsigned long long stream_id0,
+                          float* sq_layers, float* clip_layers, float* norms_layers,
+                          void* workspace, size_t workspace_bytes, void* stream);
+
 /* The whole path over a model whose layers are not all dense products: Algorithm 1 with the per-layer
  * gradients of Sec. "Fully-connected", "Convolutional" and "LayerNorm" layers in one call.
  *   kind DPCLIP_KIND_DENSE       `layer` as in dpclip_step.

@@ -104,6 +104,9 @@ def load_library():
     L.dpclip_step_host.argtypes = [ctypes.POINTER(_CLayer), _i, _i, _i, _f, _f, _u64, _u64, _vp, _vp, _vp, _sz, _vp]
     L.dpclip_step_host_arena_bytes.argtypes = [ctypes.POINTER(_CLayer), _i, _i, _i]
     L.dpclip_step_host_arena_bytes.restype = _sz
+    L.dpclip_step_per_layer.argtypes = [ctypes.POINTER(_CLayer), _i, _i, _i, ctypes.POINTER(ctypes.c_float), _f, _u64, _u64,
+                                        _vp, _vp, _vp, _vp, _sz, _vp]
+    L.dpclip_step_per_layer.restype = _i
     L.dpclip_model_step.argtypes = [ctypes.POINTER(_CModelLayer), _i, _i, _i, _f, _f, _u64, _u64, _vp, _vp, _vp, _vp,
                                     _sz, _vp]
     L.dpclip_model_step.restype = _i
@@ -671,6 +674,24 @@ class ModelPlan(StepPlan):
         dpclip_add_noise(self.gW[l], sigma, C, seed, stream_id0 + 2 * l)
         if self.gb[l] is not None:
             dpclip_add_noise(self.gb[l], sigma, C, seed, stream_id0 + 2 * l + 1)
+
+
+def dpclip_step_per_layer(plan: StepPlan, C_layer: Sequence[float], sigma: float, seed: int, stream_id0: int = 0,
+                          clip_layers: Optional[torch.Tensor] = None, norms_layers: Optional[torch.Tensor] = None,
+                          stream=None) -> torch.Tensor:
+    """Per-layer clipping over the plan's (dense) layers; returns the (L, B) factors."""
+    assert len(C_layer) == plan.L
+    if clip_layers is None:
+        clip_layers = torch.empty((plan.L, plan.B), dtype=torch.float32, device=plan.sq_layers.device)
+    assert clip_layers.dtype == torch.float32 and clip_layers.shape == (plan.L, plan.B) and clip_layers.is_contiguous()
+    assert norms_layers is None or (norms_layers.dtype == torch.float32 and norms_layers.shape == (plan.L, plan.B)
+                                    and norms_layers.is_contiguous())
+    c = (ctypes.c_float * plan.L)(*[float(v) for v in C_layer])
+    _check("dpclip_step_per_layer", load_library().dpclip_step_per_layer(
+        plan._c, plan.L, plan.B, plan.dtype_code, c, sigma, seed, stream_id0, _ptr(plan.sq_layers), _ptr(clip_layers),
+        _ptr(norms_layers) if norms_layers is not None else None, _ptr(plan.workspace), plan.workspace.numel(),
+        _stream(stream)))
+    return clip_layers
 
 
 def dpclip_model_workspace_bytes(plan: ModelPlan) -> int:

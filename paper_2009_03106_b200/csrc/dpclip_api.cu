@@ -1783,6 +1783,51 @@ int dpclip_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, fl
                         workspace_bytes, stream);
 }
 
+int dpclip_step_per_layer(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, const float* C_layer,
+                          float sigma, unsigned long long seed, unsigned long long stream_id0, float* sq_layers,
+                          float* clip_layers, float* norms_layers, void* workspace, size_t workspace_bytes,
+                          void* stream) {
+    if (!layers || L <= 0 || B <= 0 || !C_layer || !sq_layers || !clip_layers) return DPCLIP_ERR_INVALID_ARG;
+    if (!(sigma >= 0.f)) return DPCLIP_ERR_INVALID_ARG;
+    if (dtype != DPCLIP_F32 && dtype != DPCLIP_BF16) return DPCLIP_ERR_INVALID_ARG;
+    double c2 = 0.0;
+    for (int l = 0; l < L; ++l) {
+        if (!(C_layer[l] > 0.f)) return DPCLIP_ERR_INVALID_ARG;
+        c2 += (double)C_layer[l] * C_layer[l];
+    }
+    const float C_total = (float)sqrt(c2);               // sensitivity of the concatenated clipped gradient
+    // Layer by layer, norm -> factors -> clipped sum back to back: no layer waits for another one's norm, and
+    // the clipped sum re-reads inputs its own norm pass has just pulled through L2.
+    for (int l = 0; l < L; ++l) {
+        const dpclip_layer& y = layers[l];
+        float* sq = sq_layers + (size_t)l * B;
+        float* clip = clip_layers + (size_t)l * B;
+        float* gb = y.has_bias ? y.gb : nullptr;
+        if (!y.gW || (y.has_bias && !gb)) return DPCLIP_ERR_INVALID_ARG;
+        if (y.ldg != y.d_in) return DPCLIP_ERR_UNSUPPORTED;            // noise indexes the dense tensor
+        int rc = dpclip_layer_sqnorms(y.A, y.lda, y.Zbar, y.ldz, B, y.T, y.d_in, y.d_out, dtype, y.has_bias,
+                                      (dpclip_method)y.method, sq, workspace, workspace_bytes, stream);
+        if (rc) return rc;
+        rc = dpclip_factors(sq, 1, B, B, C_layer[l], clip, norms_layers ? norms_layers + (size_t)l * B : nullptr, nullptr,
+                            stream);
+        if (rc) return rc;
+        NoiseSpec ns = {sigma * C_total, seed, stream_id0 + 2ull * l, stream_id0 + 2ull * l + 1};
+        bool noise_done = false;
+        rc = clipped_grad_impl(y.A, y.lda, y.Zbar, y.ldz, B, y.T, y.d_in, y.d_out, dtype, clip, y.gW, y.ldg, gb, workspace,
+                               workspace_bytes, &ns, &noise_done, (cudaStream_t)stream);
+        if (rc) return rc;
+        if (!noise_done) {
+            rc = dpclip_add_noise(y.gW, (size_t)y.d_out * y.d_in, sigma, C_total, seed, ns.sid_w, stream);
+            if (rc) return rc;
+            if (gb) {
+                rc = dpclip_add_noise(gb, (size_t)y.d_out, sigma, C_total, seed, ns.sid_b, stream);
+                if (rc) return rc;
+            }
+        }
+    }
+    return DPCLIP_OK;
+}
+
 size_t dpclip_model_workspace_bytes(const dpclip_model_layer* layers, int L, int B, dpclip_dtype dtype) {
     size_t ws = kHeaderBytes;
     if (!layers || L <= 0 || B <= 0) return ws;

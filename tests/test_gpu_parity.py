@@ -911,6 +911,38 @@ def test_per_layer_clipping_through_the_same_entry_points(dp):
     assert dp.dpclip_read_status(ws) == 0
 
 
+@pytest.mark.parametrize("which", ["seq_bf16", "mlp_f32"])
+def test_step_per_layer_clipping(dp, which):
+    """dpclip_step_per_layer: every layer clipped to its own threshold in one call; factors, clipped sums and
+    the noise N(0, sigma^2 sum_l C_l^2) equal the oracle's layer by layer."""
+    w = workloads.seq("bf16", B=6, T=24, d=64, d_ff=136) if which == "seq_bf16" else workloads.mlp_small()
+    layers = workloads.generate(w, 8)
+    L, sigma, seed, sid0 = len(layers), 0.9, 13, 2
+    sq_ref = [oracle.layer_sqnorms(A, Z, s.has_bias) for (A, Z), s in zip(layers, w.layers)]
+    # thresholds near each layer's median norm, so that both sides of every threshold occur
+    Cl = [float(np.median(np.sqrt(q))) for q in sq_ref]
+    C_total = float(np.sqrt(np.sum(np.square(np.array(Cl, np.float32).astype(np.float64)))))
+    plan = dp.StepPlan([dp.Layer(to_device(A, w.dtype), to_device(Z, w.dtype), s.has_bias)
+                        for (A, Z), s in zip(layers, w.layers)])
+    norms = torch.empty(L, w.B, device="cuda")
+    plan.flat.fill_(float("nan"))
+    clip = dp.dpclip_step_per_layer(plan, Cl, sigma, seed, sid0, norms_layers=norms)
+    torch.cuda.synchronize()
+    assert dp.dpclip_read_status(plan.workspace) == 0
+    tol = TOL[w.dtype]
+    for l, ((A, Z), s) in enumerate(zip(layers, w.layers)):
+        n_ref, c_ref = oracle.factors(sq_ref[l][None, :], np.float32(Cl[l]))
+        assert 0 < (c_ref < 1).sum() < w.B
+        assert max_rel(norms[l].cpu().numpy(), n_ref) <= tol["norm"]
+        check_saturation(clip[l].cpu().numpy(), n_ref, c_ref, Cl[l])
+        gW_ref, gb_ref = oracle.clipped_grad(A, Z, c_ref)
+        eW = oracle.add_noise(gW_ref.reshape(-1), sigma, C_total, seed, sid0 + 2 * l).reshape(gW_ref.shape)
+        assert rel_fro(plan.gW[l].cpu().numpy(), eW) <= tol["grad"], l
+        if s.has_bias:
+            eb = oracle.add_noise(gb_ref, sigma, C_total, seed, sid0 + 2 * l + 1)
+            assert rel_fro(plan.gb[l].cpu().numpy(), eb) <= tol["grad"], l
+
+
 def test_sharded_step_single_rank_equals_step(dp):
     """The data-parallel wrapper on one rank (no process group): whole-step call without noise, then the
     noise launches, must give what one dpclip_step call gives."""
