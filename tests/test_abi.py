@@ -81,3 +81,30 @@ def test_argument_errors_are_caught_before_any_launch(lib):
     assert n(fake, 8, -1.0, 1.0, 0, 0, None) == INVALID
     assert lib.dpclip_workspace_bytes(128, 256, 512, 512, 1, 0) >= 256
     assert lib.dpclip_pick_method(128, 1, 784, 256, 784, 256, 0) == 1
+
+
+def test_workspace_queries_without_a_gpu(lib):
+    """The workspace queries are host arithmetic: the fixed scratch for ordinary layers, room for one partial
+    tile per row slice for long bf16 layers whose 64 tiles leave SMs idle in one wave, and the copies of the
+    fp32 feature-map convolution routes."""
+    lib.dpclip_workspace_bytes.restype = ctypes.c_size_t
+    lib.dpclip_workspace_bytes.argtypes = [ctypes.c_int] * 6
+    floor = lib.dpclip_workspace_bytes(1, 1, 1, 1, 1, 0)
+    assert lib.dpclip_workspace_bytes(128, 256, 512, 2048, 1, 0) == floor           # 16 tiles x 9 slices = one wave
+    assert lib.dpclip_workspace_bytes(256, 128, 1024, 4096, 1, 0) == floor          # 64 tiles, too short to re-cut
+    long64 = lib.dpclip_workspace_bytes(256, 2048, 1024, 4096, 1, 0)
+    assert long64 == 256 + 64 * 9 * (256 * 256 * 4 + 256 * 4)                       # 9 slices per tile
+    assert lib.dpclip_workspace_bytes(32, 1, 784, 256, 0, 0) == 256                 # small fp32 layer: header only
+
+    class Conv(ctypes.Structure):
+        _fields_ = [(n, ctypes.c_int) for n in ("C", "H", "W", "kh", "kw", "stride", "pad")]
+    lib.dpclip_conv_workspace_bytes.restype = ctypes.c_size_t
+    lib.dpclip_conv_workspace_bytes.argtypes = [ctypes.c_int, ctypes.POINTER(Conv), ctypes.c_int, ctypes.c_int, ctypes.c_int]
+    g = Conv(32, 16, 16, 3, 3, 1, 1)
+    rows = lib.dpclip_conv_workspace_bytes(128, ctypes.byref(g), 64, 0, 0)
+    cm = lib.dpclip_conv_workspace_bytes(128, ctypes.byref(g), 64, 0, 1)
+    assert cm == rows + 128 * 256 * 64 * 4                                          # the [B][T][d_out] copy
+    assert lib.dpclip_conv_workspace_bytes(128, ctypes.byref(g), 64, 1, 1) == floor  # bf16 reads either layout
+    g1 = Conv(3, 32, 32, 3, 3, 1, 1)
+    first = lib.dpclip_conv_workspace_bytes(128, ctypes.byref(g1), 32, 0, 0)
+    assert first == rows + 128 * 1024 * 32 * 4 + 128 * 1024 * 27 * 4                # dL/dZ rows + the patch matrix
