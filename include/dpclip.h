@@ -3,8 +3,8 @@
  * one B200 (sm_100a), after Lee & Kifer, "Scaling up Differentially Private
  * Deep Learning with Fast Per-Example Gradient Clipping".
  *
- * Problem statement (paper, Sec. "algorithm": "all that is needed" per layer
- * is the gradient w.r.t. the pre-activations and the layer's input):
+ * Problem statement (paper, Sec. "algorithm": per layer the method needs only
+ * the gradient w.r.t. the pre-activations and the layer's input):
  *
  *   layer l, example i:  A_i   in R^{T x d_in}    layer input rows
  *                        Zb_i  in R^{T x d_out}   dLoss_i/dZ rows, as given (no hidden 1/tau)
@@ -25,7 +25,13 @@
  *   - `stream` is a cudaStream_t passed as void* (NULL = legacy default stream).
  *     Calls only enqueue work; they never synchronise the stream.
  *   - The caller owns every buffer, including the workspace.  The library
- *     allocates no device memory and keeps no state between calls.  A
+ *     allocates no device memory, and no result depends on an earlier call.
+ *     What the process keeps between calls is bookkeeping only: an atomic
+ *     launch counter (dpclip_launch_count), the path-switch mask read once
+ *     from the environment (dpclip_reload_path_switches), per-device kernel
+ *     attributes set at a kernel's first launch, and the device address of
+ *     dpclip_clipped_grad_noalloc's fixed array.  Entry points may be called
+ *     from several host threads.  A
  *     workspace holds scratch (partial tiles) and, in its header, a status
  *     word, the grid-barrier counter of the one-launch T = 1 step and the
  *     item counter of the Gram kernel for T = 256 (both return to zero by
@@ -91,7 +97,9 @@ int dpclip_layer_sqnorms(const void* A, long lda, const void* Zbar, long ldz,
                          dpclip_dtype dtype, int has_bias, dpclip_method method,
                          float* sq_layer, void* workspace, size_t workspace_bytes, void* stream);
 
-/* Cross-layer accumulate and clip factors:
+/* Cross-layer accumulate and clip factors (the norm of the whole per-example gradient is the root of
+ * the sum of the per-layer squared norms: text after Eq. "weighted_loss"; the factor is Eq.
+ * "per_example_weight", nu_i = min(1, c / ||g_i||), equal to the clip_c definition of Sec. "Preliminaries"):
  *   norms[i] = sqrt(sum_l sq_layers[l*ld_sq + i]),  clip[i] = 1 if norms[i] <= C else C / norms[i].
  * The stored factor is exactly 1.0f for an unclipped example (including a zero
  * norm).  norms and n_clipped may be NULL; n_clipped[0] receives the number
@@ -143,9 +151,18 @@ int dpclip_elementwise_clipped_grad(const void* Hbar, long ldh, const void* Zbar
  * q = j / 4; word w of the block maps to u = fma(float(w), 2^-32, 2^-33) in
  * (0,1]; Box-Muller on words (0,1) gives elements 4q (cos) and 4q+1 (sin),
  * words (2,3) give 4q+2 and 4q+3.  The result depends only on (seed,
- * stream_id, j): the library is stateless, and a (seed, stream_id) pair must
+ * stream_id, j): no generator state is kept, and a (seed, stream_id) pair must
  * not be reused for two tensors.  n == 0 is a no-op.  Errors: INVALID_ARG for
- * a null g with n > 0 or negative sigma or C. */
+ * a null g with n > 0 or negative sigma or C.
+ * Limitation: the draws are an fp32 approximation of N(0,1), not exact Gaussians.  u lies on a 2^-32
+ * grid with minimum 2^-33, so |xi| <= sqrt(2 ln 2^33) = 6.76 and every draw is one of finitely many
+ * values; the device's log2 / sqrt / sin / cos approximations put each draw within 1e-5 (absolute, in
+ * units of sigma * C) of the value the same u gives in double precision.  The privacy analysis of
+ * Algorithm 1 assumes exact Gaussians; the known floating-point caveat of the Gaussian mechanism applies
+ * and is not addressed here.
+ * Releasing a step: a bounded wait inside a kernel that ran out (DPCLIP_ERR_TIMEOUT in the workspace
+ * header) leaves that step's outputs undefined while the enqueueing call has long returned DPCLIP_OK, so
+ * check dpclip_read_status() before anything computed by a step leaves the process. */
 int dpclip_add_noise(float* g, size_t n, float sigma, float C,
                      unsigned long long seed, unsigned long long stream_id, void* stream);
 
@@ -176,7 +193,10 @@ int dpclip_clipped_grad_noise(const void* A, long lda, const void* Zbar, long ld
  * workspace.  Limits and rules:
  *   - the output, padded to 256 x 256 tiles, must be at most
  *     dpclip_noalloc_max_output_bytes() (8 MB, e.g. 1024 x 2048 fp32);
- *     larger layers return DPCLIP_ERR_WORKSPACE and nothing is launched;
+ *     larger layers return DPCLIP_ERR_WORKSPACE and nothing is launched.  The
+ *     row split over CTAs is clamped to what the array holds (one partial tile
+ *     per CTA): small outputs run as wide as dpclip_clipped_grad, an output at
+ *     the limit with a bias runs unsplit (one CTA per 256 x 256 tile, slower);
  *   - no device memory is allocated or freed by this call, on any path;
  *   - the first call on each device looks up the array's device address (that
  *     device must be current); make that first call outside any stream capture;
@@ -412,6 +432,10 @@ int dpclip_pick_method(int B, int T, int d_in, int d_out, long lda, long ldz, dp
 /* Number of kernels this library has launched in this process (a host-side
  * counter for benchmarks and tests; cudaMemset calls are not counted). */
 unsigned long long dpclip_launch_count(void);
+
+/* The DPCLIP_* environment switches that force a slower kernel form (for tests and measurements) are read
+ * once, at the first call that needs them.  This re-reads them. */
+void dpclip_reload_path_switches(void);
 
 const char* dpclip_status_string(int status);
 int dpclip_version(void);

@@ -122,6 +122,8 @@ def load_library():
     L.dpclip_version.argtypes = []
     L.dpclip_launch_count.argtypes = []
     L.dpclip_launch_count.restype = _u64
+    L.dpclip_reload_path_switches.argtypes = []
+    L.dpclip_reload_path_switches.restype = None
     for name in ("dpclip_layer_sqnorms", "dpclip_factors", "dpclip_clipped_grad", "dpclip_add_noise",
                  "dpclip_step", "dpclip_step_host", "dpclip_workspace_init", "dpclip_read_status",
                  "dpclip_pick_method", "dpclip_version"):
@@ -178,6 +180,11 @@ def dpclip_version() -> int:
 
 def dpclip_launch_count() -> int:
     return load_library().dpclip_launch_count()
+
+
+def dpclip_reload_path_switches() -> None:
+    """Re-read the DPCLIP_* test/measurement switches from the environment (they are read once otherwise)."""
+    load_library().dpclip_reload_path_switches()
 
 
 def dpclip_status_string(status: int) -> str:
@@ -753,7 +760,11 @@ class HostStep:
             self.h2d_bytes += y.A.numel() * y.A.element_size() + y.Zbar.numel() * y.Zbar.element_size()
             self.d2h_bytes += gW.numel() * 4 + (gb.numel() * 4 if gb is not None else 0)
         self.clip = self._out_flat[off:off + self.B * 4].view(torch.float32); off += up(self.B * 4)
-        self.norms = self._out_flat[off:off + self.B * 4].view(torch.float32); off += up(self.B * 4)
+        self.norms = self._out_flat[off:off + self.B * 4].view(torch.float32)
+        # the merged device-to-host copy ends with the last float of `norms`: what lies behind it is not the
+        # library's to write (the bytes up to the 256-byte boundary are kept as a guard band for the tests)
+        self._out_end = off + self.B * 4
+        self._out_flat[self._out_end:].fill_(0xA5)
         self.d2h_bytes += 8 * self.B
         nbytes = load_library().dpclip_step_host_arena_bytes(self._c, self.L, self.B, self.dtype_code)
         self.arena = torch.empty((nbytes,), dtype=torch.uint8, device=device)

@@ -18,6 +18,7 @@
 #include "kernels_elementwise.cuh"
 
 #include <stdlib.h>
+#include <atomic>
 
 using namespace dpclip;
 
@@ -27,12 +28,49 @@ inline size_t elt_size(dpclip_dtype dt) { return dt == DPCLIP_F32 ? 4 : 2; }
 inline bool aligned_to(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // Kernels launched by this library since it was loaded (observability only; never read by a kernel).
-unsigned long long g_launches = 0;
+std::atomic<unsigned long long> g_launches{0};
 constexpr int kGridCounterOffset = 64;   // workspace header: status word at 0, grid-barrier counter here
 constexpr int kWorkCounterOffset = 128;  // item counter of the dynamically scheduled Gram kernel (wraps to zero by itself)
 inline int launch_status() {
-    ++g_launches;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? DPCLIP_OK : DPCLIP_ERR_CUDA;
+}
+
+// Path switches for tests and measurements (not configuration): a bit mask read ONCE from the DPCLIP_*
+// environment variables, on the first call that asks, so that no entry point touches the environment on its
+// way to a launch.  dpclip_reload_path_switches() re-reads them (the tests flip a variable, reload, and
+// reload again afterwards).
+enum PathSwitch : unsigned {
+    SW_FORCE_SIMT = 1u << 0, SW_NO_NARROW = 1u << 1, SW_NO_NARROW_RING = 1u << 2, SW_NO_NARROW_TC = 1u << 3,
+    SW_NO_NARROW_PACK = 1u << 4, SW_NARROW_PACK_BF16 = 1u << 5, SW_NO_GRAM_Q2 = 1u << 6, SW_NO_T1_TF32 = 1u << 7,
+    SW_NO_FUSED_T1 = 1u << 8, SW_NO_GRAM_GROUP = 1u << 9, SW_NO_GRAD_GROUP = 1u << 10, SW_NO_CONV_TC = 1u << 11,
+    SW_NO_CONV_PATCHES = 1u << 12, SW_TILE_M1 = 1u << 13, SW_TILE_M2 = 1u << 14, SW_T1_TWO_LAUNCHES = 1u << 15,
+    SW_LOADED = 1u << 31
+};
+std::atomic<unsigned> g_path_switches{0};
+unsigned read_path_switches() {
+    static const struct { const char* name; unsigned bit; char on; } table[] = {
+        {"DPCLIP_FORCE_SIMT", SW_FORCE_SIMT, '1'}, {"DPCLIP_NO_NARROW", SW_NO_NARROW, '1'},
+        {"DPCLIP_NO_NARROW_RING", SW_NO_NARROW_RING, '1'}, {"DPCLIP_NO_NARROW_TC", SW_NO_NARROW_TC, '1'},
+        {"DPCLIP_NO_NARROW_PACK", SW_NO_NARROW_PACK, '1'}, {"DPCLIP_NARROW_PACK_BF16", SW_NARROW_PACK_BF16, '1'},
+        {"DPCLIP_NO_GRAM_Q2", SW_NO_GRAM_Q2, '1'}, {"DPCLIP_NO_T1_TF32", SW_NO_T1_TF32, '1'},
+        {"DPCLIP_NO_FUSED_T1", SW_NO_FUSED_T1, '1'}, {"DPCLIP_NO_GRAM_GROUP", SW_NO_GRAM_GROUP, '1'},
+        {"DPCLIP_NO_GRAD_GROUP", SW_NO_GRAD_GROUP, '1'}, {"DPCLIP_NO_CONV_TC", SW_NO_CONV_TC, '1'},
+        {"DPCLIP_NO_CONV_PATCHES", SW_NO_CONV_PATCHES, '1'}, {"DPCLIP_TILE_M", SW_TILE_M1, '1'},
+        {"DPCLIP_TILE_M", SW_TILE_M2, '2'}, {"DPCLIP_T1_ONE_LAUNCH", SW_T1_TWO_LAUNCHES, '0'},
+    };
+    unsigned v = SW_LOADED;
+    for (const auto& e : table) {
+        const char* env = getenv(e.name);
+        if (env && env[0] == e.on) v |= e.bit;
+    }
+    g_path_switches.store(v, std::memory_order_relaxed);
+    return v;
+}
+inline bool path_switch(unsigned bit) {
+    unsigned v = g_path_switches.load(std::memory_order_relaxed);
+    if (!(v & SW_LOADED)) v = read_path_switches();
+    return (v & bit) != 0;
 }
 
 int check_layer_args(const void* A, long lda, const void* Z, long ldz, int B, int T, int d_in, int d_out,
@@ -77,8 +115,7 @@ int launch_t1_norms(const void* A, long lda, const void* Z, long ldz, int B, int
 
 // narrow layers (d_in + bias <= 32, d_out <= 64, T > 1): streaming kernel with one lane per column
 inline bool narrow_layer(int T, int d_in, int d_out, int has_bias, long lda, long ldz) {
-    const char* env = getenv("DPCLIP_NO_NARROW");
-    if (env && env[0] == '1') return false;
+    if (path_switch(SW_NO_NARROW)) return false;
     // dense rows: a run of rows is then one contiguous run of memory, which is what the kernel streams
     return T > 1 && d_in + (has_bias ? 1 : 0) <= 32 && d_out <= 64 && lda == d_in && ldz == d_out;
 }
@@ -103,8 +140,7 @@ int launch_narrow_ring_inst(const NarrowParams& p, int grid, cudaStream_t st) {
 
 // fp32 with every 16-row chunk starting on a 16-byte boundary (in A and in Zb): the cp.async ring form
 inline bool narrow_ring_ok(const NarrowParams& p, dpclip_dtype dtype, bool grad) {
-    const char* env = getenv("DPCLIP_NO_NARROW_RING");
-    if (env && env[0] == '1') return false;
+    if (path_switch(SW_NO_NARROW_RING)) return false;
     if (dtype != DPCLIP_F32 || !aligned_to(p.A, 16) || !aligned_to(p.Z, 16)) return false;
     // chunk starts are multiples of 16 rows from the slice start: 16 * d * 4 bytes is always a multiple of 16;
     // the slice start itself is a multiple of 32 rows (GRAD) or of T rows (NORM)
@@ -116,8 +152,7 @@ inline bool narrow_ring_ok(const NarrowParams& p, dpclip_dtype dtype, bool grad)
 // items (examples, row slices) that start and end on 16-byte boundaries in both inputs, which the bulk copies
 // into shared memory ask for
 inline bool narrow_tc_ok(const NarrowParams& p, dpclip_dtype dtype, const int* status) {
-    const char* env = getenv("DPCLIP_NO_NARROW_TC");
-    if (env && env[0] == '1') return false;
+    if (path_switch(SW_NO_NARROW_TC)) return false;
     if (dtype != DPCLIP_BF16 || status == nullptr) return false;
     if (!aligned_to(p.A, 16) || !aligned_to(p.Z, 16)) return false;
     return ((long)p.T * p.d_in) % 8 == 0 && ((long)p.T * p.d_out) % 8 == 0;
@@ -144,16 +179,14 @@ int launch_narrow_tc(const NarrowParams& p, int grid, int n_items, int* status, 
 // Narrow layers with d_out <= 32 on the tensor cores, four row groups per instruction (either dtype): the same
 // conditions as narrow_tc_ok, on 16-byte multiples of the element size
 inline bool narrow_pack_ok(const NarrowParams& p, dpclip_dtype dtype, const int* status) {
-    const char* env = getenv("DPCLIP_NO_NARROW_TC");
-    if (env && env[0] == '1') return false;
-    { const char* e2 = getenv("DPCLIP_NO_NARROW_PACK"); if (e2 && e2[0] == '1') return false; }
+    if (path_switch(SW_NO_NARROW_TC)) return false;
+    if (path_switch(SW_NO_NARROW_PACK)) return false;
     if (status == nullptr || p.d_out > 32 || p.d_in + p.has_bias > 32) return false;
     if (dtype == DPCLIP_BF16) {
         // bf16 has few instructions to save (one per 16 rows) and pays for the extra pass through shared memory in
         // the epilogue: measured 16.4 / 18.0 us against 15.2 / 17.9 us for the unpacked kernel on the first
         // convolution of the CNN.  Kept selectable for measurements.
-        const char* e3 = getenv("DPCLIP_NARROW_PACK_BF16");
-        if (!(e3 && e3[0] == '1')) return false;
+        if (!path_switch(SW_NARROW_PACK_BF16)) return false;
     }
     if (!aligned_to(p.A, 16) || !aligned_to(p.Z, 16)) return false;
     const long es = elt_size(dtype);
@@ -341,8 +374,7 @@ bool make_map_bf16(CUtensorMap* map, const void* base, long rows, long cols, lon
 // TMA needs 16-byte aligned bases and row strides.
 inline bool tc_eligible(const void* A, long lda, const void* Z, long ldz, dpclip_dtype dtype) {
     if (dtype != DPCLIP_BF16) return false;
-    const char* env = getenv("DPCLIP_FORCE_SIMT");
-    if (env && env[0] == '1') return false;
+    if (path_switch(SW_FORCE_SIMT)) return false;
     return aligned_to(A, 16) && aligned_to(Z, 16) && lda % 8 == 0 && ldz % 8 == 0;
 }
 
@@ -369,7 +401,7 @@ inline bool gram_diag_only(int T) {
 //   1: other layers whose items all sit on the diagonal (stages of two tiles, six of them)
 //   2: the rest
 inline int gram_class(int T) {
-    { const char* env = getenv("DPCLIP_NO_GRAM_Q2"); if (env && env[0] == '1') return gram_diag_only(T) ? 1 : 2; }
+    if (path_switch(SW_NO_GRAM_Q2)) return gram_diag_only(T) ? 1 : 2;
     if (T == 2 * tc::gram::BM) return 0;
     return gram_diag_only(T) ? 1 : 2;
 }
@@ -596,9 +628,8 @@ int launch_zta_tc(const void* A, long lda, const void* Z, long ldz, int B, int T
     namespace z = tc::zta;
     const long R = (long)B * T;
     int mt = d_out > 128 ? 2 : 1;
-    const char* env = getenv("DPCLIP_TILE_M");
-    if (env && env[0] == '1') mt = 1;
-    if (env && env[0] == '2') mt = 2;
+    if (path_switch(SW_TILE_M1)) mt = 1;
+    if (path_switch(SW_TILE_M2)) mt = 2;
     const int bk = mt == 2 ? z::Cfg<2>::BK : z::Cfg<1>::BK;           // rows of a TMA box = rows of a stage
     z::Maps maps;
     if (!make_map_bf16(&maps.a[0], A, R, d_in, lda, 64, bk) || !make_map_bf16(&maps.z[0], Z, R, d_out, ldz, 64, bk))
@@ -674,8 +705,7 @@ int launch_zta_tc_group(const dpclip_layer* const* ls, const int* index, int n, 
 inline bool tf32_eligible(const void* A, long lda, const void* Z, long ldz, int B, int T, int d_in, int d_out,
                           dpclip_dtype dtype) {
     if (dtype != DPCLIP_F32) return false;
-    const char* env = getenv("DPCLIP_FORCE_SIMT");
-    if (env && env[0] == '1') return false;
+    if (path_switch(SW_FORCE_SIMT)) return false;
     if (!(aligned_to(A, 16) && aligned_to(Z, 16) && lda % 4 == 0 && ldz % 4 == 0)) return false;
     // worth it once there is real contraction work; tiny layers stay on the fp32-ALU kernels
     return (double)B * T * d_in * d_out >= 32.0 * 1024 * 1024;
@@ -806,7 +836,7 @@ int launch_fused_t1_tc(tc::f1::Params& q, bool one_launch, int grid, void* works
 int launch_fused_t1_tf32(const FusedT1Params& base, bool one_launch, dpclip_dtype dtype, void* workspace,
                          size_t workspace_bytes, cudaStream_t st) {
     namespace f = tc::f1;
-    { const char* env = getenv("DPCLIP_NO_T1_TF32"); if (env && env[0] == '1') return 1; }
+    if (path_switch(SW_NO_T1_TF32)) return 1;
     if (!workspace || workspace_bytes < kHeaderBytes) return 1;
     static_assert(sizeof(f::Params) <= 4096, "kernel parameter space");
     f::Params q;
@@ -873,8 +903,8 @@ int prepare_t1_group(T1Group& g, const dpclip_layer* layers, int L, int B, dpcli
                      bool mixed_only = true) {
     g.active = false;
     if (B > FUSED_MAX_B) return 0;
-    { const char* env = getenv("DPCLIP_NO_FUSED_T1"); if (env && env[0] == '1') return 0; }
-    { const char* env = getenv("DPCLIP_NO_T1_TF32"); if (env && env[0] == '1') return 0; }
+    if (path_switch(SW_NO_FUSED_T1)) return 0;
+    if (path_switch(SW_NO_T1_TF32)) return 0;
     memset(&g.p, 0, sizeof(g.p));
     int n = 0, tiles = 0, wide = 0;
     for (int l = 0; l < L; ++l) {
@@ -902,8 +932,7 @@ int try_fused_t1_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dty
                       unsigned long long seed, unsigned long long stream_id0, float* sq, float* clip,
                       float* norms, void* workspace, size_t workspace_bytes, cudaStream_t st) {
     if (L > FUSED_MAX_LAYERS || B > FUSED_MAX_B) return 1;
-    const char* env = getenv("DPCLIP_NO_FUSED_T1");
-    if (env && env[0] == '1') return 1;
+    if (path_switch(SW_NO_FUSED_T1)) return 1;
     FusedT1Params p;
     memset(&p, 0, sizeof(p));
     // fp32-ALU form: 64 x 64 tiles, several CTAs per SM hide the global-load latency of these short (K = B)
@@ -924,7 +953,7 @@ int try_fused_t1_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dty
     const int grid_g = tiles < 4 * kNumSMs ? tiles : 4 * kNumSMs;
     const int smem64 = FusedT1Cfg<64>::SMEM_BYTES;
     bool one = true;
-    { const char* env = getenv("DPCLIP_T1_ONE_LAUNCH"); if (env && env[0] == '0') one = false; }
+    if (path_switch(SW_T1_TWO_LAUNCHES)) one = false;
     if (one) {
         const int rc = launch_fused_t1_tf32(p, true, dtype, workspace, workspace_bytes, st);
         if (rc <= 0) return rc;
@@ -945,7 +974,8 @@ extern "C" {
 
 int dpclip_version(void) { return 100; }
 
-unsigned long long dpclip_launch_count(void) { return g_launches; }
+unsigned long long dpclip_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+void dpclip_reload_path_switches(void) { read_path_switches(); }
 
 #ifdef DPCLIP_TRACE
 int dpclip_trace_copy(unsigned long long* host) {
@@ -971,8 +1001,7 @@ int dpclip_pick_method(int B, int T, int d_in, int d_out, long lda, long ldz, dp
     if (T == 1) return DPCLIP_T1;
     // alignment of the base pointers is not known here; rows must be 16-byte multiples for TMA
     if (dtype == DPCLIP_BF16 && lda % 8 == 0 && ldz % 8 == 0) {
-        const char* env = getenv("DPCLIP_FORCE_SIMT");
-        if (!(env && env[0] == '1')) {
+        if (!path_switch(SW_FORCE_SIMT)) {
             const double gram = (double)T * (T + 1.0) * ((double)d_in + d_out);      // symmetric Gram blocks
             const double mat = 2.0 * T * (double)d_in * d_out;                       // one Zb_i^T A_i product
             return gram <= mat ? DPCLIP_GRAM : DPCLIP_MATERIALIZE;
@@ -982,8 +1011,7 @@ int dpclip_pick_method(int B, int T, int d_in, int d_out, long lda, long ldz, dp
     // enough and its rows are 16-byte multiples; narrow and small layers stay on the fp32 ALUs
     if (dtype == DPCLIP_F32 && lda % 4 == 0 && ldz % 4 == 0 && !narrow_layer(T, d_in, d_out, 1, lda, ldz) &&
         (double)B * T * d_in * d_out >= 32.0 * 1024 * 1024) {
-        const char* env = getenv("DPCLIP_FORCE_SIMT");
-        if (!(env && env[0] == '1')) return DPCLIP_MATERIALIZE;
+        if (!path_switch(SW_FORCE_SIMT)) return DPCLIP_MATERIALIZE;
     }
     return DPCLIP_SIMT;
 }
@@ -1079,7 +1107,7 @@ int dpclip_gram_layers_sqnorms(const dpclip_layer* layers, int L, int B, dpclip_
     if (!layers || L <= 0 || B <= 0 || !sq_layers) return DPCLIP_ERR_INVALID_ARG;
     if (taken) for (int l = 0; l < L; ++l) taken[l] = 0;
     if (dtype != DPCLIP_BF16 || !workspace || workspace_bytes < (size_t)kHeaderBytes) return DPCLIP_OK;
-    { const char* env = getenv("DPCLIP_NO_GRAM_GROUP"); if (env && env[0] == '1') return DPCLIP_OK; }
+    if (path_switch(SW_NO_GRAM_GROUP)) return DPCLIP_OK;
     namespace g = tc::gram;
     for (int cls = 0; cls < 3; ++cls) {                    // one launch per kernel class (see gram_class)
         GramLayer batch[g::MAX_LAYERS];
@@ -1121,7 +1149,7 @@ int dpclip_same_shape_layers_clipped_grad_noise(const dpclip_layer* layers, int 
     if (!(C >= 0.f) || !(sigma >= 0.f)) return DPCLIP_ERR_INVALID_ARG;
     if (taken) for (int l = 0; l < L; ++l) taken[l] = 0;
     if (dtype != DPCLIP_BF16 || !workspace || workspace_bytes < (size_t)kHeaderBytes) return DPCLIP_OK;
-    { const char* env = getenv("DPCLIP_NO_GRAD_GROUP"); if (env && env[0] == '1') return DPCLIP_OK; }
+    if (path_switch(SW_NO_GRAD_GROUP)) return DPCLIP_OK;
     namespace z = tc::zta;
     constexpr int kMaxTracked = 256;
     if (L > kMaxTracked) return DPCLIP_OK;
@@ -1273,7 +1301,7 @@ static int conv_setup(SimtParams& p, const void* X, const void* Zbar, int z_chan
 // fp32, dL/dZ as [B][T][d_out] with 16-byte rows, enough work: the tensor-core kernel with the A operand gathered
 static bool conv_tf32_ok(const SimtParams& p, const void* X, const void* Zbar, int z_channel_major, int B, int T,
                          dpclip_dtype dtype, const void* workspace, size_t workspace_bytes, tc::ConvGather* cg) {
-    { const char* env = getenv("DPCLIP_FORCE_SIMT"); if (env && env[0] == '1') return false; }
+    if (path_switch(SW_FORCE_SIMT)) return false;
     if (dtype != DPCLIP_F32 || z_channel_major || !workspace || workspace_bytes < (size_t)kHeaderBytes) return false;
     if (!aligned_to(Zbar, 16) || p.d_out % 4 != 0 || p.kh > 255 || p.kw > 255) return false;
     if ((double)B * T * p.d_in * p.d_out < 32.0 * 1024 * 1024) return false;
@@ -1286,8 +1314,8 @@ static bool conv_tf32_ok(const SimtParams& p, const void* X, const void* Zbar, i
 // bf16 convolution layers on the tensor cores (implicit im2col): see kernels_conv_tc.cuh for the restrictions
 static bool conv_tc_ok(const SimtParams& p, const void* X, const void* Zbar, int z_channel_major, int B, int T,
                        dpclip_dtype dtype, const void* workspace, size_t workspace_bytes) {
-    { const char* env = getenv("DPCLIP_FORCE_SIMT"); if (env && env[0] == '1') return false; }
-    { const char* env = getenv("DPCLIP_NO_CONV_TC"); if (env && env[0] == '1') return false; }
+    if (path_switch(SW_FORCE_SIMT)) return false;
+    if (path_switch(SW_NO_CONV_TC)) return false;
     if (dtype != DPCLIP_BF16 || !workspace || workspace_bytes < (size_t)kHeaderBytes) return false;
     if (p.stride != 1 || !(p.Wo == 8 || p.Wo == 16 || p.Wo == 32 || p.Wo == 64) || T % 64 != 0) return false;
     if (p.d_out % 8 != 0 || p.d_out > 128) return false;
@@ -1369,7 +1397,7 @@ static const void* conv_f32_rows_of_channel_major(const SimtParams& p, const voi
                                                   cudaStream_t st, int* rc) {
     *rc = DPCLIP_OK;
     if (dtype != DPCLIP_F32 || !*channel_major || !workspace || B > 65535) return Zbar;
-    { const char* env = getenv("DPCLIP_FORCE_SIMT"); if (env && env[0] == '1') return Zbar; }
+    if (path_switch(SW_FORCE_SIMT)) return Zbar;
     if (p.d_out % 4 != 0 || p.kh > 255 || p.kw > 255) return Zbar;
     if ((double)B * T * p.d_in * p.d_out < 32.0 * 1024 * 1024) return Zbar;           // stays on the fp32-ALU tiles
     const size_t z_bytes = (size_t)B * T * p.d_out * 4;
@@ -1390,8 +1418,8 @@ static const float* conv_f32_narrow_patches(const SimtParams& p, const void* X, 
                                             cudaStream_t st, int* rc) {
     *rc = DPCLIP_OK;
     if (dtype != DPCLIP_F32 || z_cm || !workspace || p.d_out > 32 || p.d_in + (has_bias ? 1 : 0) > 32) return nullptr;
-    { const char* env = getenv("DPCLIP_FORCE_SIMT"); if (env && env[0] == '1') return nullptr; }
-    { const char* env = getenv("DPCLIP_NO_CONV_PATCHES"); if (env && env[0] == '1') return nullptr; }
+    if (path_switch(SW_FORCE_SIMT)) return nullptr;
+    if (path_switch(SW_NO_CONV_PATCHES)) return nullptr;
     if ((double)B * T * p.d_in * p.d_out < 32.0 * 1024 * 1024) return nullptr;
     if (((long)T * p.d_in * 4) % 16 != 0 || ((long)T * p.d_out * 4) % 16 != 0 || !aligned_to(z_rows, 16)) return nullptr;
     const size_t z_bytes = round_up((size_t)B * T * p.d_out * 4, 256), a_bytes = (size_t)B * T * p.d_in * 4;
@@ -1923,7 +1951,9 @@ int dpclip_step_host(const dpclip_layer* layers, int L, int B, dpclip_dtype dtyp
         in_packed = in_packed && static_cast<const char*>(y.A) - h_in0 == static_cast<const char*>(dev[l].A) - in_begin &&
                     static_cast<const char*>(y.Zbar) - h_in0 == static_cast<const char*>(dev[l].Zbar) - in_begin;
     }
-    const size_t in_bytes = (size_t)(cur - in_begin);
+    // a merged copy ends where the last tensor really ends: the host buffer need not extend to the padded end
+    const size_t in_bytes = (size_t)(static_cast<const char*>(dev[L - 1].Zbar) - in_begin) +
+                            (size_t)B * layers[L - 1].T * layers[L - 1].d_out * es;
     char* out_begin = cur;
     bool out_packed = true;
     const char* h_out0 = reinterpret_cast<const char*>(layers[0].gW);
@@ -1940,7 +1970,7 @@ int dpclip_step_host(const dpclip_layer* layers, int L, int B, dpclip_dtype dtyp
     out_packed = out_packed && host_clip && host_norms &&
                  reinterpret_cast<const char*>(host_clip) - h_out0 == reinterpret_cast<const char*>(clip) - out_begin &&
                  reinterpret_cast<const char*>(host_norms) - h_out0 == reinterpret_cast<const char*>(norms) - out_begin;
-    const size_t out_bytes = (size_t)(cur - out_begin);
+    const size_t out_bytes = (size_t)(reinterpret_cast<const char*>(norms) - out_begin) + (size_t)B * 4;
 
     if (in_packed) {
         if (cudaMemcpyAsync(in_begin, h_in0, in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return DPCLIP_ERR_CUDA;
@@ -1992,16 +2022,18 @@ static __device__ __align__(256) unsigned char g_static_scratch[kHeaderBytes + k
 // In host code `g_static_scratch` is only a handle for the runtime, not a device address, so the
 // address is looked up once per device (with that device current) and remembered.
 static void* static_scratch_for_current_device(int* rc) {
-    static void* cached[64] = {nullptr};
+    // two host threads may make the first call on a device at once: both look the same address up,
+    // and the slot is published with an atomic store
+    static std::atomic<void*> cached[64];
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { *rc = DPCLIP_ERR_CUDA; return nullptr; }
-    if (!cached[dev]) {
-        void* ptr = nullptr;
+    void* ptr = cached[dev].load(std::memory_order_acquire);
+    if (!ptr) {
         if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) { *rc = DPCLIP_ERR_CUDA; return nullptr; }
-        cached[dev] = ptr;
+        cached[dev].store(ptr, std::memory_order_release);
     }
     *rc = DPCLIP_OK;
-    return cached[dev];
+    return ptr;
 }
 
 size_t dpclip_noalloc_max_output_bytes(void) { return kStaticScratchBytes / 2; }
@@ -2013,7 +2045,10 @@ int dpclip_clipped_grad_noalloc(const void* A, long lda, const void* Zbar, long 
     if (rc) return rc;
     if (!gW || ldg < d_in) return DPCLIP_ERR_INVALID_ARG;
     if (!aligned_to(gW, 4) || (gb && !aligned_to(gb, 4))) return DPCLIP_ERR_MISALIGNED;
-    // the scratch must hold at least two partial copies of the output, padded to 256 x 256 tiles
+    // The output, padded to 256 x 256 tiles, may take at most half of the array.  Without a bias that leaves
+    // room for two partial copies; a bias adds 1 KB per partial tile, so at the very limit only one copy fits
+    // and the row split is clamped to 1: every tile then has a single CTA that stores straight to gW (bias by
+    // red.add), which is correct but uses one SM per tile.
     const size_t padded = (size_t)ceil_div(d_out, 256) * 256 * ((size_t)ceil_div(d_in, 256) * 256) * 4;
     if (padded > dpclip_noalloc_max_output_bytes()) return DPCLIP_ERR_WORKSPACE;
     void* scratch = static_scratch_for_current_device(&rc);

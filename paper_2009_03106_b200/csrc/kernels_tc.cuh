@@ -19,7 +19,9 @@
 //     swizzled 64-column TMA boxes); a transform warpgroup applies the per-row
 //     factor f to the Zb tile in shared memory between the TMA and the MMA.
 //       GRAD mode: f = clip factor of the row's example; rows split over CTAs;
-//                  the epilogue adds the tile into gW (fp32 atomics).
+//                  the epilogue writes the CTA's partial tile to the workspace
+//                  (reduce_partials_kernel adds the tiles in a fixed order), or
+//                  straight to gW when a tile has a single row slice.
 //       NORM mode: rows = one example, f masks rows outside it; the epilogue
 //                  squares and sums the tile (Frobenius norm), so the
 //                  per-example gradient never leaves the SM.

@@ -25,3 +25,18 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture
+def path_switch(monkeypatch):
+    """Set one of the library's DPCLIP_* path switches for the duration of a test.  The library reads them
+    once, so it is told to re-read after the change and again after the variable has been restored."""
+    import paper_2009_03106_b200 as pkg
+
+    def set_switch(name, value):
+        monkeypatch.setenv(name, value)
+        pkg.dpclip_reload_path_switches()
+
+    yield set_switch
+    monkeypatch.undo()
+    pkg.dpclip_reload_path_switches()

@@ -104,7 +104,8 @@ def test_sequence_workload_full_step_factors(dp):
 
 
 @pytest.mark.parametrize("B,T,d_in,d_out", [(256, 16, 1024, 1024), (256, 128, 1024, 4096), (64, 2048, 1024, 1024),
-                                            (256, 512, 1024, 4096)])
+                                            (256, 512, 1024, 4096), (1024, 16, 4096, 1024), (1024, 512, 1024, 1024),
+                                            (256, 2048, 1024, 1024)])
 def test_sweep_points(dp, B, T, d_in, d_out):
     """Points of the Gram-vs-materialise sweep (both norm forms must agree with the oracle)."""
     spec = workloads.LayerSpec("dense", T, d_in, d_out, True, "normal")
@@ -138,6 +139,89 @@ def test_sweep_points(dp, B, T, d_in, d_out):
         assert rel_fro(gW2.cpu().numpy(), gW.cpu().numpy()) <= 1e-6
         assert rel_fro(gb2.cpu().numpy(), gb.cpu().numpy()) <= 1e-6
         assert dp.dpclip_read_status(ws2) == 0
+
+
+def _probe_whole_gradient(A, Z, clip, G, rng, tol, probes=4):
+    """Random bilinear probes u^T G v of a whole clipped sum against the definition (fp64).  For unit Gaussian
+    u, v: E[(u^T E v)^2] = |E|_F^2, so the root mean square over the probes estimates the Frobenius error."""
+    G = G.astype(np.float64)
+    errs = []
+    for _ in range(probes):
+        u = rng.standard_normal(G.shape[0]); v = rng.standard_normal(G.shape[1])
+        errs.append(u @ G @ v - _probe(A, Z, clip, u, v))
+    return float(np.sqrt(np.mean(np.square(errs)))), 3 * tol * float(np.linalg.norm(G))
+
+
+def _bias_definition(Z, clip):
+    """sum_i c_i sum_t zb_{i,t} from the definition, fp64."""
+    return np.einsum("i,itd->d", clip.astype(np.float64), Z.astype(np.float64))
+
+
+@pytest.mark.parametrize("form", ["one_call", "graph_of_one_call", "graph_four_streams"])
+def test_sequence_workload_full_step_gradients(dp, form):
+    """The whole step at B=128, T=256 in the launch configurations the benchmark times (the seven layers' norms
+    in one Gram launch, the four 512->512 clipped sums stacked in one launch, one reduce with per-layer noise
+    streams): EVERY released tensor is checked, weights by random bilinear probes with the step's own factors,
+    biases element by element.  sigma = 0, so the released tensors are the clipped sums themselves."""
+    w = workloads.seq("bf16")
+    layers = workloads.generate(w, seed=2)
+    hb = [s.has_bias for s in w.layers]
+    plan = dp.StepPlan([dp.Layer(to_device(A, "bf16"), to_device(Z, "bf16"), b) for (A, Z), b in zip(layers, hb)])
+    C = 170.0                                           # norms are around 170: both sides of the threshold occur
+    if form == "one_call":
+        plan.flat.fill_(float("nan"))
+        plan.run(C, 0.0, seed=0)
+    else:
+        graph = plan.capture(C, 0.0, seed=0, branches=1 if form == "graph_of_one_call" else 4)
+        plan.flat.fill_(float("nan")); plan.clip.fill_(float("nan"))
+        graph.replay()
+    torch.cuda.synchronize()
+    assert dp.dpclip_read_status(plan.workspace) == 0
+    clip = plan.clip.cpu().numpy()
+    assert 0 < (clip < 1).sum() < w.B
+    sample = np.array([5, 77, 126])
+    sq = np.stack([oracle.layer_sqnorms(A[sample], Z[sample], b) for (A, Z), b in zip(layers, hb)])
+    n_ref, c_ref = oracle.factors(sq, C)
+    assert max_rel(plan.norms.cpu().numpy()[sample], n_ref) <= TOL["bf16"]["norm"]
+    assert np.max(np.abs(clip[sample] - c_ref)) <= 5e-3
+    rng = np.random.default_rng(11)
+    for l, ((A, Z), spec) in enumerate(zip(layers, w.layers)):
+        G = plan.gW[l].cpu().numpy()
+        assert np.all(np.isfinite(G)), spec.name
+        err, bound = _probe_whole_gradient(A, Z, clip.astype(np.float64), G, rng, TOL["bf16"]["grad"])
+        assert err <= bound, (form, spec.name, err, bound)
+        if spec.has_bias:
+            assert rel_fro(plan.gb[l].cpu().numpy(), _bias_definition(Z, clip)) <= TOL["bf16"]["grad"], spec.name
+
+
+def test_same_shape_layers_launch_full_size_against_the_oracle(dp):
+    """The launch that carries the four 512->512 projections at B=128, T=256 (their d_out tiles stacked, 14 stages
+    per CTA, one reduce over all four with per-layer outputs), called directly with factors that are zero outside
+    five examples, so that the oracle can give every output element: tensor-by-tensor comparison."""
+    w = workloads.seq("bf16")
+    data = workloads.generate(w, seed=4)[:4]
+    specs = w.layers[:4]
+    plan = dp.StepPlan([dp.Layer(to_device(A, "bf16"), to_device(Z, "bf16"), s.has_bias) for (A, Z), s in zip(data, specs)])
+    sample = np.array([0, 31, 64, 99, 127])
+    clip = np.zeros(w.B, np.float32)
+    clip[sample] = [1.0, 0.75, 0.3, 0.011, 0.6]
+    plan.clip.copy_(torch.from_numpy(clip))
+    plan.flat.fill_(float("nan"))
+    taken = dp.dpclip_same_shape_layers_clipped_grad_noise(plan, 1.0, 0.0, seed=0)
+    torch.cuda.synchronize()
+    assert all(taken)
+    assert dp.dpclip_read_status(plan.workspace) == 0
+    for l, (A, Z) in enumerate(data):
+        refW, _ = oracle.clipped_grad(A[sample], Z[sample], clip[sample])
+        assert rel_fro(plan.gW[l].cpu().numpy(), refW) <= TOL["bf16"]["grad"], l
+    # with noise: the difference to the sigma = 0 result is the oracle's noise tensor of that layer's stream
+    pre = [g.clone() for g in plan.gW]
+    dp.dpclip_same_shape_layers_clipped_grad_noise(plan, 1.0, 0.8, seed=9, stream_id0=100)
+    torch.cuda.synchronize()
+    for l in range(4):
+        xi = oracle.normals(512 * 512, 9, 100 + 2 * l).reshape(512, 512)
+        got = (plan.gW[l] - pre[l]).cpu().numpy()
+        assert np.max(np.abs(got - 0.8 * xi)) <= 1e-5 * 0.8 + 1e-6 * float(pre[l].abs().max()), l
 
 
 def test_mlp_large_graph_replay_full_size(dp):

@@ -650,9 +650,9 @@ def test_step_mlp_large(dp, C):
     assert {0.1: frac > 0.9, 1.0: 0.3 < frac < 0.7, 10.0: frac < 0.1}[C]
 
 
-def test_step_mlp_per_layer_path(dp, monkeypatch):
+def test_step_mlp_per_layer_path(dp, path_switch):
     """The general per-layer path on an all-T=1 model (the fused two-launch path is switched off)."""
-    monkeypatch.setenv("DPCLIP_NO_FUSED_T1", "1")
+    path_switch("DPCLIP_NO_FUSED_T1", "1")
     w = workloads.mlp_large(C=1.0)
     layers = workloads.generate(w, 1)
     _check_step(dp, w, _calibrate(w, layers, 1, 1.0), 1.0, w.sigma, 1)
@@ -690,7 +690,7 @@ def test_step_mlp_tensor_core_edges(dp):
     _check_step(dp, big, _calibrate(big, layers, 6, big.C), big.C, big.sigma, 6)
 
 
-def test_step_mlp_bf16_tensor_core(dp, monkeypatch):
+def test_step_mlp_bf16_tensor_core(dp, path_switch):
     """Fused T=1 step on the tensor cores with bf16 inputs (one kind::f16 instruction per 16 rows, no low
     planes): the paper-shaped MLPs, ragged tiles with a bias-free layer and a thin head, more tiles than SMs,
     and the two-launch form."""
@@ -709,7 +709,7 @@ def test_step_mlp_bf16_tensor_core(dp, monkeypatch):
                               workloads.LayerSpec("fc2", 1, 1664, 12, True, "relu")), 1.0, 0.9, 1.0 / 48)
     layers = workloads.generate(big, 6)
     _check_step(dp, big, _calibrate(big, layers, 6, big.C), big.C, big.sigma, 6)
-    monkeypatch.setenv("DPCLIP_T1_ONE_LAUNCH", "0")
+    path_switch("DPCLIP_T1_ONE_LAUNCH", "0")
     layers = workloads.generate(edges, 7)
     _check_step(dp, edges, _calibrate(edges, layers, 7, edges.C), edges.C, edges.sigma, 7)
 
@@ -752,10 +752,10 @@ def test_narrow_layers_tensor_core(dp, B, T, d_in, d_out, has_bias, dtype):
     assert rel_fro(gW.cpu().numpy(), refW1) <= 2e-5
 
 
-def test_narrow_packed_kernel_bf16(dp, monkeypatch):
+def test_narrow_packed_kernel_bf16(dp, path_switch):
     """The four-groups-per-instruction kernel with bf16 operands (fp32 layers take it by default, bf16 layers
     only on request)."""
-    monkeypatch.setenv("DPCLIP_NARROW_PACK_BF16", "1")
+    path_switch("DPCLIP_NARROW_PACK_BF16", "1")
     B, T, d_in, d_out = 150, 136, 27, 32
     A, Z = workloads.random_layer(61, B, T, d_in, d_out, "bf16", scale_z=0.05)
     idx = np.array([0, 1, 74, 149])
@@ -768,10 +768,10 @@ def test_narrow_packed_kernel_bf16(dp, monkeypatch):
     assert rel_fro(gW.cpu().numpy(), refW) <= TOL["bf16"]["grad"] and rel_fro(gb.cpu().numpy(), refb) <= TOL["bf16"]["grad"]
 
 
-def test_narrow_layer_register_staged_form(dp, monkeypatch):
+def test_narrow_layer_register_staged_form(dp, path_switch):
     """fp32 narrow layers normally take the cp.async ring kernel; the register-staged kernel (what bf16 and
     unaligned layers use) must give the same norms and clipped sums on the same fp32 input."""
-    monkeypatch.setenv("DPCLIP_NO_NARROW_RING", "1")
+    path_switch("DPCLIP_NO_NARROW_RING", "1")
     B, T, d_in, d_out = 5, 200, 27, 32
     A, Z = workloads.random_layer(33, B, T, d_in, d_out, "f32", scale_z=0.05)
     ref = oracle.layer_sqnorms(A, Z, True)
@@ -784,9 +784,9 @@ def test_narrow_layer_register_staged_form(dp, monkeypatch):
     assert rel_fro(gW.cpu().numpy(), refW) <= TOL["f32"]["grad"] and rel_fro(gb.cpu().numpy(), refb) <= TOL["f32"]["grad"]
 
 
-def test_step_mlp_fp32_alu_kernel(dp, monkeypatch):
+def test_step_mlp_fp32_alu_kernel(dp, path_switch):
     """The fp32-ALU second launch of the fused step (what models the tensor-core launch rejects fall back to)."""
-    monkeypatch.setenv("DPCLIP_NO_T1_TF32", "1")
+    path_switch("DPCLIP_NO_T1_TF32", "1")
     w = workloads.mlp_small()
     layers = workloads.generate(w, 4)
     _check_step(dp, w, _calibrate(w, layers, 4, w.C), w.C, w.sigma, 4)
@@ -856,7 +856,7 @@ def test_gram_layers_in_one_launch(dp):
     assert dp.dpclip_gram_layers_sqnorms(lone) == [False]
 
 
-def test_step_same_shape_layers_share_launches(dp, monkeypatch):
+def test_step_same_shape_layers_share_launches(dp, path_switch):
     """Layers of one shape go through one clipped-sum launch (stacked d_out tiles, one set of partial tiles,
     one reduce with every layer's own noise streams): 256-row and 128-row tile forms, ragged d_out, layers
     with and without bias in one group, a group next to single layers; and the same model layer by layer."""
@@ -873,8 +873,8 @@ def test_step_same_shape_layers_share_launches(dp, monkeypatch):
     taken = dp.dpclip_same_shape_layers_clipped_grad_noise(plan, w.C, w.sigma, 3, 0)
     torch.cuda.synchronize()
     assert taken == [True, True, True, False, True, True, False]
-    monkeypatch.setenv("DPCLIP_NO_GRAD_GROUP", "1")
-    monkeypatch.setenv("DPCLIP_NO_GRAM_GROUP", "1")
+    path_switch("DPCLIP_NO_GRAD_GROUP", "1")
+    path_switch("DPCLIP_NO_GRAM_GROUP", "1")
     single = _run_step(dp, w, cal, w.C, w.sigma, 3)
     for l in range(len(layers)):
         a, b = plan.gW[l].cpu().numpy(), single.gW[l].cpu().numpy()
@@ -977,6 +977,10 @@ def test_step_host_matches_device_step(dp):
     hp.run(w.C, w.sigma, 3, 0)
     torch.cuda.synchronize()
     assert np.array_equal(hp.clip.numpy(), hs.clip.numpy()) and np.array_equal(hp.norms.numpy(), hs.norms.numpy())
+    # the merged copies stop at the last tensor's real end (B = 32: norms take 128 of their 256-byte slot):
+    # the guard band behind the results keeps its pattern
+    for h in (hs, hp):
+        assert h._out_end % 256 != 0 and bool((h._out_flat[h._out_end:] == 0xA5).all())
     for l in range(len(layers)):
         assert np.array_equal(hp.gW[l].numpy(), hs.gW[l].numpy())
         assert np.array_equal(hp.gb[l].numpy(), hs.gb[l].numpy())

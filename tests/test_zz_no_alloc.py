@@ -1,10 +1,11 @@
 """The workspace-free clipped sum (for callers that cannot give the library device memory) must
-return what dpclip_clipped_grad returns.  Collected last on purpose: a run that stops at the first
+return what dpclip_clipped_grad returns, and what the oracle returns.  Collected last on purpose: a run that stops at the first
 failure has then already run every other test."""
 import numpy as np
 import pytest
 import torch
 
+import oracle
 import workloads
 from util import TOL, rel_fro, to_device
 
@@ -29,6 +30,11 @@ def _both(dp, B, T, d_in, d_out, dtype, seed, with_bias=True):
     got_W = torch.full((d_out, d_in), 7.0, device="cuda"); got_b = torch.full((d_out,), 7.0, device="cuda") if with_bias else None
     dp.dpclip_clipped_grad_noalloc(dA, dZ, dc, got_W, got_b)
     torch.cuda.synchronize()
+    # the oracle's clipped sum of the same inputs: the new entry point is held to the path's own tolerance
+    want_W, want_b = oracle.clipped_grad(A, Z, clip)
+    assert rel_fro(got_W.cpu().numpy(), want_W) <= TOL[dtype]["grad"]
+    if with_bias:
+        assert rel_fro(got_b.cpu().numpy(), want_b) <= TOL[dtype]["grad"]
     return ref_W.cpu().numpy(), got_W.cpu().numpy(), (ref_b.cpu().numpy() if with_bias else None), \
         (got_b.cpu().numpy() if with_bias else None)
 
@@ -41,6 +47,16 @@ def test_no_alloc_entry_matches_workspace_entry_twice_in_a_row(dp):
         # same kernels, only the row split differs: agreement far inside the bf16 tolerance
         assert rel_fro(got_W, ref_W) <= 1e-5 and rel_fro(got_W, ref_W) <= TOL["bf16"]["grad"]
         assert rel_fro(got_b, ref_b) <= 1e-5
+
+
+def test_no_alloc_entry_at_the_size_limit_with_a_bias(dp):
+    # the largest output the entry point accepts (8 MB padded), with a bias: one partial copy no longer fits
+    # next to the bias sums, so the row split is clamped to 1 and every tile is stored by a single CTA
+    ref_W, got_W, ref_b, got_b = _both(dp, 3, 96, 2048, 1024, "bf16", 5)
+    assert rel_fro(got_W, ref_W) <= 1e-5 and rel_fro(got_b, ref_b) <= 1e-5
+    # and twice in a row on the same shape with other data
+    ref_W, got_W, ref_b, got_b = _both(dp, 3, 96, 2048, 1024, "bf16", 6)
+    assert rel_fro(got_W, ref_W) <= 1e-5 and rel_fro(got_b, ref_b) <= 1e-5
 
 
 def test_no_alloc_entry_on_the_fp32_path_and_limits(dp):
