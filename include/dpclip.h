@@ -239,6 +239,30 @@ int dpclip_step(const dpclip_layer* layers /* host */, int L, int B, dpclip_dtyp
                 float* sq_layers, float* clip, float* norms,
                 void* workspace, size_t workspace_bytes, void* stream);
 
+/* dpclip_step with the launches of a stage spread over several streams INSIDE the library (Algorithm 1
+ * fixes only the order norms -> factors -> clipped sums; within the norm stage and within the clipped-sum
+ * stage the layers are independent, so one layer's kernel can start on the SMs another layer's kernel has
+ * already left).  Same arguments and results as dpclip_step, bit for bit, except:
+ *   streams     host array of n_streams (1..8) distinct cudaStream_t.  streams[0] is the caller's stream:
+ *               the step waits for nothing but what is already enqueued there, and when the call returns
+ *               everything the step enqueued, on any stream, is ordered before whatever the caller enqueues
+ *               on streams[0] next.  The other streams are used only between the library's own fork
+ *               (event record on streams[0] + waits) and join (event records + waits on streams[0]); they
+ *               must not be capturing or busy with work that conflicts with the step's buffers.
+ *   workspaces  host array of n_streams distinct device buffers of `workspace_bytes` each (the size
+ *               dpclip_step wants), each initialised once with dpclip_workspace_init; launches on different
+ *               streams overlap, so they cannot share scratch.  Check every one with dpclip_read_status.
+ * The call creates and destroys a few CUDA events (no device memory).  It may be recorded into a CUDA
+ * graph by capturing streams[0]: the fork and join become graph dependencies, and the benchmark's step is
+ * exactly one such call.  n_streams == 1 is dpclip_step.  All-T=1 models take the one-launch step on
+ * streams[0] whatever n_streams is.  Errors as dpclip_step; INVALID_ARG for n_streams outside 1..8 or
+ * repeated streams / workspaces. */
+int dpclip_step_streams(const dpclip_layer* layers /* host */, int L, int B, dpclip_dtype dtype,
+                        float C, float sigma, unsigned long long seed, unsigned long long stream_id0,
+                        float* sq_layers, float* clip, float* norms,
+                        int n_streams, void* const* streams /* host */, void* const* workspaces /* host */,
+                        size_t workspace_bytes);
+
 /* Convolution layers given by their INPUT feature map (implicit im2col).  Algorithm 3 unfolds the input into
  * the patch matrix (kh * kw copies of every pixel) and reshapes dL/dZ to [tau, c_out, T]; here element
  * (row (i, t), column (c, ky, kx)) of that matrix is read straight from
@@ -316,6 +340,13 @@ int dpclip_model_step(const dpclip_model_layer* layers /* host */, int L, int B,
                       float* sq_layers, float* clip, float* norms,
                       void* workspace, size_t workspace_bytes, void* stream);
 size_t dpclip_model_workspace_bytes(const dpclip_model_layer* layers /* host */, int L, int B, dpclip_dtype dtype);
+/* dpclip_model_step over several streams: streams, workspaces and rules as for dpclip_step_streams, every
+ * workspace of dpclip_model_workspace_bytes() bytes. */
+int dpclip_model_step_streams(const dpclip_model_layer* layers /* host */, int L, int B, dpclip_dtype dtype,
+                              float C, float sigma, unsigned long long seed, unsigned long long stream_id0,
+                              float* sq_layers, float* clip, float* norms,
+                              int n_streams, void* const* streams /* host */, void* const* workspaces /* host */,
+                              size_t workspace_bytes);
 
 /* Parameter updates with the noise folded in (one pass over the parameters instead of a noise pass and
  * an optimiser pass).  gsum is the PRE-noise clipped sum of one tensor (run the step with sigma = 0);

@@ -9,7 +9,6 @@ from __future__ import annotations
 import ctypes
 import os
 from dataclasses import dataclass
-from types import SimpleNamespace
 from typing import List, Optional, Sequence
 
 import torch
@@ -101,6 +100,12 @@ def load_library():
     L.dpclip_elementwise_clipped_grad.argtypes = [_vp, _l, _vp, _l, _i, _i, _i, _i, _vp, _vp, _vp, _vp]
     L.dpclip_elementwise_clipped_grad.restype = _i
     L.dpclip_step.argtypes = [ctypes.POINTER(_CLayer), _i, _i, _i, _f, _f, _u64, _u64, _vp, _vp, _vp, _vp, _sz, _vp]
+    L.dpclip_step_streams.argtypes = [ctypes.POINTER(_CLayer), _i, _i, _i, _f, _f, _u64, _u64, _vp, _vp, _vp, _i,
+                                      ctypes.POINTER(_vp), ctypes.POINTER(_vp), _sz]
+    L.dpclip_step_streams.restype = _i
+    L.dpclip_model_step_streams.argtypes = [ctypes.POINTER(_CModelLayer), _i, _i, _i, _f, _f, _u64, _u64, _vp, _vp, _vp,
+                                            _i, ctypes.POINTER(_vp), ctypes.POINTER(_vp), _sz]
+    L.dpclip_model_step_streams.restype = _i
     L.dpclip_step_host.argtypes = [ctypes.POINTER(_CLayer), _i, _i, _i, _f, _f, _u64, _u64, _vp, _vp, _vp, _sz, _vp]
     L.dpclip_step_host_arena_bytes.argtypes = [ctypes.POINTER(_CLayer), _i, _i, _i]
     L.dpclip_step_host_arena_bytes.restype = _sz
@@ -357,89 +362,38 @@ class StepPlan:
     def run(self, C: float, sigma: float, seed: int, stream_id0: int = 0, stream=None) -> None:
         dpclip_step(self, C, sigma, seed, stream_id0, stream)
 
-    # what `capture` needs to know about a layer (ModelPlan answers differently for the other layer kinds)
-    def _grouping(self):
-        """The object the several-layers-per-launch entry points take (dense descriptors, one per layer)."""
-        return self
-
-    def _is_t1(self, l: int) -> bool:
-        return self.layers[l].A.shape[1] == 1
-
-    def _norm(self, l: int, ws: torch.Tensor) -> None:
-        y = self.layers[l]
-        dpclip_layer_sqnorms(y.A, y.Zbar, y.has_bias, self.sq_layers[l], ws, y.method)
-
-    def _grad(self, l: int, ws: torch.Tensor, C: float, sigma: float, seed: int, stream_id0: int) -> None:
-        y = self.layers[l]
-        dpclip_clipped_grad_noise(y.A, y.Zbar, self.clip, self.gW[l], self.gb[l], sigma, C, seed,
-                                  stream_id0 + 2 * l, stream_id0 + 2 * l + 1, ws)
-
-    def capture(self, C: float, sigma: float, seed: int, stream_id0: int = 0, branches: int = 1):
-        """Record one step into a CUDA graph (the launch-bound small workloads spend most of a step
-        in launch gaps).  Returns the graph; `graph.replay()` re-runs the same kernels on the same
-        buffers with the same (C, sigma, seed, stream ids).
-
-        branches = 1 records one dpclip_step call.  branches > 1 records the same path as per-layer
-        entry-point calls spread over that many streams (layers are independent within the norm
-        stage and within the clipped-sum stage), so the graph has parallel branches and one layer's
-        kernel starts on SMs the previous layer's kernel has already left.  Pure stream plumbing:
-        the arithmetic is the same kernels either way."""
-        self.run(C, sigma, seed, stream_id0)          # warm-up outside capture (function attributes, maps)
-        torch.cuda.synchronize()
-        graph = torch.cuda.CUDAGraph()
-        if branches <= 1:
-            with torch.cuda.graph(graph):
-                self.run(C, sigma, seed, stream_id0)
-            return graph
-        if not hasattr(self, "_branch_ws"):
+    def _branches(self, branches: int):
+        """Side streams and their workspaces for the several-streams entry points (allocated once)."""
+        if len(getattr(self, "_branch_ws", [])) < branches:
             self._branch_ws = [self.workspace] + [torch.empty_like(self.workspace) for _ in range(branches - 1)]
             for w in self._branch_ws[1:]:
                 dpclip_workspace_init(w)
             self._streams = [torch.cuda.Stream() for _ in range(branches - 1)]
             torch.cuda.synchronize()
+        return self._streams[:branches - 1], self._branch_ws[:branches]
+
+    def run_streams(self, C: float, sigma: float, seed: int, stream_id0: int = 0, branches: int = 4) -> None:
+        """One dpclip_step_streams call: the library spreads the launches of a stage over `branches` streams,
+        starting from and joining back into the current stream."""
+        side, ws = self._branches(branches)
+        dpclip_step_streams(self, C, sigma, seed, stream_id0, [torch.cuda.current_stream()] + side, ws)
+
+    def workspaces(self) -> List[torch.Tensor]:
+        """Every workspace the plan has used (their status words are checked separately)."""
+        return list(getattr(self, "_branch_ws", [self.workspace]))
+
+    def capture(self, C: float, sigma: float, seed: int, stream_id0: int = 0, branches: int = 1):
+        """Record one step into a CUDA graph (the launch-bound small workloads spend most of a step
+        in launch gaps).  Returns the graph; `graph.replay()` re-runs the same kernels on the same
+        buffers with the same (C, sigma, seed, stream ids).  The graph holds exactly ONE library call:
+        dpclip_step (branches = 1) or dpclip_step_streams (the fork/join over `branches` streams happens
+        inside the library and becomes the graph's parallel branches)."""
+        step = self.run if branches <= 1 else (lambda *a: self.run_streams(*a, branches=branches))
+        step(C, sigma, seed, stream_id0)               # warm-up outside capture (function attributes, maps)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph):
-            main = torch.cuda.current_stream()
-            streams = [main] + self._streams
-
-            def fork():
-                ev = torch.cuda.Event(); ev.record(main)
-                for s in streams[1:]:
-                    s.wait_event(ev)
-
-            def join():
-                for s in streams[1:]:
-                    ev = torch.cuda.Event(); ev.record(s); main.wait_event(ev)
-
-            # the T = 1 layers of a mixed model go together (one launch per stage) when the library takes them
-            grp = self._grouping()
-            t1_together = any(self._is_t1(l) for l in range(self.L)) and dpclip_t1_layers_supported(grp)
-            last = streams[-1]
-            fork()
-            # layers whose norms go by the Gram identity share one launch (on the first branch)
-            taken = dpclip_gram_layers_sqnorms(grp, self._branch_ws[0])
-            rest = [l for l in range(self.L) if not (t1_together and self._is_t1(l))]
-            if t1_together:
-                with torch.cuda.stream(last):
-                    dpclip_t1_layers_sqnorms(grp)
-            rest_norms = [l for l in rest if not taken[l]]
-            for k, l in enumerate(rest_norms):
-                b = (k + (1 if any(taken) else 0)) % branches
-                with torch.cuda.stream(streams[b]):
-                    self._norm(l, self._branch_ws[b])
-            join()
-            dpclip_factors(self.sq_layers, C, self.clip, self.norms)
-            fork()
-            if t1_together:
-                with torch.cuda.stream(last):
-                    dpclip_t1_layers_clipped_grad_noise(grp, C, sigma, seed, stream_id0, self._branch_ws[-1])
-            # layers of one shape share a launch (first branch)
-            grouped = dpclip_same_shape_layers_clipped_grad_noise(grp, C, sigma, seed, stream_id0, self._branch_ws[0])
-            rest = [l for l in rest if not grouped[l]]
-            for k, l in enumerate(rest):
-                b = (k + (1 if any(grouped) else 0)) % branches
-                with torch.cuda.stream(streams[b]):
-                    self._grad(l, self._branch_ws[b], C, sigma, seed, stream_id0)
-            join()
+            step(C, sigma, seed, stream_id0)
         return graph
 
 
@@ -556,6 +510,29 @@ def dpclip_step(plan: StepPlan, C: float, sigma: float, seed: int, stream_id0: i
         _ptr(plan.clip), _ptr(plan.norms), _ptr(plan.workspace), plan.workspace.numel(), _stream(stream)))
 
 
+def _stream_args(streams, workspaces):
+    n = len(streams)
+    assert n == len(workspaces) and all(w.numel() == workspaces[0].numel() for w in workspaces)
+    st = (_vp * n)(*[s.cuda_stream for s in streams])
+    ws = (_vp * n)(*[w.data_ptr() for w in workspaces])
+    return n, st, ws, workspaces[0].numel()
+
+
+def dpclip_step_streams(plan: StepPlan, C: float, sigma: float, seed: int, stream_id0: int, streams, workspaces) -> None:
+    """dpclip_step with the library forking over `streams` (torch streams; streams[0] = the caller's)."""
+    n, st, ws, nbytes = _stream_args(streams, workspaces)
+    _check("dpclip_step_streams", load_library().dpclip_step_streams(
+        plan._c, plan.L, plan.B, plan.dtype_code, C, sigma, seed, stream_id0, _ptr(plan.sq_layers), _ptr(plan.clip),
+        _ptr(plan.norms), n, st, ws, nbytes))
+
+
+def dpclip_model_step_streams(plan, C: float, sigma: float, seed: int, stream_id0: int, streams, workspaces) -> None:
+    n, st, ws, nbytes = _stream_args(streams, workspaces)
+    _check("dpclip_model_step_streams", load_library().dpclip_model_step_streams(
+        plan._c, plan.L, plan.B, plan.dtype_code, C, sigma, seed, stream_id0, _ptr(plan.sq_layers), _ptr(plan.clip),
+        _ptr(plan.norms), n, st, ws, nbytes))
+
+
 DPCLIP_KIND_DENSE, DPCLIP_KIND_ELEMENTWISE, DPCLIP_KIND_CONV = 0, 1, 2
 
 
@@ -577,8 +554,8 @@ class ModelLayer:
 
 class ModelPlan(StepPlan):
     """Buffers and the C descriptor array of a model with dense, element-wise and convolution layers.
-    Holds no arithmetic: `run` is one dpclip_model_step call; `capture` with several branches records the same
-    path as per-layer entry-point calls (dense layers with the launches they share).  gW[l] is (d_out, d_in)
+    Holds no arithmetic: `run` is one dpclip_model_step call, `run_streams` one dpclip_model_step_streams call
+    (which `capture` with several branches records).  gW[l] is (d_out, d_in)
     for dense and convolution layers (d_in = C*kh*kw) and (d,) for element-wise layers; all live in `flat`."""
 
     def __init__(self, layers: Sequence[ModelLayer], device=None):
@@ -639,48 +616,9 @@ class ModelPlan(StepPlan):
     def run(self, C: float, sigma: float, seed: int, stream_id0: int = 0, stream=None) -> None:
         dpclip_model_step(self, C, sigma, seed, stream_id0, stream)
 
-    def _grouping(self):
-        # dense descriptors at their positions in the model; the other kinds as T = 0 entries, which none of
-        # the several-layers-per-launch entry points takes
-        if not hasattr(self, "_dense"):
-            arr = (_CLayer * self.L)()
-            for l, y in enumerate(self.layers):
-                if y.kind == DPCLIP_KIND_DENSE:
-                    arr[l] = self._c[l].layer
-            self._dense = SimpleNamespace(_c=arr, L=self.L, B=self.B, dtype_code=self.dtype_code,
-                                          sq_layers=self.sq_layers, clip=self.clip, norms=self.norms,
-                                          workspace=self.workspace)
-        return self._dense
-
-    def _is_t1(self, l: int) -> bool:
-        y = self.layers[l]
-        return y.kind == DPCLIP_KIND_DENSE and y.A.shape[1] == 1
-
-    def _norm(self, l: int, ws: torch.Tensor) -> None:
-        y = self.layers[l]
-        if y.kind == DPCLIP_KIND_ELEMENTWISE:
-            dpclip_elementwise_sqnorms(y.A, y.Zbar, y.has_bias, self.sq_layers[l])
-        elif y.kind == DPCLIP_KIND_CONV:
-            kh, kw, stride, pad = y.conv
-            dpclip_conv_sqnorms(y.A, y.Zbar, kh, kw, stride, pad, y.has_bias, self.sq_layers[l], y.z_channel_major, ws)
-        else:
-            dpclip_layer_sqnorms(y.A, y.Zbar, y.has_bias, self.sq_layers[l], ws, y.method)
-
-    def _grad(self, l: int, ws: torch.Tensor, C: float, sigma: float, seed: int, stream_id0: int) -> None:
-        y = self.layers[l]
-        if y.kind == DPCLIP_KIND_DENSE:
-            dpclip_clipped_grad_noise(y.A, y.Zbar, self.clip, self.gW[l], self.gb[l], sigma, C, seed,
-                                      stream_id0 + 2 * l, stream_id0 + 2 * l + 1, ws)
-            return
-        if y.kind == DPCLIP_KIND_ELEMENTWISE:
-            dpclip_elementwise_clipped_grad(y.A, y.Zbar, self.clip, self.gW[l], self.gb[l])
-        else:
-            kh, kw, stride, pad = y.conv
-            dpclip_conv_clipped_grad(y.A, y.Zbar, kh, kw, stride, pad, self.clip, self.gW[l], self.gb[l],
-                                     y.z_channel_major, ws)
-        dpclip_add_noise(self.gW[l], sigma, C, seed, stream_id0 + 2 * l)
-        if self.gb[l] is not None:
-            dpclip_add_noise(self.gb[l], sigma, C, seed, stream_id0 + 2 * l + 1)
+    def run_streams(self, C: float, sigma: float, seed: int, stream_id0: int = 0, branches: int = 4) -> None:
+        side, ws = self._branches(branches)
+        dpclip_model_step_streams(self, C, sigma, seed, stream_id0, [torch.cuda.current_stream()] + side, ws)
 
 
 def dpclip_step_per_layer(plan: StepPlan, C_layer: Sequence[float], sigma: float, seed: int, stream_id0: int = 0,

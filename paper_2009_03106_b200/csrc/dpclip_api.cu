@@ -1715,66 +1715,124 @@ static int other_kind_clipped_grad_noise(const dpclip_model_layer& m, int B, dpc
     return rc;
 }
 
-// The path layer by layer (with the launches that several layers share).  `other`, when given, is the model's
-// own descriptor array: entries of a kind other than dense have a placeholder with T = 0 in `layers`, which
-// every grouping rule below passes over, and go through the two functions above.
+// The streams a step may spread its layers over.  Lane 0 is the caller's stream: the step starts and ends
+// there.  fork() makes every other lane wait for what lane 0 has enqueued so far, join() makes lane 0 wait for
+// what the other lanes have enqueued; both are event record/wait pairs, which a stream capture records as
+// graph dependencies.  Every lane has a workspace of its own (launches on different lanes may overlap).
+struct Lanes {
+    static constexpr int kMax = 8;
+    int n = 1;
+    cudaStream_t st[kMax] = {};
+    void* ws[kMax] = {};
+    size_t ws_bytes = 0;
+    cudaEvent_t ev[2 * kMax] = {};
+    int n_ev = 0;
+    ~Lanes() { for (int i = 0; i < n_ev; ++i) cudaEventDestroy(ev[i]); }     // pending work keeps what it needs
+    // events are reused between the fork and the join of a stage: a record replaces the earlier one for later waits only
+    int event(cudaEvent_t* out) {
+        if (n_ev == 2 * kMax) return DPCLIP_ERR_CUDA;
+        if (cudaEventCreateWithFlags(&ev[n_ev], cudaEventDisableTiming) != cudaSuccess) return DPCLIP_ERR_CUDA;
+        *out = ev[n_ev++];
+        return DPCLIP_OK;
+    }
+    int fork() {
+        if (n == 1) return DPCLIP_OK;
+        cudaEvent_t e;
+        if (event(&e)) return DPCLIP_ERR_CUDA;
+        if (cudaEventRecord(e, st[0]) != cudaSuccess) return DPCLIP_ERR_CUDA;
+        for (int i = 1; i < n; ++i)
+            if (cudaStreamWaitEvent(st[i], e, 0) != cudaSuccess) return DPCLIP_ERR_CUDA;
+        return DPCLIP_OK;
+    }
+    int join() {
+        for (int i = 1; i < n; ++i) {
+            cudaEvent_t e;
+            if (event(&e)) return DPCLIP_ERR_CUDA;
+            if (cudaEventRecord(e, st[i]) != cudaSuccess || cudaStreamWaitEvent(st[0], e, 0) != cudaSuccess)
+                return DPCLIP_ERR_CUDA;
+        }
+        return DPCLIP_OK;
+    }
+};
+
+// The path layer by layer (with the launches that several layers share), Algorithm 1's order: every layer's
+// norms, then the factors, then every layer's clipped sum with its noise.  Layers are independent within the
+// norm stage and within the clipped-sum stage, so with several lanes the launches of a stage are dealt to the
+// lanes (a layer's kernel then starts on SMs the previous layer's kernel has already left): the shared Gram
+// launch and the shared same-shape launch on lane 0, the T = 1 group on the last lane, the rest round-robin.
+// `other`, when given, is the model's own descriptor array: entries of a kind other than dense have a
+// placeholder with T = 0 in `layers`, which every grouping rule below passes over, and go through the two
+// functions above.
 static int step_general(const dpclip_layer* layers, const dpclip_model_layer* other, int L, int B, dpclip_dtype dtype,
                         float C, float sigma, unsigned long long seed, unsigned long long stream_id0,
-                        float* sq_layers, float* clip, float* norms, void* workspace, size_t workspace_bytes,
-                        void* stream) {
+                        float* sq_layers, float* clip, float* norms, Lanes& lanes) {
     int rc;
+    const int last = lanes.n - 1;
+    void* const ws0 = lanes.ws[0];
+    const size_t workspace_bytes = lanes.ws_bytes;
     T1Group t1;
     rc = prepare_t1_group(t1, layers, L, B, dtype, C, sigma, seed, stream_id0, sq_layers, clip);
     if (rc) return rc;
-    if (t1.active && (!workspace || workspace_bytes < (size_t)kHeaderBytes)) t1.active = false;
+    if (t1.active && (!lanes.ws[last] || workspace_bytes < (size_t)kHeaderBytes)) t1.active = false;
+    if ((rc = lanes.fork())) return rc;
     if (t1.active) {
-        if (dtype == DPCLIP_F32) t1_all_norms_kernel<float><<<t1.p.L * B, 128, 0, (cudaStream_t)stream>>>(t1.p);
-        else t1_all_norms_kernel<__nv_bfloat16><<<t1.p.L * B, 128, 0, (cudaStream_t)stream>>>(t1.p);
+        if (dtype == DPCLIP_F32) t1_all_norms_kernel<float><<<t1.p.L * B, 128, 0, lanes.st[last]>>>(t1.p);
+        else t1_all_norms_kernel<__nv_bfloat16><<<t1.p.L * B, 128, 0, lanes.st[last]>>>(t1.p);
         if (launch_status()) return DPCLIP_ERR_CUDA;
     }
     int in_gram_group[64];
     const bool track = L <= 64;
+    bool any_gram = false;
     if (track) {
-        rc = dpclip_gram_layers_sqnorms(layers, L, B, dtype, sq_layers, in_gram_group, workspace, workspace_bytes, stream);
+        rc = dpclip_gram_layers_sqnorms(layers, L, B, dtype, sq_layers, in_gram_group, ws0, workspace_bytes, lanes.st[0]);
         if (rc) return rc;
+        for (int l = 0; l < L; ++l) any_gram = any_gram || in_gram_group[l];
     }
+    int k = any_gram ? 1 : 0;                              // lane 0 already carries the shared Gram launch
     for (int l = 0; l < L; ++l) {
         const dpclip_layer& y = layers[l];
-        if (other && other[l].kind != DPCLIP_KIND_DENSE) {
-            rc = other_kind_sqnorms(other[l], B, dtype, sq_layers + (size_t)l * B, workspace, workspace_bytes, stream);
-            if (rc) return rc;
-            continue;
-        }
-        if (t1.active && y.T == 1) continue;
-        if (track && in_gram_group[l]) continue;
-        rc = dpclip_layer_sqnorms(y.A, y.lda, y.Zbar, y.ldz, B, y.T, y.d_in, y.d_out, dtype, y.has_bias,
-                                  (dpclip_method)y.method, sq_layers + (size_t)l * B, workspace,
-                                  workspace_bytes, stream);
+        const bool is_other = other && other[l].kind != DPCLIP_KIND_DENSE;
+        if (!is_other && ((t1.active && y.T == 1) || (track && in_gram_group[l]))) continue;
+        const int b = k++ % lanes.n;
+        if (is_other)
+            rc = other_kind_sqnorms(other[l], B, dtype, sq_layers + (size_t)l * B, lanes.ws[b], workspace_bytes, lanes.st[b]);
+        else
+            rc = dpclip_layer_sqnorms(y.A, y.lda, y.Zbar, y.ldz, B, y.T, y.d_in, y.d_out, dtype, y.has_bias,
+                                      (dpclip_method)y.method, sq_layers + (size_t)l * B, lanes.ws[b],
+                                      workspace_bytes, lanes.st[b]);
         if (rc) return rc;
     }
-    rc = dpclip_factors(sq_layers, L, B, B, C, clip, norms, nullptr, stream);
+    if ((rc = lanes.join())) return rc;
+    rc = dpclip_factors(sq_layers, L, B, B, C, clip, norms, nullptr, lanes.st[0]);
     if (rc) return rc;
+    if ((rc = lanes.fork())) return rc;
     if (t1.active) {
-        rc = launch_fused_t1_tf32(t1.p, false, dtype, workspace, workspace_bytes, (cudaStream_t)stream);
+        rc = launch_fused_t1_tf32(t1.p, false, dtype, lanes.ws[last], workspace_bytes, lanes.st[last]);
         if (rc < 0) return rc;
         if (rc > 0) return DPCLIP_ERR_UNSUPPORTED;           // prepare_t1_group checked the same conditions
     }
     int in_grad_group[64];
+    bool any_group = false;
     if (track) {
         rc = dpclip_same_shape_layers_clipped_grad_noise(layers, L, B, dtype, clip, C, sigma, seed, stream_id0,
-                                                         in_grad_group, workspace, workspace_bytes, stream);
+                                                         in_grad_group, ws0, workspace_bytes, lanes.st[0]);
         if (rc) return rc;
+        for (int l = 0; l < L; ++l) any_group = any_group || in_grad_group[l];
     }
+    k = any_group ? 1 : 0;
     for (int l = 0; l < L; ++l) {
         const dpclip_layer& y = layers[l];
-        if (other && other[l].kind != DPCLIP_KIND_DENSE) {
+        const bool is_other = other && other[l].kind != DPCLIP_KIND_DENSE;
+        if (!is_other && ((t1.active && y.T == 1) || (track && in_grad_group[l]))) continue;
+        const int b = k++ % lanes.n;
+        void* const stream = lanes.st[b];
+        void* const workspace = lanes.ws[b];
+        if (is_other) {
             rc = other_kind_clipped_grad_noise(other[l], B, dtype, clip, C, sigma, seed, stream_id0 + 2ull * l,
                                                stream_id0 + 2ull * l + 1, workspace, workspace_bytes, stream);
             if (rc) return rc;
             continue;
         }
-        if (t1.active && y.T == 1) continue;
-        if (track && in_grad_group[l]) continue;
         float* gb = y.has_bias ? y.gb : nullptr;
         if (y.has_bias && !gb) return DPCLIP_ERR_INVALID_ARG;
         // noise indexes the dense d_out x d_in tensor, so the step wants unpadded output rows
@@ -1796,20 +1854,77 @@ static int step_general(const dpclip_layer* layers, const dpclip_model_layer* ot
             }
         }
     }
+    return lanes.join();
+}
+
+// Lanes of a one-stream call, and of a several-streams call (argument checks included).
+static void one_lane(Lanes& lanes, void* workspace, size_t workspace_bytes, void* stream) {
+    lanes.n = 1; lanes.st[0] = (cudaStream_t)stream; lanes.ws[0] = workspace; lanes.ws_bytes = workspace_bytes;
+}
+static int many_lanes(Lanes& lanes, int n_streams, void* const* streams, void* const* workspaces, size_t workspace_bytes) {
+    if (n_streams < 1 || n_streams > Lanes::kMax || !streams || !workspaces) return DPCLIP_ERR_INVALID_ARG;
+    lanes.n = n_streams; lanes.ws_bytes = workspace_bytes;
+    for (int i = 0; i < n_streams; ++i) {
+        lanes.st[i] = (cudaStream_t)streams[i]; lanes.ws[i] = workspaces[i];
+        for (int j = 0; j < i; ++j)
+            if (streams[i] == streams[j] || (workspaces[i] && workspaces[i] == workspaces[j])) return DPCLIP_ERR_INVALID_ARG;
+    }
     return DPCLIP_OK;
+}
+
+static int step_args_ok(const void* layers, int L, int B, dpclip_dtype dtype, float C, float sigma, const float* sq_layers,
+                        const float* clip) {
+    if (!layers || L <= 0 || B <= 0 || !sq_layers || !clip) return DPCLIP_ERR_INVALID_ARG;
+    if (!(C > 0.f) || !(sigma >= 0.f)) return DPCLIP_ERR_INVALID_ARG;
+    if (dtype != DPCLIP_F32 && dtype != DPCLIP_BF16) return DPCLIP_ERR_INVALID_ARG;
+    return DPCLIP_OK;
+}
+
+static int step_dense(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, float C, float sigma,
+                      unsigned long long seed, unsigned long long stream_id0, float* sq_layers, float* clip,
+                      float* norms, Lanes& lanes) {
+    const int rc = try_fused_t1_step(layers, L, B, dtype, C, sigma, seed, stream_id0, sq_layers, clip, norms, lanes.ws[0],
+                                     lanes.ws_bytes, lanes.st[0]);
+    if (rc <= 0) return rc;                  // done (0) or argument error (< 0); 1 = take the general path
+    return step_general(layers, nullptr, L, B, dtype, C, sigma, seed, stream_id0, sq_layers, clip, norms, lanes);
+}
+
+static int step_model(const dpclip_model_layer* layers, int L, int B, dpclip_dtype dtype, float C, float sigma,
+                      unsigned long long seed, unsigned long long stream_id0, float* sq_layers, float* clip,
+                      float* norms, Lanes& lanes) {
+    constexpr int kMaxLayers = 256;
+    if (L > kMaxLayers) return DPCLIP_ERR_INVALID_ARG;
+    dpclip_layer dense[kMaxLayers];
+    bool all_dense = true;
+    for (int l = 0; l < L; ++l) {
+        if (layers[l].kind == DPCLIP_KIND_DENSE) { dense[l] = layers[l].layer; continue; }
+        if (layers[l].kind != DPCLIP_KIND_ELEMENTWISE && layers[l].kind != DPCLIP_KIND_CONV) return DPCLIP_ERR_INVALID_ARG;
+        memset(&dense[l], 0, sizeof(dense[l]));             // T = 0: no grouping rule takes it
+        all_dense = false;
+    }
+    if (all_dense) return step_dense(dense, L, B, dtype, C, sigma, seed, stream_id0, sq_layers, clip, norms, lanes);
+    return step_general(dense, layers, L, B, dtype, C, sigma, seed, stream_id0, sq_layers, clip, norms, lanes);
 }
 
 int dpclip_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, float C, float sigma,
                 unsigned long long seed, unsigned long long stream_id0, float* sq_layers, float* clip,
                 float* norms, void* workspace, size_t workspace_bytes, void* stream) {
-    if (!layers || L <= 0 || B <= 0 || !sq_layers || !clip) return DPCLIP_ERR_INVALID_ARG;
-    if (!(C > 0.f) || !(sigma >= 0.f)) return DPCLIP_ERR_INVALID_ARG;
-    if (dtype != DPCLIP_F32 && dtype != DPCLIP_BF16) return DPCLIP_ERR_INVALID_ARG;
-    const int rc = try_fused_t1_step(layers, L, B, dtype, C, sigma, seed, stream_id0, sq_layers, clip, norms, workspace,
-                                     workspace_bytes, (cudaStream_t)stream);
-    if (rc <= 0) return rc;                  // done (0) or argument error (< 0); 1 = take the general path
-    return step_general(layers, nullptr, L, B, dtype, C, sigma, seed, stream_id0, sq_layers, clip, norms, workspace,
-                        workspace_bytes, stream);
+    int rc = step_args_ok(layers, L, B, dtype, C, sigma, sq_layers, clip);
+    if (rc) return rc;
+    Lanes lanes;
+    one_lane(lanes, workspace, workspace_bytes, stream);
+    return step_dense(layers, L, B, dtype, C, sigma, seed, stream_id0, sq_layers, clip, norms, lanes);
+}
+
+int dpclip_step_streams(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, float C, float sigma,
+                        unsigned long long seed, unsigned long long stream_id0, float* sq_layers, float* clip,
+                        float* norms, int n_streams, void* const* streams, void* const* workspaces,
+                        size_t workspace_bytes) {
+    int rc = step_args_ok(layers, L, B, dtype, C, sigma, sq_layers, clip);
+    if (rc) return rc;
+    Lanes lanes;
+    if ((rc = many_lanes(lanes, n_streams, streams, workspaces, workspace_bytes))) return rc;
+    return step_dense(layers, L, B, dtype, C, sigma, seed, stream_id0, sq_layers, clip, norms, lanes);
 }
 
 int dpclip_step_per_layer(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, const float* C_layer,
@@ -1875,23 +1990,22 @@ size_t dpclip_model_workspace_bytes(const dpclip_model_layer* layers, int L, int
 int dpclip_model_step(const dpclip_model_layer* layers, int L, int B, dpclip_dtype dtype, float C, float sigma,
                       unsigned long long seed, unsigned long long stream_id0, float* sq_layers, float* clip,
                       float* norms, void* workspace, size_t workspace_bytes, void* stream) {
-    constexpr int kMaxLayers = 256;
-    if (!layers || L <= 0 || L > kMaxLayers || B <= 0 || !sq_layers || !clip) return DPCLIP_ERR_INVALID_ARG;
-    if (!(C > 0.f) || !(sigma >= 0.f)) return DPCLIP_ERR_INVALID_ARG;
-    if (dtype != DPCLIP_F32 && dtype != DPCLIP_BF16) return DPCLIP_ERR_INVALID_ARG;
-    dpclip_layer dense[kMaxLayers];
-    bool all_dense = true;
-    for (int l = 0; l < L; ++l) {
-        if (layers[l].kind == DPCLIP_KIND_DENSE) { dense[l] = layers[l].layer; continue; }
-        if (layers[l].kind != DPCLIP_KIND_ELEMENTWISE && layers[l].kind != DPCLIP_KIND_CONV) return DPCLIP_ERR_INVALID_ARG;
-        memset(&dense[l], 0, sizeof(dense[l]));             // T = 0: no grouping rule takes it
-        all_dense = false;
-    }
-    if (all_dense)
-        return dpclip_step(dense, L, B, dtype, C, sigma, seed, stream_id0, sq_layers, clip, norms, workspace,
-                           workspace_bytes, stream);
-    return step_general(dense, layers, L, B, dtype, C, sigma, seed, stream_id0, sq_layers, clip, norms, workspace,
-                        workspace_bytes, stream);
+    int rc = step_args_ok(layers, L, B, dtype, C, sigma, sq_layers, clip);
+    if (rc) return rc;
+    Lanes lanes;
+    one_lane(lanes, workspace, workspace_bytes, stream);
+    return step_model(layers, L, B, dtype, C, sigma, seed, stream_id0, sq_layers, clip, norms, lanes);
+}
+
+int dpclip_model_step_streams(const dpclip_model_layer* layers, int L, int B, dpclip_dtype dtype, float C, float sigma,
+                              unsigned long long seed, unsigned long long stream_id0, float* sq_layers, float* clip,
+                              float* norms, int n_streams, void* const* streams, void* const* workspaces,
+                              size_t workspace_bytes) {
+    int rc = step_args_ok(layers, L, B, dtype, C, sigma, sq_layers, clip);
+    if (rc) return rc;
+    Lanes lanes;
+    if ((rc = many_lanes(lanes, n_streams, streams, workspaces, workspace_bytes))) return rc;
+    return step_model(layers, L, B, dtype, C, sigma, seed, stream_id0, sq_layers, clip, norms, lanes);
 }
 
 size_t dpclip_step_host_arena_bytes(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype) {

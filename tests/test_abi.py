@@ -83,6 +83,34 @@ def test_argument_errors_are_caught_before_any_launch(lib):
     assert lib.dpclip_pick_method(128, 1, 784, 256, 784, 256, 0) == 1
 
 
+def test_streams_step_argument_errors(lib):
+    """dpclip_step_streams checks its stream and workspace arrays on the host before anything is enqueued."""
+    fake = ctypes.c_void_p(0x1000)
+    INVALID = -1
+    f = lib.dpclip_step_streams
+    f.restype = ctypes.c_int
+    vp = ctypes.c_void_p
+
+    class Layer(ctypes.Structure):
+        _fields_ = [("A", vp), ("lda", ctypes.c_long), ("Zbar", vp), ("ldz", ctypes.c_long), ("T", ctypes.c_int),
+                    ("d_in", ctypes.c_int), ("d_out", ctypes.c_int), ("has_bias", ctypes.c_int), ("method", ctypes.c_int),
+                    ("gW", vp), ("ldg", ctypes.c_long), ("gb", vp)]
+    f.argtypes = [ctypes.POINTER(Layer), ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_float, ctypes.c_float,
+                  ctypes.c_ulonglong, ctypes.c_ulonglong, vp, vp, vp, ctypes.c_int, ctypes.POINTER(vp), ctypes.POINTER(vp),
+                  ctypes.c_size_t]
+    layers = (Layer * 1)(Layer(0x1000, 8, 0x2000, 8, 4, 8, 8, 0, 0, 0x3000, 8, None))
+    st2 = (vp * 2)(0x10, 0x20); ws2 = (vp * 2)(0x4000, 0x5000)
+    same_st = (vp * 2)(0x10, 0x10); same_ws = (vp * 2)(0x4000, 0x4000)
+    call = lambda n, st, ws: f(layers, 1, 2, 0, 1.0, 0.0, 0, 0, fake, fake, None, n, st, ws, 1 << 20)   # noqa: E731
+    assert call(0, st2, ws2) == INVALID
+    assert call(9, st2, ws2) == INVALID
+    assert call(2, None, ws2) == INVALID
+    assert call(2, st2, None) == INVALID
+    assert call(2, same_st, ws2) == INVALID
+    assert call(2, st2, same_ws) == INVALID
+    assert f(layers, 1, 2, 0, 0.0, 0.0, 0, 0, fake, fake, None, 2, st2, ws2, 1 << 20) == INVALID     # C must be > 0
+
+
 def test_workspace_queries_without_a_gpu(lib):
     """The workspace queries are host arithmetic: the fixed scratch for ordinary layers, room for one partial
     tile per row slice for long bf16 layers whose 64 tiles leave SMs idle in one wave, and the copies of the

@@ -176,7 +176,7 @@ def test_sequence_workload_full_step_gradients(dp, form):
         plan.flat.fill_(float("nan")); plan.clip.fill_(float("nan"))
         graph.replay()
     torch.cuda.synchronize()
-    assert dp.dpclip_read_status(plan.workspace) == 0
+    assert all(dp.dpclip_read_status(x) == 0 for x in plan.workspaces())
     clip = plan.clip.cpu().numpy()
     assert 0 < (clip < 1).sum() < w.B
     sample = np.array([5, 77, 126])
@@ -250,19 +250,26 @@ def test_mlp_large_graph_replay_full_size(dp):
 
 
 def test_multi_branch_graph_matches_eager_step(dp):
-    """Models with T > 1 layers are timed as a graph whose branches are per-layer entry-point calls on four
-    streams: it must give what the single dpclip_step call gives."""
+    """Models with T > 1 layers are timed as a graph that holds ONE dpclip_step_streams call (the library forks
+    over four streams and joins): it must give what the single-stream dpclip_step call gives."""
     for w in (workloads.seq("bf16", B=6, T=40, d=64, d_ff=136), workloads.cnn("f32")):
         layers = workloads.generate(w, 2)
         mk = lambda: dp.StepPlan([dp.Layer(to_device(A, w.dtype), to_device(Z, w.dtype), s.has_bias)   # noqa: E731
                                   for (A, Z), s in zip(layers, w.layers)])
         eager = mk(); eager.run(w.C, w.sigma, 7)
+        # the same call outside a graph, eager on four streams
+        direct = mk(); direct.run_streams(w.C, w.sigma, 7, branches=4)
+        torch.cuda.synchronize()
+        assert all(dp.dpclip_read_status(x) == 0 for x in direct.workspaces())
+        assert np.allclose(direct.clip.cpu().numpy(), eager.clip.cpu().numpy(), rtol=2e-6, atol=0)
+        for l in range(len(layers)):
+            assert rel_fro(direct.gW[l].cpu().numpy(), eager.gW[l].cpu().numpy()) <= 2e-6
         plan = mk()
         graph = plan.capture(w.C, w.sigma, 7, branches=4)
         plan.flat.fill_(float("nan"))
         graph.replay(); graph.replay()
         torch.cuda.synchronize()
-        assert dp.dpclip_read_status(plan.workspace) == 0
+        assert len(plan.workspaces()) == 4 and all(dp.dpclip_read_status(x) == 0 for x in plan.workspaces())
         assert np.allclose(plan.clip.cpu().numpy(), eager.clip.cpu().numpy(), rtol=2e-6, atol=0)
         for l in range(len(layers)):             # (the flat buffer has alignment gaps nobody writes)
             assert rel_fro(plan.gW[l].cpu().numpy(), eager.gW[l].cpu().numpy()) <= 2e-6
