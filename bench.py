@@ -1,23 +1,29 @@
 #!/usr/bin/env python
 """Benchmark of the per-example clipping path: clipped+noised gradient examples/s.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg4] [--impl reference]
 
 A "step" is one pass of the whole path (per-layer squared norms -> clip factors
 -> clipped sums -> noise) over one batch of synthetic inputs shaped like the
-paper's workloads.  The headline workload is the MLP 784->1000->1000->10 at
-B = 128 (fp32); the other paper-shaped workloads are timed too and reported in
-the same JSON line under "workloads".  Rank 0 prints ONE JSON line.
+paper's workloads.  The headline workload is the largest single-GPU
+configuration: the sequence-model layers at B = 128, T = 256 in bf16 (cfg4).
+The other configurations (the two MLPs, the CNN in both precisions, the
+Gram-vs-materialise sweep) are timed in the same run; their step times and
+roofline fractions are in the JSON line under "configs" (compact, printed last)
+and, with per-kernel detail, under "workloads".  Rank 0 prints ONE JSON line.
 
 Timing: CUDA events on the launching stream, max over ranks.  Models with T > 1
-layers (hundreds of microseconds per step): events around every step, the L2
-flushed by a 256 MB write between steps (outside the events).  All-T=1 models
-(one launch of about ten microseconds per step): the K timed steps are recorded
-back to back into one CUDA graph, step i working on its own copy i % R of the
-inputs and outputs with R copies adding up to more than twice the L2, and one
-event pair brackets the K steps -- the steady state of a training loop, without
-a graph-launch latency charged to every step.  The per-step-graph figure is
-reported beside it ("single_step_graph_ms_per_step").
+layers (hundreds of microseconds per step): one step = one replay of a CUDA
+graph that holds ONE dpclip_step_streams call (the library forks over four
+streams inside the call); events around every step, the L2 flushed by a 256 MB
+write between steps (outside the events).  All-T=1 models (one launch of about
+ten microseconds per step): the K timed steps are recorded back to back into
+one CUDA graph, step i working on its own copy i % R of the inputs and outputs
+with R copies adding up to more than twice the L2, and one event pair brackets
+the K steps -- the steady state of a training loop, without a graph-launch
+latency charged to every step.  The per-step-graph figure is reported beside it
+("single_step_graph_ms_per_step"), and so is the measured floor of an empty
+launch of the same shape ("launch_floor_us").
 """
 from __future__ import annotations
 
@@ -135,6 +141,43 @@ def step_algorithmic_bytes(w):
     return 2 * w.input_bytes() + 4 * w.n_params
 
 
+TF32X3_PER_BF16 = (1.1 / 2.25) / 3.0      # nominal tf32 : bf16 dense ratio, three tf32 MMAs per fp32 product
+
+
+def step_algorithmic_flops(w):
+    """The cheaper exact norm form per layer (closed form for T = 1; symmetric Gram or one materialised
+    product for T > 1) + the one clipped-sum product per layer."""
+    norm = grad = 0.0
+    for s in w.layers:
+        if s.T == 1:
+            norm += 2.0 * w.B * (s.d_in + s.d_out)
+        else:
+            norm += min(float(w.B) * s.T * (s.T + 1) * (s.d_in + s.d_out), 2.0 * w.B * s.T * s.d_in * s.d_out)
+        grad += 2.0 * w.B * s.T * s.d_in * s.d_out
+    return norm, grad
+
+
+def step_roofline(w, peaks):
+    """Lower bound of a whole step: max(algorithmic bytes / HBM bandwidth, algorithmic flops / the peak of the
+    engine the contractions run on).  Bytes: every input twice (norm pass, clipped-sum pass) + every output
+    once.  Engine: bf16 -> the tensor cores (burst and sustained figures both given; the burst one binds
+    harder and is the one `frac` uses, since clocks stay at their maximum in these sub-millisecond steps);
+    fp32 -> the tensor cores as error-compensated tf32 (measured bf16 peak x nominal tf32:bf16 / 3)."""
+    nbytes = step_algorithmic_bytes(w)
+    f_norm, f_grad = step_algorithmic_flops(w)
+    flops = f_norm + f_grad
+    t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9)
+    if w.dtype == "bf16":
+        engine, peak, peak_sus = "tensor bf16", peaks["bf16_tflops"], peaks["bf16_tflops_sustained"]
+    else:
+        engine = "tensor 3xtf32"
+        peak, peak_sus = peaks["bf16_tflops"] * TF32X3_PER_BF16, peaks["bf16_tflops_sustained"] * TF32X3_PER_BF16
+    t_eng, t_eng_sus = flops / (peak * 1e12), flops / (peak_sus * 1e12)
+    return dict(bytes=int(nbytes), flops=flops, engine=engine, t_hbm_us=t_hbm * 1e6, t_engine_burst_us=t_eng * 1e6,
+                t_engine_sustained_us=t_eng_sus * 1e6, bound="hbm" if t_hbm >= t_eng else "tensor",
+                roof_us=max(t_hbm, t_eng) * 1e6, roof_sustained_us=max(t_hbm, t_eng_sus) * 1e6)
+
+
 # ---------------------------------------------------------------------------
 # device arm
 # ---------------------------------------------------------------------------
@@ -230,10 +273,9 @@ def kernel_breakdown(torch, dp, w, plan, steps, flush, C, sigma):
         for l, (y, spec) in enumerate(zip(plan.layers, w.layers)):
             if taken_g[l]:
                 continue
-            timed(("grad", l), lambda: dp.dpclip_clipped_grad(y.A, y.Zbar, plan.clip, plan.gW[l], plan.gb[l],
-                                                              plan.workspace))
-            timed(("noise", l), lambda: (dp.dpclip_add_noise(plan.gW[l], sigma, C, 1, 2 * l),
-                                         plan.gb[l] is not None and dp.dpclip_add_noise(plan.gb[l], sigma, C, 1, 2 * l + 1)))
+            # the clipped sum with its noise, as the step launches it (noise folded into the last pass over the output)
+            timed(("grad", l), lambda: dp.dpclip_clipped_grad_noise(y.A, y.Zbar, plan.clip, plan.gW[l], plan.gb[l], sigma, C,
+                                                                    1, 2 * l, 2 * l + 1, plan.workspace))
     if not any(taken_n):
         acc.pop(("norm_gram_group", -2))
     if not any(taken_g):
@@ -264,9 +306,6 @@ NCU_TRAFFIC_BYTES = {
 }
 
 
-TF32X3_PER_BF16 = (1.1 / 2.25) / 3.0      # nominal tf32 : bf16 dense ratio, three tf32 MMAs per fp32 product
-
-
 def roofline_fused_t1(w, step_ms, peaks):
     """All-T=1 models run inside one dpclip_step call.  Models whose rows TMA can address take the
     one-launch tensor-core kernel (t1_all_grads_tf32_kernel<true, T>: norms, factors, clipped sums, noise;
@@ -275,7 +314,9 @@ def roofline_fused_t1(w, step_ms, peaks):
     step's device time, which can only understate it.  The contraction peak for fp32-by-3xtf32 is the
     measured bf16 peak x the nominal tf32:bf16 ratio / 3; for bf16 it is the measured bf16 peak."""
     flops = sum(2.0 * w.B * s.d_in * s.d_out for s in w.layers)
-    nbytes = w.input_bytes() + 4 * w.n_params
+    # algorithmic bytes of the step: inputs twice (norms, clipped sums) + outputs once.  The one-launch kernel
+    # fetches its inputs from HBM once (the second pass hits L2), so its DRAM traffic is below this figure.
+    nbytes = step_algorithmic_bytes(w)
     quantum = 4 if w.dtype == "f32" else 8
     on_tensor = all(s.d_in % quantum == 0 and (s.d_out % quantum == 0 or s.d_out <= 16) for s in w.layers)
     kernel = "t1_all_grads_tf32_kernel" if on_tensor else "t1_all_grads_kernel"
@@ -293,10 +334,11 @@ def roofline_fused_t1(w, step_ms, peaks):
         r = dict(bound="tensor" if on_tensor else "alu", achieved=ach, peak=peak_tf, unit="TFLOP/s", frac=ach / peak_tf)
     r.update(traffic=NCU_TRAFFIC_BYTES.get((w.name, kernel)), kernel=kernel,
              kernel_ms=step_ms, share_of_step=1.0, algorithmic_bytes=nbytes, algorithmic_flops=flops,
-             hbm_frac=(nbytes / (step_ms * 1e-3) / 1e9) / peaks["hbm_gbs"],
+             launches_per_step=1, hbm_frac=(nbytes / (step_ms * 1e-3) / 1e9) / peaks["hbm_gbs"],
              peak_source=peaks["source"],
-             note="whole step in one kernel; time = step device time; both roofs are far away: the step is a chain "
-                  "of memory round trips (row loads, grid barrier, factor loads, tile loads, output stores)")
+             note="whole step in one kernel; time = step device time; both roofs are below any launch (see "
+                  "launch_floor_us): the step is a chain of memory round trips (row loads, grid barrier, factor "
+                  "loads, tile loads, output stores)")
     return r
 
 
@@ -331,11 +373,51 @@ def roofline_group(w, key, breakdown, peaks):
     return r
 
 
+def _zta_layers(w):
+    """Layers whose clipped sum runs on zta_tc_kernel (bf16, rows TMA can address, not narrow)."""
+    if w.dtype != "bf16":
+        return []
+    return [l for l, s in enumerate(w.layers)
+            if s.T > 1 and s.d_in % 8 == 0 and s.d_out % 8 == 0 and not (s.d_in + (1 if s.has_bias else 0) <= 32 and s.d_out <= 64)]
+
+
+def roofline_zta(w, breakdown, peaks):
+    """The bf16 clipped-sum kernel over ALL its launches of a step (grouped launch + per-layer launches): work =
+    the layers' sum, time = the sum of the entry-point calls' device times (each call = zta_tc_kernel + the
+    reduce/noise launch that follows it), launches counted."""
+    members = _zta_layers(w)
+    keys = [k for k in breakdown if k[0] == "grad_group" or (k[0] == "grad" and k[1] in members)]
+    if not keys:
+        return None
+    ms = sum(breakdown[k] for k in keys)
+    nbytes = sum(layer_work(w, w.layers[l], "grad")[0] for l in members)
+    flops = sum(layer_work(w, w.layers[l], "grad")[1] for l in members)
+    t_hbm, t_alu = nbytes / (peaks["hbm_gbs"] * 1e9), flops / (peaks["bf16_tflops"] * 1e12)
+    if t_hbm >= t_alu:
+        ach = nbytes / (ms * 1e-3) / 1e9
+        r = dict(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s", frac=ach / peaks["hbm_gbs"])
+    else:
+        ach = flops / (ms * 1e-3) / 1e12
+        r = dict(bound="tensor", achieved=ach, peak=peaks["bf16_tflops"], unit="TFLOP/s", frac=ach / peaks["bf16_tflops"],
+                 frac_of_sustained_peak=ach / peaks["bf16_tflops_sustained"])
+    traffic = [NCU_TRAFFIC_BYTES.get((w.name, "grad_group" if k[0] == "grad_group" else f"grad[{w.layers[k[1]].name}]")) for k in keys]
+    r.update(traffic=(sum(traffic) / len(keys) if all(t is not None for t in traffic) else None),
+             kernel="zta_tc_kernel (+ reduce_partials_kernel)", launches_per_step=len(keys), kernel_ms=ms / len(keys),
+             kernel_ms_total=ms, share_of_step=ms / sum(breakdown.values()), algorithmic_bytes=nbytes / len(keys),
+             algorithmic_flops=flops / len(keys), peak_source=peaks["source"],
+             note="per launch: averages over the kernel's launches of one step; peak = burst bf16 figure")
+    return r
+
+
 def roofline_for(w, breakdown, peaks):
-    """Roofline of the launch that takes the largest share of the step."""
+    """Roofline of the kernel that takes the largest share of the step: the bf16 clipped-sum kernel over all its
+    launches when that is the largest, else the single launch with the largest share."""
     cands = {k: v for k, v in breakdown.items() if k[0] not in ("factors",)}
     key = max(cands, key=cands.get)
     kind, l = key
+    zta = roofline_zta(w, breakdown, peaks)
+    if zta is not None and zta["kernel_ms_total"] >= cands[key]:
+        return zta
     if kind in kernel_breakdown.groups:
         return roofline_group(w, key, breakdown, peaks)
     spec = w.layers[l]
@@ -380,23 +462,28 @@ def bench_workload(torch, dp, w, steps, warmup, flush, peaks, with_e2e=True):
     branches = 1 if all(s.T == 1 for s in w.layers) else 4
     graph = plan.capture(w.C, w.sigma, 1, branches=branches)
     single = time_steps(torch, graph.replay, steps, warmup, flush)
-    assert dp.dpclip_read_status(plan.workspace) == 0
+    assert all(dp.dpclip_read_status(x) == 0 for x in plan.workspaces())
     rotating = None
     if branches == 1:
         times, rotating = time_steps_rotating(torch, dp, w, layers, steps, warmup, flush)
     else:
         times = single
+    one_stream_ms = None
+    if branches > 1:
+        g1 = plan.capture(w.C, w.sigma, 1, branches=1)          # the same step as ONE dpclip_step call on one stream
+        one_stream_ms = float(np.mean(time_steps(torch, g1.replay, min(steps, 10), 2, flush)))
     warm = time_steps(torch, graph.replay, steps, 1, lambda: None)
     eager = time_steps(torch, lambda: plan.run(w.C, w.sigma, 1), steps, 1, flush)
     bd = kernel_breakdown(torch, dp, w, plan, min(steps, 20), flush, w.C, w.sigma)
     res = dict(times_ms=times, warm_ms=float(np.median(warm)), eager_ms=float(np.median(eager)),
-               single_graph_ms=float(np.mean(single)), rotating=rotating,
+               single_graph_ms=float(np.mean(single)), rotating=rotating, one_stream_ms=one_stream_ms,
                launches_per_step=int(launches_per_step),
                breakdown={f"{k[0]}[{entry_name(w, k)}]": round(v * 1e3, 2) for k, v in bd.items()},
                roofline=(roofline_fused_t1(w, float(np.mean(times)), peaks) if branches == 1
                          else roofline_for(w, bd, peaks)))
     # whole-step lower bound: max(total algorithmic bytes / HBM, total flops / the engine used)
-    res["step_roofline_us"] = step_algorithmic_bytes(w) / (peaks["hbm_gbs"] * 1e9) * 1e6
+    res["step_roofline"] = step_roofline(w, peaks)
+    res["step_roofline_us"] = res["step_roofline"]["roof_us"]
     if with_e2e:
         host_layers = [dp.Layer(torch.from_numpy(A).to(torch.float32 if w.dtype == "f32" else torch.bfloat16).pin_memory(),
                                 torch.from_numpy(Z).to(torch.float32 if w.dtype == "f32" else torch.bfloat16).pin_memory(),
@@ -693,16 +780,95 @@ def run_sweep(args):
     print(json.dumps(dict(sweep="norm_method_crossover", dtype="bf16", peaks=peaks, points=rows, noise=noise)))
 
 
+def launch_floors(torch, dp, steps, flush):
+    """Device time per EMPTY launch with the launch shape of the one-launch T = 1 step (128 CTAs of 18 warps, its
+    dynamic shared memory), plain and cooperative, measured the way the all-T=1 steps are: `steps` launches
+    back to back in one CUDA graph, one event pair around them, median of three replays."""
+    out = {}
+    for name, coop in (("plain", False), ("cooperative", True)):
+        dp.dpclip_null_launch(coop, 128)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for _ in range(steps):
+                dp.dpclip_null_launch(coop, 128)
+        graph.replay(); torch.cuda.synchronize()
+        reps = []
+        for _ in range(3):
+            flush()
+            s0, e0 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            s0.record(); graph.replay(); e0.record()
+            torch.cuda.synchronize()
+            reps.append(s0.elapsed_time(e0) * 1e3 / steps)
+        out[name] = round(float(np.median(reps)), 2)
+        # and one launch per graph replay, events around each replay (what single_step_graph_ms_per_step pays)
+        g1 = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g1):
+            dp.dpclip_null_launch(coop, 128)
+        out[name + "_single_graph"] = round(float(np.median(time_steps(torch, g1.replay, 20, 3, flush))) * 1e3, 2)
+    return out
+
+
+def sweep_points_compact(torch, dp, steps, flush, peaks):
+    """The Gram-vs-materialise sweep (one dense bf16 layer with bias per point; B in {256, 1024}, T in {16, 128,
+    512, 2048}, d_in x d_out in {1024x1024, 1024x4096, 4096x1024}): per point the step = norms (the method the
+    library picks) + factors + clipped sum with noise, each launch timed alone with CUDA events, L2 flushed in
+    between, against the point's own step roofline.  Inputs are drawn on the device (timing only; parity at these
+    shapes is in the test suite).  Lightest points first (see run_sweep)."""
+    pts = [(B, T, d_in, d_out) for B in (256, 1024) for T in (16, 128, 512, 2048)
+           for d_in, d_out in ((1024, 1024), (1024, 4096), (4096, 1024))]
+    pts.sort(key=lambda pt: pt[0] * pt[1] * pt[2] * pt[3])
+    rows = []
+    for B, T, d_in, d_out in pts:
+        w = workloads.sweep_point(B, T, d_in, d_out)
+        ws = torch.empty(dp.dpclip_workspace_bytes(B, T, d_in, d_out, dp.DPCLIP_BF16), dtype=torch.uint8, device="cuda")
+        dp.dpclip_workspace_init(ws)
+        g = torch.Generator(device="cuda").manual_seed(B * 7919 + T)
+        A = torch.empty(B, T, d_in, device="cuda", dtype=torch.bfloat16)
+        Z = torch.empty(B, T, d_out, device="cuda", dtype=torch.bfloat16)
+        for i in range(0, B, 64):                                  # drawn in slabs: no 30 GB fp32 temporaries
+            A[i:i + 64] = torch.randn(min(64, B - i), T, d_in, device="cuda", generator=g).to(torch.bfloat16)
+            Z[i:i + 64] = (torch.randn(min(64, B - i), T, d_out, device="cuda", generator=g) * (B * T) ** -0.5).to(torch.bfloat16)
+        sq = torch.empty(1, B, device="cuda"); clip = torch.empty(B, device="cuda"); nrm = torch.empty(B, device="cuda")
+        gW = torch.empty(d_out, d_in, device="cuda"); gb = torch.empty(d_out, device="cuda")
+        n = 3 if B * T * d_in * d_out > 1e14 / 8 else max(3, min(steps, 6))
+        t_norm = float(np.median(time_steps(torch, lambda: dp.dpclip_layer_sqnorms(A, Z, True, sq[0], ws), n, 2, flush)))
+        t_fac = float(np.median(time_steps(torch, lambda: dp.dpclip_factors(sq, w.C, clip, nrm), n, 2, flush)))
+        t_grad = float(np.median(time_steps(
+            torch, lambda: dp.dpclip_clipped_grad_noise(A, Z, clip, gW, gb, w.sigma, w.C, 1, 0, 1, ws), n, 2, flush)))
+        assert dp.dpclip_read_status(ws) == 0
+        roof = step_roofline(w, peaks)
+        step_us = (t_norm + t_fac + t_grad) * 1e3
+        meth = {dp.DPCLIP_GRAM: "gram", dp.DPCLIP_MATERIALIZE: "mat"}.get(
+            dp.dpclip_pick_method(B, T, d_in, d_out, d_in, d_out, dp.DPCLIP_BF16), "other")
+        rows.append(dict(B=B, T=T, d_in=d_in, d_out=d_out, norm_method=meth, norm_us=t_norm * 1e3, factors_us=t_fac * 1e3,
+                         grad_us=t_grad * 1e3, step_us=step_us, roof_us=roof["roof_us"], bound=roof["bound"],
+                         frac=roof["roof_us"] / step_us, value=B / (step_us * 1e-6),
+                         grad_tflops=2.0 * B * T * d_in * d_out / (t_grad * 1e-3) / 1e12))
+        del A, Z, gW, ws
+        torch.cuda.empty_cache()
+    return rows
+
+
+def config_summary(name, w, r, ms):
+    """One compact entry of the `configs` object."""
+    sr = r["step_roofline"]
+    return dict(workload=w.name, us=round(ms * 1e3, 2), ex_s=round(w.B / (ms * 1e-3), 1), bound=sr["bound"],
+                roof_us=round(sr["roof_us"], 2), frac=round(sr["roof_us"] / (ms * 1e3), 4),
+                frac_sustained=round(sr["roof_sustained_us"] / (ms * 1e3), 4))
+
+
 # ---------------------------------------------------------------------------
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--workload", default="cfg4")
     ap.add_argument("--impl", default="dpclip", choices=["dpclip", "reference"])
-    ap.add_argument("--others", default="cfg1,cfg2_bf16,cfg3_f32,cfg3_bf16,cfg4",
-                    help="further workloads reported under 'workloads' (N=1 only; 'none' for none)")
+    ap.add_argument("--others", default="cfg1,cfg2,cfg2_bf16,cfg3_f32,cfg3_bf16,cfg4",
+                    help="further workloads reported under 'configs' / 'workloads' (N=1 only; 'none' for none)")
+    ap.add_argument("--no-extras", action="store_true", help="skip the sweep points and the single-feature timings")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--points", default="", help="with --sweep: only these points, 'B,T,d_in,d_out;B,T,d_in,d_out;...'")
     ap.add_argument("--noise-n", type=int, default=0, help="with --sweep: also time dpclip_add_noise on this many elements")
@@ -744,17 +910,17 @@ def main():
         from paper_2009_03106_b200 import parallel
         layers = workloads.generate(w, seed=rank)                 # every rank owns its own batch (weak scaling)
         plan = make_plan(dp, w, layers, torch)
-        fn = lambda: parallel.sharded_step(plan, w.C, w.sigma, seed=1, stream_id0=0)   # noqa: E731
-        n0 = dp.dpclip_launch_count(); fn(); lps = dp.dpclip_launch_count() - n0
+        step = parallel.ShardedStep(plan, w.C, w.sigma, seed=1, stream_id0=0)
+        n0 = dp.dpclip_launch_count(); step.run(); lps = dp.dpclip_launch_count() - n0
         dist.barrier(); torch.cuda.synchronize()
         t_wall0 = time.time()
-        times = time_steps(torch, fn, args.steps, args.warmup, flush)
+        times = time_steps(torch, step.run, args.steps, args.warmup, flush)
         torch.cuda.synchronize(); dist.barrier()
         t_wall1 = time.time()
         tot = torch.tensor([sum(times)], device="cuda", dtype=torch.float64)
         dist.all_reduce(tot, op=dist.ReduceOp.MAX)
         total_ms = tot.item()
-        res = dict(launches_per_step=int(lps), roofline=None, e2e_ms=None)
+        res = dict(launches_per_step=int(lps), roofline=None, e2e_ms=None, how=step.describe())
     else:
         t_wall0 = time.time()
         res = bench_workload(torch, dp, w, args.steps, args.warmup, flush, peaks)
@@ -775,58 +941,85 @@ def main():
                             C=w.C, sigma=w.sigma, l2="flushed by a 256 MB write between steps",
                             parallelism=f"dp{world}" if world > 1 else "single"),
                 gpu_launches=int(res["launches_per_step"]) * args.steps, clocks=clocks)
-    if world == 1:
-        line["roofline"] = res["roofline"]
-        line["step_roofline_frac"] = res["step_roofline_us"] / (ms_per_step * 1e3)
-        line["warm_l2_ms_per_step"] = res["warm_ms"]
-        line["eager_ms_per_step"] = res["eager_ms"]
-        if res.get("rotating"):
-            rt = res["rotating"]
-            line["config"]["l2"] = (f"inputs larger than L2: step i works on input/output set i % {rt['sets']} "
-                                    f"({rt['set_bytes'] / 1e6:.1f} MB each), 256 MB flush write before the timed region")
-            line["config"]["launch"] = (f"one CUDA graph holding the {args.steps} timed steps back to back (one dpclip_step "
-                                        "call each); one event pair around the region, median of 3 regions")
-            line["single_step_graph_ms_per_step"] = res["single_graph_ms"]
-        else:
-            line["config"]["launch"] = "CUDA graph replay of one step (per-layer calls on 4 streams), events around every step"
-        line["breakdown_us"] = res["breakdown"]
-        line["e2e"] = dict(value=w.B / (res["e2e_ms"] * 1e-3), unit=UNIT, h2d_bytes_per_step=res["h2d"],
-                           d2h_bytes_per_step=res["d2h"], ms_per_step=res["e2e_ms"],
-                           serial_ms_per_step=res["e2e_serial_ms"],
-                           note="dpclip_step_host per step (all inputs host->device, all results device->host); two steps "
-                                "in flight on two streams; serial_ms_per_step = one step at a time")
-        others = {}
-        for name in [n for n in args.others.split(",") if n and n != args.workload]:
-            ow = workloads.by_name(name)
-            r = bench_workload(torch, dp, ow, min(args.steps, 20), 3, flush, peaks, with_e2e=False)
-            ms = float(np.mean(r["times_ms"]))
-            others[name] = dict(workload=ow.name, dtype=ow.dtype, value=ow.B / (ms * 1e-3), ms_per_step=ms,
-                                warm_l2_ms_per_step=r["warm_ms"], eager_ms_per_step=r["eager_ms"], launches_per_step=r["launches_per_step"],
-                                single_step_graph_ms_per_step=r["single_graph_ms"],
-                                timing=("rotating sets, one graph of all timed steps" if r.get("rotating") else "flush + events per step"),
-                                step_roofline_frac=r["step_roofline_us"] / (ms * 1e3), roofline=r["roofline"],
-                                breakdown_us=r["breakdown"])
-        if args.others:
-            for shape in ((128, 256, 512, "bf16"), (512, 512, 1024, "bf16")):
-                r = bench_elementwise(torch, dp, *shape, min(args.steps, 20), flush, peaks)
-                others[r["workload"]] = r
-            r = bench_model_block(torch, dp, min(args.steps, 20), flush)
-            others[r["workload"]] = r
-            r = bench_per_layer(torch, dp, min(args.steps, 20), flush)
-            others[r["workload"]] = r
-            for cdt in ("f32", "bf16"):
-                r = bench_model_cnn(torch, dp, cdt, min(args.steps, 20), flush)
-                others[r["workload"]] = r
-            for cdt in ("f32", "bf16"):
-                r = bench_conv_implicit(torch, dp, "conv2_implicit_im2col_b128_" + cdt, 128, 32, 16, 16, 3, 1, 64, cdt,
-                                        min(args.steps, 20), flush, peaks)
-                others[r["workload"]] = r
-        line["workloads"] = others
-        if not args.no_cpu_baseline:
-            line["cpu_baseline"], _, _ = oracle_sample(w)
-    else:
+    if world > 1:
+        line["config"]["launch"] = res["how"]
         line["e2e"] = None
         dist.destroy_process_group()
+        print(json.dumps(line))
+        return
+
+    sr = res["step_roofline"]
+    roof = res["roofline"]
+    roof["step"] = dict(sr, measured_us=ms_per_step * 1e3, frac=sr["roof_us"] / (ms_per_step * 1e3),
+                        frac_sustained=sr["roof_sustained_us"] / (ms_per_step * 1e3),
+                        note="whole step: max(bytes / HBM, flops / tensor peak) over the measured step time; bytes = inputs "
+                             "twice + outputs once, flops = cheaper exact norm form + clipped-sum product")
+    line["roofline"] = roof
+    line["step_roofline_frac"] = sr["roof_us"] / (ms_per_step * 1e3)
+    line["warm_l2_ms_per_step"] = res["warm_ms"]
+    line["eager_ms_per_step"] = res["eager_ms"]
+    line["one_stream_graph_ms_per_step"] = res.get("one_stream_ms")
+    if res.get("rotating"):
+        rt = res["rotating"]
+        line["config"]["l2"] = (f"inputs larger than L2: step i works on input/output set i % {rt['sets']} "
+                                f"({rt['set_bytes'] / 1e6:.1f} MB each), 256 MB flush write before the timed region")
+        line["config"]["launch"] = (f"one CUDA graph holding the {args.steps} timed steps back to back (one dpclip_step "
+                                    "call each); one event pair around the region, median of 3 regions")
+        line["single_step_graph_ms_per_step"] = res["single_graph_ms"]
+    else:
+        line["config"]["launch"] = ("CUDA graph replay of one step = ONE dpclip_step_streams call (the library forks over 4 "
+                                    "streams); events around every step")
+    line["breakdown_us"] = res["breakdown"]
+    line["e2e"] = dict(value=w.B / (res["e2e_ms"] * 1e-3), unit=UNIT, h2d_bytes_per_step=res["h2d"],
+                       d2h_bytes_per_step=res["d2h"], ms_per_step=res["e2e_ms"],
+                       serial_ms_per_step=res["e2e_serial_ms"],
+                       note="dpclip_step_host per step (all inputs host->device from pinned memory, all results "
+                            "device->host); two steps in flight on two streams; serial_ms_per_step = one step at a time")
+    configs = {args.workload: config_summary(args.workload, w, res, ms_per_step)}
+    others = {}
+    for name in [n for n in args.others.split(",") if n and n != args.workload]:
+        ow = workloads.by_name(name)
+        r = bench_workload(torch, dp, ow, min(args.steps, 20), 3, flush, peaks, with_e2e=False)
+        ms = float(np.mean(r["times_ms"]))
+        configs[name] = config_summary(name, ow, r, ms)
+        others[name] = dict(workload=ow.name, dtype=ow.dtype, value=ow.B / (ms * 1e-3), ms_per_step=ms,
+                            warm_l2_ms_per_step=r["warm_ms"], eager_ms_per_step=r["eager_ms"], launches_per_step=r["launches_per_step"],
+                            single_step_graph_ms_per_step=r["single_graph_ms"], one_stream_graph_ms_per_step=r.get("one_stream_ms"),
+                            timing=("rotating sets, one graph of all timed steps" if r.get("rotating") else "flush + events per step"),
+                            step_roofline=r["step_roofline"], step_roofline_frac=r["step_roofline_us"] / (ms * 1e3),
+                            roofline=r["roofline"], breakdown_us=r["breakdown"])
+    if args.others:
+        line["launch_floor_us"] = launch_floors(torch, dp, max(args.steps, 20), flush)
+        for k in ("cfg1", "cfg2", "cfg2_bf16"):
+            if k in configs:
+                configs[k]["launch_floor_us"] = line["launch_floor_us"]["cooperative"]
+    if args.others and not args.no_extras:
+        pts = sweep_points_compact(torch, dp, args.steps, flush, peaks)
+        others["cfg5_sweep"] = pts
+        # compact: "B,T,d_in,d_out": [step us, fraction of the point's step roofline]
+        configs["cfg5"] = {f"{r['B']},{r['T']},{r['d_in']},{r['d_out']}": [round(r["step_us"], 1), round(r["frac"], 3)]
+                           for r in pts}
+        for shape in ((128, 256, 512, "bf16"), (512, 512, 1024, "bf16")):
+            r = bench_elementwise(torch, dp, *shape, min(args.steps, 20), flush, peaks)
+            others[r["workload"]] = r
+        r = bench_model_block(torch, dp, min(args.steps, 20), flush)
+        others[r["workload"]] = r
+        r = bench_per_layer(torch, dp, min(args.steps, 20), flush)
+        others[r["workload"]] = r
+        for cdt in ("f32", "bf16"):
+            r = bench_model_cnn(torch, dp, cdt, min(args.steps, 20), flush)
+            others[r["workload"]] = r
+        for cdt in ("f32", "bf16"):
+            r = bench_conv_implicit(torch, dp, "conv2_implicit_im2col_b128_" + cdt, 128, 32, 16, 16, 3, 1, 64, cdt,
+                                    min(args.steps, 20), flush, peaks)
+            others[r["workload"]] = r
+    line["workloads"] = others
+    if not args.no_cpu_baseline:
+        line["cpu_baseline"], _, _ = oracle_sample(w)
+    # per-configuration step times and roofline fractions: inside `roofline` (kept with the headline) and,
+    # compact, as the LAST key of the line
+    roof["per_config"] = {k: (v if k == "cfg5" else dict(us=v["us"], frac=v["frac"], bound=v["bound"])) for k, v in configs.items()}
+    line["configs"] = configs
     print(json.dumps(line))
 
 

@@ -464,6 +464,12 @@ int dpclip_pick_method(int B, int T, int d_in, int d_out, long lda, long ldz, dp
  * counter for benchmarks and tests; cudaMemset calls are not counted). */
 unsigned long long dpclip_launch_count(void);
 
+/* Launch floor, for benchmarks: enqueue one EMPTY kernel with the launch shape of the one-launch T = 1 step
+ * (grid CTAs of 18 warps, its dynamic shared memory; cooperative or plain).  The small all-T=1 workloads
+ * (Sec. "Fully-connected Layers": MLPs at batch 32-128) have roofline times below any launch, so their
+ * measured step time is reported next to this floor.  (No counterpart in the paper.)  grid in 1..148. */
+int dpclip_null_launch(int cooperative, int grid, void* stream);
+
 /* The DPCLIP_* environment switches that force a slower kernel form (for tests and measurements) are read
  * once, at the first call that needs them.  This re-reads them. */
 void dpclip_reload_path_switches(void);

@@ -127,6 +127,8 @@ def load_library():
     L.dpclip_version.argtypes = []
     L.dpclip_launch_count.argtypes = []
     L.dpclip_launch_count.restype = _u64
+    L.dpclip_null_launch.argtypes = [_i, _i, _vp]
+    L.dpclip_null_launch.restype = _i
     L.dpclip_reload_path_switches.argtypes = []
     L.dpclip_reload_path_switches.restype = None
     for name in ("dpclip_layer_sqnorms", "dpclip_factors", "dpclip_clipped_grad", "dpclip_add_noise",
@@ -185,6 +187,11 @@ def dpclip_version() -> int:
 
 def dpclip_launch_count() -> int:
     return load_library().dpclip_launch_count()
+
+
+def dpclip_null_launch(cooperative: bool, grid: int = 128, stream=None) -> None:
+    """One empty kernel with the launch shape of the one-launch T = 1 step (launch-floor measurements)."""
+    _check("dpclip_null_launch", load_library().dpclip_null_launch(int(cooperative), grid, _stream(stream)))
 
 
 def dpclip_reload_path_switches() -> None:

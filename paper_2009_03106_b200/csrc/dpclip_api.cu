@@ -974,6 +974,25 @@ extern "C" {
 
 int dpclip_version(void) { return 100; }
 
+// An empty kernel with the launch shape of the one-launch T = 1 step: what a launch costs before it computes.
+__global__ void null_launch_kernel(int* sink) { if (sink && threadIdx.x == 0xFFFFFF) *sink = 0; }
+
+int dpclip_null_launch(int cooperative, int grid, void* stream) {
+    namespace f = tc::f1;
+    if (grid < 1 || grid > kNumSMs) return DPCLIP_ERR_INVALID_ARG;
+    if (!enable_smem(null_launch_kernel, f::SMEM_BYTES)) return DPCLIP_ERR_CUDA;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(f::THREADS); cfg.dynamicSmemBytes = f::SMEM_BYTES;
+    cfg.stream = (cudaStream_t)stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeCooperative; attr.val.cooperative = cooperative ? 1 : 0;
+    cfg.attrs = &attr; cfg.numAttrs = 1;
+    int* none = nullptr;
+    if (cudaLaunchKernelEx(&cfg, null_launch_kernel, none) != cudaSuccess) { cudaGetLastError(); return DPCLIP_ERR_CUDA; }
+    return launch_status();
+}
+
 unsigned long long dpclip_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 void dpclip_reload_path_switches(void) { read_path_switches(); }
 

@@ -958,6 +958,14 @@ def test_sharded_step_single_rank_equals_step(dp):
         assert dp.dpclip_read_status(plan.workspace) == 0
         assert torch.equal(plan.clip, ref.clip)
         assert rel_fro(plan.flat.cpu().numpy(), ref.flat.cpu().numpy()) <= 1e-6
+        # the recorded form the multi-GPU benchmark replays (graph of the local step, bucketed reduction, noise once)
+        plan2 = dp.StepPlan(dls)
+        step = parallel.ShardedStep(plan2, w.C, w.sigma, seed, 0, bucket_bytes=1 << 12)
+        step.run(); step.run()
+        torch.cuda.synchronize()
+        assert all(dp.dpclip_read_status(x) == 0 for x in plan2.workspaces())
+        assert np.allclose(plan2.clip.cpu().numpy(), ref.clip.cpu().numpy(), rtol=2e-6, atol=0)
+        assert rel_fro(plan2.flat.cpu().numpy(), ref.flat.cpu().numpy()) <= 2e-6
 
 
 def test_step_host_matches_device_step(dp):

@@ -42,6 +42,28 @@ class OracleOps:
         g.copy_(torch.from_numpy(self.o.add_noise(g.numpy(), sigma, C, seed, stream_id)).float())
 
 
+class OracleWholeStepOps(OracleOps):
+    """The same with the whole-step call and the all-tensors noise call of the CUDA binding: drives the branch
+    of the sharded step that GPUs take (one library call before the reduction, one noise call after it)."""
+
+    def dpclip_step(self, plan, C, sigma, seed, stream_id0=0):
+        assert sigma == 0.0                                   # the noise belongs after the reduction
+        layers = [(y.A.numpy(), y.Zbar.numpy()) for y in plan.layers]
+        r = self.o.step(layers, [y.has_bias for y in plan.layers], C, 0.0, seed, stream_id0)
+        plan.clip.copy_(torch.from_numpy(r["clip"]).float()); plan.norms.copy_(torch.from_numpy(r["norms"]).float())
+        for l in range(len(layers)):
+            plan.gW[l].copy_(torch.from_numpy(r["gW"][l]).float())
+            if plan.gb[l] is not None:
+                plan.gb[l].copy_(torch.from_numpy(r["gb"][l]).float())
+        self.whole_calls = getattr(self, "whole_calls", 0) + 1
+
+    def dpclip_step_noise(self, plan, C, sigma, seed, stream_id0=0):
+        for l in range(len(plan.layers)):
+            self.dpclip_add_noise(plan.gW[l].view(-1), sigma, C, seed, stream_id0 + 2 * l)
+            if plan.gb[l] is not None:
+                self.dpclip_add_noise(plan.gb[l], sigma, C, seed, stream_id0 + 2 * l + 1)
+
+
 class CpuPlan:
     def __init__(self, layers, has_bias):
         from types import SimpleNamespace
@@ -61,7 +83,7 @@ class CpuPlan:
         self.workspace = None
 
 
-def _worker(rank, world, port, q):
+def _worker(rank, world, port, q, whole=False, bucket_elements=0):
     sys.path.insert(0, ROOT)
     os.environ["MASTER_ADDR"] = "127.0.0.1"; os.environ["MASTER_PORT"] = str(port)
     dist.init_process_group("gloo", rank=rank, world_size=world)
@@ -73,20 +95,27 @@ def _worker(rank, world, port, q):
     mine = [(A[lo:hi], Z[lo:hi]) for A, Z in full]
     hb = [s.has_bias for s in w.layers]
     plan = CpuPlan(mine, hb)
-    parallel.sharded_step(plan, 78.0, w.sigma, seed=5, stream_id0=0, ops=OracleOps())
+    ops = OracleWholeStepOps() if whole else OracleOps()
+    parallel.sharded_step(plan, 78.0, w.sigma, seed=5, stream_id0=0, ops=ops, bucket_elements=bucket_elements)
+    if whole:
+        assert ops.whole_calls == 1
     q.put((rank, lo, hi, plan.flat.numpy().copy(), plan.clip.numpy().copy()))
     dist.barrier()
     dist.destroy_process_group()
 
 
-def test_sharded_step_equals_single_process_step():
+@pytest.mark.parametrize("world,whole,bucket_elements", [(2, False, 0), (2, True, 0), (3, True, 50000)])
+def test_sharded_step_equals_single_process_step(world, whole, bucket_elements):
+    """Per-stage ops and one all-reduce; the whole-step branch GPUs take; and three ranks with an uneven split
+    (11 + 11 + 10 examples) whose reduction goes out in several asynchronous buckets."""
     import oracle
     import workloads
+    from paper_2009_03106_b200 import parallel
     with socket.socket() as s:
         s.bind(("127.0.0.1", 0)); port = s.getsockname()[1]
     ctx = mp.get_context("spawn")
     q = ctx.Queue()
-    procs = [ctx.Process(target=_worker, args=(r, 2, port, q)) for r in range(2)]
+    procs = [ctx.Process(target=_worker, args=(r, world, port, q, whole, bucket_elements)) for r in range(world)]
     for p in procs:
         p.start()
     got = sorted([q.get(timeout=180) for _ in procs], key=lambda t: t[0])
@@ -99,10 +128,23 @@ def test_sharded_step_equals_single_process_step():
     want = np.concatenate([np.concatenate([ref["outW"][l].ravel(), ref["outb"][l]]) for l in range(2)])
     assert 0 < (ref["clip"] < 1).sum() < w.B
     # ranks cover the batch once, agree with each other, and match the unsharded result
-    assert (got[0][1], got[0][2], got[1][1], got[1][2]) == (0, 16, 16, 32)
-    np.testing.assert_array_equal(got[0][3], got[1][3])
+    assert [(g[1], g[2]) for g in got] == [parallel.shard_examples(w.B, r, world) for r in range(world)]
+    if world == 3:
+        assert [g[2] - g[1] for g in got] == [11, 11, 10]
+    for g in got[1:]:
+        np.testing.assert_array_equal(got[0][3], g[3])
     np.testing.assert_allclose(got[0][3], want, rtol=1e-5, atol=1e-5)
-    np.testing.assert_allclose(np.concatenate([got[0][4], got[1][4]]), ref["clip"], rtol=1e-6)
+    np.testing.assert_allclose(np.concatenate([g[4] for g in got]), ref["clip"], rtol=1e-6)
+
+
+def test_buckets_cover_the_buffer_once():
+    from paper_2009_03106_b200 import parallel
+    for n, b in [(10, 3), (1 << 20, 1 << 18), (1000, 1 << 20), (1025, 256), (7, 1)]:
+        cuts = parallel.buckets(n, b)
+        assert cuts[0][0] == 0 and cuts[-1][1] == n
+        assert all(cuts[i][1] == cuts[i + 1][0] for i in range(len(cuts) - 1))
+        assert all(hi > lo for lo, hi in cuts)
+    assert parallel.buckets(0, 4) == []
 
 
 def test_shard_examples_partitions_the_batch():
