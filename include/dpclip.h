@@ -194,9 +194,9 @@ int dpclip_clipped_grad_noise(const void* A, long lda, const void* Zbar, long ld
  *   - the output, padded to 256 x 256 tiles, must be at most
  *     dpclip_noalloc_max_output_bytes() (8 MB, e.g. 1024 x 2048 fp32);
  *     larger layers return DPCLIP_ERR_WORKSPACE and nothing is launched.  The
- *     row split over CTAs is clamped to what the array holds (one partial tile
- *     per CTA): small outputs run as wide as dpclip_clipped_grad, an output at
- *     the limit with a bias runs unsplit (one CTA per 256 x 256 tile, slower);
+ *     row split over SMs is clamped to what the array holds (one partial tile
+ *     per output tile and one per run of rows): small outputs run as wide as
+ *     dpclip_clipped_grad, an output at the limit on a fifth of the SMs;
  *   - no device memory is allocated or freed by this call, on any path;
  *   - the first call on each device looks up the array's device address (that
  *     device must be current); make that first call outside any stream capture;
@@ -404,10 +404,12 @@ int dpclip_gram_layers_sqnorms(const dpclip_layer* layers /* host */, int L, int
                                void* workspace, size_t workspace_bytes, void* stream);
 
 /* Clipped sums with noise (Eq. 1 applied to the sum over examples of c_i Zbar_i^T A_i, Algorithm 1's
- * last two steps) of layers that have ONE shape, taken together: bf16 layers with T > 1, equal
- * (T, d_in, d_out), rows TMA can address, dense output rows and d_in a multiple of 4 run as one
- * tensor-core launch plus one reduce launch per group of two to eight layers (e.g. the four
- * attention projections of a Transformer block).  Results and noise streams are those of
+ * last two steps) of layers taken together: bf16 layers with T > 1, rows TMA can address, dense output
+ * rows and d_in a multiple of 4.  Layers with ONE T and d_out wide enough for 512-row tiles (d_out >
+ * 256 and little padding) share a launch whatever their shapes, up to eight at a time: their tiles'
+ * work is cut into equal runs over all pairs of SMs (needs the workspace dpclip_step_workspace_bytes
+ * reports).  Other layers share a launch when they have ONE shape (T, d_in, d_out) and would be short
+ * on their own.  Each launch is followed by one reduce launch that adds the noise.  Results and noise streams are those of
  * dpclip_step: layer l of the array draws from streams stream_id0 + 2l (weights) and + 2l + 1
  * (bias).  taken (host, [L], required) is set to 1 for the layers that were handled; the caller
  * runs dpclip_clipped_grad_noise on the others.  Nothing qualifies: nothing is launched.  The
@@ -448,6 +450,13 @@ size_t dpclip_step_host_arena_bytes(const dpclip_layer* layers /* host */, int L
  * workspace of at least the 39 MB form is accepted: the layer then runs as one
  * wave. */
 size_t dpclip_workspace_bytes(int B, int T, int d_in, int d_out, dpclip_dtype dtype, dpclip_method method);
+
+/* Workspace for dpclip_step / dpclip_step_streams / dpclip_step_per_layer over these layers: the largest
+ * per-layer need, and room for the launches several layers share (bf16 layers of one T whose d_out is wide
+ * enough for 512-row tiles go into one clipped-sum launch: one fp32 partial tile of 512 x 256 per output tile
+ * of all of them and one per pair of SMs).  With less (but at least the per-layer needs) the step still
+ * runs, those layers in launches of their own. */
+size_t dpclip_step_workspace_bytes(const dpclip_layer* layers /* host */, int L, int B, dpclip_dtype dtype);
 
 /* Zero the 256-byte status header.  Call once after allocating a workspace. */
 int dpclip_workspace_init(void* workspace, size_t workspace_bytes, void* stream);

@@ -119,6 +119,8 @@ def load_library():
     L.dpclip_model_workspace_bytes.restype = _sz
     L.dpclip_workspace_bytes.argtypes = [_i, _i, _i, _i, _i, _i]
     L.dpclip_workspace_bytes.restype = _sz
+    L.dpclip_step_workspace_bytes.argtypes = [ctypes.POINTER(_CLayer), _i, _i, _i]
+    L.dpclip_step_workspace_bytes.restype = _sz
     L.dpclip_workspace_init.argtypes = [_vp, _sz, _vp]
     L.dpclip_read_status.argtypes = [_vp, ctypes.POINTER(_i), _vp]
     L.dpclip_pick_method.argtypes = [_i, _i, _i, _i, _l, _l, _i]
@@ -339,7 +341,6 @@ class StepPlan:
         self.gW: List[torch.Tensor] = []
         self.gb: List[Optional[torch.Tensor]] = []
         self._c = (_CLayer * self.L)()
-        ws = 256
         # all outputs live in one flat fp32 buffer (each tensor starts on a 256-byte boundary), so a
         # data-parallel caller can all-reduce the whole gradient with one collective
         offs, total = [], 0
@@ -359,7 +360,7 @@ class StepPlan:
             self.gW.append(gW); self.gb.append(gb)
             self._c[l] = _CLayer(_ptr(y.A), lda, _ptr(y.Zbar), ldz, T, d_in, d_out, int(y.has_bias),
                                  y.method, _ptr(gW), d_in, _ptr(gb))
-            ws = max(ws, dpclip_workspace_bytes(B, T, d_in, d_out, self.dtype_code, y.method))
+        ws = dpclip_step_workspace_bytes(self)
         self.sq_layers = torch.empty((self.L, self.B), dtype=torch.float32, device=dev)
         self.clip = torch.empty((self.B,), dtype=torch.float32, device=dev)
         self.norms = torch.empty((self.B,), dtype=torch.float32, device=dev)
@@ -509,6 +510,11 @@ def dpclip_same_shape_layers_clipped_grad_noise(plan: StepPlan, C: float, sigma:
 def dpclip_t1_layers_supported(plan: StepPlan) -> bool:
     """Whether the library takes the plan's T = 1 layers together (nothing is launched)."""
     return bool(load_library().dpclip_t1_layers_supported(plan._c, plan.L, plan.B, plan.dtype_code))
+
+
+def dpclip_step_workspace_bytes(plan) -> int:
+    """Workspace for whole-step calls over the plan's layers (per-layer needs and shared launches)."""
+    return load_library().dpclip_step_workspace_bytes(plan._c, plan.L, plan.B, plan.dtype_code)
 
 
 def dpclip_step(plan: StepPlan, C: float, sigma: float, seed: int, stream_id0: int = 0, stream=None) -> None:

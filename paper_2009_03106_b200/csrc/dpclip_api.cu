@@ -8,6 +8,7 @@
 #include "kernels_simt.cuh"
 #include "kernels_stream.cuh"
 #include "kernels_tc.cuh"
+#include "kernels_tc_pair.cuh"
 #include "kernels_fused_t1_tf32.cuh"
 #include "kernels_tf32.cuh"
 #include "kernels_fused_t1.cuh"
@@ -44,7 +45,7 @@ enum PathSwitch : unsigned {
     SW_FORCE_SIMT = 1u << 0, SW_NO_NARROW = 1u << 1, SW_NO_NARROW_RING = 1u << 2, SW_NO_NARROW_TC = 1u << 3,
     SW_NO_NARROW_PACK = 1u << 4, SW_NARROW_PACK_BF16 = 1u << 5, SW_NO_GRAM_Q2 = 1u << 6, SW_NO_T1_TF32 = 1u << 7,
     SW_NO_FUSED_T1 = 1u << 8, SW_NO_GRAM_GROUP = 1u << 9, SW_NO_GRAD_GROUP = 1u << 10, SW_NO_CONV_TC = 1u << 11,
-    SW_NO_CONV_PATCHES = 1u << 12, SW_TILE_M1 = 1u << 13, SW_TILE_M2 = 1u << 14, SW_T1_TWO_LAUNCHES = 1u << 15,
+    SW_NO_CONV_PATCHES = 1u << 12, SW_TILE_M1 = 1u << 13, SW_TILE_M2 = 1u << 14, SW_T1_TWO_LAUNCHES = 1u << 15, SW_NO_PAIR = 1u << 16,
     SW_LOADED = 1u << 31
 };
 std::atomic<unsigned> g_path_switches{0};
@@ -58,6 +59,7 @@ unsigned read_path_switches() {
         {"DPCLIP_NO_GRAD_GROUP", SW_NO_GRAD_GROUP, '1'}, {"DPCLIP_NO_CONV_TC", SW_NO_CONV_TC, '1'},
         {"DPCLIP_NO_CONV_PATCHES", SW_NO_CONV_PATCHES, '1'}, {"DPCLIP_TILE_M", SW_TILE_M1, '1'},
         {"DPCLIP_TILE_M", SW_TILE_M2, '2'}, {"DPCLIP_T1_ONE_LAUNCH", SW_T1_TWO_LAUNCHES, '0'},
+        {"DPCLIP_NO_PAIR", SW_NO_PAIR, '1'},
     };
     unsigned v = SW_LOADED;
     for (const auto& e : table) {
@@ -496,15 +498,15 @@ constexpr size_t kTcScratchBytes = (size_t)kNumSMs * 256 * 256 * 4 + (size_t)2 *
 //               stay below 4 % of an item), the smallest split whose items fill whole waves to >= 97 %; it
 //               needs one partial tile per item, which the workspace query reports for the layer.
 struct ZtaSplit { int one_wave, preferred; };
-inline ZtaSplit zta_pick_split(long nkb, int tiles, int per_sm) {
+inline ZtaSplit zta_pick_split(long nkb, int tiles, int per_sm, int slots = kNumSMs) {
     ZtaSplit r;
-    long base = ((long)per_sm * kNumSMs) / tiles;
+    long base = ((long)per_sm * slots) / tiles;
     if (base > nkb) base = nkb;
     if (base < 1) base = 1;
     r.one_wave = r.preferred = (int)base;
     auto fill = [&](long ks) {
-        const long items = (long)tiles * ks, waves = (items + kNumSMs - 1) / kNumSMs;
-        return (double)items / (double)(waves * kNumSMs);
+        const long items = (long)tiles * ks, waves = (items + slots - 1) / slots;
+        return (double)items / (double)(waves * slots);
     };
     double best = fill(base);
     if (per_sm != 1 || best >= 0.95) return r;
@@ -621,6 +623,146 @@ int launch_zta_tc_mt(const tc::zta::Maps& maps, tc::zta::Params p, int B, bool n
     return launch_reduce_partials(p, tiles, ksplit, BM, z::BN, d_in, d_out, gW, ldg, gb, noise, noise_done, st, grp);
 }
 
+// Clipped sums on CTA pairs (zta_pair_kernel): 512 x 256 tiles, the (tile, stage) units of all layers of the
+// launch cut into equal runs, one per pair.  A layer qualifies when the padding of d_out to 512-row pair tiles
+// costs at most a tenth more than its padding to 256-row tiles.
+constexpr int kNumPairs = kNumSMs / 2;
+inline bool pair_tile_ok(int d_out) {
+    if (path_switch(SW_NO_PAIR) || d_out <= 256) return false;
+    const double pad_pair = (double)ceil_div(d_out, 512) * 512, pad_single = (double)ceil_div(d_out, 256) * 256;
+    return pad_pair <= 1.1 * pad_single;
+}
+inline int pair_tiles(int d_in, int d_out) { return ceil_div(d_out, tc::ztp::BM) * ceil_div(d_in, tc::ztp::BN); }
+inline size_t pair_segment_bytes(bool bias) {
+    return tc::ztp::SEG_ELEMS * 4 + (bias ? (size_t)tc::ztp::BM * 4 : 0);
+}
+// scratch for a launch over `tiles` pair tiles with every pair busy: one segment per tile position of every
+// super-layer (at most tiles + 15 positions when narrow layers leave a super-layer part empty) and one per pair
+inline size_t pair_scratch_bytes(int tiles) { return (size_t)(tiles + 16 + kNumPairs) * pair_segment_bytes(true); }
+inline long gcd_l(long a, long b) { while (b) { const long t = a % b; a = b; b = t; } return a; }
+
+struct StreamLayer {
+    const void* A; long lda; const void* Z; long ldz; int d_in, d_out;
+    float* gW; long ldg; float* gb; unsigned long long sid_w, sid_b;
+};
+
+// Returns DPCLIP_OK, a negative status, or 1 when the workspace cannot hold even one segment per tile (the
+// caller then takes another path).
+int launch_zta_stream(const StreamLayer* ls, int n, int B, int T, const float* clip, const NoiseSpec* noise,
+                      bool* noise_done, void* workspace, size_t workspace_bytes, cudaStream_t st) {
+    namespace zp = tc::ztp;
+    if (n < 1 || n > zp::MAX_LAYERS) return 1;
+    const long R = (long)B * T;
+    tc::zta::Maps maps;
+    zp::Params p;
+    memset(&p, 0, sizeof(p));
+    p.R = (int)R; p.T = T; p.S = (int)ceil_div(R, (long)zp::BK); p.n_layers = n;
+    p.clip = clip; p.status = static_cast<int*>(workspace);
+    bool fuse_noise = noise && noise->scale > 0.f;
+    int G = 0;
+    for (int l = 0; l < n; ++l) {
+        const StreamLayer& y = ls[l];
+        if (!make_map_bf16(&maps.a[l], y.A, R, y.d_in, y.lda, 64, zp::BK) ||
+            !make_map_bf16(&maps.z[l], y.Z, R, y.d_out, y.ldz, 64, zp::BK))
+            return DPCLIP_ERR_CUDA;
+        zp::Layer& q = p.layer[l];
+        q.d_in = y.d_in; q.d_out = y.d_out;
+        q.tiles_n = ceil_div(y.d_in, zp::BN);
+        q.tile_base = G; q.tiles = pair_tiles(y.d_in, y.d_out);
+        G += q.tiles;
+        q.do_bias = y.gb ? 1 : 0;
+        q.gW = y.gW; q.gb = y.gb; q.ldg = y.ldg;
+        q.vec_ok = aligned_to(y.gW, 16) && y.ldg % 4 == 0;
+        q.sw0 = (uint32_t)y.sid_w; q.sw1 = (uint32_t)(y.sid_w >> 32);
+        q.sb0 = (uint32_t)y.sid_b; q.sb1 = (uint32_t)(y.sid_b >> 32);
+        if (y.gb) p.any_bias = 1;
+        // the noise of element j is indexed by its position in the dense tensor, one Philox block per float4
+        if (y.ldg != y.d_in || y.d_in % 4 != 0) fuse_noise = false;
+    }
+    p.G = G;
+    if (G > zp::MAX_TILES) return 1;
+    // Gang width: the widest W <= 16 for which every layer either splits into whole super-layers (tiles % W == 0)
+    // or is narrower than W (narrow layers are packed side by side), and whose gangs and super-layers leave at
+    // most a tenth of the pairs idle; else W = 1 (tile-major, no sharing of rows between tiles).
+    int W = 1, n_super = G;
+    for (int w = 16; w >= 2; --w) {
+        bool ok = true;
+        int supers = 0, open_fill = 0;              // narrow layers: first fit into the open super-layer
+        for (int l = 0; l < n && ok; ++l) {
+            const int t = p.layer[l].tiles;
+            if (t >= w) { ok = t % w == 0; supers += t / w; }
+            else if (open_fill > 0 && open_fill + t <= w) open_fill += t;
+            else { ++supers; open_fill = t; }
+        }
+        if (!ok || (long)supers * w > zp::MAX_TILES) continue;
+        const double use = (double)(kNumPairs / w) * w / kNumPairs * ((double)G / ((double)supers * w));
+        if (use >= 0.9) { W = w; n_super = supers; break; }
+    }
+    p.W = W; p.n_super = n_super;
+    for (int i = 0; i < zp::MAX_TILES; ++i) { p.super_tile[i] = -1; p.tile_slot[i] = 0; }
+    {
+        int next_super = 0, open_super = -1, open_fill = 0;
+        for (int l = 0; l < n; ++l) {
+            const zp::Layer& q = p.layer[l];
+            if (q.tiles >= W) {
+                for (int t = 0; t < q.tiles; ++t) {
+                    const int sl = next_super + t / W, j = t % W;
+                    p.super_tile[sl * W + j] = (short)(q.tile_base + t);
+                    p.tile_slot[q.tile_base + t] = (short)(sl * W + j);
+                }
+                next_super += q.tiles / W;
+            } else {
+                if (open_super < 0 || open_fill + q.tiles > W) { open_super = next_super++; open_fill = 0; }
+                for (int t = 0; t < q.tiles; ++t) {
+                    p.super_tile[open_super * W + open_fill + t] = (short)(q.tile_base + t);
+                    p.tile_slot[q.tile_base + t] = (short)(open_super * W + open_fill + t);
+                }
+                open_fill += q.tiles;
+            }
+        }
+        if (next_super != n_super || (long)n_super * W > zp::MAX_TILES) return 1;
+    }
+    p.total = (long)n_super * p.S;
+    // equal runs over all gangs; runs shorter than eight stages would be mostly set-up and drain
+    const size_t seg_bytes = pair_segment_bytes(p.any_bias != 0);
+    const size_t room = workspace && workspace_bytes > (size_t)kHeaderBytes ? workspace_bytes - kHeaderBytes : 0;
+    const long max_segments = (long)(room / seg_bytes) / W;          // per gang position
+    if (max_segments < n_super) return 1;
+    long U = ceil_div(p.total, (long)(kNumPairs / W));
+    if (U < 8) U = p.total < 8 ? p.total : 8;
+    // a small workspace (the fixed array of the entry point without one) limits the number of runs
+    while (zp::segment_of(p.total - 1, p.S, (int)U, (long)p.S / gcd_l(p.S, U) * U) + 1 > max_segments) {
+        const long runs = ceil_div(p.total, U);
+        if (runs <= 1) return 1;
+        U = ceil_div(p.total, runs - 1);
+    }
+    p.U = (int)U;
+    p.lcm = (long)p.S / gcd_l(p.S, U) * U;
+    const long n_segments = (zp::segment_of(p.total - 1, p.S, p.U, p.lcm) + 1) * W;
+    p.part = reinterpret_cast<float*>(static_cast<char*>(workspace) + kHeaderBytes);
+    p.bias_part = p.any_bias ? p.part + (size_t)n_segments * zp::SEG_ELEMS : nullptr;
+    if (fuse_noise) {
+        p.noise_scale = noise->scale;
+        p.k0 = (uint32_t)noise->seed; p.k1 = (uint32_t)(noise->seed >> 32);
+        if (noise_done) *noise_done = true;
+    }
+    if (!enable_smem(tc::zta_pair_kernel, zp::SMEM_BYTES)) return DPCLIP_ERR_CUDA;
+    const int pairs = (int)ceil_div(p.total, U) * W;
+    tc::zta_pair_kernel<<<2 * pairs, zp::THREADS, zp::SMEM_BYTES, st>>>(maps, p);
+    int rc = launch_status();
+    if (rc) return rc;
+    long most = 0;
+    for (int l = 0; l < n; ++l) {
+        const long v = (long)ls[l].d_out * ((ls[l].d_in + 3) / 4);
+        if (v > most) most = v;
+    }
+    long blocks = ceil_div(most, 256L);
+    if (blocks > 4L * kNumSMs) blocks = 4L * kNumSMs;
+    if (blocks < 1) blocks = 1;
+    tc::reduce_segments_kernel<<<dim3((unsigned)blocks, n), 256, 0, st>>>(p);
+    return launch_status();
+}
+
 int launch_zta_tc(const void* A, long lda, const void* Z, long ldz, int B, int T, int d_in, int d_out,
                   bool norm_mode, int has_bias, const float* clip, float* gW, long ldg, float* gb, float* sq,
                   void* workspace, size_t workspace_bytes, const NoiseSpec* noise, bool* noise_done,
@@ -630,6 +772,7 @@ int launch_zta_tc(const void* A, long lda, const void* Z, long ldz, int B, int T
     int mt = d_out > 128 ? 2 : 1;
     if (path_switch(SW_TILE_M1)) mt = 1;
     if (path_switch(SW_TILE_M2)) mt = 2;
+    const bool pair = !norm_mode && mt == 2 && pair_tile_ok(d_out);
     const int bk = mt == 2 ? z::Cfg<2>::BK : z::Cfg<1>::BK;           // rows of a TMA box = rows of a stage
     z::Maps maps;
     if (!make_map_bf16(&maps.a[0], A, R, d_in, lda, 64, bk) || !make_map_bf16(&maps.z[0], Z, R, d_out, ldz, 64, bk))
@@ -646,6 +789,11 @@ int launch_zta_tc(const void* A, long lda, const void* Z, long ldz, int B, int T
         p.clip = clip; p.gW = gW; p.ldg = ldg; p.gb = gb;
         p.do_bias = gb ? 1 : 0;
         p.vec_ok = aligned_to(gW, 16) && ldg % 4 == 0;
+    }
+    if (pair) {
+        const StreamLayer one = {A, lda, Z, ldz, d_in, d_out, gW, ldg, gb, noise ? noise->sid_w : 0ull, noise ? noise->sid_b : 0ull};
+        const int rc = launch_zta_stream(&one, 1, B, T, clip, noise, noise_done, workspace, workspace_bytes, st);
+        if (rc <= 0) return rc;                 // 1: not even one segment per tile fits -> the single-CTA kernel below
     }
     if (mt == 2)
         return launch_zta_tc_mt<2>(maps, p, B, norm_mode, gW, ldg, gb, sq, d_in, d_out, workspace, workspace_bytes,
@@ -1055,11 +1203,46 @@ size_t dpclip_workspace_bytes(int B, int T, int d_in, int d_out, dpclip_dtype dt
             const ZtaSplit split = zta_pick_split(ceil_div((long)B * T, 64L), tiles, 1);
             const size_t pref = zta_scratch_bytes(tiles, split.preferred, 256, true);
             if (split.preferred != split.one_wave && pref > need) need = pref;
+            if (pair_tile_ok(d_out)) {                 // the CTA-pair kernel: one segment per tile and one per pair
+                const size_t pneed = pair_scratch_bytes(pair_tiles(d_in, d_out));
+                if (pneed > need) need = pneed;
+            }
         }
         return kHeaderBytes + need;
     }
     if ((double)B * T * d_in * d_out >= 32.0 * 1024 * 1024) return kHeaderBytes + kTcScratchBytes;
     return (size_t)kHeaderBytes;
+}
+
+size_t dpclip_step_workspace_bytes(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype) {
+    size_t ws = kHeaderBytes;
+    if (!layers || L <= 0 || B <= 0) return ws;
+    for (int l = 0; l < L; ++l) {
+        const dpclip_layer& y = layers[l];
+        if (y.T <= 0) continue;
+        const size_t w = dpclip_workspace_bytes(B, y.T, y.d_in, y.d_out, dtype, (dpclip_method)y.method);
+        if (w > ws) ws = w;
+    }
+    if (dtype != DPCLIP_BF16 || path_switch(SW_NO_GRAD_GROUP)) return ws;
+    // layers of one T that share a CTA-pair launch (up to eight): one segment per tile of all of them + one per pair
+    for (int l0 = 0; l0 < L; ++l0) {
+        const dpclip_layer& y0 = layers[l0];
+        if (y0.T <= 1 || !pair_tile_ok(y0.d_out)) continue;
+        bool first = true;
+        for (int l = 0; l < l0; ++l) first = first && !(layers[l].T == y0.T && pair_tile_ok(layers[l].d_out));
+        if (!first) continue;
+        int n = 0, tiles = 0;
+        for (int l = l0; l < L; ++l) {
+            if (layers[l].T != y0.T || !pair_tile_ok(layers[l].d_out)) continue;
+            tiles += pair_tiles(layers[l].d_in, layers[l].d_out);
+            if (++n == tc::ztp::MAX_LAYERS) {
+                if (kHeaderBytes + pair_scratch_bytes(tiles) > ws) ws = kHeaderBytes + pair_scratch_bytes(tiles);
+                n = 0; tiles = 0;
+            }
+        }
+        if (n >= 2 && kHeaderBytes + pair_scratch_bytes(tiles) > ws) ws = kHeaderBytes + pair_scratch_bytes(tiles);
+    }
+    return ws;
 }
 
 int dpclip_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
@@ -1179,6 +1362,35 @@ int dpclip_same_shape_layers_clipped_grad_noise(const dpclip_layer* layers, int 
         if (!aligned_to(y.gW, 4) || (y.has_bias && !aligned_to(y.gb, 4))) return false;
         return tc_eligible(y.A, y.lda, y.Zbar, y.ldz, dtype);
     };
+    // Layers wide enough for the CTA-pair kernel need not have one shape: all that have one T (hence the same
+    // rows B*T) go into one stream-K launch, up to eight at a time.
+    for (int l0 = 0; l0 < L; ++l0) {
+        if (done[l0] || !candidate(layers[l0]) || !pair_tile_ok(layers[l0].d_out)) continue;
+        StreamLayer grp[tc::ztp::MAX_LAYERS];
+        int idx[tc::ztp::MAX_LAYERS];
+        int n = 0, tiles = 0;
+        for (int l = l0; l < L && n < tc::ztp::MAX_LAYERS; ++l) {
+            const dpclip_layer& y = layers[l];
+            if (done[l] || y.T != layers[l0].T || !pair_tile_ok(y.d_out) || !candidate(y)) continue;
+            grp[n] = {y.A, y.lda, y.Zbar, y.ldz, y.d_in, y.d_out, y.gW, y.ldg, y.has_bias ? y.gb : nullptr,
+                      stream_id0 + 2ull * l, stream_id0 + 2ull * l + 1};
+            idx[n] = l; ++n;
+            tiles += pair_tiles(y.d_in, y.d_out);
+        }
+        if (n < 2) continue;                       // a single layer takes the same kernel through its own call
+        // with less workspace than one segment per tile and pair the launch would run on fewer pairs: leave the
+        // layers to their own launches then
+        if (workspace_bytes < kHeaderBytes + pair_scratch_bytes(tiles)) continue;
+        const NoiseSpec ns = {sigma * C, seed, 0, 0};
+        bool noise_done = false;
+        const int rc = launch_zta_stream(grp, n, B, layers[l0].T, clip, &ns, &noise_done, workspace, workspace_bytes,
+                                         (cudaStream_t)stream);
+        if (rc < 0) return rc;
+        if (rc > 0) continue;
+        if (sigma * C > 0.f && !noise_done) return DPCLIP_ERR_UNSUPPORTED;    // candidate() checked dense rows, d_in % 4
+        if (!taken) return DPCLIP_ERR_INVALID_ARG;               // without `taken` the caller cannot know
+        for (int i = 0; i < n; ++i) { done[idx[i]] = true; taken[idx[i]] = 1; }
+    }
     for (int l0 = 0; l0 < L; ++l0) {
         if (done[l0] || !candidate(layers[l0])) continue;
         const dpclip_layer* grp[z::MAX_LAYERS];
@@ -1993,7 +2205,15 @@ int dpclip_step_per_layer(const dpclip_layer* layers, int L, int B, dpclip_dtype
 
 size_t dpclip_model_workspace_bytes(const dpclip_model_layer* layers, int L, int B, dpclip_dtype dtype) {
     size_t ws = kHeaderBytes;
-    if (!layers || L <= 0 || B <= 0) return ws;
+    if (!layers || L <= 0 || L > 256 || B <= 0) return ws;
+    {
+        dpclip_layer dense[256];
+        for (int l = 0; l < L; ++l) {
+            if (layers[l].kind == DPCLIP_KIND_DENSE) dense[l] = layers[l].layer;
+            else memset(&dense[l], 0, sizeof(dense[l]));
+        }
+        ws = dpclip_step_workspace_bytes(dense, L, B, dtype);
+    }
     for (int l = 0; l < L; ++l) {
         const dpclip_layer& y = layers[l].layer;
         size_t w = kHeaderBytes;
@@ -2030,11 +2250,9 @@ int dpclip_model_step_streams(const dpclip_model_layer* layers, int L, int B, dp
 size_t dpclip_step_host_arena_bytes(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype) {
     if (!layers || L <= 0 || B <= 0) return 0;
     const size_t es = elt_size(dtype);
-    size_t ws = kHeaderBytes, total = 0;
+    size_t ws = dpclip_step_workspace_bytes(layers, L, B, dtype), total = 0;
     for (int l = 0; l < L; ++l) {
         const dpclip_layer& y = layers[l];
-        size_t w = dpclip_workspace_bytes(B, y.T, y.d_in, y.d_out, dtype, (dpclip_method)y.method);
-        if (w > ws) ws = w;
         total += round_up((size_t)B * y.T * y.d_in * es, 256);
         total += round_up((size_t)B * y.T * y.d_out * es, 256);
         total += round_up((size_t)y.d_out * y.d_in * 4, 256);
@@ -2056,13 +2274,11 @@ int dpclip_step_host(const dpclip_layer* layers, int L, int B, dpclip_dtype dtyp
     char* cur = static_cast<char*>(arena);
     auto take = [&](size_t bytes) { char* p = cur; cur += round_up(bytes, 256); return (void*)p; };
 
-    size_t ws_bytes = kHeaderBytes;
+    const size_t ws_bytes = dpclip_step_workspace_bytes(layers, L, B, dtype);
     for (int l = 0; l < L; ++l) {
         const dpclip_layer& y = layers[l];
         if (y.lda != y.d_in || y.ldz != y.d_out || y.ldg != y.d_in) return DPCLIP_ERR_INVALID_ARG;
         if (!y.A || !y.Zbar || !y.gW || (y.has_bias && !y.gb)) return DPCLIP_ERR_INVALID_ARG;
-        size_t w = dpclip_workspace_bytes(B, y.T, y.d_in, y.d_out, dtype, (dpclip_method)y.method);
-        if (w > ws_bytes) ws_bytes = w;
     }
     void* ws = take(ws_bytes);
     float* sq = (float*)take((size_t)L * B * 4);
@@ -2178,10 +2394,9 @@ int dpclip_clipped_grad_noalloc(const void* A, long lda, const void* Zbar, long 
     if (rc) return rc;
     if (!gW || ldg < d_in) return DPCLIP_ERR_INVALID_ARG;
     if (!aligned_to(gW, 4) || (gb && !aligned_to(gb, 4))) return DPCLIP_ERR_MISALIGNED;
-    // The output, padded to 256 x 256 tiles, may take at most half of the array.  Without a bias that leaves
-    // room for two partial copies; a bias adds 1 KB per partial tile, so at the very limit only one copy fits
-    // and the row split is clamped to 1: every tile then has a single CTA that stores straight to gW (bias by
-    // red.add), which is correct but uses one SM per tile.
+    // The output, padded to 256 x 256 tiles, may take at most half of the array: room for one partial tile per
+    // output tile and about as many again for the row split, which is clamped to what the array holds (at the
+    // limit: 16 tiles of 512 x 256, 31 partial tiles, so 15 pairs of SMs instead of 74 -- correct, slower).
     const size_t padded = (size_t)ceil_div(d_out, 256) * 256 * ((size_t)ceil_div(d_in, 256) * 256) * 4;
     if (padded > dpclip_noalloc_max_output_bytes()) return DPCLIP_ERR_WORKSPACE;
     void* scratch = static_scratch_for_current_device(&rc);

@@ -87,7 +87,9 @@ def test_streams_step_argument_errors(lib):
     """dpclip_step_streams checks its stream and workspace arrays on the host before anything is enqueued."""
     fake = ctypes.c_void_p(0x1000)
     INVALID = -1
-    f = lib.dpclip_step_streams
+    from paper_2009_03106_b200 import binding
+    own = ctypes.CDLL(binding.library_path())      # a handle of its own: the prototypes set here stay out of the binding's
+    f = own.dpclip_step_streams
     f.restype = ctypes.c_int
     vp = ctypes.c_void_p
 
@@ -115,13 +117,19 @@ def test_workspace_queries_without_a_gpu(lib):
     """The workspace queries are host arithmetic: the fixed scratch for ordinary layers, room for one partial
     tile per row slice for long bf16 layers whose 64 tiles leave SMs idle in one wave, and the copies of the
     fp32 feature-map convolution routes."""
+    from paper_2009_03106_b200 import binding
+    lib = ctypes.CDLL(binding.library_path())      # own handle, own prototypes
     lib.dpclip_workspace_bytes.restype = ctypes.c_size_t
     lib.dpclip_workspace_bytes.argtypes = [ctypes.c_int] * 6
     floor = lib.dpclip_workspace_bytes(1, 1, 1, 1, 1, 0)
-    assert lib.dpclip_workspace_bytes(128, 256, 512, 2048, 1, 0) == floor           # 16 tiles x 9 slices = one wave
-    assert lib.dpclip_workspace_bytes(256, 128, 1024, 4096, 1, 0) == floor          # 64 tiles, too short to re-cut
+    assert lib.dpclip_workspace_bytes(128, 256, 512, 128, 1, 0) == floor            # narrow d_out: one partial tile per SM
+    # d_out wide enough for the CTA-pair kernel: one 512 x 256 segment (+ 512 bias sums) per tile (+ 16 for part-empty super-layers) and one per pair
+    seg = 512 * 256 * 4 + 512 * 4
+    assert lib.dpclip_workspace_bytes(128, 256, 512, 2048, 1, 0) == 256 + (8 + 16 + 74) * seg
+    assert lib.dpclip_workspace_bytes(256, 128, 1024, 4096, 1, 0) == 256 + (32 + 16 + 74) * seg
+    # 64 tiles of 256 x 256 and long rows: the single-CTA kernel's preferred cut (9 slices per tile) is larger still
     long64 = lib.dpclip_workspace_bytes(256, 2048, 1024, 4096, 1, 0)
-    assert long64 == 256 + 64 * 9 * (256 * 256 * 4 + 256 * 4)                       # 9 slices per tile
+    assert long64 == 256 + 64 * 9 * (256 * 256 * 4 + 256 * 4)
     assert lib.dpclip_workspace_bytes(32, 1, 784, 256, 0, 0) == 256                 # small fp32 layer: header only
 
     class Conv(ctypes.Structure):

@@ -112,8 +112,12 @@ def test_tensor_core_norms_run_twice_identically_shaped(dp):
         assert max_rel(np.sqrt(got), np.sqrt(ref)) <= 2e-5
 
 
+# the shapes with d_out = 500 ... 1024 take the CTA-pair kernel (512 x 256 tiles): exact and ragged tiles, short
+# examples (a factor per row), a single stage (one item per tile: direct stores), several row slices
 @pytest.mark.parametrize("B,T,d_in,d_out", [(128, 1, 512, 256), (4, 256, 512, 256), (3, 100, 264, 136),
-                                            (2, 2048, 64, 64), (16, 64, 576, 128)])
+                                            (2, 2048, 64, 64), (16, 64, 576, 128), (4, 256, 512, 512),
+                                            (3, 100, 264, 500), (2, 300, 200, 1000), (40, 33, 72, 512),
+                                            (1, 16, 64, 512), (24, 128, 128, 1024)])
 def test_tensor_core_clipped_grad(dp, B, T, d_in, d_out):
     A, Z = workloads.random_layer(8, B, T, d_in, d_out, "bf16", scale_z=0.05)
     clip = np.random.default_rng(B).uniform(0.05, 1.0, B).astype(np.float32)

@@ -50,8 +50,8 @@ def test_no_alloc_entry_matches_workspace_entry_twice_in_a_row(dp):
 
 
 def test_no_alloc_entry_at_the_size_limit_with_a_bias(dp):
-    # the largest output the entry point accepts (8 MB padded), with a bias: one partial copy no longer fits
-    # next to the bias sums, so the row split is clamped to 1 and every tile is stored by a single CTA
+    # the largest output the entry point accepts (8 MB padded), with a bias: the fixed array holds 31 partial
+    # tiles of 512 x 256 for the 16 output tiles, so the row split is clamped far below the usual one
     ref_W, got_W, ref_b, got_b = _both(dp, 3, 96, 2048, 1024, "bf16", 5)
     assert rel_fro(got_W, ref_W) <= 1e-5 and rel_fro(got_b, ref_b) <= 1e-5
     # and twice in a row on the same shape with other data
