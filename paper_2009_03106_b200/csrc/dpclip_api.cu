@@ -1956,12 +1956,12 @@ struct Lanes {
     cudaStream_t st[kMax] = {};
     void* ws[kMax] = {};
     size_t ws_bytes = 0;
-    cudaEvent_t ev[2 * kMax] = {};
+    cudaEvent_t ev[2 * kMax + 2] = {};
     int n_ev = 0;
     ~Lanes() { for (int i = 0; i < n_ev; ++i) cudaEventDestroy(ev[i]); }     // pending work keeps what it needs
     // events are reused between the fork and the join of a stage: a record replaces the earlier one for later waits only
     int event(cudaEvent_t* out) {
-        if (n_ev == 2 * kMax) return DPCLIP_ERR_CUDA;
+        if (n_ev == 2 * kMax + 2) return DPCLIP_ERR_CUDA;
         if (cudaEventCreateWithFlags(&ev[n_ev], cudaEventDisableTiming) != cudaSuccess) return DPCLIP_ERR_CUDA;
         *out = ev[n_ev++];
         return DPCLIP_OK;

@@ -33,11 +33,12 @@
 // 8 transform warps: scale this CTA's A half by the row's factor (bf16, one rounding), then arrive on rank
 // 0's `ready` barrier (a remote arrive for rank 1); 8 epilogue warps: during the main loop (when a layer of
 // the launch has a bias) the column sums sum_rows c * zb straight from the untouched Zb tile, in fp32, for the
-// stages dealt to this n-tile -- in parallel with the transform warps, arriving on `ready` as well -- and at
-// the end of a segment the drain of this CTA's accumulator (256 d_out rows x 256 d_in columns fp32 = all 512
-// tensor-memory columns).
-// Barriers: full[s] (local, TMA bytes) -> ready[s] (in rank 0, 16 or 32 warp arrivals from both CTAs) -> MMAs
-// -> empty[s] / acc_full (tcgen05.commit with an arrival in BOTH CTAs) -> acc_empty (in rank 0, 16 arrivals).
+// stages dealt to this n-tile -- beside the transform warps and the MMAs: they only hold up the REFILL of the
+// stage (`zfree`, local) -- and at the end of a segment the drain of this CTA's accumulator (256 d_out rows x
+// 256 d_in columns fp32 = all 512 tensor-memory columns).
+// Barriers: full[s] (local, TMA bytes) -> ready[s] (in rank 0, 16 warp arrivals from both CTAs) -> MMAs
+// -> empty[s] / acc_full (tcgen05.commit with an arrival in BOTH CTAs) -> acc_empty (in rank 0, 16 arrivals);
+// the producer refills stage s after empty[s] and zfree[s].
 // Every wait is bounded; a CTA that gives up sets the status word, unwinds, and still takes part in the
 // closing cluster barrier, so its partner neither waits for ever nor touches shared memory of a CTA that
 // has exited.
@@ -101,6 +102,8 @@ struct Params {
     Layer layer[MAX_LAYERS];
 };
 
+__device__ __forceinline__ float row_factor(const Params& p, int e) { return p.clip ? __ldg(p.clip + e) : 1.f; }
+
 __host__ __device__ __forceinline__ long segment_of(long u, int S, int U, long lcm) { return u / S + u / U - u / lcm; }
 
 struct Seg { int layer, m0, n0, tn, kb0, kb1; long slot; };       // layer < 0: this pair has no tile in the segment
@@ -141,7 +144,8 @@ zta_pair_kernel(const __grid_constant__ zta::Maps maps, const __grid_constant__ 
     uint64_t* empty = ready + STAGES;                                            // MMAs done with the stage (each CTA's own)
     uint64_t* acc_full = empty + STAGES;                                         // accumulator complete (each CTA's own)
     uint64_t* acc_empty = acc_full + 1;                                          // accumulator drained (rank 0's is used)
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 1);
+    uint64_t* zfree = acc_empty + 1;                                             // bias warps done reading the Zb tile (own)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(zfree + STAGES);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     float4* out_stage = reinterpret_cast<float4*>(smem + STAGES * STAGE_BYTES + 256);
 
@@ -152,10 +156,12 @@ zta_pair_kernel(const __grid_constant__ zta::Maps maps, const __grid_constant__ 
     const long u_begin = min((long)gang * p.U, p.total), u_end = min(u_begin + p.U, p.total);   // the gang's run
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            // with a bias the epilogue warps read every stage's Zb tile (column sums) and arrive too
             mbar_init(&full[s], 1);
-            mbar_init(&ready[s], 2 * (N_TRANSFORM_WARPS + (p.any_bias ? N_EPILOGUE_WARPS : 0)));
+            mbar_init(&ready[s], 2 * N_TRANSFORM_WARPS);
             mbar_init(&empty[s], 1);
+            // with a bias the epilogue warps read every stage's Zb tile (column sums): they hold up the refill of
+            // the stage, not the MMAs
+            mbar_init(&zfree[s], N_EPILOGUE_WARPS);
         }
         mbar_init(acc_full, 1); mbar_init(acc_empty, 2 * N_EPILOGUE_WARPS);
         *abort_flag = 0;
@@ -182,7 +188,8 @@ zta_pair_kernel(const __grid_constant__ zta::Maps maps, const __grid_constant__ 
                 const CUtensorMap* map_z = &maps.z[w.layer];
                 const int mz = w.m0 + (int)rank * BM_CTA, na = w.n0 + (int)rank * BN_CTA;
                 for (int kb = w.kb0; kb < w.kb1; ++kb) {
-                    ok = mbar_wait(&empty[stage], phase ^ 1, abort_flag, p.status);
+                    ok = mbar_wait(&empty[stage], phase ^ 1, abort_flag, p.status) &&
+                         (!p.any_bias || mbar_wait(&zfree[stage], phase ^ 1, abort_flag, p.status));
                     if (!ok) break;
                     DPCLIP_TRACE_AT(0, tr); ++tr;
                     uint8_t* dst = smem + stage * STAGE_BYTES;
@@ -266,13 +273,17 @@ zta_pair_kernel(const __grid_constant__ zta::Maps maps, const __grid_constant__ 
                 const bool uniform = (rem0 + BK <= p.T) && (blk0 + BK <= p.R);   // one example, all rows exist
                 constexpr int NR = BK / 16;
                 float fr[NR];
+                if (uniform) {
+                    const float f = row_factor(p, e_first);            // one factor for the whole stage
 #pragma unroll
-                for (int i = 0; i < NR; ++i) {
-                    const int rl = uniform ? 0 : rs + 16 * i;
-                    float f = 1.f;
-                    if (blk0 + rl >= p.R) f = 0.f;                    // past the last row (TMA filled zeros there)
-                    else if (p.clip) f = __ldg(p.clip + e_first + (rem0 + rl) / p.T);
-                    fr[i] = f;
+                    for (int i = 0; i < NR; ++i) fr[i] = f;
+                } else {
+#pragma unroll
+                    for (int i = 0; i < NR; ++i) {
+                        const int rl = rs + 16 * i;
+                        // past the last row TMA filled zeros; the factor only has to be finite there
+                        fr[i] = blk0 + rl >= p.R ? 0.f : row_factor(p, e_first + (rem0 + rl) / p.T);
+                    }
                 }
                 ok = mbar_wait(&full[stage], phase, abort_flag, p.status);
                 if (!ok) break;
@@ -327,7 +338,6 @@ zta_pair_kernel(const __grid_constant__ zta::Maps maps, const __grid_constant__ 
         const int t = threadIdx.x - 64 - 32 * N_TRANSFORM_WARPS;
         const int q = t >> 4, rs = t & 15;
         const uint32_t off = (q >> 3) * CHUNK_BYTES + rs * 128 + (((q & 7) ^ (rs & 7)) << 4);
-        const uint32_t ready0 = mapa_shared(smem_u32(ready), 0);
         int stage = 0; uint32_t phase = 0;
         int it = 0;
         bool ok = true;
@@ -352,13 +362,16 @@ zta_pair_kernel(const __grid_constant__ zta::Maps maps, const __grid_constant__ 
                         const int e_first = blk0 / p.T;
                         const int rem0 = blk0 - e_first * p.T;
                         const bool uniform = (rem0 + BK <= p.T) && (blk0 + BK <= p.R);
+                        if (uniform) {
+                            const float f = row_factor(p, e_first);
 #pragma unroll
-                        for (int i = 0; i < NR; ++i) {
-                            const int rl = uniform ? 0 : rs + 16 * i;
-                            float f = 1.f;
-                            if (blk0 + rl >= p.R) f = 0.f;
-                            else if (p.clip) f = __ldg(p.clip + e_first + (rem0 + rl) / p.T);
-                            fr[i] = f;
+                            for (int i = 0; i < NR; ++i) fr[i] = f;
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < NR; ++i) {
+                                const int rl = rs + 16 * i;
+                                fr[i] = blk0 + rl >= p.R ? 0.f : row_factor(p, e_first + (rem0 + rl) / p.T);
+                            }
                         }
                     }
                     ok = mbar_wait(&full[stage], phase, abort_flag, p.status);
@@ -384,7 +397,7 @@ zta_pair_kernel(const __grid_constant__ zta::Maps maps, const __grid_constant__ 
                             }
                     }
                     __syncwarp();
-                    if (lane == 0) mbar_arrive_cluster(ready0 + stage * 8);      // this warp is done reading the stage
+                    if (lane == 0) mbar_arrive(&zfree[stage]);                    // this warp is done reading the stage
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
                 if (!ok) break;
