@@ -78,7 +78,9 @@ typedef enum {
     DPCLIP_ERR_MISALIGNED = -3,       /* pointer not aligned to its element size                   */
     DPCLIP_ERR_WORKSPACE = -4,        /* workspace NULL or smaller than dpclip_workspace_bytes()   */
     DPCLIP_ERR_CUDA = -5,             /* a CUDA runtime/driver call or a launch failed              */
-    DPCLIP_ERR_TIMEOUT = -6           /* (device status) a bounded wait inside a kernel ran out     */
+    DPCLIP_ERR_TIMEOUT = -6,          /* (device status) a bounded wait inside a kernel ran out     */
+    DPCLIP_ERR_RANGE = -7             /* (device status, -DDPCLIP_DEBUG builds only) an index left its
+                                         buffer; the access was skipped, the kernel went on          */
 } dpclip_status;
 
 /* Squared per-example gradient norm of ONE layer, for every example:
@@ -485,6 +487,8 @@ void dpclip_reload_path_switches(void);
 
 const char* dpclip_status_string(int status);
 int dpclip_version(void);
+/* 1 when the library was compiled with -DDPCLIP_DEBUG (range-checked accesses, see DPCLIP_ERR_RANGE). */
+int dpclip_debug_build(void);
 
 #ifdef __cplusplus
 }

@@ -14,7 +14,8 @@ from typing import List, Optional, Sequence
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "libdpclip.so")
+# DPCLIP_LIBRARY selects another build of the same library (the range-checked libdpclip_debug.so)
+_LIB_PATH = os.environ.get("DPCLIP_LIBRARY") or os.path.join(_HERE, "libdpclip.so")
 _lib = None
 
 DPCLIP_F32, DPCLIP_BF16 = 0, 1
@@ -127,6 +128,7 @@ def load_library():
     L.dpclip_status_string.argtypes = [_i]
     L.dpclip_status_string.restype = ctypes.c_char_p
     L.dpclip_version.argtypes = []
+    L.dpclip_debug_build.argtypes = []
     L.dpclip_launch_count.argtypes = []
     L.dpclip_launch_count.restype = _u64
     L.dpclip_null_launch.argtypes = [_i, _i, _vp]
@@ -185,6 +187,10 @@ def _rows(t: torch.Tensor):
 # ----------------------------------------------------------------------------
 def dpclip_version() -> int:
     return load_library().dpclip_version()
+
+
+def dpclip_debug_build() -> bool:
+    return bool(load_library().dpclip_debug_build())
 
 
 def dpclip_launch_count() -> int:

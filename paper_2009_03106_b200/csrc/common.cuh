@@ -47,6 +47,21 @@ __device__ __forceinline__ float block_sum(float v, float* smem32) {
     return v;
 }
 
+// Range-checked build (-DDPCLIP_DEBUG, `python -m paper_2009_03106_b200.build --debug`): the stand-in for a
+// memory checker.  DPCLIP_IN_RANGE(i, n, status) is true when 0 <= i < n; otherwise it records
+// DPCLIP_ERR_RANGE in the workspace's status word and yields false, and the caller SKIPS the access -- no
+// trap, the kernel runs to its end.  In the normal build it is the constant true and costs nothing.
+#ifdef DPCLIP_DEBUG
+__device__ __forceinline__ bool debug_range_violation(int* status) {
+    if (status) atomicExch(status, (int)DPCLIP_ERR_RANGE);
+    return false;
+}
+#define DPCLIP_IN_RANGE(i, n, status) \
+    (((long long)(i) >= 0 && (long long)(i) < (long long)(n)) ? true : dpclip::debug_range_violation(status))
+#else
+#define DPCLIP_IN_RANGE(i, n, status) (true)
+#endif
+
 inline int ceil_div(long a, long b) { return (int)((a + b - 1) / b); }
 
 }  // namespace dpclip

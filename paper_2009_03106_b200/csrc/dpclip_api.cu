@@ -18,6 +18,7 @@
 #include "kernels_narrow_pack.cuh"
 #include "kernels_elementwise.cuh"
 
+#include <stdio.h>
 #include <stdlib.h>
 #include <atomic>
 
@@ -45,7 +46,7 @@ enum PathSwitch : unsigned {
     SW_FORCE_SIMT = 1u << 0, SW_NO_NARROW = 1u << 1, SW_NO_NARROW_RING = 1u << 2, SW_NO_NARROW_TC = 1u << 3,
     SW_NO_NARROW_PACK = 1u << 4, SW_NARROW_PACK_BF16 = 1u << 5, SW_NO_GRAM_Q2 = 1u << 6, SW_NO_T1_TF32 = 1u << 7,
     SW_NO_FUSED_T1 = 1u << 8, SW_NO_GRAM_GROUP = 1u << 9, SW_NO_GRAD_GROUP = 1u << 10, SW_NO_CONV_TC = 1u << 11,
-    SW_NO_CONV_PATCHES = 1u << 12, SW_TILE_M1 = 1u << 13, SW_TILE_M2 = 1u << 14, SW_T1_TWO_LAUNCHES = 1u << 15, SW_NO_PAIR = 1u << 16,
+    SW_NO_CONV_PATCHES = 1u << 12, SW_TILE_M1 = 1u << 13, SW_TILE_M2 = 1u << 14, SW_T1_TWO_LAUNCHES = 1u << 15, SW_NO_PAIR = 1u << 16, SW_LOG = 1u << 17,
     SW_LOADED = 1u << 31
 };
 std::atomic<unsigned> g_path_switches{0};
@@ -59,7 +60,7 @@ unsigned read_path_switches() {
         {"DPCLIP_NO_GRAD_GROUP", SW_NO_GRAD_GROUP, '1'}, {"DPCLIP_NO_CONV_TC", SW_NO_CONV_TC, '1'},
         {"DPCLIP_NO_CONV_PATCHES", SW_NO_CONV_PATCHES, '1'}, {"DPCLIP_TILE_M", SW_TILE_M1, '1'},
         {"DPCLIP_TILE_M", SW_TILE_M2, '2'}, {"DPCLIP_T1_ONE_LAUNCH", SW_T1_TWO_LAUNCHES, '0'},
-        {"DPCLIP_NO_PAIR", SW_NO_PAIR, '1'},
+        {"DPCLIP_NO_PAIR", SW_NO_PAIR, '1'}, {"DPCLIP_LOG", SW_LOG, '1'},
     };
     unsigned v = SW_LOADED;
     for (const auto& e : table) {
@@ -74,6 +75,10 @@ inline bool path_switch(unsigned bit) {
     if (!(v & SW_LOADED)) v = read_path_switches();
     return (v & bit) != 0;
 }
+
+// DPCLIP_LOG=1: one line on stderr per dispatch decision (which form of a kernel a layer takes and how its
+// work is cut) -- host side only, nothing changes on the device.
+#define DPCLIP_LOGF(...) do { if (path_switch(SW_LOG)) { fprintf(stderr, "[dpclip] " __VA_ARGS__); fputc('\n', stderr); } } while (0)
 
 int check_layer_args(const void* A, long lda, const void* Z, long ldz, int B, int T, int d_in, int d_out,
                      dpclip_dtype dtype) {
@@ -739,6 +744,7 @@ int launch_zta_stream(const StreamLayer* ls, int n, int B, int T, const float* c
     p.U = (int)U;
     p.lcm = (long)p.S / gcd_l(p.S, U) * U;
     const long n_segments = (zp::segment_of(p.total - 1, p.S, p.U, p.lcm) + 1) * W;
+    p.n_segments = n_segments;
     p.part = reinterpret_cast<float*>(static_cast<char*>(workspace) + kHeaderBytes);
     p.bias_part = p.any_bias ? p.part + (size_t)n_segments * zp::SEG_ELEMS : nullptr;
     if (fuse_noise) {
@@ -748,6 +754,9 @@ int launch_zta_stream(const StreamLayer* ls, int n, int B, int T, const float* c
     }
     if (!enable_smem(tc::zta_pair_kernel, zp::SMEM_BYTES)) return DPCLIP_ERR_CUDA;
     const int pairs = (int)ceil_div(p.total, U) * W;
+    DPCLIP_LOGF("clipped sum, CTA pairs: %d layer(s), B*T=%ld, %d tiles of 512x256 in %d super-layer(s) of %d, %d stages per tile, "
+                "%d pairs in gangs of %d, runs of %ld stages, %ld segments, noise %s", n, R, G, n_super, W, p.S, pairs, W, U,
+                n_segments, fuse_noise ? "in the reduce" : "separate");
     tc::zta_pair_kernel<<<2 * pairs, zp::THREADS, zp::SMEM_BYTES, st>>>(maps, p);
     int rc = launch_status();
     if (rc) return rc;
@@ -936,6 +945,10 @@ int launch_zta_tf32(const void* A, long lda, const void* Z, long ldz, int B, int
 int clipped_grad_impl(const void* A, long lda, const void* Zbar, long ldz, int B, int T, int d_in, int d_out,
                       dpclip_dtype dtype, const float* clip, float* gW, long ldg, float* gb, void* workspace,
                       size_t workspace_bytes, const NoiseSpec* noise, bool* noise_done, cudaStream_t st) {
+    DPCLIP_LOGF("clipped_grad B=%d T=%d %d->%d %s: %s", B, T, d_in, d_out, dtype == DPCLIP_F32 ? "f32" : "bf16",
+                tc_eligible(A, lda, Zbar, ldz, dtype) ? "tcgen05 bf16"
+                : (tf32_eligible(A, lda, Zbar, ldz, B, T, d_in, d_out, dtype) && !narrow_layer(T, d_in, d_out, gb != nullptr, lda, ldz))
+                      ? "tcgen05 3xtf32" : "fp32-ALU / narrow kernels");
     if (tc_eligible(A, lda, Zbar, ldz, dtype))
         return launch_zta_tc(A, lda, Zbar, ldz, B, T, d_in, d_out, false, 0, clip, gW, ldg, gb, nullptr, workspace,
                              workspace_bytes, noise, noise_done, st);
@@ -1121,6 +1134,13 @@ int try_fused_t1_step(const dpclip_layer* layers, int L, int B, dpclip_dtype dty
 extern "C" {
 
 int dpclip_version(void) { return 100; }
+int dpclip_debug_build(void) {
+#ifdef DPCLIP_DEBUG
+    return 1;
+#else
+    return 0;
+#endif
+}
 
 // An empty kernel with the launch shape of the one-launch T = 1 step: what a launch costs before it computes.
 __global__ void null_launch_kernel(int* sink) { if (sink && threadIdx.x == 0xFFFFFF) *sink = 0; }
@@ -1159,6 +1179,7 @@ const char* dpclip_status_string(int status) {
         case DPCLIP_ERR_WORKSPACE: return "workspace missing or too small";
         case DPCLIP_ERR_CUDA: return "CUDA call or kernel launch failed";
         case DPCLIP_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+        case DPCLIP_ERR_RANGE: return "range-checked build: an index left its buffer (access skipped)";
         default: return "unknown status";
     }
 }
@@ -1277,6 +1298,9 @@ int dpclip_layer_sqnorms(const void* A, long lda, const void* Zbar, long ldz, in
     if (!workspace || workspace_bytes < workspace_floor(B, T, d_in, d_out, dtype))
         return DPCLIP_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
+    DPCLIP_LOGF("layer_sqnorms B=%d T=%d %d->%d %s bias=%d: %s", B, T, d_in, d_out, dtype == DPCLIP_F32 ? "f32" : "bf16",
+                has_bias, method == DPCLIP_T1 ? "T1 closed form" : method == DPCLIP_SIMT ? "materialise, fp32-ALU / narrow kernels"
+                : method == DPCLIP_GRAM ? "Gram, tcgen05" : "materialise, tcgen05");
     switch (method) {
         case DPCLIP_T1:
             if (T != 1) return DPCLIP_ERR_UNSUPPORTED;

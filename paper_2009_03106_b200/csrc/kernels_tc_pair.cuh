@@ -95,6 +95,7 @@ struct Params {
     short tile_slot[MAX_TILES];    // [G]: s * W + j of every tile
     int any_bias;
     const float* clip;             // [B] or NULL
+    long n_segments;               // partial tiles the workspace holds (range checks of the debug build)
     float* part;                   // [n_segments][BM][BN] fp32
     float* bias_part;              // [n_segments][BM] fp32, or NULL when no layer has a bias
     int* status;
@@ -102,7 +103,10 @@ struct Params {
     Layer layer[MAX_LAYERS];
 };
 
-__device__ __forceinline__ float row_factor(const Params& p, int e) { return p.clip ? __ldg(p.clip + e) : 1.f; }
+__device__ __forceinline__ float row_factor(const Params& p, int e) {
+    if (!DPCLIP_IN_RANGE(e, (p.R + p.T - 1) / p.T, p.status)) return 0.f;
+    return p.clip ? __ldg(p.clip + e) : 1.f;
+}
 
 __host__ __device__ __forceinline__ long segment_of(long u, int S, int U, long lcm) { return u / S + u / U - u / lcm; }
 
@@ -412,7 +416,8 @@ zta_pair_kernel(const __grid_constant__ zta::Maps maps, const __grid_constant__ 
                         c += __shfl_xor_sync(0xFFFFFFFFu, c, 2);
                         c += __shfl_xor_sync(0xFFFFFFFFu, c, 4);
                         c += __shfl_xor_sync(0xFFFFFFFFu, c, 8);
-                        if (rs == 0) p.bias_part[(size_t)w.slot * BM + (int)rank * BM_CTA + h2 * 128 + q * 8 + j] = c;
+                        if (rs == 0 && DPCLIP_IN_RANGE(w.slot, p.n_segments, p.status))
+                            p.bias_part[(size_t)w.slot * BM + (int)rank * BM_CTA + h2 * 128 + q * 8 + j] = c;
                     }
             }
             if (!mbar_wait(acc_full, it & 1, abort_flag, p.status)) break;
@@ -442,7 +447,8 @@ zta_pair_kernel(const __grid_constant__ zta::Maps maps, const __grid_constant__ 
                     const float4 x = st[rr * 8 + (jj ^ (rr & 7))];
                     // the segment's partial tile (dense 512 x 256, no bounds: rows and columns past the layer's
                     // extent hold the zeros TMA filled in)
-                    *reinterpret_cast<float4*>(seg + (size_t)(ml0 + rr) * BN + c0 + 4 * jj) = x;
+                    if (DPCLIP_IN_RANGE(w.slot, p.n_segments, p.status) && DPCLIP_IN_RANGE(ml0 + rr, BM, p.status))
+                        *reinterpret_cast<float4*>(seg + (size_t)(ml0 + rr) * BN + c0 + 4 * jj) = x;
                 }
                 __syncwarp();
             }
@@ -481,6 +487,7 @@ reduce_segments_kernel(const __grid_constant__ ztp::Params p) {
         const long sl = ts / p.W, j = ts - sl * p.W;
         const long s0 = segment_of(sl * p.S, p.S, p.U, p.lcm), s1 = segment_of((sl + 1) * p.S - 1, p.S, p.U, p.lcm);
         const float* src = p.part + (size_t)(s0 * p.W + j) * SEG_ELEMS + (size_t)(m - tm * BM) * BN + (n - tn * BN);
+        if (!DPCLIP_IN_RANGE(s1 * p.W + j, p.n_segments, p.status) || !DPCLIP_IN_RANGE(s0, s1 + 1, p.status)) continue;
         float4 acc = __ldcs(reinterpret_cast<const float4*>(src));
         for (long s = s0 + 1; s <= s1; ++s) {
             src += (size_t)p.W * SEG_ELEMS;

@@ -6,7 +6,7 @@ import torch
 
 import oracle
 import workloads
-from util import SAT_BAND, TOL, check_saturation, max_rel, rel_fro, to_device
+from util import SAT_BAND, TOL, Guarded, check_saturation, max_rel, rel_fro, to_device
 
 pytestmark = pytest.mark.gpu
 
@@ -28,12 +28,14 @@ def _ws(dp, nbytes=None):
 
 def _sqnorms(dp, A, Z, dtype, has_bias, method=0):
     dA, dZ = to_device(A, dtype), to_device(Z, dtype)
-    sq = torch.full((A.shape[0],), -1.0, device="cuda")
+    guard = Guarded(A.shape[0], fill=-1.0)              # every norm test writes between guard bands
+    sq = guard.t
     ws = _ws(dp, max(1 << 20, dp.dpclip_workspace_bytes(A.shape[0], A.shape[1], A.shape[2], Z.shape[2],
                                                        0 if dtype == "f32" else 1, method)))
     dp.dpclip_layer_sqnorms(dA, dZ, has_bias, sq, ws, method)
     torch.cuda.synchronize()
     assert dp.dpclip_read_status(ws) == 0
+    guard.check()
     return sq.cpu().numpy()
 
 
@@ -124,10 +126,12 @@ def test_tensor_core_clipped_grad(dp, B, T, d_in, d_out):
     clip[::2] = 1.0
     refW, refb = oracle.clipped_grad(A, Z, clip)
     dA, dZ = to_device(A, "bf16"), to_device(Z, "bf16")
-    gW = torch.full((d_out, d_in), 9.0, device="cuda"); gb = torch.full((d_out,), 9.0, device="cuda")
+    guard_W, guard_b = Guarded(d_out, d_in), Guarded(d_out)       # outputs between guard bands
+    gW, gb = guard_W.t, guard_b.t
     ws = _ws(dp)
     dp.dpclip_clipped_grad(dA, dZ, torch.from_numpy(clip).cuda(), gW, gb, ws)
     assert dp.dpclip_read_status(ws) == 0
+    guard_W.check(); guard_b.check()
     assert rel_fro(gW.cpu().numpy(), refW) <= TOL["bf16"]["grad"]
     assert rel_fro(gb.cpu().numpy(), refb) <= 2e-3          # fp32 sums of the bf16-rounded clip*zbar values
     refW1, refb1 = oracle.clipped_grad(A, Z, None)
@@ -442,9 +446,11 @@ def test_clipped_grad(dp, dtype, B, T, d_in, d_out):
     clip[::3] = 1.0
     refW, refb = oracle.clipped_grad(A, Z, clip)
     dA, dZ = to_device(A, dtype), to_device(Z, dtype)
-    gW = torch.full((d_out, d_in), 9.0, device="cuda"); gb = torch.full((d_out,), 9.0, device="cuda")
+    guard_W, guard_b = Guarded(d_out, d_in), Guarded(d_out)
+    gW, gb = guard_W.t, guard_b.t
     ws = _ws(dp)
     dp.dpclip_clipped_grad(dA, dZ, torch.from_numpy(clip).cuda(), gW, gb, ws)
+    guard_W.check(); guard_b.check()
     # identical inputs and fp32 accumulation: the fp32 bound applies, except on the tensor-core path,
     # which rounds clip*zbar to bf16 in shared memory (bf16 rows that are 16-byte multiples take it)
     narrow = T > 1 and d_in + 1 <= 32 and d_out <= 64
@@ -487,8 +493,11 @@ def test_clipped_grad_noise_equals_separate_calls(dp, dtype, B, T, d_in, d_out):
 def test_noise_matches_oracle(dp, n):
     sigma, C, seed, sid = 1.1, 0.7, 0x123456789ABCDEF, (1 << 40) + 5
     base = np.random.default_rng(n).standard_normal(n).astype(np.float32)
-    g = torch.from_numpy(base).cuda()
+    guard = Guarded(n)
+    g = guard.t
+    g.copy_(torch.from_numpy(base))
     dp.dpclip_add_noise(g, sigma, C, seed, sid)
+    guard.check()
     ref = oracle.add_noise(base, sigma, C, seed, sid)
     assert np.max(np.abs(g.cpu().numpy() - ref)) <= 1e-5 * sigma * C + 1e-6 * np.max(np.abs(ref))
     # noise-only tensor, and an output that does not start on a 16-byte boundary

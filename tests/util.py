@@ -42,3 +42,24 @@ def check_saturation(clip_gpu, norms_ref, clip_ref, C):
     near = np.abs(norms_ref / C - 1.0) <= SAT_BAND
     assert not np.any(differ & ~near), np.nonzero(differ & ~near)
     assert np.all(clip_gpu[~sat_gpu] == 1.0)
+
+
+class Guarded:
+    """An fp32 output tensor carved out of a larger allocation with 256-byte guard bands before and after it,
+    filled with a bit pattern no kernel writes: stands in for a memory checker on the outputs.  `t` is the
+    tensor to hand to the library; `check()` fails if a band was touched."""
+    PATTERN = 0x7FA5A5A5          # a NaN payload
+
+    def __init__(self, *shape, fill=9.0):
+        n = int(np.prod(shape))
+        band = 64                                       # 64 floats = 256 bytes
+        pad = (-n) % 64                                 # the output keeps the 256-byte alignment of the allocation
+        self.raw = torch.full((band + n + pad + band,), 0, dtype=torch.int32, device="cuda")
+        self.raw.fill_(self.PATTERN)
+        self.t = self.raw[band:band + n].view(torch.float32).view(*shape)
+        self.t.fill_(fill)
+        self._n, self._band = n, band
+
+    def check(self):
+        lo = self.raw[:self._band]; hi = self.raw[self._band + self._n:]
+        assert bool((lo == self.PATTERN).all()) and bool((hi == self.PATTERN).all()), "guard band overwritten"
