@@ -298,11 +298,10 @@ kernel_breakdown.groups = {}          # members of the grouped launches of the l
 NCU_TRAFFIC_BYTES = {
     ("mlp_784_1000_1000_10_b128", "t1_all_grads_tf32_kernel"): 2.55e6,   # profiles/fused_t1_mlp_784_1000_1000_10_b128.txt
     ("mlp_784_1000_1000_10_b128", "t1_all_grads_kernel"): 2.54e6,
-    ("seq_b128_t256_d512_bf16", "norm_gram_group"): 775.3e6,          # profiles/tc_kernels_seq_b128_t256.txt
-    ("seq_b128_t256_d512_bf16", "grad_group"): 272.7e6,
-    ("seq_b128_t256_d512_bf16", "grad[ffn_in]"): 171.1e6,
-    ("seq_b128_t256_d512_bf16", "grad[lstm_gates]"): 171.1e6,
-    ("seq_b128_t256_d512_bf16", "grad[ffn_out]"): 171.1e6,
+    ("seq_b128_t256_d512_bf16", "norm_gram_group"): 775.4e6,          # profiles/tc_kernels_seq_b128_t256.txt
+    # zta_pair_kernel 772.8 + 24.2 MB, reduce_segments_kernel 50.5 + 0.5 MB (cold-cache capture: inside a step the
+    # reduce finds the partial tiles in L2)
+    ("seq_b128_t256_d512_bf16", "grad_group"): 848.0e6,
 }
 
 
@@ -402,7 +401,7 @@ def roofline_zta(w, breakdown, peaks):
                  frac_of_sustained_peak=ach / peaks["bf16_tflops_sustained"])
     traffic = [NCU_TRAFFIC_BYTES.get((w.name, "grad_group" if k[0] == "grad_group" else f"grad[{w.layers[k[1]].name}]")) for k in keys]
     r.update(traffic=(sum(traffic) / len(keys) if all(t is not None for t in traffic) else None),
-             kernel="zta_tc_kernel (+ reduce_partials_kernel)", launches_per_step=len(keys), kernel_ms=ms / len(keys),
+             kernel="zta_pair_kernel + reduce_segments_kernel (bf16 clipped sums)", launches_per_step=len(keys), kernel_ms=ms / len(keys),
              kernel_ms_total=ms, share_of_step=ms / sum(breakdown.values()), algorithmic_bytes=nbytes / len(keys),
              algorithmic_flops=flops / len(keys), peak_source=peaks["source"],
              note="per launch: averages over the kernel's launches of one step; peak = burst bf16 figure")

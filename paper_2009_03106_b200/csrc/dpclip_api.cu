@@ -33,6 +33,7 @@ inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 std::atomic<unsigned long long> g_launches{0};
 constexpr int kGridCounterOffset = 64;   // workspace header: status word at 0, grid-barrier counter here
 constexpr int kWorkCounterOffset = 128;  // item counter of the dynamically scheduled Gram kernel (wraps to zero by itself)
+constexpr int kTailCounterOffset = 192;  // CTAs done, for the factors tail of a Gram launch (reset by the last CTA)
 inline int launch_status() {
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? DPCLIP_OK : DPCLIP_ERR_CUDA;
@@ -46,7 +47,7 @@ enum PathSwitch : unsigned {
     SW_FORCE_SIMT = 1u << 0, SW_NO_NARROW = 1u << 1, SW_NO_NARROW_RING = 1u << 2, SW_NO_NARROW_TC = 1u << 3,
     SW_NO_NARROW_PACK = 1u << 4, SW_NARROW_PACK_BF16 = 1u << 5, SW_NO_GRAM_Q2 = 1u << 6, SW_NO_T1_TF32 = 1u << 7,
     SW_NO_FUSED_T1 = 1u << 8, SW_NO_GRAM_GROUP = 1u << 9, SW_NO_GRAD_GROUP = 1u << 10, SW_NO_CONV_TC = 1u << 11,
-    SW_NO_CONV_PATCHES = 1u << 12, SW_TILE_M1 = 1u << 13, SW_TILE_M2 = 1u << 14, SW_T1_TWO_LAUNCHES = 1u << 15, SW_NO_PAIR = 1u << 16, SW_LOG = 1u << 17,
+    SW_NO_CONV_PATCHES = 1u << 12, SW_TILE_M1 = 1u << 13, SW_TILE_M2 = 1u << 14, SW_T1_TWO_LAUNCHES = 1u << 15, SW_NO_PAIR = 1u << 16, SW_LOG = 1u << 17, SW_NO_FACTORS_TAIL = 1u << 18,
     SW_LOADED = 1u << 31
 };
 std::atomic<unsigned> g_path_switches{0};
@@ -61,6 +62,7 @@ unsigned read_path_switches() {
         {"DPCLIP_NO_CONV_PATCHES", SW_NO_CONV_PATCHES, '1'}, {"DPCLIP_TILE_M", SW_TILE_M1, '1'},
         {"DPCLIP_TILE_M", SW_TILE_M2, '2'}, {"DPCLIP_T1_ONE_LAUNCH", SW_T1_TWO_LAUNCHES, '0'},
         {"DPCLIP_NO_PAIR", SW_NO_PAIR, '1'}, {"DPCLIP_LOG", SW_LOG, '1'},
+        {"DPCLIP_NO_FACTORS_TAIL", SW_NO_FACTORS_TAIL, '1'},
     };
     unsigned v = SW_LOADED;
     for (const auto& e : table) {
@@ -416,7 +418,8 @@ inline int gram_class(int T) {
 // Norms of up to gram::MAX_LAYERS layers by the Gram identity in ONE launch.  All layers must agree on
 // gram_class(T).  Layers go in descending order of bytes per group, so that the round-robin deal
 // leaves the small items for the end of every CTA's queue.
-int launch_gram_group(const GramLayer* ls, int n, int* status, cudaStream_t st) {
+int launch_gram_group(const GramLayer* ls, int n, int* status, cudaStream_t st,
+                      const tc::gram::FactorsTail* tail = nullptr) {
     namespace g = tc::gram;
     if (n <= 0 || n > g::MAX_LAYERS) return DPCLIP_ERR_INVALID_ARG;
     int order[g::MAX_LAYERS];
@@ -470,6 +473,10 @@ int launch_gram_group(const GramLayer* ls, int n, int* status, cudaStream_t st) 
     }
     q.group_begin[n] = groups;
     q.total_groups = groups;
+    if (tail) {
+        q.tail = *tail;
+        q.tail.done = reinterpret_cast<unsigned int*>(reinterpret_cast<char*>(status) + kTailCounterOffset);
+    }
     const int grid = groups < kNumSMs ? groups : kNumSMs;
     if (cls == 0) {
         q.work_counter = reinterpret_cast<unsigned int*>(reinterpret_cast<char*>(status) + kWorkCounterOffset);
@@ -1328,8 +1335,21 @@ int dpclip_layer_sqnorms(const void* A, long lda, const void* Zbar, long ldz, in
     }
 }
 
+static int gram_layers_sqnorms(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, float* sq_layers,
+                               int* taken, void* workspace, size_t workspace_bytes, void* stream,
+                               const tc::gram::FactorsTail* tail, bool* tail_done);
+
 int dpclip_gram_layers_sqnorms(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, float* sq_layers,
                                int* taken, void* workspace, size_t workspace_bytes, void* stream) {
+    return gram_layers_sqnorms(layers, L, B, dtype, sq_layers, taken, workspace, workspace_bytes, stream, nullptr, nullptr);
+}
+
+// tail: factors in the tail of the launch -- only when ONE launch takes every layer (all L rows of sq come from
+// it); *tail_done says whether that happened.
+static int gram_layers_sqnorms(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype, float* sq_layers,
+                               int* taken, void* workspace, size_t workspace_bytes, void* stream,
+                               const tc::gram::FactorsTail* tail, bool* tail_done) {
+    if (tail_done) *tail_done = false;
     if (!layers || L <= 0 || B <= 0 || !sq_layers) return DPCLIP_ERR_INVALID_ARG;
     if (taken) for (int l = 0; l < L; ++l) taken[l] = 0;
     if (dtype != DPCLIP_BF16 || !workspace || workspace_bytes < (size_t)kHeaderBytes) return DPCLIP_OK;
@@ -1342,9 +1362,11 @@ int dpclip_gram_layers_sqnorms(const dpclip_layer* layers, int L, int B, dpclip_
         auto flush = [&]() -> int {
             // a single layer gains nothing from this entry point: leave it to the per-layer call
             if (n >= 2) {
-                const int rc = launch_gram_group(batch, n, (int*)workspace, (cudaStream_t)stream);
+                const bool with_tail = tail && n == L;             // this launch writes every row of sq
+                const int rc = launch_gram_group(batch, n, (int*)workspace, (cudaStream_t)stream, with_tail ? tail : nullptr);
                 if (rc) return rc;
                 if (taken) for (int i = 0; i < n; ++i) taken[idx[i]] = 1;
+                if (with_tail && tail_done) *tail_done = true;
             }
             n = 0;
             return DPCLIP_OK;
@@ -2038,8 +2060,12 @@ static int step_general(const dpclip_layer* layers, const dpclip_model_layer* ot
     int in_gram_group[64];
     const bool track = L <= 64;
     bool any_gram = false;
+    bool factors_done = false;
     if (track) {
-        rc = dpclip_gram_layers_sqnorms(layers, L, B, dtype, sq_layers, in_gram_group, ws0, workspace_bytes, lanes.st[0]);
+        // when one Gram launch takes every layer of the model, its last CTA also computes the factors
+        const tc::gram::FactorsTail tail = {sq_layers, L, (long)B, B, C, clip, norms, nullptr};
+        rc = gram_layers_sqnorms(layers, L, B, dtype, sq_layers, in_gram_group, ws0, workspace_bytes, lanes.st[0],
+                                 (!t1.active && !other && !path_switch(SW_NO_FACTORS_TAIL)) ? &tail : nullptr, &factors_done);
         if (rc) return rc;
         for (int l = 0; l < L; ++l) any_gram = any_gram || in_gram_group[l];
     }
@@ -2058,8 +2084,10 @@ static int step_general(const dpclip_layer* layers, const dpclip_model_layer* ot
         if (rc) return rc;
     }
     if ((rc = lanes.join())) return rc;
-    rc = dpclip_factors(sq_layers, L, B, B, C, clip, norms, nullptr, lanes.st[0]);
-    if (rc) return rc;
+    if (!factors_done) {
+        rc = dpclip_factors(sq_layers, L, B, B, C, clip, norms, nullptr, lanes.st[0]);
+        if (rc) return rc;
+    }
     if ((rc = lanes.fork())) return rc;
     if (t1.active) {
         rc = launch_fused_t1_tf32(t1.p, false, dtype, lanes.ws[last], workspace_bytes, lanes.st[last]);

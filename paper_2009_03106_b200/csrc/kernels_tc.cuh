@@ -77,6 +77,16 @@ struct Params {            // one layer
 // first).  With one example per CTA a single layer of a small batch is a latency chain (set-up, first
 // load, the second row block and both epilogues are all exposed); several layers in one launch give every
 // CTA a queue of items, so loads of the next item run under the MMAs and epilogues of the current one.
+// Clip factors in the tail of a norm launch that produces EVERY row of sq[L][B] (the text after Eq.
+// "weighted_loss" and Eq. "per_example_weight": n_i = sqrt(sum_l sq[l][i]), c_i = min(1, C / n_i)): the CTA
+// that finishes last computes them, so the step needs no factors launch between its norms and its clipped
+// sums.  Same arithmetic, in the same order, as factors_kernel.
+struct FactorsTail {
+    const float* sq; int L; long ld; int B; float C;
+    float* clip; float* norms;           // clip == NULL: no tail
+    unsigned int* done;                  // CTAs finished so far (workspace header; back at zero after the launch)
+};
+
 struct Launch {
     CUtensorMap map_a[MAX_LAYERS], map_z[MAX_LAYERS];
     Params layer[MAX_LAYERS];
@@ -84,7 +94,30 @@ struct Launch {
     int L, total_groups;
     int* status;
     unsigned int* work_counter;    // gram_norm_q2_kernel: items are handed out in order from this counter
+    FactorsTail tail;
 };
+
+// Called by every thread of a CTA after its last atomic into sq has been issued.
+__device__ __forceinline__ void factors_tail(const FactorsTail& t) {
+    if (!t.clip) return;
+    __shared__ unsigned int s_prev;
+    __threadfence();                                   // this thread's atomics on sq before the CTA's count
+    __syncthreads();
+    if (threadIdx.x == 0) s_prev = atomicAdd(t.done, 1u);
+    __syncthreads();
+    if (s_prev != gridDim.x - 1) return;               // not the last CTA
+    __threadfence();
+    for (int i = threadIdx.x; i < t.B; i += blockDim.x) {
+        float s = 0.f;
+        for (int l = 0; l < t.L; ++l) s += __ldcg(t.sq + (size_t)l * t.ld + i);      // L2: where the atomics landed
+        const float n = sqrtf(s);
+        float c = 1.0f;
+        if (n > t.C) c = t.C / n;                      // tie and zero norm stay exactly 1
+        t.clip[i] = c;
+        if (t.norms) t.norms[i] = n;
+    }
+    if (threadIdx.x == 0) *t.done = 0u;                // ready for the next launch
+}
 
 // layer of group g (group_begin is ascending; L is small)
 __device__ __forceinline__ int layer_of(const Launch& q, int g) {
@@ -323,6 +356,7 @@ gram_norm_kernel(const __grid_constant__ gram::Launch q) {
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) { tc_fence_after_sync(); tmem_dealloc(tmem_base, 512); }
+    factors_tail(q.tail);
 }
 
 // ---------------------------------------------------------------------------
@@ -558,6 +592,7 @@ gram_norm_q2_kernel(const __grid_constant__ gram::Launch q) {
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) { tc_fence_after_sync(); tmem_dealloc(tmem_base, 512); }
+    factors_tail(q.tail);
 }
 
 // ===========================================================================

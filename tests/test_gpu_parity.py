@@ -869,6 +869,45 @@ def test_gram_layers_in_one_launch(dp):
     assert dp.dpclip_gram_layers_sqnorms(lone) == [False]
 
 
+def test_step_factors_in_the_tail_of_the_gram_launch(dp, path_switch):
+    """When one Gram launch takes every layer of the model, its last CTA computes the clip factors (no factors
+    launch): same bits as the factors kernel (the path with the shared launch switched off), equal to the oracle,
+    and repeatable (the CTA counter in the workspace header returns to zero)."""
+    w = workloads.seq("bf16", B=40, T=256, d=64, d_ff=136)
+    data = workloads.generate(w, 5)
+    cal = _calibrate(w, data, 5, w.C)
+    mk = lambda: dp.StepPlan([dp.Layer(to_device(A, "bf16"), to_device(Z, "bf16"), s.has_bias, dp.DPCLIP_GRAM)   # noqa: E731
+                              for (A, Z), s in zip(cal, w.layers)])
+    plan = mk()
+    n0 = dp.dpclip_launch_count()
+    plan.run(w.C, 0.0, 3)
+    launches_with_tail = dp.dpclip_launch_count() - n0
+    torch.cuda.synchronize()
+    assert dp.dpclip_read_status(plan.workspace) == 0
+    hb = [s.has_bias for s in w.layers]
+    sq = np.stack([oracle.layer_sqnorms(A, Z, b) for (A, Z), b in zip(cal, hb)])
+    n_ref, c_ref = oracle.factors(sq, w.C)
+    assert max_rel(plan.norms.cpu().numpy(), n_ref) <= TOL["bf16"]["norm"]
+    check_saturation(plan.clip.cpu().numpy(), n_ref, c_ref, w.C)
+    assert 0 < (c_ref < 1).sum() < w.B
+    first_clip, first_flat = plan.clip.clone(), plan.flat.clone()
+    for _ in range(50):
+        plan.clip.fill_(float("nan"))
+        plan.run(w.C, 0.0, 3)
+    torch.cuda.synchronize()
+    assert dp.dpclip_read_status(plan.workspace) == 0
+    # the norms are combined with atomics (order of arrival): factors equal up to that, clipped sums follow
+    assert np.allclose(plan.clip.cpu().numpy(), first_clip.cpu().numpy(), rtol=2e-6, atol=0)
+    assert rel_fro(plan.flat.cpu().numpy(), first_flat.cpu().numpy()) <= 2e-6
+    path_switch("DPCLIP_NO_GRAM_GROUP", "1")
+    other = mk()
+    n0 = dp.dpclip_launch_count()
+    other.run(w.C, 0.0, 3)
+    assert dp.dpclip_launch_count() - n0 > launches_with_tail          # per-layer norms + a factors launch
+    torch.cuda.synchronize()
+    assert np.allclose(other.clip.cpu().numpy(), first_clip.cpu().numpy(), rtol=2e-6, atol=0)
+
+
 def test_step_same_shape_layers_share_launches(dp, path_switch):
     """Layers of one shape go through one clipped-sum launch (stacked d_out tiles, one set of partial tiles,
     one reduce with every layer's own noise streams): 256-row and 128-row tile forms, ragged d_out, layers
