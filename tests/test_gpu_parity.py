@@ -908,6 +908,58 @@ def test_step_factors_in_the_tail_of_the_gram_launch(dp, path_switch):
     assert np.allclose(other.clip.cpu().numpy(), first_clip.cpu().numpy(), rtol=2e-6, atol=0)
 
 
+@pytest.mark.parametrize("shapes", [
+    # three 512 -> 512 layers (2 tiles each) and a 256 -> 1024 layer (2 tiles): gangs of 8, one super-layer
+    [(512, 512, False), (512, 512, True), (512, 512, False), (256, 1024, True)],
+    # 2 + 2 + 8 tiles: the narrow layers share a super-layer that stays half empty (pairs without a tile)
+    [(512, 512, True), (512, 504, False), (512, 2048, True)],
+    # 3 + 2 tiles: five tiles side by side in gangs of 5
+    [(768, 512, True), (512, 512, False)],
+    # 8 + 7 tiles: gangs of 8, the second super-layer has a position without a tile (that pair idles there)
+    [(512, 2048, True), (256, 3584, False)],
+    # 17 tiles: no gang width divides it -> tile-major runs (W = 1)
+    [(256, 8704, True)],
+])
+def test_wide_layers_of_any_shape_share_one_pair_launch(dp, shapes):
+    """Layers wide enough for the CTA-pair kernel share ONE clipped-sum launch whatever their shapes (same T):
+    packed into super-layers, runs cut per gang, segments reduced per tile.  Every output against the oracle;
+    with noise, the difference to the sigma = 0 result is each layer's own noise stream."""
+    B, T = 3, 192                                   # 9 stages per tile: runs of 8 stages cross tile boundaries
+    L = workloads.LayerSpec
+    specs = tuple(L(f"l{i}", T, d_in, d_out, hb, "normal") for i, (d_in, d_out, hb) in enumerate(shapes))
+    w = workloads.Workload("wide_mixed", B, "bf16", specs, 1.0, 0.7, 1.0 / (B * T))
+    data = workloads.generate(w, 11)
+    plan = dp.StepPlan([dp.Layer(to_device(A, "bf16"), to_device(Z, "bf16"), s.has_bias) for (A, Z), s in zip(data, specs)])
+    clip = np.array([1.0, 0.37, 0.052], np.float32)
+    plan.clip.copy_(torch.from_numpy(clip))
+    plan.flat.fill_(float("nan"))
+    taken = dp.dpclip_same_shape_layers_clipped_grad_noise(plan, 1.0, 0.0, seed=0)
+    torch.cuda.synchronize()
+    assert (all(taken) or len(shapes) == 1) and dp.dpclip_read_status(plan.workspace) == 0
+    if len(shapes) == 1:            # a single layer takes the same kernel through its own entry point
+        dp.dpclip_clipped_grad(plan.layers[0].A, plan.layers[0].Zbar, plan.clip, plan.gW[0], plan.gb[0], plan.workspace)
+        torch.cuda.synchronize()
+    for l, ((A, Z), s) in enumerate(zip(data, specs)):
+        refW, refb = oracle.clipped_grad(A, Z, clip)
+        assert rel_fro(plan.gW[l].cpu().numpy(), refW) <= TOL["bf16"]["grad"], l
+        if s.has_bias:
+            assert rel_fro(plan.gb[l].cpu().numpy(), refb) <= 1e-5, l        # bias sums are taken in fp32
+    if len(shapes) == 1:
+        return
+    pre = plan.flat.clone()
+    dp.dpclip_same_shape_layers_clipped_grad_noise(plan, 1.3, 0.7, seed=5, stream_id0=40)
+    torch.cuda.synchronize()
+    for l, s in enumerate(specs):
+        xi = oracle.normals(s.d_out * s.d_in, 5, 40 + 2 * l).reshape(s.d_out, s.d_in)
+        off = plan.gW[l].data_ptr() - plan.flat.data_ptr()
+        base = pre[off // 4: off // 4 + s.d_out * s.d_in].view(s.d_out, s.d_in)
+        assert np.max(np.abs((plan.gW[l] - base).cpu().numpy() - 0.7 * 1.3 * xi)) <= 1e-5 * 0.91 + 1e-6 * float(base.abs().max()), l
+        if s.has_bias:
+            xb = oracle.normals(s.d_out, 5, 40 + 2 * l + 1)
+            offb = (plan.gb[l].data_ptr() - plan.flat.data_ptr()) // 4
+            assert np.max(np.abs((plan.gb[l] - pre[offb:offb + s.d_out]).cpu().numpy() - 0.91 * xb)) <= 1e-5, l
+
+
 def test_step_same_shape_layers_share_launches(dp, path_switch):
     """Layers of one shape go through one clipped-sum launch (stacked d_out tiles, one set of partial tiles,
     one reduce with every layer's own noise streams): 256-row and 128-row tile forms, ragged d_out, layers
