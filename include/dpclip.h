@@ -300,13 +300,15 @@ size_t dpclip_conv_workspace_bytes(int B, const dpclip_conv* geom, int d_out, dp
 
 /* Per-layer clipping: every layer's per-example gradient is clipped to its own threshold C_layer[l] (for
  * instance C / sqrt(L), so that the concatenated gradient stays within C), the variant that per-layer norms
- * make possible (Sec. "Related Work", per-layer clipping).  For each layer in turn: squared norms -> factors
- * from that row alone -> clipped sum -> noise N(0, sigma^2 * sum_l C_layer[l]^2) on every coordinate (the
+ * make possible (Sec. "Related Work", per-layer clipping).  The stages of dpclip_step with a factor vector per
+ * layer: squared norms of every layer -> factors of layer l from row l alone, against C_layer[l] -> clipped sums,
+ * layer l with its own factors -> noise N(0, sigma^2 * sum_l C_layer[l]^2) on every coordinate (the
  * sensitivity of the concatenated clipped gradient), streams stream_id0 + 2l / + 2l + 1 as in dpclip_step.
+ * The launches several layers share under global clipping (Gram norms; the clipped sums of wide bf16 layers)
+ * are shared here too.
  *   C_layer       host [L], each > 0
  *   sq_layers     [L][B], clip_layers [L][B] (row l = layer l's factors), norms_layers [L][B] or NULL
- * No layer waits for another layer's norm, and a layer's clipped sum follows its own norm pass while its
- * inputs are still in L2.  Errors as for dpclip_step. */
+ * workspace >= dpclip_step_workspace_bytes().  Errors as for dpclip_step. */
 int dpclip_step_per_layer(const dpclip_layer* layers /* host */, int L, int B, dpclip_dtype dtype,
                           const float* C_layer /* host */, float sigma,
                           unsigned long long seed, unsigned long long stream_id0,

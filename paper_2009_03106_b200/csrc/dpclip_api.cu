@@ -656,11 +656,12 @@ inline long gcd_l(long a, long b) { while (b) { const long t = a % b; a = b; b =
 struct StreamLayer {
     const void* A; long lda; const void* Z; long ldz; int d_in, d_out;
     float* gW; long ldg; float* gb; unsigned long long sid_w, sid_b;
+    const float* clip;             // this layer's factors [B], or NULL
 };
 
 // Returns DPCLIP_OK, a negative status, or 1 when the workspace cannot hold even one segment per tile (the
 // caller then takes another path).
-int launch_zta_stream(const StreamLayer* ls, int n, int B, int T, const float* clip, const NoiseSpec* noise,
+int launch_zta_stream(const StreamLayer* ls, int n, int B, int T, const NoiseSpec* noise,
                       bool* noise_done, void* workspace, size_t workspace_bytes, cudaStream_t st) {
     namespace zp = tc::ztp;
     if (n < 1 || n > zp::MAX_LAYERS) return 1;
@@ -669,7 +670,7 @@ int launch_zta_stream(const StreamLayer* ls, int n, int B, int T, const float* c
     zp::Params p;
     memset(&p, 0, sizeof(p));
     p.R = (int)R; p.T = T; p.S = (int)ceil_div(R, (long)zp::BK); p.n_layers = n;
-    p.clip = clip; p.status = static_cast<int*>(workspace);
+    p.status = static_cast<int*>(workspace);
     bool fuse_noise = noise && noise->scale > 0.f;
     int G = 0;
     for (int l = 0; l < n; ++l) {
@@ -683,6 +684,7 @@ int launch_zta_stream(const StreamLayer* ls, int n, int B, int T, const float* c
         q.tile_base = G; q.tiles = pair_tiles(y.d_in, y.d_out);
         G += q.tiles;
         q.do_bias = y.gb ? 1 : 0;
+        q.clip = y.clip;
         q.gW = y.gW; q.gb = y.gb; q.ldg = y.ldg;
         q.vec_ok = aligned_to(y.gW, 16) && y.ldg % 4 == 0;
         q.sw0 = (uint32_t)y.sid_w; q.sw1 = (uint32_t)(y.sid_w >> 32);
@@ -807,8 +809,8 @@ int launch_zta_tc(const void* A, long lda, const void* Z, long ldz, int B, int T
         p.vec_ok = aligned_to(gW, 16) && ldg % 4 == 0;
     }
     if (pair) {
-        const StreamLayer one = {A, lda, Z, ldz, d_in, d_out, gW, ldg, gb, noise ? noise->sid_w : 0ull, noise ? noise->sid_b : 0ull};
-        const int rc = launch_zta_stream(&one, 1, B, T, clip, noise, noise_done, workspace, workspace_bytes, st);
+        const StreamLayer one = {A, lda, Z, ldz, d_in, d_out, gW, ldg, gb, noise ? noise->sid_w : 0ull, noise ? noise->sid_b : 0ull, clip};
+        const int rc = launch_zta_stream(&one, 1, B, T, noise, noise_done, workspace, workspace_bytes, st);
         if (rc <= 0) return rc;                 // 1: not even one segment per tile fits -> the single-CTA kernel below
     }
     if (mt == 2)
@@ -1389,10 +1391,25 @@ static int gram_layers_sqnorms(const dpclip_layer* layers, int L, int B, dpclip_
     return DPCLIP_OK;
 }
 
+static int shared_clipped_grad_launches(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype,
+                                        const float* clip, long clip_ld, float C, float sigma, unsigned long long seed,
+                                        unsigned long long stream_id0, int* taken, void* workspace,
+                                        size_t workspace_bytes, void* stream);
+
 int dpclip_same_shape_layers_clipped_grad_noise(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype,
                                                 const float* clip, float C, float sigma, unsigned long long seed,
                                                 unsigned long long stream_id0, int* taken, void* workspace,
                                                 size_t workspace_bytes, void* stream) {
+    return shared_clipped_grad_launches(layers, L, B, dtype, clip, 0, C, sigma, seed, stream_id0, taken, workspace,
+                                        workspace_bytes, stream);
+}
+
+// clip_ld = 0: one factor vector for all layers (global clipping); clip_ld > 0: layer l's factors are row l of
+// clip[L][clip_ld] (per-layer clipping) -- then only the CTA-pair launches, which take a vector per layer, are made.
+static int shared_clipped_grad_launches(const dpclip_layer* layers, int L, int B, dpclip_dtype dtype,
+                                        const float* clip, long clip_ld, float C, float sigma, unsigned long long seed,
+                                        unsigned long long stream_id0, int* taken, void* workspace,
+                                        size_t workspace_bytes, void* stream) {
     if (!layers || L <= 0 || B <= 0) return DPCLIP_ERR_INVALID_ARG;
     if (!(C >= 0.f) || !(sigma >= 0.f)) return DPCLIP_ERR_INVALID_ARG;
     if (taken) for (int l = 0; l < L; ++l) taken[l] = 0;
@@ -1419,7 +1436,7 @@ int dpclip_same_shape_layers_clipped_grad_noise(const dpclip_layer* layers, int 
             const dpclip_layer& y = layers[l];
             if (done[l] || y.T != layers[l0].T || !pair_tile_ok(y.d_out) || !candidate(y)) continue;
             grp[n] = {y.A, y.lda, y.Zbar, y.ldz, y.d_in, y.d_out, y.gW, y.ldg, y.has_bias ? y.gb : nullptr,
-                      stream_id0 + 2ull * l, stream_id0 + 2ull * l + 1};
+                      stream_id0 + 2ull * l, stream_id0 + 2ull * l + 1, clip ? clip + (size_t)l * clip_ld : nullptr};
             idx[n] = l; ++n;
             tiles += pair_tiles(y.d_in, y.d_out);
         }
@@ -1429,7 +1446,7 @@ int dpclip_same_shape_layers_clipped_grad_noise(const dpclip_layer* layers, int 
         if (workspace_bytes < kHeaderBytes + pair_scratch_bytes(tiles)) continue;
         const NoiseSpec ns = {sigma * C, seed, 0, 0};
         bool noise_done = false;
-        const int rc = launch_zta_stream(grp, n, B, layers[l0].T, clip, &ns, &noise_done, workspace, workspace_bytes,
+        const int rc = launch_zta_stream(grp, n, B, layers[l0].T, &ns, &noise_done, workspace, workspace_bytes,
                                          (cudaStream_t)stream);
         if (rc < 0) return rc;
         if (rc > 0) continue;
@@ -1437,6 +1454,7 @@ int dpclip_same_shape_layers_clipped_grad_noise(const dpclip_layer* layers, int 
         if (!taken) return DPCLIP_ERR_INVALID_ARG;               // without `taken` the caller cannot know
         for (int i = 0; i < n; ++i) { done[idx[i]] = true; taken[idx[i]] = 1; }
     }
+    if (clip_ld > 0) return DPCLIP_OK;
     for (int l0 = 0; l0 < L; ++l0) {
         if (done[l0] || !candidate(layers[l0])) continue;
         const dpclip_layer* grp[z::MAX_LAYERS];
@@ -2223,25 +2241,55 @@ int dpclip_step_per_layer(const dpclip_layer* layers, int L, int B, dpclip_dtype
         c2 += (double)C_layer[l] * C_layer[l];
     }
     const float C_total = (float)sqrt(c2);               // sensitivity of the concatenated clipped gradient
-    // Layer by layer, norm -> factors -> clipped sum back to back: no layer waits for another one's norm, and
-    // the clipped sum re-reads inputs its own norm pass has just pulled through L2.
     for (int l = 0; l < L; ++l) {
         const dpclip_layer& y = layers[l];
-        float* sq = sq_layers + (size_t)l * B;
-        float* clip = clip_layers + (size_t)l * B;
-        float* gb = y.has_bias ? y.gb : nullptr;
-        if (!y.gW || (y.has_bias && !gb)) return DPCLIP_ERR_INVALID_ARG;
+        if (!y.gW || (y.has_bias && !y.gb)) return DPCLIP_ERR_INVALID_ARG;
         if (y.ldg != y.d_in) return DPCLIP_ERR_UNSUPPORTED;            // noise indexes the dense tensor
-        int rc = dpclip_layer_sqnorms(y.A, y.lda, y.Zbar, y.ldz, B, y.T, y.d_in, y.d_out, dtype, y.has_bias,
-                                      (dpclip_method)y.method, sq, workspace, workspace_bytes, stream);
+    }
+    int rc;
+    // The stages of the global step with a factor vector per layer: every layer's norms (the layers that go by
+    // the Gram identity in one launch), then ALL rows of factors in one launch (row l against C_layer[l]), then
+    // the clipped sums -- the wide bf16 layers of one T in one CTA-pair launch, each with its own factor row --
+    // with the noise N(0, sigma^2 * sum_l C_l^2).  (Layer after layer, norm -> factors -> clipped sum, so that a
+    // layer's second pass finds its inputs in L2, took 566 us on the sequence workload: it gives up both shared
+    // launches, and a wide layer's inputs do not fit L2 anyway.)
+    constexpr int kMaxTracked = 64;
+    int in_gram[kMaxTracked], in_pairs[kMaxTracked];
+    const bool track = L <= kMaxTracked;
+    if (track) {
+        rc = dpclip_gram_layers_sqnorms(layers, L, B, dtype, sq_layers, in_gram, workspace, workspace_bytes, stream);
         if (rc) return rc;
-        rc = dpclip_factors(sq, 1, B, B, C_layer[l], clip, norms_layers ? norms_layers + (size_t)l * B : nullptr, nullptr,
-                            stream);
+    }
+    for (int l = 0; l < L; ++l) {
+        const dpclip_layer& y = layers[l];
+        if (track && in_gram[l]) continue;
+        rc = dpclip_layer_sqnorms(y.A, y.lda, y.Zbar, y.ldz, B, y.T, y.d_in, y.d_out, dtype, y.has_bias,
+                                  (dpclip_method)y.method, sq_layers + (size_t)l * B, workspace, workspace_bytes, stream);
         if (rc) return rc;
+    }
+    if (track) {
+        LayerThresholds th;
+        for (int l = 0; l < L; ++l) th.C[l] = C_layer[l];
+        factors_rows_kernel<<<L, 256, 0, (cudaStream_t)stream>>>(sq_layers, (long)B, B, th, clip_layers, norms_layers);
+        if (launch_status()) return DPCLIP_ERR_CUDA;
+        rc = shared_clipped_grad_launches(layers, L, B, dtype, clip_layers, (long)B, C_total, sigma, seed, stream_id0,
+                                          in_pairs, workspace, workspace_bytes, stream);
+        if (rc) return rc;
+    } else {
+        for (int l = 0; l < L; ++l) {
+            rc = dpclip_factors(sq_layers + (size_t)l * B, 1, B, B, C_layer[l], clip_layers + (size_t)l * B,
+                                norms_layers ? norms_layers + (size_t)l * B : nullptr, nullptr, stream);
+            if (rc) return rc;
+        }
+    }
+    for (int l = 0; l < L; ++l) {
+        const dpclip_layer& y = layers[l];
+        if (track && in_pairs[l]) continue;
+        float* gb = y.has_bias ? y.gb : nullptr;
         NoiseSpec ns = {sigma * C_total, seed, stream_id0 + 2ull * l, stream_id0 + 2ull * l + 1};
         bool noise_done = false;
-        rc = clipped_grad_impl(y.A, y.lda, y.Zbar, y.ldz, B, y.T, y.d_in, y.d_out, dtype, clip, y.gW, y.ldg, gb, workspace,
-                               workspace_bytes, &ns, &noise_done, (cudaStream_t)stream);
+        rc = clipped_grad_impl(y.A, y.lda, y.Zbar, y.ldz, B, y.T, y.d_in, y.d_out, dtype, clip_layers + (size_t)l * B, y.gW,
+                               y.ldg, gb, workspace, workspace_bytes, &ns, &noise_done, (cudaStream_t)stream);
         if (rc) return rc;
         if (!noise_done) {
             rc = dpclip_add_noise(y.gW, (size_t)y.d_out * y.d_in, sigma, C_total, seed, ns.sid_w, stream);

@@ -68,6 +68,23 @@ factors_kernel(const float* __restrict__ sq_layers, int L, long ld_sq, int B, fl
     }
 }
 
+// Per-layer clipping (Sec. "Related Work"): row l of sq[L][B] gives layer l's own factors against its own
+// threshold C[l].  One CTA per layer.
+struct LayerThresholds { float C[64]; };
+__global__ void __launch_bounds__(256)
+factors_rows_kernel(const float* __restrict__ sq_layers, long ld_sq, int B, const LayerThresholds th,
+                    float* __restrict__ clip_layers, float* __restrict__ norms_layers) {
+    const int l = blockIdx.x;
+    const float C = th.C[l];
+    for (int i = threadIdx.x; i < B; i += blockDim.x) {
+        const float n = sqrtf(sq_layers[(size_t)l * ld_sq + i]);
+        float c = 1.0f;
+        if (n > C) c = C / n;                         // tie and zero norm stay exactly 1
+        clip_layers[(size_t)l * B + i] = c;
+        if (norms_layers) norms_layers[(size_t)l * B + i] = n;
+    }
+}
+
 // ---------------------------------------------------------------------------
 // Gaussian noise: Philox4x32-10 counter-based generator + Box-Muller.
 // One 128-bit block gives four normals; a thread owns block q = elements

@@ -77,6 +77,8 @@ struct Layer {
     int tiles_n;                   // pair tiles along d_in
     int tile_base, tiles;          // this layer's tiles are tile_base .. tile_base + tiles - 1 of the launch
     int do_bias;
+    const float* clip;             // [B] factors of THIS layer, or NULL (all ones): one vector for the whole model under
+                                   // global clipping, one per layer under per-layer clipping
     float* gW; float* gb;          // outputs (dense rows: ldg = d_in for the noise; see ldg)
     long ldg; int vec_ok;
     uint32_t sw0, sw1, sb0, sb1;   // noise streams of gW and gb
@@ -94,7 +96,6 @@ struct Params {
     short super_tile[MAX_TILES];   // [n_super][W]: tile of the launch at position j of super-layer s, or -1
     short tile_slot[MAX_TILES];    // [G]: s * W + j of every tile
     int any_bias;
-    const float* clip;             // [B] or NULL
     long n_segments;               // partial tiles the workspace holds (range checks of the debug build)
     float* part;                   // [n_segments][BM][BN] fp32
     float* bias_part;              // [n_segments][BM] fp32, or NULL when no layer has a bias
@@ -103,9 +104,9 @@ struct Params {
     Layer layer[MAX_LAYERS];
 };
 
-__device__ __forceinline__ float row_factor(const Params& p, int e) {
+__device__ __forceinline__ float row_factor(const Params& p, const float* clip, int e) {
     if (!DPCLIP_IN_RANGE(e, (p.R + p.T - 1) / p.T, p.status)) return 0.f;
-    return p.clip ? __ldg(p.clip + e) : 1.f;
+    return clip ? __ldg(clip + e) : 1.f;
 }
 
 __host__ __device__ __forceinline__ long segment_of(long u, int S, int U, long lcm) { return u / S + u / U - u / lcm; }
@@ -268,6 +269,7 @@ zta_pair_kernel(const __grid_constant__ zta::Maps maps, const __grid_constant__ 
         for (long u = u_begin; u < u_end && ok;) {
             const Seg w = segment_at(p, u, u_end, gj);
             if (w.layer < 0) { u += w.kb1 - w.kb0; continue; }
+            const float* lclip = p.layer[w.layer].clip;
             for (int kb = w.kb0; kb < w.kb1; ++kb) {
                 // the factors of this stage's rows are fetched BEFORE waiting for the tile, so the global-load
                 // latency overlaps the wait instead of sitting between TMA and MMA
@@ -278,7 +280,7 @@ zta_pair_kernel(const __grid_constant__ zta::Maps maps, const __grid_constant__ 
                 constexpr int NR = BK / 16;
                 float fr[NR];
                 if (uniform) {
-                    const float f = row_factor(p, e_first);            // one factor for the whole stage
+                    const float f = row_factor(p, lclip, e_first);     // one factor for the whole stage
 #pragma unroll
                     for (int i = 0; i < NR; ++i) fr[i] = f;
                 } else {
@@ -286,7 +288,7 @@ zta_pair_kernel(const __grid_constant__ zta::Maps maps, const __grid_constant__ 
                     for (int i = 0; i < NR; ++i) {
                         const int rl = rs + 16 * i;
                         // past the last row TMA filled zeros; the factor only has to be finite there
-                        fr[i] = blk0 + rl >= p.R ? 0.f : row_factor(p, e_first + (rem0 + rl) / p.T);
+                        fr[i] = blk0 + rl >= p.R ? 0.f : row_factor(p, lclip, e_first + (rem0 + rl) / p.T);
                     }
                 }
                 ok = mbar_wait(&full[stage], phase, abort_flag, p.status);
@@ -349,6 +351,7 @@ zta_pair_kernel(const __grid_constant__ zta::Maps maps, const __grid_constant__ 
             const Seg w = segment_at(p, u, u_end, gj);
             if (w.layer < 0) { u += w.kb1 - w.kb0; continue; }
             const Layer& y = p.layer[w.layer];
+            const float* lclip = y.clip;
             if (p.any_bias) {
                 float cs[2][8];
 #pragma unroll
@@ -367,14 +370,14 @@ zta_pair_kernel(const __grid_constant__ zta::Maps maps, const __grid_constant__ 
                         const int rem0 = blk0 - e_first * p.T;
                         const bool uniform = (rem0 + BK <= p.T) && (blk0 + BK <= p.R);
                         if (uniform) {
-                            const float f = row_factor(p, e_first);
+                            const float f = row_factor(p, lclip, e_first);
 #pragma unroll
                             for (int i = 0; i < NR; ++i) fr[i] = f;
                         } else {
 #pragma unroll
                             for (int i = 0; i < NR; ++i) {
                                 const int rl = rs + 16 * i;
-                                fr[i] = blk0 + rl >= p.R ? 0.f : row_factor(p, e_first + (rem0 + rl) / p.T);
+                                fr[i] = blk0 + rl >= p.R ? 0.f : row_factor(p, lclip, e_first + (rem0 + rl) / p.T);
                             }
                         }
                     }

@@ -194,6 +194,37 @@ def test_sequence_workload_full_step_gradients(dp, form):
             assert rel_fro(plan.gb[l].cpu().numpy(), _bias_definition(Z, clip)) <= TOL["bf16"]["grad"], spec.name
 
 
+def test_sequence_workload_full_step_per_layer_clipping(dp):
+    """Per-layer clipping at B=128, T=256 (every layer against its own threshold, Sec. "Related Work"): one Gram launch
+    for the norms, one launch for all rows of factors, one CTA-pair launch in which every layer carries its own
+    factor vector.  Factors of sampled examples against the oracle; every released tensor by probes with that
+    layer's own factor row."""
+    w = workloads.seq("bf16")
+    layers = workloads.generate(w, seed=3)
+    hb = [s.has_bias for s in w.layers]
+    plan = dp.StepPlan([dp.Layer(to_device(A, "bf16"), to_device(Z, "bf16"), b) for (A, Z), b in zip(layers, hb)])
+    sample = np.array([1, 66, 120])
+    sq = np.stack([oracle.layer_sqnorms(A[sample], Z[sample], b) for (A, Z), b in zip(layers, hb)])
+    # thresholds near each layer's own typical norm, so that both sides of every threshold occur
+    Cl = [float(np.sqrt(np.median(sq[l]))) for l in range(plan.L)]
+    plan.flat.fill_(float("nan"))
+    clip_layers = dp.dpclip_step_per_layer(plan, Cl, 0.0, seed=0)
+    torch.cuda.synchronize()
+    assert dp.dpclip_read_status(plan.workspace) == 0
+    clips = clip_layers.cpu().numpy()
+    rng = np.random.default_rng(13)
+    for l, ((A, Z), spec) in enumerate(zip(layers, w.layers)):
+        n_ref, c_ref = oracle.factors(sq[l:l + 1], Cl[l])
+        assert np.max(np.abs(clips[l][sample] - c_ref)) <= 5e-3, spec.name
+        assert 0 < (clips[l] < 1).sum() < w.B, spec.name
+        G = plan.gW[l].cpu().numpy()
+        assert np.all(np.isfinite(G)), spec.name
+        err, bound = _probe_whole_gradient(A, Z, clips[l].astype(np.float64), G, rng, TOL["bf16"]["grad"])
+        assert err <= bound, (spec.name, err, bound)
+        if spec.has_bias:
+            assert rel_fro(plan.gb[l].cpu().numpy(), _bias_definition(Z, clips[l])) <= TOL["bf16"]["grad"], spec.name
+
+
 def test_same_shape_layers_launch_full_size_against_the_oracle(dp):
     """The launch that carries the four 512->512 projections at B=128, T=256 (their d_out tiles stacked, 14 stages
     per CTA, one reduce over all four with per-layer outputs), called directly with factors that are zero outside
