@@ -47,7 +47,7 @@ enum PathSwitch : unsigned {
     SW_FORCE_SIMT = 1u << 0, SW_NO_NARROW = 1u << 1, SW_NO_NARROW_RING = 1u << 2, SW_NO_NARROW_TC = 1u << 3,
     SW_NO_NARROW_PACK = 1u << 4, SW_NARROW_PACK_BF16 = 1u << 5, SW_NO_GRAM_Q2 = 1u << 6, SW_NO_T1_TF32 = 1u << 7,
     SW_NO_FUSED_T1 = 1u << 8, SW_NO_GRAM_GROUP = 1u << 9, SW_NO_GRAD_GROUP = 1u << 10, SW_NO_CONV_TC = 1u << 11,
-    SW_NO_CONV_PATCHES = 1u << 12, SW_TILE_M1 = 1u << 13, SW_TILE_M2 = 1u << 14, SW_T1_TWO_LAUNCHES = 1u << 15, SW_NO_PAIR = 1u << 16, SW_LOG = 1u << 17, SW_NO_FACTORS_TAIL = 1u << 18,
+    SW_NO_CONV_PATCHES = 1u << 12, SW_TILE_M1 = 1u << 13, SW_TILE_M2 = 1u << 14, SW_T1_TWO_LAUNCHES = 1u << 15, SW_NO_PAIR = 1u << 16, SW_LOG = 1u << 17, SW_NO_FACTORS_TAIL = 1u << 18, SW_NO_SM_BUDGET = 1u << 19,
     SW_LOADED = 1u << 31
 };
 std::atomic<unsigned> g_path_switches{0};
@@ -62,7 +62,7 @@ unsigned read_path_switches() {
         {"DPCLIP_NO_CONV_PATCHES", SW_NO_CONV_PATCHES, '1'}, {"DPCLIP_TILE_M", SW_TILE_M1, '1'},
         {"DPCLIP_TILE_M", SW_TILE_M2, '2'}, {"DPCLIP_T1_ONE_LAUNCH", SW_T1_TWO_LAUNCHES, '0'},
         {"DPCLIP_NO_PAIR", SW_NO_PAIR, '1'}, {"DPCLIP_LOG", SW_LOG, '1'},
-        {"DPCLIP_NO_FACTORS_TAIL", SW_NO_FACTORS_TAIL, '1'},
+        {"DPCLIP_NO_FACTORS_TAIL", SW_NO_FACTORS_TAIL, '1'}, {"DPCLIP_NO_SM_BUDGET", SW_NO_SM_BUDGET, '1'},
     };
     unsigned v = SW_LOADED;
     for (const auto& e : table) {
@@ -77,6 +77,19 @@ inline bool path_switch(unsigned bit) {
     if (!(v & SW_LOADED)) v = read_path_switches();
     return (v & bit) != 0;
 }
+
+// SM budget of the calling thread's next launches (0 = the whole GPU).  A step that spreads small layers over
+// several streams gives each launch a share of the SMs in proportion to its bytes: launches of a few
+// megabytes are chains of round trips, not throughput problems, so running four of them side by side on a
+// quarter of the SMs each costs each one little and hides the others' latency; launched at full width they
+// queue for the SMs (one CTA per SM) and run one after the other.
+thread_local int t_sm_budget = 0;
+inline int sm_budget() { return t_sm_budget > 0 && t_sm_budget < kNumSMs ? t_sm_budget : kNumSMs; }
+struct SmBudgetScope {
+    int prev;
+    explicit SmBudgetScope(int b) : prev(t_sm_budget) { t_sm_budget = b; }
+    ~SmBudgetScope() { t_sm_budget = prev; }
+};
 
 // DPCLIP_LOG=1: one line on stderr per dispatch decision (which form of a kernel a layer takes and how its
 // work is cut) -- host side only, nothing changes on the device.
@@ -245,9 +258,9 @@ int launch_simt_norms(const void* A, long lda, const void* Z, long ldz, int B, i
         q.A = A; q.lda = lda; q.Z = Z; q.ldz = ldz; q.T = T; q.d_in = d_in; q.d_out = d_out;
         q.has_bias = has_bias ? 1 : 0; q.sq = sq;
         if (narrow_pack_ok(q, dtype, status))
-            return launch_narrow_pack<false>(q, B < kNumSMs ? B : kNumSMs, B, dtype, status, st);
+            return launch_narrow_pack<false>(q, B < sm_budget() ? B : sm_budget(), B, dtype, status, st);
         if (narrow_tc_ok(q, dtype, status))
-            return launch_narrow_tc<false>(q, B < kNumSMs ? B : kNumSMs, B, status, st);
+            return launch_narrow_tc<false>(q, B < sm_budget() ? B : sm_budget(), B, status, st);
         return launch_narrow<false>(q, B, d_out, dtype, st);
     }
     SimtParams p;
@@ -282,7 +295,7 @@ int launch_simt_grad(const void* A, long lda, const void* Z, long ldz, int B, in
         const bool on_pack = narrow_pack_ok(q, dtype, status);
         const bool on_tc = on_pack || narrow_tc_ok(q, dtype, status);
         // one wave: a CTA of the register-staged kernel holds a whole SM; the cp.async form runs two per SM
-        int grid = (!on_tc && narrow_ring_ok(q, dtype, true)) ? 2 * kNumSMs : kNumSMs;
+        int grid = (!on_tc && narrow_ring_ok(q, dtype, true)) ? 2 * sm_budget() : sm_budget();
         const long min_rows = NARROW_WARPS * 32;                   // at least one chunk per warp
         if ((long)grid * min_rows > q.rows_total) grid = (int)((q.rows_total + min_rows - 1) / min_rows);
         // whole 32-row chunks per CTA: every chunk of a dense layer then starts on a 16-byte boundary whatever
@@ -477,7 +490,7 @@ int launch_gram_group(const GramLayer* ls, int n, int* status, cudaStream_t st,
         q.tail = *tail;
         q.tail.done = reinterpret_cast<unsigned int*>(reinterpret_cast<char*>(status) + kTailCounterOffset);
     }
-    const int grid = groups < kNumSMs ? groups : kNumSMs;
+    const int grid = groups < sm_budget() ? groups : sm_budget();
     if (cls == 0) {
         q.work_counter = reinterpret_cast<unsigned int*>(reinterpret_cast<char*>(status) + kWorkCounterOffset);
         if (!enable_smem(tc::gram_norm_q2_kernel, g::SMEM_BYTES)) return DPCLIP_ERR_CUDA;
@@ -597,8 +610,9 @@ int launch_zta_tc_mt(const tc::zta::Maps& maps, tc::zta::Params p, int B, bool n
         // One wave of equally long items: the kernel is bound by L2->SM traffic, so what matters is that
         // every SM streams the same number of row blocks.  (MT = 1 has two accumulator buffers and can
         // overlap the epilogue of one item with the next, so it takes two items per SM when they stay long.)
-        const int per_sm = (MT == 1 && tiles <= kNumSMs && nkb / ((2 * kNumSMs) / tiles) >= 16) ? 2 : 1;
-        const ZtaSplit split = zta_pick_split(nkb, tiles, per_sm);
+        const int sms = sm_budget();
+        const int per_sm = (MT == 1 && tiles <= sms && nkb / ((2 * sms) / tiles) >= 16) ? 2 : 1;
+        const ZtaSplit split = zta_pick_split(nkb, tiles, per_sm, sms);
         // the preferred split when the workspace holds its partial tiles, else one wave
         ksplit = split.one_wave;
         if (split.preferred != split.one_wave && !fit_to_workspace &&
@@ -627,7 +641,7 @@ int launch_zta_tc_mt(const tc::zta::Maps& maps, tc::zta::Params p, int B, bool n
         }
     }
     if (!enable_smem(tc::zta_tc_kernel<MT>, z::SMEM_BYTES)) return DPCLIP_ERR_CUDA;
-    const int grid = p.n_items < kNumSMs ? p.n_items : kNumSMs;
+    const int grid = p.n_items < sm_budget() ? p.n_items : sm_budget();
     tc::zta_tc_kernel<MT><<<grid, z::THREADS, z::SMEM_BYTES, st>>>(maps, p);
     int rc = launch_status();
     if (rc || norm_mode || ksplit == 1) return rc;
@@ -918,8 +932,9 @@ int launch_zta_tf32(const void* A, long lda, const void* Z, long ldz, int B, int
         p.vec_ok = aligned_to(gW, 16) && ldg % 4 == 0;
         const int nkb = ceil_div(R, t::BK);
         // two accumulator buffers: two items per SM when they stay long enough, else one wave
-        const int per_sm = (tiles <= kNumSMs && nkb / ((2 * kNumSMs) / tiles) >= 16) ? 2 : 1;
-        ksplit = (per_sm * kNumSMs) / tiles;
+        const int sms = sm_budget();
+        const int per_sm = (tiles <= sms && nkb / ((2 * sms) / tiles) >= 16) ? 2 : 1;
+        ksplit = (per_sm * sms) / tiles;
         if (ksplit > nkb) ksplit = nkb;
         if (ksplit < 1) ksplit = 1;
         p.kb_per_split = ceil_div(nkb, ksplit);
@@ -935,7 +950,7 @@ int launch_zta_tf32(const void* A, long lda, const void* Z, long ldz, int B, int
             return DPCLIP_ERR_CUDA;
         }
     }
-    const int grid = p.n_items < kNumSMs ? p.n_items : kNumSMs;
+    const int grid = p.n_items < sm_budget() ? p.n_items : sm_budget();
     if (conv) {
         if (!enable_smem(tc::zta_tf32_kernel<true>, t::SMEM_BYTES)) return DPCLIP_ERR_CUDA;
         tc::zta_tf32_kernel<true><<<grid, t::THREADS, t::SMEM_BYTES, st>>>(ma, mz, p, *conv);
@@ -1642,7 +1657,7 @@ static int launch_conv_tc(const SimtParams& sp, const void* X, const void* Zbar,
     int slices = 1;
     if (GRAD) {
         // one wave: as many slices of examples as there are SMs per block of patch columns
-        slices = kNumSMs / p.tiles_n;
+        slices = sm_budget() / p.tiles_n;
         if (slices > B) slices = B;
         if (slices < 1) slices = 1;
         p.ex_per_item = ceil_div(B, slices);
@@ -1659,7 +1674,7 @@ static int launch_conv_tc(const SimtParams& sp, const void* X, const void* Zbar,
         if (cudaMemsetAsync(sq, 0, sizeof(float) * (size_t)B, st) != cudaSuccess) return DPCLIP_ERR_CUDA;
     }
     if (!enable_smem(tc::conv_tc_kernel<GRAD>, c::SMEM_BYTES)) return DPCLIP_ERR_CUDA;
-    const int grid = p.n_items < kNumSMs ? p.n_items : kNumSMs;
+    const int grid = p.n_items < sm_budget() ? p.n_items : sm_budget();
     tc::conv_tc_kernel<GRAD><<<grid, c::THREADS, c::SMEM_BYTES, st>>>(mz, p);
     int rc = launch_status();
     if (rc || !GRAD) return rc;
@@ -2087,11 +2102,48 @@ static int step_general(const dpclip_layer* layers, const dpclip_model_layer* ot
         if (rc) return rc;
         for (int l = 0; l < L; ++l) any_gram = any_gram || in_gram_group[l];
     }
+    // SM shares for the per-layer launches of a stage (see t_sm_budget): only when several of them run side by
+    // side on different lanes, no launch shared by several layers is in the stage, and the stage is small
+    const size_t es = elt_size(dtype);
+    auto layer_bytes = [&](int l) -> double {
+        if (other && other[l].kind == DPCLIP_KIND_CONV) {
+            const dpclip_conv& g = other[l].conv;
+            const double Ho = (g.H + 2 * g.pad - g.kh) / g.stride + 1, Wo = (g.W + 2 * g.pad - g.kw) / g.stride + 1;
+            return (double)B * ((double)g.C * g.H * g.W + Ho * Wo * other[l].layer.d_out) * es;
+        }
+        const dpclip_layer& y = other && other[l].kind != DPCLIP_KIND_DENSE ? other[l].layer : layers[l];
+        return (double)B * y.T * ((double)y.d_in + y.d_out) * es;
+    };
+    auto stage_budgets = [&](const int* skip, bool shared_launch, int* budget) {
+        int n_ent = 0;
+        double total = 0.0;
+        for (int l = 0; l < L; ++l) {
+            budget[l] = 0;
+            const bool is_other = other && other[l].kind != DPCLIP_KIND_DENSE;
+            if (!is_other && ((t1.active && layers[l].T == 1) || (skip && skip[l]))) continue;
+            ++n_ent; total += layer_bytes(l);
+        }
+        // bf16 only: the fp32 forms (three tf32 MMAs per product, four operand planes to prepare, gathers) are
+        // bound by their own work, and a share of the SMs stretches them in proportion (measured: the feature-map
+        // CNN in fp32 242 -> 312 us with shares, in bf16 98 -> 86 us; the patch-matrix CNN in bf16 94 -> 79 us)
+        if (dtype != DPCLIP_BF16 || lanes.n < 2 || n_ent < 2 || shared_launch || total > 400e6 ||
+            path_switch(SW_NO_SM_BUDGET)) return;
+        const double widen = n_ent > lanes.n ? (double)n_ent / lanes.n : 1.0;      // more launches than lanes: some queue
+        for (int l = 0; l < L; ++l) {
+            const bool is_other = other && other[l].kind != DPCLIP_KIND_DENSE;
+            if (!is_other && ((t1.active && layers[l].T == 1) || (skip && skip[l]))) continue;
+            int b = (int)(kNumSMs * layer_bytes(l) / total * widen + 0.5);
+            budget[l] = b < 16 ? 16 : (b > kNumSMs ? kNumSMs : b);
+        }
+    };
+    int budget[64] = {0};
+    if (track) stage_budgets(in_gram_group, any_gram, budget);
     int k = any_gram ? 1 : 0;                              // lane 0 already carries the shared Gram launch
     for (int l = 0; l < L; ++l) {
         const dpclip_layer& y = layers[l];
         const bool is_other = other && other[l].kind != DPCLIP_KIND_DENSE;
         if (!is_other && ((t1.active && y.T == 1) || (track && in_gram_group[l]))) continue;
+        const SmBudgetScope share(track ? budget[l] : 0);
         const int b = k++ % lanes.n;
         if (is_other)
             rc = other_kind_sqnorms(other[l], B, dtype, sq_layers + (size_t)l * B, lanes.ws[b], workspace_bytes, lanes.st[b]);
@@ -2120,11 +2172,13 @@ static int step_general(const dpclip_layer* layers, const dpclip_model_layer* ot
         if (rc) return rc;
         for (int l = 0; l < L; ++l) any_group = any_group || in_grad_group[l];
     }
+    if (track) stage_budgets(in_grad_group, any_group, budget);
     k = any_group ? 1 : 0;
     for (int l = 0; l < L; ++l) {
         const dpclip_layer& y = layers[l];
         const bool is_other = other && other[l].kind != DPCLIP_KIND_DENSE;
         if (!is_other && ((t1.active && y.T == 1) || (track && in_grad_group[l]))) continue;
+        const SmBudgetScope share(track ? budget[l] : 0);
         const int b = k++ % lanes.n;
         void* const stream = lanes.st[b];
         void* const workspace = lanes.ws[b];
