@@ -469,8 +469,9 @@ int launch_gram_group(const GramLayer* ls, int n, int* status, cudaStream_t st,
         q.group_begin[k] = groups;
         groups += p.n_groups;
     }
-    // the kernel accumulates with atomics: clear the rows, adjacent rows of sq in one memset
-    {
+    // the general kernels accumulate with atomics: clear the rows, adjacent rows of sq in one memset (the kernel
+    // for examples of two row blocks stores every norm, so its rows need no clearing)
+    if (cls != 0) {
         int by_ptr[g::MAX_LAYERS];
         for (int i = 0; i < n; ++i) by_ptr[i] = i;
         for (int i = 1; i < n; ++i)
@@ -768,6 +769,14 @@ int launch_zta_stream(const StreamLayer* ls, int n, int B, int T, const NoiseSpe
     p.lcm = (long)p.S / gcd_l(p.S, U) * U;
     const long n_segments = (zp::segment_of(p.total - 1, p.S, p.U, p.lcm) + 1) * W;
     p.n_segments = n_segments;
+    for (int t = 0; t < G; ++t) {                                   // the reduce kernel's view of the same cut
+        const long sl = p.tile_slot[t] / W, j = p.tile_slot[t] % W;
+        const long s0 = zp::segment_of(sl * p.S, p.S, p.U, p.lcm), s1 = zp::segment_of((sl + 1) * p.S - 1, p.S, p.U, p.lcm);
+        p.seg_first[t] = (int)(s0 * W + j);
+        p.seg_count[t] = (short)(s1 - s0 + 1);
+    }
+    for (int l = 0; l < n; ++l)
+        for (int t = 0; t < p.layer[l].tiles; ++t) p.tile_layer[p.layer[l].tile_base + t] = (unsigned char)l;
     p.part = reinterpret_cast<float*>(static_cast<char*>(workspace) + kHeaderBytes);
     p.bias_part = p.any_bias ? p.part + (size_t)n_segments * zp::SEG_ELEMS : nullptr;
     if (fuse_noise) {
@@ -783,15 +792,10 @@ int launch_zta_stream(const StreamLayer* ls, int n, int B, int T, const NoiseSpe
     tc::zta_pair_kernel<<<2 * pairs, zp::THREADS, zp::SMEM_BYTES, st>>>(maps, p);
     int rc = launch_status();
     if (rc) return rc;
-    long most = 0;
-    for (int l = 0; l < n; ++l) {
-        const long v = (long)ls[l].d_out * ((ls[l].d_in + 3) / 4);
-        if (v > most) most = v;
-    }
-    long blocks = ceil_div(most, 256L);
-    if (blocks > 4L * kNumSMs) blocks = 4L * kNumSMs;
-    if (blocks < 1) blocks = 1;
-    tc::reduce_segments_kernel<<<dim3((unsigned)blocks, n), 256, 0, st>>>(p);
+    // one wave of CTAs (six of 256 threads and 40 registers per SM) over the 4-row blocks of all tiles
+    long blocks = (long)G * (zp::BM / 4);
+    if (blocks > 6L * kNumSMs) blocks = 6L * kNumSMs;
+    tc::reduce_segments_kernel<<<(unsigned)blocks, 256, 0, st>>>(p);
     return launch_status();
 }
 

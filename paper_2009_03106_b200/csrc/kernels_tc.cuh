@@ -62,7 +62,7 @@ template <bool DIAG_ONLY> struct Cfg {
 };
 constexpr int N_EPILOGUE_WARPS = 8;
 constexpr int THREADS = 64 + 32 * N_EPILOGUE_WARPS;   // warp 0 TMA, warp 1 MMA, warps 2..9 epilogue
-constexpr int SMEM_BYTES = 4 * 3 * TILE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;   // = 6 * 2 tiles
+constexpr int SMEM_BYTES = 4 * 3 * TILE_BYTES + 1024 /*alignment slack*/ + 512 /*barriers, queues, warp sums*/;   // = 6 * 2 tiles
 
 constexpr int MAX_LAYERS = 8;                 // layers one launch can take
 
@@ -374,6 +374,10 @@ gram_norm_kernel(const __grid_constant__ gram::Launch q) {
 //                                                                            block (0,1) counted twice
 // Only the narrower operand's second half is read twice, a few hundred KB apart (an L2 hit).  All 512
 // columns are in use, so E1 must finish before P3 starts and E0 before the next example's P1.
+//
+// An example belongs to one CTA, so its squared norm is STORED, not accumulated: the eight epilogue warps leave
+// their sums in shared memory and the first of them adds these in a fixed order.  The row of sq needs no
+// clearing before the launch and the result does not depend on the order of atomics.
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(gram::THREADS, 1)
 gram_norm_q2_kernel(const __grid_constant__ gram::Launch q) {
@@ -391,12 +395,18 @@ gram_norm_q2_kernel(const __grid_constant__ gram::Launch q) {
     volatile int* sched_item = reinterpret_cast<volatile int*>(sched_empty + SCHED);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(const_cast<int*>(sched_item) + SCHED);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    // barriers and queue end 200 bytes into their area; the next 8-byte boundary is three ints past the flag's address
+    static_assert((2 * STAGES + 2 + 2 * SCHED) * 8 + SCHED * 4 + 4 == 196, "offset of the abort flag");
+    uint64_t* sums_full = reinterpret_cast<uint64_t*>(const_cast<int*>(abort_flag) + 3);   // [2]: warp sums of an example are in
+    volatile float* sums = reinterpret_cast<volatile float*>(sums_full + 2);               // [2][N_EPILOGUE_WARPS]
+    static_assert(STAGES * STAGE_BYTES + 208 + 16 + 2 * N_EPILOGUE_WARPS * 4 + 1024 <= SMEM_BYTES, "shared memory layout");
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
         mbar_init(acc_full, 1); mbar_init(acc_empty, N_EPILOGUE_WARPS);
         for (int s = 0; s < SCHED; ++s) { mbar_init(&sched_full[s], 1); mbar_init(&sched_empty[s], 1 + N_EPILOGUE_WARPS); }
+        mbar_init(&sums_full[0], N_EPILOGUE_WARPS); mbar_init(&sums_full[1], N_EPILOGUE_WARPS);
         *abort_flag = 0;
         mbar_fence_init();
         for (int l = 0; l < q.L; ++l) { tma_prefetch_desc(&q.map_a[l]); tma_prefetch_desc(&q.map_z[l]); }
@@ -531,6 +541,7 @@ gram_norm_q2_kernel(const __grid_constant__ gram::Launch q) {
         const int half = (warp - 2) >> 2;
         uint32_t acc_phase = 0;
         int slot = 0; uint32_t sphase = 0;
+        int buf = 0; uint32_t sums_phase = 0;                  // bit b: phase of sums_full[b]
         bool ok = true;
         [[maybe_unused]] int etr = 0;
         const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16);
@@ -581,7 +592,21 @@ gram_norm_q2_kernel(const __grid_constant__ gram::Launch q) {
             }
             if (!ok) break;
             val = warp_sum(val);
-            if (lane == 0) atomicAdd(p.sq + e, val);
+            // Two buffers suffice: a warp writes the sums of example k + 2 only after the accumulators of that
+            // example were handed over, which needs the first warp's arrival for example k + 1, after its read here.
+            if (lane == 0) { sums[buf * N_EPILOGUE_WARPS + (warp - 2)] = val; mbar_arrive(&sums_full[buf]); }
+            if (warp == 2) {
+                ok = mbar_wait(&sums_full[buf], (sums_phase >> buf) & 1u, abort_flag, q.status);
+                if (!ok) break;
+                if (lane == 0) {
+                    float total = 0.f;
+#pragma unroll
+                    for (int w = 0; w < N_EPILOGUE_WARPS; ++w) total += sums[buf * N_EPILOGUE_WARPS + w];
+                    p.sq[e] = total;
+                }
+            }
+            sums_phase ^= 1u << buf;
+            buf ^= 1;
         }
     }
 

@@ -95,6 +95,9 @@ struct Params {
     long total, lcm;               // n_super * S; lcm(S, U)
     short super_tile[MAX_TILES];   // [n_super][W]: tile of the launch at position j of super-layer s, or -1
     short tile_slot[MAX_TILES];    // [G]: s * W + j of every tile
+    int seg_first[MAX_TILES];      // [G]: slot of the tile's first segment (first segment of its super-layer * W + j)
+    short seg_count[MAX_TILES];    // [G]: segments its stages are cut into; they lie W slots apart
+    unsigned char tile_layer[MAX_TILES];   // [G]: layer of the launch a tile belongs to
     int any_bias;
     long n_segments;               // partial tiles the workspace holds (range checks of the debug build)
     float* part;                   // [n_segments][BM][BN] fp32
@@ -475,34 +478,51 @@ zta_pair_kernel(const __grid_constant__ zta::Maps maps, const __grid_constant__ 
 
 // ---------------------------------------------------------------------------
 // Second stage: every output element = the fixed-order sum of its tile's segments (+ Philox noise), every bias =
-// the sum over the n-tiles and segments of its tile row.  blockIdx.y = layer.
+// the sum over the n-tiles and segments of its tile row.
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
 reduce_segments_kernel(const __grid_constant__ ztp::Params p) {
     using namespace ztp;
-    const Layer& y = p.layer[blockIdx.y];
-    const int n4 = (y.d_in + 3) >> 2;
-    const long total = (long)y.d_out * n4;
-    for (long idx = (long)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (long)gridDim.x * blockDim.x) {
-        const int m = (int)(idx / n4), n = (int)(idx - (long)m * n4) << 2;
-        const int tm = m / BM, tn = n / BN;
-        const int ts = p.tile_slot[y.tile_base + tm * y.tiles_n + tn];
-        const long sl = ts / p.W, j = ts - sl * p.W;
-        const long s0 = segment_of(sl * p.S, p.S, p.U, p.lcm), s1 = segment_of((sl + 1) * p.S - 1, p.S, p.U, p.lcm);
-        const float* src = p.part + (size_t)(s0 * p.W + j) * SEG_ELEMS + (size_t)(m - tm * BM) * BN + (n - tn * BN);
-        if (!DPCLIP_IN_RANGE(s1 * p.W + j, p.n_segments, p.status) || !DPCLIP_IN_RANGE(s0, s1 + 1, p.status)) continue;
-        float4 acc = __ldcs(reinterpret_cast<const float4*>(src));
-        for (long s = s0 + 1; s <= s1; ++s) {
-            src += (size_t)p.W * SEG_ELEMS;
-            const float4 v = __ldcs(reinterpret_cast<const float4*>(src));
-            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
-        }
+    // One wave of CTAs over the 4-row x 256-column blocks of every tile of every layer, one float4 per thread and
+    // block.  A tile's layer and segment range come from the host's tables (working the range out here cost six
+    // 64-bit divisions per block).  A thread issues the loads of up to four segments before the first add and draws
+    // its noise while they are in flight: with one load in flight per thread the kernel was bound by the latency of
+    // its serial loads; what binds it now is instruction issue (the Philox rounds and Box-Muller of every float4).
+    constexpr int ROWS = 4, SG = 4;
+    constexpr int ROW_BLOCKS = BM / ROWS;
+    const int n_blocks = p.G * ROW_BLOCKS;
+    const size_t seg_stride = (size_t)p.W * SEG_ELEMS;
+    const int c4 = (threadIdx.x & 63) << 2, r = threadIdx.x >> 6;
+    for (int blk = blockIdx.x; blk < n_blocks; blk += gridDim.x) {
+        const int t = blk / ROW_BLOCKS, rb = blk - t * ROW_BLOCKS;
+        const Layer& y = p.layer[p.tile_layer[t]];
+        const int tile = t - y.tile_base;
+        const int tm = tile / y.tiles_n, tn = tile - tm * y.tiles_n;
+        const int m = tm * BM + rb * ROWS + r, n = tn * BN + c4;
+        if (m >= y.d_out || n >= y.d_in) continue;
+        const int first = p.seg_first[t], n_seg = p.seg_count[t];
+        if (!DPCLIP_IN_RANGE(first + (long)(n_seg - 1) * p.W, p.n_segments, p.status) || n_seg < 1) continue;
+        const float* src = p.part + (size_t)first * SEG_ELEMS + (size_t)(rb * ROWS + r) * BN + c4;
+        float4 v[SG];
+#pragma unroll
+        for (int k = 0; k < SG; ++k)
+            v[k] = k < n_seg ? __ldcs(reinterpret_cast<const float4*>(src + (size_t)k * seg_stride))
+                             : make_float4(0.f, 0.f, 0.f, 0.f);
+        float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;
         if (p.noise_scale > 0.f) {
             const size_t qd = ((size_t)m * y.d_in + n) >> 2;
             PhiloxBlock b = philox_block((uint32_t)qd, (uint32_t)(qd >> 32), y.sw0, y.sw1, p.k0, p.k1);
-            float z0, z1, z2, z3;
             box_muller(b.v[0], b.v[1], z0, z1);
             box_muller(b.v[2], b.v[3], z2, z3);
+        }
+        float4 acc = v[0];                                                  // segment order
+#pragma unroll
+        for (int k = 1; k < SG; ++k) { acc.x += v[k].x; acc.y += v[k].y; acc.z += v[k].z; acc.w += v[k].w; }
+        for (int sb = SG; sb < n_seg; ++sb) {                               // runs shorter than a quarter of a tile: rare
+            const float4 w = __ldcs(reinterpret_cast<const float4*>(src + (size_t)sb * seg_stride));
+            acc.x += w.x; acc.y += w.y; acc.z += w.z; acc.w += w.w;
+        }
+        if (p.noise_scale > 0.f) {
             acc.x = fmaf(p.noise_scale, z0, acc.x); acc.y = fmaf(p.noise_scale, z1, acc.y);
             acc.z = fmaf(p.noise_scale, z2, acc.z); acc.w = fmaf(p.noise_scale, z3, acc.w);
         }
@@ -511,10 +531,12 @@ reduce_segments_kernel(const __grid_constant__ ztp::Params p) {
             *reinterpret_cast<float4*>(dst) = acc;
         } else {
             const float xs[4] = {acc.x, acc.y, acc.z, acc.w};
-            for (int u = 0; u < 4; ++u)
-                if (n + u < y.d_in) dst[u] = xs[u];
+            for (int q = 0; q < 4; ++q)
+                if (n + q < y.d_in) dst[q] = xs[q];
         }
     }
+    for (int l = 0; l < p.n_layers; ++l) {
+    const Layer& y = p.layer[l];
     if (y.do_bias && y.gb) {
         // bias: one warp per output; lanes over the (n-tile, segment) partial sums of its tile row
         const int lane = threadIdx.x & 31;
@@ -522,10 +544,10 @@ reduce_segments_kernel(const __grid_constant__ ztp::Params p) {
             const int tm = m / BM;
             float acc = 0.f;
             for (int tn = 0; tn < y.tiles_n; ++tn) {
-                const int ts = p.tile_slot[y.tile_base + tm * y.tiles_n + tn];
-                const long sl = ts / p.W, j = ts - sl * p.W;
-                const long s0 = segment_of(sl * p.S, p.S, p.U, p.lcm), s1 = segment_of((sl + 1) * p.S - 1, p.S, p.U, p.lcm);
-                for (long s = s0 + lane; s <= s1; s += 32) acc += p.bias_part[(size_t)(s * p.W + j) * BM + (m - tm * BM)];
+                const int t = y.tile_base + tm * y.tiles_n + tn;
+                const int first = p.seg_first[t], n_seg = p.seg_count[t];
+                for (int k = lane; k < n_seg; k += 32)
+                    acc += p.bias_part[(size_t)(first + (long)k * p.W) * BM + (m - tm * BM)];
             }
             acc = warp_sum(acc);
             if (lane != 0) continue;
@@ -538,6 +560,7 @@ reduce_segments_kernel(const __grid_constant__ ztp::Params p) {
             }
             y.gb[m] = acc;
         }
+    }
     }
 }
 
