@@ -684,6 +684,13 @@ def oracle_sample(w, budget_s=12.0):
                        f"(fp64, single thread, {dt:.1f} s)"), dt / reps, n
 
 
+def workload_config(w, world):
+    """The `config` object of the JSON line: the same for both arms, so that their lines can be matched."""
+    return dict(workload=w.name, B_per_gpu=w.B, layers=[f"{s.name}:T{s.T}:{s.d_in}->{s.d_out}" for s in w.layers],
+                C=w.C, sigma=w.sigma, l2="flushed by a 256 MB write between steps",
+                parallelism=f"dp{world}" if world > 1 else "single")
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -699,7 +706,7 @@ def run_reference(args):
     line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
                 warmup=args.warmup, ms_per_step=total_t / args.steps * 1e3, higher_is_better=True,
                 scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
-                config=dict(workload=w.name, B=w.B, sample=info["sample"]),
+                config=workload_config(w, args.gpus), sample=info["sample"],
                 cpu_baseline=dict(value=value, unit=UNIT, cores=1, kind="oracle", sample=info["sample"]),
                 e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0),
                 gpu_launches=0)
@@ -936,12 +943,10 @@ def main():
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
                 ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None,
                 dtype=w.dtype, data="synthetic",
-                config=dict(workload=w.name, B_per_gpu=w.B, layers=[f"{s.name}:T{s.T}:{s.d_in}->{s.d_out}" for s in w.layers],
-                            C=w.C, sigma=w.sigma, l2="flushed by a 256 MB write between steps",
-                            parallelism=f"dp{world}" if world > 1 else "single"),
+                config=workload_config(w, world),
                 gpu_launches=int(res["launches_per_step"]) * args.steps, clocks=clocks)
     if world > 1:
-        line["config"]["launch"] = res["how"]
+        line["launch"] = res["how"]
         line["e2e"] = None
         dist.destroy_process_group()
         print(json.dumps(line))
@@ -962,11 +967,11 @@ def main():
         rt = res["rotating"]
         line["config"]["l2"] = (f"inputs larger than L2: step i works on input/output set i % {rt['sets']} "
                                 f"({rt['set_bytes'] / 1e6:.1f} MB each), 256 MB flush write before the timed region")
-        line["config"]["launch"] = (f"one CUDA graph holding the {args.steps} timed steps back to back (one dpclip_step "
+        line["launch"] = (f"one CUDA graph holding the {args.steps} timed steps back to back (one dpclip_step "
                                     "call each); one event pair around the region, median of 3 regions")
         line["single_step_graph_ms_per_step"] = res["single_graph_ms"]
     else:
-        line["config"]["launch"] = ("CUDA graph replay of one step = ONE dpclip_step_streams call (the library forks over 4 "
+        line["launch"] = ("CUDA graph replay of one step = ONE dpclip_step_streams call (the library forks over 4 "
                                     "streams); events around every step")
     line["breakdown_us"] = res["breakdown"]
     line["e2e"] = dict(value=w.B / (res["e2e_ms"] * 1e-3), unit=UNIT, h2d_bytes_per_step=res["h2d"],
