@@ -47,7 +47,7 @@ enum PathSwitch : unsigned {
     SW_FORCE_SIMT = 1u << 0, SW_NO_NARROW = 1u << 1, SW_NO_NARROW_RING = 1u << 2, SW_NO_NARROW_TC = 1u << 3,
     SW_NO_NARROW_PACK = 1u << 4, SW_NARROW_PACK_BF16 = 1u << 5, SW_NO_GRAM_Q2 = 1u << 6, SW_NO_T1_TF32 = 1u << 7,
     SW_NO_FUSED_T1 = 1u << 8, SW_NO_GRAM_GROUP = 1u << 9, SW_NO_GRAD_GROUP = 1u << 10, SW_NO_CONV_TC = 1u << 11,
-    SW_NO_CONV_PATCHES = 1u << 12, SW_TILE_M1 = 1u << 13, SW_TILE_M2 = 1u << 14, SW_T1_TWO_LAUNCHES = 1u << 15, SW_NO_PAIR = 1u << 16, SW_LOG = 1u << 17, SW_NO_FACTORS_TAIL = 1u << 18, SW_NO_SM_BUDGET = 1u << 19,
+    SW_NO_CONV_PATCHES = 1u << 12, SW_TILE_M1 = 1u << 13, SW_TILE_M2 = 1u << 14, SW_T1_TWO_LAUNCHES = 1u << 15, SW_NO_PAIR = 1u << 16, SW_LOG = 1u << 17, SW_NO_FACTORS_TAIL = 1u << 18, SW_NO_SM_BUDGET = 1u << 19, SW_NO_OVERLAP = 1u << 20,
     SW_LOADED = 1u << 31
 };
 std::atomic<unsigned> g_path_switches{0};
@@ -63,6 +63,7 @@ unsigned read_path_switches() {
         {"DPCLIP_TILE_M", SW_TILE_M2, '2'}, {"DPCLIP_T1_ONE_LAUNCH", SW_T1_TWO_LAUNCHES, '0'},
         {"DPCLIP_NO_PAIR", SW_NO_PAIR, '1'}, {"DPCLIP_LOG", SW_LOG, '1'},
         {"DPCLIP_NO_FACTORS_TAIL", SW_NO_FACTORS_TAIL, '1'}, {"DPCLIP_NO_SM_BUDGET", SW_NO_SM_BUDGET, '1'},
+        {"DPCLIP_NO_OVERLAP", SW_NO_OVERLAP, '1'},
     };
     unsigned v = SW_LOADED;
     for (const auto& e : table) {
@@ -85,6 +86,14 @@ inline bool path_switch(unsigned bit) {
 // queue for the SMs (one CTA per SM) and run one after the other.
 thread_local int t_sm_budget = 0;
 inline int sm_budget() { return t_sm_budget > 0 && t_sm_budget < kNumSMs ? t_sm_budget : kNumSMs; }
+// Set while the next clipped-sum launch of this thread directly follows, in its stream, the Gram launch whose tail
+// computed the factors: the launch then asks for programmatic serialization (see griddep_wait in tc_common.cuh).
+thread_local bool t_overlap_prev = false;
+struct OverlapPrevScope {
+    bool prev;
+    explicit OverlapPrevScope(bool on) : prev(t_overlap_prev) { t_overlap_prev = on; }
+    ~OverlapPrevScope() { t_overlap_prev = prev; }
+};
 struct SmBudgetScope {
     int prev;
     explicit SmBudgetScope(int b) : prev(t_sm_budget) { t_sm_budget = b; }
@@ -789,7 +798,20 @@ int launch_zta_stream(const StreamLayer* ls, int n, int B, int T, const NoiseSpe
     DPCLIP_LOGF("clipped sum, CTA pairs: %d layer(s), B*T=%ld, %d tiles of 512x256 in %d super-layer(s) of %d, %d stages per tile, "
                 "%d pairs in gangs of %d, runs of %ld stages, %ld segments, noise %s", n, R, G, n_super, W, p.S, pairs, W, U,
                 n_segments, fuse_noise ? "in the reduce" : "separate");
-    tc::zta_pair_kernel<<<2 * pairs, zp::THREADS, zp::SMEM_BYTES, st>>>(maps, p);
+    if (t_overlap_prev && !path_switch(SW_NO_OVERLAP)) {
+        t_overlap_prev = false;                    // only the launch that directly follows
+        cudaLaunchConfig_t cfg;
+        memset(&cfg, 0, sizeof(cfg));
+        cfg.gridDim = dim3(2 * pairs); cfg.blockDim = dim3(zp::THREADS);
+        cfg.dynamicSmemBytes = zp::SMEM_BYTES; cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, tc::zta_pair_kernel, maps, p) != cudaSuccess) { cudaGetLastError(); return DPCLIP_ERR_CUDA; }
+    } else {
+        tc::zta_pair_kernel<<<2 * pairs, zp::THREADS, zp::SMEM_BYTES, st>>>(maps, p);
+    }
     int rc = launch_status();
     if (rc) return rc;
     // one wave of CTAs (six of 256 threads and 40 registers per SM) over the 4-row blocks of all tiles
@@ -2171,6 +2193,9 @@ static int step_general(const dpclip_layer* layers, const dpclip_model_layer* ot
     int in_grad_group[64];
     bool any_group = false;
     if (track) {
+        // the factors came from the tail of the Gram launch, the last kernel of this stream: the first clipped-sum
+        // launch may start loading while that tail runs
+        const OverlapPrevScope overlap(factors_done);
         rc = dpclip_same_shape_layers_clipped_grad_noise(layers, L, B, dtype, clip, C, sigma, seed, stream_id0,
                                                          in_grad_group, ws0, workspace_bytes, lanes.st[0]);
         if (rc) return rc;

@@ -416,6 +416,7 @@ gram_norm_q2_kernel(const __grid_constant__ gram::Launch q) {
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    griddep_launch_dependents();    // the clipped-sum launch that follows may place its CTAs as SMs fall idle
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer

@@ -181,6 +181,10 @@ zta_pair_kernel(const __grid_constant__ zta::Maps maps, const __grid_constant__ 
     cluster_sync_all();             // both CTAs' barriers initialised and tensor memory allocated before anyone proceeds
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    // When the launch overlaps the tail of the kernel that computes the factors, only the loads of the layers'
+    // inputs (which no kernel of a step writes) may run ahead: the warps that read the factors or write the
+    // workspace wait for that kernel here.
+    if (warp >= 2) griddep_wait();
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer (each CTA loads its own operands)
@@ -518,9 +522,13 @@ reduce_segments_kernel(const __grid_constant__ ztp::Params p) {
         float4 acc = v[0];                                                  // segment order
 #pragma unroll
         for (int k = 1; k < SG; ++k) { acc.x += v[k].x; acc.y += v[k].y; acc.z += v[k].z; acc.w += v[k].w; }
-        for (int sb = SG; sb < n_seg; ++sb) {                               // runs shorter than a quarter of a tile: rare
-            const float4 w = __ldcs(reinterpret_cast<const float4*>(src + (size_t)sb * seg_stride));
-            acc.x += w.x; acc.y += w.y; acc.z += w.z; acc.w += w.w;
+        for (int sb = SG; sb < n_seg; sb += SG) {                           // tiles cut into more than four runs
+#pragma unroll
+            for (int k = 0; k < SG; ++k)
+                v[k] = sb + k < n_seg ? __ldcs(reinterpret_cast<const float4*>(src + (size_t)(sb + k) * seg_stride))
+                                      : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int k = 0; k < SG; ++k) { acc.x += v[k].x; acc.y += v[k].y; acc.z += v[k].z; acc.w += v[k].w; }
         }
         if (p.noise_scale > 0.f) {
             acc.x = fmaf(p.noise_scale, z0, acc.x); acc.y = fmaf(p.noise_scale, z1, acc.y);

@@ -179,6 +179,14 @@ __device__ __forceinline__ void red_add_v4_f32(float* addr, float a, float b, fl
 // Two CTAs of a cluster (ranks 0 and 1, on the two SMs of one TPC) run ONE MMA: rank 0 issues it, each CTA
 // supplies its own 128 rows of the M-side operand and HALF of the N-side operand from its own shared memory
 // (same offsets in both CTAs) and receives its 128 rows of D in its own tensor memory.
+// Programmatic dependent launch.  A kernel that calls griddep_launch_dependents lets the next kernel of its stream,
+// if that one was launched with the programmatic-serialization attribute, start its CTAs as soon as every CTA of
+// this grid has made the call (or exited) and there is room for them; that kernel's threads call griddep_wait
+// before they touch anything this grid (or an earlier one) writes or reads for writing: the wait returns once
+// this grid has completed and its writes are visible.  Without the attribute both are no-ops.
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
