@@ -484,7 +484,7 @@ zta_pair_kernel(const __grid_constant__ zta::Maps maps, const __grid_constant__ 
 // Second stage: every output element = the fixed-order sum of its tile's segments (+ Philox noise), every bias =
 // the sum over the n-tiles and segments of its tile row.
 // ---------------------------------------------------------------------------
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 6)            // six CTAs per SM: the launch is one wave of 6 x SMs
 reduce_segments_kernel(const __grid_constant__ ztp::Params p) {
     using namespace ztp;
     // One wave of CTAs over the 4-row x 256-column blocks of every tile of every layer, one float4 per thread and
@@ -543,18 +543,28 @@ reduce_segments_kernel(const __grid_constant__ ztp::Params p) {
                 if (n + q < y.d_in) dst[q] = xs[q];
         }
     }
-    for (int l = 0; l < p.n_layers; ++l) {
-    const Layer& y = p.layer[l];
-    if (y.do_bias && y.gb) {
-        // bias: one warp per output; lanes over the (n-tile, segment) partial sums of its tile row
+    if (p.any_bias) {
+        // bias: one warp per output, the outputs of all layers with a bias numbered in one sequence (so every warp
+        // of the grid has at most one or two of them).  Its lanes take eight n-tiles x four segments of the tile row
+        // at a time: the partial sums of a row are usually fetched by one load per lane (a serial walk over layers
+        // and n-tiles left a tail of several microseconds at the end of the kernel).
         const int lane = threadIdx.x & 31;
-        for (int m = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; m < y.d_out; m += (gridDim.x * blockDim.x) >> 5) {
+        int total = 0;
+        for (int l = 0; l < p.n_layers; ++l) total += (p.layer[l].do_bias && p.layer[l].gb) ? p.layer[l].d_out : 0;
+        for (int g = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; g < total; g += (gridDim.x * blockDim.x) >> 5) {
+            int l = 0, m = g;
+            for (; l < p.n_layers; ++l) {
+                const int rows = (p.layer[l].do_bias && p.layer[l].gb) ? p.layer[l].d_out : 0;
+                if (m < rows) break;
+                m -= rows;
+            }
+            const Layer& y = p.layer[l];
             const int tm = m / BM;
             float acc = 0.f;
-            for (int tn = 0; tn < y.tiles_n; ++tn) {
+            for (int tn = lane >> 2; tn < y.tiles_n; tn += 8) {
                 const int t = y.tile_base + tm * y.tiles_n + tn;
                 const int first = p.seg_first[t], n_seg = p.seg_count[t];
-                for (int k = lane; k < n_seg; k += 32)
+                for (int k = lane & 3; k < n_seg; k += 4)
                     acc += p.bias_part[(size_t)(first + (long)k * p.W) * BM + (m - tm * BM)];
             }
             acc = warp_sum(acc);
@@ -568,7 +578,6 @@ reduce_segments_kernel(const __grid_constant__ ztp::Params p) {
             }
             y.gb[m] = acc;
         }
-    }
     }
 }
 
