@@ -474,6 +474,18 @@ def bench_workload(torch, dp, w, steps, warmup, flush, peaks, with_e2e=True):
     warm = time_steps(torch, graph.replay, steps, 1, lambda: None)
     eager = time_steps(torch, lambda: plan.run(w.C, w.sigma, 1), steps, 1, flush)
     bd = kernel_breakdown(torch, dp, w, plan, min(steps, 20), flush, w.C, w.sigma)
+    # The literal inputs clip every example (the worst case for the clipped sum: stages whose factor is exactly one
+    # skip the rescaling in shared memory): the same step with the threshold at the median norm and above every norm.
+    clip_cases = None
+    if with_e2e:
+        norms = plan.norms.float()
+        clip_cases = {"literal": dict(clipped_fraction=float((plan.clip < 1).float().mean().item()))}
+        for name, c in (("half_clipped", float(norms.median().item())), ("unclipped", 2.0 * float(norms.max().item()))):
+            g = plan.capture(c, w.sigma, 1, branches=branches)
+            ms = float(np.mean(time_steps(torch, g.replay, min(steps, 20), 3, flush)))
+            clip_cases[name] = dict(C=c, ms_per_step=ms, clipped_fraction=float((plan.clip < 1).float().mean().item()))
+        plan.run(w.C, w.sigma, 1)
+        torch.cuda.synchronize()
     res = dict(times_ms=times, warm_ms=float(np.median(warm)), eager_ms=float(np.median(eager)),
                single_graph_ms=float(np.mean(single)), rotating=rotating, one_stream_ms=one_stream_ms,
                launches_per_step=int(launches_per_step),
@@ -483,6 +495,7 @@ def bench_workload(torch, dp, w, steps, warmup, flush, peaks, with_e2e=True):
     # whole-step lower bound: max(total algorithmic bytes / HBM, total flops / the engine used)
     res["step_roofline"] = step_roofline(w, peaks)
     res["step_roofline_us"] = res["step_roofline"]["roof_us"]
+    res["clip_cases"] = clip_cases
     if with_e2e:
         host_layers = [dp.Layer(torch.from_numpy(A).to(torch.float32 if w.dtype == "f32" else torch.bfloat16).pin_memory(),
                                 torch.from_numpy(Z).to(torch.float32 if w.dtype == "f32" else torch.bfloat16).pin_memory(),
@@ -868,8 +881,8 @@ def config_summary(name, w, r, ms):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default="cfg4")
     ap.add_argument("--impl", default="dpclip", choices=["dpclip", "reference"])
     ap.add_argument("--others", default="cfg1,cfg2,cfg2_bf16,cfg3_f32,cfg3_bf16,cfg4",
@@ -952,6 +965,8 @@ def main():
         print(json.dumps(line))
         return
 
+    if res.get("clip_cases"):
+        line["clip_cases"] = res["clip_cases"]
     sr = res["step_roofline"]
     roof = res["roofline"]
     roof["step"] = dict(sr, measured_us=ms_per_step * 1e3, frac=sr["roof_us"] / (ms_per_step * 1e3),
@@ -998,7 +1013,7 @@ def main():
             if k in configs:
                 configs[k]["launch_floor_us"] = line["launch_floor_us"]["cooperative"]
     if args.others and not args.no_extras:
-        pts = sweep_points_compact(torch, dp, args.steps, flush, peaks)
+        pts = sweep_points_compact(torch, dp, min(args.steps, 30), flush, peaks)
         others["cfg5_sweep"] = pts
         # compact: "B,T,d_in,d_out": [step us, fraction of the point's step roofline]
         configs["cfg5"] = {f"{r['B']},{r['T']},{r['d_in']},{r['d_out']}": [round(r["step_us"], 1), round(r["frac"], 3)]
