@@ -460,6 +460,13 @@ def bench_workload(torch, dp, w, steps, warmup, flush, peaks, with_e2e=True):
     # take the fused two-launch step inside one dpclip_step call
     branches = 1 if all(s.T == 1 for s in w.layers) else 4
     graph = plan.capture(w.C, w.sigma, 1, branches=branches)
+    # per-call times first, while the GPU is still in the state in which the burst peaks were measured (a kernel
+    # timed alone is compared with the burst figure; after the long loops below the power cap lowers the clocks)
+    for _ in range(3):
+        flush(); graph.replay()
+    bd = kernel_breakdown(torch, dp, w, plan, min(steps, 20), flush, w.C, w.sigma)
+    torch.cuda.synchronize()
+    time.sleep(0.5)                  # the timed loop starts from an idle GPU (see rest() below), then its warm-up steps
     single = time_steps(torch, graph.replay, steps, warmup, flush)
     assert all(dp.dpclip_read_status(x) == 0 for x in plan.workspaces())
     rotating = None
@@ -467,13 +474,21 @@ def bench_workload(torch, dp, w, steps, warmup, flush, peaks, with_e2e=True):
         times, rotating = time_steps_rotating(torch, dp, w, layers, steps, warmup, flush)
     else:
         times = single
+    def rest():
+        # the other launch modes are measured for comparison, each from the same starting state: half a second of
+        # idle lets the power cap's running average recover after the loop before
+        torch.cuda.synchronize()
+        time.sleep(0.5)
+
     one_stream_ms = None
     if branches > 1:
         g1 = plan.capture(w.C, w.sigma, 1, branches=1)          # the same step as ONE dpclip_step call on one stream
-        one_stream_ms = float(np.mean(time_steps(torch, g1.replay, min(steps, 10), 2, flush)))
-    warm = time_steps(torch, graph.replay, steps, 1, lambda: None)
-    eager = time_steps(torch, lambda: plan.run(w.C, w.sigma, 1), steps, 1, flush)
-    bd = kernel_breakdown(torch, dp, w, plan, min(steps, 20), flush, w.C, w.sigma)
+        rest()
+        one_stream_ms = float(np.mean(time_steps(torch, g1.replay, min(steps, 30), 3, flush)))
+    rest()
+    eager = time_steps(torch, lambda: plan.run(w.C, w.sigma, 1), min(steps, 30), 3, flush)
+    rest()
+    warm = time_steps(torch, graph.replay, steps, 3, lambda: None)
     # The literal inputs clip every example (the worst case for the clipped sum: stages whose factor is exactly one
     # skip the rescaling in shared memory): the same step with the threshold at the median norm and above every norm.
     clip_cases = None
@@ -881,7 +896,7 @@ def config_summary(name, w, r, ms):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default="cfg4")
     ap.add_argument("--impl", default="dpclip", choices=["dpclip", "reference"])
@@ -967,6 +982,10 @@ def main():
 
     if res.get("clip_cases"):
         line["clip_cases"] = res["clip_cases"]
+    if len(res["times_ms"]) >= 8 and not res.get("rotating"):
+        # the timed steps in four quarters: shows whether the power cap lowered the clocks during the run
+        q = np.array_split(np.asarray(res["times_ms"]), 4)
+        line["ms_per_step_by_quarter"] = [round(float(x.mean()), 5) for x in q]
     sr = res["step_roofline"]
     roof = res["roofline"]
     roof["step"] = dict(sr, measured_us=ms_per_step * 1e3, frac=sr["roof_us"] / (ms_per_step * 1e3),
